@@ -1,0 +1,37 @@
+"""CPU oracle for the BiCache attention hot path.
+
+TEST INFRASTRUCTURE ONLY.  This package is the plain, slow, fp64 statement of
+what the library must compute.  It is imported by the tests, by the smoke
+check and by the benchmark's CPU-baseline leg, and by nothing else; the
+product path never routes through it.  It shares no code with the CUDA path
+and imports nothing from it.
+
+Parity status of each function (what pins it, see tests/test_oracle_*.py):
+
+  reuse_depth      pinned (hand-computed cases, ranges, monotonicity).  The
+                   *contents* of the depth table are an input; the paper
+                   prints no table values, so the stand-in table used by the
+                   workloads is "parity unpinned".
+  PagedPrefixStore pinned (independent trace simulation, conservation laws).
+  attention        pinned (scalar brute force, torch SDPA fp64, closed forms,
+                   rational-weight golden cases, invariances).
+  merge            pinned (any split of the key set equals the direct result).
+  attend/attend_full/stack
+                   pinned (brute force over the concatenated key list, depth-0
+                   and depth-L special cases, cached == fresh special case).
+"""
+from .bicache_oracle import (  # noqa: F401
+    OracleError,
+    InvalidArgument,
+    OutOfPages,
+    NotFound,
+    reuse_depth,
+    PagedPrefixStore,
+    attention,
+    merge,
+    attend,
+    attend_full,
+    attend_rows,
+    attend_full_rows,
+    stack,
+)

@@ -1,0 +1,390 @@
+"""Plain fp64 definition of the BiCache per-denoising-step attention.
+
+TEST INFRASTRUCTURE ONLY: never imported by the product path.
+
+Everything here is written from the paper's statement of the method:
+
+  * Eq. 2  (bidirectional softmax attention over all tokens of the input),
+  * Eq. 4  (shallow layers l <= b use the cached shared-prefix KVs),
+  * Sec. 5.1/5.2 (ratio r of shared-prefix tokens to all tokens -> lookup
+    table T -> shallow depth b; layer l reuses iff l <= b, else recomputes),
+  * Sec. 5.2 + implementation appendix (hash-indexed KV store H holding the
+    prefix KVs of all L layers; first-in-first-out eviction).
+
+All floating-point work is numpy float64.  A matrix product (numpy matmul) is
+used as a library step; there is no tiling, fusion, online softmax or any
+other reordering, so each function can be compared with the paper by eye.
+Inputs arrive as float64 arrays that are exact widenings of the bytes the GPU
+gets (bf16 or fp32 -> fp64 is exact).
+
+Conventions (0-based, as in the C API): layer index l in [0, L); a request
+with depth b reuses the cache in layers l < b (the paper's 1-based l <= b).
+Tensors: q [rows, Hq, D]; k, v [rows, Hkv, D]; query head h reads KV head
+h // (Hq // Hkv).
+"""
+from __future__ import annotations
+
+import math
+from collections import OrderedDict, deque
+
+import numpy as np
+
+
+class OracleError(Exception):
+    """Base class; subclasses mirror the library's status codes."""
+
+
+class InvalidArgument(OracleError):
+    pass
+
+
+class OutOfPages(OracleError):
+    pass
+
+
+class NotFound(OracleError):
+    pass
+
+
+# ---------------------------------------------------------------------------
+# Reuse-depth rule (Sec. 5.1 "profiling dataset": r = shared-prefix tokens /
+# all tokens of the input string; Sec. 5.2: r -> T -> b).
+# ---------------------------------------------------------------------------
+
+def reuse_depth(prefix_len, nonshared_len, table, num_layers):
+    """Per-request shallow depth b in [0, L].
+
+    r = m / (m + n) is quantised DOWN to the table's 1/100 grid in integer
+    arithmetic (the paper profiles r in {0.01, ..., 1.00}; it does not state
+    the rounding; flooring is the conservative reading because b grows with
+    r).  table has 101 entries, table[idx] for idx = floor(100 m / (m + n)).
+    m <= 0 (no shared prefix) gives depth 0.
+    """
+    table = [int(x) for x in table]
+    if len(table) != 101:
+        raise InvalidArgument("depth table must have 101 entries")
+    out = []
+    for m, n in zip(prefix_len, nonshared_len):
+        m = int(m)
+        n = int(n)
+        if n < 0:
+            raise InvalidArgument("negative non-shared length")
+        if m <= 0:
+            out.append(0)
+            continue
+        idx = (100 * m) // (m + n)
+        b = table[idx]
+        b = max(0, min(int(num_layers), b))
+        out.append(b)
+    return np.asarray(out, dtype=np.int32)
+
+
+# ---------------------------------------------------------------------------
+# KV store H (Sec. 5.2: hit -> load the cached KVs of all L layers; miss ->
+# insert; implementation appendix: FIFO eviction).  Storage is paged.
+# ---------------------------------------------------------------------------
+
+class PagedPrefixStore:
+    """Prefix-KV store over fixed-size pages with FIFO eviction.
+
+    One page index addresses the same slot in every layer.  Token t of a
+    prefix lives in page pages[t // P], slot t % P.  The free list is a FIFO
+    queue: pages are taken from its head; an evicted prefix's pages are
+    appended to its tail in page-table order.  Prefix ids come from a counter
+    that is never reused.
+    """
+
+    def __init__(self, num_layers, num_kv_heads, head_dim, page_size, num_pages,
+                 free_order=None):
+        self.L = int(num_layers)
+        self.Hkv = int(num_kv_heads)
+        self.D = int(head_dim)
+        self.P = int(page_size)
+        self.num_pages = int(num_pages)
+        if free_order is None:
+            free_order = range(self.num_pages)
+        free_order = [int(p) for p in free_order]
+        if sorted(free_order) != list(range(self.num_pages)):
+            raise InvalidArgument("free_order must be a permutation of the pages")
+        self.free = deque(free_order)
+        # [layer][page][slot][kv head][dim]
+        shape = (self.L, self.num_pages, self.P, self.Hkv, self.D)
+        self.k_pool = np.zeros(shape, dtype=np.float64)
+        self.v_pool = np.zeros(shape, dtype=np.float64)
+        self.by_key = OrderedDict()   # key -> prefix id, in insertion order
+        self.entries = {}             # prefix id -> (key, m, [pages])
+        self.next_id = 0
+
+    def pages_needed(self, m):
+        return (int(m) + self.P - 1) // self.P
+
+    def put(self, key, k, v):
+        """Insert prefix KVs k, v of shape [L, m, Hkv, D].  Returns
+        (prefix_id, was_hit, pages)."""
+        k = np.asarray(k, dtype=np.float64)
+        v = np.asarray(v, dtype=np.float64)
+        if k.shape != v.shape or k.ndim != 4 or k.shape[0] != self.L \
+                or k.shape[2] != self.Hkv or k.shape[3] != self.D:
+            raise InvalidArgument("bad prefix KV shape")
+        m = k.shape[1]
+        if m < 1:
+            raise InvalidArgument("empty prefix")
+        key = int(key)
+        if key in self.by_key:
+            pid = self.by_key[key]
+            if self.entries[pid][1] != m:
+                raise InvalidArgument("key already present with another length")
+            return pid, True, list(self.entries[pid][2])
+        need = self.pages_needed(m)
+        if need > self.num_pages:
+            raise OutOfPages("prefix larger than the whole pool")
+        while len(self.free) < need:
+            old_key, old_id = next(iter(self.by_key.items()))   # oldest insertion
+            del self.by_key[old_key]
+            for p in self.entries.pop(old_id)[2]:
+                self.free.append(p)
+        pages = [self.free.popleft() for _ in range(need)]
+        pid = self.next_id
+        self.next_id += 1
+        self.by_key[key] = pid
+        self.entries[pid] = (key, m, pages)
+        for t in range(m):
+            self.k_pool[:, pages[t // self.P], t % self.P] = k[:, t]
+            self.v_pool[:, pages[t // self.P], t % self.P] = v[:, t]
+        return pid, False, list(pages)
+
+    def lookup(self, key):
+        key = int(key)
+        if key not in self.by_key:
+            raise NotFound("unknown key")
+        pid = self.by_key[key]
+        return pid, self.entries[pid][1]
+
+    def pages(self, prefix_id):
+        if prefix_id not in self.entries:
+            raise NotFound("unknown or evicted prefix id")
+        return list(self.entries[prefix_id][2])
+
+    def prefix_len(self, prefix_id):
+        if prefix_id not in self.entries:
+            raise NotFound("unknown or evicted prefix id")
+        return self.entries[prefix_id][1]
+
+    def prefix_kv(self, layer, prefix_id):
+        """Cached K, V of one layer, read back through the page table:
+        two arrays [m, Hkv, D]."""
+        if not 0 <= layer < self.L:
+            raise InvalidArgument("layer out of range")
+        if prefix_id not in self.entries:
+            raise NotFound("unknown or evicted prefix id")
+        _, m, pages = self.entries[prefix_id]
+        k = np.empty((m, self.Hkv, self.D), dtype=np.float64)
+        v = np.empty((m, self.Hkv, self.D), dtype=np.float64)
+        for t in range(m):
+            k[t] = self.k_pool[layer, pages[t // self.P], t % self.P]
+            v[t] = self.v_pool[layer, pages[t // self.P], t % self.P]
+        return k, v
+
+
+# ---------------------------------------------------------------------------
+# Eq. 2: o = sum_j softmax_j(q . k_j * scale) v_j over ALL keys, no mask.
+# ---------------------------------------------------------------------------
+
+def attention(q, k, v, scale):
+    """q [nq, Hq, D]; k, v [nk, Hkv, D] -> (o [nq, Hq, D], lse [nq, Hq]).
+
+    lse is the natural log of sum_j exp(scale * q.k_j).  With no keys the
+    output is 0 and lse is -inf (the empty partial result of a merge).
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    nq, Hq, D = q.shape
+    nk, Hkv, _ = k.shape
+    if Hq % Hkv:
+        raise InvalidArgument("query heads must be a multiple of KV heads")
+    group = Hq // Hkv
+    o = np.zeros((nq, Hq, D), dtype=np.float64)
+    lse = np.full((nq, Hq), -np.inf, dtype=np.float64)
+    if nq == 0 or nk == 0:
+        return o, lse
+    for h in range(Hq):
+        hk = h // group
+        s = float(scale) * (q[:, h, :] @ k[:, hk, :].T)          # [nq, nk]
+        mx = s.max(axis=1, keepdims=True)
+        p = np.exp(s - mx)
+        z = p.sum(axis=1, keepdims=True)
+        o[:, h, :] = (p @ v[:, hk, :]) / z
+        lse[:, h] = (mx + np.log(z))[:, 0]
+    return o, lse
+
+
+def merge(parts):
+    """Log-sum-exp merge of partial results over disjoint key sets.
+
+    parts: sequence of (o [.., D], lse [..]).  Returns (o, lse) equal to Eq. 2
+    over the union of the key sets:  lse = log sum_i exp(lse_i),
+    o = sum_i exp(lse_i - lse) o_i.  A part with lse = -inf weighs 0.
+    """
+    parts = [(np.asarray(o, dtype=np.float64), np.asarray(l, dtype=np.float64))
+             for o, l in parts]
+    lses = np.stack([l for _, l in parts])                       # [parts, ...]
+    mx = lses.max(axis=0)
+    safe = np.where(np.isfinite(mx), mx, 0.0)
+    w = np.exp(lses - safe)                                       # exp(-inf) = 0
+    tot = w.sum(axis=0)
+    with np.errstate(divide="ignore"):
+        lse = safe + np.log(tot)
+    lse = np.where(tot > 0, lse, -np.inf)
+    o = np.zeros_like(parts[0][0])
+    for (oi, _), wi in zip(parts, w):
+        frac = np.where(tot > 0, wi / np.where(tot > 0, tot, 1.0), 0.0)
+        o = o + frac[..., None] * oi
+    return o, lse
+
+
+# ---------------------------------------------------------------------------
+# The two calls of the hot path.
+# ---------------------------------------------------------------------------
+
+def _check_batch(row_off, seqlen, rows):
+    for off, n in zip(row_off, seqlen):
+        if n < 0 or off < 0 or off + n > rows:
+            raise InvalidArgument("request rows out of range")
+
+
+def attend(store, layer, prefix_id, row_off, seqlen, q, k, v, scale):
+    """Shallow-layer attention (Eq. 2 with the key set Eq. 4 prescribes).
+
+    For request i with suffix rows row_off[i] .. row_off[i] + seqlen[i] of
+    q/k/v: every suffix query attends, without any mask, over
+    [cached prefix K/V of prefix_id[i] at `layer` | the request's own suffix
+    K/V].  prefix_id[i] = -1 means no prefix.  Returns (out, lse) shaped like
+    q and q[..., 0]; rows that belong to no request are left at 0 / -inf.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    _check_batch(row_off, seqlen, q.shape[0])
+    out = np.zeros_like(q)
+    lse = np.full(q.shape[:2], -np.inf)
+    for pid, off, n in zip(prefix_id, row_off, seqlen):
+        off = int(off)
+        n = int(n)
+        if n == 0:
+            continue
+        ks, vs = k[off:off + n], v[off:off + n]
+        if pid >= 0:
+            kc, vc = store.prefix_kv(layer, int(pid))
+            ks = np.concatenate([kc, ks], axis=0)
+            vs = np.concatenate([vc, vs], axis=0)
+        out[off:off + n], lse[off:off + n] = attention(q[off:off + n], ks, vs, scale)
+    return out, lse
+
+
+def attend_full(row_off, seqlen, q, k, v, scale):
+    """Deep-layer fallback: full bidirectional attention (Eq. 2) of each
+    request over its own N_i fresh rows; all N_i rows are queries."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    _check_batch(row_off, seqlen, q.shape[0])
+    out = np.zeros_like(q)
+    lse = np.full(q.shape[:2], -np.inf)
+    for off, n in zip(row_off, seqlen):
+        off = int(off)
+        n = int(n)
+        if n == 0:
+            continue
+        out[off:off + n], lse[off:off + n] = attention(
+            q[off:off + n], k[off:off + n], v[off:off + n], scale)
+    return out, lse
+
+
+def _one_row(q_row, ks, vs, hk, scale):
+    s = float(scale) * (ks[:, hk, :] @ q_row)
+    mx = s.max()
+    p = np.exp(s - mx)
+    z = p.sum()
+    return (p @ vs[:, hk, :]) / z, mx + math.log(z)
+
+
+def attend_rows(store, layer, prefix_id, row_off, seqlen, q, k, v, scale, samples):
+    """Same definition as `attend`, evaluated only at the sampled
+    (request, head, row-within-suffix) triples, each over ALL its keys.
+    Returns (o [len(samples), D], lse [len(samples)])."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    Hq, Hkv = q.shape[1], k.shape[1]
+    o = np.zeros((len(samples), q.shape[2]))
+    lse = np.zeros(len(samples))
+    cache = {}
+    for si, (i, h, a) in enumerate(samples):
+        off, n, pid = int(row_off[i]), int(seqlen[i]), int(prefix_id[i])
+        if not 0 <= a < n:
+            raise InvalidArgument("sampled row outside the request")
+        if i not in cache:
+            ks, vs = k[off:off + n], v[off:off + n]
+            if pid >= 0:
+                kc, vc = store.prefix_kv(layer, pid)
+                ks = np.concatenate([kc, ks], axis=0)
+                vs = np.concatenate([vc, vs], axis=0)
+            cache = {i: (ks, vs)}
+        ks, vs = cache[i]
+        o[si], lse[si] = _one_row(q[off + a, h], ks, vs, h // (Hq // Hkv), scale)
+    return o, lse
+
+
+def attend_full_rows(row_off, seqlen, q, k, v, scale, samples):
+    """`attend_full` at sampled (request, head, row) triples."""
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    Hq, Hkv = q.shape[1], k.shape[1]
+    o = np.zeros((len(samples), q.shape[2]))
+    lse = np.zeros(len(samples))
+    for si, (i, h, a) in enumerate(samples):
+        off, n = int(row_off[i]), int(seqlen[i])
+        if not 0 <= a < n:
+            raise InvalidArgument("sampled row outside the request")
+        o[si], lse[si] = _one_row(q[off + a, h], k[off:off + n], v[off:off + n],
+                                  h // (Hq // Hkv), scale)
+    return o, lse
+
+
+def stack(store, depth, prefix_id, prefix_len, full_row_off, full_len, q, k, v, scale):
+    """One denoising step's attention over all L layers (Sec. 5.2 dispatch).
+
+    Request i owns rows full_row_off[i] .. + full_len[i] of q/k/v (its whole
+    input: prefix_len[i] prefix tokens then the suffix).  q, k, v are lists
+    with one [rows, H, D] array per layer.  In layer l, requests with
+    l < depth[i] go through `attend` on their suffix rows (the tail of their
+    row range); the others go through `attend_full` on all their rows.
+    Returns a list of per-layer (out, lse); rows not computed in a layer
+    (prefix rows of reusing requests) stay 0 / -inf.
+    """
+    R = len(depth)
+    results = []
+    for l in range(store.L if store is not None else len(q)):
+        reuse = [i for i in range(R) if l < depth[i]]
+        full = [i for i in range(R) if l >= depth[i]]
+        out = np.zeros_like(np.asarray(q[l], dtype=np.float64))
+        lse = np.full(out.shape[:2], -np.inf)
+        if reuse:
+            offs = [full_row_off[i] + prefix_len[i] for i in reuse]
+            lens = [full_len[i] - prefix_len[i] for i in reuse]
+            o1, l1 = attend(store, l, [prefix_id[i] for i in reuse], offs, lens,
+                            q[l], k[l], v[l], scale)
+            for off, n in zip(offs, lens):
+                out[off:off + n] = o1[off:off + n]
+                lse[off:off + n] = l1[off:off + n]
+        if full:
+            offs = [full_row_off[i] for i in full]
+            lens = [full_len[i] for i in full]
+            o2, l2 = attend_full(offs, lens, q[l], k[l], v[l], scale)
+            for off, n in zip(offs, lens):
+                out[off:off + n] = o2[off:off + n]
+                lse[off:off + n] = l2[off:off + n]
+        results.append((out, lse))
+    return results

@@ -1,0 +1,152 @@
+"""Pins for the oracle's reuse-depth rule and paged FIFO prefix store (CPU)."""
+import os
+
+import numpy as np
+import pytest
+from hypothesis import given, settings, strategies as st
+
+import oracle
+from paper_2606_07571_b200 import workloads
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _depth_cases():
+    with open(os.path.join(GOLDEN, "depth_cases.txt")) as f:
+        return [tuple(int(x) for x in ln.split()) for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+def test_depth_rule_hand_cases():
+    """An identity table turns the rule into its ratio-bin index."""
+    table = list(range(101))
+    for m, n, idx in _depth_cases():
+        assert oracle.reuse_depth([m], [n], table, 1000)[0] == idx
+    # clamped into [0, L]; no prefix -> 0
+    assert oracle.reuse_depth([99, 0, 50], [1, 10, 50], table, 32).tolist() == [32, 0, 32]
+    assert oracle.reuse_depth([10], [10], [-3] * 101, 32)[0] == 0
+    with pytest.raises(oracle.InvalidArgument):
+        oracle.reuse_depth([1], [1], list(range(100)), 32)
+    with pytest.raises(oracle.InvalidArgument):
+        oracle.reuse_depth([1], [-1], table, 32)
+
+
+@given(st.integers(1, 5000), st.integers(0, 5000), st.integers(1, 64))
+@settings(max_examples=200, deadline=None)
+def test_depth_rule_ranges_and_monotonicity(m, n, L):
+    t = workloads.standin_depth_table(L)
+    d = oracle.reuse_depth([m, m + 1, m], [n, n, n + 1], t, L)
+    assert 1 <= d[0] <= L                      # a shared prefix always allows layer 1
+    assert d[1] >= d[0] >= d[2]                # more prefix -> deeper; more suffix -> shallower
+    # the bin index is the floor of 100 r, never beyond the true ratio
+    idx = oracle.reuse_depth([m], [n], list(range(101)), 1000)[0]
+    assert idx * (m + n) <= 100 * m < (idx + 1) * (m + n)
+
+
+def test_standin_table_shape():
+    t = workloads.standin_depth_table(32)
+    assert len(t) == 101 and t[100] == 32 and t[85] == 16 and t[0] == 1
+    assert (np.diff(t) >= 0).all() and t.min() >= 1
+
+
+# -- store: an independent trace simulation -----------------------------------
+
+class ModelStore:
+    """Deliberately different bookkeeping: a flat owner array plus an explicit
+    arrival list, re-deriving the free queue by replaying events."""
+
+    def __init__(self, num_pages, P, order):
+        self.P = P
+        self.queue = list(order)
+        self.live = []          # [key, m, pages] in arrival order
+        self.count = 0
+
+    def put(self, key, m):
+        for e in self.live:
+            if e[0] == key:
+                return ("hit", e[3], e[2]) if e[1] == m else ("invalid",)
+        need = -(-m // self.P)
+        if need > len(self.queue) + sum(len(e[2]) for e in self.live):
+            return ("nomem",)
+        while len(self.queue) < need:
+            self.queue.extend(self.live.pop(0)[2])
+        pages, self.queue = self.queue[:need], self.queue[need:]
+        self.live.append([key, m, pages, self.count])
+        self.count += 1
+        return ("miss", self.count - 1, pages)
+
+
+@given(st.lists(st.tuples(st.integers(0, 6), st.integers(1, 70)), min_size=1, max_size=40),
+       st.integers(1, 12), st.integers(0, 3))
+@settings(max_examples=150, deadline=None)
+def test_store_traces_against_model(trace, num_pages, seed):
+    P, L, H, D = 8, 1, 1, 2
+    order = list(range(num_pages)) if seed == 0 else np.random.default_rng(seed).permutation(num_pages).tolist()
+    real = oracle.PagedPrefixStore(L, H, D, P, num_pages, free_order=order)
+    model = ModelStore(num_pages, P, order)
+    key_len = {}
+    for key, m in trace:
+        m = key_len.setdefault(key, m) if seed % 2 == 0 else m
+        want = model.put(key, m)
+        kv = np.full((L, m, H, D), float(key))
+        if want[0] == "invalid":
+            with pytest.raises(oracle.InvalidArgument):
+                real.put(key, kv, kv)
+        elif want[0] == "nomem":
+            with pytest.raises(oracle.OutOfPages):
+                real.put(key, kv, kv)
+        else:
+            pid, hit, pages = real.put(key, kv, kv)
+            assert (hit, pid, pages) == (want[0] == "hit", want[1], want[2])
+        # conservation: every page is free or owned exactly once
+        owned = [p for pid in real.entries for p in real.pages(pid)]
+        assert sorted(owned + list(real.free)) == list(range(num_pages))
+        # live keys agree, evicted keys are gone
+        live = {e[0] for e in model.live}
+        for k in range(7):
+            if k in live:
+                pid, mm = real.lookup(k)
+                kk, _ = real.prefix_kv(0, pid)
+                assert kk.shape[0] == mm and (kk == float(k)).all()
+            else:
+                with pytest.raises(oracle.NotFound):
+                    real.lookup(k)
+
+
+def test_store_fifo_not_lru_and_ids_never_reused():
+    s = oracle.PagedPrefixStore(1, 1, 2, 16, 4)
+    kv = lambda m: np.ones((1, m, 1, 2))
+    a, _, pa = s.put(10, kv(32), kv(32))       # pages 0,1
+    b, _, pb = s.put(11, kv(16), kv(16))       # page 2
+    assert (a, b, pa, pb) == (0, 1, [0, 1], [2])
+    assert s.put(10, kv(32), kv(32))[1] is True            # a hit does not refresh age
+    c, hit, pc = s.put(12, kv(32), kv(32))     # needs 2, 1 free -> evict oldest (key 10)
+    assert (c, hit, pc) == (2, False, [3, 0])  # free queue was [3] + evicted [0, 1]
+    with pytest.raises(oracle.NotFound):
+        s.lookup(10)
+    with pytest.raises(oracle.NotFound):
+        s.pages(a)
+    d, _, pd = s.put(10, kv(16), kv(16))       # re-put after eviction: new id, next free page
+    assert (d, pd) == (3, [1])
+    with pytest.raises(oracle.OutOfPages):
+        s.put(13, kv(16 * 5), kv(16 * 5))
+    with pytest.raises(oracle.InvalidArgument):
+        s.put(11, kv(17), kv(17))
+    with pytest.raises(oracle.InvalidArgument):
+        oracle.PagedPrefixStore(1, 1, 2, 16, 4, free_order=[0, 1, 1, 2])
+
+
+def test_workload_recipes_are_deterministic_and_shaped():
+    w = workloads.config4()
+    w2 = workloads.config4()
+    assert w.prefix_lens == w2.prefix_lens and w.suffix_lens == w2.suffix_lens
+    assert len(w.prefix_lens) == 8 and w.num_requests == 256
+    assert all(512 <= m <= 4096 for m in w.prefix_lens)
+    assert all(32 <= n <= 1024 for n in w.suffix_lens)
+    assert w.req_prefix == sorted(w.req_prefix)
+    w3 = workloads.config3()
+    assert w3.num_requests == 64 and all(64 <= n <= 512 for n in w3.suffix_lens)
+    q, k, v = workloads.draw_full_qkv(workloads.config1())
+    q2, _, _ = workloads.draw_full_qkv(workloads.config1())
+    assert q.shape == (4 * 96, 4, 64) and (q == q2).all()
+    small = workloads.scaled_down(w, num_layers=2, max_requests=12, prefix_div=16, suffix_div=8)
+    assert small.num_requests == 12 and small.req_prefix == sorted(small.req_prefix)
