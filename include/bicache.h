@@ -1,0 +1,191 @@
+/*
+ * bicache.h - C ABI of the BiCache attention hot path for NVIDIA B200 (sm_100a).
+ *
+ * BiCache serves diffusion language models with a shared-prefix KV cache: in
+ * the shallow layers 1..b of a request the cached KVs of the shared prefix are
+ * reused (Eq. 4), in the deep layers they are recomputed (Sec. 5.2).  This
+ * library is the attention of one denoising step under that scheme:
+ *
+ *   bicache_put_prefix    KV store H: insert the prefix KVs of all L layers
+ *                         (Sec. 5.2 "On a miss ... stores them in H[k]"),
+ *                         paged, with first-in-first-out eviction
+ *                         (implementation appendix).
+ *   bicache_reuse_depth   r = shared-prefix tokens / all tokens of the input
+ *                         string -> lookup table T -> shallow depth b
+ *                         (Sec. 5.1, Sec. 5.2 first paragraph).
+ *   bicache_attend        layers l < b: suffix queries attend, without a
+ *                         causal mask, over [cached prefix K/V | own suffix
+ *                         K/V] (Eq. 2 with the key set of Eq. 4).
+ *   bicache_attend_full   layers l >= b: full bidirectional attention of a
+ *                         request over its own freshly computed rows (Eq. 2).
+ *
+ * General rules
+ *   - Every function returns a bicache_status.  Nothing aborts, throws or
+ *     traps the device.  Host-detectable errors return before any launch and
+ *     leave all outputs untouched.
+ *   - The caller owns every device buffer (pools, workspace, tensors) and the
+ *     CUDA stream.  The library allocates no device memory; it owns host
+ *     bookkeeping only (key map, FIFO list, free-page queue, schedules).
+ *   - Pointers documented "device" must be device pointers on cfg.device and
+ *     16-byte aligned; row strides are in elements and must keep every row
+ *     16-byte aligned.  Pointers documented "host" are ordinary host memory.
+ *   - Calls enqueue work on `stream` and return without synchronising (except
+ *     bicache_destroy and bicache_device_status).  One stream per context at a
+ *     time; a context is not thread-safe.  Evicting a prefix while work that
+ *     reads it is still enqueued is safe only because everything is ordered on
+ *     that one stream.
+ *   - Layers are 0-based: layer l reuses the cache iff l < depth (the paper's
+ *     1-based l <= b).
+ */
+#ifndef BICACHE_H_
+#define BICACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct bicache_ctx bicache_ctx;
+
+typedef enum {
+  BICACHE_OK = 0,
+  BICACHE_ERR_INVALID = 1,     /* bad argument (null/unaligned pointer, range, ungrouped ids, ...) */
+  BICACHE_ERR_NOMEM = 2,       /* prefix larger than the pool, or workspace too small             */
+  BICACHE_ERR_NOTFOUND = 3,    /* unknown or evicted key / prefix id                              */
+  BICACHE_ERR_CUDA = 4,        /* a CUDA runtime call failed                                      */
+  BICACHE_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (see bicache_device_status)  */
+  BICACHE_ERR_UNSUPPORTED = 6  /* dtype / head_dim / page size outside what is built              */
+} bicache_status;
+
+enum { BICACHE_F32 = 0, BICACHE_BF16 = 1 };
+
+/* Which kernels serve bf16 head_dim-128 attention.  AUTO picks the tensor-core
+ * path when it applies; SIMT forces the plain CUDA-core kernels (used as an
+ * on-device cross-check).  fp32 and other head dims always run SIMT. */
+enum { BICACHE_PATH_AUTO = 0, BICACHE_PATH_SIMT = 1, BICACHE_PATH_TENSOR = 2 };
+
+typedef struct {
+  int32_t num_layers;        /* L >= 1                                                         */
+  int32_t num_q_heads;       /* Hq, a multiple of num_kv_heads                                 */
+  int32_t num_kv_heads;      /* Hkv                                                            */
+  int32_t head_dim;          /* D: 128 for the tensor-core path; any multiple of 32 up to 256
+                                on the SIMT path                                               */
+  int32_t page_size;         /* tokens per page; must be 16                                    */
+  int32_t num_pages;         /* pool capacity; page p addresses the same slot in every layer   */
+  int32_t dtype;             /* BICACHE_F32 or BICACHE_BF16: type of q/k/v/out and the pools   */
+  int32_t device;            /* CUDA device ordinal.  A negative value creates a host-only
+                                context: the store's bookkeeping and the depth rule work (pools
+                                and workspace may be NULL, put_prefix moves no data), the
+                                attention calls return UNSUPPORTED.  It exists so that the host
+                                logic can be exercised on a machine without a GPU; it computes
+                                nothing.                                                       */
+  const int32_t* initial_free_order; /* host, num_pages entries, a permutation of 0..num_pages-1
+                                giving the initial order of the free-page queue; NULL = 0,1,2,...
+                                Read during bicache_create only.                               */
+  void* k_pool;              /* device, bicache_pool_bytes() bytes, caller-owned               */
+  void* v_pool;              /* device, same size                                              */
+  void* workspace;           /* device scratch, caller-owned, 256-byte aligned                 */
+  size_t workspace_bytes;    /* >= bicache_workspace_bytes() for the batches to be run         */
+} bicache_config;
+
+/* Bytes of ONE pool (K or V): L * num_pages * Hkv * page_size * D elements.  The order of
+ * elements inside a page is private to the library: only bicache_put_prefix writes pools. */
+size_t bicache_pool_bytes(const bicache_config* cfg);
+
+/* Workspace needed to run batches of at most max_requests requests and max_total_rows query rows
+ * per call (bicache_attend: suffix rows; bicache_attend_full: all rows). */
+size_t bicache_workspace_bytes(const bicache_config* cfg, int64_t max_total_rows, int32_t max_requests);
+
+/* Create a context.  Clears the library's part of the workspace with a synchronous memset.
+ * INVALID for inconsistent sizes/pointers, UNSUPPORTED for page_size != 16 or an unsupported
+ * dtype/head_dim, NOMEM if the workspace cannot hold even an empty batch. */
+int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out);
+
+/* Synchronises the device and frees host state.  Device buffers stay the caller's. */
+int32_t bicache_destroy(bicache_ctx* ctx);
+
+/* Select the kernel family (BICACHE_PATH_*).  UNSUPPORTED if TENSOR is asked for a
+ * dtype/head_dim it does not cover. */
+int32_t bicache_set_path(bicache_ctx* ctx, int32_t path);
+
+/* Install the lookup table T (Sec. 5.1): table[idx] is the shallow depth for ratio bin
+ * idx = floor(100 * m / (m + n)), idx in 0..100.  n must be 101.  Host pointer; copied. */
+int32_t bicache_set_depth_table(bicache_ctx* ctx, const int32_t* table, int32_t n);
+
+/* (1) KV store insert (Sec. 5.2).  k, v: device, [L][m][Hkv][D] with `layer_stride` elements
+ * between layers (>= m*Hkv*D), rows dense.  m >= 1.
+ *   key present with the same m : hit, nothing is written, *was_hit = 1.
+ *   key present with another m  : INVALID.
+ *   ceil(m/16) > num_pages      : NOMEM, nothing evicted.
+ *   otherwise: evict whole prefixes, oldest insertion first (hits do not refresh age), until
+ *   enough pages are free (their pages join the tail of the free queue in page-table order),
+ *   take ceil(m/16) pages from the head of the queue, and enqueue the scatter of all L layers
+ *   on `stream`.  The caller may free k, v once the stream has passed this point.
+ * prefix_id (host, required) receives an id that is never reused.  was_hit (host, optional).
+ * pages_out (host, optional, capacity pages_cap) receives the page ids in token order;
+ * INVALID if pages_cap is too small (checked before anything changes). */
+int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const void* v,
+                           int64_t layer_stride, void* stream,
+                           int32_t* prefix_id, int32_t* was_hit, int32_t* pages_out, int32_t pages_cap);
+
+/* KV store lookup (Sec. 5.2 "On a cache hit").  NOTFOUND if the key is absent or evicted. */
+int32_t bicache_lookup_prefix(const bicache_ctx* ctx, uint64_t key, int32_t* prefix_id, int32_t* m);
+
+/* Page list of a live prefix, in token order.  *n receives the page count; pages_out (host) may be
+ * NULL to query the count only.  NOTFOUND for an evicted id, INVALID if cap is too small. */
+int32_t bicache_prefix_pages(const bicache_ctx* ctx, int32_t prefix_id, int32_t* pages_out, int32_t cap,
+                             int32_t* n);
+
+/* (2) Per-request shallow depth (Sec. 5.1/5.2).  Host arrays of length R.  prefix_len[i] = m_i
+ * shared-prefix tokens, nonshared_len[i] = n_i = every other token of the input string (prompt
+ * and all mask positions).  depth_out[i] = clamp(T[floor(100 m / (m + n))], 0, L); m <= 0 gives 0.
+ * Pure integer arithmetic, no device work.  INVALID if no table is installed or n_i < 0. */
+int32_t bicache_reuse_depth(const bicache_ctx* ctx, int32_t R, const int32_t* prefix_len,
+                            const int32_t* nonshared_len, int32_t* depth_out);
+
+/* (3) Shallow-layer attention of a ragged batch grouped by prefix, one layer (Eq. 2 + Eq. 4).
+ * Host metadata arrays of length R:
+ *   prefix_id[i]  live prefix id, or -1 for "no prefix"; equal ids must be contiguous (INVALID
+ *                 otherwise); NOTFOUND for an evicted id.
+ *   row_off[i]    first row of request i's suffix inside q, k, v, out, lse_out.
+ *   seqlen[i]     n_i >= 0 suffix rows (0 contributes nothing).
+ * Device tensors: q, out [rows][Hq][D] with q_row_stride / out_row_stride elements between rows;
+ * k, v [rows][Hkv][D] with kv_row_stride.  Heads are dense within a row.  Query head h reads KV
+ * head h / (Hq / Hkv).  lse_out: device fp32 [rows][Hq] (dense) or NULL; natural log of the sum of
+ * exp(softmax_scale * q.k) over all keys.  Each suffix row i,a attends over the prefix's m cached
+ * keys of `layer` and the request's own n_i suffix keys (itself included), no mask.  Only rows that
+ * belong to a request are written.  out is rounded to the context dtype (round to nearest even). */
+int32_t bicache_attend(bicache_ctx* ctx, int32_t layer, int32_t R, const int32_t* prefix_id,
+                       const int64_t* row_off, const int32_t* seqlen,
+                       const void* q, const void* k, const void* v,
+                       int64_t q_row_stride, int64_t kv_row_stride,
+                       void* out, int64_t out_row_stride, float* lse_out,
+                       float softmax_scale, void* stream);
+
+/* (4) Deep-layer fallback: full bidirectional attention (Eq. 2) of each request over its own
+ * seqlen[i] = N_i rows starting at row_off[i]; every row is a query.  Same tensor conventions as
+ * bicache_attend; `layer` is only range-checked (no cache is read). */
+int32_t bicache_attend_full(bicache_ctx* ctx, int32_t layer, int32_t R,
+                            const int64_t* row_off, const int32_t* seqlen,
+                            const void* q, const void* k, const void* v,
+                            int64_t q_row_stride, int64_t kv_row_stride,
+                            void* out, int64_t out_row_stride, float* lse_out,
+                            float softmax_scale, void* stream);
+
+/* Synchronises `stream` and returns the sticky device status: OK, or TIMEOUT if a kernel gave up
+ * on a bounded wait (its outputs are then undefined), or CUDA for a runtime error.  `clear` != 0
+ * resets the word. */
+int32_t bicache_device_status(bicache_ctx* ctx, void* stream, int32_t clear);
+
+/* Number of kernels this context has launched so far (for benchmarks' launch accounting). */
+int64_t bicache_launch_count(const bicache_ctx* ctx);
+
+/* Human-readable text for the last error of this context (host string, valid until next call). */
+const char* bicache_last_error(const bicache_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BICACHE_H_ */

@@ -1,0 +1,241 @@
+"""ctypes binding of libbicache.so: same names as the C ABI, argument marshalling only.
+
+Every step of the path runs inside the shared library's CUDA kernels; PyTorch is used for device
+buffers and streams.  A missing or unloadable library raises at first use: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+OK, ERR_INVALID, ERR_NOMEM, ERR_NOTFOUND, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = range(7)
+F32, BF16 = 0, 1
+PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+_STATUS_NAMES = ["OK", "INVALID", "NOMEM", "NOTFOUND", "CUDA", "TIMEOUT", "UNSUPPORTED"]
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbicache.so")
+
+EXPORTED = [
+    "bicache_pool_bytes", "bicache_workspace_bytes", "bicache_create", "bicache_destroy",
+    "bicache_set_path", "bicache_set_depth_table", "bicache_put_prefix", "bicache_lookup_prefix",
+    "bicache_prefix_pages", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
+    "bicache_device_status", "bicache_launch_count", "bicache_last_error",
+]
+
+
+class BiCacheError(RuntimeError):
+    def __init__(self, status, where, detail=""):
+        self.status = status
+        name = _STATUS_NAMES[status] if 0 <= status < len(_STATUS_NAMES) else str(status)
+        super().__init__("%s: BICACHE_ERR_%s %s" % (where, name, detail))
+
+
+class Config(C.Structure):
+    _fields_ = [
+        ("num_layers", C.c_int32), ("num_q_heads", C.c_int32), ("num_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("page_size", C.c_int32), ("num_pages", C.c_int32),
+        ("dtype", C.c_int32), ("device", C.c_int32),
+        ("initial_free_order", C.POINTER(C.c_int32)),
+        ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+    ]
+
+
+_lib = None
+
+
+def load_library():
+    """Load libbicache.so (built in-tree by __graft_entry__.build()).  Raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libbicache.so is not built (run __graft_entry__.build()); "
+                           "there is no fallback path: " + LIB_PATH)
+    lib = C.CDLL(LIB_PATH)
+    i32p, i64p, vp = C.POINTER(C.c_int32), C.POINTER(C.c_int64), C.c_void_p
+    lib.bicache_pool_bytes.restype = C.c_size_t
+    lib.bicache_pool_bytes.argtypes = [C.POINTER(Config)]
+    lib.bicache_workspace_bytes.restype = C.c_size_t
+    lib.bicache_workspace_bytes.argtypes = [C.POINTER(Config), C.c_int64, C.c_int32]
+    lib.bicache_create.restype = C.c_int32
+    lib.bicache_create.argtypes = [C.POINTER(Config), C.POINTER(vp)]
+    lib.bicache_destroy.restype = C.c_int32
+    lib.bicache_destroy.argtypes = [vp]
+    lib.bicache_set_path.restype = C.c_int32
+    lib.bicache_set_path.argtypes = [vp, C.c_int32]
+    lib.bicache_set_depth_table.restype = C.c_int32
+    lib.bicache_set_depth_table.argtypes = [vp, i32p, C.c_int32]
+    lib.bicache_put_prefix.restype = C.c_int32
+    lib.bicache_put_prefix.argtypes = [vp, C.c_uint64, C.c_int32, vp, vp, C.c_int64, vp, i32p, i32p, i32p, C.c_int32]
+    lib.bicache_lookup_prefix.restype = C.c_int32
+    lib.bicache_lookup_prefix.argtypes = [vp, C.c_uint64, i32p, i32p]
+    lib.bicache_prefix_pages.restype = C.c_int32
+    lib.bicache_prefix_pages.argtypes = [vp, C.c_int32, i32p, C.c_int32, i32p]
+    lib.bicache_reuse_depth.restype = C.c_int32
+    lib.bicache_reuse_depth.argtypes = [vp, C.c_int32, i32p, i32p, i32p]
+    lib.bicache_attend.restype = C.c_int32
+    lib.bicache_attend.argtypes = [vp, C.c_int32, C.c_int32, i32p, i64p, i32p, vp, vp, vp, C.c_int64, C.c_int64,
+                                   vp, C.c_int64, vp, C.c_float, vp]
+    lib.bicache_attend_full.restype = C.c_int32
+    lib.bicache_attend_full.argtypes = [vp, C.c_int32, C.c_int32, i64p, i32p, vp, vp, vp, C.c_int64, C.c_int64,
+                                        vp, C.c_int64, vp, C.c_float, vp]
+    lib.bicache_device_status.restype = C.c_int32
+    lib.bicache_device_status.argtypes = [vp, vp, C.c_int32]
+    lib.bicache_launch_count.restype = C.c_int64
+    lib.bicache_launch_count.argtypes = [vp]
+    lib.bicache_last_error.restype = C.c_char_p
+    lib.bicache_last_error.argtypes = [vp]
+    _lib = lib
+    return lib
+
+
+def _i32(a):
+    a = np.ascontiguousarray(a, dtype=np.int32)
+    return a, a.ctypes.data_as(C.POINTER(C.c_int32))
+
+
+def _i64(a):
+    a = np.ascontiguousarray(a, dtype=np.int64)
+    return a, a.ctypes.data_as(C.POINTER(C.c_int64))
+
+
+def _dtype_code(dtype):
+    if dtype == torch.float32:
+        return F32
+    if dtype == torch.bfloat16:
+        return BF16
+    raise BiCacheError(ERR_UNSUPPORTED, "dtype", str(dtype))
+
+
+class BiCache:
+    """One library context plus the torch-owned device buffers it needs."""
+
+    def __init__(self, num_layers, num_q_heads, num_kv_heads, head_dim, num_pages, dtype,
+                 max_total_rows, max_requests, device=0, page_size=16, free_order=None):
+        self.lib = load_library()
+        if not torch.cuda.is_available():
+            raise RuntimeError("BiCache needs a CUDA device; there is no CPU path")
+        self.device = torch.device("cuda", device)
+        self.dtype = dtype
+        self.L, self.Hq, self.Hkv, self.D = num_layers, num_q_heads, num_kv_heads, head_dim
+        cfg = Config(num_layers, num_q_heads, num_kv_heads, head_dim, page_size, num_pages,
+                     _dtype_code(dtype), device)
+        pool_bytes = self.lib.bicache_pool_bytes(C.byref(cfg))
+        ws_bytes = self.lib.bicache_workspace_bytes(C.byref(cfg), int(max_total_rows), int(max_requests))
+        if pool_bytes == 0 or ws_bytes == 0:
+            raise BiCacheError(ERR_INVALID, "bicache_pool_bytes/workspace_bytes")
+        # torch allocations are 512-byte aligned
+        self.k_pool = torch.empty(pool_bytes, dtype=torch.uint8, device=self.device)
+        self.v_pool = torch.empty(pool_bytes, dtype=torch.uint8, device=self.device)
+        self.workspace = torch.empty(ws_bytes, dtype=torch.uint8, device=self.device)
+        self._order = None
+        if free_order is not None:
+            self._order, ptr = _i32(free_order)
+            cfg.initial_free_order = ptr
+        cfg.k_pool, cfg.v_pool = self.k_pool.data_ptr(), self.v_pool.data_ptr()
+        cfg.workspace, cfg.workspace_bytes = self.workspace.data_ptr(), ws_bytes
+        self.ctx = C.c_void_p()
+        self._check(self.lib.bicache_create(C.byref(cfg), C.byref(self.ctx)), "bicache_create", use_ctx=False)
+
+    # -- helpers ---------------------------------------------------------------------------
+    def _check(self, status, where, use_ctx=True):
+        if status != OK:
+            detail = ""
+            if use_ctx and self.ctx:
+                detail = (self.lib.bicache_last_error(self.ctx) or b"").decode()
+            raise BiCacheError(status, where, detail)
+
+    @staticmethod
+    def _stream():
+        return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+    def close(self):
+        if getattr(self, "ctx", None) and self.ctx:
+            self.lib.bicache_destroy(self.ctx)
+            self.ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the C ABI, one method per call -----------------------------------------------------
+    def set_path(self, path):
+        self._check(self.lib.bicache_set_path(self.ctx, path), "bicache_set_path")
+
+    def set_depth_table(self, table):
+        arr, ptr = _i32(table)
+        self._check(self.lib.bicache_set_depth_table(self.ctx, ptr, len(arr)), "bicache_set_depth_table")
+
+    def put_prefix(self, key, k, v):
+        """k, v: [L, m, Hkv, D] device tensors.  Returns (prefix_id, was_hit, pages)."""
+        assert k.is_cuda and v.is_cuda and k.dtype == self.dtype and k.shape == v.shape
+        assert k.stride()[1:] == (self.Hkv * self.D, self.D, 1) and v.stride() == k.stride()
+        m = k.shape[1]
+        pid, hit = C.c_int32(-1), C.c_int32(0)
+        cap = (m + 15) // 16
+        pages = np.zeros(max(cap, 1), dtype=np.int32)
+        st = self.lib.bicache_put_prefix(self.ctx, C.c_uint64(key), m, k.data_ptr(), v.data_ptr(),
+                                         k.stride(0), self._stream(), C.byref(pid), C.byref(hit),
+                                         pages.ctypes.data_as(C.POINTER(C.c_int32)), cap)
+        self._check(st, "bicache_put_prefix")
+        return pid.value, bool(hit.value), pages[:cap].tolist()
+
+    def lookup_prefix(self, key):
+        pid, m = C.c_int32(-1), C.c_int32(0)
+        self._check(self.lib.bicache_lookup_prefix(self.ctx, C.c_uint64(key), C.byref(pid), C.byref(m)),
+                    "bicache_lookup_prefix")
+        return pid.value, m.value
+
+    def prefix_pages(self, prefix_id):
+        n = C.c_int32(0)
+        self._check(self.lib.bicache_prefix_pages(self.ctx, prefix_id, None, 0, C.byref(n)), "bicache_prefix_pages")
+        pages = np.zeros(max(n.value, 1), dtype=np.int32)
+        self._check(self.lib.bicache_prefix_pages(self.ctx, prefix_id, pages.ctypes.data_as(C.POINTER(C.c_int32)),
+                                                  n.value, C.byref(n)), "bicache_prefix_pages")
+        return pages[:n.value].tolist()
+
+    def reuse_depth(self, prefix_len, nonshared_len):
+        a, pa = _i32(prefix_len)
+        b, pb = _i32(nonshared_len)
+        out = np.zeros(max(len(a), 1), dtype=np.int32)
+        self._check(self.lib.bicache_reuse_depth(self.ctx, len(a), pa, pb, out.ctypes.data_as(C.POINTER(C.c_int32))),
+                    "bicache_reuse_depth")
+        return out[:len(a)]
+
+    def _tensor_args(self, q, k, v, out, lse):
+        for t in (q, k, v, out):
+            assert t.is_cuda and t.dtype == self.dtype and t.dim() == 3 and t.stride(2) == 1 and t.stride(1) == self.D
+        assert lse is None or (lse.dtype == torch.float32 and lse.is_contiguous())
+        return (q.data_ptr(), k.data_ptr(), v.data_ptr(), q.stride(0), k.stride(0),
+                out.data_ptr(), out.stride(0), lse.data_ptr() if lse is not None else None)
+
+    def attend(self, layer, prefix_id, row_off, seqlen, q, k, v, out, lse=None, scale=None):
+        pid, ppid = _i32(prefix_id)
+        off, poff = _i64(row_off)
+        n, pn = _i32(seqlen)
+        qp, kp, vp_, qs, ks, op, os_, lp = self._tensor_args(q, k, v, out, lse)
+        scale = self.D ** -0.5 if scale is None else scale
+        st = self.lib.bicache_attend(self.ctx, layer, len(n), ppid, poff, pn, qp, kp, vp_, qs, ks, op, os_, lp,
+                                     C.c_float(scale), self._stream())
+        self._check(st, "bicache_attend")
+
+    def attend_full(self, layer, row_off, seqlen, q, k, v, out, lse=None, scale=None):
+        off, poff = _i64(row_off)
+        n, pn = _i32(seqlen)
+        qp, kp, vp_, qs, ks, op, os_, lp = self._tensor_args(q, k, v, out, lse)
+        scale = self.D ** -0.5 if scale is None else scale
+        st = self.lib.bicache_attend_full(self.ctx, layer, len(n), poff, pn, qp, kp, vp_, qs, ks, op, os_, lp,
+                                          C.c_float(scale), self._stream())
+        self._check(st, "bicache_attend_full")
+
+    def device_status(self, clear=False):
+        return self.lib.bicache_device_status(self.ctx, self._stream(), 1 if clear else 0)
+
+    def launch_count(self):
+        return int(self.lib.bicache_launch_count(self.ctx))

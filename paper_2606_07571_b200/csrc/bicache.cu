@@ -1,0 +1,619 @@
+// Host runtime and C ABI of the BiCache attention library (see include/bicache.h).
+//
+// Host side: the prefix KV store's bookkeeping (key map, FIFO eviction, free-page queue), the
+// reuse-depth rule, and the per-call schedule (which 128-row work items exist, which keys they
+// cover), cached across the layers of a denoising step.  Device side: kernels in the .cuh files.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <list>
+#include <new>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/bicache.h"
+#include "common.cuh"
+#include "simt_kernels.cuh"
+#include "tc_attention.cuh"
+
+using namespace bicache;
+
+namespace {
+
+constexpr int kNumSlots = 4;                 // cached schedules kept on the device
+constexpr size_t kStatusBytes = 256;
+constexpr int kTargetCtas = 296;             // two waves of 148 SMs: aim of the key split
+constexpr long long kMaxPartialRowHeads = (long long)kTargetCtas * kTileRows;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct PrefixEntry {
+  uint64_t key;
+  int32_t id;
+  int32_t m;
+  std::vector<int32_t> pages;
+};
+
+struct CachedSchedule {
+  bool valid = false;
+  uint64_t last_use = 0;
+  int kind = 0;                               // 0 attend, 1 attend_full
+  std::vector<int32_t> prefix_id;
+  std::vector<int64_t> row_off;
+  std::vector<int32_t> seqlen;
+  int num_items = 0, num_splits = 1, split_keys = 0, total_tokens = 0;
+  size_t reqs_off = 0, pages_off = 0, items_off = 0;   // byte offsets inside the slot
+};
+
+}  // namespace
+
+struct bicache_ctx {
+  bicache_config cfg;
+  int esize = 2;
+  bool swizzled = false;
+  bool tensor_ok = false;
+  bool host_only = false;                                         // cfg.device < 0: bookkeeping only
+  int path = BICACHE_PATH_AUTO;
+  std::deque<int32_t> free_pages;
+  std::list<PrefixEntry> fifo;                                    // insertion order, oldest first
+  std::unordered_map<uint64_t, std::list<PrefixEntry>::iterator> by_key;
+  std::unordered_map<int32_t, std::list<PrefixEntry>::iterator> by_id;
+  int32_t next_id = 0;
+  std::vector<int32_t> depth_table;
+  // workspace carving
+  int* d_status = nullptr;
+  char* d_slots = nullptr;
+  size_t slot_bytes = 0;
+  float* d_part_o = nullptr;
+  float* d_part_lse = nullptr;
+  long long part_capacity_rowheads = 0;
+  int* d_put_pages = nullptr;                                     // page list staging for put_prefix
+  CachedSchedule slots[kNumSlots];
+  uint64_t use_counter = 0;
+  int64_t launches = 0;
+  int sm_count = 148;
+  std::string last_error;
+};
+
+namespace {
+
+int fail(const bicache_ctx* ctx, int code, const std::string& msg) {
+  if (ctx) const_cast<bicache_ctx*>(ctx)->last_error = msg;
+  return code;
+}
+
+bool supported(const bicache_config* c, int* esize, bool* swz, bool* tensor_ok) {
+  if (c->dtype != BICACHE_F32 && c->dtype != BICACHE_BF16) return false;
+  if (c->page_size != kPageSize) return false;
+  if (c->head_dim < 32 || c->head_dim > kSimtMaxD || c->head_dim % 32) return false;
+  *esize = c->dtype == BICACHE_F32 ? 4 : 2;
+  *swz = c->dtype == BICACHE_BF16 && c->head_dim == 128;
+  *tensor_ok = *swz && kTensorPathBuilt;
+  return true;
+}
+
+bool sane(const bicache_config* c) {
+  return c && c->num_layers >= 1 && c->num_kv_heads >= 1 && c->num_q_heads >= c->num_kv_heads &&
+         c->num_q_heads % c->num_kv_heads == 0 && c->num_pages >= 1 && c->head_dim >= 1;
+}
+
+size_t slot_bytes_for(const bicache_config* c, int64_t max_rows, int32_t max_req) {
+  const int G = c->num_q_heads / c->num_kv_heads;
+  const long long tiles = (max_rows * G + kTileRows - 1) / kTileRows + max_req;
+  const long long max_items = std::max<long long>(tiles * c->num_kv_heads, 1) + 2LL * kTargetCtas;
+  return align_up((size_t)max_req * sizeof(ReqMeta) + 16, 256) +
+         align_up((size_t)c->num_pages * sizeof(int) + 16, 256) +
+         align_up((size_t)max_items * sizeof(WorkItem) + 16, 256);
+}
+
+size_t partial_bytes_for(const bicache_config* c) {
+  return align_up((size_t)kMaxPartialRowHeads * (c->head_dim + 1) * sizeof(float), 256);
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+PoolView pool_view(const bicache_ctx* ctx) {
+  PoolView p;
+  p.k = static_cast<const char*>(ctx->cfg.k_pool);
+  p.v = static_cast<const char*>(ctx->cfg.v_pool);
+  p.page_bytes = kPageSize * ctx->cfg.head_dim * ctx->esize;
+  p.num_kv_heads = ctx->cfg.num_kv_heads;
+  p.layer_bytes = (long long)ctx->cfg.num_pages * ctx->cfg.num_kv_heads * p.page_bytes;
+  p.swizzled = ctx->swizzled ? 1 : 0;
+  return p;
+}
+
+// Build (or find) the device-resident schedule for this batch.  Returns the slot index or -1.
+int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id, const int64_t* row_off,
+                     const int32_t* seqlen, cudaStream_t stream, int* status) {
+  *status = BICACHE_OK;
+  ctx->use_counter++;
+  for (int s = 0; s < kNumSlots; ++s) {
+    CachedSchedule& c = ctx->slots[s];
+    if (!c.valid || c.kind != kind || (int)c.seqlen.size() != R) continue;
+    if (std::memcmp(c.row_off.data(), row_off, sizeof(int64_t) * R) != 0) continue;
+    if (std::memcmp(c.seqlen.data(), seqlen, sizeof(int32_t) * R) != 0) continue;
+    if (kind == 0 && std::memcmp(c.prefix_id.data(), prefix_id, sizeof(int32_t) * R) != 0) continue;
+    c.last_use = ctx->use_counter;
+    return s;
+  }
+  const int Hkv = ctx->cfg.num_kv_heads, G = ctx->cfg.num_q_heads / Hkv;
+  std::vector<ReqMeta> reqs(R);
+  std::vector<int> pages;
+  long long tok = 0;
+  int max_keys = 0;
+  long long unsplit_items = 0;
+  int last_pid = -1, last_page_off = 0;
+  for (int i = 0; i < R; ++i) {
+    ReqMeta& r = reqs[i];
+    r.row_off = row_off[i];
+    r.n = seqlen[i];
+    r.m = 0;
+    r.page_off = 0;
+    r.tok_off = (int)tok;
+    tok += seqlen[i];
+    if (kind == 0 && prefix_id[i] >= 0) {
+      const PrefixEntry& e = *ctx->by_id.at(prefix_id[i]);
+      r.m = e.m;
+      if (prefix_id[i] != last_pid) {
+        last_pid = prefix_id[i];
+        last_page_off = (int)pages.size();
+        pages.insert(pages.end(), e.pages.begin(), e.pages.end());
+      }
+      r.page_off = last_page_off;
+    }
+    if (r.n > 0) {
+      max_keys = std::max(max_keys, r.m + r.n);
+      unsplit_items += (long long)((r.n * (long long)G + kTileRows - 1) / kTileRows) * Hkv;
+    }
+  }
+  // Split the keys across CTAs when the batch has too few row tiles to fill the GPU.
+  int num_splits = 1, split_keys = 0;
+  if (unsplit_items > 0 && unsplit_items * 2 <= ctx->sm_count && max_keys >= 8 * kTileKeys) {
+    const int key_tiles = (max_keys + kTileKeys - 1) / kTileKeys;
+    int want = (int)std::min<long long>((kTargetCtas + unsplit_items - 1) / unsplit_items, key_tiles / 2);
+    while (want > 1 && tok * ctx->cfg.num_q_heads * want > ctx->part_capacity_rowheads) --want;
+    if (want > 1) {
+      const int tiles_per_split = (key_tiles + want - 1) / want;
+      split_keys = tiles_per_split * kTileKeys;
+      num_splits = (key_tiles + tiles_per_split - 1) / tiles_per_split;
+    }
+  }
+  std::vector<WorkItem> items;
+  items.reserve((size_t)unsplit_items * num_splits);
+  for (int sp = 0; sp < num_splits; ++sp) {
+    const size_t first = items.size();
+    for (int i = 0; i < R; ++i) {
+      if (reqs[i].n <= 0) continue;
+      const int prow = reqs[i].n * G;
+      for (int hk = 0; hk < Hkv; ++hk)
+        for (int r0 = 0; r0 < prow; r0 += kTileRows) items.push_back(WorkItem{i, hk, r0, sp});
+    }
+    // Longest key range first (the tail of the launch is then made of short items); items of one
+    // KV head and request stay adjacent so that concurrently running CTAs share K/V tiles in L2.
+    std::stable_sort(items.begin() + first, items.end(), [&](const WorkItem& a, const WorkItem& b) {
+      const int ka = reqs[a.req].m + reqs[a.req].n, kb = reqs[b.req].m + reqs[b.req].n;
+      return ka > kb;
+    });
+  }
+  const size_t reqs_off = 0;
+  const size_t pages_off = align_up(reqs_off + reqs.size() * sizeof(ReqMeta) + 16, 256);
+  const size_t items_off = align_up(pages_off + pages.size() * sizeof(int) + 16, 256);
+  const size_t total = items_off + items.size() * sizeof(WorkItem);
+  if (total > ctx->slot_bytes) {
+    *status = fail(ctx, BICACHE_ERR_NOMEM, "workspace too small for this batch's schedule");
+    return -1;
+  }
+  int victim = 0;
+  for (int s = 0; s < kNumSlots; ++s) {
+    if (!ctx->slots[s].valid) { victim = s; break; }
+    if (ctx->slots[s].last_use < ctx->slots[victim].last_use) victim = s;
+  }
+  std::vector<char> blob(total, 0);
+  if (!reqs.empty()) std::memcpy(blob.data() + reqs_off, reqs.data(), reqs.size() * sizeof(ReqMeta));
+  if (!pages.empty()) std::memcpy(blob.data() + pages_off, pages.data(), pages.size() * sizeof(int));
+  if (!items.empty()) std::memcpy(blob.data() + items_off, items.data(), items.size() * sizeof(WorkItem));
+  CachedSchedule& c = ctx->slots[victim];
+  c.valid = false;
+  if (total > 0) {
+    // Pageable source: the runtime stages it before returning, so `blob` may die with this scope.
+    cudaError_t e = cudaMemcpyAsync(ctx->d_slots + (size_t)victim * ctx->slot_bytes, blob.data(), total,
+                                    cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) {
+      *status = fail(ctx, BICACHE_ERR_CUDA, std::string("schedule upload: ") + cudaGetErrorString(e));
+      return -1;
+    }
+  }
+  c.kind = kind;
+  c.prefix_id.assign(prefix_id ? prefix_id : nullptr, prefix_id ? prefix_id + R : nullptr);
+  c.row_off.assign(row_off, row_off + R);
+  c.seqlen.assign(seqlen, seqlen + R);
+  c.num_items = (int)items.size();
+  c.num_splits = num_splits;
+  c.split_keys = split_keys;
+  c.total_tokens = (int)tok;
+  c.reqs_off = reqs_off;
+  c.pages_off = pages_off;
+  c.items_off = items_off;
+  c.last_use = ctx->use_counter;
+  c.valid = true;
+  return victim;
+}
+
+void drop_schedules(bicache_ctx* ctx) {
+  for (int s = 0; s < kNumSlots; ++s) ctx->slots[s].valid = false;
+}
+
+int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const int32_t* prefix_id,
+                  const int64_t* row_off, const int32_t* seqlen, const void* q, const void* k, const void* v,
+                  int64_t q_row_stride, int64_t kv_row_stride, void* out, int64_t out_row_stride,
+                  float* lse_out, float softmax_scale, void* stream_) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  if (ctx->host_only) return fail(ctx, BICACHE_ERR_UNSUPPORTED, "host-only context has no device path");
+  const bicache_config& cfg = ctx->cfg;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  if (layer < 0 || layer >= cfg.num_layers) return fail(ctx, BICACHE_ERR_INVALID, "layer out of range");
+  if (R < 0) return fail(ctx, BICACHE_ERR_INVALID, "negative request count");
+  if (R == 0) return BICACHE_OK;
+  if (!row_off || !seqlen || (kind == 0 && !prefix_id))
+    return fail(ctx, BICACHE_ERR_INVALID, "null metadata array");
+  if (!q || !k || !v || !out) return fail(ctx, BICACHE_ERR_INVALID, "null tensor pointer");
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) ||
+      (lse_out && (reinterpret_cast<uintptr_t>(lse_out) & 3)))
+    return fail(ctx, BICACHE_ERR_INVALID, "tensor pointer not 16-byte aligned");
+  const int D = cfg.head_dim;
+  if (q_row_stride < (int64_t)cfg.num_q_heads * D || out_row_stride < (int64_t)cfg.num_q_heads * D ||
+      kv_row_stride < (int64_t)cfg.num_kv_heads * D || (q_row_stride * ctx->esize) % 16 ||
+      (kv_row_stride * ctx->esize) % 16 || (out_row_stride * ctx->esize) % 16)
+    return fail(ctx, BICACHE_ERR_INVALID, "bad row stride");
+  long long total = 0;
+  for (int i = 0; i < R; ++i) {
+    if (seqlen[i] < 0 || row_off[i] < 0) return fail(ctx, BICACHE_ERR_INVALID, "negative length or offset");
+    total += seqlen[i];
+  }
+  if (total > 0x7fffffffLL / std::max(1, cfg.num_q_heads / cfg.num_kv_heads))
+    return fail(ctx, BICACHE_ERR_INVALID, "batch too large");
+  if (kind == 0) {
+    // equal ids contiguous; every id live
+    std::vector<int32_t> seen;
+    for (int i = 0; i < R; ++i) {
+      const int32_t p = prefix_id[i];
+      if (p < -1) return fail(ctx, BICACHE_ERR_INVALID, "bad prefix id");
+      if (i > 0 && p == prefix_id[i - 1]) continue;
+      if (p >= 0) {
+        if (std::find(seen.begin(), seen.end(), p) != seen.end())
+          return fail(ctx, BICACHE_ERR_INVALID, "requests of one prefix are not contiguous");
+        seen.push_back(p);
+        if (ctx->by_id.find(p) == ctx->by_id.end())
+          return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+      }
+    }
+  }
+  if (total == 0) return BICACHE_OK;
+
+  int st = BICACHE_OK;
+  const int slot = prepare_schedule(ctx, kind, R, prefix_id, row_off, seqlen, stream, &st);
+  if (slot < 0) return st;
+  const CachedSchedule& c = ctx->slots[slot];
+  char* base = ctx->d_slots + (size_t)slot * ctx->slot_bytes;
+  ScheduleView sv;
+  sv.reqs = reinterpret_cast<const ReqMeta*>(base + c.reqs_off);
+  sv.pages = reinterpret_cast<const int*>(base + c.pages_off);
+  sv.items = reinterpret_cast<const WorkItem*>(base + c.items_off);
+  sv.num_items = c.num_items;
+  sv.num_splits = c.num_splits;
+  sv.split_keys = c.split_keys;
+
+  TensorArgs t;
+  t.q = static_cast<const char*>(q);
+  t.k = static_cast<const char*>(k);
+  t.v = static_cast<const char*>(v);
+  t.out = static_cast<char*>(out);
+  t.lse = lse_out;
+  t.q_stride = q_row_stride;
+  t.kv_stride = kv_row_stride;
+  t.out_stride = out_row_stride;
+  t.Hq = cfg.num_q_heads;
+  t.Hkv = cfg.num_kv_heads;
+  t.D = D;
+  t.layer = layer;
+  t.scale = softmax_scale;
+  t.part_o = ctx->d_part_o;
+  t.part_lse = ctx->d_part_lse;
+  t.total_tokens = c.total_tokens;
+  const PoolView pool = pool_view(ctx);
+
+  const bool use_tensor = ctx->tensor_ok && ctx->path != BICACHE_PATH_SIMT;
+  cudaError_t e;
+  if (use_tensor) {
+    e = launch_tc_attention(sv, pool, t, ctx->d_status, stream);
+  } else if (cfg.dtype == BICACHE_F32) {
+    simt_attention_kernel<float><<<c.num_items, kSimtWarps * 32, 0, stream>>>(sv, pool, t);
+    e = cudaGetLastError();
+  } else {
+    simt_attention_kernel<__nv_bfloat16><<<c.num_items, kSimtWarps * 32, 0, stream>>>(sv, pool, t);
+    e = cudaGetLastError();
+  }
+  ctx->launches++;
+  if (e != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
+  if (c.num_splits > 1) {
+    const int grid = c.num_items / c.num_splits;
+    if (cfg.dtype == BICACHE_F32)
+      merge_partials_kernel<float><<<grid, kSimtWarps * 32, 0, stream>>>(sv, t);
+    else
+      merge_partials_kernel<__nv_bfloat16><<<grid, kSimtWarps * 32, 0, stream>>>(sv, t);
+    ctx->launches++;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("merge launch: ") + cudaGetErrorString(e));
+  }
+  return BICACHE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t bicache_pool_bytes(const bicache_config* cfg) {
+  if (!sane(cfg)) return 0;
+  const size_t es = cfg->dtype == BICACHE_F32 ? 4 : 2;
+  return (size_t)cfg->num_layers * cfg->num_pages * cfg->num_kv_heads * cfg->page_size * cfg->head_dim * es;
+}
+
+size_t bicache_workspace_bytes(const bicache_config* cfg, int64_t max_total_rows, int32_t max_requests) {
+  if (!sane(cfg) || max_total_rows < 0 || max_requests < 0) return 0;
+  return kStatusBytes + kNumSlots * slot_bytes_for(cfg, max_total_rows, max_requests) +
+         partial_bytes_for(cfg) + align_up((size_t)cfg->num_pages * sizeof(int) + 16, 256);
+}
+
+int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
+  if (!out) return BICACHE_ERR_INVALID;
+  *out = nullptr;
+  if (!sane(cfg)) return BICACHE_ERR_INVALID;
+  int esize;
+  bool swz, tensor_ok;
+  if (!supported(cfg, &esize, &swz, &tensor_ok)) return BICACHE_ERR_UNSUPPORTED;
+  const bool host_only = cfg->device < 0;
+  const size_t part = partial_bytes_for(cfg);
+  const size_t put_pages = align_up((size_t)cfg->num_pages * sizeof(int) + 16, 256);
+  if (!host_only) {
+    if (!cfg->k_pool || !cfg->v_pool || !cfg->workspace) return BICACHE_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(cfg->k_pool) & 255) || (reinterpret_cast<uintptr_t>(cfg->v_pool) & 255) ||
+        (reinterpret_cast<uintptr_t>(cfg->workspace) & 255))
+      return BICACHE_ERR_INVALID;
+    if (cfg->workspace_bytes < kStatusBytes + part + put_pages + kNumSlots * slot_bytes_for(cfg, 0, 0))
+      return BICACHE_ERR_NOMEM;
+  }
+  std::vector<int32_t> order(cfg->num_pages);
+  if (cfg->initial_free_order) {
+    std::vector<char> seen(cfg->num_pages, 0);
+    for (int i = 0; i < cfg->num_pages; ++i) {
+      const int32_t p = cfg->initial_free_order[i];
+      if (p < 0 || p >= cfg->num_pages || seen[p]) return BICACHE_ERR_INVALID;
+      seen[p] = 1;
+      order[i] = p;
+    }
+  } else {
+    for (int i = 0; i < cfg->num_pages; ++i) order[i] = i;
+  }
+  if (!host_only && cudaSetDevice(cfg->device) != cudaSuccess) return BICACHE_ERR_CUDA;
+  bicache_ctx* ctx = new (std::nothrow) bicache_ctx();
+  if (!ctx) return BICACHE_ERR_NOMEM;
+  ctx->host_only = host_only;
+  ctx->cfg = *cfg;
+  ctx->cfg.initial_free_order = nullptr;
+  ctx->esize = esize;
+  ctx->swizzled = swz;
+  ctx->tensor_ok = tensor_ok;
+  ctx->free_pages.assign(order.begin(), order.end());
+  if (host_only) {
+    *out = ctx;
+    return BICACHE_OK;
+  }
+  char* ws = static_cast<char*>(cfg->workspace);
+  ctx->d_status = reinterpret_cast<int*>(ws);
+  ctx->d_part_o = reinterpret_cast<float*>(ws + kStatusBytes);
+  ctx->d_part_lse = ctx->d_part_o + (size_t)kMaxPartialRowHeads * cfg->head_dim;
+  ctx->part_capacity_rowheads = kMaxPartialRowHeads;
+  ctx->d_put_pages = reinterpret_cast<int*>(ws + kStatusBytes + part);
+  ctx->d_slots = ws + kStatusBytes + part + put_pages;
+  ctx->slot_bytes = (cfg->workspace_bytes - (kStatusBytes + part + put_pages)) / kNumSlots / 256 * 256;
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess && sms > 0)
+    ctx->sm_count = sms;
+  if (cudaMemset(ws, 0, kStatusBytes) != cudaSuccess) {
+    delete ctx;
+    return BICACHE_ERR_CUDA;
+  }
+  if (tensor_ok) {
+    cudaError_t e = configure_tc_attention();
+    if (e != cudaSuccess) {
+      delete ctx;
+      return BICACHE_ERR_CUDA;
+    }
+  }
+  *out = ctx;
+  return BICACHE_OK;
+}
+
+int32_t bicache_destroy(bicache_ctx* ctx) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  if (ctx->host_only) {
+    delete ctx;
+    return BICACHE_OK;
+  }
+  cudaSetDevice(ctx->cfg.device);
+  cudaError_t e = cudaDeviceSynchronize();
+  delete ctx;
+  return e == cudaSuccess ? BICACHE_OK : BICACHE_ERR_CUDA;
+}
+
+int32_t bicache_set_path(bicache_ctx* ctx, int32_t path) {
+  if (!ctx || path < BICACHE_PATH_AUTO || path > BICACHE_PATH_TENSOR) return BICACHE_ERR_INVALID;
+  if (path == BICACHE_PATH_TENSOR && !ctx->tensor_ok)
+    return fail(ctx, BICACHE_ERR_UNSUPPORTED, "tensor-core path needs bf16 and head_dim 128");
+  ctx->path = path;
+  return BICACHE_OK;
+}
+
+int32_t bicache_set_depth_table(bicache_ctx* ctx, const int32_t* table, int32_t n) {
+  if (!ctx || !table || n != 101) return fail(ctx, BICACHE_ERR_INVALID, "depth table must have 101 entries");
+  ctx->depth_table.assign(table, table + n);
+  return BICACHE_OK;
+}
+
+int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const void* v,
+                           int64_t layer_stride, void* stream_, int32_t* prefix_id, int32_t* was_hit,
+                           int32_t* pages_out, int32_t pages_cap) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  if (!prefix_id) return fail(ctx, BICACHE_ERR_INVALID, "prefix_id is required");
+  if (m < 1) return fail(ctx, BICACHE_ERR_INVALID, "empty prefix");
+  const bicache_config& cfg = ctx->cfg;
+  const int need = (m + kPageSize - 1) / kPageSize;
+  auto found = ctx->by_key.find(key);
+  if (found != ctx->by_key.end()) {
+    const PrefixEntry& e = *found->second;
+    if (e.m != m) return fail(ctx, BICACHE_ERR_INVALID, "key already present with another length");
+    if (pages_out && pages_cap < need) return fail(ctx, BICACHE_ERR_INVALID, "pages_out too small");
+    *prefix_id = e.id;
+    if (was_hit) *was_hit = 1;
+    if (pages_out) std::copy(e.pages.begin(), e.pages.end(), pages_out);
+    return BICACHE_OK;
+  }
+  if (!ctx->host_only && (!k || !v || !aligned16(k) || !aligned16(v)))
+    return fail(ctx, BICACHE_ERR_INVALID, "bad k/v pointer");
+  const int64_t row_elems = (int64_t)cfg.num_kv_heads * cfg.head_dim;
+  if (layer_stride < (int64_t)m * row_elems || (layer_stride * ctx->esize) % 16)
+    return fail(ctx, BICACHE_ERR_INVALID, "bad layer stride");
+  if (need > cfg.num_pages) return fail(ctx, BICACHE_ERR_NOMEM, "prefix larger than the whole pool");
+  if (pages_out && pages_cap < need) return fail(ctx, BICACHE_ERR_INVALID, "pages_out too small");
+  while ((int)ctx->free_pages.size() < need) {
+    PrefixEntry& old = ctx->fifo.front();
+    for (int32_t p : old.pages) ctx->free_pages.push_back(p);
+    ctx->by_key.erase(old.key);
+    ctx->by_id.erase(old.id);
+    ctx->fifo.pop_front();
+    drop_schedules(ctx);
+  }
+  PrefixEntry e;
+  e.key = key;
+  e.m = m;
+  e.id = ctx->next_id++;
+  e.pages.resize(need);
+  for (int i = 0; i < need; ++i) {
+    e.pages[i] = ctx->free_pages.front();
+    ctx->free_pages.pop_front();
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  cudaError_t ce = cudaSuccess;
+  if (!ctx->host_only)
+    ce = cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+  if (ce == cudaSuccess && !ctx->host_only) {
+    const int chunks_per_row = cfg.head_dim * ctx->esize / 16;
+    const long long total = (long long)cfg.num_layers * need * kPageSize * cfg.num_kv_heads * chunks_per_row;
+    const int threads = 256;
+    const int blocks = (int)std::min<long long>((total + threads - 1) / threads, (long long)ctx->sm_count * 16);
+    const PoolView pv = pool_view(ctx);
+    scatter_prefix_kernel<<<blocks, threads, 0, stream>>>(
+        static_cast<const char*>(k), static_cast<const char*>(v), static_cast<char*>(cfg.k_pool),
+        static_cast<char*>(cfg.v_pool), ctx->d_put_pages, need, m, cfg.num_layers, cfg.num_kv_heads,
+        chunks_per_row, layer_stride * ctx->esize, pv.layer_bytes, pv.page_bytes, pv.swizzled);
+    ctx->launches++;
+    ce = cudaGetLastError();
+  }
+  if (ce != cudaSuccess) {
+    for (auto it = e.pages.rbegin(); it != e.pages.rend(); ++it) ctx->free_pages.push_front(*it);
+    ctx->next_id--;
+    return fail(ctx, BICACHE_ERR_CUDA, std::string("put_prefix: ") + cudaGetErrorString(ce));
+  }
+  *prefix_id = e.id;
+  if (was_hit) *was_hit = 0;
+  if (pages_out) std::copy(e.pages.begin(), e.pages.end(), pages_out);
+  ctx->fifo.push_back(std::move(e));
+  auto it = std::prev(ctx->fifo.end());
+  ctx->by_key[key] = it;
+  ctx->by_id[it->id] = it;
+  return BICACHE_OK;
+}
+
+int32_t bicache_lookup_prefix(const bicache_ctx* ctx, uint64_t key, int32_t* prefix_id, int32_t* m) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  auto found = ctx->by_key.find(key);
+  if (found == ctx->by_key.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown key");
+  if (prefix_id) *prefix_id = found->second->id;
+  if (m) *m = found->second->m;
+  return BICACHE_OK;
+}
+
+int32_t bicache_prefix_pages(const bicache_ctx* ctx, int32_t prefix_id, int32_t* pages_out, int32_t cap,
+                             int32_t* n) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  auto found = ctx->by_id.find(prefix_id);
+  if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+  const PrefixEntry& e = *found->second;
+  if (n) *n = (int32_t)e.pages.size();
+  if (pages_out) {
+    if (cap < (int32_t)e.pages.size()) return fail(ctx, BICACHE_ERR_INVALID, "pages_out too small");
+    std::copy(e.pages.begin(), e.pages.end(), pages_out);
+  }
+  return BICACHE_OK;
+}
+
+int32_t bicache_reuse_depth(const bicache_ctx* ctx, int32_t R, const int32_t* prefix_len,
+                            const int32_t* nonshared_len, int32_t* depth_out) {
+  if (!ctx || R < 0 || (R > 0 && (!prefix_len || !nonshared_len || !depth_out)))
+    return fail(ctx, BICACHE_ERR_INVALID, "bad arguments");
+  if (ctx->depth_table.size() != 101) return fail(ctx, BICACHE_ERR_INVALID, "no depth table installed");
+  for (int i = 0; i < R; ++i)
+    if (nonshared_len[i] < 0) return fail(ctx, BICACHE_ERR_INVALID, "negative non-shared length");
+  for (int i = 0; i < R; ++i) {
+    const int64_t m = prefix_len[i], n = nonshared_len[i];
+    int32_t b = 0;
+    if (m > 0) {
+      const int64_t idx = (100 * m) / (m + n);
+      b = ctx->depth_table[(size_t)idx];
+      b = std::max<int32_t>(0, std::min<int32_t>(ctx->cfg.num_layers, b));
+    }
+    depth_out[i] = b;
+  }
+  return BICACHE_OK;
+}
+
+int32_t bicache_attend(bicache_ctx* ctx, int32_t layer, int32_t R, const int32_t* prefix_id,
+                       const int64_t* row_off, const int32_t* seqlen, const void* q, const void* k,
+                       const void* v, int64_t q_row_stride, int64_t kv_row_stride, void* out,
+                       int64_t out_row_stride, float* lse_out, float softmax_scale, void* stream) {
+  return run_attention(ctx, 0, layer, R, prefix_id, row_off, seqlen, q, k, v, q_row_stride, kv_row_stride, out,
+                       out_row_stride, lse_out, softmax_scale, stream);
+}
+
+int32_t bicache_attend_full(bicache_ctx* ctx, int32_t layer, int32_t R, const int64_t* row_off,
+                            const int32_t* seqlen, const void* q, const void* k, const void* v,
+                            int64_t q_row_stride, int64_t kv_row_stride, void* out, int64_t out_row_stride,
+                            float* lse_out, float softmax_scale, void* stream) {
+  return run_attention(ctx, 1, layer, R, nullptr, row_off, seqlen, q, k, v, q_row_stride, kv_row_stride, out,
+                       out_row_stride, lse_out, softmax_scale, stream);
+}
+
+int32_t bicache_device_status(bicache_ctx* ctx, void* stream, int32_t clear) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  if (ctx->host_only) return BICACHE_OK;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(s) != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, "stream synchronize failed");
+  int word = 0;
+  if (cudaMemcpy(&word, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return fail(ctx, BICACHE_ERR_CUDA, "status read failed");
+  if (clear && word != 0) cudaMemset(ctx->d_status, 0, kStatusBytes);
+  if (word == kDevOk) return BICACHE_OK;
+  return fail(ctx, word == kDevTimeout ? BICACHE_ERR_TIMEOUT : BICACHE_ERR_CUDA, "device-side wait gave up");
+}
+
+int64_t bicache_launch_count(const bicache_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* bicache_last_error(const bicache_ctx* ctx) { return ctx ? ctx->last_error.c_str() : "null context"; }
+
+}  // extern "C"

@@ -1,0 +1,72 @@
+// Shared host/device definitions of the BiCache attention library: the device-side batch
+// description ("schedule") and the private element order of a cache page.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace bicache {
+
+constexpr int kPageSize = 16;          // tokens per page
+constexpr int kTileRows = 128;         // query rows of one work item (one tensor-core M tile)
+constexpr int kTileKeys = 128;         // keys per K/V tile
+
+// One request of a call.  Rows are rows of the caller's q/k/v/out tensors.
+struct ReqMeta {
+  long long row_off;   // first row of the request (suffix rows for attend, all rows for attend_full)
+  int n;               // number of rows = number of queries = number of own keys
+  int m;               // cached prefix length (0: none)
+  int page_off;        // index of the prefix's first page id inside the schedule's page list
+  int tok_off;         // sum of n over the earlier requests of the call (row index into partials)
+};
+
+// 128 packed query rows of one request and one KV head, over a range of its keys.  Packed row p of
+// a request enumerates (token a, query head j within the KV head's group of G = Hq / Hkv):
+// p = a * G + j.  Keys are numbered 0..m-1 (cached prefix) then m..m+n-1 (own rows).
+struct WorkItem {
+  int req;
+  int kv_head;
+  int row0;            // first packed row of the item
+  int split;           // index of the key split this item covers (0 when the keys are not split)
+};
+
+// Device view of a schedule: everything a kernel needs besides the tensors.
+struct ScheduleView {
+  const ReqMeta* reqs;
+  const int* pages;          // concatenated page lists
+  const WorkItem* items;
+  int num_items;
+  int num_splits;            // > 1: every item covers keys [split * split_keys, (split+1) * split_keys)
+  int split_keys;            // multiple of kTileKeys
+};
+
+// Bytes from the start of a (page, kv head) slice to the 16-byte chunk `c16` of token slot `slot`.
+// For bf16 with D = 128 a page is stored as the shared-memory image the tensor-core descriptors
+// read: four 1 KB blocks [slots 0-7, dims 0-63 | slots 0-7, dims 64-127 | slots 8-15, dims 0-63 |
+// slots 8-15, dims 64-127], each 8 rows of 128 bytes with the 16-byte chunks of row r XOR-permuted
+// by r (the 128-byte swizzle).  Every other dtype/D keeps plain [slot][dim] order.
+__host__ __device__ inline unsigned page_chunk_offset(bool swizzled, int slot, int c16, int row_bytes) {
+  if (swizzled) {
+    const int g = slot >> 3, r = slot & 7, h = c16 >> 3, c = c16 & 7;
+    return (unsigned)(g * 2048 + h * 1024 + r * 128 + ((c ^ r) << 4));
+  }
+  return (unsigned)(slot * row_bytes + c16 * 16);
+}
+
+struct PoolView {
+  const char* k;
+  const char* v;
+  long long layer_bytes;     // num_pages * Hkv * page_bytes
+  int page_bytes;            // kPageSize * D * elem size (bytes of one (page, head) slice)
+  int num_kv_heads;
+  int swizzled;
+};
+
+__host__ __device__ inline long long pool_slice_offset(const PoolView& p, int layer, int page, int hk) {
+  return (long long)layer * p.layer_bytes + ((long long)page * p.num_kv_heads + hk) * p.page_bytes;
+}
+
+// Sticky device status word codes (first error wins).
+constexpr int kDevOk = 0;
+constexpr int kDevTimeout = 5;
+
+}  // namespace bicache

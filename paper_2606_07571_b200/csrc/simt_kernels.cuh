@@ -1,0 +1,271 @@
+// Plain CUDA-core kernels: the page scatter of put_prefix, a straightforward fp32-accumulating
+// attention (one warp per query row, online softmax with warp-shuffle reductions) that serves
+// fp32 inputs and head dims the tensor-core path does not cover, and the log-sum-exp merge of
+// partial results over disjoint key ranges.
+#pragma once
+#include <cuda_bf16.h>
+#include "common.cuh"
+
+namespace bicache {
+
+struct TensorArgs {
+  const char* q;
+  const char* k;
+  const char* v;
+  char* out;
+  float* lse;            // [rows][Hq] or nullptr
+  long long q_stride;    // elements between rows
+  long long kv_stride;
+  long long out_stride;
+  int Hq, Hkv, D;
+  int layer;
+  float scale;
+  float* part_o;         // [splits][tokens][Hq][D] fp32, used when the keys are split
+  float* part_lse;       // [splits][tokens][Hq]
+  int total_tokens;      // sum of n over the call's requests
+};
+
+template <typename T> struct ElemTraits;
+template <> struct ElemTraits<float> {
+  static constexpr int kPerChunk = 4;
+  static __device__ __forceinline__ void unpack(const uint4& c, float* f) {
+    f[0] = __uint_as_float(c.x); f[1] = __uint_as_float(c.y);
+    f[2] = __uint_as_float(c.z); f[3] = __uint_as_float(c.w);
+  }
+  static __device__ __forceinline__ float load(const char* p) { return *reinterpret_cast<const float*>(p); }
+  static __device__ __forceinline__ void store(char* p, float x) { *reinterpret_cast<float*>(p) = x; }
+};
+template <> struct ElemTraits<__nv_bfloat16> {
+  static constexpr int kPerChunk = 8;
+  static __device__ __forceinline__ void unpack(const uint4& c, float* f) {
+    const unsigned w[4] = {c.x, c.y, c.z, c.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      f[2 * i] = __uint_as_float(w[i] << 16);
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  static __device__ __forceinline__ float load(const char* p) {
+    return __bfloat162float(*reinterpret_cast<const __nv_bfloat16*>(p));
+  }
+  static __device__ __forceinline__ void store(char* p, float x) {
+    *reinterpret_cast<__nv_bfloat16*>(p) = __float2bfloat16_rn(x);
+  }
+};
+
+// ---------------------------------------------------------------------------------------------
+// put_prefix: scatter [L][m][Hkv][D] rows into pool pages (both K and V), zero-filling the unused
+// slots of the last page so that a tile which covers them multiplies weight 0 by a finite value.
+// One thread moves one 16-byte chunk.
+// ---------------------------------------------------------------------------------------------
+__global__ void scatter_prefix_kernel(const char* __restrict__ src_k, const char* __restrict__ src_v,
+                                      char* __restrict__ pool_k, char* __restrict__ pool_v,
+                                      const int* __restrict__ pages, int num_prefix_pages, int m,
+                                      int num_layers, int num_kv_heads, int chunks_per_row,
+                                      long long layer_stride_bytes, long long pool_layer_bytes,
+                                      int page_bytes, int swizzled) {
+  const long long per_layer = (long long)num_prefix_pages * kPageSize * num_kv_heads * chunks_per_row;
+  const long long total = per_layer * num_layers;
+  const int row_bytes = chunks_per_row * 16;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const int layer = (int)(idx / per_layer);
+    long long rem = idx - (long long)layer * per_layer;
+    const int c16 = (int)(rem % chunks_per_row); rem /= chunks_per_row;
+    const int hk = (int)(rem % num_kv_heads); rem /= num_kv_heads;
+    const int t = (int)rem;                        // token index, may be >= m inside the last page
+    const int page = pages[t / kPageSize];
+    const int slot = t % kPageSize;
+    uint4 ck = make_uint4(0, 0, 0, 0), cv = ck;
+    if (t < m) {
+      const long long so = (long long)layer * layer_stride_bytes +
+                           ((long long)t * num_kv_heads + hk) * row_bytes + c16 * 16;
+      ck = *reinterpret_cast<const uint4*>(src_k + so);
+      cv = *reinterpret_cast<const uint4*>(src_v + so);
+    }
+    const long long po = (long long)layer * pool_layer_bytes +
+                         ((long long)page * num_kv_heads + hk) * page_bytes +
+                         page_chunk_offset(swizzled != 0, slot, c16, row_bytes);
+    *reinterpret_cast<uint4*>(pool_k + po) = ck;
+    *reinterpret_cast<uint4*>(pool_v + po) = cv;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// SIMT attention.  One block = one work item (128 packed rows of one request and KV head); each
+// warp takes packed rows warp, warp + nwarps, ...  Keys are visited 32 at a time: lane j scores
+// key j, the chunk maximum and sum are reduced with shuffles, and P.V is accumulated with each lane
+// owning dims lane, lane + 32, ...
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float warp_max(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+  return x;
+}
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+
+constexpr int kSimtWarps = 4;
+constexpr int kSimtMaxD = 256;
+
+template <typename T>
+__global__ void __launch_bounds__(kSimtWarps * 32)
+simt_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t) {
+  using Tr = ElemTraits<T>;
+  constexpr int kEsize = (int)sizeof(T);
+  __shared__ float qs[kSimtWarps][kSimtMaxD];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const WorkItem item = s.items[blockIdx.x];
+  const ReqMeta req = s.reqs[item.req];
+  const int G = t.Hq / t.Hkv;
+  const int D = t.D;
+  const int row_bytes = D * kEsize;
+  const int chunks = row_bytes / 16;
+  const int dims_per_lane = D / 32;
+  const int total_keys = req.m + req.n;
+  int key_begin = 0, key_end = total_keys;
+  if (s.num_splits > 1) {
+    key_begin = min(total_keys, item.split * s.split_keys);
+    key_end = min(total_keys, key_begin + s.split_keys);
+  }
+  const int* pages = s.pages + req.page_off;
+  const int row_end = min(item.row0 + kTileRows, req.n * G);
+
+  for (int p = item.row0 + warp; p < row_end; p += kSimtWarps) {
+    const int a = p / G;
+    const int h = item.kv_head * G + (p - a * G);
+    const char* qrow = t.q + ((req.row_off + a) * t.q_stride + (long long)h * D) * kEsize;
+    __syncwarp();
+    for (int d = lane; d < D; d += 32) qs[warp][d] = Tr::load(qrow + d * kEsize);
+    __syncwarp();
+
+    float m_run = -INFINITY, l_run = 0.f;
+    float acc[kSimtMaxD / 32];
+#pragma unroll
+    for (int i = 0; i < kSimtMaxD / 32; ++i) acc[i] = 0.f;
+
+    for (int key0 = key_begin; key0 < key_end; key0 += 32) {
+      const int j = key0 + lane;
+      const bool valid = j < key_end;
+      float sc = -INFINITY;
+      if (valid) {
+        const char* base;
+        int slot = 0;
+        bool paged = j < req.m;
+        if (paged) {
+          base = pool.k + pool_slice_offset(pool, t.layer, pages[j / kPageSize], item.kv_head);
+          slot = j % kPageSize;
+        } else {
+          base = t.k + ((req.row_off + (j - req.m)) * t.kv_stride + (long long)item.kv_head * D) * kEsize;
+        }
+        float dot = 0.f;
+        for (int c = 0; c < chunks; ++c) {
+          const char* cp = paged ? base + page_chunk_offset(pool.swizzled != 0, slot, c, row_bytes)
+                                 : base + c * 16;
+          const uint4 raw = *reinterpret_cast<const uint4*>(cp);
+          float f[Tr::kPerChunk];
+          Tr::unpack(raw, f);
+#pragma unroll
+          for (int e = 0; e < Tr::kPerChunk; ++e) dot = fmaf(f[e], qs[warp][c * Tr::kPerChunk + e], dot);
+        }
+        sc = t.scale * dot;
+      }
+      const float m_new = fmaxf(m_run, warp_max(sc));
+      const float pj = valid ? expf(sc - m_new) : 0.f;
+      const float alpha = expf(m_run - m_new);          // exp(-inf) = 0 on the first chunk
+      l_run = l_run * alpha + warp_sum(pj);
+#pragma unroll
+      for (int i = 0; i < kSimtMaxD / 32; ++i) acc[i] *= alpha;
+      m_run = m_new;
+      const int cnt = min(32, key_end - key0);
+      for (int jj = 0; jj < cnt; ++jj) {
+        const float w = __shfl_sync(0xffffffffu, pj, jj);
+        const int key = key0 + jj;
+        const char* base;
+        int slot = 0;
+        const bool paged = key < req.m;
+        if (paged) {
+          base = pool.v + pool_slice_offset(pool, t.layer, pages[key / kPageSize], item.kv_head);
+          slot = key % kPageSize;
+        } else {
+          base = t.v + ((req.row_off + (key - req.m)) * t.kv_stride + (long long)item.kv_head * D) * kEsize;
+        }
+#pragma unroll
+        for (int i = 0; i < kSimtMaxD / 32; ++i) {
+          if (i < dims_per_lane) {
+            const int d = lane + 32 * i;
+            const int c = d / Tr::kPerChunk, e = d % Tr::kPerChunk;
+            const char* ep = paged ? base + page_chunk_offset(pool.swizzled != 0, slot, c, row_bytes) + e * kEsize
+                                   : base + d * kEsize;
+            acc[i] = fmaf(w, Tr::load(ep), acc[i]);
+          }
+        }
+      }
+    }
+
+    const bool any = key_end > key_begin;
+    const float inv = any ? 1.f / l_run : 0.f;
+    const float lse = any ? m_run + logf(l_run) : -INFINITY;
+    if (s.num_splits > 1) {
+      const long long pr = ((long long)item.split * t.total_tokens + req.tok_off + a) * t.Hq + h;
+#pragma unroll
+      for (int i = 0; i < kSimtMaxD / 32; ++i)
+        if (i < dims_per_lane) t.part_o[pr * D + lane + 32 * i] = acc[i] * inv;
+      if (lane == 0) t.part_lse[pr] = lse;
+    } else {
+      char* orow = t.out + ((req.row_off + a) * t.out_stride + (long long)h * D) * kEsize;
+#pragma unroll
+      for (int i = 0; i < kSimtMaxD / 32; ++i)
+        if (i < dims_per_lane) Tr::store(orow + (lane + 32 * i) * kEsize, acc[i] * inv);
+      if (lane == 0 && t.lse != nullptr) t.lse[(req.row_off + a) * t.Hq + h] = lse;
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Log-sum-exp merge of the partial results of `num_splits` disjoint key ranges:
+//   lse = log sum_s exp(lse_s),  o = sum_s exp(lse_s - lse) o_s.
+// An empty part carries lse = -inf and weighs 0.  One block per split-0 work item, one warp per
+// packed row.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kSimtWarps * 32)
+merge_partials_kernel(ScheduleView s, TensorArgs t) {
+  using Tr = ElemTraits<T>;
+  constexpr int kEsize = (int)sizeof(T);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const WorkItem item = s.items[blockIdx.x];       // the first num_items / num_splits items are split 0
+  const ReqMeta req = s.reqs[item.req];
+  const int G = t.Hq / t.Hkv;
+  const int D = t.D;
+  const int row_end = min(item.row0 + kTileRows, req.n * G);
+  for (int p = item.row0 + warp; p < row_end; p += kSimtWarps) {
+    const int a = p / G;
+    const int h = item.kv_head * G + (p - a * G);
+    const long long pr0 = ((long long)req.tok_off + a) * t.Hq + h;
+    const long long split_stride = (long long)t.total_tokens * t.Hq;
+    float mx = -INFINITY;
+    for (int sp = 0; sp < s.num_splits; ++sp) mx = fmaxf(mx, t.part_lse[pr0 + sp * split_stride]);
+    float tot = 0.f;
+    for (int sp = 0; sp < s.num_splits; ++sp) tot += expf(t.part_lse[pr0 + sp * split_stride] - mx);
+    const bool any = mx > -INFINITY;
+    char* orow = t.out + ((req.row_off + a) * t.out_stride + (long long)h * D) * kEsize;
+    for (int d = lane; d < D; d += 32) {
+      float o = 0.f;
+      if (any) {
+        for (int sp = 0; sp < s.num_splits; ++sp) {
+          const float w = expf(t.part_lse[pr0 + sp * split_stride] - mx) / tot;
+          o = fmaf(w, t.part_o[(pr0 + sp * split_stride) * D + d], o);
+        }
+      }
+      Tr::store(orow + d * kEsize, o);
+    }
+    if (lane == 0 && t.lse != nullptr)
+      t.lse[(req.row_off + a) * t.Hq + h] = any ? mx + logf(tot) : -INFINITY;
+  }
+}
+
+}  // namespace bicache

@@ -1,0 +1,156 @@
+"""CPU tests of the C-ABI library: it builds, loads, exports every declared symbol, and its host
+logic (store bookkeeping, FIFO eviction, depth rule) matches the oracle bit-exactly through a
+host-only context.  No compute call is made here."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+from hypothesis import given, settings, strategies as st
+
+import oracle
+import __graft_entry__ as entry
+from paper_2606_07571_b200 import binding, workloads
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    entry.build()
+    return binding.load_library()
+
+
+def test_every_declared_symbol_is_exported(lib):
+    hdr = open(os.path.join(ROOT, "include", "bicache.h")).read()
+    declared = set(re.findall(r"\b(bicache_[a-z_]+)\s*\(", hdr))
+    assert declared == set(binding.EXPORTED)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def host_ctx(lib, L=2, Hq=4, Hkv=2, D=128, pages=8, dtype=binding.BF16, order=None):
+    cfg = binding.Config(L, Hq, Hkv, D, 16, pages, dtype, -1)
+    keep = None
+    if order is not None:
+        keep = np.ascontiguousarray(order, dtype=np.int32)
+        cfg.initial_free_order = keep.ctypes.data_as(C.POINTER(C.c_int32))
+    ctx = C.c_void_p()
+    assert lib.bicache_create(C.byref(cfg), C.byref(ctx)) == binding.OK
+    return ctx
+
+
+def put(lib, ctx, key, m, cap=None):
+    pid, hit = C.c_int32(-1), C.c_int32(-1)
+    cap = (m + 15) // 16 if cap is None else cap
+    pages = np.full(max(cap, 1), -1, dtype=np.int32)
+    st_ = lib.bicache_put_prefix(ctx, C.c_uint64(key), m, None, None, m * 2 * 128, None, C.byref(pid), C.byref(hit),
+                                 pages.ctypes.data_as(C.POINTER(C.c_int32)), cap)
+    return st_, pid.value, hit.value, pages[:cap].tolist()
+
+
+def test_sizes_and_create_errors(lib):
+    cfg = binding.Config(32, 32, 32, 128, 16, 128, binding.BF16, -1)
+    assert lib.bicache_pool_bytes(C.byref(cfg)) == 32 * 128 * 32 * 16 * 128 * 2
+    assert lib.bicache_workspace_bytes(C.byref(cfg), 4096, 16) > 0
+    ctx = C.c_void_p()
+    bad = binding.Config(32, 32, 5, 128, 16, 128, binding.BF16, -1)        # Hq % Hkv != 0
+    assert lib.bicache_create(C.byref(bad), C.byref(ctx)) == binding.ERR_INVALID
+    bad = binding.Config(32, 32, 32, 128, 32, 128, binding.BF16, -1)       # page size
+    assert lib.bicache_create(C.byref(bad), C.byref(ctx)) == binding.ERR_UNSUPPORTED
+    bad = binding.Config(32, 32, 32, 128, 16, 128, 7, -1)                  # dtype
+    assert lib.bicache_create(C.byref(bad), C.byref(ctx)) == binding.ERR_UNSUPPORTED
+    order = np.array([0, 1, 1, 2], dtype=np.int32)
+    bad = binding.Config(1, 1, 1, 128, 16, 4, binding.BF16, -1)
+    bad.initial_free_order = order.ctypes.data_as(C.POINTER(C.c_int32))
+    assert lib.bicache_create(C.byref(bad), C.byref(ctx)) == binding.ERR_INVALID
+    dev = binding.Config(1, 1, 1, 128, 16, 4, binding.BF16, 0)             # device context needs buffers
+    assert lib.bicache_create(C.byref(dev), C.byref(ctx)) == binding.ERR_INVALID
+
+
+def test_depth_rule_matches_oracle(lib):
+    ctx = host_ctx(lib, L=32, Hq=32, Hkv=32, pages=4)
+    m = np.array([2048, 85, 1, 5, 0, 1024, 512], dtype=np.int32)
+    n = np.array([362, 15, 1000, 0, 9, 256, 1024], dtype=np.int32)
+    out = np.zeros(7, dtype=np.int32)
+    p = lambda a: a.ctypes.data_as(C.POINTER(C.c_int32))
+    assert lib.bicache_reuse_depth(ctx, 7, p(m), p(n), p(out)) == binding.ERR_INVALID     # no table yet
+    t = workloads.standin_depth_table(32)
+    assert lib.bicache_set_depth_table(ctx, p(t), 100) == binding.ERR_INVALID
+    assert lib.bicache_set_depth_table(ctx, p(t), 101) == binding.OK
+    assert lib.bicache_reuse_depth(ctx, 7, p(m), p(n), p(out)) == binding.OK
+    assert out.tolist() == oracle.reuse_depth(m, n, t, 32).tolist()
+    ident = np.arange(101, dtype=np.int32)
+    lib.bicache_set_depth_table(ctx, p(ident), 101)
+    lib.bicache_reuse_depth(ctx, 7, p(m), p(n), p(out))
+    assert out.tolist() == [32, 32, 0, 32, 0, 32, 32] and oracle.reuse_depth(m, n, ident, 32).tolist() == out.tolist()
+    n[2] = -1
+    assert lib.bicache_reuse_depth(ctx, 7, p(m), p(n), p(out)) == binding.ERR_INVALID
+    rng = np.random.default_rng(0)
+    m = rng.integers(0, 20000, 4000).astype(np.int32)
+    n = rng.integers(0, 20000, 4000).astype(np.int32)
+    out = np.zeros(4000, dtype=np.int32)
+    lib.bicache_set_depth_table(ctx, p(t), 101)
+    assert lib.bicache_reuse_depth(ctx, 4000, p(m), p(n), p(out)) == binding.OK
+    assert (out == oracle.reuse_depth(m, n, t, 32)).all()
+    lib.bicache_destroy(ctx)
+
+
+def test_store_fifo_sequence_matches_oracle(lib):
+    ctx = host_ctx(lib, L=1, Hq=2, Hkv=2, pages=4)
+    assert put(lib, ctx, 10, 32) == (binding.OK, 0, 0, [0, 1])
+    assert put(lib, ctx, 11, 16) == (binding.OK, 1, 0, [2])
+    assert put(lib, ctx, 10, 32) == (binding.OK, 0, 1, [0, 1])                  # hit, age not refreshed
+    assert put(lib, ctx, 10, 31)[0] == binding.ERR_INVALID                     # same key, other length
+    assert put(lib, ctx, 12, 32) == (binding.OK, 2, 0, [3, 0])                  # evicts key 10 (oldest)
+    pid, m = C.c_int32(), C.c_int32()
+    assert lib.bicache_lookup_prefix(ctx, C.c_uint64(10), C.byref(pid), C.byref(m)) == binding.ERR_NOTFOUND
+    assert lib.bicache_lookup_prefix(ctx, C.c_uint64(12), C.byref(pid), C.byref(m)) == binding.OK
+    assert (pid.value, m.value) == (2, 32)
+    n = C.c_int32()
+    assert lib.bicache_prefix_pages(ctx, 0, None, 0, C.byref(n)) == binding.ERR_NOTFOUND
+    assert put(lib, ctx, 10, 16) == (binding.OK, 3, 0, [1])                     # new id after eviction
+    assert put(lib, ctx, 13, 16 * 5)[0] == binding.ERR_NOMEM
+    assert put(lib, ctx, 14, 0)[0] == binding.ERR_INVALID
+    assert put(lib, ctx, 15, 32, cap=1)[0] == binding.ERR_INVALID               # pages_out too small, nothing changes
+    assert lib.bicache_lookup_prefix(ctx, C.c_uint64(11), C.byref(pid), C.byref(m)) == binding.OK
+    # attention on a host-only context is refused, not emulated
+    z = np.zeros(1, dtype=np.int64)
+    assert lib.bicache_attend_full(ctx, 0, 1, z.ctypes.data_as(C.POINTER(C.c_int64)),
+                                   np.ones(1, np.int32).ctypes.data_as(C.POINTER(C.c_int32)),
+                                   None, None, None, 256, 256, None, 256, None, C.c_float(1.0), None) \
+        == binding.ERR_UNSUPPORTED
+    lib.bicache_destroy(ctx)
+
+
+@given(st.lists(st.tuples(st.integers(0, 6), st.integers(1, 130)), min_size=1, max_size=40),
+       st.integers(1, 12), st.integers(0, 3))
+@settings(max_examples=100, deadline=None)
+def test_store_traces_match_oracle_bit_exactly(trace, num_pages, seed):
+    entry.build()
+    lib = binding.load_library()
+    order = None if seed == 0 else workloads.shuffled_page_order(num_pages, seed)
+    ctx = host_ctx(lib, L=1, Hq=1, Hkv=1, pages=num_pages, order=order)
+    ref = oracle.PagedPrefixStore(1, 1, 2, 16, num_pages, free_order=order)
+    for key, m in trace:
+        kv = np.zeros((1, m, 1, 2))
+        try:
+            want = (binding.OK,) + tuple(ref.put(key, kv, kv))
+        except oracle.InvalidArgument:
+            want = (binding.ERR_INVALID,)
+        except oracle.OutOfPages:
+            want = (binding.ERR_NOMEM,)
+        got = put(lib, ctx, key, m)
+        if want[0] == binding.OK:
+            assert got == (binding.OK, want[1], int(want[2]), want[3])
+        else:
+            assert got[0] == want[0]
+        for k in range(7):
+            pid, mm = C.c_int32(), C.c_int32()
+            stt = lib.bicache_lookup_prefix(ctx, C.c_uint64(k), C.byref(pid), C.byref(mm))
+            try:
+                assert (stt, pid.value, mm.value) == (binding.OK,) + tuple(ref.lookup(k))
+            except oracle.NotFound:
+                assert stt == binding.ERR_NOTFOUND
+    lib.bicache_destroy(ctx)
