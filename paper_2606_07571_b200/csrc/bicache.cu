@@ -46,7 +46,7 @@ struct CachedSchedule {
   std::vector<int32_t> prefix_id;
   std::vector<int64_t> row_off;
   std::vector<int32_t> seqlen;
-  int num_items = 0, num_splits = 1, split_keys = 0, total_tokens = 0;
+  int num_items = 0, num_splits = 1, tiles_per_split = 0, total_tokens = 0;
   size_t reqs_off = 0, pages_off = 0, items_off = 0;   // byte offsets inside the slot
 };
 
@@ -146,7 +146,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   std::vector<ReqMeta> reqs(R);
   std::vector<int> pages;
   long long tok = 0;
-  int max_keys = 0;
+  int max_key_tiles = 0;
   long long unsplit_items = 0;
   int last_pid = -1, last_page_off = 0;
   for (int i = 0; i < R; ++i) {
@@ -168,19 +168,18 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
       r.page_off = last_page_off;
     }
     if (r.n > 0) {
-      max_keys = std::max(max_keys, r.m + r.n);
+      max_key_tiles = std::max(max_key_tiles, (r.m + kTileKeys - 1) / kTileKeys + (r.n + kTileKeys - 1) / kTileKeys);
       unsplit_items += (long long)((r.n * (long long)G + kTileRows - 1) / kTileRows) * Hkv;
     }
   }
   // Split the keys across CTAs when the batch has too few row tiles to fill the GPU.
-  int num_splits = 1, split_keys = 0;
-  if (unsplit_items > 0 && unsplit_items * 2 <= ctx->sm_count && max_keys >= 8 * kTileKeys) {
-    const int key_tiles = (max_keys + kTileKeys - 1) / kTileKeys;
+  int num_splits = 1, tiles_per_split = 0;
+  if (unsplit_items > 0 && unsplit_items * 2 <= ctx->sm_count && max_key_tiles >= 8) {
+    const int key_tiles = max_key_tiles;
     int want = (int)std::min<long long>((kTargetCtas + unsplit_items - 1) / unsplit_items, key_tiles / 2);
     while (want > 1 && tok * ctx->cfg.num_q_heads * want > ctx->part_capacity_rowheads) --want;
     if (want > 1) {
-      const int tiles_per_split = (key_tiles + want - 1) / want;
-      split_keys = tiles_per_split * kTileKeys;
+      tiles_per_split = (key_tiles + want - 1) / want;
       num_splits = (key_tiles + tiles_per_split - 1) / tiles_per_split;
     }
   }
@@ -235,7 +234,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   c.seqlen.assign(seqlen, seqlen + R);
   c.num_items = (int)items.size();
   c.num_splits = num_splits;
-  c.split_keys = split_keys;
+  c.tiles_per_split = tiles_per_split;
   c.total_tokens = (int)tok;
   c.reqs_off = reqs_off;
   c.pages_off = pages_off;
@@ -307,7 +306,7 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   sv.items = reinterpret_cast<const WorkItem*>(base + c.items_off);
   sv.num_items = c.num_items;
   sv.num_splits = c.num_splits;
-  sv.split_keys = c.split_keys;
+  sv.tiles_per_split = c.tiles_per_split;
 
   TensorArgs t;
   t.q = static_cast<const char*>(q);

@@ -35,8 +35,8 @@ struct ScheduleView {
   const int* pages;          // concatenated page lists
   const WorkItem* items;
   int num_items;
-  int num_splits;            // > 1: every item covers keys [split * split_keys, (split+1) * split_keys)
-  int split_keys;            // multiple of kTileKeys
+  int num_splits;            // > 1: item covers key tiles [split * tiles_per_split, (split + 1) * tiles_per_split)
+  int tiles_per_split;       // key tiles: ceil(m/128) prefix tiles followed by ceil(n/128) own tiles
 };
 
 // Bytes from the start of a (page, kv head) slice to the 16-byte chunk `c16` of token slot `slot`.

@@ -125,12 +125,18 @@ simt_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t) {
   const int row_bytes = D * kEsize;
   const int chunks = row_bytes / 16;
   const int dims_per_lane = D / 32;
-  const int total_keys = req.m + req.n;
-  int key_begin = 0, key_end = total_keys;
+  // Key tiles: ceil(m/128) tiles of cached prefix keys, then ceil(n/128) tiles of own keys; a key
+  // split covers a contiguous range of tiles.
+  const int prefix_tiles = (req.m + kTileKeys - 1) / kTileKeys;
+  const int all_tiles = prefix_tiles + (req.n + kTileKeys - 1) / kTileKeys;
+  int tile_begin = 0, tile_end = all_tiles;
   if (s.num_splits > 1) {
-    key_begin = min(total_keys, item.split * s.split_keys);
-    key_end = min(total_keys, key_begin + s.split_keys);
+    tile_begin = min(all_tiles, item.split * s.tiles_per_split);
+    tile_end = min(all_tiles, tile_begin + s.tiles_per_split);
   }
+  const int pre_begin = min(req.m, tile_begin * kTileKeys), pre_end = min(req.m, tile_end * kTileKeys);
+  const int own_begin = min(req.n, max(0, tile_begin - prefix_tiles) * kTileKeys);
+  const int own_end = min(req.n, max(0, tile_end - prefix_tiles) * kTileKeys);
   const int* pages = s.pages + req.page_off;
   const int row_end = min(item.row0 + kTileRows, req.n * G);
 
@@ -147,66 +153,69 @@ simt_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t) {
 #pragma unroll
     for (int i = 0; i < kSimtMaxD / 32; ++i) acc[i] = 0.f;
 
-    for (int key0 = key_begin; key0 < key_end; key0 += 32) {
-      const int j = key0 + lane;
-      const bool valid = j < key_end;
-      float sc = -INFINITY;
-      if (valid) {
-        const char* base;
-        int slot = 0;
-        bool paged = j < req.m;
-        if (paged) {
-          base = pool.k + pool_slice_offset(pool, t.layer, pages[j / kPageSize], item.kv_head);
-          slot = j % kPageSize;
-        } else {
-          base = t.k + ((req.row_off + (j - req.m)) * t.kv_stride + (long long)item.kv_head * D) * kEsize;
-        }
-        float dot = 0.f;
-        for (int c = 0; c < chunks; ++c) {
-          const char* cp = paged ? base + page_chunk_offset(pool.swizzled != 0, slot, c, row_bytes)
-                                 : base + c * 16;
-          const uint4 raw = *reinterpret_cast<const uint4*>(cp);
-          float f[Tr::kPerChunk];
-          Tr::unpack(raw, f);
+    for (int part = 0; part < 2; ++part) {
+      const bool paged = part == 0;
+      const int key_begin = paged ? pre_begin : own_begin;
+      const int key_end = paged ? pre_end : own_end;
+      for (int key0 = key_begin; key0 < key_end; key0 += 32) {
+        const int j = key0 + lane;
+        const bool valid = j < key_end;
+        float sc = -INFINITY;
+        if (valid) {
+          const char* base;
+          int slot = 0;
+          if (paged) {
+            base = pool.k + pool_slice_offset(pool, t.layer, pages[j / kPageSize], item.kv_head);
+            slot = j % kPageSize;
+          } else {
+            base = t.k + ((req.row_off + j) * t.kv_stride + (long long)item.kv_head * D) * kEsize;
+          }
+          float dot = 0.f;
+          for (int c = 0; c < chunks; ++c) {
+            const char* cp = paged ? base + page_chunk_offset(pool.swizzled != 0, slot, c, row_bytes)
+                                   : base + c * 16;
+            const uint4 raw = *reinterpret_cast<const uint4*>(cp);
+            float f[Tr::kPerChunk];
+            Tr::unpack(raw, f);
 #pragma unroll
-          for (int e = 0; e < Tr::kPerChunk; ++e) dot = fmaf(f[e], qs[warp][c * Tr::kPerChunk + e], dot);
+            for (int e = 0; e < Tr::kPerChunk; ++e) dot = fmaf(f[e], qs[warp][c * Tr::kPerChunk + e], dot);
+          }
+          sc = t.scale * dot;
         }
-        sc = t.scale * dot;
-      }
-      const float m_new = fmaxf(m_run, warp_max(sc));
-      const float pj = valid ? expf(sc - m_new) : 0.f;
-      const float alpha = expf(m_run - m_new);          // exp(-inf) = 0 on the first chunk
-      l_run = l_run * alpha + warp_sum(pj);
+        const float m_new = fmaxf(m_run, warp_max(sc));
+        const float pj = valid ? expf(sc - m_new) : 0.f;
+        const float alpha = expf(m_run - m_new);          // exp(-inf) = 0 on the first chunk
+        l_run = l_run * alpha + warp_sum(pj);
 #pragma unroll
-      for (int i = 0; i < kSimtMaxD / 32; ++i) acc[i] *= alpha;
-      m_run = m_new;
-      const int cnt = min(32, key_end - key0);
-      for (int jj = 0; jj < cnt; ++jj) {
-        const float w = __shfl_sync(0xffffffffu, pj, jj);
-        const int key = key0 + jj;
-        const char* base;
-        int slot = 0;
-        const bool paged = key < req.m;
-        if (paged) {
-          base = pool.v + pool_slice_offset(pool, t.layer, pages[key / kPageSize], item.kv_head);
-          slot = key % kPageSize;
-        } else {
-          base = t.v + ((req.row_off + (key - req.m)) * t.kv_stride + (long long)item.kv_head * D) * kEsize;
-        }
+        for (int i = 0; i < kSimtMaxD / 32; ++i) acc[i] *= alpha;
+        m_run = m_new;
+        const int cnt = min(32, key_end - key0);
+        for (int jj = 0; jj < cnt; ++jj) {
+          const float w = __shfl_sync(0xffffffffu, pj, jj);
+          const int key = key0 + jj;
+          const char* base;
+          int slot = 0;
+          if (paged) {
+            base = pool.v + pool_slice_offset(pool, t.layer, pages[key / kPageSize], item.kv_head);
+            slot = key % kPageSize;
+          } else {
+            base = t.v + ((req.row_off + key) * t.kv_stride + (long long)item.kv_head * D) * kEsize;
+          }
 #pragma unroll
-        for (int i = 0; i < kSimtMaxD / 32; ++i) {
-          if (i < dims_per_lane) {
-            const int d = lane + 32 * i;
-            const int c = d / Tr::kPerChunk, e = d % Tr::kPerChunk;
-            const char* ep = paged ? base + page_chunk_offset(pool.swizzled != 0, slot, c, row_bytes) + e * kEsize
-                                   : base + d * kEsize;
-            acc[i] = fmaf(w, Tr::load(ep), acc[i]);
+          for (int i = 0; i < kSimtMaxD / 32; ++i) {
+            if (i < dims_per_lane) {
+              const int d = lane + 32 * i;
+              const int c = d / Tr::kPerChunk, e = d % Tr::kPerChunk;
+              const char* ep = paged ? base + page_chunk_offset(pool.swizzled != 0, slot, c, row_bytes) + e * kEsize
+                                     : base + d * kEsize;
+              acc[i] = fmaf(w, Tr::load(ep), acc[i]);
+            }
           }
         }
       }
     }
 
-    const bool any = key_end > key_begin;
+    const bool any = pre_end > pre_begin || own_end > own_begin;
     const float inv = any ? 1.f / l_run : 0.f;
     const float lse = any ? m_run + logf(l_run) : -INFINITY;
     if (s.num_splits > 1) {
