@@ -174,6 +174,22 @@ int32_t bicache_attend_full(bicache_ctx* ctx, int32_t layer, int32_t R,
                             void* out, int64_t out_row_stride, float* lse_out,
                             float softmax_scale, void* stream);
 
+/* Layer-partitioned dispatch of one layer (Sec. 5.2: "for each layer l, determine whether l <= b"):
+ * request i, whose whole input (prefix rows, then suffix rows) occupies seqlen[i] = N_i rows from
+ * row_off[i], goes through bicache_attend on its suffix rows (row_off[i] + m_i, N_i - m_i rows, m_i =
+ * length of prefix_id[i]) if layer < depth[i] and prefix_id[i] >= 0, and through bicache_attend_full
+ * on all its rows otherwise.  depth, prefix_id, row_off, seqlen: host arrays of length R; the reusing
+ * requests' prefix ids must be grouped.  Tensor arguments as for bicache_attend.  Outputs: suffix rows
+ * of reusing requests, all rows of the others.  INVALID if a reusing request is shorter than its
+ * prefix; other errors as for the two calls.  The reuse half is validated and enqueued first; if
+ * the second half then fails validation the first has already been enqueued. */
+int32_t bicache_attend_layer(bicache_ctx* ctx, int32_t layer, int32_t R, const int32_t* depth,
+                             const int32_t* prefix_id, const int64_t* row_off, const int32_t* seqlen,
+                             const void* q, const void* k, const void* v,
+                             int64_t q_row_stride, int64_t kv_row_stride,
+                             void* out, int64_t out_row_stride, float* lse_out,
+                             float softmax_scale, void* stream);
+
 /* Synchronises `stream` and returns the sticky device status: OK, or TIMEOUT if a kernel gave up
  * on a bounded wait (its outputs are then undefined), or CUDA for a runtime error.  `clear` != 0
  * resets the word. */

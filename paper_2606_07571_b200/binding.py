@@ -22,6 +22,7 @@ EXPORTED = [
     "bicache_pool_bytes", "bicache_workspace_bytes", "bicache_create", "bicache_destroy",
     "bicache_set_path", "bicache_set_depth_table", "bicache_put_prefix", "bicache_lookup_prefix",
     "bicache_prefix_pages", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
+    "bicache_attend_layer",
     "bicache_device_status", "bicache_launch_count", "bicache_last_error",
 ]
 
@@ -83,6 +84,9 @@ def load_library():
     lib.bicache_attend_full.restype = C.c_int32
     lib.bicache_attend_full.argtypes = [vp, C.c_int32, C.c_int32, i64p, i32p, vp, vp, vp, C.c_int64, C.c_int64,
                                         vp, C.c_int64, vp, C.c_float, vp]
+    lib.bicache_attend_layer.restype = C.c_int32
+    lib.bicache_attend_layer.argtypes = [vp, C.c_int32, C.c_int32, i32p, i32p, i64p, i32p, vp, vp, vp, C.c_int64,
+                                         C.c_int64, vp, C.c_int64, vp, C.c_float, vp]
     lib.bicache_device_status.restype = C.c_int32
     lib.bicache_device_status.argtypes = [vp, vp, C.c_int32]
     lib.bicache_launch_count.restype = C.c_int64
@@ -233,6 +237,17 @@ class BiCache:
         st = self.lib.bicache_attend_full(self.ctx, layer, len(n), poff, pn, qp, kp, vp_, qs, ks, op, os_, lp,
                                           C.c_float(scale), self._stream())
         self._check(st, "bicache_attend_full")
+
+    def attend_layer(self, layer, depth, prefix_id, row_off, seqlen, q, k, v, out, lse=None, scale=None):
+        d, pd = _i32(depth)
+        pid, ppid = _i32(prefix_id)
+        off, poff = _i64(row_off)
+        n, pn = _i32(seqlen)
+        qp, kp, vp_, qs, ks, op, os_, lp = self._tensor_args(q, k, v, out, lse)
+        scale = self.D ** -0.5 if scale is None else scale
+        st = self.lib.bicache_attend_layer(self.ctx, layer, len(n), pd, ppid, poff, pn, qp, kp, vp_, qs, ks, op, os_,
+                                           lp, C.c_float(scale), self._stream())
+        self._check(st, "bicache_attend_layer")
 
     def device_status(self, clear=False):
         return self.lib.bicache_device_status(self.ctx, self._stream(), 1 if clear else 0)

@@ -598,6 +598,52 @@ int32_t bicache_attend_full(bicache_ctx* ctx, int32_t layer, int32_t R, const in
                        out_row_stride, lse_out, softmax_scale, stream);
 }
 
+int32_t bicache_attend_layer(bicache_ctx* ctx, int32_t layer, int32_t R, const int32_t* depth,
+                             const int32_t* prefix_id, const int64_t* row_off, const int32_t* seqlen,
+                             const void* q, const void* k, const void* v, int64_t q_row_stride,
+                             int64_t kv_row_stride, void* out, int64_t out_row_stride, float* lse_out,
+                             float softmax_scale, void* stream) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  if (R < 0 || (R > 0 && (!depth || !prefix_id || !row_off || !seqlen)))
+    return fail(ctx, BICACHE_ERR_INVALID, "null metadata array");
+  // Layer-partitioned dispatch: request i reuses the cached prefix in this layer iff layer < depth[i].
+  std::vector<int32_t> r_pid, r_len, f_len;
+  std::vector<int64_t> r_off, f_off;
+  for (int i = 0; i < R; ++i) {
+    if (seqlen[i] < 0 || row_off[i] < 0) return fail(ctx, BICACHE_ERR_INVALID, "negative length or offset");
+    if (layer < depth[i] && prefix_id[i] >= 0) {
+      auto found = ctx->by_id.find(prefix_id[i]);
+      if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+      const int32_t m = found->second->m;
+      if (seqlen[i] < m) return fail(ctx, BICACHE_ERR_INVALID, "request shorter than its prefix");
+      r_pid.push_back(prefix_id[i]);
+      r_off.push_back(row_off[i] + m);
+      r_len.push_back(seqlen[i] - m);
+    } else {
+      f_off.push_back(row_off[i]);
+      f_len.push_back(seqlen[i]);
+    }
+  }
+  // Validate both halves before launching either, so that an error leaves the outputs untouched.
+  if (!r_len.empty()) {
+    for (size_t i = 1; i < r_pid.size(); ++i)
+      if (r_pid[i] != r_pid[i - 1] &&
+          std::find(r_pid.begin(), r_pid.begin() + i, r_pid[i]) != r_pid.begin() + i)
+        return fail(ctx, BICACHE_ERR_INVALID, "requests of one prefix are not contiguous");
+    const int32_t st = run_attention(ctx, 0, layer, (int32_t)r_len.size(), r_pid.data(), r_off.data(), r_len.data(),
+                                     q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                                     softmax_scale, stream);
+    if (st != BICACHE_OK) return st;
+  }
+  if (!f_len.empty()) {
+    const int32_t st = run_attention(ctx, 1, layer, (int32_t)f_len.size(), nullptr, f_off.data(), f_len.data(),
+                                     q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                                     softmax_scale, stream);
+    if (st != BICACHE_OK) return st;
+  }
+  return BICACHE_OK;
+}
+
 int32_t bicache_device_status(bicache_ctx* ctx, void* stream, int32_t clear) {
   if (!ctx) return BICACHE_ERR_INVALID;
   if (ctx->host_only) return BICACHE_OK;
