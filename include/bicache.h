@@ -195,6 +195,36 @@ int32_t bicache_attend_layer(bicache_ctx* ctx, int32_t layer, int32_t R, const i
  * resets the word. */
 int32_t bicache_device_status(bicache_ctx* ctx, void* stream, int32_t clear);
 
+/* Allocation-free full attention of ONE request (the paper has no counterpart: this entry point
+ * exists for callers, not for the method).
+ *
+ * Some callers cannot allocate device memory where they need attention: code embedded in another
+ * framework's fixed memory plan, a serving loop that must stay clear of the allocator once it is
+ * running, a process whose GPU budget was handed out before this library was loaded.  The calls
+ * above need a context and a caller-allocated workspace; this one needs neither.  Its scratch
+ * (partial results of BICACHE_STATIC_KEY_SPLITS key ranges) is a fixed array inside the library's
+ * device image: about 8.1 MB on every GPU that loads the library, held until the process exits.
+ * The call allocates and frees nothing, on the host or on the device.
+ *
+ * Computes what bicache_attend_full computes for a single request occupying rows 0..n_rows-1:
+ * every row attends, without a mask, over all n_rows keys.  dtype: BICACHE_F32 or BICACHE_BF16;
+ * head_dim: 32, 64, 96 or 128; q, out: device [n_rows][Hq][D]; k, v: device [n_rows][Hkv][D]; row
+ * strides in elements; heads dense within a row.  Runs on the current device, on `stream`.
+ *   NOMEM        n_rows * num_q_heads > BICACHE_STATIC_MAX_ROW_HEADS (the array's capacity)
+ *   UNSUPPORTED  dtype or head_dim outside the list above
+ *   INVALID      null pointers, bad strides or head counts
+ * The first call on each device looks up the array's device address (a host-side set-up step that
+ * enqueues nothing); make that first call before starting any stream capture.  All calls on a
+ * device share the one array and every call overwrites the part it uses, so nothing has to be
+ * cleared between calls - but two calls whose kernels may overlap on the GPU (different streams,
+ * or different threads) race on it.  Issue them on one stream, or serialise them yourself. */
+#define BICACHE_STATIC_MAX_ROW_HEADS 4096
+#define BICACHE_STATIC_KEY_SPLITS 4
+int32_t bicache_attend_full_static(int32_t dtype, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
+                                   int32_t n_rows, const void* q, const void* k, const void* v,
+                                   int64_t q_row_stride, int64_t kv_row_stride,
+                                   void* out, int64_t out_row_stride, float softmax_scale, void* stream);
+
 /* Number of kernels this context has launched so far (for benchmarks' launch accounting). */
 int64_t bicache_launch_count(const bicache_ctx* ctx);
 

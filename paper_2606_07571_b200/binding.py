@@ -22,7 +22,7 @@ EXPORTED = [
     "bicache_pool_bytes", "bicache_workspace_bytes", "bicache_create", "bicache_destroy",
     "bicache_set_path", "bicache_set_depth_table", "bicache_put_prefix", "bicache_lookup_prefix",
     "bicache_prefix_pages", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
-    "bicache_attend_layer",
+    "bicache_attend_layer", "bicache_attend_full_static",
     "bicache_device_status", "bicache_launch_count", "bicache_last_error",
 ]
 
@@ -87,6 +87,9 @@ def load_library():
     lib.bicache_attend_layer.restype = C.c_int32
     lib.bicache_attend_layer.argtypes = [vp, C.c_int32, C.c_int32, i32p, i32p, i64p, i32p, vp, vp, vp, C.c_int64,
                                          C.c_int64, vp, C.c_int64, vp, C.c_float, vp]
+    lib.bicache_attend_full_static.restype = C.c_int32
+    lib.bicache_attend_full_static.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp, vp, vp,
+                                               C.c_int64, C.c_int64, vp, C.c_int64, C.c_float, vp]
     lib.bicache_device_status.restype = C.c_int32
     lib.bicache_device_status.argtypes = [vp, vp, C.c_int32]
     lib.bicache_launch_count.restype = C.c_int64
@@ -254,3 +257,21 @@ class BiCache:
 
     def launch_count(self):
         return int(self.lib.bicache_launch_count(self.ctx))
+
+
+STATIC_MAX_ROW_HEADS = 4096
+
+
+def attend_full_static(q, k, v, out, scale=None):
+    """bicache_attend_full_static: full attention of one request without a context or workspace.
+
+    For callers that may not allocate device memory: the scratch is a fixed array inside the
+    library.  q, out [n, Hq, D]; k, v [n, Hkv, D] on the current CUDA device.  Returns the status
+    code (0 = OK); n * Hq above STATIC_MAX_ROW_HEADS is refused with ERR_NOMEM."""
+    lib = load_library()
+    n, Hq, D = q.shape
+    Hkv = k.shape[1]
+    scale = D ** -0.5 if scale is None else scale
+    return lib.bicache_attend_full_static(_dtype_code(q.dtype), Hq, Hkv, D, n, q.data_ptr(), k.data_ptr(),
+                                          v.data_ptr(), q.stride(0), k.stride(0), out.data_ptr(), out.stride(0),
+                                          C.c_float(scale), C.c_void_p(torch.cuda.current_stream().cuda_stream))
