@@ -327,7 +327,8 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   t.total_tokens = c.total_tokens;
   const PoolView pool = pool_view(ctx);
 
-  const bool use_tensor = ctx->tensor_ok && ctx->path != BICACHE_PATH_SIMT;
+  // the tensor-core kernel takes the row maximum before scaling, which needs a positive scale
+  const bool use_tensor = ctx->tensor_ok && ctx->path != BICACHE_PATH_SIMT && softmax_scale > 0.f;
   cudaError_t e;
   if (use_tensor) {
     e = launch_tc_attention(sv, pool, t, ctx->d_status, stream);
@@ -656,6 +657,13 @@ int32_t bicache_device_status(bicache_ctx* ctx, void* stream, int32_t clear) {
   if (word == kDevOk) return BICACHE_OK;
   return fail(ctx, word == kDevTimeout ? BICACHE_ERR_TIMEOUT : BICACHE_ERR_CUDA, "device-side wait gave up");
 }
+
+#ifdef BICACHE_TRACE
+// Debug build only: copy the traced CTA's clock stamps to the host.
+int32_t bicache_debug_read_trace(long long* out, int32_t n) {
+  return cudaMemcpyFromSymbol(out, bicache::tc::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : 4;
+}
+#endif
 
 int64_t bicache_launch_count(const bicache_ctx* ctx) { return ctx ? ctx->launches : 0; }
 

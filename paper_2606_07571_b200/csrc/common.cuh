@@ -7,7 +7,7 @@
 namespace bicache {
 
 constexpr int kPageSize = 16;          // tokens per page
-constexpr int kTileRows = 128;         // query rows of one work item (one tensor-core M tile)
+constexpr int kTileRows = 256;         // query rows of one work item (two tensor-core M tiles of 128)
 constexpr int kTileKeys = 128;         // keys per K/V tile
 
 // One request of a call.  Rows are rows of the caller's q/k/v/out tensors.
@@ -19,7 +19,7 @@ struct ReqMeta {
   int tok_off;         // sum of n over the earlier requests of the call (row index into partials)
 };
 
-// 128 packed query rows of one request and one KV head, over a range of its keys.  Packed row p of
+// Up to 256 packed query rows of one request and one KV head, over a range of its keys.  Packed row p of
 // a request enumerates (token a, query head j within the KV head's group of G = Hq / Hkv):
 // p = a * G + j.  Keys are numbered 0..m-1 (cached prefix) then m..m+n-1 (own rows).
 struct WorkItem {

@@ -1,17 +1,20 @@
 // Tensor-core attention for bf16, head_dim 128, on sm_100a: tcgen05.mma with TMEM accumulators.
 //
-// One CTA computes one work item: 128 packed query rows (one request, one KV head) against a
-// range of key tiles of 128 keys - first the cached prefix (pages of 16 tokens, staged with
-// cp.async.bulk because a pool page already is the shared-memory image the MMA reads), then the
-// request's own rows (16-byte cp.async gathers from the caller's row-major K/V, zero-filled past
-// the end).  Per tile: S = Q K^T (tcgen05, fp32 in TMEM) -> online softmax in registers
-// (one thread per row) -> P as bf16 back to TMEM -> O += P V (tcgen05, A operand from TMEM).
-// The running maximum only moves when it grew by more than 2^8, so rescaling O is rare; the
-// final normalisation uses the same reference, which keeps the result exact.
+// One CTA (one per SM) computes one work item: up to 256 packed query rows (one request, one KV
+// head) as two 128-row tiles A and B that share every K/V tile, against a range of key tiles of
+// 128 keys - first the cached prefix (pages of 16 tokens, staged with cp.async.bulk because a pool
+// page already is the shared-memory image the MMA reads), then the request's own rows (16-byte
+// cp.async gathers from the caller's row-major K/V, zero-filled past the end).
+// Per key tile and query tile: S = Q K^T (tcgen05, fp32 in TMEM) -> online softmax in registers
+// (one thread per row) -> P as bf16 written over S in TMEM -> O += P V (tcgen05, A from TMEM).
+// The tensor pipe alternates  S_A(j), O_B(j-1), S_B(j), O_A(j)  so that each softmax warpgroup
+// works while the other tile's MMAs run.  The running maximum only moves when it grew by more
+// than 2^8, so rescaling O is rare; the final normalisation uses the same reference, which keeps
+// the result exact.
 //
-// Roles: warps 0-3 softmax / correction / epilogue, warp 4 MMA issue and TMEM ownership,
-// warps 5-8 loads.  All waits are bounded; a wait that gives up raises a sticky status word
-// and the CTA drains and exits.
+// Roles: warps 0-3 softmax/correction/epilogue of tile A, warps 4-7 of tile B, warp 8 MMA issue
+// and TMEM ownership, warps 9-10 loads (warp 11 idles; 384 threads leave each 168 registers).  All waits are bounded; a wait that gives up raises a sticky status word and
+// the CTA drains and exits.
 #pragma once
 #include <cuda_bf16.h>
 #include "common.cuh"
@@ -23,28 +26,28 @@ constexpr bool kTensorPathBuilt = true;
 
 namespace tc {
 
-constexpr int kStages = 3;                       // K/V ring depth
 constexpr int kTileBytes = kTileKeys * 128 * 2;  // 32 KB: one 128 x 128 bf16 tile
 constexpr int kPageBytes = 4096;
-constexpr int kThreads = 288;
-constexpr int kSoftmaxThreads = 128;
-constexpr int kLoadThreads = 128;
-constexpr unsigned kMaxPolls = 1u << 21;         // bounded waits: about a quarter of a second
+constexpr int kRing = 5;                         // K/V ring slots of one tile each: K0 V0 K1 V1 ...
+constexpr int kThreads = 384;
+constexpr int kGroupThreads = 128;               // threads of one softmax warpgroup
+constexpr int kLoadThreads = 64;
+constexpr long long kWaitCycles = 400000000LL;   // bounded waits: about 0.2 s of SM clocks
 
-// shared-memory layout (dynamic, 1024-byte aligned by hand)
+// shared-memory layout (dynamic, 1024-byte aligned by hand): Q_A, Q_B, ring, barriers
 struct alignas(8) Barriers {
   unsigned long long q_full;
-  unsigned long long kv_full[kStages];
-  unsigned long long kv_free[kStages];
-  unsigned long long s_full[2];
-  unsigned long long s_free[2];
-  unsigned long long p_full[2];
-  unsigned long long o_done;
+  unsigned long long full[kRing];        // ring slot holds its tile
+  unsigned long long free_[kRing];       // the MMAs reading the slot have completed
+  unsigned long long s_full[2];          // S = Q K^T of the current key tile is in TMEM (per query tile)
+  unsigned long long p_full[2];          // P is in TMEM and O is rescaled (per query tile)
+  unsigned long long o_done;             // every MMA of the item has completed
   unsigned long long drain;
   unsigned tmem_base;
   int abort_flag;
 };
-constexpr int kSmemBytes = 1024 + kTileBytes * (1 + 2 * kStages) + (int)sizeof(Barriers) + 64;
+constexpr int kTmemCols = 512;           // S_A 0-127, S_B 128-255 (P over the first 64 of each), O_A 256-383, O_B 384-511
+constexpr int kSmemBytes = 1024 + kTileBytes * (2 + kRing) + (int)sizeof(Barriers) + 64;
 
 // ----- raw PTX wrappers --------------------------------------------------------------------
 __device__ __forceinline__ unsigned smem_u32(const void* p) {
@@ -70,13 +73,17 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
-// Bounded wait.  Returns false (and raises the CTA's abort flag) if the phase never completes.
+// Bounded wait.  try_wait suspends the thread in hardware until the phase completes or a short
+// system time limit passes, so the loop itself needs no sleep; the SM clock bounds the total.
+// Returns false (and raises the CTA's abort flag) if the phase never completes.
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
-  for (unsigned it = 0; it < kMaxPolls; ++it) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (unsigned it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (it >= 32) {
-      __nanosleep(64);
+    if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
+      if (clock64() - t0 > kWaitCycles) break;
     }
   }
   *abort_flag = 1;
@@ -202,6 +209,15 @@ __device__ __forceinline__ unsigned tile_chunk_offset(int r, int c16) {
   return (unsigned)((r >> 4) * kPageBytes) + page_chunk_offset(true, r & 15, c16, 256);
 }
 
+#ifdef BICACHE_TRACE
+// Debug build only: per-phase SM clock stamps of one CTA (three roles x 1024 slots).
+__device__ long long g_trace[3 * 1024];
+#define BICACHE_STAMP(role, idx) \
+  do { if (blockIdx.x == BICACHE_TRACE && (idx) < 1024) g_trace[(role) * 1024 + (idx)++] = clock64(); } while (0)
+#else
+#define BICACHE_STAMP(role, idx) do { } while (0)
+#endif
+
 }  // namespace tc
 
 __global__ void __launch_bounds__(tc::kThreads, 1)
@@ -210,10 +226,10 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  Barriers* bars = reinterpret_cast<Barriers*>(smem + kTileBytes * (1 + 2 * kStages));
+  Barriers* bars = reinterpret_cast<Barriers*>(smem + kTileBytes * (2 + kRing));
   volatile int* abort_flag = &bars->abort_flag;
-  const unsigned q_smem = smem_u32(smem);
-  const unsigned kv_smem = q_smem + kTileBytes;             // stage i: K at 2i, V at 2i + 1
+  const unsigned q_smem = smem_u32(smem);                  // Q_A, then Q_B
+  const unsigned ring_smem = q_smem + 2 * kTileBytes;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const WorkItem item = s.items[blockIdx.x];
@@ -228,66 +244,75 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
   }
   const int T = tile_end - tile_begin;
   const int packed_rows = req.n * G;
+  const bool b_active = item.row0 + 128 < packed_rows;     // the item has a second query tile
 
   if (tid == 0) {
     bars->abort_flag = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
     mbar_init(smem_u32(&bars->q_full), kLoadThreads);
-    for (int i = 0; i < kStages; ++i) {
-      mbar_init(smem_u32(&bars->kv_full[i]), kLoadThreads);
-      mbar_init(smem_u32(&bars->kv_free[i]), 1);
+    for (int i = 0; i < kRing; ++i) {
+      mbar_init(smem_u32(&bars->full[i]), kLoadThreads);
+      mbar_init(smem_u32(&bars->free_[i]), 1);
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&bars->s_full[i]), 1);
-      mbar_init(smem_u32(&bars->s_free[i]), kSoftmaxThreads);
-      mbar_init(smem_u32(&bars->p_full[i]), kSoftmaxThreads);
+      mbar_init(smem_u32(&bars->p_full[i]), kGroupThreads);
     }
     mbar_init(smem_u32(&bars->o_done), 1);
     mbar_init(smem_u32(&bars->drain), 1);
     fence_barrier_init();
   }
-  if (warp == 4) {
-    tmem_alloc(smem_u32(&bars->tmem_base), 512);
+  if (warp == 8) {
+    tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&bars->tmem_base);
-  const unsigned tmem_o = tmem + 256;
   const bool dead = *abort_flag != 0;        // an earlier CTA already gave up: do no work
 
-  if (!dead && warp < 4) {
-    // =========================== softmax / correction / epilogue ===========================
-    const unsigned lane_base = (unsigned)(warp * 32) << 16;  // this warp's quarter of the TMEM lanes
+  if (warp < 8) {
+    // ====================== softmax / correction / epilogue of one query tile ======================
+    const int X = warp >> 2;                                 // 0: tile A, 1: tile B
+    const int gt = tid & 127;                                // row of the tile = TMEM lane
+    const unsigned lane_base = (unsigned)((warp & 3) * 32) << 16;
+    const unsigned tmem_s = tmem + X * 128 + lane_base;      // S, and P written over its first 64 columns
+    const unsigned tmem_o = tmem + 256 + X * 128 + lane_base;
+    const bool active = !dead && (X == 0 || b_active);
     const float sl2 = t.scale * 1.4426950408889634f;         // scores are handled in the log2 domain
     float m_ref = -INFINITY, l_sum = 0.f;
-    bool ok = true;
-    for (int j = 0; j < T; ++j) {
-      const int b = j & 1;
-      const unsigned tmem_s = tmem + b * 128 + lane_base;
-      const unsigned tmem_p = tmem + 384 + b * 64 + lane_base;
+    bool ok = active;
+    int ti = 0; (void)ti;
+    for (int j = 0; j < T && active; ++j) {
       const int jg = tile_begin + j;
       const int cnt = jg < prefix_tiles ? min(kTileKeys, req.m - jg * kTileKeys)
                                         : min(kTileKeys, req.n - (jg - prefix_tiles) * kTileKeys);
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_full[b]), (j >> 1) & 1, abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_full[X]), j & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
-      // pass 1: row maximum of the scaled scores (columns >= cnt do not exist)
-      float mx = -INFINITY;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        unsigned r[32];
-        tmem_ld32(tmem_s + c * 32, r);
-        tmem_wait_ld();
-        if (cnt >= kTileKeys) {
+      if (gt == 0 && X == 0) BICACHE_STAMP(0, ti);
+      // the whole row of S into registers: four loads in flight, one wait
+      unsigned r[128];
+      tmem_ld32(tmem_s, r);
+      tmem_ld32(tmem_s + 32, r + 32);
+      tmem_ld32(tmem_s + 64, r + 64);
+      tmem_ld32(tmem_s + 96, r + 96);
+      tmem_wait_ld();
+      if (cnt < kTileKeys) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]) * sl2);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (c * 32 + i < cnt) mx = fmaxf(mx, __uint_as_float(r[i]) * sl2);
-        }
+        for (int i = 0; i < 128; ++i)
+          if (i >= cnt) r[i] = 0xff800000u;                  // -inf: columns past the last key
       }
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 128; i += 4) {
+        mx0 = fmaxf(mx0, __uint_as_float(r[i]));
+        mx1 = fmaxf(mx1, __uint_as_float(r[i + 1]));
+        mx2 = fmaxf(mx2, __uint_as_float(r[i + 2]));
+        mx3 = fmaxf(mx3, __uint_as_float(r[i + 3]));
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sl2;     // scale > 0
+      if (gt == 0 && X == 0) BICACHE_STAMP(0, ti);
       // The reference maximum moves only when the row maximum outgrew it by more than 2^8.
       float alpha = 1.f;
       if (j == 0) {
@@ -296,59 +321,45 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         alpha = ex2(m_ref - mx);
         m_ref = mx;
       }
-      if (j > 0) {
-        // P[b] was read by the P.V product of tile j-2 and O is accumulated by that of tile j-1:
-        // both have finished once o_done completed its phase for tile j-1.
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->o_done), (j - 1) & 1, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+      // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
+      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            unsigned r[32];
-            tmem_ld32(tmem_o + lane_base + c * 32, r);
-            tmem_wait_ld();
+        for (int c = 0; c < 4; ++c) {
+          unsigned o[32];
+          tmem_ld32(tmem_o + c * 32, o);
+          tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-            tmem_st32(tmem_o + lane_base + c * 32, r);
-          }
-          tmem_wait_st();
+          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+          tmem_st32(tmem_o + c * 32, o);
         }
       }
-      // pass 2: p = 2^(s - m_ref), row sum, P as bf16 into TMEM (two values per 32-bit column)
-      float psum = 0.f;
-#pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        unsigned r[32];
-        tmem_ld32(tmem_s + c * 32, r);
-        tmem_wait_ld();
-        unsigned pk[16];
+      if (gt == 0 && X == 0) BICACHE_STAMP(0, ti);
+      // p = 2^(s - m_ref), row sum, P as bf16 (two values per 32-bit column) over S
+      float ps0 = 0.f, ps1 = 0.f;
+      const float neg_m = -m_ref;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), sl2, -m_ref));
-          float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), sl2, -m_ref));
-          if (cnt < kTileKeys) {
-            if (c * 32 + 2 * i >= cnt) p0 = 0.f;
-            if (c * 32 + 2 * i + 1 >= cnt) p1 = 0.f;
-          }
-          psum += p0 + p1;
-          pk[i] = pack_bf16(p0, p1);
-        }
-        tmem_st16(tmem_p + c * 16, pk);
+      for (int i = 0; i < 64; ++i) {
+        const float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), sl2, neg_m));
+        const float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), sl2, neg_m));
+        ps0 += p0;
+        ps1 += p1;
+        r[i] = pack_bf16(p0, p1);
       }
+      tmem_st32(tmem_s, r);
+      tmem_st32(tmem_s + 32, r + 32);
       tmem_wait_st();
-      l_sum = l_sum * alpha + psum;
+      if (gt == 0 && X == 0) BICACHE_STAMP(0, ti);
+      l_sum = l_sum * alpha + (ps0 + ps1);
       tc_fence_before();
-      mbar_arrive(smem_u32(&bars->s_free[b]));      // S[b] may be overwritten by tile j + 2
-      mbar_arrive(smem_u32(&bars->p_full[b]));      // P[b] is complete, O is rescaled
+      mbar_arrive(smem_u32(&bars->p_full[X]));
     }
     // ------------------------------- epilogue -------------------------------------------
-    const int prow = item.row0 + tid;                // packed row of this thread
+    const int prow = item.row0 + X * 128 + gt;       // packed row of this thread
     const bool row_valid = prow < packed_rows;
     const int a = prow / G;
     const int h = item.kv_head * G + (prow - a * G);
     if (ok && T > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->o_done), (T - 1) & 1, abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->o_done), 0, abort_flag));
       if (ok) tc_fence_after();
     }
     if (ok) {
@@ -359,19 +370,19 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         float* po = t.part_o + pr * 128;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
-          unsigned r[32];
+          unsigned o[32];
           if (T > 0) {
-            tmem_ld32(tmem_o + lane_base + c * 32, r);
+            tmem_ld32(tmem_o + c * 32, o);
             tmem_wait_ld();
           } else {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) r[i] = 0u;
+            for (int i = 0; i < 32; ++i) o[i] = 0u;
           }
           if (row_valid) {
 #pragma unroll
             for (int i = 0; i < 32; i += 4) {
-              float4 v4 = make_float4(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv,
-                                      __uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
+              float4 v4 = make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv,
+                                      __uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
               *reinterpret_cast<float4*>(po + c * 32 + i) = v4;
             }
           }
@@ -381,17 +392,17 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         char* orow = t.out + ((req.row_off + a) * t.out_stride + (long long)h * 128) * 2;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
-          unsigned r[32];
-          tmem_ld32(tmem_o + lane_base + c * 32, r);
+          unsigned o[32];
+          tmem_ld32(tmem_o + c * 32, o);
           tmem_wait_ld();
           if (row_valid) {
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
               uint4 v4;
-              v4.x = pack_bf16(__uint_as_float(r[i]) * inv, __uint_as_float(r[i + 1]) * inv);
-              v4.y = pack_bf16(__uint_as_float(r[i + 2]) * inv, __uint_as_float(r[i + 3]) * inv);
-              v4.z = pack_bf16(__uint_as_float(r[i + 4]) * inv, __uint_as_float(r[i + 5]) * inv);
-              v4.w = pack_bf16(__uint_as_float(r[i + 6]) * inv, __uint_as_float(r[i + 7]) * inv);
+              v4.x = pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+              v4.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+              v4.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+              v4.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
               *reinterpret_cast<uint4*>(orow + (c * 32 + i) * 2) = v4;
             }
           }
@@ -400,95 +411,56 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       }
     }
     tc_fence_before();
-  } else if (!dead && warp == 4) {
-    // ===================================== MMA issue =====================================
-    if (lane == 0 && T > 0) {
-      bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
-      // software pipeline: S(j) = Q K_j^T is issued before O += P(j-1) V_(j-1)
-      for (int j = 0; j <= T && ok; ++j) {
-        if (j < T) {
-          const int st = j % kStages, b = j & 1;
-          ok = mbar_wait(smem_u32(&bars->kv_full[st]), (j / kStages) & 1, abort_flag);
-          if (ok) ok = mbar_wait(smem_u32(&bars->s_free[b]), ((j >> 1) & 1) ^ 1, abort_flag);
-          if (!ok) break;
-          fence_proxy_async();
-          tc_fence_after();
-          const unsigned k_smem = kv_smem + (2 * st) * kTileBytes;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const unsigned off = (k >> 2) * 1024 + (k & 3) * 32;
-            mma_ss(tmem + b * 128, make_desc(q_smem + off, 16, 2048), make_desc(k_smem + off, 16, 2048),
-                   kIdescQK, k > 0 ? 1u : 0u);
-          }
-          mma_commit(smem_u32(&bars->s_full[b]));
-        }
-        if (j >= 1) {
-          const int jp = j - 1, st = jp % kStages, b = jp & 1;
-          const int jg = tile_begin + jp;
-          const int cnt = jg < prefix_tiles ? min(kTileKeys, req.m - jg * kTileKeys)
-                                            : min(kTileKeys, req.n - (jg - prefix_tiles) * kTileKeys);
-          const int ksteps = (cnt + 15) >> 4;
-          ok = mbar_wait(smem_u32(&bars->p_full[b]), (jp >> 1) & 1, abort_flag);
-          if (!ok) break;
-          tc_fence_after();
-          const unsigned v_smem = kv_smem + (2 * st + 1) * kTileBytes;
-          for (int k = 0; k < ksteps; ++k) {
-            mma_ts(tmem_o, tmem + 384 + b * 64 + k * 8, make_desc(v_smem + k * kPageBytes, 1024, 2048),
-                   kIdescPV, (jp > 0 || k > 0) ? 1u : 0u);
-          }
-          mma_commit(smem_u32(&bars->kv_free[st]));
-          mma_commit(smem_u32(&bars->o_done));
+  } else if (warp == 9 || warp == 10) {
+    // ====================================== loads =======================================
+    const int lt = tid - 9 * 32;                      // 0..63
+    // A 128-row tile is fetched as 16 passes of 8 rows: thread lt takes 16-byte chunk (lt & 15) of
+    // rows (lt >> 4) + 8 i and (lt >> 4) + 4 + 8 i.  In the tile image those chunks sit 2048 bytes
+    // after the ones of pass i-1.
+    const int r0 = lt >> 4, c16 = lt & 15;
+    const unsigned dst_a = tile_chunk_offset(r0, c16), dst_b = tile_chunk_offset(r0 + 4, c16);
+    bool ok = !dead;
+    if (ok) {
+      // Q tiles: packed rows (token, head within the KV group); rows past the end are zero-filled
+      for (int x = 0; x < (b_active ? 2 : 1); ++x) {
+#pragma unroll 4
+        for (int i = 0; i < 32; ++i) {
+          const int prow = item.row0 + x * 128 + r0 + 4 * i;
+          const bool valid = prow < packed_rows;
+          const int a = valid ? prow / G : 0;
+          const int h = item.kv_head * G + (valid ? prow - a * G : 0);
+          const char* src = t.q + ((req.row_off + a) * t.q_stride + (long long)h * 128) * 2 + c16 * 16;
+          cp_async16(q_smem + x * kTileBytes + ((i & 1) ? dst_b : dst_a) + (i >> 1) * 2048, src, valid ? 16u : 0u);
         }
       }
-      // Whatever happened, let every MMA issued so far finish before TMEM is released.
-      mma_commit(smem_u32(&bars->drain));
-      mbar_wait(smem_u32(&bars->drain), 0, abort_flag);
+      cp_async_commit();
+      cp_async_wait<0>();
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&bars->q_full));
     }
-    __syncwarp();
-  } else if (!dead && warp >= 5) {
-    // ====================================== loads =======================================
-    const int lt = tid - 5 * 32;                      // 0..127
-    const int G_ = G;
-    // Q tile: 128 packed rows x 256 bytes; 16 consecutive threads fetch one row; rows past the
-    // request's end are zero-filled.
-#pragma unroll 4
-    for (int i = 0; i < 16; ++i) {
-      const int idx = i * kLoadThreads + lt;
-      const int r = idx >> 4, c16 = idx & 15;
-      const int prow = item.row0 + r;
-      const bool valid = prow < packed_rows;
-      const int a = valid ? prow / G_ : 0;
-      const int h = item.kv_head * G_ + (valid ? prow - a * G_ : 0);
-      const char* src = t.q + ((req.row_off + a) * t.q_stride + (long long)h * 128) * 2 + c16 * 16;
-      cp_async16(q_smem + tile_chunk_offset(r, c16), src, valid ? 16u : 0u);
-    }
-    cp_async_commit();
-    cp_async_wait<0>();
-    fence_proxy_async();
-    mbar_arrive(smem_u32(&bars->q_full));
-
     const int* pages = s.pages + req.page_off;
-    bool ok = true;
-    int pending_async = -1;                           // tile whose cp.async group is still in flight
-    for (int j = 0; j < T; ++j) {
-      const int st = j % kStages;
-      const int jg = tile_begin + j;
-      ok = mbar_wait(smem_u32(&bars->kv_free[st]), ((j / kStages) & 1) ^ 1, abort_flag);
+    int pending = -1;                                 // ring slot whose cp.async group is in flight
+    int ti = 0; (void)ti;
+    for (int u = 0; u < 2 * T && ok; ++u) {           // u = 2 j: K of tile j, u = 2 j + 1: V of tile j
+      const int slot = u % kRing;
+      const int jg = tile_begin + (u >> 1);
+      const bool is_v = u & 1;
+      ok = mbar_wait(smem_u32(&bars->free_[slot]), ((u / kRing) & 1) ^ 1, abort_flag);
       if (!ok) break;
-      const unsigned k_smem = kv_smem + (2 * st) * kTileBytes;
-      const unsigned v_smem = k_smem + kTileBytes;
-      const unsigned full = smem_u32(&bars->kv_full[st]);
+      if (lt == 0) BICACHE_STAMP(2, ti);
+      const unsigned dst = ring_smem + slot * kTileBytes;
+      const unsigned full = smem_u32(&bars->full[slot]);
       if (jg < prefix_tiles) {
-        // cached prefix tile: one bulk copy per page and tensor; a page is already the image
+        // cached prefix tile: one bulk copy per page; a pool page already is the tile image
         const int cnt = min(kTileKeys, req.m - jg * kTileKeys);
         const int npages = (cnt + kPageSize - 1) / kPageSize;
         if (lt == 0) {
-          mbar_arrive_expect_tx(full, (unsigned)(2 * npages * kPageBytes));
-          for (int pg = 0; pg < npages; ++pg) {
-            const long long off = pool_slice_offset(pool, t.layer, pages[jg * 8 + pg], item.kv_head);
-            bulk_copy_g2s(k_smem + pg * kPageBytes, pool.k + off, kPageBytes, full);
-            bulk_copy_g2s(v_smem + pg * kPageBytes, pool.v + off, kPageBytes, full);
-          }
+          const char* pool_base = is_v ? pool.v : pool.k;
+          mbar_arrive_expect_tx(full, (unsigned)(npages * kPageBytes));
+          for (int pg = 0; pg < npages; ++pg)
+            bulk_copy_g2s(dst + pg * kPageBytes,
+                          pool_base + pool_slice_offset(pool, t.layer, pages[jg * 8 + pg], item.kv_head),
+                          kPageBytes, full);
         } else {
           mbar_arrive(full);
         }
@@ -496,48 +468,133 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         // own rows: 16-byte gathers from row-major K/V into the image, zero-filled past the end
         const int key0 = (jg - prefix_tiles) * kTileKeys;
         const int cnt = min(kTileKeys, req.n - key0);
+        const char* row0 = (is_v ? t.v : t.k) +
+                           ((req.row_off + key0) * t.kv_stride + (long long)item.kv_head * 128) * 2 + c16 * 16;
+        const long long row_bytes = t.kv_stride * 2;
+        const char* src = row0 + r0 * row_bytes;
 #pragma unroll 4
         for (int i = 0; i < 16; ++i) {
-          const int idx = i * kLoadThreads + lt;
-          const int r = idx >> 4, c16 = idx & 15;
-          const bool valid = r < cnt;
-          const long long roff = ((req.row_off + key0 + (valid ? r : 0)) * t.kv_stride +
-                                  (long long)item.kv_head * 128) * 2 + c16 * 16;
-          const unsigned dst = tile_chunk_offset(r, c16);
-          cp_async16(k_smem + dst, t.k + roff, valid ? 16u : 0u);
-          cp_async16(v_smem + dst, t.v + roff, valid ? 16u : 0u);
+          const bool va = r0 + 8 * i < cnt, vb = r0 + 4 + 8 * i < cnt;
+          cp_async16(dst + dst_a + i * 2048, va ? src : row0, va ? 16u : 0u);
+          cp_async16(dst + dst_b + i * 2048, vb ? src + 4 * row_bytes : row0, vb ? 16u : 0u);
+          src += 8 * row_bytes;
         }
         cp_async_commit();
-        if (pending_async >= 0) {
+        if (pending >= 0) {
           cp_async_wait<1>();                         // the previous gathered tile has landed
           fence_proxy_async();
-          mbar_arrive(smem_u32(&bars->kv_full[pending_async % kStages]));
+          mbar_arrive(smem_u32(&bars->full[pending]));
         }
-        pending_async = j;
+        pending = slot;
       }
+      if (lt == 0) BICACHE_STAMP(2, ti);
     }
     cp_async_wait<0>();
-    if (pending_async >= 0) {
+    if (pending >= 0) {
       fence_proxy_async();
-      mbar_arrive(smem_u32(&bars->kv_full[pending_async % kStages]));
+      mbar_arrive(smem_u32(&bars->full[pending]));
     }
     // On the normal path every tile loaded has been consumed by the time the CTA ends (the
-    // epilogue waits for the last P.V).  After a give-up, bulk copies may still be in flight:
-    // wait (bounded) for the stages this thread armed.
-    if (!ok || *abort_flag) {
-      if (lt == 0) {
-        for (int j = max(0, T - kStages); j < T; ++j)
-          if (tile_begin + j < prefix_tiles)
-            for (unsigned it = 0; it < 4096 && !mbar_try_wait(smem_u32(&bars->kv_full[j % kStages]), (j / kStages) & 1); ++it)
-              __nanosleep(256);
-      }
+    // epilogue waits for the last MMA).  After a give-up, bulk copies may still be in flight:
+    // wait (bounded) for the last barriers this thread armed.
+    if (!dead && (!ok || *abort_flag) && lt == 0) {
+      for (int u = max(0, 2 * T - kRing); u < 2 * T; ++u)
+        if (tile_begin + (u >> 1) < prefix_tiles)
+          for (unsigned it = 0; it < 4096 && !mbar_try_wait(smem_u32(&bars->full[u % kRing]), (u / kRing) & 1); ++it)
+            __nanosleep(256);
     }
+  } else if (warp == 8) {
+    // ===================================== MMA issue =====================================
+    if (!dead && lane == 0 && T > 0) {
+      const unsigned tmem_sa = tmem, tmem_sb = tmem + 128, tmem_oa = tmem + 256, tmem_ob = tmem + 384;
+      const unsigned long long qa_desc = make_desc(q_smem, 16, 2048);
+      const unsigned long long qb_desc = make_desc(q_smem + kTileBytes, 16, 2048);
+      bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
+      int ti = 0; (void)ti;
+      BICACHE_STAMP(1, ti);
+      int prev_ksteps = 0;
+      for (int j = 0; j < T && ok; ++j) {
+        const int jg = tile_begin + j;
+        const int cnt = jg < prefix_tiles ? min(kTileKeys, req.m - jg * kTileKeys)
+                                          : min(kTileKeys, req.n - (jg - prefix_tiles) * kTileKeys);
+        const int ksteps = (cnt + 15) >> 4;
+        const int uk = 2 * j, uv = 2 * j + 1;
+        const int slot_k = uk % kRing, slot_v = uv % kRing;
+        ok = mbar_wait(smem_u32(&bars->full[slot_k]), (uk / kRing) & 1, abort_flag);
+        if (!ok) break;
+        BICACHE_STAMP(1, ti);
+        fence_proxy_async();
+        tc_fence_after();
+        // The descriptor's address field counts 16-byte units: a K step of 16 dims is +2, the second
+        // 64-dim half +64.
+        const unsigned long long k_desc = make_desc(ring_smem + slot_k * kTileBytes, 16, 2048);
+        // S_A = Q_A K^T.  It overwrites P_A of the previous key tile; the tensor pipe runs MMAs in
+        // issue order, so O_A += P_A V (issued earlier) has read P_A before this writes.
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const unsigned off = (k >> 2) * 64 + (k & 3) * 2;
+          mma_ss(tmem_sa, qa_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
+        }
+        mma_commit(smem_u32(&bars->s_full[0]));
+        BICACHE_STAMP(1, ti);
+        if (b_active) {
+          if (j > 0) {
+            // O_B += P_B V of the previous key tile
+            const int pv = 2 * (j - 1) + 1, pslot = pv % kRing;
+            ok = mbar_wait(smem_u32(&bars->p_full[1]), (j - 1) & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const unsigned long long v_desc = make_desc(ring_smem + pslot * kTileBytes, 1024, 2048);
+            for (int k = 0; k < prev_ksteps; ++k)
+              mma_ts(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, (j > 1 || k > 0) ? 1u : 0u);
+            mma_commit(smem_u32(&bars->free_[pslot]));
+          }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const unsigned off = (k >> 2) * 64 + (k & 3) * 2;
+            mma_ss(tmem_sb, qb_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
+          }
+          mma_commit(smem_u32(&bars->s_full[1]));
+        }
+        mma_commit(smem_u32(&bars->free_[slot_k]));
+        BICACHE_STAMP(1, ti);
+        // O_A += P_A V
+        ok = mbar_wait(smem_u32(&bars->p_full[0]), j & 1, abort_flag);
+        BICACHE_STAMP(1, ti);
+        if (ok) ok = mbar_wait(smem_u32(&bars->full[slot_v]), (uv / kRing) & 1, abort_flag);
+        if (!ok) break;
+        fence_proxy_async();
+        tc_fence_after();
+        const unsigned long long v_desc = make_desc(ring_smem + slot_v * kTileBytes, 1024, 2048);
+        for (int k = 0; k < ksteps; ++k)
+          mma_ts(tmem_oa, tmem_sa + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
+        if (!b_active) mma_commit(smem_u32(&bars->free_[slot_v]));
+        BICACHE_STAMP(1, ti);
+        prev_ksteps = ksteps;
+      }
+      if (ok && b_active) {
+        const int pv = 2 * (T - 1) + 1, pslot = pv % kRing;
+        ok = mbar_wait(smem_u32(&bars->p_full[1]), (T - 1) & 1, abort_flag);
+        if (ok) {
+          tc_fence_after();
+          const unsigned long long v_desc = make_desc(ring_smem + pslot * kTileBytes, 1024, 2048);
+          for (int k = 0; k < prev_ksteps; ++k)
+            mma_ts(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, (T > 1 || k > 0) ? 1u : 0u);
+          mma_commit(smem_u32(&bars->free_[pslot]));
+        }
+      }
+      if (ok) mma_commit(smem_u32(&bars->o_done));
+      // Whatever happened, let every MMA issued so far finish before TMEM is released.
+      mma_commit(smem_u32(&bars->drain));
+      mbar_wait(smem_u32(&bars->drain), 0, abort_flag);
+    }
+    __syncwarp();
   }
 
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 8) {
     tc_fence_after();
-    tmem_dealloc(tmem, 512);
+    tmem_dealloc(tmem, kTmemCols);
   }
   if (tid == 0 && !dead && *abort_flag) atomicCAS(status, kDevOk, kDevTimeout);
 }
