@@ -12,8 +12,10 @@
 // than 2^8, so rescaling O is rare; the final normalisation uses the same reference, which keeps
 // the result exact.
 //
-// Roles: warps 0-3 softmax/correction/epilogue of tile A, warps 4-7 of tile B, warp 8 MMA issue
-// and TMEM ownership, warps 9-10 loads (warp 11 idles; 384 threads leave each 168 registers).  All waits are bounded; a wait that gives up raises a sticky status word and
+// Roles: warps 0-3 softmax/correction/epilogue of tile A, warps 4-7 of tile B (one thread per
+// row), warp 8 MMA issue and TMEM ownership, warps 9-10 loads.  The whole SM is bound by
+// instruction issue, so the softmax uses packed fp32 instructions, 3-input maxima and as few
+// instructions per score as possible; MMAs are issued branch-free by an elected lane.  All waits are bounded; a wait that gives up raises a sticky status word and
 // the CTA drains and exits.
 #pragma once
 #include <cuda_bf16.h>
@@ -28,10 +30,14 @@ namespace tc {
 
 constexpr int kTileBytes = kTileKeys * 128 * 2;  // 32 KB: one 128 x 128 bf16 tile
 constexpr int kPageBytes = 4096;
-constexpr int kRing = 5;                         // K/V ring slots of one tile each: K0 V0 K1 V1 ...
+constexpr int kRing = 4;                         // K/V ring slots of one tile each: K0 V0 K1 V1
 constexpr int kThreads = 384;
-constexpr int kGroupThreads = 128;               // threads of one softmax warpgroup
+constexpr int kGroupThreads = 128;               // softmax threads of one query tile (one per row)
 constexpr int kLoadThreads = 64;
+constexpr int kSoftmaxRegs = 208;                // registers per thread after setmaxnreg
+constexpr int kOtherRegs = 80;
+constexpr int kMmaWarp = 8;
+constexpr int kPolyPeriod = 2;                   // of every kPolyPeriod groups of 4 scores, one sends 2 scores to the FMA-pipe cubic (0: none)
 constexpr long long kWaitCycles = 400000000LL;   // bounded waits: about 0.2 s of SM clocks
 
 // shared-memory layout (dynamic, 1024-byte aligned by hand): Q_A, Q_B, ring, barriers
@@ -119,6 +125,38 @@ __device__ __forceinline__ void tmem_dealloc(unsigned taddr, unsigned cols) {
 __device__ __forceinline__ void mma_commit(unsigned bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// The same two MMAs issued by one elected lane of a converged warp, without a branch: the election
+// and the accumulate flag are predicates inside one asm block.  `enable` = 0 skips the MMA.
+__device__ __forceinline__ void mma_ss_elect(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                             unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred P, Q;\n\t"
+      "elect.sync _|P, 0xffffffff;\n\t"
+      "setp.ne.b32 Q, %4, 0;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, Q;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ts_elect(unsigned d_tmem, unsigned a_tmem, unsigned long long b_desc,
+                                             unsigned idesc, unsigned accumulate, unsigned enable) {
+  asm volatile(
+      "{\n\t.reg .pred P, Q, E;\n\t"
+      "elect.sync _|P, 0xffffffff;\n\t"
+      "setp.ne.b32 Q, %4, 0;\n\t"
+      "setp.ne.b32 E, %5, 0;\n\t"
+      "and.pred P, P, E;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, Q;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(enable)
+      : "memory");
+}
+__device__ __forceinline__ void mma_commit_elect(unsigned bar) {
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "elect.sync _|P, 0xffffffff;\n\t"
+      "@P tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar)
+      : "memory");
+}
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
                                        unsigned idesc, unsigned accumulate) {
@@ -173,10 +211,60 @@ __device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* r) {
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// One lane of a converged warp (all 32 lanes must call this together).
+__device__ __forceinline__ bool elect_one() {
+  unsigned pred;
+  asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// two fp32 values in one 64-bit register, for the packed fp32 instructions
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+  unsigned long long d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ unsigned long long fma2(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long add2(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// 2^x for a pair of arguments on the FMA pipe (the exp unit is the scarce resource of the softmax):
+// x = n + f with n = round(x), f in [-0.5, 0.5]; 2^f by a cubic (relative error 7.5e-5, far below
+// the bf16 rounding of P); 2^n by adding n to the exponent field.  x is clamped at -126.
+__device__ __forceinline__ void ex2_poly2(unsigned long long x2, float& p0, float& p1) {
+  float x0, x1;
+  unpack2(x2, x0, x1);
+  x2 = pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
+  const unsigned long long magic = pack2(12582912.f, 12582912.f);          // 1.5 * 2^23
+  const unsigned long long t2 = add2(x2, magic);                            // low mantissa bits = round(x)
+  const unsigned long long neg_n2 = fma2(t2, pack2(-1.f, -1.f), magic);     // -(round(x))
+  const unsigned long long f2 = add2(x2, neg_n2);
+  unsigned long long q2 = fma2(f2, pack2(0.055171650f, 0.055171650f), pack2(0.24261113f, 0.24261113f));
+  q2 = fma2(q2, f2, pack2(0.69326097f, 0.69326097f));
+  q2 = fma2(q2, f2, pack2(0.99992806f, 0.99992806f));
+  float q0, q1, t0, t1;
+  unpack2(q2, q0, q1);
+  unpack2(t2, t0, t1);
+  p0 = __int_as_float(__float_as_int(q0) + (__float_as_int(t0) << 23));
+  p1 = __int_as_float(__float_as_int(q1) + (__float_as_int(t1) << 23));
 }
 __device__ __forceinline__ unsigned pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);     // .x = lo (low 16 bits), .y = hi
@@ -261,7 +349,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
     mbar_init(smem_u32(&bars->drain), 1);
     fence_barrier_init();
   }
-  if (warp == 8) {
+  if (warp == kMmaWarp) {
     tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
     tmem_relinquish();
   }
@@ -271,6 +359,15 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&bars->tmem_base);
   const bool dead = *abort_flag != 0;        // an earlier CTA already gave up: do no work
 
+  // Registers move from the MMA/load warpgroup to the two softmax warpgroups, which hold a whole
+  // row of S (128 values) per thread.  The counts must fit the CTA's launch allocation:
+  // 256 * kSoftmaxRegs + 128 * kOtherRegs <= 384 * (registers per thread at launch); the host
+  // checks this before the first launch, because an increase that cannot be met never returns.
+  if (warp < 8) {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
+  } else {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
+  }
   if (warp < 8) {
     // ====================== softmax / correction / epilogue of one query tile ======================
     const int X = warp >> 2;                                 // 0: tile A, 1: tile B
@@ -280,6 +377,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
     const unsigned tmem_o = tmem + 256 + X * 128 + lane_base;
     const bool active = !dead && (X == 0 || b_active);
     const float sl2 = t.scale * 1.4426950408889634f;         // scores are handled in the log2 domain
+    const unsigned long long sl2_2 = pack2(sl2, sl2);
     float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = active;
     int ti = 0; (void)ti;
@@ -290,7 +388,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_full[X]), j & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
-      if (gt == 0 && X == 0) BICACHE_STAMP(0, ti);
+      if (tid == 0) BICACHE_STAMP(0, ti);
       // the whole row of S into registers: four loads in flight, one wait
       unsigned r[128];
       tmem_ld32(tmem_s, r);
@@ -298,58 +396,137 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       tmem_ld32(tmem_s + 64, r + 64);
       tmem_ld32(tmem_s + 96, r + 96);
       tmem_wait_ld();
-      if (cnt < kTileKeys) {
-#pragma unroll
-        for (int i = 0; i < 128; ++i)
-          if (i >= cnt) r[i] = 0xff800000u;                  // -inf: columns past the last key
-      }
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-      for (int i = 0; i < 128; i += 4) {
-        mx0 = fmaxf(mx0, __uint_as_float(r[i]));
-        mx1 = fmaxf(mx1, __uint_as_float(r[i + 1]));
-        mx2 = fmaxf(mx2, __uint_as_float(r[i + 2]));
-        mx3 = fmaxf(mx3, __uint_as_float(r[i + 3]));
-      }
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sl2;     // scale > 0
-      if (gt == 0 && X == 0) BICACHE_STAMP(0, ti);
-      // The reference maximum moves only when the row maximum outgrew it by more than 2^8.
       float alpha = 1.f;
-      if (j == 0) {
-        m_ref = mx;
-      } else if (mx > m_ref + 8.f) {
-        alpha = ex2(m_ref - mx);
-        m_ref = mx;
-      }
-      // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
-      if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          unsigned o[32];
-          tmem_ld32(tmem_o + c * 32, o);
-          tmem_wait_ld();
+      unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
+      if (j > 0 && cnt >= kTileKeys) {
+        // Common case (a full tile after the first): the exponentials use the reference maximum of
+        // the earlier tiles and do not wait for this tile's maximum, which is computed alongside.
+        // If the row maximum turns out to exceed the reference by more than 2^8 (rare: checked per
+        // warp), the tile is redone below with the new reference.
+        const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
+        float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-          tmem_st32(tmem_o + c * 32, o);
+        for (int i = 0; i < 32; ++i) {
+          const float s0 = __uint_as_float(r[4 * i]), s1 = __uint_as_float(r[4 * i + 1]);
+          const float s2 = __uint_as_float(r[4 * i + 2]), s3 = __uint_as_float(r[4 * i + 3]);
+          mx0 = max3(mx0, s0, s1);
+          mx1 = max3(mx1, s2, s3);
+          const unsigned long long xa = fma2(pack2(s0, s1), sl2_2, neg_m2);
+          const unsigned long long xb = fma2(pack2(s2, s3), sl2_2, neg_m2);
+          float xa0, xa1, p0, p1, p2, p3;
+          unpack2(xa, xa0, xa1);
+          p0 = ex2(xa0);
+          p1 = ex2(xa1);
+          if (kPolyPeriod > 0 && (i % (kPolyPeriod > 0 ? kPolyPeriod : 1)) == 0) {
+            ex2_poly2(xb, p2, p3);
+          } else {
+            float xb0, xb1;
+            unpack2(xb, xb0, xb1);
+            p2 = ex2(xb0);
+            p3 = ex2(xb1);
+          }
+          acc_a = add2(acc_a, pack2(p0, p1));
+          acc_b = add2(acc_b, pack2(p2, p3));
+          r[2 * i] = pack_bf16(p0, p1);
+          r[2 * i + 1] = pack_bf16(p2, p3);
+        }
+        const float mx = fmaxf(mx0, mx1) * sl2;              // scale > 0
+        if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+          // redo with the new reference: S is still intact in TMEM
+          if (mx > m_ref + 8.f) {
+            alpha = ex2(m_ref - mx);
+            m_ref = mx;
+          }
+          unsigned s4[32];
+          const float neg_m = -m_ref;
+          float ps = 0.f;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tmem_s + c * 32, s4);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float p0 = ex2(fmaf(__uint_as_float(s4[2 * i]), sl2, neg_m));
+              const float p1 = ex2(fmaf(__uint_as_float(s4[2 * i + 1]), sl2, neg_m));
+              ps += p0 + p1;
+              r[c * 16 + i] = pack_bf16(p0, p1);
+            }
+          }
+          acc_a = pack2(ps, 0.f);
+          acc_b = pack2(0.f, 0.f);
+          // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tmem_o + c * 32, s4);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) s4[i] = __float_as_uint(__uint_as_float(s4[i]) * alpha);
+            tmem_st32(tmem_o + c * 32, s4);
+          }
+        }
+      } else {
+        // First tile of the item, or a ragged tile: maximum first, every exponential on the exp
+        // unit so that masked columns give exactly 0.
+        if (cnt < kTileKeys) {
+#pragma unroll
+          for (int i = 0; i < 128; ++i)
+            if (i >= cnt) r[i] = 0xff800000u;                // -inf: columns past the last key
+        }
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 128; i += 8) {
+          mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+          mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+          mx2 = max3(mx2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+          mx3 = max3(mx3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sl2;   // scale > 0
+        if (j == 0) {
+          m_ref = mx;
+        } else if (mx > m_ref + 8.f) {
+          alpha = ex2(m_ref - mx);
+          m_ref = mx;
+        }
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            unsigned o[32];
+            tmem_ld32(tmem_o + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            tmem_st32(tmem_o + c * 32, o);
+          }
+        }
+        const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const unsigned long long xa =
+              fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+          const unsigned long long xb =
+              fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+          float x0, x1, x2, x3;
+          unpack2(xa, x0, x1);
+          unpack2(xb, x2, x3);
+          const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+          acc_a = add2(acc_a, pack2(p0, p1));
+          acc_b = add2(acc_b, pack2(p2, p3));
+          r[2 * i] = pack_bf16(p0, p1);
+          r[2 * i + 1] = pack_bf16(p2, p3);
         }
       }
-      if (gt == 0 && X == 0) BICACHE_STAMP(0, ti);
-      // p = 2^(s - m_ref), row sum, P as bf16 (two values per 32-bit column) over S
-      float ps0 = 0.f, ps1 = 0.f;
-      const float neg_m = -m_ref;
-#pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        const float p0 = ex2(fmaf(__uint_as_float(r[2 * i]), sl2, neg_m));
-        const float p1 = ex2(fmaf(__uint_as_float(r[2 * i + 1]), sl2, neg_m));
-        ps0 += p0;
-        ps1 += p1;
-        r[i] = pack_bf16(p0, p1);
-      }
+      if (tid == 0) BICACHE_STAMP(0, ti);
+      if (tid == 0) BICACHE_STAMP(0, ti);
       tmem_st32(tmem_s, r);
       tmem_st32(tmem_s + 32, r + 32);
       tmem_wait_st();
-      if (gt == 0 && X == 0) BICACHE_STAMP(0, ti);
-      l_sum = l_sum * alpha + (ps0 + ps1);
+      if (tid == 0) BICACHE_STAMP(0, ti);
+      {
+        float s0, s1, s2, s3;
+        unpack2(acc_a, s0, s1);
+        unpack2(acc_b, s2, s3);
+        l_sum = l_sum * alpha + ((s0 + s1) + (s2 + s3));
+      }
       tc_fence_before();
       mbar_arrive(smem_u32(&bars->p_full[X]));
     }
@@ -433,11 +610,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
           cp_async16(q_smem + x * kTileBytes + ((i & 1) ? dst_b : dst_a) + (i >> 1) * 2048, src, valid ? 16u : 0u);
         }
       }
-      cp_async_commit();
-      cp_async_wait<0>();
-      fence_proxy_async();
-      mbar_arrive(smem_u32(&bars->q_full));
+      cp_async_commit();                              // lands while the first K/V loads are issued
     }
+    bool q_pending = ok;
     const int* pages = s.pages + req.page_off;
     int pending = -1;                                 // ring slot whose cp.async group is in flight
     int ti = 0; (void)ti;
@@ -464,6 +639,12 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         } else {
           mbar_arrive(full);
         }
+        if (q_pending) {
+          cp_async_wait<0>();
+          fence_proxy_async();
+          mbar_arrive(smem_u32(&bars->q_full));
+          q_pending = false;
+        }
       } else {
         // own rows: 16-byte gathers from row-major K/V into the image, zero-filled past the end
         const int key0 = (jg - prefix_tiles) * kTileKeys;
@@ -480,20 +661,21 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
           src += 8 * row_bytes;
         }
         cp_async_commit();
-        if (pending >= 0) {
-          cp_async_wait<1>();                         // the previous gathered tile has landed
+        if (pending >= 0 || q_pending) {
+          cp_async_wait<1>();                         // everything but the tile just issued has landed
           fence_proxy_async();
-          mbar_arrive(smem_u32(&bars->full[pending]));
+          if (q_pending) mbar_arrive(smem_u32(&bars->q_full));
+          if (pending >= 0) mbar_arrive(smem_u32(&bars->full[pending]));
+          q_pending = false;
         }
         pending = slot;
       }
       if (lt == 0) BICACHE_STAMP(2, ti);
     }
     cp_async_wait<0>();
-    if (pending >= 0) {
-      fence_proxy_async();
-      mbar_arrive(smem_u32(&bars->full[pending]));
-    }
+    fence_proxy_async();
+    if (q_pending) mbar_arrive(smem_u32(&bars->q_full));
+    if (pending >= 0) mbar_arrive(smem_u32(&bars->full[pending]));
     // On the normal path every tile loaded has been consumed by the time the CTA ends (the
     // epilogue waits for the last MMA).  After a give-up, bulk copies may still be in flight:
     // wait (bounded) for the last barriers this thread armed.
@@ -503,15 +685,18 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
           for (unsigned it = 0; it < 4096 && !mbar_try_wait(smem_u32(&bars->full[u % kRing]), (u / kRing) & 1); ++it)
             __nanosleep(256);
     }
-  } else if (warp == 8) {
+  } else if (warp == kMmaWarp) {
     // ===================================== MMA issue =====================================
-    if (!dead && lane == 0 && T > 0) {
+    // The whole warp runs this control flow converged and one elected lane issues each tcgen05
+    // instruction: descriptor arithmetic then stays in the uniform datapath and the MMAs can be
+    // issued back to back (a single diverged lane cannot feed the tensor pipe fast enough).
+    if (!dead && T > 0) {
       const unsigned tmem_sa = tmem, tmem_sb = tmem + 128, tmem_oa = tmem + 256, tmem_ob = tmem + 384;
       const unsigned long long qa_desc = make_desc(q_smem, 16, 2048);
       const unsigned long long qb_desc = make_desc(q_smem + kTileBytes, 16, 2048);
-      bool ok = mbar_wait(smem_u32(&bars->q_full), 0, abort_flag);
+      bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_full), 0, abort_flag));
       int ti = 0; (void)ti;
-      BICACHE_STAMP(1, ti);
+      if (lane == 0) BICACHE_STAMP(1, ti);
       int prev_ksteps = 0;
       for (int j = 0; j < T && ok; ++j) {
         const int jg = tile_begin + j;
@@ -520,9 +705,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         const int ksteps = (cnt + 15) >> 4;
         const int uk = 2 * j, uv = 2 * j + 1;
         const int slot_k = uk % kRing, slot_v = uv % kRing;
-        ok = mbar_wait(smem_u32(&bars->full[slot_k]), (uk / kRing) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_k]), (uk / kRing) & 1, abort_flag));
         if (!ok) break;
-        BICACHE_STAMP(1, ti);
+        if (lane == 0) BICACHE_STAMP(1, ti);
         fence_proxy_async();
         tc_fence_after();
         // The descriptor's address field counts 16-byte units: a K step of 16 dims is +2, the second
@@ -533,66 +718,76 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
           const unsigned off = (k >> 2) * 64 + (k & 3) * 2;
-          mma_ss(tmem_sa, qa_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
+          mma_ss_elect(tmem_sa, qa_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
         }
-        mma_commit(smem_u32(&bars->s_full[0]));
-        BICACHE_STAMP(1, ti);
+        mma_commit_elect(smem_u32(&bars->s_full[0]));
+        if (lane == 0) BICACHE_STAMP(1, ti);
         if (b_active) {
           if (j > 0) {
             // O_B += P_B V of the previous key tile
             const int pv = 2 * (j - 1) + 1, pslot = pv % kRing;
-            ok = mbar_wait(smem_u32(&bars->p_full[1]), (j - 1) & 1, abort_flag);
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_full[1]), (j - 1) & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
             const unsigned long long v_desc = make_desc(ring_smem + pslot * kTileBytes, 1024, 2048);
-            for (int k = 0; k < prev_ksteps; ++k)
-              mma_ts(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, (j > 1 || k > 0) ? 1u : 0u);
-            mma_commit(smem_u32(&bars->free_[pslot]));
+            const unsigned acc0 = j > 1 ? 1u : 0u;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              mma_ts_elect(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
+                           k < prev_ksteps ? 1u : 0u);
+            mma_commit_elect(smem_u32(&bars->free_[pslot]));
           }
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const unsigned off = (k >> 2) * 64 + (k & 3) * 2;
-            mma_ss(tmem_sb, qb_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
+            mma_ss_elect(tmem_sb, qb_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
           }
-          mma_commit(smem_u32(&bars->s_full[1]));
+          mma_commit_elect(smem_u32(&bars->s_full[1]));
         }
-        mma_commit(smem_u32(&bars->free_[slot_k]));
-        BICACHE_STAMP(1, ti);
+        mma_commit_elect(smem_u32(&bars->free_[slot_k]));
+        if (lane == 0) BICACHE_STAMP(1, ti);
         // O_A += P_A V
-        ok = mbar_wait(smem_u32(&bars->p_full[0]), j & 1, abort_flag);
-        BICACHE_STAMP(1, ti);
-        if (ok) ok = mbar_wait(smem_u32(&bars->full[slot_v]), (uv / kRing) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_full[0]), j & 1, abort_flag));
+        if (lane == 0) BICACHE_STAMP(1, ti);
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_v]), (uv / kRing) & 1, abort_flag));
         if (!ok) break;
         fence_proxy_async();
         tc_fence_after();
         const unsigned long long v_desc = make_desc(ring_smem + slot_v * kTileBytes, 1024, 2048);
-        for (int k = 0; k < ksteps; ++k)
-          mma_ts(tmem_oa, tmem_sa + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, (j > 0 || k > 0) ? 1u : 0u);
-        if (!b_active) mma_commit(smem_u32(&bars->free_[slot_v]));
-        BICACHE_STAMP(1, ti);
+        const unsigned acc0 = j > 0 ? 1u : 0u;
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          mma_ts_elect(tmem_oa, tmem_sa + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
+                       k < ksteps ? 1u : 0u);
+        if (!b_active) mma_commit_elect(smem_u32(&bars->free_[slot_v]));
+        if (lane == 0) BICACHE_STAMP(1, ti);
         prev_ksteps = ksteps;
       }
       if (ok && b_active) {
         const int pv = 2 * (T - 1) + 1, pslot = pv % kRing;
-        ok = mbar_wait(smem_u32(&bars->p_full[1]), (T - 1) & 1, abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_full[1]), (T - 1) & 1, abort_flag));
         if (ok) {
           tc_fence_after();
           const unsigned long long v_desc = make_desc(ring_smem + pslot * kTileBytes, 1024, 2048);
-          for (int k = 0; k < prev_ksteps; ++k)
-            mma_ts(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, (T > 1 || k > 0) ? 1u : 0u);
-          mma_commit(smem_u32(&bars->free_[pslot]));
+          const unsigned acc0 = T > 1 ? 1u : 0u;
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            mma_ts_elect(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
+                         k < prev_ksteps ? 1u : 0u);
+          mma_commit_elect(smem_u32(&bars->free_[pslot]));
         }
       }
-      if (ok) mma_commit(smem_u32(&bars->o_done));
+      if (ok) mma_commit_elect(smem_u32(&bars->o_done));
       // Whatever happened, let every MMA issued so far finish before TMEM is released.
-      mma_commit(smem_u32(&bars->drain));
+      __syncwarp();
+      mma_commit_elect(smem_u32(&bars->drain));
       mbar_wait(smem_u32(&bars->drain), 0, abort_flag);
     }
     __syncwarp();
   }
 
   __syncthreads();
-  if (warp == 8) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
@@ -600,6 +795,12 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
 }
 
 inline cudaError_t configure_tc_attention() {
+  cudaFuncAttributes attr;
+  cudaError_t e = cudaFuncGetAttributes(&attr, tc_attention_kernel);
+  if (e != cudaSuccess) return e;
+  // the register pool the kernel redistributes is the launch allocation of the CTA
+  if (attr.numRegs * tc::kThreads < 2 * tc::kGroupThreads * tc::kSoftmaxRegs + 128 * tc::kOtherRegs)
+    return cudaErrorLaunchOutOfResources;
   return cudaFuncSetAttribute(tc_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes);
 }
 
