@@ -46,7 +46,7 @@ struct alignas(8) Barriers {
   unsigned long long full[kRing];        // ring slot holds its tile
   unsigned long long free_[kRing];       // the MMAs reading the slot have completed
   unsigned long long s_full[2];          // S = Q K^T of the current key tile is in TMEM (per query tile)
-  unsigned long long p_full[2];          // P is in TMEM and O is rescaled (per query tile)
+  unsigned long long p_half[2][2];       // P of keys 0-63 / 64-127 is in TMEM and O is rescaled (per query tile)
   unsigned long long o_done;             // every MMA of the item has completed
   unsigned long long drain;
   unsigned tmem_base;
@@ -343,7 +343,8 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&bars->s_full[i]), 1);
-      mbar_init(smem_u32(&bars->p_full[i]), kGroupThreads);
+      mbar_init(smem_u32(&bars->p_half[i][0]), kGroupThreads);
+      mbar_init(smem_u32(&bars->p_half[i][1]), kGroupThreads);
     }
     mbar_init(smem_u32(&bars->o_done), 1);
     mbar_init(smem_u32(&bars->drain), 1);
@@ -389,49 +390,70 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       if (!ok) break;
       tc_fence_after();
       if (tid == 0) BICACHE_STAMP(0, ti);
-      // the whole row of S into registers: four loads in flight, one wait
+      // S of keys 0-63 first; the load of keys 64-127 is issued right after and lands while the
+      // first half is processed.
       unsigned r[128];
       tmem_ld32(tmem_s, r);
       tmem_ld32(tmem_s + 32, r + 32);
+      tmem_wait_ld();
       tmem_ld32(tmem_s + 64, r + 64);
       tmem_ld32(tmem_s + 96, r + 96);
-      tmem_wait_ld();
       float alpha = 1.f;
       unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
+      bool stored = false;                                   // P already stored and signalled
       if (j > 0 && cnt >= kTileKeys) {
         // Common case (a full tile after the first): the exponentials use the reference maximum of
         // the earlier tiles and do not wait for this tile's maximum, which is computed alongside.
+        // P of the first 64 keys is handed to the tensor pipe before the second half is computed.
         // If the row maximum turns out to exceed the reference by more than 2^8 (rare: checked per
-        // warp), the tile is redone below with the new reference.
+        // warp before anything is handed over), the tile is redone below with the new reference.
         const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
         float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float s0 = __uint_as_float(r[4 * i]), s1 = __uint_as_float(r[4 * i + 1]);
-          const float s2 = __uint_as_float(r[4 * i + 2]), s3 = __uint_as_float(r[4 * i + 3]);
-          mx0 = max3(mx0, s0, s1);
-          mx1 = max3(mx1, s2, s3);
-          const unsigned long long xa = fma2(pack2(s0, s1), sl2_2, neg_m2);
-          const unsigned long long xb = fma2(pack2(s2, s3), sl2_2, neg_m2);
-          float xa0, xa1, p0, p1, p2, p3;
-          unpack2(xa, xa0, xa1);
-          p0 = ex2(xa0);
-          p1 = ex2(xa1);
-          if (kPolyPeriod > 0 && (i % (kPolyPeriod > 0 ? kPolyPeriod : 1)) == 0) {
-            ex2_poly2(xb, p2, p3);
-          } else {
-            float xb0, xb1;
-            unpack2(xb, xb0, xb1);
-            p2 = ex2(xb0);
-            p3 = ex2(xb1);
-          }
-          acc_a = add2(acc_a, pack2(p0, p1));
-          acc_b = add2(acc_b, pack2(p2, p3));
-          r[2 * i] = pack_bf16(p0, p1);
-          r[2 * i + 1] = pack_bf16(p2, p3);
+        for (int i = 0; i < 16; ++i) {
+          mx0 = max3(mx0, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
+          mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+        }
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 16; i < 32; ++i) {
+          mx0 = max3(mx0, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
+          mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
         }
         const float mx = fmaxf(mx0, mx1) * sl2;              // scale > 0
-        if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+        if (!__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+#pragma unroll
+          for (int half = 0; half < 2; ++half) {
+#pragma unroll
+            for (int i = half * 16; i < half * 16 + 16; ++i) {
+              const unsigned long long xa =
+                  fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+              const unsigned long long xb =
+                  fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+              float xa0, xa1, p0, p1, p2, p3;
+              unpack2(xa, xa0, xa1);
+              p0 = ex2(xa0);
+              p1 = ex2(xa1);
+              if (kPolyPeriod > 0 && (i % (kPolyPeriod > 0 ? kPolyPeriod : 1)) == 0) {
+                ex2_poly2(xb, p2, p3);
+              } else {
+                float xb0, xb1;
+                unpack2(xb, xb0, xb1);
+                p2 = ex2(xb0);
+                p3 = ex2(xb1);
+              }
+              acc_a = add2(acc_a, pack2(p0, p1));
+              acc_b = add2(acc_b, pack2(p2, p3));
+              r[2 * i] = pack_bf16(p0, p1);
+              r[2 * i + 1] = pack_bf16(p2, p3);
+            }
+            tmem_st32(tmem_s + half * 32, r + half * 32);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->p_half[X][half]));
+          }
+          stored = true;
+        } else {
           // redo with the new reference: S is still intact in TMEM
           if (mx > m_ref + 8.f) {
             alpha = ex2(m_ref - mx);
@@ -453,7 +475,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
             }
           }
           acc_a = pack2(ps, 0.f);
-          acc_b = pack2(0.f, 0.f);
           // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
@@ -467,6 +488,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       } else {
         // First tile of the item, or a ragged tile: maximum first, every exponential on the exp
         // unit so that masked columns give exactly 0.
+        tmem_wait_ld();
         if (cnt < kTileKeys) {
 #pragma unroll
           for (int i = 0; i < 128; ++i)
@@ -517,9 +539,14 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       }
       if (tid == 0) BICACHE_STAMP(0, ti);
       if (tid == 0) BICACHE_STAMP(0, ti);
-      tmem_st32(tmem_s, r);
-      tmem_st32(tmem_s + 32, r + 32);
-      tmem_wait_st();
+      if (!stored) {
+        tmem_st32(tmem_s, r);
+        tmem_st32(tmem_s + 32, r + 32);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars->p_half[X][0]));
+        mbar_arrive(smem_u32(&bars->p_half[X][1]));
+      }
       if (tid == 0) BICACHE_STAMP(0, ti);
       {
         float s0, s1, s2, s3;
@@ -527,8 +554,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         unpack2(acc_b, s2, s3);
         l_sum = l_sum * alpha + ((s0 + s1) + (s2 + s3));
       }
-      tc_fence_before();
-      mbar_arrive(smem_u32(&bars->p_full[X]));
     }
     // ------------------------------- epilogue -------------------------------------------
     const int prow = item.row0 + X * 128 + gt;       // packed row of this thread
@@ -726,15 +751,19 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
           if (j > 0) {
             // O_B += P_B V of the previous key tile
             const int pv = 2 * (j - 1) + 1, pslot = pv % kRing;
-            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_full[1]), (j - 1) & 1, abort_flag));
-            if (!ok) break;
-            tc_fence_after();
             const unsigned long long v_desc = make_desc(ring_smem + pslot * kTileBytes, 1024, 2048);
             const unsigned acc0 = j > 1 ? 1u : 0u;
 #pragma unroll
-            for (int k = 0; k < 8; ++k)
-              mma_ts_elect(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
-                           k < prev_ksteps ? 1u : 0u);
+            for (int half = 0; half < 2 && ok; ++half) {
+              ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[1][half]), (j - 1) & 1, abort_flag));
+              if (!ok) break;
+              tc_fence_after();
+#pragma unroll
+              for (int k = half * 4; k < half * 4 + 4; ++k)
+                mma_ts_elect(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
+                             k < prev_ksteps ? 1u : 0u);
+            }
+            if (!ok) break;
             mma_commit_elect(smem_u32(&bars->free_[pslot]));
           }
 #pragma unroll
@@ -747,35 +776,42 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         mma_commit_elect(smem_u32(&bars->free_[slot_k]));
         if (lane == 0) BICACHE_STAMP(1, ti);
         // O_A += P_A V
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_full[0]), j & 1, abort_flag));
-        if (lane == 0) BICACHE_STAMP(1, ti);
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_v]), (uv / kRing) & 1, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_v]), (uv / kRing) & 1, abort_flag));
         if (!ok) break;
         fence_proxy_async();
-        tc_fence_after();
         const unsigned long long v_desc = make_desc(ring_smem + slot_v * kTileBytes, 1024, 2048);
         const unsigned acc0 = j > 0 ? 1u : 0u;
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          mma_ts_elect(tmem_oa, tmem_sa + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
-                       k < ksteps ? 1u : 0u);
+        for (int half = 0; half < 2 && ok; ++half) {
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[0][half]), j & 1, abort_flag));
+          if (!ok) break;
+          if (lane == 0 && half == 0) BICACHE_STAMP(1, ti);
+          tc_fence_after();
+#pragma unroll
+          for (int k = half * 4; k < half * 4 + 4; ++k)
+            mma_ts_elect(tmem_oa, tmem_sa + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
+                         k < ksteps ? 1u : 0u);
+        }
+        if (!ok) break;
         if (!b_active) mma_commit_elect(smem_u32(&bars->free_[slot_v]));
         if (lane == 0) BICACHE_STAMP(1, ti);
         prev_ksteps = ksteps;
       }
       if (ok && b_active) {
         const int pv = 2 * (T - 1) + 1, pslot = pv % kRing;
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_full[1]), (T - 1) & 1, abort_flag));
-        if (ok) {
-          tc_fence_after();
-          const unsigned long long v_desc = make_desc(ring_smem + pslot * kTileBytes, 1024, 2048);
-          const unsigned acc0 = T > 1 ? 1u : 0u;
+        const unsigned long long v_desc = make_desc(ring_smem + pslot * kTileBytes, 1024, 2048);
+        const unsigned acc0 = T > 1 ? 1u : 0u;
 #pragma unroll
-          for (int k = 0; k < 8; ++k)
+        for (int half = 0; half < 2 && ok; ++half) {
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[1][half]), (T - 1) & 1, abort_flag));
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int k = half * 4; k < half * 4 + 4; ++k)
             mma_ts_elect(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
                          k < prev_ksteps ? 1u : 0u);
-          mma_commit_elect(smem_u32(&bars->free_[pslot]));
         }
+        if (ok) mma_commit_elect(smem_u32(&bars->free_[pslot]));
       }
       if (ok) mma_commit_elect(smem_u32(&bars->o_done));
       // Whatever happened, let every MMA issued so far finish before TMEM is released.
