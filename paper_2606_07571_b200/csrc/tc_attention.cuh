@@ -37,7 +37,10 @@ constexpr int kLoadThreads = 64;
 constexpr int kSoftmaxRegs = 208;                // registers per thread after setmaxnreg
 constexpr int kOtherRegs = 80;
 constexpr int kMmaWarp = 8;
-constexpr int kPolyPeriod = 2;                   // of every kPolyPeriod groups of 4 scores, one sends 2 scores to the FMA-pipe cubic (0: none)
+#ifndef BICACHE_POLY_PERIOD
+#define BICACHE_POLY_PERIOD 0
+#endif
+constexpr int kPolyPeriod = BICACHE_POLY_PERIOD;                   // of every kPolyPeriod groups of 4 scores, one sends 2 scores to the FMA-pipe cubic (0: none)
 constexpr long long kWaitCycles = 400000000LL;   // bounded waits: about 0.2 s of SM clocks
 
 // shared-memory layout (dynamic, 1024-byte aligned by hand): Q_A, Q_B, ring, barriers
