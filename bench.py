@@ -33,7 +33,7 @@ UNIT = "tokens/s"
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from ncu captures summarised
 # under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {"config2": {"full": 652.7e6, "attend": 134.7e6}}     # profiles/tc_attention_kernel_config2.md
 
 
 def load_peaks():
@@ -166,6 +166,14 @@ def time_call(fn, iters, flush):
         b.record()
     torch.cuda.synchronize()
     return sum(a.elapsed_time(b) for a, b in ev) / iters
+
+
+def max_over_ranks(value, dist, device):
+    """Maximum of a per-rank scalar over all ranks (identity when not distributed)."""
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
 
 
 def oracle_one_request(w, workloads, oracle, i):
@@ -322,11 +330,9 @@ def main():
         torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
     assert job.bc.device_status() == 0
-    t = torch.tensor([step_ms], dtype=torch.float64, device="cuda")
+    step_ms_max = max_over_ranks(step_ms, dist, "cuda")
     if dist is not None:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
         dist.barrier()
-    step_ms_max = float(t.item())
     value = world * w.suffix_tokens / (step_ms_max * 1e-3)
 
     # ---- per-call timing for the roofline (CUDA events around the single kernel launch) ------
@@ -380,10 +386,7 @@ def main():
         torch.cuda.synchronize()
         n_e2e = max(3, min(args.steps, 10))
         e2e_ms = time_call(e2e_step, n_e2e, flush)
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        if dist is not None:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+        e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
         h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hv))
         d2h = ho.numel() * ho.element_size() * (2 if ho2 is not None else 1)
         e2e = {"value": world * w.suffix_tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
