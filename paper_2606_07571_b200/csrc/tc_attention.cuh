@@ -13,10 +13,10 @@
 // the result exact.
 //
 // Roles: warps 0-3 softmax/correction/epilogue of tile A, warps 4-7 of tile B (one thread per
-// row), warp 8 MMA issue and TMEM ownership, warps 9-10 loads.  The whole SM is bound by
-// instruction issue, so the softmax uses packed fp32 instructions, 3-input maxima and as few
-// instructions per score as possible; MMAs are issued branch-free by an elected lane.  All waits are bounded; a wait that gives up raises a sticky status word and
-// the CTA drains and exits.
+// row), warp 8 MMA issue and TMEM ownership, warps 9-10 loads.  The softmax uses packed fp32
+// instructions and 3-input maxima; MMAs are issued branch-free by an elected lane of a converged
+// warp.  All waits are bounded; a wait that gives up raises a sticky status word and the CTA
+// drains and exits.
 #pragma once
 #include <cuda_bf16.h>
 #include "common.cuh"
@@ -401,6 +401,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       tmem_wait_ld();
       tmem_ld32(tmem_s + 64, r + 64);
       tmem_ld32(tmem_s + 96, r + 96);
+      if (tid == 0) BICACHE_STAMP(0, ti);
       float alpha = 1.f;
       unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
       bool stored = false;                                   // P already stored and signalled
@@ -424,6 +425,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
           mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
         }
         const float mx = fmaxf(mx0, mx1) * sl2;              // scale > 0
+        if (tid == 0) BICACHE_STAMP(0, ti);
         if (!__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
@@ -450,10 +452,12 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
               r[2 * i] = pack_bf16(p0, p1);
               r[2 * i + 1] = pack_bf16(p2, p3);
             }
+            if (tid == 0) BICACHE_STAMP(0, ti);
             tmem_st32(tmem_s + half * 32, r + half * 32);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(smem_u32(&bars->p_half[X][half]));
+            if (tid == 0) BICACHE_STAMP(0, ti);
           }
           stored = true;
         } else {
@@ -540,8 +544,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
           r[2 * i + 1] = pack_bf16(p2, p3);
         }
       }
-      if (tid == 0) BICACHE_STAMP(0, ti);
-      if (tid == 0) BICACHE_STAMP(0, ti);
       if (!stored) {
         tmem_st32(tmem_s, r);
         tmem_st32(tmem_s + 32, r + 32);
@@ -550,7 +552,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         mbar_arrive(smem_u32(&bars->p_half[X][0]));
         mbar_arrive(smem_u32(&bars->p_half[X][1]));
       }
-      if (tid == 0) BICACHE_STAMP(0, ti);
       {
         float s0, s1, s2, s3;
         unpack2(acc_a, s0, s1);
@@ -719,102 +720,79 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
     // instruction: descriptor arithmetic then stays in the uniform datapath and the MMAs can be
     // issued back to back (a single diverged lane cannot feed the tensor pipe fast enough).
     if (!dead && T > 0) {
-      const unsigned tmem_sa = tmem, tmem_sb = tmem + 128, tmem_oa = tmem + 256, tmem_ob = tmem + 384;
-      const unsigned long long qa_desc = make_desc(q_smem, 16, 2048);
-      const unsigned long long qb_desc = make_desc(q_smem + kTileBytes, 16, 2048);
+      const unsigned tmem_s2[2] = {tmem, tmem + 128};
+      const unsigned tmem_o2[2] = {tmem + 256, tmem + 384};
+      const unsigned long long q_desc[2] = {make_desc(q_smem, 16, 2048), make_desc(q_smem + kTileBytes, 16, 2048)};
+      const int nx = b_active ? 2 : 1;
       bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_full), 0, abort_flag));
       int ti = 0; (void)ti;
       if (lane == 0) BICACHE_STAMP(1, ti);
-      int prev_ksteps = 0;
+      // Issue order: S_A(0) S_B(0) | O_A(0) S_A(1) | O_B(0) S_B(1) | O_A(1) S_A(2) | ...
+      // O_X(j) += P_X V is issued in two halves as P arrives, and S_X(j+1) = Q_X K^T follows it
+      // back to back (it overwrites P_X; the tensor pipe runs MMAs in issue order).  The K/V tiles
+      // an iteration needs are waited for before the wait on P, so nothing stands between the
+      // arrival of P and the MMAs.
+      // prologue: S_X(0)
+      ok = ok && __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[0]), 0, abort_flag));
+      if (ok) {
+        fence_proxy_async();
+        tc_fence_after();
+        const unsigned long long k_desc = make_desc(ring_smem, 16, 2048);
+        for (int x = 0; x < nx; ++x) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const unsigned off = (k >> 2) * 64 + (k & 3) * 2;
+            mma_ss_elect(tmem_s2[x], q_desc[x] + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
+          }
+          mma_commit_elect(smem_u32(&bars->s_full[x]));
+        }
+        mma_commit_elect(smem_u32(&bars->free_[0]));
+      }
       for (int j = 0; j < T && ok; ++j) {
         const int jg = tile_begin + j;
         const int cnt = jg < prefix_tiles ? min(kTileKeys, req.m - jg * kTileKeys)
                                           : min(kTileKeys, req.n - (jg - prefix_tiles) * kTileKeys);
         const int ksteps = (cnt + 15) >> 4;
-        const int uk = 2 * j, uv = 2 * j + 1;
-        const int slot_k = uk % kRing, slot_v = uv % kRing;
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_k]), (uk / kRing) & 1, abort_flag));
-        if (!ok) break;
-        if (lane == 0) BICACHE_STAMP(1, ti);
-        fence_proxy_async();
-        tc_fence_after();
-        // The descriptor's address field counts 16-byte units: a K step of 16 dims is +2, the second
-        // 64-dim half +64.
-        const unsigned long long k_desc = make_desc(ring_smem + slot_k * kTileBytes, 16, 2048);
-        // S_A = Q_A K^T.  It overwrites P_A of the previous key tile; the tensor pipe runs MMAs in
-        // issue order, so O_A += P_A V (issued earlier) has read P_A before this writes.
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-          const unsigned off = (k >> 2) * 64 + (k & 3) * 2;
-          mma_ss_elect(tmem_sa, qa_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
-        }
-        mma_commit_elect(smem_u32(&bars->s_full[0]));
-        if (lane == 0) BICACHE_STAMP(1, ti);
-        if (b_active) {
-          if (j > 0) {
-            // O_B += P_B V of the previous key tile
-            const int pv = 2 * (j - 1) + 1, pslot = pv % kRing;
-            const unsigned long long v_desc = make_desc(ring_smem + pslot * kTileBytes, 1024, 2048);
-            const unsigned acc0 = j > 1 ? 1u : 0u;
-#pragma unroll
-            for (int half = 0; half < 2 && ok; ++half) {
-              ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[1][half]), (j - 1) & 1, abort_flag));
-              if (!ok) break;
-              tc_fence_after();
-#pragma unroll
-              for (int k = half * 4; k < half * 4 + 4; ++k)
-                mma_ts_elect(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
-                             k < prev_ksteps ? 1u : 0u);
-            }
-            if (!ok) break;
-            mma_commit_elect(smem_u32(&bars->free_[pslot]));
-          }
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const unsigned off = (k >> 2) * 64 + (k & 3) * 2;
-            mma_ss_elect(tmem_sb, qb_desc + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
-          }
-          mma_commit_elect(smem_u32(&bars->s_full[1]));
-        }
-        mma_commit_elect(smem_u32(&bars->free_[slot_k]));
-        if (lane == 0) BICACHE_STAMP(1, ti);
-        // O_A += P_A V
+        const int uv = 2 * j + 1, un = 2 * j + 2;          // ring uses: V of tile j, K of tile j + 1
+        const int slot_v = uv % kRing, slot_n = un % kRing;
+        const bool more = j + 1 < T;
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_v]), (uv / kRing) & 1, abort_flag));
+        if (ok && more)
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_n]), (un / kRing) & 1, abort_flag));
         if (!ok) break;
         fence_proxy_async();
         const unsigned long long v_desc = make_desc(ring_smem + slot_v * kTileBytes, 1024, 2048);
+        const unsigned long long k_desc = make_desc(ring_smem + slot_n * kTileBytes, 16, 2048);
         const unsigned acc0 = j > 0 ? 1u : 0u;
+        for (int x = 0; x < nx && ok; ++x) {
+          // O_X += P_X V, 16 keys (one page image) per MMA; P is the A operand, read from TMEM
 #pragma unroll
-        for (int half = 0; half < 2 && ok; ++half) {
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[0][half]), j & 1, abort_flag));
+          for (int half = 0; half < 2; ++half) {
+            ok = ok && __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[x][half]), j & 1, abort_flag));
+            if (ok) {
+              if (lane == 0 && x == 0 && half == 0) BICACHE_STAMP(1, ti);
+              tc_fence_after();
+#pragma unroll
+              for (int k = half * 4; k < half * 4 + 4; ++k)
+                mma_ts_elect(tmem_o2[x], tmem_s2[x] + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV,
+                             k > 0 ? 1u : acc0, k < ksteps ? 1u : 0u);
+            }
+          }
           if (!ok) break;
-          if (lane == 0 && half == 0) BICACHE_STAMP(1, ti);
-          tc_fence_after();
+          // S_X of the next key tile
+          if (more) {
 #pragma unroll
-          for (int k = half * 4; k < half * 4 + 4; ++k)
-            mma_ts_elect(tmem_oa, tmem_sa + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
-                         k < ksteps ? 1u : 0u);
+            for (int k = 0; k < 8; ++k) {
+              const unsigned off = (k >> 2) * 64 + (k & 3) * 2;
+              mma_ss_elect(tmem_s2[x], q_desc[x] + off, k_desc + off, kIdescQK, k > 0 ? 1u : 0u);
+            }
+            mma_commit_elect(smem_u32(&bars->s_full[x]));
+          }
+          if (lane == 0 && x == 0) BICACHE_STAMP(1, ti);
         }
         if (!ok) break;
-        if (!b_active) mma_commit_elect(smem_u32(&bars->free_[slot_v]));
-        if (lane == 0) BICACHE_STAMP(1, ti);
-        prev_ksteps = ksteps;
-      }
-      if (ok && b_active) {
-        const int pv = 2 * (T - 1) + 1, pslot = pv % kRing;
-        const unsigned long long v_desc = make_desc(ring_smem + pslot * kTileBytes, 1024, 2048);
-        const unsigned acc0 = T > 1 ? 1u : 0u;
-#pragma unroll
-        for (int half = 0; half < 2 && ok; ++half) {
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[1][half]), (T - 1) & 1, abort_flag));
-          if (!ok) break;
-          tc_fence_after();
-#pragma unroll
-          for (int k = half * 4; k < half * 4 + 4; ++k)
-            mma_ts_elect(tmem_ob, tmem_sb + k * 8, v_desc + k * (kPageBytes >> 4), kIdescPV, k > 0 ? 1u : acc0,
-                         k < prev_ksteps ? 1u : 0u);
-        }
-        if (ok) mma_commit_elect(smem_u32(&bars->free_[pslot]));
+        mma_commit_elect(smem_u32(&bars->free_[slot_v]));
+        if (more) mma_commit_elect(smem_u32(&bars->free_[slot_n]));
       }
       if (ok) mma_commit_elect(smem_u32(&bars->o_done));
       // Whatever happened, let every MMA issued so far finish before TMEM is released.
