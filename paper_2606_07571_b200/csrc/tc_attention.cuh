@@ -13,7 +13,7 @@
 // the result exact.
 //
 // Roles: warps 0-3 softmax/correction/epilogue of tile A, warps 4-7 of tile B (one thread per
-// row), warp 8 MMA issue and TMEM ownership, warps 9-10 loads.  The softmax uses packed fp32
+// row), warp 8 MMA issue and TMEM ownership, warps 9-11 loads.  The softmax uses packed fp32
 // instructions and 3-input maxima; MMAs are issued branch-free by an elected lane of a converged
 // warp.  All waits are bounded; a wait that gives up raises a sticky status word and the CTA
 // drains and exits.
@@ -33,7 +33,7 @@ constexpr int kPageBytes = 4096;
 constexpr int kRing = 4;                         // K/V ring slots of one tile each: K0 V0 K1 V1
 constexpr int kThreads = 384;
 constexpr int kGroupThreads = 128;               // softmax threads of one query tile (one per row)
-constexpr int kLoadThreads = 64;
+constexpr int kLoadThreads = 32;                 // one warp loads a whole tile
 constexpr int kSoftmaxRegs = 208;                // registers per thread after setmaxnreg
 constexpr int kOtherRegs = 80;
 constexpr int kMmaWarp = 8;
@@ -339,7 +339,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
 
   if (tid == 0) {
     bars->abort_flag = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
-    mbar_init(smem_u32(&bars->q_full), kLoadThreads);
+    mbar_init(smem_u32(&bars->q_full), 64);               // the two warps that fetch Q_A and Q_B
     for (int i = 0; i < kRing; ++i) {
       mbar_init(smem_u32(&bars->full[i]), kLoadThreads);
       mbar_init(smem_u32(&bars->free_[i]), 1);
@@ -617,48 +617,51 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       }
     }
     tc_fence_before();
-  } else if (warp == 9 || warp == 10) {
+  } else if (warp >= 9) {
     // ====================================== loads =======================================
-    const int lt = tid - 9 * 32;                      // 0..63
-    // A 128-row tile is fetched as 16 passes of 8 rows: thread lt takes 16-byte chunk (lt & 15) of
-    // rows (lt >> 4) + 8 i and (lt >> 4) + 4 + 8 i.  In the tile image those chunks sit 2048 bytes
-    // after the ones of pass i-1.
-    const int r0 = lt >> 4, c16 = lt & 15;
-    const unsigned dst_a = tile_chunk_offset(r0, c16), dst_b = tile_chunk_offset(r0 + 4, c16);
+    // Three load warps, each responsible for whole tiles: warp w takes ring uses u = w, w + 3, ...
+    // (u = 2 j: K of key tile j, u = 2 j + 1: V of key tile j).  A warp issues its tile, waits for
+    // it to land, fences and signals, while the other two warps are already issuing theirs.
+    const int w = warp - 9;
+    // A 128-row tile is fetched as 64 passes of 2 rows: lane l takes 16-byte chunk (l & 15) of rows
+    // (l >> 4) + 2 i.  In the tile image, rows r, r + 8, r + 16, ... are 2048 bytes apart.
+    const int r0 = lane >> 4, c16 = lane & 15;
+    unsigned dst_q[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) dst_q[q] = tile_chunk_offset(r0 + 2 * q, c16);
     bool ok = !dead;
-    if (ok) {
-      // Q tiles: packed rows (token, head within the KV group); rows past the end are zero-filled
-      for (int x = 0; x < (b_active ? 2 : 1); ++x) {
+    bool q_pending = false;
+    if (ok && w < 2) {
+      // Q tiles (warp 0: A, warp 1: B): packed rows (token, head within the KV group); rows past
+      // the end are zero-filled
+      if (w == 0 || b_active) {
 #pragma unroll 4
-        for (int i = 0; i < 32; ++i) {
-          const int prow = item.row0 + x * 128 + r0 + 4 * i;
+        for (int i = 0; i < 64; ++i) {
+          const int prow = item.row0 + w * 128 + r0 + 2 * i;
           const bool valid = prow < packed_rows;
           const int a = valid ? prow / G : 0;
           const int h = item.kv_head * G + (valid ? prow - a * G : 0);
           const char* src = t.q + ((req.row_off + a) * t.q_stride + (long long)h * 128) * 2 + c16 * 16;
-          cp_async16(q_smem + x * kTileBytes + ((i & 1) ? dst_b : dst_a) + (i >> 1) * 2048, src, valid ? 16u : 0u);
+          cp_async16(q_smem + w * kTileBytes + dst_q[i & 3] + (i >> 2) * 2048, src, valid ? 16u : 0u);
         }
       }
-      cp_async_commit();                              // lands while the first K/V loads are issued
+      cp_async_commit();                              // lands while the first K/V tile is issued
+      q_pending = true;
     }
-    bool q_pending = ok;
     const int* pages = s.pages + req.page_off;
-    int pending = -1;                                 // ring slot whose cp.async group is in flight
-    int ti = 0; (void)ti;
-    for (int u = 0; u < 2 * T && ok; ++u) {           // u = 2 j: K of tile j, u = 2 j + 1: V of tile j
+    for (int u = w; u < 2 * T && ok; u += 3) {
       const int slot = u % kRing;
       const int jg = tile_begin + (u >> 1);
       const bool is_v = u & 1;
       ok = mbar_wait(smem_u32(&bars->free_[slot]), ((u / kRing) & 1) ^ 1, abort_flag);
       if (!ok) break;
-      if (lt == 0) BICACHE_STAMP(2, ti);
       const unsigned dst = ring_smem + slot * kTileBytes;
       const unsigned full = smem_u32(&bars->full[slot]);
       if (jg < prefix_tiles) {
         // cached prefix tile: one bulk copy per page; a pool page already is the tile image
         const int cnt = min(kTileKeys, req.m - jg * kTileKeys);
         const int npages = (cnt + kPageSize - 1) / kPageSize;
-        if (lt == 0) {
+        if (lane == 0) {
           const char* pool_base = is_v ? pool.v : pool.k;
           mbar_arrive_expect_tx(full, (unsigned)(npages * kPageBytes));
           for (int pg = 0; pg < npages; ++pg)
@@ -668,12 +671,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         } else {
           mbar_arrive(full);
         }
-        if (q_pending) {
-          cp_async_wait<0>();
-          fence_proxy_async();
-          mbar_arrive(smem_u32(&bars->q_full));
-          q_pending = false;
-        }
       } else {
         // own rows: 16-byte gathers from row-major K/V into the image, zero-filled past the end
         const int key0 = (jg - prefix_tiles) * kTileKeys;
@@ -682,35 +679,44 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
                            ((req.row_off + key0) * t.kv_stride + (long long)item.kv_head * 128) * 2 + c16 * 16;
         const long long row_bytes = t.kv_stride * 2;
         const char* src = row0 + r0 * row_bytes;
+#ifdef BICACHE_SKIP_LOADS
+        if (false)
+#endif
 #pragma unroll 4
-        for (int i = 0; i < 16; ++i) {
-          const bool va = r0 + 8 * i < cnt, vb = r0 + 4 + 8 * i < cnt;
-          cp_async16(dst + dst_a + i * 2048, va ? src : row0, va ? 16u : 0u);
-          cp_async16(dst + dst_b + i * 2048, vb ? src + 4 * row_bytes : row0, vb ? 16u : 0u);
-          src += 8 * row_bytes;
+        for (int i = 0; i < 64; ++i) {
+          const bool valid = r0 + 2 * i < cnt;
+          cp_async16(dst + dst_q[i & 3] + (i >> 2) * 2048, valid ? src : row0, valid ? 16u : 0u);
+          src += 2 * row_bytes;
         }
         cp_async_commit();
-        if (pending >= 0 || q_pending) {
-          cp_async_wait<1>();                         // everything but the tile just issued has landed
+        if (q_pending) {
+          cp_async_wait<1>();                         // the Q tile has landed
           fence_proxy_async();
-          if (q_pending) mbar_arrive(smem_u32(&bars->q_full));
-          if (pending >= 0) mbar_arrive(smem_u32(&bars->full[pending]));
+          mbar_arrive(smem_u32(&bars->q_full));
           q_pending = false;
         }
-        pending = slot;
+        cp_async_wait<0>();
+        fence_proxy_async();
+        mbar_arrive(full);
       }
-      if (lt == 0) BICACHE_STAMP(2, ti);
+      if (q_pending) {
+        cp_async_wait<0>();
+        fence_proxy_async();
+        mbar_arrive(smem_u32(&bars->q_full));
+        q_pending = false;
+      }
     }
     cp_async_wait<0>();
-    fence_proxy_async();
-    if (q_pending) mbar_arrive(smem_u32(&bars->q_full));
-    if (pending >= 0) mbar_arrive(smem_u32(&bars->full[pending]));
+    if (q_pending) {
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&bars->q_full));
+    }
     // On the normal path every tile loaded has been consumed by the time the CTA ends (the
     // epilogue waits for the last MMA).  After a give-up, bulk copies may still be in flight:
-    // wait (bounded) for the last barriers this thread armed.
-    if (!dead && (!ok || *abort_flag) && lt == 0) {
+    // wait (bounded) for the last barriers this lane armed.
+    if (!dead && (!ok || *abort_flag) && lane == 0) {
       for (int u = max(0, 2 * T - kRing); u < 2 * T; ++u)
-        if (tile_begin + (u >> 1) < prefix_tiles)
+        if (u % 3 == w && tile_begin + (u >> 1) < prefix_tiles)
           for (unsigned it = 0; it < 4096 && !mbar_try_wait(smem_u32(&bars->full[u % kRing]), (u / kRing) & 1); ++it)
             __nanosleep(256);
     }
@@ -739,6 +745,14 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         tc_fence_after();
         const unsigned long long k_desc = make_desc(ring_smem, 16, 2048);
         for (int x = 0; x < nx; ++x) {
+          if (x == 1) {
+            // Stagger the two query tiles by half a period: tile B starts when tile A's softmax is
+            // half done, so that afterwards each tile's softmax runs while the tensor pipe works for
+            // the other tile (started together, the two softmaxes share the exp unit and the MMAs
+            // of both tiles then queue behind each other).
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[0][0]), 0, abort_flag));
+            if (!ok) break;
+          }
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
             const unsigned off = (k >> 2) * 64 + (k & 3) * 2;
@@ -746,7 +760,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
           }
           mma_commit_elect(smem_u32(&bars->s_full[x]));
         }
-        mma_commit_elect(smem_u32(&bars->free_[0]));
+        if (ok) mma_commit_elect(smem_u32(&bars->free_[0]));
       }
       for (int j = 0; j < T && ok; ++j) {
         const int jg = tile_begin + j;
