@@ -323,6 +323,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
   const unsigned ring_smem = q_smem + 2 * kTileBytes;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef BICACHE_TRACE
+  if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1000] = clock64();
+#endif
   const WorkItem item = s.items[blockIdx.x];
   const ReqMeta req = s.reqs[item.req];
   const int G = t.Hq / t.Hkv;
@@ -339,7 +342,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
 
   if (tid == 0) {
     bars->abort_flag = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
-    mbar_init(smem_u32(&bars->q_full), 64);               // the two warps that fetch Q_A and Q_B
+    mbar_init(smem_u32(&bars->q_full), 256);              // the eight softmax warps fetch the Q tiles
     for (int i = 0; i < kRing; ++i) {
       mbar_init(smem_u32(&bars->full[i]), kLoadThreads);
       mbar_init(smem_u32(&bars->free_[i]), 1);
@@ -360,6 +363,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+#ifdef BICACHE_TRACE
+  if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1001] = clock64();
+#endif
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&bars->tmem_base);
   const bool dead = *abort_flag != 0;        // an earlier CTA already gave up: do no work
 
@@ -382,6 +388,36 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
     const bool active = !dead && (X == 0 || b_active);
     const float sl2 = t.scale * 1.4426950408889634f;         // scores are handled in the log2 domain
     const unsigned long long sl2_2 = pack2(sl2, sl2);
+    // Each softmax warp first fetches its own 32 rows of the Q tile (packed rows: token a, head jj
+    // within the KV group, p = a * G + jj; rows past the end are zero-filled): eight warps in
+    // parallel hide the DRAM latency of this cold read far better than one load warp could.
+    if (!dead) {
+      if (active) {
+        const int r0 = (warp & 3) * 32 + (lane >> 4), c16 = lane & 15;
+        int prow = item.row0 + X * 128 + r0;
+        const int a0 = prow / G;
+        int jj = prow - a0 * G;
+        const long long q_row_bytes = t.q_stride * 2;
+        const char* q_base = t.q + (req.row_off * t.q_stride + (long long)item.kv_head * G * 128) * 2 + c16 * 16;
+        const char* src_row = q_base + a0 * q_row_bytes;
+        const unsigned q_dst = q_smem + X * kTileBytes;
+#pragma unroll 4
+        for (int i = 0; i < 16; ++i) {
+          const bool valid = prow < packed_rows;
+          cp_async16(q_dst + tile_chunk_offset(r0 + 2 * i, c16), valid ? src_row + jj * 256 : q_base, valid ? 16u : 0u);
+          prow += 2;
+          jj += 2;
+          while (jj >= G) {                           // at most twice (G >= 1)
+            jj -= G;
+            src_row += q_row_bytes;
+          }
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        fence_proxy_async();
+      }
+      mbar_arrive(smem_u32(&bars->q_full));
+    }
     float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = active;
     int ti = 0; (void)ti;
@@ -568,6 +604,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->o_done), 0, abort_flag));
       if (ok) tc_fence_after();
     }
+#ifdef BICACHE_TRACE
+    if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1003] = clock64();
+#endif
     if (ok) {
       const float inv = T > 0 ? 1.f / l_sum : 0.f;
       const float lse = T > 0 ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
@@ -630,24 +669,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
 #pragma unroll
     for (int q = 0; q < 4; ++q) dst_q[q] = tile_chunk_offset(r0 + 2 * q, c16);
     bool ok = !dead;
-    bool q_pending = false;
-    if (ok && w < 2) {
-      // Q tiles (warp 0: A, warp 1: B): packed rows (token, head within the KV group); rows past
-      // the end are zero-filled
-      if (w == 0 || b_active) {
-#pragma unroll 4
-        for (int i = 0; i < 64; ++i) {
-          const int prow = item.row0 + w * 128 + r0 + 2 * i;
-          const bool valid = prow < packed_rows;
-          const int a = valid ? prow / G : 0;
-          const int h = item.kv_head * G + (valid ? prow - a * G : 0);
-          const char* src = t.q + ((req.row_off + a) * t.q_stride + (long long)h * 128) * 2 + c16 * 16;
-          cp_async16(q_smem + w * kTileBytes + dst_q[i & 3] + (i >> 2) * 2048, src, valid ? 16u : 0u);
-        }
-      }
-      cp_async_commit();                              // lands while the first K/V tile is issued
-      q_pending = true;
-    }
+    int ti = 0; (void)ti;
     const int* pages = s.pages + req.page_off;
     for (int u = w; u < 2 * T && ok; u += 3) {
       const int slot = u % kRing;
@@ -679,38 +701,29 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
                            ((req.row_off + key0) * t.kv_stride + (long long)item.kv_head * 128) * 2 + c16 * 16;
         const long long row_bytes = t.kv_stride * 2;
         const char* src = row0 + r0 * row_bytes;
-#ifdef BICACHE_SKIP_LOADS
-        if (false)
-#endif
+        if (cnt >= kTileKeys) {
+#pragma unroll 8
+          for (int i = 0; i < 64; ++i) {
+            cp_async16(dst + dst_q[i & 3] + (i >> 2) * 2048, src, 16u);
+            src += 2 * row_bytes;
+          }
+        } else {
 #pragma unroll 4
-        for (int i = 0; i < 64; ++i) {
-          const bool valid = r0 + 2 * i < cnt;
-          cp_async16(dst + dst_q[i & 3] + (i >> 2) * 2048, valid ? src : row0, valid ? 16u : 0u);
-          src += 2 * row_bytes;
+          for (int i = 0; i < 64; ++i) {
+            const bool valid = r0 + 2 * i < cnt;
+            cp_async16(dst + dst_q[i & 3] + (i >> 2) * 2048, valid ? src : row0, valid ? 16u : 0u);
+            src += 2 * row_bytes;
+          }
         }
         cp_async_commit();
-        if (q_pending) {
-          cp_async_wait<1>();                         // the Q tile has landed
-          fence_proxy_async();
-          mbar_arrive(smem_u32(&bars->q_full));
-          q_pending = false;
-        }
+        if (w == 0 && lane == 0) BICACHE_STAMP(2, ti);
         cp_async_wait<0>();
         fence_proxy_async();
         mbar_arrive(full);
-      }
-      if (q_pending) {
-        cp_async_wait<0>();
-        fence_proxy_async();
-        mbar_arrive(smem_u32(&bars->q_full));
-        q_pending = false;
+        if (w == 0 && lane == 0) BICACHE_STAMP(2, ti);
       }
     }
     cp_async_wait<0>();
-    if (q_pending) {
-      fence_proxy_async();
-      mbar_arrive(smem_u32(&bars->q_full));
-    }
     // On the normal path every tile loaded has been consumed by the time the CTA ends (the
     // epilogue waits for the last MMA).  After a give-up, bulk copies may still be in flight:
     // wait (bounded) for the last barriers this lane armed.
@@ -818,6 +831,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
   }
 
   __syncthreads();
+#ifdef BICACHE_TRACE
+  if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1002] = clock64();
+#endif
   if (warp == kMmaWarp) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
