@@ -634,21 +634,47 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         }
         if (row_valid) t.part_lse[pr] = lse;
       } else if (T > 0) {
-        char* orow = t.out + ((req.row_off + a) * t.out_stride + (long long)h * 128) * 2;
+        // Each thread holds one output row; a row-per-thread store would touch 32 rows per
+        // instruction.  Stage the warp's 32 rows (256 bytes each) in this warp's quarter of the Q
+        // tile's shared memory (Q is no longer needed) and write them out two whole rows per
+        // instruction.  Chunks are XOR-placed by row to keep both directions conflict-light.
+        unsigned char* stage = smem + X * kTileBytes + (warp & 3) * 8192;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
           unsigned o[32];
           tmem_ld32(tmem_o + c * 32, o);
           tmem_wait_ld();
-          if (row_valid) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              uint4 v4;
-              v4.x = pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
-              v4.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-              v4.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
-              v4.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
-              *reinterpret_cast<uint4*>(orow + (c * 32 + i) * 2) = v4;
+          for (int i = 0; i < 32; i += 8) {
+            uint4 v4;
+            v4.x = pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+            v4.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+            v4.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+            v4.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+            const int cc = c * 4 + (i >> 3);
+            *reinterpret_cast<uint4*>(stage + lane * 256 + ((cc ^ (lane & 15)) << 4)) = v4;
+          }
+        }
+        __syncwarp();
+        {
+          const int cc = lane & 15;
+          int row = lane >> 4;                                 // rows row, row + 2, ... of this warp
+          int prow2 = item.row0 + X * 128 + (warp & 3) * 32 + row;
+          const int a2 = prow2 / G;
+          int jj = prow2 - a2 * G;
+          const long long o_row_bytes = t.out_stride * 2;
+          char* dst_row = t.out + (req.row_off * t.out_stride + (long long)item.kv_head * G * 128) * 2 + cc * 16 +
+                          a2 * o_row_bytes;
+#pragma unroll 4
+          for (int it = 0; it < 16; ++it) {
+            const uint4 v4 = *reinterpret_cast<const uint4*>(stage + row * 256 + ((cc ^ (row & 15)) << 4));
+            if (prow2 < packed_rows) *reinterpret_cast<uint4*>(dst_row + jj * 256) = v4;
+            row += 2;
+            prow2 += 2;
+            jj += 2;
+            while (jj >= G) {
+              jj -= G;
+              dst_row += o_row_bytes;
             }
           }
         }
