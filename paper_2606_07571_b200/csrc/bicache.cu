@@ -342,11 +342,11 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   ctx->launches++;
   if (e != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
   if (c.num_splits > 1) {
-    const int grid = c.num_items / c.num_splits;
+    const int grid = c.num_items / c.num_splits * (kTileRows / kMergeRowsPerBlock);
     if (cfg.dtype == BICACHE_F32)
-      merge_partials_kernel<float><<<grid, kSimtWarps * 32, 0, stream>>>(sv, t);
+      merge_partials_kernel<float><<<grid, kMergeRowsPerBlock * 32, 0, stream>>>(sv, t);
     else
-      merge_partials_kernel<__nv_bfloat16><<<grid, kSimtWarps * 32, 0, stream>>>(sv, t);
+      merge_partials_kernel<__nv_bfloat16><<<grid, kMergeRowsPerBlock * 32, 0, stream>>>(sv, t);
     ctx->launches++;
     e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("merge launch: ") + cudaGetErrorString(e));

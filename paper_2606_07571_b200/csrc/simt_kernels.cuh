@@ -240,41 +240,54 @@ simt_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t) {
 // An empty part carries lse = -inf and weighs 0.  One block per split-0 work item, one warp per
 // packed row.
 // ---------------------------------------------------------------------------------------------
+constexpr int kMergeRowsPerBlock = 8;   // packed rows per block of the merge kernel (one warp each)
+
 template <typename T>
-__global__ void __launch_bounds__(kSimtWarps * 32)
+__global__ void __launch_bounds__(kMergeRowsPerBlock * 32)
 merge_partials_kernel(ScheduleView s, TensorArgs t) {
   using Tr = ElemTraits<T>;
   constexpr int kEsize = (int)sizeof(T);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const WorkItem item = s.items[blockIdx.x];       // the first num_items / num_splits items are split 0
+  // blockIdx.x enumerates (split-0 work item, group of kMergeRowsPerBlock packed rows); the first
+  // num_items / num_splits items of the schedule are the split-0 items.
+  constexpr int kBlocksPerItem = kTileRows / kMergeRowsPerBlock;
+  const WorkItem item = s.items[blockIdx.x / kBlocksPerItem];
   const ReqMeta req = s.reqs[item.req];
   const int G = t.Hq / t.Hkv;
   const int D = t.D;
-  const int row_end = min(item.row0 + kTileRows, req.n * G);
-  for (int p = item.row0 + warp; p < row_end; p += kSimtWarps) {
-    const int a = p / G;
-    const int h = item.kv_head * G + (p - a * G);
-    const long long pr0 = ((long long)req.tok_off + a) * t.Hq + h;
-    const long long split_stride = (long long)t.total_tokens * t.Hq;
-    float mx = -INFINITY;
-    for (int sp = 0; sp < s.num_splits; ++sp) mx = fmaxf(mx, t.part_lse[pr0 + sp * split_stride]);
-    float tot = 0.f;
-    for (int sp = 0; sp < s.num_splits; ++sp) tot += expf(t.part_lse[pr0 + sp * split_stride] - mx);
-    const bool any = mx > -INFINITY;
-    char* orow = t.out + ((req.row_off + a) * t.out_stride + (long long)h * D) * kEsize;
-    for (int d = lane; d < D; d += 32) {
-      float o = 0.f;
-      if (any) {
-        for (int sp = 0; sp < s.num_splits; ++sp) {
-          const float w = expf(t.part_lse[pr0 + sp * split_stride] - mx) / tot;
-          o = fmaf(w, t.part_o[(pr0 + sp * split_stride) * D + d], o);
-        }
-      }
-      Tr::store(orow + d * kEsize, o);
+  const int p = item.row0 + (blockIdx.x % kBlocksPerItem) * kMergeRowsPerBlock + warp;
+  if (p >= req.n * G) return;
+  const int a = p / G;
+  const int h = item.kv_head * G + (p - a * G);
+  const long long pr0 = ((long long)req.tok_off + a) * t.Hq + h;
+  const long long split_stride = (long long)t.total_tokens * t.Hq;
+  // lane sp holds the lse of split sp (+32, ...): maximum and total weight by shuffles
+  float mx = -INFINITY;
+  for (int sp = lane; sp < s.num_splits; sp += 32) mx = fmaxf(mx, t.part_lse[pr0 + sp * split_stride]);
+  mx = warp_max(mx);
+  float tot = 0.f;
+  for (int sp = lane; sp < s.num_splits; sp += 32) tot += expf(t.part_lse[pr0 + sp * split_stride] - mx);
+  tot = warp_sum(tot);
+  const bool any = mx > -INFINITY;
+  const float inv_tot = any ? 1.f / tot : 0.f;
+  char* orow = t.out + ((req.row_off + a) * t.out_stride + (long long)h * D) * kEsize;
+  float acc[kSimtMaxD / 32];
+#pragma unroll
+  for (int i = 0; i < kSimtMaxD / 32; ++i) acc[i] = 0.f;
+  if (any) {
+    for (int sp = 0; sp < s.num_splits; ++sp) {
+      const float w = expf(t.part_lse[pr0 + sp * split_stride] - mx) * inv_tot;
+      const float* po = t.part_o + (pr0 + sp * split_stride) * D;
+#pragma unroll
+      for (int i = 0; i < kSimtMaxD / 32; ++i)
+        if (lane + 32 * i < D) acc[i] = fmaf(w, po[lane + 32 * i], acc[i]);
     }
-    if (lane == 0 && t.lse != nullptr)
-      t.lse[(req.row_off + a) * t.Hq + h] = any ? mx + logf(tot) : -INFINITY;
   }
+#pragma unroll
+  for (int i = 0; i < kSimtMaxD / 32; ++i)
+    if (lane + 32 * i < D) Tr::store(orow + (lane + 32 * i) * kEsize, acc[i]);
+  if (lane == 0 && t.lse != nullptr)
+    t.lse[(req.row_off + a) * t.Hq + h] = any ? mx + logf(tot) : -INFINITY;
 }
 
 }  // namespace bicache
