@@ -429,14 +429,13 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       if (!ok) break;
       tc_fence_after();
       if (tid == 0) BICACHE_STAMP(0, ti);
-      // S of keys 0-63 first; the load of keys 64-127 is issued right after and lands while the
-      // first half is processed.
+      // the whole row of S into registers: four loads in flight, one wait
       unsigned r[128];
       tmem_ld32(tmem_s, r);
       tmem_ld32(tmem_s + 32, r + 32);
-      tmem_wait_ld();
       tmem_ld32(tmem_s + 64, r + 64);
       tmem_ld32(tmem_s + 96, r + 96);
+      tmem_wait_ld();
       if (tid == 0) BICACHE_STAMP(0, ti);
       float alpha = 1.f;
       unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
@@ -449,52 +448,57 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
         // warp before anything is handed over), the tile is redone below with the new reference.
         const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
         float mx0 = -INFINITY, mx1 = -INFINITY;
+        // first half of the exponentials, with the maximum over all 128 scores computed alongside
+        // (independent instructions that fill the exp unit's latency)
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
           mx0 = max3(mx0, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
           mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
-        }
-        tmem_wait_ld();
-#pragma unroll
-        for (int i = 16; i < 32; ++i) {
-          mx0 = max3(mx0, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
-          mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+          mx0 = max3(mx0, __uint_as_float(r[64 + 4 * i]), __uint_as_float(r[64 + 4 * i + 1]));
+          mx1 = max3(mx1, __uint_as_float(r[64 + 4 * i + 2]), __uint_as_float(r[64 + 4 * i + 3]));
+          const unsigned long long xa =
+              fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+          const unsigned long long xb =
+              fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+          float xa0, xa1, xb0, xb1;
+          unpack2(xa, xa0, xa1);
+          unpack2(xb, xb0, xb1);
+          const float p0 = ex2(xa0), p1 = ex2(xa1), p2 = ex2(xb0), p3 = ex2(xb1);
+          acc_a = add2(acc_a, pack2(p0, p1));
+          acc_b = add2(acc_b, pack2(p2, p3));
+          r[2 * i] = pack_bf16(p0, p1);
+          r[2 * i + 1] = pack_bf16(p2, p3);
         }
         const float mx = fmaxf(mx0, mx1) * sl2;              // scale > 0
         if (tid == 0) BICACHE_STAMP(0, ti);
         if (!__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+          if (tid == 0) BICACHE_STAMP(0, ti);
+          tmem_st32(tmem_s, r);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(smem_u32(&bars->p_half[X][0]));
+          if (tid == 0) BICACHE_STAMP(0, ti);
 #pragma unroll
-          for (int half = 0; half < 2; ++half) {
-#pragma unroll
-            for (int i = half * 16; i < half * 16 + 16; ++i) {
-              const unsigned long long xa =
-                  fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
-              const unsigned long long xb =
-                  fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
-              float xa0, xa1, p0, p1, p2, p3;
-              unpack2(xa, xa0, xa1);
-              p0 = ex2(xa0);
-              p1 = ex2(xa1);
-              if (kPolyPeriod > 0 && (i % (kPolyPeriod > 0 ? kPolyPeriod : 1)) == 0) {
-                ex2_poly2(xb, p2, p3);
-              } else {
-                float xb0, xb1;
-                unpack2(xb, xb0, xb1);
-                p2 = ex2(xb0);
-                p3 = ex2(xb1);
-              }
-              acc_a = add2(acc_a, pack2(p0, p1));
-              acc_b = add2(acc_b, pack2(p2, p3));
-              r[2 * i] = pack_bf16(p0, p1);
-              r[2 * i + 1] = pack_bf16(p2, p3);
-            }
-            if (tid == 0) BICACHE_STAMP(0, ti);
-            tmem_st32(tmem_s + half * 32, r + half * 32);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(smem_u32(&bars->p_half[X][half]));
-            if (tid == 0) BICACHE_STAMP(0, ti);
+          for (int i = 16; i < 32; ++i) {
+            const unsigned long long xa =
+                fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+            const unsigned long long xb =
+                fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+            float xa0, xa1, xb0, xb1;
+            unpack2(xa, xa0, xa1);
+            unpack2(xb, xb0, xb1);
+            const float p0 = ex2(xa0), p1 = ex2(xa1), p2 = ex2(xb0), p3 = ex2(xb1);
+            acc_a = add2(acc_a, pack2(p0, p1));
+            acc_b = add2(acc_b, pack2(p2, p3));
+            r[2 * i] = pack_bf16(p0, p1);
+            r[2 * i + 1] = pack_bf16(p2, p3);
           }
+          if (tid == 0) BICACHE_STAMP(0, ti);
+          tmem_st32(tmem_s + 32, r + 32);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(smem_u32(&bars->p_half[X][1]));
+          if (tid == 0) BICACHE_STAMP(0, ti);
           stored = true;
         } else {
           // redo with the new reference: S is still intact in TMEM
@@ -518,6 +522,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
             }
           }
           acc_a = pack2(ps, 0.f);
+          acc_b = pack2(0.f, 0.f);
           // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
@@ -531,7 +536,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status) {
       } else {
         // First tile of the item, or a ragged tile: maximum first, every exponential on the exp
         // unit so that masked columns give exactly 0.
-        tmem_wait_ld();
         if (cnt < kTileKeys) {
 #pragma unroll
           for (int i = 0; i < 128; ++i)
