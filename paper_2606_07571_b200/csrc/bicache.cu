@@ -13,6 +13,7 @@
 #include <unordered_map>
 #include <vector>
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
@@ -126,6 +127,37 @@ PoolView pool_view(const bicache_ctx* ctx) {
   p.layer_bytes = (long long)ctx->cfg.num_pages * ctx->cfg.num_kv_heads * p.page_bytes;
   p.swizzled = ctx->swizzled ? 1 : 0;
   return p;
+}
+
+// cuTensorMapEncodeTiled, fetched through the runtime so that the library does not link libcuda.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor [rows][heads][128] with `row_stride` elements between rows; box = (64 dims, box_heads,
+// box_rows), 128-byte swizzle, zero fill outside.
+bool encode_map(CUtensorMap* m, const void* base, long long rows, int heads, long long row_stride, int box_heads,
+                int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[3] = {128, (cuuint64_t)heads, (cuuint64_t)rows};
+  const cuuint64_t strides[2] = {256, (cuuint64_t)row_stride * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_heads, (cuuint32_t)box_rows};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // Build (or find) the device-resident schedule for this batch.  Returns the slot index or -1.
@@ -331,7 +363,18 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   const bool use_tensor = ctx->tensor_ok && ctx->path != BICACHE_PATH_SIMT && softmax_scale > 0.f;
   cudaError_t e;
   if (use_tensor) {
-    e = launch_tc_attention(sv, pool, t, ctx->d_status, stream);
+    // rows the tensors are known to have: up to the end of the last request
+    long long rows_total = 0;
+    for (int i = 0; i < R; ++i) rows_total = std::max<long long>(rows_total, row_off[i] + seqlen[i]);
+    const int G = cfg.num_q_heads / cfg.num_kv_heads;
+    TcTensorMaps maps;
+    maps.q_tma = (128 % G == 0) ? 1 : 0;
+    bool okm = encode_map(&maps.k, k, rows_total, cfg.num_kv_heads, kv_row_stride, 1, 128) &&
+               encode_map(&maps.v, v, rows_total, cfg.num_kv_heads, kv_row_stride, 1, 128) &&
+               encode_map(&maps.q, q, rows_total, cfg.num_q_heads, q_row_stride, maps.q_tma ? G : 1,
+                          maps.q_tma ? 128 / G : 128);
+    if (!okm) return fail(ctx, BICACHE_ERR_CUDA, "tensor map encoding failed");
+    e = launch_tc_attention(sv, pool, t, ctx->d_status, ctx->sm_count, maps, stream);
   } else if (cfg.dtype == BICACHE_F32) {
     simt_attention_kernel<float><<<c.num_items, kSimtWarps * 32, 0, stream>>>(sv, pool, t);
     e = cudaGetLastError();
