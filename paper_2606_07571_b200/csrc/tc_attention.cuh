@@ -46,20 +46,18 @@ constexpr long long kWaitCycles = 400000000LL;   // bounded waits: about 0.2 s o
 
 // shared-memory layout (dynamic, 1024-byte aligned by hand): Q_A, Q_B, ring, barriers
 struct alignas(8) Barriers {
-  unsigned long long q_full;             // the item's Q tiles are in shared memory
-  unsigned long long q_free;             // the last S of the item has been computed: Q may be replaced
+  unsigned long long q_full;
   unsigned long long full[kRing];        // ring slot holds its tile
   unsigned long long free_[kRing];       // the MMAs reading the slot have completed
   unsigned long long s_full[2];          // S = Q K^T of the current key tile is in TMEM (per query tile)
   unsigned long long p_half[2][2];       // P of keys 0-63 / 64-127 is in TMEM and O is rescaled (per query tile)
   unsigned long long o_done;             // every MMA of the item has completed
-  unsigned long long o_free[2];          // the epilogue has read O (per query tile)
   unsigned long long drain;
   unsigned tmem_base;
   int abort_flag;
 };
 constexpr int kTmemCols = 512;           // S_A 0-127, S_B 128-255 (P over the first 64 of each), O_A 256-383, O_B 384-511
-constexpr int kSmemBytes = 1024 + kTileBytes * (3 + kRing) + (int)sizeof(Barriers) + 64;   // Q_A Q_B, ring, output staging
+constexpr int kSmemBytes = 1024 + kTileBytes * (2 + kRing) + (int)sizeof(Barriers) + 64;
 
 // ----- raw PTX wrappers --------------------------------------------------------------------
 __device__ __forceinline__ unsigned smem_u32(const void* p) {
@@ -320,38 +318,8 @@ __device__ long long g_trace[3 * 1024];
 #define BICACHE_STAMP(role, idx) do { } while (0)
 #endif
 
-// Geometry of one work item, derived by every role from the schedule.
-struct ItemGeom {
-  WorkItem item;
-  ReqMeta req;
-  int prefix_tiles, tile_begin, T, packed_rows;
-  bool b_active;
-};
-__device__ __forceinline__ ItemGeom load_geom(const ScheduleView& s, int G, int it) {
-  ItemGeom g;
-  g.item = s.items[it];
-  g.req = s.reqs[g.item.req];
-  g.prefix_tiles = (g.req.m + kTileKeys - 1) / kTileKeys;
-  const int all_tiles = g.prefix_tiles + (g.req.n + kTileKeys - 1) / kTileKeys;
-  int tile_end = all_tiles;
-  g.tile_begin = 0;
-  if (s.num_splits > 1) {
-    g.tile_begin = min(all_tiles, g.item.split * s.tiles_per_split);
-    tile_end = min(all_tiles, g.tile_begin + s.tiles_per_split);
-  }
-  g.T = tile_end - g.tile_begin;
-  g.packed_rows = g.req.n * G;
-  g.b_active = g.item.row0 + 128 < g.packed_rows;        // the item has a second query tile
-  return g;
-}
-
 }  // namespace tc
 
-// Persistent kernel: one CTA per SM walks the work items blockIdx.x, blockIdx.x + gridDim.x, ...
-// All barriers keep their phases across items (every role counts its own uses), TMEM is allocated
-// once, and the load warps run ahead into the next item (its Q tiles as soon as the last S of the
-// current item has been issued, its K/V tiles as ring slots free up), so the prologue of an item
-// hides behind the tail and the epilogue of the previous one.
 __global__ void __launch_bounds__(tc::kThreads, 1)
 tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
                     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -360,19 +328,32 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  Barriers* bars = reinterpret_cast<Barriers*>(smem + kTileBytes * (3 + kRing));
+  Barriers* bars = reinterpret_cast<Barriers*>(smem + kTileBytes * (2 + kRing));
   volatile int* abort_flag = &bars->abort_flag;
   const unsigned q_smem = smem_u32(smem);                  // Q_A, then Q_B
   const unsigned ring_smem = q_smem + 2 * kTileBytes;
-  unsigned char* stage_smem = smem + kTileBytes * (2 + kRing);       // 32 KB: output staging
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef BICACHE_TRACE
+  if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1000] = clock64();
+#endif
+  const WorkItem item = s.items[blockIdx.x];
+  const ReqMeta req = s.reqs[item.req];
   const int G = t.Hq / t.Hkv;
+  const int prefix_tiles = (req.m + kTileKeys - 1) / kTileKeys;
+  const int all_tiles = prefix_tiles + (req.n + kTileKeys - 1) / kTileKeys;
+  int tile_begin = 0, tile_end = all_tiles;
+  if (s.num_splits > 1) {
+    tile_begin = min(all_tiles, item.split * s.tiles_per_split);
+    tile_end = min(all_tiles, tile_begin + s.tiles_per_split);
+  }
+  const int T = tile_end - tile_begin;
+  const int packed_rows = req.n * G;
+  const bool b_active = item.row0 + 128 < packed_rows;     // the item has a second query tile
 
   if (tid == 0) {
     bars->abort_flag = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
-    mbar_init(smem_u32(&bars->q_full), 64);               // the two load warps that fetch Q_A and Q_B
-    mbar_init(smem_u32(&bars->q_free), 1);
+    mbar_init(smem_u32(&bars->q_full), 256);              // the eight softmax warps fetch the Q tiles
     for (int i = 0; i < kRing; ++i) {
       mbar_init(smem_u32(&bars->full[i]), kLoadThreads);
       mbar_init(smem_u32(&bars->free_[i]), 1);
@@ -381,7 +362,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       mbar_init(smem_u32(&bars->s_full[i]), 1);
       mbar_init(smem_u32(&bars->p_half[i][0]), kGroupThreads);
       mbar_init(smem_u32(&bars->p_half[i][1]), kGroupThreads);
-      mbar_init(smem_u32(&bars->o_free[i]), kGroupThreads);
     }
     mbar_init(smem_u32(&bars->o_done), 1);
     mbar_init(smem_u32(&bars->drain), 1);
@@ -394,8 +374,11 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+#ifdef BICACHE_TRACE
+  if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1001] = clock64();
+#endif
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&bars->tmem_base);
-  const bool dead = *abort_flag != 0;        // an earlier launch or CTA already gave up: do no work
+  const bool dead = *abort_flag != 0;        // an earlier CTA already gave up: do no work
 
   // Registers move from the MMA/load warpgroup to the two softmax warpgroups, which hold a whole
   // row of S (128 values) per thread.  The counts must fit the CTA's launch allocation:
@@ -413,55 +396,117 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
     const unsigned lane_base = (unsigned)((warp & 3) * 32) << 16;
     const unsigned tmem_s = tmem + X * 128 + lane_base;      // S, and P written over its first 64 columns
     const unsigned tmem_o = tmem + 256 + X * 128 + lane_base;
+    const bool active = !dead && (X == 0 || b_active);
     const float sl2 = t.scale * 1.4426950408889634f;         // scores are handled in the log2 domain
     const unsigned long long sl2_2 = pack2(sl2, sl2);
-    unsigned tcnt = 0;                                       // key tiles this warpgroup has processed so far
-    int ti = 0; (void)ti;
-    bool ok = !dead;
-    for (int it = blockIdx.x, n_it = 0; it < s.num_items && ok; it += gridDim.x, ++n_it) {
-      const ItemGeom geo = load_geom(s, G, it);
-      const WorkItem item = geo.item;
-      const ReqMeta req = geo.req;
-      const int prefix_tiles = geo.prefix_tiles, tile_begin = geo.tile_begin, T = geo.T;
-      const int packed_rows = geo.packed_rows;
-      const bool active = X == 0 || geo.b_active;
-      float m_ref = -INFINITY, l_sum = 0.f;
-      for (int j = 0; j < T && active; ++j, ++tcnt) {
-        const int jg = tile_begin + j;
-        const int cnt = jg < prefix_tiles ? min(kTileKeys, req.m - jg * kTileKeys)
-                                          : min(kTileKeys, req.n - (jg - prefix_tiles) * kTileKeys);
-        const unsigned tpar = tcnt & 1;                      // phase parity of this stream's tile barriers
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_full[X]), tpar, abort_flag));
-        if (!ok) break;
-        tc_fence_after();
-        if (tid == 0) BICACHE_STAMP(0, ti);
-        // the whole row of S into registers: four loads in flight, one wait
-        unsigned r[128];
-        tmem_ld32(tmem_s, r);
-        tmem_ld32(tmem_s + 32, r + 32);
-        tmem_ld32(tmem_s + 64, r + 64);
-        tmem_ld32(tmem_s + 96, r + 96);
-        tmem_wait_ld();
-        if (tid == 0) BICACHE_STAMP(0, ti);
-        float alpha = 1.f;
-        unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
-        bool stored = false;                                   // P already stored and signalled
-        if (j > 0 && cnt >= kTileKeys) {
-          // Common case (a full tile after the first): the exponentials use the reference maximum of
-          // the earlier tiles and do not wait for this tile's maximum, which is computed alongside.
-          // P of the first 64 keys is handed to the tensor pipe before the second half is computed.
-          // If the row maximum turns out to exceed the reference by more than 2^8 (rare: checked per
-          // warp before anything is handed over), the tile is redone below with the new reference.
-          const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
-          float mx0 = -INFINITY, mx1 = -INFINITY;
-          // first half of the exponentials, with the maximum over all 128 scores computed alongside
-          // (independent instructions that fill the exp unit's latency)
-  #pragma unroll
+    // Each softmax warp first fetches its own 32 rows of the Q tile (packed rows: token a, head jj
+    // within the KV group, p = a * G + jj; rows past the end are zero-filled): eight warps in
+    // parallel hide the DRAM latency of this cold read far better than one load warp could.
+    if (!dead) {
+      if (q_tma) {
+        // 128 packed rows = 128 / G tokens x G heads of the KV group: one TMA box per 64-dim half,
+        // in the dense swizzled layout (row r at r * 128 bytes, halves 16 KB apart).  The first
+        // lane of each tile's first warp issues it; every softmax thread arrives.
+        if ((warp & 3) == 0 && lane == 0 && active) {
+          const unsigned qf = smem_u32(&bars->q_full);
+          const unsigned q_dst = q_smem + X * kTileBytes;
+          const int tok = (int)req.row_off + (item.row0 + X * 128) / G;
+          mbar_arrive_expect_tx(qf, (unsigned)kTileBytes);
+          tma_load_3d(q_dst, &tm_q, 0, item.kv_head * G, tok, qf);
+          tma_load_3d(q_dst + kTileBytes / 2, &tm_q, 64, item.kv_head * G, tok, qf);
+        } else {
+          mbar_arrive(smem_u32(&bars->q_full));
+        }
+      } else {
+        if (active) {
+          const int r0 = (warp & 3) * 32 + (lane >> 4), c16 = lane & 15;
+          int prow = item.row0 + X * 128 + r0;
+          const int a0 = prow / G;
+          int jj = prow - a0 * G;
+          const long long q_row_bytes = t.q_stride * 2;
+          const char* q_base = t.q + (req.row_off * t.q_stride + (long long)item.kv_head * G * 128) * 2 + c16 * 16;
+          const char* src_row = q_base + a0 * q_row_bytes;
+          const unsigned q_dst = q_smem + X * kTileBytes;
+#pragma unroll 4
           for (int i = 0; i < 16; ++i) {
-            mx0 = max3(mx0, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
-            mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
-            mx0 = max3(mx0, __uint_as_float(r[64 + 4 * i]), __uint_as_float(r[64 + 4 * i + 1]));
-            mx1 = max3(mx1, __uint_as_float(r[64 + 4 * i + 2]), __uint_as_float(r[64 + 4 * i + 3]));
+            const bool valid = prow < packed_rows;
+            cp_async16(q_dst + tile_chunk_offset(r0 + 2 * i, c16), valid ? src_row + jj * 256 : q_base, valid ? 16u : 0u);
+            prow += 2;
+            jj += 2;
+            while (jj >= G) {                         // at most twice (G >= 1)
+              jj -= G;
+              src_row += q_row_bytes;
+            }
+          }
+          cp_async_commit();
+          cp_async_wait<0>();
+          fence_proxy_async();
+        }
+        mbar_arrive(smem_u32(&bars->q_full));
+      }
+    }
+    float m_ref = -INFINITY, l_sum = 0.f;
+    bool ok = active;
+    int ti = 0; (void)ti;
+    for (int j = 0; j < T && active; ++j) {
+      const int jg = tile_begin + j;
+      const int cnt = jg < prefix_tiles ? min(kTileKeys, req.m - jg * kTileKeys)
+                                        : min(kTileKeys, req.n - (jg - prefix_tiles) * kTileKeys);
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_full[X]), j & 1, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      if (tid == 0) BICACHE_STAMP(0, ti);
+      // the whole row of S into registers: four loads in flight, one wait
+      unsigned r[128];
+      tmem_ld32(tmem_s, r);
+      tmem_ld32(tmem_s + 32, r + 32);
+      tmem_ld32(tmem_s + 64, r + 64);
+      tmem_ld32(tmem_s + 96, r + 96);
+      tmem_wait_ld();
+      if (tid == 0) BICACHE_STAMP(0, ti);
+      float alpha = 1.f;
+      unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
+      bool stored = false;                                   // P already stored and signalled
+      if (j > 0 && cnt >= kTileKeys) {
+        // Common case (a full tile after the first): the exponentials use the reference maximum of
+        // the earlier tiles and do not wait for this tile's maximum, which is computed alongside.
+        // P of the first 64 keys is handed to the tensor pipe before the second half is computed.
+        // If the row maximum turns out to exceed the reference by more than 2^8 (rare: checked per
+        // warp before anything is handed over), the tile is redone below with the new reference.
+        const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+        // first half of the exponentials, with the maximum over all 128 scores computed alongside
+        // (independent instructions that fill the exp unit's latency)
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          mx0 = max3(mx0, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
+          mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+          mx0 = max3(mx0, __uint_as_float(r[64 + 4 * i]), __uint_as_float(r[64 + 4 * i + 1]));
+          mx1 = max3(mx1, __uint_as_float(r[64 + 4 * i + 2]), __uint_as_float(r[64 + 4 * i + 3]));
+          const unsigned long long xa =
+              fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+          const unsigned long long xb =
+              fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+          float xa0, xa1, xb0, xb1;
+          unpack2(xa, xa0, xa1);
+          unpack2(xb, xb0, xb1);
+          const float p0 = ex2(xa0), p1 = ex2(xa1), p2 = ex2(xb0), p3 = ex2(xb1);
+          acc_a = add2(acc_a, pack2(p0, p1));
+          acc_b = add2(acc_b, pack2(p2, p3));
+          r[2 * i] = pack_bf16(p0, p1);
+          r[2 * i + 1] = pack_bf16(p2, p3);
+        }
+        const float mx = fmaxf(mx0, mx1) * sl2;              // scale > 0
+        if (tid == 0) BICACHE_STAMP(0, ti);
+        if (!__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+          if (tid == 0) BICACHE_STAMP(0, ti);
+          tmem_st32(tmem_s, r);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(smem_u32(&bars->p_half[X][0]));
+          if (tid == 0) BICACHE_STAMP(0, ti);
+#pragma unroll
+          for (int i = 16; i < 32; ++i) {
             const unsigned long long xa =
                 fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
             const unsigned long long xb =
@@ -475,155 +520,134 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             r[2 * i] = pack_bf16(p0, p1);
             r[2 * i + 1] = pack_bf16(p2, p3);
           }
-          const float mx = fmaxf(mx0, mx1) * sl2;              // scale > 0
           if (tid == 0) BICACHE_STAMP(0, ti);
-          if (!__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
-            if (tid == 0) BICACHE_STAMP(0, ti);
-            tmem_st32(tmem_s, r);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(smem_u32(&bars->p_half[X][0]));
-            if (tid == 0) BICACHE_STAMP(0, ti);
-  #pragma unroll
-            for (int i = 16; i < 32; ++i) {
-              const unsigned long long xa =
-                  fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
-              const unsigned long long xb =
-                  fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
-              float xa0, xa1, xb0, xb1;
-              unpack2(xa, xa0, xa1);
-              unpack2(xb, xb0, xb1);
-              const float p0 = ex2(xa0), p1 = ex2(xa1), p2 = ex2(xb0), p3 = ex2(xb1);
-              acc_a = add2(acc_a, pack2(p0, p1));
-              acc_b = add2(acc_b, pack2(p2, p3));
-              r[2 * i] = pack_bf16(p0, p1);
-              r[2 * i + 1] = pack_bf16(p2, p3);
-            }
-            if (tid == 0) BICACHE_STAMP(0, ti);
-            tmem_st32(tmem_s + 32, r + 32);
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(smem_u32(&bars->p_half[X][1]));
-            if (tid == 0) BICACHE_STAMP(0, ti);
-            stored = true;
-          } else {
-            // redo with the new reference: S is still intact in TMEM
-            if (mx > m_ref + 8.f) {
-              alpha = ex2(m_ref - mx);
-              m_ref = mx;
-            }
-            unsigned s4[32];
-            const float neg_m = -m_ref;
-            float ps = 0.f;
-  #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              tmem_ld32(tmem_s + c * 32, s4);
-              tmem_wait_ld();
-  #pragma unroll
-              for (int i = 0; i < 16; ++i) {
-                const float p0 = ex2(fmaf(__uint_as_float(s4[2 * i]), sl2, neg_m));
-                const float p1 = ex2(fmaf(__uint_as_float(s4[2 * i + 1]), sl2, neg_m));
-                ps += p0 + p1;
-                r[c * 16 + i] = pack_bf16(p0, p1);
-              }
-            }
-            acc_a = pack2(ps, 0.f);
-            acc_b = pack2(0.f, 0.f);
-            // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
-  #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              tmem_ld32(tmem_o + c * 32, s4);
-              tmem_wait_ld();
-  #pragma unroll
-              for (int i = 0; i < 32; ++i) s4[i] = __float_as_uint(__uint_as_float(s4[i]) * alpha);
-              tmem_st32(tmem_o + c * 32, s4);
-            }
-          }
-        } else {
-          // First tile of the item, or a ragged tile: maximum first, every exponential on the exp
-          // unit so that masked columns give exactly 0.
-          if (cnt < kTileKeys) {
-  #pragma unroll
-            for (int i = 0; i < 128; ++i)
-              if (i >= cnt) r[i] = 0xff800000u;                // -inf: columns past the last key
-          }
-          float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-  #pragma unroll
-          for (int i = 0; i < 128; i += 8) {
-            mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-            mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-            mx2 = max3(mx2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-            mx3 = max3(mx3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-          }
-          const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sl2;   // scale > 0
-          if (j == 0) {
-            m_ref = mx;
-          } else if (mx > m_ref + 8.f) {
-            alpha = ex2(m_ref - mx);
-            m_ref = mx;
-          }
-          if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-  #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              unsigned o[32];
-              tmem_ld32(tmem_o + c * 32, o);
-              tmem_wait_ld();
-  #pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-              tmem_st32(tmem_o + c * 32, o);
-            }
-          }
-          const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
-  #pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const unsigned long long xa =
-                fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
-            const unsigned long long xb =
-                fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
-            float x0, x1, x2, x3;
-            unpack2(xa, x0, x1);
-            unpack2(xb, x2, x3);
-            const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-            acc_a = add2(acc_a, pack2(p0, p1));
-            acc_b = add2(acc_b, pack2(p2, p3));
-            r[2 * i] = pack_bf16(p0, p1);
-            r[2 * i + 1] = pack_bf16(p2, p3);
-          }
-        }
-        if (!stored) {
-          tmem_st32(tmem_s, r);
           tmem_st32(tmem_s + 32, r + 32);
           tmem_wait_st();
           tc_fence_before();
-          mbar_arrive(smem_u32(&bars->p_half[X][0]));
           mbar_arrive(smem_u32(&bars->p_half[X][1]));
+          if (tid == 0) BICACHE_STAMP(0, ti);
+          stored = true;
+        } else {
+          // redo with the new reference: S is still intact in TMEM
+          if (mx > m_ref + 8.f) {
+            alpha = ex2(m_ref - mx);
+            m_ref = mx;
+          }
+          unsigned s4[32];
+          const float neg_m = -m_ref;
+          float ps = 0.f;
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tmem_s + c * 32, s4);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float p0 = ex2(fmaf(__uint_as_float(s4[2 * i]), sl2, neg_m));
+              const float p1 = ex2(fmaf(__uint_as_float(s4[2 * i + 1]), sl2, neg_m));
+              ps += p0 + p1;
+              r[c * 16 + i] = pack_bf16(p0, p1);
+            }
+          }
+          acc_a = pack2(ps, 0.f);
+          acc_b = pack2(0.f, 0.f);
+          // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            tmem_ld32(tmem_o + c * 32, s4);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) s4[i] = __float_as_uint(__uint_as_float(s4[i]) * alpha);
+            tmem_st32(tmem_o + c * 32, s4);
+          }
         }
-        {
-          float s0, s1, s2, s3;
-          unpack2(acc_a, s0, s1);
-          unpack2(acc_b, s2, s3);
-          l_sum = l_sum * alpha + ((s0 + s1) + (s2 + s3));
+      } else {
+        // First tile of the item, or a ragged tile: maximum first, every exponential on the exp
+        // unit so that masked columns give exactly 0.
+        if (cnt < kTileKeys) {
+#pragma unroll
+          for (int i = 0; i < 128; ++i)
+            if (i >= cnt) r[i] = 0xff800000u;                // -inf: columns past the last key
+        }
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 128; i += 8) {
+          mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+          mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+          mx2 = max3(mx2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+          mx3 = max3(mx3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+        }
+        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sl2;   // scale > 0
+        if (j == 0) {
+          m_ref = mx;
+        } else if (mx > m_ref + 8.f) {
+          alpha = ex2(m_ref - mx);
+          m_ref = mx;
+        }
+        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            unsigned o[32];
+            tmem_ld32(tmem_o + c * 32, o);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+            tmem_st32(tmem_o + c * 32, o);
+          }
+        }
+        const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const unsigned long long xa =
+              fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+          const unsigned long long xb =
+              fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+          float x0, x1, x2, x3;
+          unpack2(xa, x0, x1);
+          unpack2(xb, x2, x3);
+          const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+          acc_a = add2(acc_a, pack2(p0, p1));
+          acc_b = add2(acc_b, pack2(p2, p3));
+          r[2 * i] = pack_bf16(p0, p1);
+          r[2 * i + 1] = pack_bf16(p2, p3);
         }
       }
-      if (!ok) break;
-      // ------------------------------- epilogue -------------------------------------------
-      const int prow = item.row0 + X * 128 + gt;       // packed row of this thread
-      const bool row_valid = active && prow < packed_rows;
-      const int a = prow / G;
-      const int h = item.kv_head * G + (prow - a * G);
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->o_done), n_it & 1, abort_flag));
-      if (!ok) break;
-      tc_fence_after();
-      const bool have = active && T > 0;
-      const float inv = have ? 1.f / l_sum : 0.f;
-      const float lse = have ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
+      if (!stored) {
+        tmem_st32(tmem_s, r);
+        tmem_st32(tmem_s + 32, r + 32);
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(smem_u32(&bars->p_half[X][0]));
+        mbar_arrive(smem_u32(&bars->p_half[X][1]));
+      }
+      {
+        float s0, s1, s2, s3;
+        unpack2(acc_a, s0, s1);
+        unpack2(acc_b, s2, s3);
+        l_sum = l_sum * alpha + ((s0 + s1) + (s2 + s3));
+      }
+    }
+    // ------------------------------- epilogue -------------------------------------------
+    const int prow = item.row0 + X * 128 + gt;       // packed row of this thread
+    const bool row_valid = prow < packed_rows;
+    const int a = prow / G;
+    const int h = item.kv_head * G + (prow - a * G);
+    if (ok && T > 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->o_done), 0, abort_flag));
+      if (ok) tc_fence_after();
+    }
+#ifdef BICACHE_TRACE
+    if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1003] = clock64();
+#endif
+    if (ok) {
+      const float inv = T > 0 ? 1.f / l_sum : 0.f;
+      const float lse = T > 0 ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
       if (s.num_splits > 1) {
         const long long pr = ((long long)item.split * t.total_tokens + req.tok_off + a) * t.Hq + h;
         float* po = t.part_o + pr * 128;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
           unsigned o[32];
-          if (have) {
+          if (T > 0) {
             tmem_ld32(tmem_o + c * 32, o);
             tmem_wait_ld();
           } else {
@@ -640,76 +664,60 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           }
         }
         if (row_valid) t.part_lse[pr] = lse;
-        tc_fence_before();
-        mbar_arrive(smem_u32(&bars->o_free[X]));             // O may be overwritten by the next item
-      } else {
+      } else if (T > 0) {
         // Each thread holds one output row; a row-per-thread store would touch 32 rows per
-        // instruction.  The warp's 32 rows are staged in shared memory, 64 columns (128 bytes per
-        // row) at a time, and written out four half rows per instruction.  Chunks are XOR-placed
-        // by row to keep both directions conflict-light.
-        unsigned char* stage = stage_smem + warp * 4096;
-        const int cc = lane & 7;
-        const long long o_row_bytes = t.out_stride * 2;
+        // instruction.  Stage the warp's 32 rows (256 bytes each) in this warp's quarter of the Q
+        // tile's shared memory (Q is no longer needed) and write them out two whole rows per
+        // instruction.  Chunks are XOR-placed by row to keep both directions conflict-light.
+        unsigned char* stage = smem + X * kTileBytes + (warp & 3) * 8192;
 #pragma unroll 1
-        for (int ph = 0; ph < 2; ++ph) {
+        for (int c = 0; c < 4; ++c) {
+          unsigned o[32];
+          tmem_ld32(tmem_o + c * 32, o);
+          tmem_wait_ld();
 #pragma unroll
-          for (int c2 = 0; c2 < 2; ++c2) {
-            unsigned o[32];
-            if (have) {
-              tmem_ld32(tmem_o + (ph * 2 + c2) * 32, o);
-              tmem_wait_ld();
-            } else {
-#pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = 0u;
-            }
-            if (ph == 1 && c2 == 1) {
-              tc_fence_before();
-              mbar_arrive(smem_u32(&bars->o_free[X]));       // all of O is in registers / staged
-            }
-#pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              uint4 v4;
-              v4.x = pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
-              v4.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-              v4.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
-              v4.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
-              const int ch = c2 * 4 + (i >> 3);
-              *reinterpret_cast<uint4*>(stage + lane * 128 + ((ch ^ (lane & 7)) << 4)) = v4;
-            }
+          for (int i = 0; i < 32; i += 8) {
+            uint4 v4;
+            v4.x = pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+            v4.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+            v4.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+            v4.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+            const int cc = c * 4 + (i >> 3);
+            *reinterpret_cast<uint4*>(stage + lane * 256 + ((cc ^ (lane & 15)) << 4)) = v4;
           }
-          __syncwarp();
-          if (active && T > 0) {
-            int row = lane >> 3;                               // rows row, row + 4, ... of this warp
-            int prow2 = item.row0 + X * 128 + (warp & 3) * 32 + row;
-            const int a2 = prow2 / G;
-            int jj = prow2 - a2 * G;
-            char* dst_row = t.out + (req.row_off * t.out_stride + (long long)item.kv_head * G * 128) * 2 +
-                            ph * 128 + cc * 16 + a2 * o_row_bytes;
-#pragma unroll 4
-            for (int k = 0; k < 8; ++k) {
-              const uint4 v4 = *reinterpret_cast<const uint4*>(stage + row * 128 + ((cc ^ (row & 7)) << 4));
-              if (prow2 < packed_rows) *reinterpret_cast<uint4*>(dst_row + jj * 256) = v4;
-              row += 4;
-              prow2 += 4;
-              jj += 4;
-              while (jj >= G) {
-                jj -= G;
-                dst_row += o_row_bytes;
-              }
-            }
-          }
-          __syncwarp();
         }
-        if (row_valid && T > 0 && t.lse != nullptr) t.lse[(req.row_off + a) * t.Hq + h] = lse;
+        __syncwarp();
+        {
+          const int cc = lane & 15;
+          int row = lane >> 4;                                 // rows row, row + 2, ... of this warp
+          int prow2 = item.row0 + X * 128 + (warp & 3) * 32 + row;
+          const int a2 = prow2 / G;
+          int jj = prow2 - a2 * G;
+          const long long o_row_bytes = t.out_stride * 2;
+          char* dst_row = t.out + (req.row_off * t.out_stride + (long long)item.kv_head * G * 128) * 2 + cc * 16 +
+                          a2 * o_row_bytes;
+#pragma unroll 4
+          for (int it = 0; it < 16; ++it) {
+            const uint4 v4 = *reinterpret_cast<const uint4*>(stage + row * 256 + ((cc ^ (row & 15)) << 4));
+            if (prow2 < packed_rows) *reinterpret_cast<uint4*>(dst_row + jj * 256) = v4;
+            row += 2;
+            prow2 += 2;
+            jj += 2;
+            while (jj >= G) {
+              jj -= G;
+              dst_row += o_row_bytes;
+            }
+          }
+        }
+        if (row_valid && t.lse != nullptr) t.lse[(req.row_off + a) * t.Hq + h] = lse;
       }
     }
     tc_fence_before();
   } else if (warp >= 9) {
     // ====================================== loads =======================================
-    // Three load warps, each responsible for whole tiles: ring use g (counted over all items of
-    // this CTA; within an item u = 2 j is K of key tile j, u = 2 j + 1 is V) belongs to warp g % 3.
-    // A warp issues its tile, waits for it to land, fences and signals, while the other two warps
-    // are already issuing theirs.  Warps 0 and 1 also fetch the item's Q tiles A and B.
+    // Three load warps, each responsible for whole tiles: warp w takes ring uses u = w, w + 3, ...
+    // (u = 2 j: K of key tile j, u = 2 j + 1: V of key tile j).  A warp issues its tile, waits for
+    // it to land, fences and signals, while the other two warps are already issuing theirs.
     const int w = warp - 9;
     // A 128-row tile is fetched as 64 passes of 2 rows: lane l takes 16-byte chunk (l & 15) of rows
     // (l >> 4) + 2 i.  In the tile image, rows r, r + 8, r + 16, ... are 2048 bytes apart.
@@ -718,180 +726,118 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
 #pragma unroll
     for (int q = 0; q < 4; ++q) dst_q[q] = tile_chunk_offset(r0 + 2 * q, c16);
     bool ok = !dead;
-    unsigned g_use = 0;                               // ring uses of all earlier items of this CTA
     int ti = 0; (void)ti;
-    for (int it = blockIdx.x, n_it = 0; it < s.num_items && ok; it += gridDim.x, ++n_it) {
-      const ItemGeom geo = load_geom(s, G, it);
-      const WorkItem item = geo.item;
-      const ReqMeta req = geo.req;
-      const int prefix_tiles = geo.prefix_tiles, tile_begin = geo.tile_begin, T = geo.T;
-      const int packed_rows = geo.packed_rows;
-      if (w < 2) {
-        // Q tiles (warp 0: A, warp 1: B): packed rows (token a, head jj within the KV group,
-        // p = a * G + jj) advance without divisions; rows past the end are zero-filled.  The Q
-        // buffers are free once the last S of the previous item has been computed.
-        ok = mbar_wait(smem_u32(&bars->q_free), (n_it & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        if (q_tma) {
-          // 128 packed rows = 128 / G tokens x G heads of the KV group: one TMA box per 64-dim half,
-          // written in the dense swizzled layout (row r at r * 128 bytes, halves 16 KB apart).
-          if (lane == 0) {
-            if (w == 0 || geo.b_active) {
-              const unsigned qf = smem_u32(&bars->q_full);
-              const unsigned q_dst = q_smem + w * kTileBytes;
-              const int tok = (int)req.row_off + (item.row0 + w * 128) / G;
-              mbar_arrive_expect_tx(qf, (unsigned)kTileBytes);
-              tma_load_3d(q_dst, &tm_q, 0, item.kv_head * G, tok, qf);
-              tma_load_3d(q_dst + kTileBytes / 2, &tm_q, 64, item.kv_head * G, tok, qf);
-            } else {
-              mbar_arrive(smem_u32(&bars->q_full));
-            }
-          } else {
-            mbar_arrive(smem_u32(&bars->q_full));
-          }
+    const int* pages = s.pages + req.page_off;
+    for (int u = w; u < 2 * T && ok; u += 3) {
+      const int slot = u % kRing;
+      const int jg = tile_begin + (u >> 1);
+      const bool is_v = u & 1;
+      ok = mbar_wait(smem_u32(&bars->free_[slot]), ((u / kRing) & 1) ^ 1, abort_flag);
+      if (!ok) break;
+      const unsigned dst = ring_smem + slot * kTileBytes;
+      const unsigned full = smem_u32(&bars->full[slot]);
+      if (jg < prefix_tiles) {
+        // cached prefix tile: one bulk copy per page; a pool page already is the tile image
+        const int cnt = min(kTileKeys, req.m - jg * kTileKeys);
+        const int npages = (cnt + kPageSize - 1) / kPageSize;
+        if (lane == 0) {
+          const char* pool_base = is_v ? pool.v : pool.k;
+          mbar_arrive_expect_tx(full, (unsigned)(npages * kPageBytes));
+          for (int pg = 0; pg < npages; ++pg)
+            bulk_copy_g2s(dst + pg * kPageBytes,
+                          pool_base + pool_slice_offset(pool, t.layer, pages[jg * 8 + pg], item.kv_head),
+                          kPageBytes, full);
         } else {
-          if (w == 0 || geo.b_active) {
-            int prow = item.row0 + w * 128 + r0;
-            const int a0 = prow / G;
-            int jj = prow - a0 * G;
-            const long long q_row_bytes = t.q_stride * 2;
-            const char* q_base = t.q + (req.row_off * t.q_stride + (long long)item.kv_head * G * 128) * 2 + c16 * 16;
-            const char* src_row = q_base + a0 * q_row_bytes;
-            const unsigned q_dst = q_smem + w * kTileBytes;
-#pragma unroll 4
-            for (int i = 0; i < 64; ++i) {
-              const bool valid = prow < packed_rows;
-              cp_async16(q_dst + dst_q[i & 3] + (i >> 2) * 2048, valid ? src_row + jj * 256 : q_base, valid ? 16u : 0u);
-              prow += 2;
-              jj += 2;
-              while (jj >= G) {                       // at most twice (G >= 1)
-                jj -= G;
-                src_row += q_row_bytes;
-              }
-            }
-          }
-          cp_async_commit();
-          cp_async_wait<0>();                         // the other load warps issue K/V tiles meanwhile
-          fence_proxy_async();
-          mbar_arrive(smem_u32(&bars->q_full));
+          mbar_arrive(full);
         }
-      }
-      const int* pages = s.pages + req.page_off;
-      for (int u = 0; u < 2 * T && ok; ++u) {
-        const unsigned g = g_use + u;
-        if ((int)(g % 3) != w) continue;
-        const int slot = g % kRing;
-        const int jg = tile_begin + (u >> 1);
-        const bool is_v = u & 1;
-        ok = mbar_wait(smem_u32(&bars->free_[slot]), ((g / kRing) & 1) ^ 1, abort_flag);
-        if (!ok) break;
-        const unsigned dst = ring_smem + slot * kTileBytes;
-        const unsigned full = smem_u32(&bars->full[slot]);
-        if (jg < prefix_tiles) {
-          // cached prefix tile: one bulk copy per page; a pool page already is the tile image
-          const int cnt = min(kTileKeys, req.m - jg * kTileKeys);
-          const int npages = (cnt + kPageSize - 1) / kPageSize;
+      } else {
+        // own rows: 16-byte gathers from row-major K/V into the image, zero-filled past the end
+        const int key0 = (jg - prefix_tiles) * kTileKeys;
+        const int cnt = min(kTileKeys, req.n - key0);
+        const char* row0 = (is_v ? t.v : t.k) +
+                           ((req.row_off + key0) * t.kv_stride + (long long)item.kv_head * 128) * 2 + c16 * 16;
+        const long long row_bytes = t.kv_stride * 2;
+        const char* src = row0 + r0 * row_bytes;
+        if (cnt >= kTileKeys) {
+          // a full tile of the request's own rows: two TMA boxes (dense swizzled layout)
           if (lane == 0) {
-            const char* pool_base = is_v ? pool.v : pool.k;
-            mbar_arrive_expect_tx(full, (unsigned)(npages * kPageBytes));
-            for (int pg = 0; pg < npages; ++pg)
-              bulk_copy_g2s(dst + pg * kPageBytes,
-                            pool_base + pool_slice_offset(pool, t.layer, pages[jg * 8 + pg], item.kv_head),
-                            kPageBytes, full);
+            const int row = (int)req.row_off + key0;
+            const void* tm = is_v ? (const void*)&tm_v : (const void*)&tm_k;
+            mbar_arrive_expect_tx(full, (unsigned)kTileBytes);
+            tma_load_3d(dst, tm, 0, item.kv_head, row, full);
+            tma_load_3d(dst + kTileBytes / 2, tm, 64, item.kv_head, row, full);
           } else {
             mbar_arrive(full);
           }
-        } else {
-          // own rows: 16-byte gathers from row-major K/V into the image, zero-filled past the end
-          const int key0 = (jg - prefix_tiles) * kTileKeys;
-          const int cnt = min(kTileKeys, req.n - key0);
-          const char* row0 = (is_v ? t.v : t.k) +
-                             ((req.row_off + key0) * t.kv_stride + (long long)item.kv_head * 128) * 2 + c16 * 16;
-          const long long row_bytes = t.kv_stride * 2;
-          const char* src = row0 + r0 * row_bytes;
-          if (cnt >= kTileKeys) {
-            // a full tile of the request's own rows: two TMA boxes (dense swizzled layout)
-            if (lane == 0) {
-              const int row = (int)req.row_off + key0;
-              const void* tm = is_v ? (const void*)&tm_v : (const void*)&tm_k;
-              mbar_arrive_expect_tx(full, (unsigned)kTileBytes);
-              tma_load_3d(dst, tm, 0, item.kv_head, row, full);
-              tma_load_3d(dst + kTileBytes / 2, tm, 64, item.kv_head, row, full);
-            } else {
-              mbar_arrive(full);
-            }
-          } else {
-            // ragged last tile: 16-byte gathers into the page-image layout, zero-filled past the end
-#pragma unroll 4
-            for (int i = 0; i < 64; ++i) {
-              const bool valid = r0 + 2 * i < cnt;
-              cp_async16(dst + dst_q[i & 3] + (i >> 2) * 2048, valid ? src : row0, valid ? 16u : 0u);
-              src += 2 * row_bytes;
-            }
-            cp_async_commit();
-            cp_async_wait<0>();
-            fence_proxy_async();
-            mbar_arrive(full);
-          }
+          continue;
         }
+        // ragged last tile: 16-byte gathers into the page-image layout, zero-filled past the end
+#pragma unroll 4
+        for (int i = 0; i < 64; ++i) {
+          const bool valid = r0 + 2 * i < cnt;
+          cp_async16(dst + dst_q[i & 3] + (i >> 2) * 2048, valid ? src : row0, valid ? 16u : 0u);
+          src += 2 * row_bytes;
+        }
+        cp_async_commit();
+        if (w == 0 && lane == 0) BICACHE_STAMP(2, ti);
+        cp_async_wait<0>();
+        fence_proxy_async();
+        mbar_arrive(full);
+        if (w == 0 && lane == 0) BICACHE_STAMP(2, ti);
       }
-      g_use += 2u * (unsigned)T;
     }
     cp_async_wait<0>();
     // On the normal path every tile loaded has been consumed by the time the CTA ends (the
-    // epilogue waits for the last MMA).  After a give-up, bulk copies may still be in flight: give
-    // them time to land before the CTA's shared memory is released.
+    // epilogue waits for the last MMA).  After a give-up, bulk copies may still be in flight:
+    // wait (bounded) for the last barriers this lane armed.
     if (!dead && (!ok || *abort_flag) && lane == 0) {
-      for (unsigned itw = 0; itw < 64; ++itw) __nanosleep(1000);
+      for (int u = max(0, 2 * T - kRing); u < 2 * T; ++u)
+        if (u % 3 == w && tile_begin + (u >> 1) < prefix_tiles)
+          for (unsigned it = 0; it < 4096 && !mbar_try_wait(smem_u32(&bars->full[u % kRing]), (u / kRing) & 1); ++it)
+            __nanosleep(256);
     }
   } else if (warp == kMmaWarp) {
     // ===================================== MMA issue =====================================
     // The whole warp runs this control flow converged and one elected lane issues each tcgen05
     // instruction: descriptor arithmetic then stays in the uniform datapath and the MMAs can be
     // issued back to back (a single diverged lane cannot feed the tensor pipe fast enough).
-    const unsigned tmem_s2[2] = {tmem, tmem + 128};
-    const unsigned tmem_o2[2] = {tmem + 256, tmem + 384};
-    // Two shared-memory layouts occur (see make_desc): the page image (cached tiles, gathered ragged
-    // tiles, gathered Q) and the dense layout TMA writes (full own-row tiles, TMA-loaded Q): 8-row
-    // groups 1024 bytes apart, the two 64-dim halves 16 KB apart.
-    const unsigned q_sbo = q_tma ? 1024u : 2048u, q_hi = q_tma ? 1024u : 64u;
-    const unsigned long long q_desc[2] = {make_desc(q_smem, 16, q_sbo), make_desc(q_smem + kTileBytes, 16, q_sbo)};
-    bool ok = !dead;
-    unsigned g_use = 0;                               // ring uses of all earlier items of this CTA
-    unsigned tcnt[2] = {0, 0};                        // key tiles issued so far, per query tile
-    int ti = 0; (void)ti;
-    for (int it = blockIdx.x, n_it = 0; it < s.num_items && ok; it += gridDim.x, ++n_it) {
-      const ItemGeom geo = load_geom(s, G, it);
-      const ReqMeta req = geo.req;
-      const int prefix_tiles = geo.prefix_tiles, tile_begin = geo.tile_begin, T = geo.T;
-      const int nx = geo.b_active ? 2 : 1;
+    if (!dead && T > 0) {
+      const unsigned tmem_s2[2] = {tmem, tmem + 128};
+      const unsigned tmem_o2[2] = {tmem + 256, tmem + 384};
+      // Two shared-memory layouts occur (see make_desc): the page image (cached tiles, gathered ragged
+      // tiles, gathered Q) and the dense layout TMA writes (full own-row tiles, TMA-loaded Q): 8-row
+      // groups 1024 bytes apart, the two 64-dim halves 16 KB apart.
+      const unsigned q_sbo = q_tma ? 1024u : 2048u, q_hi = q_tma ? 1024u : 64u;
+      const unsigned long long q_desc[2] = {make_desc(q_smem, 16, q_sbo), make_desc(q_smem + kTileBytes, 16, q_sbo)};
+      const int nx = b_active ? 2 : 1;
       // a key tile is in the dense (TMA) layout iff it is a full tile of the request's own rows
       auto dense_tile = [&](int jt) {
         const int jgt = tile_begin + jt;
         return jgt >= prefix_tiles && req.n - (jgt - prefix_tiles) * kTileKeys >= kTileKeys;
       };
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_full), n_it & 1, abort_flag));
-      if (!ok) break;
+      bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_full), 0, abort_flag));
+      int ti = 0; (void)ti;
       if (lane == 0) BICACHE_STAMP(1, ti);
-      // Issue order: S_A(0) [S_B(0) once P_A(0) is half done] | O_A(0) S_A(1) | O_B(0) S_B(1) | ...
+      // Issue order: S_A(0) S_B(0) | O_A(0) S_A(1) | O_B(0) S_B(1) | O_A(1) S_A(2) | ...
       // O_X(j) += P_X V is issued in two halves as P arrives, and S_X(j+1) = Q_X K^T follows it
       // back to back (it overwrites P_X; the tensor pipe runs MMAs in issue order).  The K/V tiles
-      // an iteration needs are waited for before the wait on P.
-      if (T > 0) {
-        const unsigned g0 = g_use;
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[g0 % kRing]), (g0 / kRing) & 1, abort_flag));
-        if (!ok) break;
+      // an iteration needs are waited for before the wait on P, so nothing stands between the
+      // arrival of P and the MMAs.
+      // prologue: S_X(0)
+      ok = ok && __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[0]), 0, abort_flag));
+      if (ok) {
         fence_proxy_async();
         tc_fence_after();
         const bool kd0 = dense_tile(0);
         const unsigned k_hi0 = kd0 ? 1024u : 64u;
-        const unsigned long long k_desc = make_desc(ring_smem + (g0 % kRing) * kTileBytes, 16, kd0 ? 1024u : 2048u);
+        const unsigned long long k_desc = make_desc(ring_smem, 16, kd0 ? 1024u : 2048u);
         for (int x = 0; x < nx; ++x) {
           if (x == 1) {
             // Stagger the two query tiles by half a period: tile B starts when tile A's softmax is
             // half done, so that afterwards each tile's softmax runs while the tensor pipe works for
-            // the other tile.
-            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[0][0]), tcnt[0] & 1, abort_flag));
+            // the other tile (started together, the two softmaxes share the exp unit and the MMAs
+            // of both tiles then queue behind each other).
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[0][0]), 0, abort_flag));
             if (!ok) break;
           }
 #pragma unroll
@@ -900,27 +846,19 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
                          kIdescQK, k > 0 ? 1u : 0u);
           mma_commit_elect(smem_u32(&bars->s_full[x]));
         }
-        if (!ok) break;
-        mma_commit_elect(smem_u32(&bars->free_[g0 % kRing]));
-        if (T == 1) mma_commit_elect(smem_u32(&bars->q_free));    // that was the last S of the item
-      } else {
-        mma_commit_elect(smem_u32(&bars->q_free));
+        if (ok) mma_commit_elect(smem_u32(&bars->free_[0]));
       }
-      // O of the previous item must have been read out before it is overwritten
-      for (int x = 0; x < 2 && ok; ++x)
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->o_free[x]), (n_it & 1) ^ 1, abort_flag));
-      if (!ok) break;
       for (int j = 0; j < T && ok; ++j) {
         const int jg = tile_begin + j;
         const int cnt = jg < prefix_tiles ? min(kTileKeys, req.m - jg * kTileKeys)
                                           : min(kTileKeys, req.n - (jg - prefix_tiles) * kTileKeys);
         const int ksteps = (cnt + 15) >> 4;
-        const unsigned gv = g_use + 2 * j + 1, gn = g_use + 2 * j + 2;    // ring uses: V of tile j, K of tile j + 1
-        const int slot_v = gv % kRing, slot_n = gn % kRing;
+        const int uv = 2 * j + 1, un = 2 * j + 2;          // ring uses: V of tile j, K of tile j + 1
+        const int slot_v = uv % kRing, slot_n = un % kRing;
         const bool more = j + 1 < T;
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_v]), (gv / kRing) & 1, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_v]), (uv / kRing) & 1, abort_flag));
         if (ok && more)
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_n]), (gn / kRing) & 1, abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_n]), (un / kRing) & 1, abort_flag));
         if (!ok) break;
         fence_proxy_async();
         const bool vd = dense_tile(j), kd = more && dense_tile(j + 1);
@@ -934,7 +872,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           // O_X += P_X V, 16 keys (one page image) per MMA; P is the A operand, read from TMEM
 #pragma unroll
           for (int half = 0; half < 2; ++half) {
-            ok = ok && __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[x][half]), (tcnt[x] + j) & 1, abort_flag));
+            ok = ok && __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[x][half]), j & 1, abort_flag));
             if (ok) {
               if (lane == 0 && x == 0 && half == 0) BICACHE_STAMP(1, ti);
               tc_fence_after();
@@ -958,17 +896,10 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
         if (!ok) break;
         mma_commit_elect(smem_u32(&bars->free_[slot_v]));
         if (more) mma_commit_elect(smem_u32(&bars->free_[slot_n]));
-        if (j + 2 == T) mma_commit_elect(smem_u32(&bars->q_free));      // the last S of the item has been issued
       }
-      if (!ok) break;
-      mma_commit_elect(smem_u32(&bars->o_done));
-      g_use += 2u * (unsigned)T;
-      tcnt[0] += (unsigned)T;
-      if (nx == 2) tcnt[1] += (unsigned)T;
-    }
-    // Whatever happened, let every MMA issued so far finish before TMEM is released.
-    __syncwarp();
-    if (!dead) {
+      if (ok) mma_commit_elect(smem_u32(&bars->o_done));
+      // Whatever happened, let every MMA issued so far finish before TMEM is released.
+      __syncwarp();
       mma_commit_elect(smem_u32(&bars->drain));
       mbar_wait(smem_u32(&bars->drain), 0, abort_flag);
     }
@@ -976,6 +907,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
   }
 
   __syncthreads();
+#ifdef BICACHE_TRACE
+  if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1002] = clock64();
+#endif
   if (warp == kMmaWarp) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
@@ -1002,9 +936,9 @@ struct TcTensorMaps {
 
 inline cudaError_t launch_tc_attention(const ScheduleView& s, const PoolView& pool, const TensorArgs& t,
                                        int* status, int num_sms, const TcTensorMaps& maps, cudaStream_t stream) {
-  const int grid = s.num_items < num_sms ? s.num_items : num_sms;
-  tc_attention_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(s, pool, t, status, maps.q, maps.k, maps.v,
-                                                                       maps.q_tma);
+  (void)num_sms;             // one CTA per work item; the hardware scheduler balances ragged items
+  tc_attention_kernel<<<s.num_items, tc::kThreads, tc::kSmemBytes, stream>>>(s, pool, t, status, maps.q, maps.k,
+                                                                              maps.v, maps.q_tma);
   return cudaGetLastError();
 }
 
