@@ -204,15 +204,31 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
       unsplit_items += (long long)((r.n * (long long)G + kTileRows - 1) / kTileRows) * Hkv;
     }
   }
-  // Split the keys across CTAs when the batch has too few row tiles to fill the GPU.
+  // Split the keys across CTAs when the batch has too few row tiles to fill the GPU.  The number of
+  // splits minimises a simple cost model: waves of CTAs (one CTA per SM) times the time of one CTA
+  // (a fixed prologue/epilogue plus a per-key-tile cost), plus the merge pass over the partials.
   int num_splits = 1, tiles_per_split = 0;
-  if (unsplit_items > 0 && unsplit_items * 2 <= ctx->sm_count && max_key_tiles >= 8) {
+  if (unsplit_items > 0 && unsplit_items < 2LL * ctx->sm_count && max_key_tiles >= 8) {
     const int key_tiles = max_key_tiles;
-    int want = (int)std::min<long long>((kTargetCtas + unsplit_items - 1) / unsplit_items, key_tiles / 2);
-    while (want > 1 && tok * ctx->cfg.num_q_heads * want > ctx->part_capacity_rowheads) --want;
-    if (want > 1) {
-      tiles_per_split = (key_tiles + want - 1) / want;
-      num_splits = (key_tiles + tiles_per_split - 1) / tiles_per_split;
+    const double c_tile = 3000.0, c_cta = 8000.0;          // SM clocks
+    auto cost = [&](int nsplit, int tps) {
+      const long long ctas = unsplit_items * nsplit;
+      const double waves = (double)((ctas + ctx->sm_count - 1) / ctx->sm_count);
+      double c = waves * (c_cta + c_tile * tps);
+      if (nsplit > 1) c += 6000.0 + (double)tok * ctx->cfg.num_q_heads * nsplit * 516.0 / 3300.0;
+      return c;
+    };
+    double best = cost(1, key_tiles);
+    for (int want = 2; want <= std::min(64, key_tiles / 2); ++want) {
+      if (tok * ctx->cfg.num_q_heads * want > ctx->part_capacity_rowheads) break;
+      const int tps = (key_tiles + want - 1) / want;
+      const int ns = (key_tiles + tps - 1) / tps;
+      const double c = cost(ns, tps);
+      if (ns > 1 && c < best) {
+        best = c;
+        num_splits = ns;
+        tiles_per_split = tps;
+      }
     }
   }
   std::vector<WorkItem> items;
