@@ -3,11 +3,13 @@
 // One CTA (one per SM) computes one work item: up to 256 packed query rows (one request, one KV
 // head) as two 128-row tiles A and B that share every K/V tile, against a range of key tiles of
 // 128 keys - first the cached prefix (pages of 16 tokens, staged with cp.async.bulk because a pool
-// page already is the shared-memory image the MMA reads), then the request's own rows (16-byte
-// cp.async gathers from the caller's row-major K/V, zero-filled past the end).
+// page already is the shared-memory image the MMA reads), then the request's own rows (full tiles
+// by tiled TMA loads through tensor maps of the caller's row-major K/V; the ragged last tile by
+// 16-byte cp.async gathers, zero-filled past the end).  Q tiles come by TMA as well when the
+// query heads of a KV group divide 128, else by gathers.
 // Per key tile and query tile: S = Q K^T (tcgen05, fp32 in TMEM) -> online softmax in registers
 // (one thread per row) -> P as bf16 written over S in TMEM -> O += P V (tcgen05, A from TMEM).
-// The tensor pipe alternates  S_A(j), O_B(j-1), S_B(j), O_A(j)  so that each softmax warpgroup
+// The MMA warp issues  O_A(j), S_A(j+1), O_B(j), S_B(j+1)  so that each softmax warpgroup
 // works while the other tile's MMAs run.  The running maximum only moves when it grew by more
 // than 2^8, so rescaling O is rare; the final normalisation uses the same reference, which keeps
 // the result exact.
