@@ -389,6 +389,9 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
                encode_map(&maps.v, v, rows_total, cfg.num_kv_heads, kv_row_stride, 1, 128) &&
                encode_map(&maps.q, q, rows_total, cfg.num_q_heads, q_row_stride, maps.q_tma ? G : 1,
                           maps.q_tma ? 128 / G : 128);
+    maps.o_tma = (32 % G == 0) ? 1 : 0;
+    okm = okm && encode_map(&maps.o, out, rows_total, cfg.num_q_heads, out_row_stride, maps.o_tma ? G : 1,
+                            maps.o_tma ? 32 / G : 32);
     if (!okm) return fail(ctx, BICACHE_ERR_CUDA, "tensor map encoding failed");
     e = launch_tc_attention(sv, pool, t, ctx->d_status, ctx->sm_count, maps, stream);
   } else if (cfg.dtype == BICACHE_F32) {

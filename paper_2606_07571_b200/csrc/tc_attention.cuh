@@ -1,26 +1,31 @@
 // Tensor-core attention for bf16, head_dim 128, on sm_100a: tcgen05.mma with TMEM accumulators.
 //
-// One CTA (one per SM) computes one work item: up to 256 packed query rows (one request, one KV
-// head) as two 128-row tiles A and B that share every K/V tile, against a range of key tiles of
-// 128 keys - first the cached prefix (pages of 16 tokens, staged with cp.async.bulk because a pool
-// page already is the shared-memory image the MMA reads), then the request's own rows (full tiles
-// by tiled TMA loads through tensor maps of the caller's row-major K/V; the ragged last tile by
-// 16-byte cp.async gathers, zero-filled past the end).  Q tiles come by TMA as well when the
-// query heads of a KV group divide 128, else by gathers.
+// Persistent kernel: one CTA per SM takes work items from a shared counter (longest items first).
+// A work item is up to 256 packed query rows (one request, one KV head) as two 128-row tiles A
+// and B that share every K/V tile, against a range of key tiles of 128 keys - first the cached
+// prefix (pages of 16 tokens, staged with cp.async.bulk because a pool page already is the
+// shared-memory image the MMA reads), then the request's own rows (full tiles by tiled TMA loads
+// through tensor maps of the caller's row-major K/V; the ragged last tile by 16-byte cp.async
+// gathers, zero-filled past the end).  Q tiles come by TMA as well when the query heads of a KV
+// group divide 128, else by gathers.
 // Per key tile and query tile: S = Q K^T (tcgen05, fp32 in TMEM) -> online softmax in registers
 // (one thread per row) -> P as bf16 written over S in TMEM -> O += P V (tcgen05, A from TMEM).
-// The MMA warp issues  O_A(j), S_A(j+1), O_B(j), S_B(j+1)  so that each softmax warpgroup
-// works while the other tile's MMAs run.  The running maximum only moves when it grew by more
-// than 2^8, so rescaling O is rare; the final normalisation uses the same reference, which keeps
-// the result exact.
+// The MMA warp issues  O_A(j), S_A(j+1), O_B(j), S_B(j+1)  so that each softmax warpgroup works
+// while the other tile's MMAs run, and the stream of key tiles runs on across item boundaries:
+// after the last O_X of an item comes the first S_X of the next item, whose Q, K and V were
+// fetched while the current item was computed, so only the epilogue of a query tile (TMEM ->
+// registers -> bf16 -> shared memory -> TMA store) stands between two items.  The running maximum
+// only moves when it grew by more than 2^8, so rescaling O is rare; the final normalisation uses
+// the same reference, which keeps the result exact.
 //
 // Roles: warps 0-3 softmax/correction/epilogue of tile A, warps 4-7 of tile B (one thread per
-// row), warp 8 MMA issue and TMEM ownership, warps 9-11 loads.  The softmax uses packed fp32
-// instructions and 3-input maxima; MMAs are issued branch-free by an elected lane of a converged
-// warp.  All waits are bounded; a wait that gives up raises a sticky status word and the CTA
-// drains and exits.
+// row), warp 8 MMA issue and TMEM ownership, warp 9 item fetch and Q loads, warp 10 K tiles,
+// warp 11 V tiles.  The softmax uses packed fp32 instructions and 3-input maxima; MMAs are issued
+// branch-free by an elected lane of a converged warp.  All waits are bounded; a wait that gives
+// up raises a sticky status word and the CTA drains and exits.
 #pragma once
 #include <cuda.h>
+#include <type_traits>
 #include <cuda_bf16.h>
 #include "common.cuh"
 #include "simt_kernels.cuh"
@@ -37,8 +42,8 @@ constexpr int kRing = 4;                         // K/V ring slots of one tile e
 constexpr int kThreads = 384;
 constexpr int kGroupThreads = 128;               // softmax threads of one query tile (one per row)
 constexpr int kLoadThreads = 32;                 // one warp loads a whole tile
-constexpr int kSoftmaxRegs = 208;                // registers per thread after setmaxnreg
-constexpr int kOtherRegs = 80;
+constexpr int kSoftmaxRegs = 184;                // registers per thread after setmaxnreg
+constexpr int kOtherRegs = 136;
 constexpr int kMmaWarp = 8;
 #ifndef BICACHE_POLY_PERIOD
 #define BICACHE_POLY_PERIOD 0
@@ -46,20 +51,35 @@ constexpr int kMmaWarp = 8;
 constexpr int kPolyPeriod = BICACHE_POLY_PERIOD;                   // of every kPolyPeriod groups of 4 scores, one sends 2 scores to the FMA-pipe cubic (0: none)
 constexpr long long kWaitCycles = 400000000LL;   // bounded waits: about 0.2 s of SM clocks
 
-// shared-memory layout (dynamic, 1024-byte aligned by hand): Q_A, Q_B, ring, barriers
+// shared-memory layout (dynamic, 1024-byte aligned by hand): Q_A, Q_B, ring, output staging
+// (4 KB per softmax warp), barriers and item records
+struct ItemInfo {                        // one work item, written by the fetching lane of warp 9
+  int valid;                             // 0: the items are exhausted
+  int kv_head, row0, split;
+  int n, m, page_off, tok_off;
+  long long row_off;
+};
 struct alignas(8) Barriers {
-  unsigned long long q_full;
+  unsigned long long info_full[2];       // item record (double-buffered by item parity) is written
+  unsigned long long info_free[2];       // every role is done with the record
+  unsigned long long q_full[2];          // Q tile of the item is in shared memory (per query tile)
+  unsigned long long q_free[2];          // the last S of the item has been computed: Q may be replaced
   unsigned long long full[kRing];        // ring slot holds its tile
   unsigned long long free_[kRing];       // the MMAs reading the slot have completed
   unsigned long long s_full[2];          // S = Q K^T of the current key tile is in TMEM (per query tile)
   unsigned long long p_half[2][2];       // P of keys 0-63 / 64-127 is in TMEM and O is rescaled (per query tile)
-  unsigned long long o_done;             // every MMA of the item has completed
+  unsigned long long o_done[2];          // the last O += P V of the item has completed (per query tile)
+  unsigned long long o_free[2];          // the epilogue has read O out of TMEM (per query tile)
   unsigned long long drain;
   unsigned tmem_base;
   int abort_flag;
+  ItemInfo info[2];
 };
+constexpr int kInfoReaders = 8 + 1 + 2;  // arrivals on info_free: softmax warps, the MMA warp, the two load warps
+constexpr int kStageBytes = 8 * 4096;
 constexpr int kTmemCols = 512;           // S_A 0-127, S_B 128-255 (P over the first 64 of each), O_A 256-383, O_B 384-511
-constexpr int kSmemBytes = 1024 + kTileBytes * (2 + kRing) + (int)sizeof(Barriers) + 64;
+constexpr int kSmemBytes = 1024 + kTileBytes * (2 + kRing) + kStageBytes + (int)sizeof(Barriers) + 64;
+static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 
 // ----- raw PTX wrappers --------------------------------------------------------------------
 __device__ __forceinline__ unsigned smem_u32(const void* p) {
@@ -127,6 +147,17 @@ __device__ __forceinline__ void tma_load_3d(unsigned dst, const void* tmap, int 
       ::"r"(dst), "l"(reinterpret_cast<unsigned long long>(tmap)), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
       : "memory");
 }
+// Tiled TMA store of a 3-D box from shared memory (bulk async-group completion).
+__device__ __forceinline__ void tma_store_3d(const void* tmap, unsigned src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(reinterpret_cast<unsigned long long>(tmap)), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// the shared-memory source of every committed bulk store has been read
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// every committed bulk store has completed
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(unsigned smem_slot, unsigned cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(cols) : "memory");
 }
@@ -311,6 +342,53 @@ __device__ __forceinline__ unsigned tile_chunk_offset(int r, int c16) {
   return (unsigned)((r >> 4) * kPageBytes) + page_chunk_offset(true, r & 15, c16, 256);
 }
 
+// Geometry of one work item, derived from its record.
+struct Geo {
+  int valid, m, n, prefix_tiles, tile_begin, T, b_active;
+};
+__device__ __forceinline__ Geo read_geo(const ItemInfo* inf, int num_splits, int tiles_per_split, int G) {
+  Geo g;
+  g.valid = inf->valid;
+  g.m = inf->m;
+  g.n = inf->n;
+  g.prefix_tiles = (g.m + kTileKeys - 1) / kTileKeys;
+  const int all_tiles = g.prefix_tiles + (g.n + kTileKeys - 1) / kTileKeys;
+  int tb = 0, te = all_tiles;
+  if (num_splits > 1) {
+    tb = min(all_tiles, inf->split * tiles_per_split);
+    te = min(all_tiles, tb + tiles_per_split);
+  }
+  g.tile_begin = tb;
+  g.T = g.valid ? te - tb : 0;
+  g.b_active = inf->row0 + 128 < g.n * G;                   // the item has a second query tile
+  return g;
+}
+// The same, with every field broadcast from lane 0 of a converged warp: the compiler then knows the
+// values to be warp-uniform and keeps what derives from them (loop counters, MMA descriptors) in
+// the uniform datapath, which the MMA issue path needs to run at full rate.
+__device__ __forceinline__ Geo read_geo_uniform(const ItemInfo* inf, int num_splits, int tiles_per_split, int G) {
+  Geo g = read_geo(inf, num_splits, tiles_per_split, G);
+  g.valid = __shfl_sync(0xffffffffu, g.valid, 0);
+  g.m = __shfl_sync(0xffffffffu, g.m, 0);
+  g.n = __shfl_sync(0xffffffffu, g.n, 0);
+  g.prefix_tiles = __shfl_sync(0xffffffffu, g.prefix_tiles, 0);
+  g.tile_begin = __shfl_sync(0xffffffffu, g.tile_begin, 0);
+  g.T = __shfl_sync(0xffffffffu, g.T, 0);
+  g.b_active = __shfl_sync(0xffffffffu, g.b_active, 0);
+  return g;
+}
+// keys of key tile j of the item
+__device__ __forceinline__ int tile_keys(const Geo& g, int j) {
+  const int jg = g.tile_begin + j;
+  return jg < g.prefix_tiles ? min(kTileKeys, g.m - jg * kTileKeys)
+                             : min(kTileKeys, g.n - (jg - g.prefix_tiles) * kTileKeys);
+}
+// a key tile is in the dense (TMA) layout iff it is a full tile of the request's own rows
+__device__ __forceinline__ bool tile_dense(const Geo& g, int j) {
+  const int jg = g.tile_begin + j;
+  return jg >= g.prefix_tiles && g.n - (jg - g.prefix_tiles) * kTileKeys >= kTileKeys;
+}
+
 #ifdef BICACHE_TRACE
 // Debug build only: per-phase SM clock stamps of one CTA (three roles x 1024 slots).
 __device__ long long g_trace[3 * 1024];
@@ -322,50 +400,46 @@ __device__ long long g_trace[3 * 1024];
 
 }  // namespace tc
 
+
 __global__ void __launch_bounds__(tc::kThreads, 1)
 tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
                     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                    const __grid_constant__ CUtensorMap tm_v, int q_tma) {
+                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int q_tma,
+                    int o_tma) {
   using namespace tc;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  Barriers* bars = reinterpret_cast<Barriers*>(smem + kTileBytes * (2 + kRing));
+  Barriers* bars = reinterpret_cast<Barriers*>(smem + kTileBytes * (2 + kRing) + kStageBytes);
   volatile int* abort_flag = &bars->abort_flag;
   const unsigned q_smem = smem_u32(smem);                  // Q_A, then Q_B
   const unsigned ring_smem = q_smem + 2 * kTileBytes;
+  int* const next_item = status + 16;                      // items handed out beyond the first gridDim.x
+  int* const ctas_done = status + 17;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 #ifdef BICACHE_TRACE
   if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1000] = clock64();
 #endif
-  const WorkItem item = s.items[blockIdx.x];
-  const ReqMeta req = s.reqs[item.req];
   const int G = t.Hq / t.Hkv;
-  const int prefix_tiles = (req.m + kTileKeys - 1) / kTileKeys;
-  const int all_tiles = prefix_tiles + (req.n + kTileKeys - 1) / kTileKeys;
-  int tile_begin = 0, tile_end = all_tiles;
-  if (s.num_splits > 1) {
-    tile_begin = min(all_tiles, item.split * s.tiles_per_split);
-    tile_end = min(all_tiles, tile_begin + s.tiles_per_split);
-  }
-  const int T = tile_end - tile_begin;
-  const int packed_rows = req.n * G;
-  const bool b_active = item.row0 + 128 < packed_rows;     // the item has a second query tile
 
   if (tid == 0) {
     bars->abort_flag = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
-    mbar_init(smem_u32(&bars->q_full), 256);              // the eight softmax warps fetch the Q tiles
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&bars->info_full[i]), 1);
+      mbar_init(smem_u32(&bars->info_free[i]), kInfoReaders);
+      mbar_init(smem_u32(&bars->q_full[i]), kLoadThreads);
+      mbar_init(smem_u32(&bars->q_free[i]), 1);
+      mbar_init(smem_u32(&bars->s_full[i]), 1);
+      mbar_init(smem_u32(&bars->p_half[i][0]), kGroupThreads);
+      mbar_init(smem_u32(&bars->p_half[i][1]), kGroupThreads);
+      mbar_init(smem_u32(&bars->o_done[i]), 1);
+      mbar_init(smem_u32(&bars->o_free[i]), kGroupThreads);
+    }
     for (int i = 0; i < kRing; ++i) {
       mbar_init(smem_u32(&bars->full[i]), kLoadThreads);
       mbar_init(smem_u32(&bars->free_[i]), 1);
     }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(smem_u32(&bars->s_full[i]), 1);
-      mbar_init(smem_u32(&bars->p_half[i][0]), kGroupThreads);
-      mbar_init(smem_u32(&bars->p_half[i][1]), kGroupThreads);
-    }
-    mbar_init(smem_u32(&bars->o_done), 1);
     mbar_init(smem_u32(&bars->drain), 1);
     fence_barrier_init();
   }
@@ -380,7 +454,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
   if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1001] = clock64();
 #endif
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&bars->tmem_base);
-  const bool dead = *abort_flag != 0;        // an earlier CTA already gave up: do no work
+  const bool dead = *abort_flag != 0;        // an earlier launch or CTA already gave up: do no work
 
   // Registers move from the MMA/load warpgroup to the two softmax warpgroups, which hold a whole
   // row of S (128 values) per thread.  The counts must fit the CTA's launch allocation:
@@ -398,117 +472,56 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
     const unsigned lane_base = (unsigned)((warp & 3) * 32) << 16;
     const unsigned tmem_s = tmem + X * 128 + lane_base;      // S, and P written over its first 64 columns
     const unsigned tmem_o = tmem + 256 + X * 128 + lane_base;
-    const bool active = !dead && (X == 0 || b_active);
     const float sl2 = t.scale * 1.4426950408889634f;         // scores are handled in the log2 domain
     const unsigned long long sl2_2 = pack2(sl2, sl2);
-    // Each softmax warp first fetches its own 32 rows of the Q tile (packed rows: token a, head jj
-    // within the KV group, p = a * G + jj; rows past the end are zero-filled): eight warps in
-    // parallel hide the DRAM latency of this cold read far better than one load warp could.
-    if (!dead) {
-      if (q_tma) {
-        // 128 packed rows = 128 / G tokens x G heads of the KV group: one TMA box per 64-dim half,
-        // in the dense swizzled layout (row r at r * 128 bytes, halves 16 KB apart).  The first
-        // lane of each tile's first warp issues it; every softmax thread arrives.
-        if ((warp & 3) == 0 && lane == 0 && active) {
-          const unsigned qf = smem_u32(&bars->q_full);
-          const unsigned q_dst = q_smem + X * kTileBytes;
-          const int tok = (int)req.row_off + (item.row0 + X * 128) / G;
-          mbar_arrive_expect_tx(qf, (unsigned)kTileBytes);
-          tma_load_3d(q_dst, &tm_q, 0, item.kv_head * G, tok, qf);
-          tma_load_3d(q_dst + kTileBytes / 2, &tm_q, 64, item.kv_head * G, tok, qf);
-        } else {
-          mbar_arrive(smem_u32(&bars->q_full));
-        }
-      } else {
-        if (active) {
-          const int r0 = (warp & 3) * 32 + (lane >> 4), c16 = lane & 15;
-          int prow = item.row0 + X * 128 + r0;
-          const int a0 = prow / G;
-          int jj = prow - a0 * G;
-          const long long q_row_bytes = t.q_stride * 2;
-          const char* q_base = t.q + (req.row_off * t.q_stride + (long long)item.kv_head * G * 128) * 2 + c16 * 16;
-          const char* src_row = q_base + a0 * q_row_bytes;
-          const unsigned q_dst = q_smem + X * kTileBytes;
-#pragma unroll 4
-          for (int i = 0; i < 16; ++i) {
-            const bool valid = prow < packed_rows;
-            cp_async16(q_dst + tile_chunk_offset(r0 + 2 * i, c16), valid ? src_row + jj * 256 : q_base, valid ? 16u : 0u);
-            prow += 2;
-            jj += 2;
-            while (jj >= G) {                         // at most twice (G >= 1)
-              jj -= G;
-              src_row += q_row_bytes;
-            }
-          }
-          cp_async_commit();
-          cp_async_wait<0>();
-          fence_proxy_async();
-        }
-        mbar_arrive(smem_u32(&bars->q_full));
-      }
-    }
-    float m_ref = -INFINITY, l_sum = 0.f;
-    bool ok = active;
+    unsigned char* const stage = smem + kTileBytes * (2 + kRing) + warp * 4096;   // this warp's 32 rows x 128 bytes
+    bool ok = !dead;
+    int n_it = 0;                // items seen by this CTA
+    int c_tile = 0;              // key tiles this query tile has processed (phase of s_full / p_half)
+    int e_item = 0;              // items this query tile has taken part in (phase of o_done)
     int ti = 0; (void)ti;
-    for (int j = 0; j < T && active; ++j) {
-      const int jg = tile_begin + j;
-      const int cnt = jg < prefix_tiles ? min(kTileKeys, req.m - jg * kTileKeys)
-                                        : min(kTileKeys, req.n - (jg - prefix_tiles) * kTileKeys);
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_full[X]), j & 1, abort_flag));
+    while (ok) {
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->info_full[n_it & 1]), (n_it >> 1) & 1, abort_flag));
       if (!ok) break;
-      tc_fence_after();
-      if (tid == 0) BICACHE_STAMP(0, ti);
-      // the whole row of S into registers: four loads in flight, one wait
-      unsigned r[128];
-      tmem_ld32(tmem_s, r);
-      tmem_ld32(tmem_s + 32, r + 32);
-      tmem_ld32(tmem_s + 64, r + 64);
-      tmem_ld32(tmem_s + 96, r + 96);
-      tmem_wait_ld();
-      if (tid == 0) BICACHE_STAMP(0, ti);
-      float alpha = 1.f;
-      unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
-      bool stored = false;                                   // P already stored and signalled
-      if (j > 0 && cnt >= kTileKeys) {
-        // Common case (a full tile after the first): the exponentials use the reference maximum of
-        // the earlier tiles and do not wait for this tile's maximum, which is computed alongside.
-        // P of the first 64 keys is handed to the tensor pipe before the second half is computed.
-        // If the row maximum turns out to exceed the reference by more than 2^8 (rare: checked per
-        // warp before anything is handed over), the tile is redone below with the new reference.
-        const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
-        float mx0 = -INFINITY, mx1 = -INFINITY;
-        // first half of the exponentials, with the maximum over all 128 scores computed alongside
-        // (independent instructions that fill the exp unit's latency)
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          mx0 = max3(mx0, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
-          mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
-          mx0 = max3(mx0, __uint_as_float(r[64 + 4 * i]), __uint_as_float(r[64 + 4 * i + 1]));
-          mx1 = max3(mx1, __uint_as_float(r[64 + 4 * i + 2]), __uint_as_float(r[64 + 4 * i + 3]));
-          const unsigned long long xa =
-              fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
-          const unsigned long long xb =
-              fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
-          float xa0, xa1, xb0, xb1;
-          unpack2(xa, xa0, xa1);
-          unpack2(xb, xb0, xb1);
-          const float p0 = ex2(xa0), p1 = ex2(xa1), p2 = ex2(xb0), p3 = ex2(xb1);
-          acc_a = add2(acc_a, pack2(p0, p1));
-          acc_b = add2(acc_b, pack2(p2, p3));
-          r[2 * i] = pack_bf16(p0, p1);
-          r[2 * i + 1] = pack_bf16(p2, p3);
-        }
-        const float mx = fmaxf(mx0, mx1) * sl2;              // scale > 0
-        if (tid == 0) BICACHE_STAMP(0, ti);
-        if (!__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
-          if (tid == 0) BICACHE_STAMP(0, ti);
-          tmem_st32(tmem_s, r);
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(smem_u32(&bars->p_half[X][0]));
-          if (tid == 0) BICACHE_STAMP(0, ti);
-#pragma unroll
-          for (int i = 16; i < 32; ++i) {
+      const ItemInfo* inf = &bars->info[n_it & 1];
+      const Geo g = read_geo_uniform(inf, s.num_splits, s.tiles_per_split, G);
+      if (!g.valid) break;
+      const int T = g.T;
+      const bool active = X == 0 || g.b_active;
+      float m_ref = -INFINITY, l_sum = 0.f;
+      for (int j = 0; j < T && active; ++j) {
+        const int cnt = tile_keys(g, j);
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_full[X]), c_tile & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        if (tid == 0) BICACHE_STAMP(0, ti); if (tid == 128) BICACHE_STAMP(2, ti);
+        // the whole row of S into registers: four loads in flight, one wait
+        unsigned r[128];
+        tmem_ld32(tmem_s, r);
+        tmem_ld32(tmem_s + 32, r + 32);
+        tmem_ld32(tmem_s + 64, r + 64);
+        tmem_ld32(tmem_s + 96, r + 96);
+        tmem_wait_ld();
+
+        float alpha = 1.f;
+        unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
+        bool stored = false;                                   // P already stored and signalled
+        if (j > 0 && cnt >= kTileKeys) {
+          // Common case (a full tile after the first): the exponentials use the reference maximum of
+          // the earlier tiles and do not wait for this tile's maximum, which is computed alongside.
+          // P of the first 64 keys is handed to the tensor pipe before the second half is computed.
+          // If the row maximum turns out to exceed the reference by more than 2^8 (rare: checked per
+          // warp before anything is handed over), the tile is redone below with the new reference.
+          const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
+          float mx0 = -INFINITY, mx1 = -INFINITY;
+          // first half of the exponentials, with the maximum over all 128 scores computed alongside
+          // (independent instructions that fill the exp unit's latency)
+  #pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            mx0 = max3(mx0, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
+            mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+            mx0 = max3(mx0, __uint_as_float(r[64 + 4 * i]), __uint_as_float(r[64 + 4 * i + 1]));
+            mx1 = max3(mx1, __uint_as_float(r[64 + 4 * i + 2]), __uint_as_float(r[64 + 4 * i + 3]));
             const unsigned long long xa =
                 fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
             const unsigned long long xb =
@@ -522,384 +535,646 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             r[2 * i] = pack_bf16(p0, p1);
             r[2 * i + 1] = pack_bf16(p2, p3);
           }
-          if (tid == 0) BICACHE_STAMP(0, ti);
-          tmem_st32(tmem_s + 32, r + 32);
-          tmem_wait_st();
-          tc_fence_before();
-          mbar_arrive(smem_u32(&bars->p_half[X][1]));
-          if (tid == 0) BICACHE_STAMP(0, ti);
-          stored = true;
+          const float mx = fmaxf(mx0, mx1) * sl2;              // scale > 0
+
+          if (!__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+            tmem_st32(tmem_s, r);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->p_half[X][0]));
+
+  #pragma unroll
+            for (int i = 16; i < 32; ++i) {
+              const unsigned long long xa =
+                  fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+              const unsigned long long xb =
+                  fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+              float xa0, xa1, xb0, xb1;
+              unpack2(xa, xa0, xa1);
+              unpack2(xb, xb0, xb1);
+              const float p0 = ex2(xa0), p1 = ex2(xa1), p2 = ex2(xb0), p3 = ex2(xb1);
+              acc_a = add2(acc_a, pack2(p0, p1));
+              acc_b = add2(acc_b, pack2(p2, p3));
+              r[2 * i] = pack_bf16(p0, p1);
+              r[2 * i + 1] = pack_bf16(p2, p3);
+            }
+            tmem_st32(tmem_s + 32, r + 32);
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars->p_half[X][1]));
+            if (tid == 0) BICACHE_STAMP(0, ti); if (tid == 128) BICACHE_STAMP(2, ti);
+            stored = true;
+          } else {
+            // redo with the new reference: S is still intact in TMEM
+            if (mx > m_ref + 8.f) {
+              alpha = ex2(m_ref - mx);
+              m_ref = mx;
+            }
+            unsigned s4[32];
+            const float neg_m = -m_ref;
+            float ps = 0.f;
+  #pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              tmem_ld32(tmem_s + c * 32, s4);
+              tmem_wait_ld();
+  #pragma unroll
+              for (int i = 0; i < 16; ++i) {
+                const float p0 = ex2(fmaf(__uint_as_float(s4[2 * i]), sl2, neg_m));
+                const float p1 = ex2(fmaf(__uint_as_float(s4[2 * i + 1]), sl2, neg_m));
+                ps += p0 + p1;
+                r[c * 16 + i] = pack_bf16(p0, p1);
+              }
+            }
+            acc_a = pack2(ps, 0.f);
+            acc_b = pack2(0.f, 0.f);
+            // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
+  #pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              tmem_ld32(tmem_o + c * 32, s4);
+              tmem_wait_ld();
+  #pragma unroll
+              for (int i = 0; i < 32; ++i) s4[i] = __float_as_uint(__uint_as_float(s4[i]) * alpha);
+              tmem_st32(tmem_o + c * 32, s4);
+            }
+          }
         } else {
-          // redo with the new reference: S is still intact in TMEM
-          if (mx > m_ref + 8.f) {
+          // First tile of the item, or a ragged tile: maximum first, every exponential on the exp
+          // unit so that masked columns give exactly 0.
+          if (cnt < kTileKeys) {
+  #pragma unroll
+            for (int i = 0; i < 128; ++i)
+              if (i >= cnt) r[i] = 0xff800000u;                // -inf: columns past the last key
+          }
+          float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+  #pragma unroll
+          for (int i = 0; i < 128; i += 8) {
+            mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+            mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+            mx2 = max3(mx2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+            mx3 = max3(mx3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+          }
+          const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sl2;   // scale > 0
+          if (j == 0) {
+            m_ref = mx;
+          } else if (mx > m_ref + 8.f) {
             alpha = ex2(m_ref - mx);
             m_ref = mx;
           }
-          unsigned s4[32];
-          const float neg_m = -m_ref;
-          float ps = 0.f;
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            tmem_ld32(tmem_s + c * 32, s4);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float p0 = ex2(fmaf(__uint_as_float(s4[2 * i]), sl2, neg_m));
-              const float p1 = ex2(fmaf(__uint_as_float(s4[2 * i + 1]), sl2, neg_m));
-              ps += p0 + p1;
-              r[c * 16 + i] = pack_bf16(p0, p1);
+          if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+  #pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              unsigned o[32];
+              tmem_ld32(tmem_o + c * 32, o);
+              tmem_wait_ld();
+  #pragma unroll
+              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+              tmem_st32(tmem_o + c * 32, o);
             }
           }
-          acc_a = pack2(ps, 0.f);
-          acc_b = pack2(0.f, 0.f);
-          // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            tmem_ld32(tmem_o + c * 32, s4);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) s4[i] = __float_as_uint(__uint_as_float(s4[i]) * alpha);
-            tmem_st32(tmem_o + c * 32, s4);
+          const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
+  #pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const unsigned long long xa =
+                fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+            const unsigned long long xb =
+                fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+            float x0, x1, x2, x3;
+            unpack2(xa, x0, x1);
+            unpack2(xb, x2, x3);
+            const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+            acc_a = add2(acc_a, pack2(p0, p1));
+            acc_b = add2(acc_b, pack2(p2, p3));
+            r[2 * i] = pack_bf16(p0, p1);
+            r[2 * i + 1] = pack_bf16(p2, p3);
           }
         }
-      } else {
-        // First tile of the item, or a ragged tile: maximum first, every exponential on the exp
-        // unit so that masked columns give exactly 0.
-        if (cnt < kTileKeys) {
-#pragma unroll
-          for (int i = 0; i < 128; ++i)
-            if (i >= cnt) r[i] = 0xff800000u;                // -inf: columns past the last key
+        if (!stored) {
+          tmem_st32(tmem_s, r);
+          tmem_st32(tmem_s + 32, r + 32);
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(smem_u32(&bars->p_half[X][0]));
+          mbar_arrive(smem_u32(&bars->p_half[X][1]));
         }
-        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < 128; i += 8) {
-          mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-          mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-          mx2 = max3(mx2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-          mx3 = max3(mx3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-        }
-        const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sl2;   // scale > 0
-        if (j == 0) {
-          m_ref = mx;
-        } else if (mx > m_ref + 8.f) {
-          alpha = ex2(m_ref - mx);
-          m_ref = mx;
-        }
-        if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll 1
-          for (int c = 0; c < 4; ++c) {
-            unsigned o[32];
-            tmem_ld32(tmem_o + c * 32, o);
-            tmem_wait_ld();
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-            tmem_st32(tmem_o + c * 32, o);
-          }
-        }
-        const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
-#pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const unsigned long long xa =
-              fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
-          const unsigned long long xb =
-              fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
-          float x0, x1, x2, x3;
-          unpack2(xa, x0, x1);
-          unpack2(xb, x2, x3);
-          const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-          acc_a = add2(acc_a, pack2(p0, p1));
-          acc_b = add2(acc_b, pack2(p2, p3));
-          r[2 * i] = pack_bf16(p0, p1);
-          r[2 * i + 1] = pack_bf16(p2, p3);
-        }
-      }
-      if (!stored) {
-        tmem_st32(tmem_s, r);
-        tmem_st32(tmem_s + 32, r + 32);
-        tmem_wait_st();
-        tc_fence_before();
-        mbar_arrive(smem_u32(&bars->p_half[X][0]));
-        mbar_arrive(smem_u32(&bars->p_half[X][1]));
-      }
-      {
-        float s0, s1, s2, s3;
-        unpack2(acc_a, s0, s1);
-        unpack2(acc_b, s2, s3);
-        l_sum = l_sum * alpha + ((s0 + s1) + (s2 + s3));
-      }
-    }
-    // ------------------------------- epilogue -------------------------------------------
-    const int prow = item.row0 + X * 128 + gt;       // packed row of this thread
-    const bool row_valid = prow < packed_rows;
-    const int a = prow / G;
-    const int h = item.kv_head * G + (prow - a * G);
-    if (ok && T > 0) {
-      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->o_done), 0, abort_flag));
-      if (ok) tc_fence_after();
-    }
-#ifdef BICACHE_TRACE
-    if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1003] = clock64();
-#endif
-    if (ok) {
-      const float inv = T > 0 ? 1.f / l_sum : 0.f;
-      const float lse = T > 0 ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
-      if (s.num_splits > 1) {
-        const long long pr = ((long long)item.split * t.total_tokens + req.tok_off + a) * t.Hq + h;
-        float* po = t.part_o + pr * 128;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          unsigned o[32];
-          if (T > 0) {
-            tmem_ld32(tmem_o + c * 32, o);
-            tmem_wait_ld();
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) o[i] = 0u;
-          }
-          if (row_valid) {
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-              float4 v4 = make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv,
-                                      __uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-              *reinterpret_cast<float4*>(po + c * 32 + i) = v4;
-            }
-          }
-        }
-        if (row_valid) t.part_lse[pr] = lse;
-      } else if (T > 0) {
-        // Each thread holds one output row; a row-per-thread store would touch 32 rows per
-        // instruction.  Stage the warp's 32 rows (256 bytes each) in this warp's quarter of the Q
-        // tile's shared memory (Q is no longer needed) and write them out two whole rows per
-        // instruction.  Chunks are XOR-placed by row to keep both directions conflict-light.
-        unsigned char* stage = smem + X * kTileBytes + (warp & 3) * 8192;
-#pragma unroll 1
-        for (int c = 0; c < 4; ++c) {
-          unsigned o[32];
-          tmem_ld32(tmem_o + c * 32, o);
-          tmem_wait_ld();
-#pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            uint4 v4;
-            v4.x = pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
-            v4.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-            v4.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
-            v4.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
-            const int cc = c * 4 + (i >> 3);
-            *reinterpret_cast<uint4*>(stage + lane * 256 + ((cc ^ (lane & 15)) << 4)) = v4;
-          }
-        }
-        __syncwarp();
         {
-          const int cc = lane & 15;
-          int row = lane >> 4;                                 // rows row, row + 2, ... of this warp
-          int prow2 = item.row0 + X * 128 + (warp & 3) * 32 + row;
-          const int a2 = prow2 / G;
-          int jj = prow2 - a2 * G;
-          const long long o_row_bytes = t.out_stride * 2;
-          char* dst_row = t.out + (req.row_off * t.out_stride + (long long)item.kv_head * G * 128) * 2 + cc * 16 +
-                          a2 * o_row_bytes;
-#pragma unroll 4
-          for (int it = 0; it < 16; ++it) {
-            const uint4 v4 = *reinterpret_cast<const uint4*>(stage + row * 256 + ((cc ^ (row & 15)) << 4));
-            if (prow2 < packed_rows) *reinterpret_cast<uint4*>(dst_row + jj * 256) = v4;
-            row += 2;
-            prow2 += 2;
-            jj += 2;
-            while (jj >= G) {
-              jj -= G;
-              dst_row += o_row_bytes;
+          float s0, s1, s2, s3;
+          unpack2(acc_a, s0, s1);
+          unpack2(acc_b, s2, s3);
+          l_sum = l_sum * alpha + ((s0 + s1) + (s2 + s3));
+        }
+        ++c_tile;
+      }
+      if (!ok) break;
+      // ------------------------------- epilogue -------------------------------------------
+      if (active) {
+        const int row0 = inf->row0, kv_head = inf->kv_head;
+        const long long row_off = inf->row_off;
+        const int packed_rows = g.n * G;
+        const int prow = row0 + X * 128 + gt;                // packed row of this thread
+        const bool row_valid = prow < packed_rows;
+        const int a = prow / G;
+        const int h = kv_head * G + (prow - a * G);
+        unsigned o[128];
+        if (T > 0) {
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->o_done[X]), e_item & 1, abort_flag));
+          if (!ok) break;
+          tc_fence_after();
+          ++e_item;
+          if (tid == 0) BICACHE_STAMP(0, ti); if (tid == 128) BICACHE_STAMP(2, ti);
+          tmem_ld32(tmem_o, o);
+          tmem_ld32(tmem_o + 32, o + 32);
+          tmem_ld32(tmem_o + 64, o + 64);
+          tmem_ld32(tmem_o + 96, o + 96);
+          tmem_wait_ld();
+          tc_fence_before();
+          mbar_arrive(smem_u32(&bars->o_free[X]));           // the next item may overwrite O
+        } else {
+#pragma unroll
+          for (int i = 0; i < 128; ++i) o[i] = 0u;
+        }
+        const float inv = T > 0 ? 1.f / l_sum : 0.f;
+        const float lse = T > 0 ? (m_ref + log2f(l_sum)) * 0.6931471805599453f : -INFINITY;
+        if (s.num_splits > 1) {
+          // key-split call: normalised fp32 partial and its lse, merged by a second kernel
+          if (row_valid) {
+            const long long pr = ((long long)inf->split * t.total_tokens + inf->tok_off + a) * t.Hq + h;
+            float* po = t.part_o + pr * 128;
+#pragma unroll
+            for (int i = 0; i < 128; i += 4)
+              *reinterpret_cast<float4*>(po + i) =
+                  make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv,
+                              __uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+            t.part_lse[pr] = lse;
+          }
+        } else if (T > 0) {
+          // Each thread holds one output row.  The warp stages its 32 rows, one 64-dim half at a
+          // time (128 bytes per row, 16-byte chunks XOR-placed by row: the 128-byte swizzle), and
+          // one TMA store writes the half out; a warp whose rows are not all valid, or a head
+          // grouping the box cannot express, copies the staged rows out itself, four rows per
+          // instruction.
+          const int p0w = row0 + X * 128 + (warp & 3) * 32;  // first packed row of this warp
+          const bool by_tma = o_tma && p0w + 32 <= packed_rows;
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            if (lane == 0) bulk_wait_read();                 // the previous store has read the staging rows
+            __syncwarp();
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              const int i = hh * 64 + c * 8;
+              uint4 v4;
+              v4.x = pack_bf16(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv);
+              v4.y = pack_bf16(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+              v4.z = pack_bf16(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+              v4.w = pack_bf16(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+              *reinterpret_cast<uint4*>(stage + lane * 128 + ((c ^ (lane & 7)) << 4)) = v4;
+            }
+            if (by_tma) {
+              fence_proxy_async();
+              __syncwarp();
+              if (lane == 0) {
+                tma_store_3d(&tm_o, smem_u32(stage), hh * 64, kv_head * G, (int)row_off + p0w / G);
+                bulk_commit_group();
+              }
+            } else {
+              __syncwarp();
+              const int ch = lane & 7;
+#pragma unroll 2
+              for (int it = 0; it < 8; ++it) {
+                const int row = it * 4 + (lane >> 3);
+                const int pr = p0w + row;
+                if (pr < packed_rows) {
+                  const int a2 = pr / G, jj = pr - a2 * G;
+                  char* dst = t.out + ((row_off + a2) * t.out_stride + (long long)(kv_head * G + jj) * 128 + hh * 64) * 2 +
+                              ch * 16;
+                  *reinterpret_cast<uint4*>(dst) =
+                      *reinterpret_cast<const uint4*>(stage + row * 128 + ((ch ^ (row & 7)) << 4));
+                }
+              }
+              __syncwarp();
             }
           }
+          if (row_valid && t.lse != nullptr) t.lse[(row_off + a) * t.Hq + h] = lse;
         }
-        if (row_valid && t.lse != nullptr) t.lse[(req.row_off + a) * t.Hq + h] = lse;
+        if (tid == 0) BICACHE_STAMP(0, ti); if (tid == 128) BICACHE_STAMP(2, ti);
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->info_free[n_it & 1]));
+      ++n_it;
     }
+    if (lane == 0) bulk_wait_all();                          // the output stores of this warp have completed
     tc_fence_before();
-  } else if (warp >= 9) {
+  } else if (warp == 9) {
+    // ============================== item fetch and Q loads ===============================
+    // Lane 0 writes the record of the CTA's first item (its block index) and, while item n is
+    // computed, fetches item n + 1 from the shared counter.  The warp loads the Q tiles of item n
+    // as soon as the last S of item n - 1 has been computed.
+    bool ok = !dead;
+    int n_it = 0;
+    int eq[2] = {0, 0};          // items each query tile has taken part in (phase of q_free / q_full)
+    auto write_info = [&](ItemInfo* dst, int idx) {
+      if (idx < s.num_items) {
+        const WorkItem wi = s.items[idx];
+        const ReqMeta rq = s.reqs[wi.req];
+        dst->kv_head = wi.kv_head;
+        dst->row0 = wi.row0;
+        dst->split = wi.split;
+        dst->n = rq.n;
+        dst->m = rq.m;
+        dst->page_off = rq.page_off;
+        dst->tok_off = rq.tok_off;
+        dst->row_off = rq.row_off;
+        dst->valid = 1;
+      } else {
+        dst->valid = 0;
+      }
+    };
+    if (ok && lane == 0) {
+      write_info(&bars->info[0], (int)blockIdx.x);
+      mbar_arrive(smem_u32(&bars->info_full[0]));
+    }
+    __syncwarp();
+    while (ok) {
+      const ItemInfo* inf = &bars->info[n_it & 1];
+      const Geo g = read_geo_uniform(inf, s.num_splits, s.tiles_per_split, G);
+      if (!g.valid) break;
+      if (g.T > 0) {
+        const int packed_rows = g.n * G;
+        for (int x = 0; x < 2 && ok; ++x) {
+          if (x == 1 && !g.b_active) break;
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_free[x]), (eq[x] & 1) ^ 1, abort_flag));
+          if (!ok) break;
+          ++eq[x];
+          const unsigned qf = smem_u32(&bars->q_full[x]);
+          const unsigned q_dst = q_smem + x * kTileBytes;
+          if (q_tma) {
+            // 128 packed rows = 128 / G tokens x G heads of the KV group: one TMA box per 64-dim half,
+            // in the dense swizzled layout (row r at r * 128 bytes, halves 16 KB apart)
+            if (lane == 0) {
+              const int tok = (int)inf->row_off + (inf->row0 + x * 128) / G;
+              mbar_arrive_expect_tx(qf, (unsigned)kTileBytes);
+              tma_load_3d(q_dst, &tm_q, 0, inf->kv_head * G, tok, qf);
+              tma_load_3d(q_dst + kTileBytes / 2, &tm_q, 64, inf->kv_head * G, tok, qf);
+            } else {
+              mbar_arrive(qf);
+            }
+          } else {
+            // gathers into the page-image layout: packed row p = token a * G + head jj of the KV
+            // group; rows past the end are zero-filled
+            const int r0 = lane >> 4, c16 = lane & 15;
+            int prow = inf->row0 + x * 128 + r0;
+            const int a0 = prow / G;
+            int jj = prow - a0 * G;
+            const long long q_row_bytes = t.q_stride * 2;
+            const char* q_base = t.q + (inf->row_off * t.q_stride + (long long)inf->kv_head * G * 128) * 2 + c16 * 16;
+            const char* src_row = q_base + a0 * q_row_bytes;
+#pragma unroll 4
+            for (int i = 0; i < 64; ++i) {
+              const bool valid = prow < packed_rows;
+              cp_async16(q_dst + tile_chunk_offset(r0 + 2 * i, c16), valid ? src_row + jj * 256 : q_base, valid ? 16u : 0u);
+              prow += 2;
+              jj += 2;
+              while (jj >= G) {                         // at most twice (G >= 1)
+                jj -= G;
+                src_row += q_row_bytes;
+              }
+            }
+            cp_async_commit();
+            cp_async_wait<0>();
+            fence_proxy_async();
+            mbar_arrive(qf);
+          }
+        }
+        if (!ok) break;
+      }
+      // the next item: its record slot must have been released by every role (item n - 1)
+      if (lane == 0) {
+        const int nn = n_it + 1;
+        ok = mbar_wait(smem_u32(&bars->info_free[nn & 1]), ((nn >> 1) & 1) ^ 1, abort_flag);
+        if (ok) {
+          write_info(&bars->info[nn & 1], (int)gridDim.x + atomicAdd(next_item, 1));
+          mbar_arrive(smem_u32(&bars->info_full[nn & 1]));
+        }
+      }
+      ok = __all_sync(0xffffffffu, ok);
+      __syncwarp();                                          // lane 0's record is visible to the warp
+      ++n_it;
+    }
+  } else if (warp >= 10) {
     // ====================================== loads =======================================
-    // Three load warps, each responsible for whole tiles: warp w takes ring uses u = w, w + 3, ...
-    // (u = 2 j: K of key tile j, u = 2 j + 1: V of key tile j).  A warp issues its tile, waits for
-    // it to land, fences and signals, while the other two warps are already issuing theirs.
-    const int w = warp - 9;
-    // A 128-row tile is fetched as 64 passes of 2 rows: lane l takes 16-byte chunk (l & 15) of rows
-    // (l >> 4) + 2 i.  In the tile image, rows r, r + 8, r + 16, ... are 2048 bytes apart.
+    // Warp 10 stages the K tiles, warp 11 the V tiles, each running ahead of the MMAs by the depth
+    // of the ring (K0 V0 K1 V1) and on into the next item.  Ring uses are counted over the whole
+    // life of the CTA: use u = 2 * (key tiles before) + (0: K, 1: V).
+    const int is_v = warp - 10;
+    // A gathered 128-row tile is fetched as 64 passes of 2 rows: lane l takes 16-byte chunk (l & 15)
+    // of rows (l >> 4) + 2 i.  In the tile image, rows r, r + 8, r + 16, ... are 2048 bytes apart.
     const int r0 = lane >> 4, c16 = lane & 15;
     unsigned dst_q[4];
 #pragma unroll
     for (int q = 0; q < 4; ++q) dst_q[q] = tile_chunk_offset(r0 + 2 * q, c16);
     bool ok = !dead;
-    int ti = 0; (void)ti;
-    const int* pages = s.pages + req.page_off;
-    for (int u = w; u < 2 * T && ok; u += 3) {
-      const int slot = u % kRing;
-      const int jg = tile_begin + (u >> 1);
-      const bool is_v = u & 1;
-      ok = mbar_wait(smem_u32(&bars->free_[slot]), ((u / kRing) & 1) ^ 1, abort_flag);
+    int n_it = 0, U = 0;
+    int armed[kRing] = {-1, -1, -1, -1};     // the last use armed with bulk copies, per slot
+    while (ok) {
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->info_full[n_it & 1]), (n_it >> 1) & 1, abort_flag));
       if (!ok) break;
-      const unsigned dst = ring_smem + slot * kTileBytes;
-      const unsigned full = smem_u32(&bars->full[slot]);
-      if (jg < prefix_tiles) {
-        // cached prefix tile: one bulk copy per page; a pool page already is the tile image
-        const int cnt = min(kTileKeys, req.m - jg * kTileKeys);
-        const int npages = (cnt + kPageSize - 1) / kPageSize;
-        if (lane == 0) {
-          const char* pool_base = is_v ? pool.v : pool.k;
-          mbar_arrive_expect_tx(full, (unsigned)(npages * kPageBytes));
-          for (int pg = 0; pg < npages; ++pg)
-            bulk_copy_g2s(dst + pg * kPageBytes,
-                          pool_base + pool_slice_offset(pool, t.layer, pages[jg * 8 + pg], item.kv_head),
-                          kPageBytes, full);
-        } else {
-          mbar_arrive(full);
+      const ItemInfo* inf = &bars->info[n_it & 1];
+      const Geo g = read_geo_uniform(inf, s.num_splits, s.tiles_per_split, G);
+      if (!g.valid) break;
+      const int kv_head = inf->kv_head;
+      const long long row_off = inf->row_off;
+      const int* pages = s.pages + inf->page_off;
+      for (int j = 0; j < g.T; ++j) {
+        const int u = U + 2 * j + is_v;
+        const int slot = u % kRing;
+        const int jg = g.tile_begin + j;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->free_[slot]), ((u / kRing) & 1) ^ 1, abort_flag));
+        if (!ok) break;
+        const unsigned dst = ring_smem + slot * kTileBytes;
+        const unsigned full = smem_u32(&bars->full[slot]);
+        if (jg < g.prefix_tiles) {
+          // cached prefix tile: one bulk copy per page (a pool page already is the tile image), each
+          // issued by its own lane so that the page-table reads overlap
+          const int cnt = min(kTileKeys, g.m - jg * kTileKeys);
+          const int npages = (cnt + kPageSize - 1) / kPageSize;
+          if (lane < npages) {
+            const char* pool_base = is_v ? pool.v : pool.k;
+            bulk_copy_g2s(dst + lane * kPageBytes,
+                          pool_base + pool_slice_offset(pool, t.layer, pages[jg * 8 + lane], kv_head), kPageBytes, full);
+          }
+          // every lane arrives, so the phase cannot complete before lane 0 has announced the bytes
+          if (lane == 0) {
+            mbar_arrive_expect_tx(full, (unsigned)(npages * kPageBytes));
+            armed[slot] = u;
+          } else {
+            mbar_arrive(full);
+          }
+          continue;
         }
-      } else {
-        // own rows: 16-byte gathers from row-major K/V into the image, zero-filled past the end
-        const int key0 = (jg - prefix_tiles) * kTileKeys;
-        const int cnt = min(kTileKeys, req.n - key0);
-        const char* row0 = (is_v ? t.v : t.k) +
-                           ((req.row_off + key0) * t.kv_stride + (long long)item.kv_head * 128) * 2 + c16 * 16;
-        const long long row_bytes = t.kv_stride * 2;
-        const char* src = row0 + r0 * row_bytes;
+        const int key0 = (jg - g.prefix_tiles) * kTileKeys;
+        const int cnt = min(kTileKeys, g.n - key0);
         if (cnt >= kTileKeys) {
           // a full tile of the request's own rows: two TMA boxes (dense swizzled layout)
           if (lane == 0) {
-            const int row = (int)req.row_off + key0;
+            const int row = (int)row_off + key0;
             const void* tm = is_v ? (const void*)&tm_v : (const void*)&tm_k;
             mbar_arrive_expect_tx(full, (unsigned)kTileBytes);
-            tma_load_3d(dst, tm, 0, item.kv_head, row, full);
-            tma_load_3d(dst + kTileBytes / 2, tm, 64, item.kv_head, row, full);
+            tma_load_3d(dst, tm, 0, kv_head, row, full);
+            tma_load_3d(dst + kTileBytes / 2, tm, 64, kv_head, row, full);
+            armed[slot] = u;
           } else {
             mbar_arrive(full);
           }
           continue;
         }
         // ragged last tile: 16-byte gathers into the page-image layout, zero-filled past the end
+        const char* rowp = (is_v ? t.v : t.k) + ((row_off + key0) * t.kv_stride + (long long)kv_head * 128) * 2 + c16 * 16;
+        const long long row_bytes = t.kv_stride * 2;
+        const char* src = rowp + r0 * row_bytes;
 #pragma unroll 4
         for (int i = 0; i < 64; ++i) {
           const bool valid = r0 + 2 * i < cnt;
-          cp_async16(dst + dst_q[i & 3] + (i >> 2) * 2048, valid ? src : row0, valid ? 16u : 0u);
+          cp_async16(dst + dst_q[i & 3] + (i >> 2) * 2048, valid ? src : rowp, valid ? 16u : 0u);
           src += 2 * row_bytes;
         }
         cp_async_commit();
-        if (w == 0 && lane == 0) BICACHE_STAMP(2, ti);
         cp_async_wait<0>();
         fence_proxy_async();
         mbar_arrive(full);
-        if (w == 0 && lane == 0) BICACHE_STAMP(2, ti);
       }
+      if (!ok) break;
+      U += 2 * g.T;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->info_free[n_it & 1]));
+      ++n_it;
     }
     cp_async_wait<0>();
     // On the normal path every tile loaded has been consumed by the time the CTA ends (the
     // epilogue waits for the last MMA).  After a give-up, bulk copies may still be in flight:
     // wait (bounded) for the last barriers this lane armed.
     if (!dead && (!ok || *abort_flag) && lane == 0) {
-      for (int u = max(0, 2 * T - kRing); u < 2 * T; ++u)
-        if (u % 3 == w && tile_begin + (u >> 1) < prefix_tiles)
-          for (unsigned it = 0; it < 4096 && !mbar_try_wait(smem_u32(&bars->full[u % kRing]), (u / kRing) & 1); ++it)
+      for (int i = 0; i < kRing; ++i)
+        if (armed[i] >= 0)
+          for (unsigned it = 0;
+               it < 4096 && !mbar_try_wait(smem_u32(&bars->full[armed[i] % kRing]), (armed[i] / kRing) & 1); ++it)
             __nanosleep(256);
     }
   } else if (warp == kMmaWarp) {
     // ===================================== MMA issue =====================================
-    // The whole warp runs this control flow converged and one elected lane issues each tcgen05
-    // instruction: descriptor arithmetic then stays in the uniform datapath and the MMAs can be
-    // issued back to back (a single diverged lane cannot feed the tensor pipe fast enough).
-    if (!dead && T > 0) {
-      const unsigned tmem_s2[2] = {tmem, tmem + 128};
-      const unsigned tmem_o2[2] = {tmem + 256, tmem + 384};
+    // The whole warp runs this control flow converged and one elected lane issues each batch of
+    // tcgen05 instructions.  Issue order inside an item:
+    //   S_A(0) S_B(0) | O_A(0) S_A(1) | O_B(0) S_B(1) | O_A(1) S_A(2) | ...
+    // O_X(j) += P_X V is issued in two halves as P arrives, and the next S_X = Q_X K^T follows it
+    // back to back (it overwrites P_X; the tensor pipe runs MMAs in issue order).  After the last
+    // O_X of an item the next S_X is the first one of the next item.  Alternating between the two
+    // tiles keeps their softmaxes half a period apart, which the exp unit they share needs.
+    // This warp shares its scheduler with two busy softmax warps and gets through its own
+    // instructions slowly, so everything but the MMAs - waits for K/V tiles, descriptors, what
+    // follows each O - sits in the shadow of the waits for the second half of P.
+    bool ok = !dead;
+    if (ok) {
+      const unsigned bar_full = smem_u32(&bars->full[0]), bar_free = smem_u32(&bars->free_[0]);   // slot i: + 8 i
+      const unsigned bar_p = smem_u32(&bars->p_half[0][0]);     // [x][half]: + 16 x + 8 half
+      const unsigned bar_s = smem_u32(&bars->s_full[0]), bar_qfull = smem_u32(&bars->q_full[0]);   // [x]: + 8 x
+      const unsigned bar_qfree = smem_u32(&bars->q_free[0]), bar_odone = smem_u32(&bars->o_done[0]);
+      const unsigned bar_ofree = smem_u32(&bars->o_free[0]);
       // Two shared-memory layouts occur (see make_desc): the page image (cached tiles, gathered ragged
       // tiles, gathered Q) and the dense layout TMA writes (full own-row tiles, TMA-loaded Q): 8-row
-      // groups 1024 bytes apart, the two 64-dim halves 16 KB apart.
-      const unsigned q_sbo = q_tma ? 1024u : 2048u, q_hi = q_tma ? 1024u : 64u;
-      const unsigned long long q_desc[2] = {make_desc(q_smem, 16, q_sbo), make_desc(q_smem + kTileBytes, 16, q_sbo)};
-      const int nx = b_active ? 2 : 1;
-      // a key tile is in the dense (TMA) layout iff it is a full tile of the request's own rows
-      auto dense_tile = [&](int jt) {
-        const int jgt = tile_begin + jt;
-        return jgt >= prefix_tiles && req.n - (jgt - prefix_tiles) * kTileKeys >= kTileKeys;
+      // groups 1024 bytes apart, the two 64-dim halves 16 KB apart.  Descriptors of ring slot 0 in
+      // both layouts; slot i adds i * (tile bytes / 16) to the address field.
+      const unsigned q_hi = q_tma ? 1024u : 64u;
+      const unsigned long long q_desc0 = make_desc(q_smem, 16, q_tma ? 1024u : 2048u);
+      const unsigned long long q_desc1 = q_desc0 + (kTileBytes >> 4);
+      const unsigned long long kb_img = make_desc(ring_smem, 16, 2048), kb_dense = make_desc(ring_smem, 16, 1024);
+      const unsigned long long vb_img = make_desc(ring_smem, 1024, 2048), vb_dense = make_desc(ring_smem, 16384, 1024);
+      constexpr unsigned kSlotUnits = kTileBytes >> 4;
+      const unsigned tmem_u = __shfl_sync(0xffffffffu, tmem, 0);   // warp-uniform copy of the TMEM base
+      const unsigned tmem_s1 = tmem_u + 128, tmem_o0 = tmem_u + 256, tmem_o1 = tmem_u + 384;
+#define BICACHE_WAIT(bar, parity) __all_sync(0xffffffffu, mbar_wait((bar), (parity), abort_flag))
+      // the eight MMAs (K steps of 16 dims) of S_X = Q_X K^T
+      auto issue_s = [&](unsigned d_tmem, unsigned long long qd, unsigned long long kd, unsigned k_hi) {
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          mma_ss_elect(d_tmem, qd + (k >> 2) * q_hi + (k & 3) * 2, kd + (k >> 2) * k_hi + (k & 3) * 2, kIdescQK,
+                       k > 0 ? 1u : 0u);
       };
-      bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_full), 0, abort_flag));
+      int n_it = 0;
+      int c0 = 0, c1 = 0;        // key tiles each query tile has been through (phase of p_half)
+      int e0 = 0, e1 = 0;        // items each query tile has taken part in (phase of q_full / o_free)
+      unsigned u = 0;            // ring use of the current key tile's K; its V is u + 1, the next tile's K u + 2
       int ti = 0; (void)ti;
-      if (lane == 0) BICACHE_STAMP(1, ti);
-      // Issue order: S_A(0) S_B(0) | O_A(0) S_A(1) | O_B(0) S_B(1) | O_A(1) S_A(2) | ...
-      // O_X(j) += P_X V is issued in two halves as P arrives, and S_X(j+1) = Q_X K^T follows it
-      // back to back (it overwrites P_X; the tensor pipe runs MMAs in issue order).  The K/V tiles
-      // an iteration needs are waited for before the wait on P, so nothing stands between the
-      // arrival of P and the MMAs.
-      // prologue: S_X(0)
-      ok = ok && __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[0]), 0, abort_flag));
-      if (ok) {
-        fence_proxy_async();
-        tc_fence_after();
-        const bool kd0 = dense_tile(0);
-        const unsigned k_hi0 = kd0 ? 1024u : 64u;
-        const unsigned long long k_desc = make_desc(ring_smem, 16, kd0 ? 1024u : 2048u);
-        for (int x = 0; x < nx; ++x) {
-          if (x == 1) {
-            // Stagger the two query tiles by half a period: tile B starts when tile A's softmax is
-            // half done, so that afterwards each tile's softmax runs while the tensor pipe works for
-            // the other tile (started together, the two softmaxes share the exp unit and the MMAs
-            // of both tiles then queue behind each other).
-            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[0][0]), 0, abort_flag));
+      ok = BICACHE_WAIT(smem_u32(&bars->info_full[0]), 0);
+      Geo cur = read_geo_uniform(&bars->info[0], s.num_splits, s.tiles_per_split, G);
+      bool pre = false;          // the first S of the current item was issued at the end of the previous one
+      while (ok && cur.valid) {
+        Geo nxt;
+        nxt.valid = 0;
+        bool have_next = false, can_pre = false;
+        const int T = cur.T;
+        if (T > 0) {
+          const bool b_on = cur.b_active;
+          bool dn = tile_dense(cur, 0);                        // layout of the current key tile
+          if (!pre) {
+            // the first S of an item that could not be issued ahead (the CTA's first item)
+            ok = BICACHE_WAIT(bar_full + (u & 3) * 8, (u >> 2) & 1) && BICACHE_WAIT(bar_qfull, e0 & 1);
             if (!ok) break;
-          }
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            mma_ss_elect(tmem_s2[x], q_desc[x] + (k >> 2) * q_hi + (k & 3) * 2, k_desc + (k >> 2) * k_hi0 + (k & 3) * 2,
-                         kIdescQK, k > 0 ? 1u : 0u);
-          mma_commit_elect(smem_u32(&bars->s_full[x]));
-        }
-        if (ok) mma_commit_elect(smem_u32(&bars->free_[0]));
-      }
-      for (int j = 0; j < T && ok; ++j) {
-        const int jg = tile_begin + j;
-        const int cnt = jg < prefix_tiles ? min(kTileKeys, req.m - jg * kTileKeys)
-                                          : min(kTileKeys, req.n - (jg - prefix_tiles) * kTileKeys);
-        const int ksteps = (cnt + 15) >> 4;
-        const int uv = 2 * j + 1, un = 2 * j + 2;          // ring uses: V of tile j, K of tile j + 1
-        const int slot_v = uv % kRing, slot_n = un % kRing;
-        const bool more = j + 1 < T;
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_v]), (uv / kRing) & 1, abort_flag));
-        if (ok && more)
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->full[slot_n]), (un / kRing) & 1, abort_flag));
-        if (!ok) break;
-        fence_proxy_async();
-        const bool vd = dense_tile(j), kd = more && dense_tile(j + 1);
-        const unsigned long long v_desc = vd ? make_desc(ring_smem + slot_v * kTileBytes, 16384, 1024)
-                                             : make_desc(ring_smem + slot_v * kTileBytes, 1024, 2048);
-        const unsigned v_step = vd ? 128u : 256u;          // 16 keys further, in 16-byte units
-        const unsigned long long k_desc = make_desc(ring_smem + slot_n * kTileBytes, 16, kd ? 1024u : 2048u);
-        const unsigned k_hi = kd ? 1024u : 64u;
-        const unsigned acc0 = j > 0 ? 1u : 0u;
-        for (int x = 0; x < nx && ok; ++x) {
-          // O_X += P_X V, 16 keys (one page image) per MMA; P is the A operand, read from TMEM
-#pragma unroll
-          for (int half = 0; half < 2; ++half) {
-            ok = ok && __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->p_half[x][half]), j & 1, abort_flag));
-            if (ok) {
-              if (lane == 0 && x == 0 && half == 0) BICACHE_STAMP(1, ti);
-              tc_fence_after();
-#pragma unroll
-              for (int k = half * 4; k < half * 4 + 4; ++k)
-                mma_ts_elect(tmem_o2[x], tmem_s2[x] + k * 8, v_desc + k * v_step, kIdescPV,
-                             k > 0 ? 1u : acc0, k < ksteps ? 1u : 0u);
+            tc_fence_after();
+            const unsigned long long kd0 = (dn ? kb_dense : kb_img) + (u & 3) * kSlotUnits;
+            issue_s(tmem_u, q_desc0, kd0, dn ? 1024u : 64u);
+            mma_commit_elect(bar_s);
+            if (T == 1) mma_commit_elect(bar_qfree);
+            if (b_on) {
+              // Stagger the two query tiles by half a period: tile B starts when tile A's softmax is
+              // half done (started together, the two softmaxes share the exp unit and the MMAs of
+              // both tiles then queue behind each other).
+              ok = BICACHE_WAIT(bar_p, c0 & 1) && BICACHE_WAIT(bar_qfull + 8, e1 & 1);
+              if (!ok) break;
+              issue_s(tmem_s1, q_desc1, kd0, dn ? 1024u : 64u);
+              mma_commit_elect(bar_s + 8);
+              if (T == 1) mma_commit_elect(bar_qfree + 8);
             }
+            mma_commit_elect(bar_free + (u & 3) * 8);
           }
+          // V of the first key tile; the previous item's epilogue must have read O_A out of TMEM
+          ok = BICACHE_WAIT(bar_full + ((u + 1) & 3) * 8, ((u + 1) >> 2) & 1) && BICACHE_WAIT(bar_ofree, (e0 & 1) ^ 1);
           if (!ok) break;
-          // S_X of the next key tile
-          if (more) {
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-              mma_ss_elect(tmem_s2[x], q_desc[x] + (k >> 2) * q_hi + (k & 3) * 2, k_desc + (k >> 2) * k_hi + (k & 3) * 2,
-                           kIdescQK, k > 0 ? 1u : 0u);
-            mma_commit_elect(smem_u32(&bars->s_full[x]));
-          }
-          if (lane == 0 && x == 0) BICACHE_STAMP(1, ti);
+          int ksteps = (tile_keys(cur, 0) + 15) >> 4;
+          // One key tile.  The body exists twice: the lean one for every tile but the last, and the
+          // one for the last tile, which also looks at the next item.
+          auto tile_iter = [&](auto last_c, int j) {
+            constexpr bool last = decltype(last_c)::value;
+            const unsigned sv = (u + 1) & 3, sn = (u + 2) & 3;  // ring slots: V of this tile, K of the next
+            const unsigned long long v_desc = (dn ? vb_dense : vb_img) + sv * kSlotUnits;
+            const unsigned v_step = dn ? 128u : 256u;           // 16 keys further, in 16-byte units
+            const unsigned acc0 = j > 0 ? 1u : 0u;
+            // ---- tile A: first half of O += P V as soon as P of keys 0-63 is there ----
+            ok = BICACHE_WAIT(bar_p, c0 & 1);
+            if (!ok) return;
+            if (lane == 0) BICACHE_STAMP(1, ti);
+            tc_fence_after();
+            #pragma unroll
+              for (int k = 0; k < 4; ++k)
+                mma_ts_elect(tmem_o0, tmem_u + k * 8, v_desc + k * v_step, kIdescPV, k > 0 ? 1u : acc0, k < ksteps ? 1u : 0u);
+            if (lane == 0) BICACHE_STAMP(1, ti);
+            // ---- shadow of A's second half of the exponentials: what follows the O of this iteration ----
+            bool s_on0 = true, s_on1 = b_on;                   // an S follows O_A / O_B
+            bool q_last = j + 2 == T;                           // ... and it is the last S of its item
+            bool dn_next;
+            if (!last) {
+              dn_next = tile_dense(cur, j + 1);
+            } else {
+              // the next item (fetched long ago): its first S follows this item's last O
+              const int nn = n_it + 1;
+              ok = BICACHE_WAIT(smem_u32(&bars->info_full[nn & 1]), (nn >> 1) & 1);
+              if (!ok) return;
+              nxt = read_geo_uniform(&bars->info[nn & 1], s.num_splits, s.tiles_per_split, G);
+              have_next = true;
+              can_pre = nxt.valid && nxt.T > 0;
+              s_on0 = can_pre;
+              s_on1 = can_pre && nxt.b_active;
+              q_last = nxt.T == 1;
+              dn_next = can_pre && tile_dense(nxt, 0);
+            }
+            if (s_on0) {
+              ok = BICACHE_WAIT(bar_full + sn * 8, ((u + 2) >> 2) & 1);
+              if (!ok) return;
+            }
+            const unsigned long long k_desc = (dn_next ? kb_dense : kb_img) + sn * kSlotUnits;
+            const unsigned k_hi = dn_next ? 1024u : 64u;
+            if (lane == 0) BICACHE_STAMP(1, ti);
+            // ---- tile A: second half, then the next S_A back to back ----
+            ok = BICACHE_WAIT(bar_p + 8, c0 & 1);
+            if (!ok) return;
+            if (lane == 0) BICACHE_STAMP(1, ti);
+            tc_fence_after();
+            #pragma unroll
+              for (int k = 4; k < 8; ++k)
+                mma_ts_elect(tmem_o0, tmem_u + k * 8, v_desc + k * v_step, kIdescPV, 1u, k < ksteps ? 1u : 0u);
+            ++c0;
+            if (last) {
+              mma_commit_elect(bar_odone);
+              ++e0;
+            }
+            if (s_on0) {
+              if (last) {
+                ok = BICACHE_WAIT(bar_qfull, e0 & 1);           // the next item's Q tile must have landed
+                if (!ok) return;
+              }
+              issue_s(tmem_u, q_desc0, k_desc, k_hi);
+              mma_commit_elect(bar_s);
+              if (q_last) mma_commit_elect(bar_qfree);
+            }
+            if (lane == 0) BICACHE_STAMP(1, ti);
+            // ---- tile B: first half ----
+            if (b_on) {
+              if (j == 0) {
+                ok = BICACHE_WAIT(bar_ofree + 8, (e1 & 1) ^ 1);  // the previous epilogue has read O_B
+                if (!ok) return;
+              }
+              ok = BICACHE_WAIT(bar_p + 16, c1 & 1);
+              if (!ok) return;
+              if (lane == 0) BICACHE_STAMP(1, ti);
+              tc_fence_after();
+              #pragma unroll
+                for (int k = 0; k < 4; ++k)
+                  mma_ts_elect(tmem_o1, tmem_s1 + k * 8, v_desc + k * v_step, kIdescPV, k > 0 ? 1u : acc0,
+                               k < ksteps ? 1u : 0u);
+            }
+            // ---- shadow of B's second half: the next tile's key count ----
+            const int ks_next = last ? 8 : (tile_keys(cur, j + 1) + 15) >> 4;
+            // ---- tile B: second half, then the next S_B ----
+            if (b_on) {
+              ok = BICACHE_WAIT(bar_p + 24, c1 & 1);
+              if (!ok) return;
+              tc_fence_after();
+              #pragma unroll
+                for (int k = 4; k < 8; ++k)
+                  mma_ts_elect(tmem_o1, tmem_s1 + k * 8, v_desc + k * v_step, kIdescPV, 1u, k < ksteps ? 1u : 0u);
+              ++c1;
+              if (last) {
+                mma_commit_elect(bar_odone + 8);
+                ++e1;
+              }
+            }
+            if (s_on1) {
+              if (last) {
+                ok = BICACHE_WAIT(bar_qfull + 8, e1 & 1);
+                if (!ok) return;
+              }
+              issue_s(tmem_s1, q_desc1, k_desc, k_hi);
+              mma_commit_elect(bar_s + 8);
+              if (q_last) mma_commit_elect(bar_qfree + 8);
+            }
+            if (lane == 0) BICACHE_STAMP(1, ti);
+            // release V of this tile and K of the next
+            mma_commit_elect(bar_free + sv * 8);
+            if (s_on0) mma_commit_elect(bar_free + sn * 8);
+            u += 2;
+            dn = dn_next;
+            ksteps = ks_next;
+            // V of the next key tile (its slot was released one iteration ago: it lands about now)
+            if (!last) {
+              ok = BICACHE_WAIT(bar_full + ((u + 1) & 3) * 8, ((u + 1) >> 2) & 1);
+              if (!ok) return;
+            }
+          };
+          for (int j = 0; j + 1 < T && ok; ++j) tile_iter(std::false_type{}, j);
+          if (ok) tile_iter(std::true_type{}, T - 1);
+          if (!ok) break;
         }
-        if (!ok) break;
-        mma_commit_elect(smem_u32(&bars->free_[slot_v]));
-        if (more) mma_commit_elect(smem_u32(&bars->free_[slot_n]));
+        // done with this item's record; move on
+        if (!have_next) {
+          const int nn = n_it + 1;
+          ok = BICACHE_WAIT(smem_u32(&bars->info_full[nn & 1]), (nn >> 1) & 1);
+          if (!ok) break;
+          nxt = read_geo_uniform(&bars->info[nn & 1], s.num_splits, s.tiles_per_split, G);
+        }
+        if (elect_one()) mbar_arrive(smem_u32(&bars->info_free[n_it & 1]));
+        __syncwarp();
+        pre = can_pre;
+        cur = nxt;
+        ++n_it;
       }
-      if (ok) mma_commit_elect(smem_u32(&bars->o_done));
+#undef BICACHE_WAIT
       // Whatever happened, let every MMA issued so far finish before TMEM is released.
       __syncwarp();
       mma_commit_elect(smem_u32(&bars->drain));
@@ -916,7 +1191,16 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);
   }
-  if (tid == 0 && !dead && *abort_flag) atomicCAS(status, kDevOk, kDevTimeout);
+  if (tid == 0) {
+    if (!dead && *abort_flag) atomicCAS(status, kDevOk, kDevTimeout);
+    // the last CTA to finish rewinds the item counter for the next launch
+    __threadfence();
+    if (atomicAdd(ctas_done, 1) == (int)gridDim.x - 1) {
+      *next_item = 0;
+      *ctas_done = 0;
+      __threadfence();
+    }
+  }
 }
 
 inline cudaError_t configure_tc_attention() {
@@ -930,17 +1214,21 @@ inline cudaError_t configure_tc_attention() {
 }
 
 // Tensor maps of one call: q [rows][Hq][128] with a box of (64 dims, G heads, 128 / G rows) so that
-// a box is 128 packed rows; k, v [rows][Hkv][128] with a box of (64 dims, 1 head, 128 rows).
+// a box is 128 packed rows; k, v [rows][Hkv][128] with a box of (64 dims, 1 head, 128 rows); out like
+// q with a box of 32 packed rows (the rows of one softmax warp).
 struct TcTensorMaps {
-  CUtensorMap q, k, v;
+  CUtensorMap q, k, v, o;
   int q_tma;                 // 0: G does not divide 128, Q is gathered instead
+  int o_tma;                 // 0: G does not divide 32, the output rows are copied out by the warps
 };
 
+// `status` points at the context's status area: word 0 is the sticky device status, words 16 and 17
+// are the item counter and the count of finished CTAs (both zero between launches).
 inline cudaError_t launch_tc_attention(const ScheduleView& s, const PoolView& pool, const TensorArgs& t,
                                        int* status, int num_sms, const TcTensorMaps& maps, cudaStream_t stream) {
-  (void)num_sms;             // one CTA per work item; the hardware scheduler balances ragged items
-  tc_attention_kernel<<<s.num_items, tc::kThreads, tc::kSmemBytes, stream>>>(s, pool, t, status, maps.q, maps.k,
-                                                                              maps.v, maps.q_tma);
+  const int grid = s.num_items < num_sms ? s.num_items : num_sms;
+  tc_attention_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(s, pool, t, status, maps.q, maps.k, maps.v,
+                                                                        maps.o, maps.q_tma, maps.o_tma);
   return cudaGetLastError();
 }
 
