@@ -526,10 +526,17 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
                 fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
             const unsigned long long xb =
                 fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
-            float xa0, xa1, xb0, xb1;
+            float xa0, xa1, p2, p3;
             unpack2(xa, xa0, xa1);
-            unpack2(xb, xb0, xb1);
-            const float p0 = ex2(xa0), p1 = ex2(xa1), p2 = ex2(xb0), p3 = ex2(xb1);
+            const float p0 = ex2(xa0), p1 = ex2(xa1);
+            if (kPolyPeriod > 0 && i % (kPolyPeriod > 0 ? kPolyPeriod : 1) == 0) {
+              ex2_poly2(xb, p2, p3);                            // this pair on the FMA pipe
+            } else {
+              float xb0, xb1;
+              unpack2(xb, xb0, xb1);
+              p2 = ex2(xb0);
+              p3 = ex2(xb1);
+            }
             acc_a = add2(acc_a, pack2(p0, p1));
             acc_b = add2(acc_b, pack2(p2, p3));
             r[2 * i] = pack_bf16(p0, p1);
@@ -549,10 +556,17 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
                   fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
               const unsigned long long xb =
                   fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
-              float xa0, xa1, xb0, xb1;
+              float xa0, xa1, p2, p3;
               unpack2(xa, xa0, xa1);
-              unpack2(xb, xb0, xb1);
-              const float p0 = ex2(xa0), p1 = ex2(xa1), p2 = ex2(xb0), p3 = ex2(xb1);
+              const float p0 = ex2(xa0), p1 = ex2(xa1);
+              if (kPolyPeriod > 0 && i % (kPolyPeriod > 0 ? kPolyPeriod : 1) == 0) {
+                ex2_poly2(xb, p2, p3);                            // this pair on the FMA pipe
+              } else {
+                float xb0, xb1;
+                unpack2(xb, xb0, xb1);
+                p2 = ex2(xb0);
+                p3 = ex2(xb1);
+              }
               acc_a = add2(acc_a, pack2(p0, p1));
               acc_b = add2(acc_b, pack2(p2, p3));
               r[2 * i] = pack_bf16(p0, p1);
