@@ -202,6 +202,56 @@ __device__ __forceinline__ void mma_commit_elect(unsigned bar) {
       ::"r"(bar)
       : "memory");
 }
+// Batches of MMAs issued by the elected lane (`el` = elect_one() of a converged warp) under one
+// predicate, every descriptor computed by the caller (warp-uniform values stay in the uniform
+// datapath): the issuing warp then spends two instructions per MMA instead of five.
+// S = Q K^T: eight K steps of 16 dims; the first overwrites, the rest accumulate.
+__device__ __forceinline__ void mma_ss_batch8(unsigned el, unsigned d_tmem, const unsigned long long (&a)[8],
+                                              const unsigned long long (&b)[8], unsigned idesc) {
+  asm volatile(
+      "{\n\t.reg .pred P, T, F;\n\t"
+      "setp.ne.b32 P, %18, 0;\n\t"
+      "setp.eq.u32 T, 0, 0;\n\t"
+      "setp.ne.u32 F, 0, 0;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %9, %17, F;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %2, %10, %17, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %3, %11, %17, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %4, %12, %17, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %5, %13, %17, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %6, %14, %17, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %7, %15, %17, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %8, %16, %17, T;\n\t}"
+      ::"r"(d_tmem), "l"(a[0]), "l"(a[1]), "l"(a[2]), "l"(a[3]), "l"(a[4]), "l"(a[5]), "l"(a[6]), "l"(a[7]),
+        "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7]), "r"(idesc), "r"(el)
+      : "memory");
+}
+// O (+)= P V: four K steps of 16 keys, P read from TMEM at p + 8 k; the first accumulates iff acc0.
+__device__ __forceinline__ void mma_ts_batch4(unsigned el, unsigned o_tmem, unsigned p_tmem,
+                                              const unsigned long long (&b)[4], unsigned idesc, unsigned acc0) {
+  asm volatile(
+      "{\n\t.reg .pred P, T, Q;\n\t.reg .b32 p1, p2, p3;\n\t"
+      "setp.ne.b32 P, %8, 0;\n\t"
+      "setp.eq.u32 T, 0, 0;\n\t"
+      "setp.ne.b32 Q, %7, 0;\n\t"
+      "add.u32 p1, %1, 8;\n\t"
+      "add.u32 p2, %1, 16;\n\t"
+      "add.u32 p3, %1, 24;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %6, Q;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p1], %3, %6, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p2], %4, %6, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p3], %5, %6, T;\n\t}"
+      ::"r"(o_tmem), "r"(p_tmem), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "r"(idesc), "r"(acc0), "r"(el)
+      : "memory");
+}
+// tcgen05.commit by the same elected lane (a commit covers the MMAs its own thread issued)
+__device__ __forceinline__ void mma_commit_pred(unsigned el, unsigned bar) {
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "setp.ne.b32 P, %1, 0;\n\t"
+      "@P tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar), "r"(el)
+      : "memory");
+}
 // D[tmem] (+)= A[smem] * B[smem]
 __device__ __forceinline__ void mma_ss(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
                                        unsigned idesc, unsigned accumulate) {
@@ -1004,12 +1054,30 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       const unsigned tmem_u = __shfl_sync(0xffffffffu, tmem, 0);   // warp-uniform copy of the TMEM base
       const unsigned tmem_s1 = tmem_u + 128, tmem_o0 = tmem_u + 256, tmem_o1 = tmem_u + 384;
 #define BICACHE_WAIT(bar, parity) __all_sync(0xffffffffu, mbar_wait((bar), (parity), abort_flag))
+      const unsigned el = elect_one() ? 1u : 0u;               // the lane that issues every MMA of this warp
       // the eight MMAs (K steps of 16 dims) of S_X = Q_X K^T
       auto issue_s = [&](unsigned d_tmem, unsigned long long qd, unsigned long long kd, unsigned k_hi) {
+        unsigned long long a[8], b[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          mma_ss_elect(d_tmem, qd + (k >> 2) * q_hi + (k & 3) * 2, kd + (k >> 2) * k_hi + (k & 3) * 2, kIdescQK,
-                       k > 0 ? 1u : 0u);
+        for (int k = 0; k < 8; ++k) {
+          a[k] = qd + (k >> 2) * q_hi + (k & 3) * 2;
+          b[k] = kd + (k >> 2) * k_hi + (k & 3) * 2;
+        }
+        mma_ss_batch8(el, d_tmem, a, b, kIdescQK);
+      };
+      // four of the eight MMAs (K steps of 16 keys) of O_X += P_X V
+      auto issue_pv = [&](unsigned o_tmem, unsigned p_tmem, unsigned long long vd, unsigned v_step, int half,
+                          unsigned acc0, int ksteps) {
+        if (ksteps == 8) {
+          unsigned long long b[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k) b[k] = vd + (half * 4 + k) * v_step;
+          mma_ts_batch4(el, o_tmem, p_tmem + half * 32, b, kIdescPV, half ? 1u : acc0);
+        } else {
+#pragma unroll
+          for (int k = half * 4; k < half * 4 + 4; ++k)
+            mma_ts_elect(o_tmem, p_tmem + k * 8, vd + k * v_step, kIdescPV, k > 0 ? 1u : acc0, k < ksteps ? 1u : 0u);
+        }
       };
       int n_it = 0;
       int c0 = 0, c1 = 0;        // key tiles each query tile has been through (phase of p_half)
@@ -1034,8 +1102,8 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             tc_fence_after();
             const unsigned long long kd0 = (dn ? kb_dense : kb_img) + (u & 3) * kSlotUnits;
             issue_s(tmem_u, q_desc0, kd0, dn ? 1024u : 64u);
-            mma_commit_elect(bar_s);
-            if (T == 1) mma_commit_elect(bar_qfree);
+            mma_commit_pred(el, bar_s);
+            if (T == 1) mma_commit_pred(el, bar_qfree);
             if (b_on) {
               // Stagger the two query tiles by half a period: tile B starts when tile A's softmax is
               // half done (started together, the two softmaxes share the exp unit and the MMAs of
@@ -1043,10 +1111,10 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               ok = BICACHE_WAIT(bar_p, c0 & 1) && BICACHE_WAIT(bar_qfull + 8, e1 & 1);
               if (!ok) break;
               issue_s(tmem_s1, q_desc1, kd0, dn ? 1024u : 64u);
-              mma_commit_elect(bar_s + 8);
-              if (T == 1) mma_commit_elect(bar_qfree + 8);
+              mma_commit_pred(el, bar_s + 8);
+              if (T == 1) mma_commit_pred(el, bar_qfree + 8);
             }
-            mma_commit_elect(bar_free + (u & 3) * 8);
+            mma_commit_pred(el, bar_free + (u & 3) * 8);
           }
           // V of the first key tile; the previous item's epilogue must have read O_A out of TMEM
           ok = BICACHE_WAIT(bar_full + ((u + 1) & 3) * 8, ((u + 1) >> 2) & 1) && BICACHE_WAIT(bar_ofree, (e0 & 1) ^ 1);
@@ -1065,9 +1133,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             if (!ok) return;
             if (lane == 0) BICACHE_STAMP(1, ti);
             tc_fence_after();
-            #pragma unroll
-              for (int k = 0; k < 4; ++k)
-                mma_ts_elect(tmem_o0, tmem_u + k * 8, v_desc + k * v_step, kIdescPV, k > 0 ? 1u : acc0, k < ksteps ? 1u : 0u);
+                        issue_pv(tmem_o0, tmem_u, v_desc, v_step, 0, acc0, ksteps);
             if (lane == 0) BICACHE_STAMP(1, ti);
             // ---- shadow of A's second half of the exponentials: what follows the O of this iteration ----
             bool s_on0 = true, s_on1 = b_on;                   // an S follows O_A / O_B
@@ -1100,12 +1166,10 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             if (!ok) return;
             if (lane == 0) BICACHE_STAMP(1, ti);
             tc_fence_after();
-            #pragma unroll
-              for (int k = 4; k < 8; ++k)
-                mma_ts_elect(tmem_o0, tmem_u + k * 8, v_desc + k * v_step, kIdescPV, 1u, k < ksteps ? 1u : 0u);
+                        issue_pv(tmem_o0, tmem_u, v_desc, v_step, 1, acc0, ksteps);
             ++c0;
             if (last) {
-              mma_commit_elect(bar_odone);
+              mma_commit_pred(el, bar_odone);
               ++e0;
             }
             if (s_on0) {
@@ -1114,8 +1178,8 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
                 if (!ok) return;
               }
               issue_s(tmem_u, q_desc0, k_desc, k_hi);
-              mma_commit_elect(bar_s);
-              if (q_last) mma_commit_elect(bar_qfree);
+              mma_commit_pred(el, bar_s);
+              if (q_last) mma_commit_pred(el, bar_qfree);
             }
             if (lane == 0) BICACHE_STAMP(1, ti);
             // ---- tile B: first half ----
@@ -1128,10 +1192,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               if (!ok) return;
               if (lane == 0) BICACHE_STAMP(1, ti);
               tc_fence_after();
-              #pragma unroll
-                for (int k = 0; k < 4; ++k)
-                  mma_ts_elect(tmem_o1, tmem_s1 + k * 8, v_desc + k * v_step, kIdescPV, k > 0 ? 1u : acc0,
-                               k < ksteps ? 1u : 0u);
+                            issue_pv(tmem_o1, tmem_s1, v_desc, v_step, 0, acc0, ksteps);
             }
             // ---- shadow of B's second half: the next tile's key count ----
             const int ks_next = last ? 8 : (tile_keys(cur, j + 1) + 15) >> 4;
@@ -1140,12 +1201,10 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               ok = BICACHE_WAIT(bar_p + 24, c1 & 1);
               if (!ok) return;
               tc_fence_after();
-              #pragma unroll
-                for (int k = 4; k < 8; ++k)
-                  mma_ts_elect(tmem_o1, tmem_s1 + k * 8, v_desc + k * v_step, kIdescPV, 1u, k < ksteps ? 1u : 0u);
+                            issue_pv(tmem_o1, tmem_s1, v_desc, v_step, 1, acc0, ksteps);
               ++c1;
               if (last) {
-                mma_commit_elect(bar_odone + 8);
+                mma_commit_pred(el, bar_odone + 8);
                 ++e1;
               }
             }
@@ -1155,13 +1214,13 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
                 if (!ok) return;
               }
               issue_s(tmem_s1, q_desc1, k_desc, k_hi);
-              mma_commit_elect(bar_s + 8);
-              if (q_last) mma_commit_elect(bar_qfree + 8);
+              mma_commit_pred(el, bar_s + 8);
+              if (q_last) mma_commit_pred(el, bar_qfree + 8);
             }
             if (lane == 0) BICACHE_STAMP(1, ti);
             // release V of this tile and K of the next
-            mma_commit_elect(bar_free + sv * 8);
-            if (s_on0) mma_commit_elect(bar_free + sn * 8);
+            mma_commit_pred(el, bar_free + sv * 8);
+            if (s_on0) mma_commit_pred(el, bar_free + sn * 8);
             u += 2;
             dn = dn_next;
             ksteps = ks_next;
@@ -1191,7 +1250,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
 #undef BICACHE_WAIT
       // Whatever happened, let every MMA issued so far finish before TMEM is released.
       __syncwarp();
-      mma_commit_elect(smem_u32(&bars->drain));
+      mma_commit_elect(smem_u32(&bars->drain));               // elect.sync names the same lane as `el`
       mbar_wait(smem_u32(&bars->drain), 0, abort_flag);
     }
     __syncwarp();
