@@ -399,6 +399,29 @@ def main():
         sec, desc, _ = oracle_step_seconds(w, workloads, oracle, depth)
         cpu = {"value": w.suffix_tokens / sec, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": desc}
 
+    # ---- prefix store put (bandwidth-bound scatter into page images), off the per-step path ----
+    # Timed last: every put of a fresh key evicts the oldest prefix (FIFO), the workload's own first.
+    roofline_put = None
+    put_bytes = 4 * w.num_layers * w.prefix_lens[0] * w.num_kv_heads * w.head_dim * (2 if w.dtype == torch.bfloat16 else 4)
+    if put_bytes >= (256 << 20):
+        kc, vc = workloads.draw_prefix_kv(w, 0, "cuda")
+        ts = []
+        for i in range(5):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            bc.put_prefix(0x7000000000000000 + i, kc, vc)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        del kc, vc
+        ms_put = sorted(ts[1:])[len(ts[1:]) // 2]
+        gbs = put_bytes / (ms_put * 1e-3) / 1e9
+        roofline_put = {"bound": "hbm", "kernel": "scatter_prefix_kernel (put_prefix of prefix 0, all layers)",
+                        "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                        "peak_source": peaks["source"], "bytes_per_launch": put_bytes, "ms_per_launch": ms_put,
+                        "traffic": None}
+
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": step_ms_max, "higher_is_better": True, "scaling": "weak",
@@ -410,7 +433,8 @@ def main():
                            "depth_min": int(min(depth)), "depth_max": int(max(depth))},
                 "tflops": flops / (step_ms_max * 1e-3) / 1e12, "step_flops": flops,
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-                "roofline": roofline, "roofline_attend": roofline_attend, "cpu_baseline": cpu}
+                "roofline": roofline, "roofline_attend": roofline_attend, "roofline_put": roofline_put,
+                "cpu_baseline": cpu}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

@@ -19,6 +19,12 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
   attend/attend_full/stack
                    pinned (brute force over the concatenated key list, depth-0
                    and depth-L special cases, cached == fresh special case).
+  is_refresh_step/attend_step (Eq. 5)
+                   pinned (refresh steps enumerated by hand for Delta = 16;
+                   Delta = 1 equals full recompute at every step; a separate
+                   brute force that looks up "the step whose prefix KVs are in
+                   use" in closed form and concatenates; prefix KVs constant
+                   over the steps make the result independent of Delta).
 """
 from .bicache_oracle import (  # noqa: F401
     OracleError,
@@ -28,6 +34,8 @@ from .bicache_oracle import (  # noqa: F401
     reuse_depth,
     PagedPrefixStore,
     attention,
+    is_refresh_step,
+    attend_step,
     merge,
     attend,
     attend_full,

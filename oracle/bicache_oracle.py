@@ -9,7 +9,9 @@ Everything here is written from the paper's statement of the method:
   * Sec. 5.1/5.2 (ratio r of shared-prefix tokens to all tokens -> lookup
     table T -> shallow depth b; layer l reuses iff l <= b, else recomputes),
   * Sec. 5.2 + implementation appendix (hash-indexed KV store H holding the
-    prefix KVs of all L layers; first-in-first-out eviction).
+    prefix KVs of all L layers; first-in-first-out eviction),
+  * Eq. 5  (deep layers l > b: the prefix KVs computed within the request are
+    kept and reused across denoising steps, recomputed every Delta steps).
 
 All floating-point work is numpy float64.  A matrix product (numpy matmul) is
 used as a library step; there is no tiling, fusion, online softmax or any
@@ -152,6 +154,29 @@ class PagedPrefixStore:
             self.k_pool[:, pages[t // self.P], t % self.P] = k[:, t]
             self.v_pool[:, pages[t // self.P], t % self.P] = v[:, t]
         return pid, False, list(pages)
+
+    def reserve(self, key, m):
+        """Allocate pages for a prefix of m tokens without writing any KV (the
+        per-request deep-layer cache of Eq. 5, filled layer by layer at refresh
+        steps).  Same allocation and eviction rules as `put`."""
+        zeros = np.zeros((self.L, int(m), self.Hkv, self.D), dtype=np.float64)
+        return self.put(key, zeros, zeros)
+
+    def update_layer(self, prefix_id, layer, k, v):
+        """Overwrite one layer of an existing prefix with k, v [m, Hkv, D]
+        (Eq. 5, refresh step: KV^use <- KV^ref of the current step)."""
+        if not 0 <= layer < self.L:
+            raise InvalidArgument("layer out of range")
+        if prefix_id not in self.entries:
+            raise NotFound("unknown or evicted prefix id")
+        _, m, pages = self.entries[prefix_id]
+        k = np.asarray(k, dtype=np.float64)
+        v = np.asarray(v, dtype=np.float64)
+        if k.shape != (m, self.Hkv, self.D) or v.shape != k.shape:
+            raise InvalidArgument("bad layer KV shape")
+        for t in range(m):
+            self.k_pool[layer, pages[t // self.P], t % self.P] = k[t]
+            self.v_pool[layer, pages[t // self.P], t % self.P] = v[t]
 
     def lookup(self, key):
         key = int(key)
@@ -388,3 +413,66 @@ def stack(store, depth, prefix_id, prefix_len, full_row_off, full_len, q, k, v, 
                 lse[off:off + n] = l2[off:off + n]
         results.append((out, lse))
     return results
+
+
+# ---------------------------------------------------------------------------
+# Eq. 5: deep layers reuse the request's own prefix KVs across steps and
+# recompute them every Delta steps.
+# ---------------------------------------------------------------------------
+
+def is_refresh_step(t, delta):
+    """Eq. 5's condition (t - 1) mod Delta = 0 for the 1-based step t."""
+    if t < 1 or delta < 1:
+        raise InvalidArgument("t and delta start at 1")
+    return (t - 1) % delta == 0
+
+
+def attend_step(store, layer, t, delta, depth, shared_id, private_id, full_row_off, full_len,
+                q, k, v, scale):
+    """One layer of denoising step t with both kinds of reuse (Sec. 5.2).
+
+    Request i owns rows full_row_off[i] .. + full_len[i] of q/k/v (prefix
+    tokens first).  Per request, in this order:
+      * layer < depth[i] and shared_id[i] >= 0: the suffix queries attend over
+        [shared cached prefix KVs | own suffix KVs]              (Eq. 4);
+      * else, private_id[i] >= 0 and t is not a refresh step: the suffix
+        queries attend over [the request's own prefix KVs kept from the last
+        refresh step | own suffix KVs]                           (Eq. 5, 2nd case);
+      * else: full attention over all the request's rows; if private_id[i] >= 0
+        (a refresh step) the fresh prefix KVs of this layer, rows
+        0 .. m of the request, replace the kept ones             (Eq. 5, 1st case).
+    Returns (out, lse); rows not computed stay 0 / -inf.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    _check_batch(full_row_off, full_len, q.shape[0])
+    refresh = is_refresh_step(t, delta)
+    out = np.zeros_like(q)
+    lse = np.full(q.shape[:2], -np.inf)
+    for i in range(len(depth)):
+        off, N = int(full_row_off[i]), int(full_len[i])
+        if layer < depth[i] and shared_id[i] >= 0:
+            pid = int(shared_id[i])
+        elif private_id[i] >= 0 and not refresh:
+            pid = int(private_id[i])
+        else:
+            pid = -1
+        if pid >= 0:
+            m = store.prefix_len(pid)
+            if N < m:
+                raise InvalidArgument("request shorter than its prefix")
+            kc, vc = store.prefix_kv(layer, pid)
+            ks = np.concatenate([kc, k[off + m:off + N]], axis=0)
+            vs = np.concatenate([vc, v[off + m:off + N]], axis=0)
+            if N > m:
+                out[off + m:off + N], lse[off + m:off + N] = attention(q[off + m:off + N], ks, vs, scale)
+        else:
+            if N > 0:
+                out[off:off + N], lse[off:off + N] = attention(q[off:off + N], k[off:off + N], v[off:off + N], scale)
+            if private_id[i] >= 0:
+                m = store.prefix_len(int(private_id[i]))
+                if N < m:
+                    raise InvalidArgument("request shorter than its prefix")
+                store.update_layer(int(private_id[i]), layer, k[off:off + m], v[off:off + m])
+    return out, lse
