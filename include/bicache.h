@@ -190,6 +190,51 @@ int32_t bicache_attend_layer(bicache_ctx* ctx, int32_t layer, int32_t R, const i
                              void* out, int64_t out_row_stride, float* lse_out,
                              float softmax_scale, void* stream);
 
+/* ---- Deep layers: reuse within a request with periodic refresh (Sec. 5.2, Eq. 5) ------------------
+ * In layers l >= depth a request does not read the shared cache; it keeps the prefix K/V it computed
+ * itself and reuses them across denoising steps, recomputing them every delta steps.  The kept K/V
+ * live in the same paged store under a per-request key ("private" prefix). */
+
+/* Eq. 5's condition for the 1-based denoising step t: 1 if (t - 1) mod delta == 0 (recompute), 0 if
+ * not (reuse the kept K/V), -1 if t < 1 or delta < 1.  Pure integer, no context. */
+int32_t bicache_is_refresh_step(int32_t t, int32_t delta);
+
+/* Allocate pages for a prefix of m tokens under `key` without writing K/V: same hit / miss / FIFO
+ * eviction rules, outputs and errors as bicache_put_prefix, no kernel is launched.  The content of
+ * the pages is unspecified until bicache_update_prefix_layer has written a layer. */
+int32_t bicache_reserve_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, int32_t* prefix_id,
+                               int32_t* was_hit, int32_t* pages_out, int32_t pages_cap);
+
+/* Overwrite ONE layer of an existing prefix (Eq. 5, refresh step: the kept K/V become the ones just
+ * computed).  k, v: device, rows [m][Hkv][D] of the context's dtype, `kv_row_stride` elements between
+ * consecutive rows (so k may point at the request's first row inside a packed [rows][Hkv][D] tensor),
+ * 16-byte aligned rows.  Copies on `stream`; unused slots of the last page are zero-filled.
+ * NOTFOUND for an unknown or evicted id, INVALID for a bad layer, pointer or stride. */
+int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, const void* k,
+                                    const void* v, int64_t kv_row_stride, void* stream);
+
+/* One layer of denoising step t with both kinds of reuse.  Request i owns seqlen[i] = N_i rows from
+ * row_off[i] (prefix rows first).  Per request, in this order:
+ *   layer < depth[i] and shared_id[i] >= 0      -> suffix rows attend over [shared cached prefix | own
+ *                                                  suffix]                              (Eq. 4);
+ *   else private_id[i] >= 0 and not a refresh step -> suffix rows attend over [kept prefix K/V of
+ *                                                  private_id[i] | own suffix]          (Eq. 5, reuse);
+ *   else                                         -> full attention over all N_i rows; on a refresh
+ *                                                  step with private_id[i] >= 0, rows 0 .. m_i of k, v
+ *                                                  then replace the kept K/V of this layer
+ *                                                                                       (Eq. 5, recompute).
+ * depth, shared_id, private_id, row_off, seqlen: host arrays of length R (requests of one shared prefix
+ * need not be contiguous here: the call groups them).  Tensor arguments, outputs and errors as for
+ * bicache_attend_layer; INVALID also if t < 1 or delta < 1.  Everything is validated before the first
+ * launch. */
+int32_t bicache_attend_step(bicache_ctx* ctx, int32_t layer, int32_t t, int32_t delta, int32_t R,
+                            const int32_t* depth, const int32_t* shared_id, const int32_t* private_id,
+                            const int64_t* row_off, const int32_t* seqlen,
+                            const void* q, const void* k, const void* v,
+                            int64_t q_row_stride, int64_t kv_row_stride,
+                            void* out, int64_t out_row_stride, float* lse_out,
+                            float softmax_scale, void* stream);
+
 /* Synchronises `stream` and returns the sticky device status: OK, or TIMEOUT if a kernel gave up
  * on a bounded wait (its outputs are then undefined), or CUDA for a runtime error.  `clear` != 0
  * resets the word. */

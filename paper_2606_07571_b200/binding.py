@@ -23,6 +23,7 @@ EXPORTED = [
     "bicache_set_path", "bicache_set_depth_table", "bicache_put_prefix", "bicache_lookup_prefix",
     "bicache_prefix_pages", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
     "bicache_attend_layer", "bicache_attend_full_static",
+    "bicache_is_refresh_step", "bicache_reserve_prefix", "bicache_update_prefix_layer", "bicache_attend_step",
     "bicache_device_status", "bicache_launch_count", "bicache_last_error",
 ]
 
@@ -87,6 +88,15 @@ def load_library():
     lib.bicache_attend_layer.restype = C.c_int32
     lib.bicache_attend_layer.argtypes = [vp, C.c_int32, C.c_int32, i32p, i32p, i64p, i32p, vp, vp, vp, C.c_int64,
                                          C.c_int64, vp, C.c_int64, vp, C.c_float, vp]
+    lib.bicache_is_refresh_step.restype = C.c_int32
+    lib.bicache_is_refresh_step.argtypes = [C.c_int32, C.c_int32]
+    lib.bicache_reserve_prefix.restype = C.c_int32
+    lib.bicache_reserve_prefix.argtypes = [vp, C.c_uint64, C.c_int32, i32p, i32p, i32p, C.c_int32]
+    lib.bicache_update_prefix_layer.restype = C.c_int32
+    lib.bicache_update_prefix_layer.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, C.c_int64, vp]
+    lib.bicache_attend_step.restype = C.c_int32
+    lib.bicache_attend_step.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, i32p, i32p, i32p, i64p, i32p,
+                                        vp, vp, vp, C.c_int64, C.c_int64, vp, C.c_int64, vp, C.c_float, vp]
     lib.bicache_attend_full_static.restype = C.c_int32
     lib.bicache_attend_full_static.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp, vp, vp,
                                                C.c_int64, C.c_int64, vp, C.c_int64, C.c_float, vp]
@@ -192,6 +202,41 @@ class BiCache:
                                          pages.ctypes.data_as(C.POINTER(C.c_int32)), cap)
         self._check(st, "bicache_put_prefix")
         return pid.value, bool(hit.value), pages[:cap].tolist()
+
+    def reserve_prefix(self, key, m):
+        """Pages for a prefix of m tokens, no K/V written (Eq. 5's per-request cache).  Returns
+        (prefix_id, was_hit, pages)."""
+        pid, hit = C.c_int32(-1), C.c_int32(0)
+        cap = (m + 15) // 16
+        pages = np.zeros(max(cap, 1), dtype=np.int32)
+        st = self.lib.bicache_reserve_prefix(self.ctx, C.c_uint64(key), m, C.byref(pid), C.byref(hit),
+                                             pages.ctypes.data_as(C.POINTER(C.c_int32)), cap)
+        self._check(st, "bicache_reserve_prefix")
+        return pid.value, bool(hit.value), pages[:cap].tolist()
+
+    def update_prefix_layer(self, prefix_id, layer, k, v):
+        """k, v: [m, Hkv, D] device tensors (rows may be strided) that replace one layer of a prefix."""
+        assert k.is_cuda and v.is_cuda and k.dtype == self.dtype and k.shape == v.shape
+        assert k.stride()[1:] == (self.D, 1) and v.stride() == k.stride()
+        st = self.lib.bicache_update_prefix_layer(self.ctx, prefix_id, layer, k.data_ptr(), v.data_ptr(),
+                                                  k.stride(0), self._stream())
+        self._check(st, "bicache_update_prefix_layer")
+
+    def is_refresh_step(self, t, delta):
+        return int(self.lib.bicache_is_refresh_step(t, delta))
+
+    def attend_step(self, layer, t, delta, depth, shared_id, private_id, row_off, seqlen, q, k, v, out, lse=None,
+                    scale=None):
+        d, pd = _i32(depth)
+        sid, psid = _i32(shared_id)
+        prid, pprid = _i32(private_id)
+        off, poff = _i64(row_off)
+        n, pn = _i32(seqlen)
+        qp, kp, vp_, qs, ks, op, os_, lp = self._tensor_args(q, k, v, out, lse)
+        scale = self.D ** -0.5 if scale is None else scale
+        st = self.lib.bicache_attend_step(self.ctx, layer, t, delta, len(n), pd, psid, pprid, poff, pn, qp, kp, vp_,
+                                          qs, ks, op, os_, lp, C.c_float(scale), self._stream())
+        self._check(st, "bicache_attend_step")
 
     def lookup_prefix(self, key):
         pid, m = C.c_int32(-1), C.c_int32(0)

@@ -528,9 +528,14 @@ int32_t bicache_set_depth_table(bicache_ctx* ctx, const int32_t* table, int32_t 
   return BICACHE_OK;
 }
 
-int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const void* v,
-                           int64_t layer_stride, void* stream_, int32_t* prefix_id, int32_t* was_hit,
-                           int32_t* pages_out, int32_t pages_cap) {
+}  // extern "C"
+
+namespace {
+// Insert a prefix: hit / miss / FIFO eviction / page allocation, and (write = true) the scatter of all
+// layers' K/V into the page images.
+int32_t put_impl(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const void* v, int64_t layer_stride,
+                 void* stream_, int32_t* prefix_id, int32_t* was_hit, int32_t* pages_out, int32_t pages_cap,
+                 bool write) {
   if (!ctx) return BICACHE_ERR_INVALID;
   if (!prefix_id) return fail(ctx, BICACHE_ERR_INVALID, "prefix_id is required");
   if (m < 1) return fail(ctx, BICACHE_ERR_INVALID, "empty prefix");
@@ -546,10 +551,10 @@ int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void
     if (pages_out) std::copy(e.pages.begin(), e.pages.end(), pages_out);
     return BICACHE_OK;
   }
-  if (!ctx->host_only && (!k || !v || !aligned16(k) || !aligned16(v)))
-    return fail(ctx, BICACHE_ERR_INVALID, "bad k/v pointer");
+  write = write && !ctx->host_only;
+  if (write && (!k || !v || !aligned16(k) || !aligned16(v))) return fail(ctx, BICACHE_ERR_INVALID, "bad k/v pointer");
   const int64_t row_elems = (int64_t)cfg.num_kv_heads * cfg.head_dim;
-  if (layer_stride < (int64_t)m * row_elems || (layer_stride * ctx->esize) % 16)
+  if (write && (layer_stride < (int64_t)m * row_elems || (layer_stride * ctx->esize) % 16))
     return fail(ctx, BICACHE_ERR_INVALID, "bad layer stride");
   if (need > cfg.num_pages) return fail(ctx, BICACHE_ERR_NOMEM, "prefix larger than the whole pool");
   if (pages_out && pages_cap < need) return fail(ctx, BICACHE_ERR_INVALID, "pages_out too small");
@@ -572,9 +577,9 @@ int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void
   }
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   cudaError_t ce = cudaSuccess;
-  if (!ctx->host_only)
+  if (write)
     ce = cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
-  if (ce == cudaSuccess && !ctx->host_only) {
+  if (ce == cudaSuccess && write) {
     const int chunks_per_row = cfg.head_dim * ctx->esize / 16;
     const long long total = (long long)cfg.num_layers * need * kPageSize * cfg.num_kv_heads * chunks_per_row;
     const int threads = 256;
@@ -583,7 +588,8 @@ int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void
     scatter_prefix_kernel<<<blocks, threads, 0, stream>>>(
         static_cast<const char*>(k), static_cast<const char*>(v), static_cast<char*>(cfg.k_pool),
         static_cast<char*>(cfg.v_pool), ctx->d_put_pages, need, m, cfg.num_layers, cfg.num_kv_heads,
-        chunks_per_row, layer_stride * ctx->esize, pv.layer_bytes, pv.page_bytes, pv.swizzled);
+        chunks_per_row, layer_stride * ctx->esize, (long long)row_elems * ctx->esize, pv.layer_bytes,
+        pv.page_bytes, pv.swizzled);
     ctx->launches++;
     ce = cudaGetLastError();
   }
@@ -600,6 +606,60 @@ int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void
   ctx->by_key[key] = it;
   ctx->by_id[it->id] = it;
   return BICACHE_OK;
+}
+}  // namespace
+
+extern "C" {
+
+int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const void* v,
+                           int64_t layer_stride, void* stream, int32_t* prefix_id, int32_t* was_hit,
+                           int32_t* pages_out, int32_t pages_cap) {
+  return put_impl(ctx, key, m, k, v, layer_stride, stream, prefix_id, was_hit, pages_out, pages_cap, true);
+}
+
+int32_t bicache_reserve_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, int32_t* prefix_id, int32_t* was_hit,
+                               int32_t* pages_out, int32_t pages_cap) {
+  return put_impl(ctx, key, m, nullptr, nullptr, 0, nullptr, prefix_id, was_hit, pages_out, pages_cap, false);
+}
+
+int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, const void* k,
+                                    const void* v, int64_t kv_row_stride, void* stream_) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  const bicache_config& cfg = ctx->cfg;
+  auto found = ctx->by_id.find(prefix_id);
+  if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+  if (layer < 0 || layer >= cfg.num_layers) return fail(ctx, BICACHE_ERR_INVALID, "layer out of range");
+  const PrefixEntry& e = *found->second;
+  const int64_t row_elems = (int64_t)cfg.num_kv_heads * cfg.head_dim;
+  if (kv_row_stride < row_elems || (kv_row_stride * ctx->esize) % 16)
+    return fail(ctx, BICACHE_ERR_INVALID, "bad row stride");
+  if (ctx->host_only) return BICACHE_OK;
+  if (!k || !v || !aligned16(k) || !aligned16(v)) return fail(ctx, BICACHE_ERR_INVALID, "bad k/v pointer");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int need = (int)e.pages.size();
+  cudaError_t ce =
+      cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+  if (ce == cudaSuccess) {
+    const int chunks_per_row = cfg.head_dim * ctx->esize / 16;
+    const long long total = (long long)need * kPageSize * cfg.num_kv_heads * chunks_per_row;
+    const int threads = 256;
+    const int blocks = (int)std::min<long long>((total + threads - 1) / threads, (long long)ctx->sm_count * 16);
+    const PoolView pv = pool_view(ctx);
+    scatter_prefix_kernel<<<blocks, threads, 0, stream>>>(
+        static_cast<const char*>(k), static_cast<const char*>(v),
+        static_cast<char*>(cfg.k_pool) + (long long)layer * pv.layer_bytes,
+        static_cast<char*>(cfg.v_pool) + (long long)layer * pv.layer_bytes, ctx->d_put_pages, need, e.m, 1,
+        cfg.num_kv_heads, chunks_per_row, 0, kv_row_stride * ctx->esize, pv.layer_bytes, pv.page_bytes, pv.swizzled);
+    ctx->launches++;
+    ce = cudaGetLastError();
+  }
+  if (ce != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("update_prefix_layer: ") + cudaGetErrorString(ce));
+  return BICACHE_OK;
+}
+
+int32_t bicache_is_refresh_step(int32_t t, int32_t delta) {
+  if (t < 1 || delta < 1) return -1;
+  return (t - 1) % delta == 0 ? 1 : 0;
 }
 
 int32_t bicache_lookup_prefix(const bicache_ctx* ctx, uint64_t key, int32_t* prefix_id, int32_t* m) {
@@ -702,6 +762,78 @@ int32_t bicache_attend_layer(bicache_ctx* ctx, int32_t layer, int32_t R, const i
     const int32_t st = run_attention(ctx, 1, layer, (int32_t)f_len.size(), nullptr, f_off.data(), f_len.data(),
                                      q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
                                      softmax_scale, stream);
+    if (st != BICACHE_OK) return st;
+  }
+  return BICACHE_OK;
+}
+
+int32_t bicache_attend_step(bicache_ctx* ctx, int32_t layer, int32_t t, int32_t delta, int32_t R,
+                            const int32_t* depth, const int32_t* shared_id, const int32_t* private_id,
+                            const int64_t* row_off, const int32_t* seqlen, const void* q, const void* k,
+                            const void* v, int64_t q_row_stride, int64_t kv_row_stride, void* out,
+                            int64_t out_row_stride, float* lse_out, float softmax_scale, void* stream) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  if (R < 0 || (R > 0 && (!depth || !shared_id || !private_id || !row_off || !seqlen)))
+    return fail(ctx, BICACHE_ERR_INVALID, "null metadata array");
+  const int refresh = bicache_is_refresh_step(t, delta);
+  if (refresh < 0) return fail(ctx, BICACHE_ERR_INVALID, "t and delta start at 1");
+  if (layer < 0 || layer >= ctx->cfg.num_layers) return fail(ctx, BICACHE_ERR_INVALID, "layer out of range");
+  // Per request: which cached prefix (if any) its suffix rows read in this layer at this step.
+  struct Reuse { int32_t pid; int64_t off; int32_t len; int order; };
+  std::vector<Reuse> reuse;
+  std::vector<int32_t> f_len, upd_id;
+  std::vector<int64_t> f_off, upd_off;
+  std::unordered_map<int32_t, int> first_seen;
+  for (int i = 0; i < R; ++i) {
+    if (seqlen[i] < 0 || row_off[i] < 0) return fail(ctx, BICACHE_ERR_INVALID, "negative length or offset");
+    int32_t pid = -1;
+    if (layer < depth[i] && shared_id[i] >= 0) pid = shared_id[i];
+    else if (private_id[i] >= 0 && !refresh) pid = private_id[i];
+    if (pid >= 0) {
+      auto found = ctx->by_id.find(pid);
+      if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+      const int32_t m = found->second->m;
+      if (seqlen[i] < m) return fail(ctx, BICACHE_ERR_INVALID, "request shorter than its prefix");
+      const int order = first_seen.emplace(pid, (int)first_seen.size()).first->second;
+      reuse.push_back(Reuse{pid, row_off[i] + m, seqlen[i] - m, order});
+    } else {
+      f_off.push_back(row_off[i]);
+      f_len.push_back(seqlen[i]);
+      if (private_id[i] >= 0) {
+        auto found = ctx->by_id.find(private_id[i]);
+        if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+        if (seqlen[i] < found->second->m) return fail(ctx, BICACHE_ERR_INVALID, "request shorter than its prefix");
+        upd_id.push_back(private_id[i]);
+        upd_off.push_back(row_off[i]);
+      }
+    }
+  }
+  // requests of one prefix side by side, in order of first appearance
+  std::stable_sort(reuse.begin(), reuse.end(), [](const Reuse& a, const Reuse& b) { return a.order < b.order; });
+  if (!reuse.empty()) {
+    std::vector<int32_t> r_pid, r_len;
+    std::vector<int64_t> r_off;
+    for (const Reuse& r : reuse) {
+      r_pid.push_back(r.pid);
+      r_off.push_back(r.off);
+      r_len.push_back(r.len);
+    }
+    const int32_t st = run_attention(ctx, 0, layer, (int32_t)r_len.size(), r_pid.data(), r_off.data(), r_len.data(),
+                                     q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                                     softmax_scale, stream);
+    if (st != BICACHE_OK) return st;
+  }
+  if (!f_len.empty()) {
+    const int32_t st = run_attention(ctx, 1, layer, (int32_t)f_len.size(), nullptr, f_off.data(), f_len.data(),
+                                     q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                                     softmax_scale, stream);
+    if (st != BICACHE_OK) return st;
+  }
+  // refresh: the prefix rows just used become the kept K/V of this layer (Eq. 5, first case)
+  for (size_t i = 0; i < upd_id.size(); ++i) {
+    const char* kp = static_cast<const char*>(k) + upd_off[i] * kv_row_stride * ctx->esize;
+    const char* vp = static_cast<const char*>(v) + upd_off[i] * kv_row_stride * ctx->esize;
+    const int32_t st = bicache_update_prefix_layer(ctx, upd_id[i], layer, kp, vp, kv_row_stride, stream);
     if (st != BICACHE_OK) return st;
   }
   return BICACHE_OK;

@@ -62,8 +62,8 @@ __global__ void scatter_prefix_kernel(const char* __restrict__ src_k, const char
                                       char* __restrict__ pool_k, char* __restrict__ pool_v,
                                       const int* __restrict__ pages, int num_prefix_pages, int m,
                                       int num_layers, int num_kv_heads, int chunks_per_row,
-                                      long long layer_stride_bytes, long long pool_layer_bytes,
-                                      int page_bytes, int swizzled) {
+                                      long long layer_stride_bytes, long long src_row_stride_bytes,
+                                      long long pool_layer_bytes, int page_bytes, int swizzled) {
   const long long per_layer = (long long)num_prefix_pages * kPageSize * num_kv_heads * chunks_per_row;
   const long long total = per_layer * num_layers;
   const int row_bytes = chunks_per_row * 16;
@@ -78,8 +78,8 @@ __global__ void scatter_prefix_kernel(const char* __restrict__ src_k, const char
     const int slot = t % kPageSize;
     uint4 ck = make_uint4(0, 0, 0, 0), cv = ck;
     if (t < m) {
-      const long long so = (long long)layer * layer_stride_bytes +
-                           ((long long)t * num_kv_heads + hk) * row_bytes + c16 * 16;
+      const long long so = (long long)layer * layer_stride_bytes + (long long)t * src_row_stride_bytes +
+                           (long long)hk * row_bytes + c16 * 16;
       ck = *reinterpret_cast<const uint4*>(src_k + so);
       cv = *reinterpret_cast<const uint4*>(src_v + so);
     }

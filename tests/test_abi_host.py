@@ -154,3 +154,45 @@ def test_store_traces_match_oracle_bit_exactly(trace, num_pages, seed):
             except oracle.NotFound:
                 assert stt == binding.ERR_NOTFOUND
     lib.bicache_destroy(ctx)
+
+
+def test_refresh_rule_and_reserve_on_host_context(lib):
+    """Eq. 5's step rule and the page bookkeeping of a reserved (per-request) prefix, no GPU."""
+    for t in range(1, 70):
+        for delta in (1, 3, 16):
+            assert lib.bicache_is_refresh_step(t, delta) == int(oracle.is_refresh_step(t, delta))
+    assert lib.bicache_is_refresh_step(0, 16) == -1
+    assert lib.bicache_is_refresh_step(5, 0) == -1
+    ctx = host_ctx(lib, L=2, Hq=2, Hkv=2, pages=4)
+    ref = oracle.PagedPrefixStore(2, 2, 2, 16, 4)
+    pid, hit = C.c_int32(-1), C.c_int32(-1)
+    pages = np.full(8, -1, dtype=np.int32)
+    pp = pages.ctypes.data_as(C.POINTER(C.c_int32))
+    assert put(lib, ctx, 10, 20) == (binding.OK, 0, 0, [0, 1])
+    ref.put(10, np.zeros((2, 20, 2, 2)), np.zeros((2, 20, 2, 2)))
+    assert lib.bicache_reserve_prefix(ctx, C.c_uint64(77), 17, C.byref(pid), C.byref(hit), pp, 8) == binding.OK
+    want = ref.reserve(77, 17)
+    assert (pid.value, bool(hit.value), pages[:2].tolist()) == want
+    assert lib.bicache_reserve_prefix(ctx, C.c_uint64(77), 17, C.byref(pid), C.byref(hit), pp, 8) == binding.OK
+    assert hit.value == 1
+    assert lib.bicache_reserve_prefix(ctx, C.c_uint64(77), 18, C.byref(pid), C.byref(hit), pp, 8) == binding.ERR_INVALID
+    # update: id, layer and stride are checked on the host
+    assert lib.bicache_update_prefix_layer(ctx, 99, 0, None, None, 256, None) == binding.ERR_NOTFOUND
+    assert lib.bicache_update_prefix_layer(ctx, pid.value, 2, None, None, 256, None) == binding.ERR_INVALID
+    assert lib.bicache_update_prefix_layer(ctx, pid.value, 0, None, None, 255, None) == binding.ERR_INVALID
+    assert lib.bicache_update_prefix_layer(ctx, pid.value, 1, None, None, 256, None) == binding.OK   # host-only: no copy
+    # a third prefix evicts the oldest (key 10), the reserved one stays
+    assert put(lib, ctx, 11, 20)[0] == binding.OK
+    m = C.c_int32()
+    assert lib.bicache_lookup_prefix(ctx, C.c_uint64(10), C.byref(pid), C.byref(m)) == binding.ERR_NOTFOUND
+    assert lib.bicache_lookup_prefix(ctx, C.c_uint64(77), C.byref(pid), C.byref(m)) == binding.OK
+    # the step dispatch validates before it would launch
+    i32 = lambda *a: np.asarray(a, dtype=np.int32).ctypes.data_as(C.POINTER(C.c_int32))
+    i64 = lambda *a: np.asarray(a, dtype=np.int64).ctypes.data_as(C.POINTER(C.c_int64))
+    args = (None, None, None, 256, 256, None, 256, None, C.c_float(1.0), None)
+    assert lib.bicache_attend_step(ctx, 0, 0, 16, 1, i32(1), i32(-1), i32(-1), i64(0), i32(4), *args) == binding.ERR_INVALID
+    assert lib.bicache_attend_step(ctx, 5, 1, 16, 1, i32(1), i32(-1), i32(-1), i64(0), i32(4), *args) == binding.ERR_INVALID
+    assert lib.bicache_attend_step(ctx, 0, 2, 16, 1, i32(0), i32(-1), i32(55), i64(0), i32(40), *args) == binding.ERR_NOTFOUND
+    assert lib.bicache_attend_step(ctx, 0, 2, 16, 1, i32(0), i32(-1), i32(pid.value), i64(0), i32(5), *args) \
+        == binding.ERR_INVALID                                                   # shorter than its kept prefix
+    lib.bicache_destroy(ctx)
