@@ -102,11 +102,15 @@ class ClockSampler:
 class Job:
     """Device state of one workload: context, store, tensors, and the step function."""
 
-    def __init__(self, w, device):
+    def __init__(self, w, device, delta=0):
         from paper_2606_07571_b200 import binding, workloads
         self.w, self.binding, self.workloads = w, binding, workloads
         torch.cuda.set_device(device)
+        self.delta = delta if w.num_layers > 1 else 0
+        self.t = 1                                    # 1-based denoising step (Eq. 5)
         npages = w.pages_needed() + 1
+        if self.delta > 0:                            # per-request kept prefix K/V of the deep layers
+            npages += sum((w.prefix_lens[g] + 15) // 16 for g in w.req_prefix)
         order = workloads.shuffled_page_order(npages, 7) if w.shuffle_pages else None
         self.bc = binding.BiCache(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim, npages, w.dtype,
                                   w.total_rows, w.num_requests, device=device, free_order=order)
@@ -116,6 +120,10 @@ class Job:
             kc, vc = workloads.draw_prefix_kv(w, g, "cuda")
             self.bc.put_prefix(self.keys[g], kc, vc)
             del kc, vc
+        self.private = [-1] * w.num_requests
+        if self.delta > 0:
+            self.private = [self.bc.reserve_prefix(0x6000000000000000 + i, w.prefix_lens[g])[0]
+                            for i, g in enumerate(w.req_prefix)]
         self.q, self.k, self.v = workloads.draw_full_qkv(w, "cuda")
         self.out = torch.empty_like(self.q)
         self.single_layer = w.num_layers == 1
@@ -136,6 +144,12 @@ class Job:
             bc.attend_layer(0, depth, req_pid, w.full_row_off, w.full_lens, q, k, v, self.out, None, w.softmax_scale)
             bc.attend_layer(0, [0] * w.num_requests, req_pid, w.full_row_off, w.full_lens, q, k, v, self.out2, None,
                             w.softmax_scale)
+        elif self.delta > 0:
+            # deep layers keep the request's own prefix K/V and recompute them every delta steps
+            for l in range(w.num_layers):
+                bc.attend_step(l, self.t, self.delta, depth, req_pid, self.private, w.full_row_off, w.full_lens,
+                               q, k, v, self.out, None, w.softmax_scale)
+            self.t += 1
         else:
             for l in range(w.num_layers):
                 bc.attend_layer(l, depth, req_pid, w.full_row_off, w.full_lens, q, k, v, self.out, None,
@@ -154,6 +168,12 @@ class Job:
         for i in range(w.num_requests):
             tot += int(depth[i]) * per_req_attend[i] + (w.num_layers - int(depth[i])) * per_req_full[i]
         return tot, depth
+
+    def reuse_step_flops(self):
+        """A step between two refresh steps: every layer reads a cached prefix (shared or kept)."""
+        w = self.w
+        return w.num_layers * sum(4 * w.head_dim * w.num_q_heads * n * (w.prefix_lens[g] + n)
+                                  for g, n in zip(w.req_prefix, w.suffix_lens))
 
 
 def time_call(fn, iters, flush):
@@ -274,6 +294,8 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--delta", type=int, default=0,
+                    help="refresh interval of the deep layers' kept prefix K/V (Eq. 5); 0: recompute every step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -298,7 +320,7 @@ def main():
         if rank != 0:
             entry.build()
     peaks = load_peaks()
-    job = Job(w, local_rank)
+    job = Job(w, local_rank, args.delta)
     flops, depth = job.step_flops()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")       # 2x the 126 MB L2
 
@@ -315,6 +337,7 @@ def main():
         sampler.start()
     launches0 = job.bc.launch_count()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    job.t = 1                                         # the timed steps are denoising steps 1 .. K
     for a, b in ev:
         flush.zero_()
         a.record()
@@ -322,7 +345,17 @@ def main():
         b.record()
     torch.cuda.synchronize()
     launches = job.bc.launch_count() - launches0
-    step_ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
+    per_step_ms = [a.elapsed_time(b) for a, b in ev]
+    step_ms = sum(per_step_ms) / args.steps
+    refresh_info = None
+    if job.delta > 0:
+        is_ref = [(t - 1) % job.delta == 0 for t in range(1, args.steps + 1)]
+        ref_ms = [m for m, r in zip(per_step_ms, is_ref) if r]
+        reu_ms = [m for m, r in zip(per_step_ms, is_ref) if not r]
+        flops = (len(ref_ms) * flops + len(reu_ms) * job.reuse_step_flops()) / args.steps   # mean FLOPs per step
+        refresh_info = {"delta": job.delta, "refresh_steps": len(ref_ms), "reuse_steps": len(reu_ms),
+                        "ms_refresh_step": sum(ref_ms) / max(1, len(ref_ms)),
+                        "ms_reuse_step": sum(reu_ms) / max(1, len(reu_ms)) if reu_ms else None}
     # a short sustained stretch so that the clock sampler sees the kernels under load
     t_end = time.time() + 0.6
     while time.time() < t_end:
@@ -430,7 +463,8 @@ def main():
                            "suffix_tokens": w.suffix_tokens, "l2": "flushed between timed steps (256 MB write)",
                            "step": ("shallow-layer pass + deep-layer pass of the single layer"
                                     if job.single_layer else "all layers, per-request depths from the rule"),
-                           "depth_min": int(min(depth)), "depth_max": int(max(depth))},
+                           "depth_min": int(min(depth)), "depth_max": int(max(depth)),
+                           "deep_layer_refresh": refresh_info},
                 "tflops": flops / (step_ms_max * 1e-3) / 1e12, "step_flops": flops,
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
                 "roofline": roofline, "roofline_attend": roofline_attend, "roofline_put": roofline_put,
