@@ -25,6 +25,11 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
                    brute force that looks up "the step whose prefix KVs are in
                    use" in closed form and concatenates; prefix KVs constant
                    over the steps make the result independent of Delta).
+  kv_similarity/depth_from_similarity/build_depth_table (Eq. 3, Sec. 5.1)
+                   pinned (closed forms: identical, negated, scaled and
+                   orthogonally mixed tensors with cos = a / sqrt(a^2 + b^2);
+                   scalar-loop brute force; hand-written threshold and
+                   averaging cases).
 """
 from .bicache_oracle import (  # noqa: F401
     OracleError,
@@ -36,6 +41,9 @@ from .bicache_oracle import (  # noqa: F401
     attention,
     is_refresh_step,
     attend_step,
+    kv_similarity,
+    depth_from_similarity,
+    build_depth_table,
     merge,
     attend,
     attend_full,

@@ -11,7 +11,9 @@ Everything here is written from the paper's statement of the method:
   * Sec. 5.2 + implementation appendix (hash-indexed KV store H holding the
     prefix KVs of all L layers; first-in-first-out eviction),
   * Eq. 5  (deep layers l > b: the prefix KVs computed within the request are
-    kept and reused across denoising steps, recomputed every Delta steps).
+    kept and reused across denoising steps, recomputed every Delta steps),
+  * Eq. 3 + Sec. 4.2/5.1 (profiler: cosine similarity between cached and
+    reference prefix KVs per layer -> depth b_i under threshold tau -> table T).
 
 All floating-point work is numpy float64.  A matrix product (numpy matmul) is
 used as a library step; there is no tiling, fusion, online softmax or any
@@ -476,3 +478,68 @@ def attend_step(store, layer, t, delta, depth, shared_id, private_id, full_row_o
                     raise InvalidArgument("request shorter than its prefix")
                 store.update_layer(int(private_id[i]), layer, k[off:off + m], v[off:off + m])
     return out, lse
+
+
+# ---------------------------------------------------------------------------
+# Profiler (Sec. 4.1 Eq. 3, Sec. 4.2, Sec. 5.1): similarity of the cached prefix
+# KVs to the ones a request computes itself, per layer; the depth it allows;
+# the lookup table built from many requests.
+# ---------------------------------------------------------------------------
+
+def kv_similarity(store, prefix_id, k_ref, v_ref):
+    """sim_l = cos(KV$_l, KVref_l) for every layer l (Eq. 3).
+
+    "Each KV representation is flattened into a single vector" (Sec. 4.1
+    footnote) is read as: layer l's keys and values of all prefix positions
+    and heads, concatenated, form one vector per side.  k_ref, v_ref:
+    [L, m, Hkv, D].  A zero vector on either side gives similarity 0.
+    """
+    k_ref = np.asarray(k_ref, dtype=np.float64)
+    v_ref = np.asarray(v_ref, dtype=np.float64)
+    m = store.prefix_len(prefix_id)
+    if k_ref.shape != (store.L, m, store.Hkv, store.D) or v_ref.shape != k_ref.shape:
+        raise InvalidArgument("bad reference KV shape")
+    sim = np.zeros(store.L)
+    for l in range(store.L):
+        kc, vc = store.prefix_kv(l, prefix_id)
+        a = np.concatenate([kc.reshape(-1), vc.reshape(-1)])
+        b = np.concatenate([k_ref[l].reshape(-1), v_ref[l].reshape(-1)])
+        na, nb = math.sqrt(float(a @ a)), math.sqrt(float(b @ b))
+        sim[l] = float(a @ b) / (na * nb) if na > 0 and nb > 0 else 0.0
+    return sim
+
+
+def depth_from_similarity(sim, tau):
+    """Sec. 4.2 / 5.1: b = the largest layer count such that every layer
+    1 .. b has sim_l >= tau, i.e. the number of leading layers at or above the
+    threshold."""
+    b = 0
+    for x in sim:
+        if not x >= tau:
+            break
+        b += 1
+    return b
+
+
+def build_depth_table(ratio_idx, depths, num_layers):
+    """Sec. 5.1 "lookup table T": for each ratio bin, the average of the b_i of
+    the requests profiled at that ratio, as an integer (floored: the smaller,
+    safer depth).  Returns 101 entries.  A bin without samples takes the value
+    of the nearest filled bin below it (b does not decrease with the ratio, so
+    this never overstates it); bins below the first filled one take min(1, L)
+    (layer 1's KVs do not depend on the rest of the input, Sec. 4.2 footnote).
+    """
+    sums = [0] * 101
+    cnts = [0] * 101
+    for idx, b in zip(ratio_idx, depths):
+        if not 0 <= idx <= 100 or not 0 <= b <= num_layers:
+            raise InvalidArgument("ratio bin or depth out of range")
+        sums[idx] += int(b)
+        cnts[idx] += 1
+    table = []
+    last = min(1, num_layers)
+    for idx in range(101):
+        if cnts[idx]:
+            last = sums[idx] // cnts[idx]
+        table.append(last)
+    return table
