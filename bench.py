@@ -436,8 +436,25 @@ def main():
     # Timed last: every put of a fresh key evicts the oldest prefix (FIFO), the workload's own first.
     roofline_put = None
     put_bytes = 4 * w.num_layers * w.prefix_lens[0] * w.num_kv_heads * w.head_dim * (2 if w.dtype == torch.bfloat16 else 4)
+    roofline_sim = None
     if put_bytes >= (256 << 20):
         kc, vc = workloads.draw_prefix_kv(w, 0, "cuda")
+        # profiler reduction (Eq. 3): cached prefix 0 against a reference K/V of the same shape; reads both once
+        ts = []
+        for i in range(5):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            bc.prefix_similarity(pid[0], kc, vc)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        ms_sim = sorted(ts[1:])[len(ts[1:]) // 2]
+        gbs = put_bytes / (ms_sim * 1e-3) / 1e9
+        roofline_sim = {"bound": "hbm", "kernel": "kv_similarity_partial_kernel (prefix_similarity of prefix 0)",
+                        "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                        "peak_source": peaks["source"], "bytes_per_launch": put_bytes, "ms_per_launch": ms_sim,
+                        "traffic": None}
         ts = []
         for i in range(5):
             flush.zero_()
@@ -468,6 +485,7 @@ def main():
                 "tflops": flops / (step_ms_max * 1e-3) / 1e12, "step_flops": flops,
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
                 "roofline": roofline, "roofline_attend": roofline_attend, "roofline_put": roofline_put,
+                "roofline_similarity": roofline_sim,
                 "cpu_baseline": cpu}
         print(json.dumps(line))
     if dist is not None:

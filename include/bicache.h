@@ -235,6 +235,32 @@ int32_t bicache_attend_step(bicache_ctx* ctx, int32_t layer, int32_t t, int32_t 
                             void* out, int64_t out_row_stride, float* lse_out,
                             float softmax_scale, void* stream);
 
+/* ---- Profiler pieces (Sec. 4.1 Eq. 3, Sec. 4.2, Sec. 5.1) -------------------------------------------
+ * How close the cached K/V of a prefix are to the K/V a request computes for the same tokens, per
+ * layer; the depth that allows under a threshold; the lookup table from many profiled requests. */
+
+/* sim_out[l] = cos(KV$_l, KVref_l), l = 0 .. L-1 (Eq. 3): per layer, the cached keys and values of all
+ * prefix positions and heads form one vector, the reference ones the other.  k_ref, v_ref: device,
+ * [L][m][Hkv][D] of the context's dtype, `layer_stride` elements between layers (m = the prefix's
+ * length).  sim_out: HOST array of L floats.  Runs on `stream` and synchronises it before returning
+ * (an offline call).  A zero vector on either side gives 0.  Uses the context's workspace as scratch.
+ * NOTFOUND for an unknown or evicted id, INVALID for a bad pointer or stride, UNSUPPORTED on a
+ * host-only context. */
+int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const void* k_ref, const void* v_ref,
+                                  int64_t layer_stride, float* sim_out, void* stream);
+
+/* *depth = the number of leading layers whose similarity is >= tau (Sec. 4.2: the largest b such that
+ * every layer 1 .. b is at or above the threshold; tau = 0.97 in the paper).  Host arrays, no context;
+ * a NaN ends the run. */
+int32_t bicache_depth_from_similarity(const float* sim, int32_t num_layers, float tau, int32_t* depth);
+
+/* table_out[0..100] from n profiled requests (ratio_idx[i] = floor(100 r_i) in 0..100, depth[i] in
+ * 0..num_layers): per ratio bin the mean of the depths, floored; a bin without samples takes the
+ * value of the nearest filled bin below it, bins below the first filled one take min(1, num_layers)
+ * (Sec. 5.1 "lookup table").  Host arrays, no context; INVALID for values out of range. */
+int32_t bicache_build_depth_table(const int32_t* ratio_idx, const int32_t* depth, int32_t n,
+                                  int32_t num_layers, int32_t* table_out);
+
 /* Synchronises `stream` and returns the sticky device status: OK, or TIMEOUT if a kernel gave up
  * on a bounded wait (its outputs are then undefined), or CUDA for a runtime error.  `clear` != 0
  * resets the word. */

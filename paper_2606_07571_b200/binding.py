@@ -24,6 +24,7 @@ EXPORTED = [
     "bicache_prefix_pages", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
     "bicache_attend_layer", "bicache_attend_full_static",
     "bicache_is_refresh_step", "bicache_reserve_prefix", "bicache_update_prefix_layer", "bicache_attend_step",
+    "bicache_prefix_similarity", "bicache_depth_from_similarity", "bicache_build_depth_table",
     "bicache_device_status", "bicache_launch_count", "bicache_last_error",
 ]
 
@@ -97,6 +98,13 @@ def load_library():
     lib.bicache_attend_step.restype = C.c_int32
     lib.bicache_attend_step.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, i32p, i32p, i32p, i64p, i32p,
                                         vp, vp, vp, C.c_int64, C.c_int64, vp, C.c_int64, vp, C.c_float, vp]
+    f32p = C.POINTER(C.c_float)
+    lib.bicache_prefix_similarity.restype = C.c_int32
+    lib.bicache_prefix_similarity.argtypes = [vp, C.c_int32, vp, vp, C.c_int64, f32p, vp]
+    lib.bicache_depth_from_similarity.restype = C.c_int32
+    lib.bicache_depth_from_similarity.argtypes = [f32p, C.c_int32, C.c_float, i32p]
+    lib.bicache_build_depth_table.restype = C.c_int32
+    lib.bicache_build_depth_table.argtypes = [i32p, i32p, C.c_int32, C.c_int32, i32p]
     lib.bicache_attend_full_static.restype = C.c_int32
     lib.bicache_attend_full_static.argtypes = [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp, vp, vp,
                                                C.c_int64, C.c_int64, vp, C.c_int64, C.c_float, vp]
@@ -222,6 +230,17 @@ class BiCache:
                                                   k.stride(0), self._stream())
         self._check(st, "bicache_update_prefix_layer")
 
+    def prefix_similarity(self, prefix_id, k_ref, v_ref):
+        """Eq. 3 per layer: cosine between the cached K/V of a prefix and k_ref, v_ref [L, m, Hkv, D]."""
+        assert k_ref.is_cuda and v_ref.is_cuda and k_ref.dtype == self.dtype and k_ref.shape == v_ref.shape
+        assert k_ref.stride()[1:] == (self.Hkv * self.D, self.D, 1) and v_ref.stride() == k_ref.stride()
+        sim = np.zeros(self.L, dtype=np.float32)
+        st = self.lib.bicache_prefix_similarity(self.ctx, prefix_id, k_ref.data_ptr(), v_ref.data_ptr(),
+                                                k_ref.stride(0), sim.ctypes.data_as(C.POINTER(C.c_float)),
+                                                self._stream())
+        self._check(st, "bicache_prefix_similarity")
+        return sim
+
     def is_refresh_step(self, t, delta):
         return int(self.lib.bicache_is_refresh_step(t, delta))
 
@@ -320,3 +339,28 @@ def attend_full_static(q, k, v, out, scale=None):
     return lib.bicache_attend_full_static(_dtype_code(q.dtype), Hq, Hkv, D, n, q.data_ptr(), k.data_ptr(),
                                           v.data_ptr(), q.stride(0), k.stride(0), out.data_ptr(), out.stride(0),
                                           C.c_float(scale), C.c_void_p(torch.cuda.current_stream().cuda_stream))
+
+
+def depth_from_similarity(sim, tau):
+    """bicache_depth_from_similarity: leading layers with similarity >= tau."""
+    lib = load_library()
+    a = np.ascontiguousarray(sim, dtype=np.float32)
+    d = C.c_int32(-1)
+    st = lib.bicache_depth_from_similarity(a.ctypes.data_as(C.POINTER(C.c_float)), len(a), C.c_float(tau), C.byref(d))
+    if st != OK:
+        raise BiCacheError(st, "bicache_depth_from_similarity")
+    return d.value
+
+
+def build_depth_table(ratio_idx, depth, num_layers):
+    """bicache_build_depth_table: the 101-entry lookup table from profiled (ratio bin, depth) pairs."""
+    lib = load_library()
+    r = np.ascontiguousarray(ratio_idx, dtype=np.int32)
+    d = np.ascontiguousarray(depth, dtype=np.int32)
+    out = np.zeros(101, dtype=np.int32)
+    i32p = C.POINTER(C.c_int32)
+    st = lib.bicache_build_depth_table(r.ctypes.data_as(i32p), d.ctypes.data_as(i32p), len(r), num_layers,
+                                       out.ctypes.data_as(i32p))
+    if st != OK:
+        raise BiCacheError(st, "bicache_build_depth_table")
+    return out.tolist()

@@ -657,6 +657,80 @@ int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t
   return BICACHE_OK;
 }
 
+int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const void* k_ref, const void* v_ref,
+                                  int64_t layer_stride, float* sim_out, void* stream_) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  const bicache_config& cfg = ctx->cfg;
+  auto found = ctx->by_id.find(prefix_id);
+  if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+  if (!sim_out) return fail(ctx, BICACHE_ERR_INVALID, "sim_out is required");
+  const PrefixEntry& e = *found->second;
+  const int64_t row_elems = (int64_t)cfg.num_kv_heads * cfg.head_dim;
+  if (layer_stride < (int64_t)e.m * row_elems || (layer_stride * ctx->esize) % 16)
+    return fail(ctx, BICACHE_ERR_INVALID, "bad layer stride");
+  if (ctx->host_only) return fail(ctx, BICACHE_ERR_UNSUPPORTED, "host-only context");
+  if (!k_ref || !v_ref || !aligned16(k_ref) || !aligned16(v_ref))
+    return fail(ctx, BICACHE_ERR_INVALID, "bad k/v pointer");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int need = (int)e.pages.size();
+  // scratch: the key-split partials area (no attention call of this context can be running on it:
+  // calls on one context are stream-ordered)
+  double* partials = reinterpret_cast<double*>(ctx->d_part_o);
+  float* d_sim = reinterpret_cast<float*>(partials + (size_t)cfg.num_layers * kSimBlocksPerLayer * 3);
+  cudaError_t ce =
+      cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+  if (ce == cudaSuccess) {
+    const int chunks_per_row = cfg.head_dim * ctx->esize / 16;
+    const PoolView pv = pool_view(ctx);
+    const dim3 grid(kSimBlocksPerLayer, cfg.num_layers);
+    if (cfg.dtype == BICACHE_F32)
+      kv_similarity_partial_kernel<float><<<grid, kSimThreads, 0, stream>>>(
+          pv.k, pv.v, static_cast<const char*>(k_ref), static_cast<const char*>(v_ref), ctx->d_put_pages, e.m,
+          cfg.num_kv_heads, chunks_per_row, layer_stride * ctx->esize, pv.layer_bytes, pv.page_bytes, pv.swizzled,
+          partials);
+    else
+      kv_similarity_partial_kernel<__nv_bfloat16><<<grid, kSimThreads, 0, stream>>>(
+          pv.k, pv.v, static_cast<const char*>(k_ref), static_cast<const char*>(v_ref), ctx->d_put_pages, e.m,
+          cfg.num_kv_heads, chunks_per_row, layer_stride * ctx->esize, pv.layer_bytes, pv.page_bytes, pv.swizzled,
+          partials);
+    kv_similarity_final_kernel<<<(cfg.num_layers + 63) / 64, 64, 0, stream>>>(partials, kSimBlocksPerLayer,
+                                                                               cfg.num_layers, d_sim);
+    ctx->launches += 2;
+    ce = cudaGetLastError();
+  }
+  if (ce == cudaSuccess)
+    ce = cudaMemcpyAsync(sim_out, d_sim, sizeof(float) * cfg.num_layers, cudaMemcpyDeviceToHost, stream);
+  if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
+  if (ce != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("prefix_similarity: ") + cudaGetErrorString(ce));
+  return BICACHE_OK;
+}
+
+int32_t bicache_depth_from_similarity(const float* sim, int32_t num_layers, float tau, int32_t* depth) {
+  if (num_layers < 0 || (num_layers > 0 && !sim) || !depth) return BICACHE_ERR_INVALID;
+  int32_t b = 0;
+  while (b < num_layers && sim[b] >= tau) ++b;          // NaN compares false: it ends the run
+  *depth = b;
+  return BICACHE_OK;
+}
+
+int32_t bicache_build_depth_table(const int32_t* ratio_idx, const int32_t* depth, int32_t n, int32_t num_layers,
+                                  int32_t* table_out) {
+  if (n < 0 || num_layers < 0 || !table_out || (n > 0 && (!ratio_idx || !depth))) return BICACHE_ERR_INVALID;
+  long long sums[101] = {0};
+  long long cnts[101] = {0};
+  for (int i = 0; i < n; ++i) {
+    if (ratio_idx[i] < 0 || ratio_idx[i] > 100 || depth[i] < 0 || depth[i] > num_layers) return BICACHE_ERR_INVALID;
+    sums[ratio_idx[i]] += depth[i];
+    cnts[ratio_idx[i]] += 1;
+  }
+  int32_t last = num_layers < 1 ? num_layers : 1;
+  for (int idx = 0; idx <= 100; ++idx) {
+    if (cnts[idx]) last = (int32_t)(sums[idx] / cnts[idx]);
+    table_out[idx] = last;
+  }
+  return BICACHE_OK;
+}
+
 int32_t bicache_is_refresh_step(int32_t t, int32_t delta) {
   if (t < 1 || delta < 1) return -1;
   return (t - 1) % delta == 0 ? 1 : 0;

@@ -92,6 +92,124 @@ __global__ void scatter_prefix_kernel(const char* __restrict__ src_k, const char
 }
 
 // ---------------------------------------------------------------------------------------------
+// Profiler reduction (Eq. 3): for every layer the three sums behind
+//   sim_l = cos(KV$_l, KVref_l) = <a, b> / (|a| |b|),
+// a = the cached prefix's K and V of layer l read through the page table, b = the reference K and V
+// [L][m][Hkv][D], each side taken as one vector.  HBM bound: both sides are read once, 16 bytes per
+// thread and step; consecutive threads walk the reference in memory order (the page image holds the
+// same chunks permuted inside 128-byte rows).  Products and squares are summed in fp32 inside a
+// chunk, in fp64 across chunks; each block writes its three partial sums and a second kernel adds
+// them in a fixed order, so the result does not depend on scheduling.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSimBlocksPerLayer = 128;
+constexpr int kSimThreads = 256;
+
+template <typename T>
+__device__ __forceinline__ void chunk_sums(const uint4& a, const uint4& b, float& dot, float& na, float& nb);
+template <>
+__device__ __forceinline__ void chunk_sums<float>(const uint4& a, const uint4& b, float& dot, float& na, float& nb) {
+  const float* x = reinterpret_cast<const float*>(&a);
+  const float* y = reinterpret_cast<const float*>(&b);
+  dot = na = nb = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    dot = fmaf(x[i], y[i], dot);
+    na = fmaf(x[i], x[i], na);
+    nb = fmaf(y[i], y[i], nb);
+  }
+}
+template <>
+__device__ __forceinline__ void chunk_sums<__nv_bfloat16>(const uint4& a, const uint4& b, float& dot, float& na,
+                                                           float& nb) {
+  const __nv_bfloat162* x = reinterpret_cast<const __nv_bfloat162*>(&a);
+  const __nv_bfloat162* y = reinterpret_cast<const __nv_bfloat162*>(&b);
+  dot = na = nb = 0.f;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 xf = __bfloat1622float2(x[i]), yf = __bfloat1622float2(y[i]);
+    dot = fmaf(xf.x, yf.x, fmaf(xf.y, yf.y, dot));
+    na = fmaf(xf.x, xf.x, fmaf(xf.y, xf.y, na));
+    nb = fmaf(yf.x, yf.x, fmaf(yf.y, yf.y, nb));
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kSimThreads)
+kv_similarity_partial_kernel(const char* __restrict__ pool_k, const char* __restrict__ pool_v,
+                             const char* __restrict__ ref_k, const char* __restrict__ ref_v,
+                             const int* __restrict__ pages, int m, int num_kv_heads, int chunks_per_row,
+                             long long ref_layer_stride_bytes, long long pool_layer_bytes, int page_bytes,
+                             int swizzled, double* __restrict__ partials) {
+  const int layer = blockIdx.y;
+  const int row_bytes = chunks_per_row * 16;
+  const long long per_tensor = (long long)m * num_kv_heads * chunks_per_row;
+  double dot = 0.0, na = 0.0, nb = 0.0;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < 2 * per_tensor;
+       idx += (long long)gridDim.x * blockDim.x) {
+    const bool is_v = idx >= per_tensor;
+    long long rem = is_v ? idx - per_tensor : idx;
+    const int c16 = (int)(rem % chunks_per_row); rem /= chunks_per_row;
+    const int hk = (int)(rem % num_kv_heads);
+    const int t = (int)(rem / num_kv_heads);
+    const int page = pages[t / kPageSize];
+    const char* pa = (is_v ? pool_v : pool_k) + (long long)layer * pool_layer_bytes +
+                     ((long long)page * num_kv_heads + hk) * page_bytes +
+                     page_chunk_offset(swizzled != 0, t % kPageSize, c16, row_bytes);
+    const char* pb = (is_v ? ref_v : ref_k) + (long long)layer * ref_layer_stride_bytes +
+                     ((long long)t * num_kv_heads + hk) * row_bytes + c16 * 16;
+    const uint4 a = *reinterpret_cast<const uint4*>(pa);
+    const uint4 b = *reinterpret_cast<const uint4*>(pb);
+    float d, x, y;
+    chunk_sums<T>(a, b, d, x, y);
+    dot += d;
+    na += x;
+    nb += y;
+  }
+  // block reduction in a fixed order: shuffles inside a warp, then warp 0 over the warps' sums
+  __shared__ double red[3][kSimThreads / 32];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    dot += __shfl_down_sync(0xffffffffu, dot, o);
+    na += __shfl_down_sync(0xffffffffu, na, o);
+    nb += __shfl_down_sync(0xffffffffu, nb, o);
+  }
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) {
+    red[0][warp] = dot;
+    red[1][warp] = na;
+    red[2][warp] = nb;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s0 = 0.0, s1 = 0.0, s2 = 0.0;
+    for (int w = 0; w < kSimThreads / 32; ++w) {
+      s0 += red[0][w];
+      s1 += red[1][w];
+      s2 += red[2][w];
+    }
+    double* out = partials + ((long long)layer * gridDim.x + blockIdx.x) * 3;
+    out[0] = s0;
+    out[1] = s1;
+    out[2] = s2;
+  }
+}
+
+// One thread per layer adds the blocks' partial sums in block order and forms the cosine.
+__global__ void kv_similarity_final_kernel(const double* __restrict__ partials, int blocks_per_layer, int num_layers,
+                                           float* __restrict__ sim) {
+  const int layer = blockIdx.x * blockDim.x + threadIdx.x;
+  if (layer >= num_layers) return;
+  double dot = 0.0, na = 0.0, nb = 0.0;
+  for (int b = 0; b < blocks_per_layer; ++b) {
+    const double* p = partials + ((long long)layer * blocks_per_layer + b) * 3;
+    dot += p[0];
+    na += p[1];
+    nb += p[2];
+  }
+  sim[layer] = (na > 0.0 && nb > 0.0) ? (float)(dot / (sqrt(na) * sqrt(nb))) : 0.f;
+}
+
+// ---------------------------------------------------------------------------------------------
 // SIMT attention.  One block = one work item (128 packed rows of one request and KV head); each
 // warp takes packed rows warp, warp + nwarps, ...  Keys are visited 32 at a time: lane j scores
 // key j, the chunk maximum and sum are reduced with shuffles, and P.V is accumulated with each lane

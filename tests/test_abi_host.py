@@ -196,3 +196,31 @@ def test_refresh_rule_and_reserve_on_host_context(lib):
     assert lib.bicache_attend_step(ctx, 0, 2, 16, 1, i32(0), i32(-1), i32(pid.value), i64(0), i32(5), *args) \
         == binding.ERR_INVALID                                                   # shorter than its kept prefix
     lib.bicache_destroy(ctx)
+
+
+def test_profiler_host_pieces_match_oracle(lib):
+    """Depth under a threshold and the table from profiled depths: pure host functions."""
+    from hypothesis import strategies as hst
+    cases = [([1.0, 0.99, 0.98, 0.96, 0.99], 0.97), ([1.0, 0.97, 0.97], 0.97), ([0.5, 1.0], 0.97), ([], 0.5),
+             ([1.0, float("nan"), 1.0], 0.97)]
+    for sim, tau in cases:
+        assert binding.depth_from_similarity(sim, tau) == oracle.depth_from_similarity(np.float32(sim), np.float32(tau))
+    rng = np.random.default_rng(0)
+    for _ in range(50):
+        n = int(rng.integers(0, 60))
+        L = int(rng.integers(0, 40))
+        idx = rng.integers(0, 101, n).tolist()
+        b = rng.integers(0, L + 1, n).tolist()
+        assert binding.build_depth_table(idx, b, L) == oracle.build_depth_table(idx, b, L)
+    with pytest.raises(binding.BiCacheError):
+        binding.build_depth_table([101], [1], 32)
+    with pytest.raises(binding.BiCacheError):
+        binding.build_depth_table([5], [33], 32)
+    ctx = host_ctx(lib)
+    sim = np.zeros(2, dtype=np.float32)
+    sp = sim.ctypes.data_as(C.POINTER(C.c_float))
+    assert lib.bicache_prefix_similarity(ctx, 0, None, None, 1 << 20, sp, None) == binding.ERR_NOTFOUND
+    assert put(lib, ctx, 1, 20)[0] == binding.OK
+    assert lib.bicache_prefix_similarity(ctx, 0, None, None, 8, sp, None) == binding.ERR_INVALID        # stride < m rows
+    assert lib.bicache_prefix_similarity(ctx, 0, None, None, 1 << 20, sp, None) == binding.ERR_UNSUPPORTED
+    lib.bicache_destroy(ctx)
