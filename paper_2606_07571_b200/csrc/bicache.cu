@@ -682,7 +682,8 @@ int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const voi
   if (ce == cudaSuccess) {
     const int chunks_per_row = cfg.head_dim * ctx->esize / 16;
     const PoolView pv = pool_view(ctx);
-    const dim3 grid(kSimBlocksPerLayer, cfg.num_layers);
+    const int bpl = std::max(1, std::min(kSimBlocksPerLayer, 2 * e.m));       // a block takes whole rows
+    const dim3 grid(bpl, cfg.num_layers);
     if (cfg.dtype == BICACHE_F32)
       kv_similarity_partial_kernel<float><<<grid, kSimThreads, 0, stream>>>(
           pv.k, pv.v, static_cast<const char*>(k_ref), static_cast<const char*>(v_ref), ctx->d_put_pages, e.m,
@@ -693,8 +694,7 @@ int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const voi
           pv.k, pv.v, static_cast<const char*>(k_ref), static_cast<const char*>(v_ref), ctx->d_put_pages, e.m,
           cfg.num_kv_heads, chunks_per_row, layer_stride * ctx->esize, pv.layer_bytes, pv.page_bytes, pv.swizzled,
           partials);
-    kv_similarity_final_kernel<<<(cfg.num_layers + 63) / 64, 64, 0, stream>>>(partials, kSimBlocksPerLayer,
-                                                                               cfg.num_layers, d_sim);
+    kv_similarity_final_kernel<<<(cfg.num_layers + 63) / 64, 64, 0, stream>>>(partials, bpl, cfg.num_layers, d_sim);
     ctx->launches += 2;
     ce = cudaGetLastError();
   }

@@ -140,30 +140,57 @@ kv_similarity_partial_kernel(const char* __restrict__ pool_k, const char* __rest
                              const int* __restrict__ pages, int m, int num_kv_heads, int chunks_per_row,
                              long long ref_layer_stride_bytes, long long pool_layer_bytes, int page_bytes,
                              int swizzled, double* __restrict__ partials) {
+  // Rows of the layer: the m K rows, then the m V rows; a block takes a contiguous range of them.
+  // A thread keeps its chunk column(s) of the row and walks down the rows, so the per-chunk work is
+  // two loads, a handful of integer operations and the sums (no division in the loop).
   const int layer = blockIdx.y;
   const int row_bytes = chunks_per_row * 16;
-  const long long per_tensor = (long long)m * num_kv_heads * chunks_per_row;
+  const int row_chunks = num_kv_heads * chunks_per_row;     // 16-byte chunks of one token row
+  const int tpr = min(row_chunks, (int)blockDim.x);         // threads that share a row
+  const int rpp = (int)blockDim.x / tpr;                    // rows in flight per pass
+  const int r_local = (int)threadIdx.x / tpr, c0 = (int)threadIdx.x - r_local * tpr;
+  const int rows = 2 * m;
+  const int per_block = (rows + (int)gridDim.x - 1) / (int)gridDim.x;
+  const int row_begin = (int)blockIdx.x * per_block, row_end = min(rows, row_begin + per_block);
+  const char* pool_k_l = pool_k + (long long)layer * pool_layer_bytes;
+  const char* pool_v_l = pool_v + (long long)layer * pool_layer_bytes;
+  const char* ref_k_l = ref_k + (long long)layer * ref_layer_stride_bytes;
+  const char* ref_v_l = ref_v + (long long)layer * ref_layer_stride_bytes;
+  const long long page_stride = (long long)num_kv_heads * page_bytes;
   double dot = 0.0, na = 0.0, nb = 0.0;
-  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < 2 * per_tensor;
-       idx += (long long)gridDim.x * blockDim.x) {
-    const bool is_v = idx >= per_tensor;
-    long long rem = is_v ? idx - per_tensor : idx;
-    const int c16 = (int)(rem % chunks_per_row); rem /= chunks_per_row;
-    const int hk = (int)(rem % num_kv_heads);
-    const int t = (int)(rem / num_kv_heads);
-    const int page = pages[t / kPageSize];
-    const char* pa = (is_v ? pool_v : pool_k) + (long long)layer * pool_layer_bytes +
-                     ((long long)page * num_kv_heads + hk) * page_bytes +
-                     page_chunk_offset(swizzled != 0, t % kPageSize, c16, row_bytes);
-    const char* pb = (is_v ? ref_v : ref_k) + (long long)layer * ref_layer_stride_bytes +
-                     ((long long)t * num_kv_heads + hk) * row_bytes + c16 * 16;
-    const uint4 a = *reinterpret_cast<const uint4*>(pa);
-    const uint4 b = *reinterpret_cast<const uint4*>(pb);
-    float d, x, y;
-    chunk_sums<T>(a, b, d, x, y);
-    dot += d;
-    na += x;
-    nb += y;
+  constexpr int kUnroll = 4;                      // loads of four rows in flight before any arithmetic
+  if (r_local < rpp) {
+    for (int c = c0; c < row_chunks; c += tpr) {
+      const int hk = c / chunks_per_row, c16 = c - hk * chunks_per_row;
+      const long long slice = (long long)hk * page_bytes;
+      for (int base = row_begin + r_local; base < row_end; base += kUnroll * rpp) {
+        uint4 a[kUnroll], b[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+          const int row = base + u * rpp;
+          a[u] = make_uint4(0, 0, 0, 0);
+          b[u] = a[u];
+          if (row < row_end) {
+            const bool is_v = row >= m;
+            const int t = is_v ? row - m : row;
+            const int page = pages[t / kPageSize];
+            const char* pa = (is_v ? pool_v_l : pool_k_l) + page * page_stride + slice +
+                             page_chunk_offset(swizzled != 0, t % kPageSize, c16, row_bytes);
+            const char* pb = (is_v ? ref_v_l : ref_k_l) + ((long long)t * row_chunks + c) * 16;
+            a[u] = *reinterpret_cast<const uint4*>(pa);
+            b[u] = *reinterpret_cast<const uint4*>(pb);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {       // rows past the end are zeros and add nothing
+          float d, x, y;
+          chunk_sums<T>(a[u], b[u], d, x, y);
+          dot += d;
+          na += x;
+          nb += y;
+        }
+      }
+    }
   }
   // block reduction in a fixed order: shuffles inside a warp, then warp 0 over the warps' sums
   __shared__ double red[3][kSimThreads / 32];
