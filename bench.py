@@ -33,7 +33,8 @@ UNIT = "tokens/s"
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from ncu captures summarised
 # under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {"config2": {"full": 651.0e6, "attend": 138.2e6}}     # profiles/tc_attention_kernel_config2.md
+NCU_TRAFFIC_BYTES = {"config2": {"full": 651.0e6, "attend": 138.2e6},
+                     "config3": {"put": 2104.6e6, "similarity": 2147.6e6}}     # profiles/tc_attention_kernel_config2.md
 
 
 def load_peaks():
@@ -441,11 +442,12 @@ def main():
         kc, vc = workloads.draw_prefix_kv(w, 0, "cuda")
         # profiler reduction (Eq. 3): cached prefix 0 against a reference K/V of the same shape; reads both once
         ts = []
+        sim_dev = torch.zeros(w.num_layers, dtype=torch.float32, device="cuda")
         for i in range(5):
             flush.zero_()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
-            bc.prefix_similarity(pid[0], kc, vc)
+            bc.prefix_similarity_async(pid[0], kc, vc, sim_dev)
             b.record()
             torch.cuda.synchronize()
             ts.append(a.elapsed_time(b))
@@ -454,7 +456,7 @@ def main():
         roofline_sim = {"bound": "hbm", "kernel": "kv_similarity_partial_kernel (prefix_similarity of prefix 0)",
                         "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                         "peak_source": peaks["source"], "bytes_per_launch": put_bytes, "ms_per_launch": ms_sim,
-                        "traffic": None}
+                        "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("similarity")}
         ts = []
         for i in range(5):
             flush.zero_()
@@ -470,7 +472,7 @@ def main():
         roofline_put = {"bound": "hbm", "kernel": "scatter_prefix_kernel (put_prefix of prefix 0, all layers)",
                         "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                         "peak_source": peaks["source"], "bytes_per_launch": put_bytes, "ms_per_launch": ms_put,
-                        "traffic": None}
+                        "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("put")}
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -249,6 +249,11 @@ int32_t bicache_attend_step(bicache_ctx* ctx, int32_t layer, int32_t t, int32_t 
 int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const void* k_ref, const void* v_ref,
                                   int64_t layer_stride, float* sim_out, void* stream);
 
+/* The same reduction without the copy to the host and without the synchronisation: sim_dev is a DEVICE
+ * array of L floats, written on `stream`. */
+int32_t bicache_prefix_similarity_async(bicache_ctx* ctx, int32_t prefix_id, const void* k_ref,
+                                        const void* v_ref, int64_t layer_stride, float* sim_dev, void* stream);
+
 /* *depth = the number of leading layers whose similarity is >= tau (Sec. 4.2: the largest b such that
  * every layer 1 .. b is at or above the threshold; tau = 0.97 in the paper).  Host arrays, no context;
  * a NaN ends the run. */

@@ -24,7 +24,8 @@ EXPORTED = [
     "bicache_prefix_pages", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
     "bicache_attend_layer", "bicache_attend_full_static",
     "bicache_is_refresh_step", "bicache_reserve_prefix", "bicache_update_prefix_layer", "bicache_attend_step",
-    "bicache_prefix_similarity", "bicache_depth_from_similarity", "bicache_build_depth_table",
+    "bicache_prefix_similarity", "bicache_prefix_similarity_async", "bicache_depth_from_similarity",
+    "bicache_build_depth_table",
     "bicache_device_status", "bicache_launch_count", "bicache_last_error",
 ]
 
@@ -101,6 +102,8 @@ def load_library():
     f32p = C.POINTER(C.c_float)
     lib.bicache_prefix_similarity.restype = C.c_int32
     lib.bicache_prefix_similarity.argtypes = [vp, C.c_int32, vp, vp, C.c_int64, f32p, vp]
+    lib.bicache_prefix_similarity_async.restype = C.c_int32
+    lib.bicache_prefix_similarity_async.argtypes = [vp, C.c_int32, vp, vp, C.c_int64, vp, vp]
     lib.bicache_depth_from_similarity.restype = C.c_int32
     lib.bicache_depth_from_similarity.argtypes = [f32p, C.c_int32, C.c_float, i32p]
     lib.bicache_build_depth_table.restype = C.c_int32
@@ -240,6 +243,15 @@ class BiCache:
                                                 self._stream())
         self._check(st, "bicache_prefix_similarity")
         return sim
+
+    def prefix_similarity_async(self, prefix_id, k_ref, v_ref, sim_dev):
+        """As prefix_similarity, result into the device tensor sim_dev [L] (float32), no synchronisation."""
+        assert k_ref.is_cuda and v_ref.is_cuda and k_ref.dtype == self.dtype and k_ref.shape == v_ref.shape
+        assert k_ref.stride()[1:] == (self.Hkv * self.D, self.D, 1) and v_ref.stride() == k_ref.stride()
+        assert sim_dev.is_cuda and sim_dev.dtype == torch.float32 and sim_dev.numel() >= self.L and sim_dev.is_contiguous()
+        st = self.lib.bicache_prefix_similarity_async(self.ctx, prefix_id, k_ref.data_ptr(), v_ref.data_ptr(),
+                                                      k_ref.stride(0), sim_dev.data_ptr(), self._stream())
+        self._check(st, "bicache_prefix_similarity_async")
 
     def is_refresh_step(self, t, delta):
         return int(self.lib.bicache_is_refresh_step(t, delta))

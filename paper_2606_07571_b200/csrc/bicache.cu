@@ -657,13 +657,13 @@ int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t
   return BICACHE_OK;
 }
 
-int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const void* k_ref, const void* v_ref,
-                                  int64_t layer_stride, float* sim_out, void* stream_) {
+int32_t bicache_prefix_similarity_async(bicache_ctx* ctx, int32_t prefix_id, const void* k_ref, const void* v_ref,
+                                        int64_t layer_stride, float* sim_dev, void* stream_) {
   if (!ctx) return BICACHE_ERR_INVALID;
   const bicache_config& cfg = ctx->cfg;
   auto found = ctx->by_id.find(prefix_id);
   if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
-  if (!sim_out) return fail(ctx, BICACHE_ERR_INVALID, "sim_out is required");
+  if (!sim_dev) return fail(ctx, BICACHE_ERR_INVALID, "the output array is required");
   const PrefixEntry& e = *found->second;
   const int64_t row_elems = (int64_t)cfg.num_kv_heads * cfg.head_dim;
   if (layer_stride < (int64_t)e.m * row_elems || (layer_stride * ctx->esize) % 16)
@@ -676,7 +676,6 @@ int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const voi
   // scratch: the key-split partials area (no attention call of this context can be running on it:
   // calls on one context are stream-ordered)
   double* partials = reinterpret_cast<double*>(ctx->d_part_o);
-  float* d_sim = reinterpret_cast<float*>(partials + (size_t)cfg.num_layers * kSimBlocksPerLayer * 3);
   cudaError_t ce =
       cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
   if (ce == cudaSuccess) {
@@ -694,12 +693,25 @@ int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const voi
           pv.k, pv.v, static_cast<const char*>(k_ref), static_cast<const char*>(v_ref), ctx->d_put_pages, e.m,
           cfg.num_kv_heads, chunks_per_row, layer_stride * ctx->esize, pv.layer_bytes, pv.page_bytes, pv.swizzled,
           partials);
-    kv_similarity_final_kernel<<<(cfg.num_layers + 63) / 64, 64, 0, stream>>>(partials, bpl, cfg.num_layers, d_sim);
+    kv_similarity_final_kernel<<<(cfg.num_layers + 63) / 64, 64, 0, stream>>>(partials, bpl, cfg.num_layers, sim_dev);
     ctx->launches += 2;
     ce = cudaGetLastError();
   }
-  if (ce == cudaSuccess)
-    ce = cudaMemcpyAsync(sim_out, d_sim, sizeof(float) * cfg.num_layers, cudaMemcpyDeviceToHost, stream);
+  if (ce != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("prefix_similarity: ") + cudaGetErrorString(ce));
+  return BICACHE_OK;
+}
+
+int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const void* k_ref, const void* v_ref,
+                                  int64_t layer_stride, float* sim_out, void* stream_) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  if (!sim_out) return fail(ctx, BICACHE_ERR_INVALID, "sim_out is required");
+  // device copy of the result: behind the block partials in the key-split scratch area
+  float* d_sim = reinterpret_cast<float*>(reinterpret_cast<double*>(ctx->d_part_o) +
+                                          (size_t)ctx->cfg.num_layers * kSimBlocksPerLayer * 3);
+  const int32_t st = bicache_prefix_similarity_async(ctx, prefix_id, k_ref, v_ref, layer_stride, d_sim, stream_);
+  if (st != BICACHE_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  cudaError_t ce = cudaMemcpyAsync(sim_out, d_sim, sizeof(float) * ctx->cfg.num_layers, cudaMemcpyDeviceToHost, stream);
   if (ce == cudaSuccess) ce = cudaStreamSynchronize(stream);
   if (ce != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("prefix_similarity: ") + cudaGetErrorString(ce));
   return BICACHE_OK;

@@ -50,6 +50,9 @@ def test_similarity_matches_oracle(dtype, L, Hq, Hkv, D, m, shuffle):
     ref = oracle.kv_similarity(st, opid, workloads.to_f64(kr), workloads.to_f64(vr))
     assert np.abs(sim - ref).max() <= 1e-5, (sim, ref)
     assert sim[0] == pytest.approx(1.0, abs=1e-6)           # layer 0 has no noise
+    sim_dev = torch.full((L,), 7.0, dtype=torch.float32, device="cuda")
+    bc.prefix_similarity_async(pid, kr, vr, sim_dev)        # same numbers without the host copy
+    assert (sim_dev.cpu().numpy() == sim).all()
     for tau in (0.97, 0.9, 0.5):
         assert binding.depth_from_similarity(sim, tau) == oracle.depth_from_similarity(np.float32(ref), np.float32(tau))
     # identical / negated / zero references
