@@ -167,11 +167,8 @@ __device__ __forceinline__ void tmem_relinquish() {
 __device__ __forceinline__ void tmem_dealloc(unsigned taddr, unsigned cols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-__device__ __forceinline__ void mma_commit(unsigned bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// The same two MMAs issued by one elected lane of a converged warp, without a branch: the election
-// and the accumulate flag are predicates inside one asm block.  `enable` = 0 skips the MMA.
+// An MMA issued by one elected lane of a converged warp, without a branch: the election and the
+// accumulate flag are predicates inside one asm block.  `enable` = 0 skips the MMA.
 __device__ __forceinline__ void mma_ss_elect(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
                                              unsigned idesc, unsigned accumulate) {
   asm volatile(
@@ -252,26 +249,6 @@ __device__ __forceinline__ void mma_commit_pred(unsigned el, unsigned bar) {
       ::"r"(bar), "r"(el)
       : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
-                                       unsigned idesc, unsigned accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(unsigned d_tmem, unsigned a_tmem, unsigned long long b_desc,
-                                       unsigned idesc, unsigned accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
 __device__ __forceinline__ void tmem_ld32(unsigned taddr, unsigned* r) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -293,14 +270,6 @@ __device__ __forceinline__ void tmem_st32(unsigned taddr, const unsigned* r) {
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
         "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* r) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -566,7 +535,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           float mx0 = -INFINITY, mx1 = -INFINITY;
           // first half of the exponentials, with the maximum over all 128 scores computed alongside
           // (independent instructions that fill the exp unit's latency)
-  #pragma unroll
+#pragma unroll
           for (int i = 0; i < 16; ++i) {
             mx0 = max3(mx0, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]));
             mx1 = max3(mx1, __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
@@ -600,7 +569,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             tc_fence_before();
             mbar_arrive(smem_u32(&bars->p_half[X][0]));
 
-  #pragma unroll
+#pragma unroll
             for (int i = 16; i < 32; ++i) {
               const unsigned long long xa =
                   fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
@@ -637,11 +606,11 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             unsigned s4[32];
             const float neg_m = -m_ref;
             float ps = 0.f;
-  #pragma unroll
+#pragma unroll
             for (int c = 0; c < 4; ++c) {
               tmem_ld32(tmem_s + c * 32, s4);
               tmem_wait_ld();
-  #pragma unroll
+#pragma unroll
               for (int i = 0; i < 16; ++i) {
                 const float p0 = ex2(fmaf(__uint_as_float(s4[2 * i]), sl2, neg_m));
                 const float p1 = ex2(fmaf(__uint_as_float(s4[2 * i + 1]), sl2, neg_m));
@@ -652,11 +621,11 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             acc_a = pack2(ps, 0.f);
             acc_b = pack2(0.f, 0.f);
             // S(j) was committed after O += P V of tile j-1 was issued, so O is quiescent here.
-  #pragma unroll 1
+#pragma unroll 1
             for (int c = 0; c < 4; ++c) {
               tmem_ld32(tmem_o + c * 32, s4);
               tmem_wait_ld();
-  #pragma unroll
+#pragma unroll
               for (int i = 0; i < 32; ++i) s4[i] = __float_as_uint(__uint_as_float(s4[i]) * alpha);
               tmem_st32(tmem_o + c * 32, s4);
             }
@@ -665,12 +634,12 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           // First tile of the item, or a ragged tile: maximum first, every exponential on the exp
           // unit so that masked columns give exactly 0.
           if (cnt < kTileKeys) {
-  #pragma unroll
+#pragma unroll
             for (int i = 0; i < 128; ++i)
               if (i >= cnt) r[i] = 0xff800000u;                // -inf: columns past the last key
           }
           float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-  #pragma unroll
+#pragma unroll
           for (int i = 0; i < 128; i += 8) {
             mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
             mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
@@ -685,18 +654,18 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             m_ref = mx;
           }
           if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-  #pragma unroll 1
+#pragma unroll 1
             for (int c = 0; c < 4; ++c) {
               unsigned o[32];
               tmem_ld32(tmem_o + c * 32, o);
               tmem_wait_ld();
-  #pragma unroll
+#pragma unroll
               for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
               tmem_st32(tmem_o + c * 32, o);
             }
           }
           const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
-  #pragma unroll
+#pragma unroll
           for (int i = 0; i < 32; ++i) {
             const unsigned long long xa =
                 fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
