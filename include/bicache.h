@@ -271,6 +271,14 @@ int32_t bicache_build_depth_table(const int32_t* ratio_idx, const int32_t* depth
  * resets the word. */
 int32_t bicache_device_status(bicache_ctx* ctx, void* stream, int32_t clear);
 
+/* Budget, in SM clock cycles, of every device-side wait of the tensor-core kernel (on a barrier that a
+ * copy, an MMA or another warp completes).  A wait that exceeds it gives up: the CTA drains its copies
+ * and MMAs, releases its tensor memory and exits, and bicache_device_status reports TIMEOUT; outputs of
+ * that call are then undefined, the context stays usable once the status is cleared.  0 restores the
+ * default (about 0.2 s).  A tiny budget makes ordinary waits run out: that is how the tests exercise
+ * the give-up path without any barrier that could never complete.  INVALID for a negative value. */
+int32_t bicache_set_wait_budget(bicache_ctx* ctx, int64_t sm_cycles);
+
 /* Allocation-free full attention of ONE request (the paper has no counterpart: this entry point
  * exists for callers, not for the method).
  *

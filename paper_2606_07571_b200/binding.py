@@ -26,7 +26,7 @@ EXPORTED = [
     "bicache_is_refresh_step", "bicache_reserve_prefix", "bicache_update_prefix_layer", "bicache_attend_step",
     "bicache_prefix_similarity", "bicache_prefix_similarity_async", "bicache_depth_from_similarity",
     "bicache_build_depth_table",
-    "bicache_device_status", "bicache_launch_count", "bicache_last_error",
+    "bicache_device_status", "bicache_set_wait_budget", "bicache_launch_count", "bicache_last_error",
 ]
 
 
@@ -113,6 +113,8 @@ def load_library():
                                                C.c_int64, C.c_int64, vp, C.c_int64, C.c_float, vp]
     lib.bicache_device_status.restype = C.c_int32
     lib.bicache_device_status.argtypes = [vp, vp, C.c_int32]
+    lib.bicache_set_wait_budget.restype = C.c_int32
+    lib.bicache_set_wait_budget.argtypes = [vp, C.c_int64]
     lib.bicache_launch_count.restype = C.c_int64
     lib.bicache_launch_count.argtypes = [vp]
     lib.bicache_last_error.restype = C.c_char_p
@@ -330,6 +332,9 @@ class BiCache:
 
     def device_status(self, clear=False):
         return self.lib.bicache_device_status(self.ctx, self._stream(), 1 if clear else 0)
+
+    def set_wait_budget(self, sm_cycles):
+        self._check(self.lib.bicache_set_wait_budget(self.ctx, sm_cycles), "bicache_set_wait_budget")
 
     def launch_count(self):
         return int(self.lib.bicache_launch_count(self.ctx))

@@ -68,6 +68,7 @@ struct bicache_ctx {
   std::vector<int32_t> depth_table;
   // workspace carving
   int* d_status = nullptr;
+  long long wait_cycles = 0;       // SM-clock budget of the device-side waits (0: the kernel's default)
   char* d_slots = nullptr;
   size_t slot_bytes = 0;
   float* d_part_o = nullptr;
@@ -393,7 +394,7 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
     okm = okm && encode_map(&maps.o, out, rows_total, cfg.num_q_heads, out_row_stride, maps.o_tma ? G : 1,
                             maps.o_tma ? 32 / G : 32);
     if (!okm) return fail(ctx, BICACHE_ERR_CUDA, "tensor map encoding failed");
-    e = launch_tc_attention(sv, pool, t, ctx->d_status, ctx->sm_count, maps, stream);
+    e = launch_tc_attention(sv, pool, t, ctx->d_status, ctx->sm_count, maps, ctx->wait_cycles, stream);
   } else if (cfg.dtype == BICACHE_F32) {
     simt_attention_kernel<float><<<c.num_items, kSimtWarps * 32, 0, stream>>>(sv, pool, t);
     e = cudaGetLastError();
@@ -944,6 +945,12 @@ int32_t bicache_debug_read_trace(long long* out, int32_t n) {
   return cudaMemcpyFromSymbol(out, bicache::tc::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : 4;
 }
 #endif
+
+int32_t bicache_set_wait_budget(bicache_ctx* ctx, int64_t sm_cycles) {
+  if (!ctx || sm_cycles < 0) return BICACHE_ERR_INVALID;
+  ctx->wait_cycles = sm_cycles;
+  return BICACHE_OK;
+}
 
 int64_t bicache_launch_count(const bicache_ctx* ctx) { return ctx ? ctx->launches : 0; }
 

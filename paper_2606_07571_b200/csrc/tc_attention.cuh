@@ -49,7 +49,7 @@ constexpr int kMmaWarp = 8;
 #define BICACHE_POLY_PERIOD 0
 #endif
 constexpr int kPolyPeriod = BICACHE_POLY_PERIOD;                   // of every kPolyPeriod groups of 4 scores, one sends 2 scores to the FMA-pipe cubic (0: none)
-constexpr long long kWaitCycles = 400000000LL;   // bounded waits: about 0.2 s of SM clocks
+constexpr long long kWaitCycles = 400000000LL;   // default budget of a bounded wait: about 0.2 s of SM clocks
 
 // shared-memory layout (dynamic, 1024-byte aligned by hand): Q_A, Q_B, ring, output staging
 // (4 KB per softmax warp), barriers and item records
@@ -71,8 +71,10 @@ struct alignas(8) Barriers {
   unsigned long long o_done[2];          // the last O += P V of the item has completed (per query tile)
   unsigned long long o_free[2];          // the epilogue has read O out of TMEM (per query tile)
   unsigned long long drain;
-  unsigned tmem_base;
+  long long wait_cycles;                 // SM-clock budget of every wait; directly before abort_flag (mbar_wait reads it)
   int abort_flag;
+  unsigned tmem_base;
+  int dead;                              // the context's status word was already set when the CTA started
   ItemInfo info[2];
 };
 constexpr int kInfoReaders = 8 + 1 + 2;  // arrivals on info_free: softmax warps, the MMA warp, the two load warps
@@ -107,19 +109,33 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
 }
 // Bounded wait.  try_wait suspends the thread in hardware until the phase completes or a short
 // system time limit passes, so the loop itself needs no sleep; the SM clock bounds the total.
-// Returns false (and raises the CTA's abort flag) if the phase never completes.
+// Returns false if the CTA's abort flag is up or (raising it) if the budget runs out.
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (unsigned it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 0u) {
+    if ((it & 63u) == 1u) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitCycles) break;
+      // the budget sits in shared memory directly before the abort flag
+      if (clock64() - t0 > *reinterpret_cast<const volatile long long*>(abort_flag - 2)) break;
     }
   }
   *abort_flag = 1;
   return false;
+}
+// A budget below this is the tests' way to walk the give-up path with barriers that all complete:
+// the abort flag is up from the start, so every wait that is not over within its first two polls
+// gives up, and the launch reports a timeout.
+constexpr long long kStrictBudget = 1024;
+// Wait for work that is certain to finish (MMAs already issued): the default budget, whatever the
+// per-wait budget or the abort flag say, because tensor memory must not be released under them.
+__device__ __forceinline__ bool mbar_wait_issued(unsigned bar, unsigned parity) {
+  const long long t0 = clock64();
+  for (unsigned it = 0;; ++it) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((it & 63u) == 63u && clock64() - t0 > kWaitCycles) return false;
+  }
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
@@ -424,7 +440,7 @@ __global__ void __launch_bounds__(tc::kThreads, 1)
 tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
                     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int q_tma,
-                    int o_tma) {
+                    int o_tma, long long wait_cycles) {
   using namespace tc;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem =
@@ -443,7 +459,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
   const int G = t.Hq / t.Hkv;
 
   if (tid == 0) {
-    bars->abort_flag = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
+    bars->wait_cycles = wait_cycles;
+    bars->dead = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
+    bars->abort_flag = (bars->dead || wait_cycles < kStrictBudget) ? 1 : 0;
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&bars->info_full[i]), 1);
       mbar_init(smem_u32(&bars->info_free[i]), kInfoReaders);
@@ -473,7 +491,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
   if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1001] = clock64();
 #endif
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&bars->tmem_base);
-  const bool dead = *abort_flag != 0;        // an earlier launch or CTA already gave up: do no work
+  const bool dead = *reinterpret_cast<volatile int*>(&bars->dead) != 0;   // an earlier launch or CTA gave up: do no work
 
   // Registers move from the MMA/load warpgroup to the two softmax warpgroups, which hold a whole
   // row of S (128 values) per thread.  The counts must fit the CTA's launch allocation:
@@ -892,6 +910,14 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       __syncwarp();                                          // lane 0's record is visible to the warp
       ++n_it;
     }
+    cp_async_wait<0>();
+    // After a give-up, the Q loads issued last may still be in flight: wait (bounded) for them.
+    if (!dead && (!ok || *abort_flag) && lane == 0) {
+      for (int x = 0; x < 2; ++x)
+        if (eq[x] > 0)
+          for (unsigned it = 0; it < 4096 && !mbar_try_wait(smem_u32(&bars->q_full[x]), (eq[x] - 1) & 1); ++it)
+            __nanosleep(256);
+    }
   } else if (warp >= 10) {
     // ====================================== loads =======================================
     // Warp 10 stages the K tiles, warp 11 the V tiles, each running ahead of the MMAs by the depth
@@ -1220,7 +1246,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       // Whatever happened, let every MMA issued so far finish before TMEM is released.
       __syncwarp();
       mma_commit_elect(smem_u32(&bars->drain));               // elect.sync names the same lane as `el`
-      mbar_wait(smem_u32(&bars->drain), 0, abort_flag);
+      mbar_wait_issued(smem_u32(&bars->drain), 0);
     }
     __syncwarp();
   }
@@ -1267,10 +1293,12 @@ struct TcTensorMaps {
 // `status` points at the context's status area: word 0 is the sticky device status, words 16 and 17
 // are the item counter and the count of finished CTAs (both zero between launches).
 inline cudaError_t launch_tc_attention(const ScheduleView& s, const PoolView& pool, const TensorArgs& t,
-                                       int* status, int num_sms, const TcTensorMaps& maps, cudaStream_t stream) {
+                                       int* status, int num_sms, const TcTensorMaps& maps, long long wait_cycles,
+                                       cudaStream_t stream) {
   const int grid = s.num_items < num_sms ? s.num_items : num_sms;
-  tc_attention_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(s, pool, t, status, maps.q, maps.k, maps.v,
-                                                                        maps.o, maps.q_tma, maps.o_tma);
+  tc_attention_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(
+      s, pool, t, status, maps.q, maps.k, maps.v, maps.o, maps.q_tma, maps.o_tma,
+      wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
   return cudaGetLastError();
 }
 
