@@ -130,6 +130,12 @@ int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void
                            int64_t layer_stride, void* stream,
                            int32_t* prefix_id, int32_t* was_hit, int32_t* pages_out, int32_t pages_cap);
 
+/* k = h(p) (Sec. 5.2): the 64-bit identifier of a tokenised prefix, for use as the `key` of the store
+ * calls.  XXH64 with seed 0 over the n token ids taken as little-endian 32-bit integers (the paper's
+ * implementation hashes the token id sequence with xxHash).  Host array, no context; n = 0 gives the
+ * hash of the empty input; a negative n or a null array with n > 0 gives 0. */
+uint64_t bicache_hash_tokens(const int32_t* tokens, int64_t n);
+
 /* KV store lookup (Sec. 5.2 "On a cache hit").  NOTFOUND if the key is absent or evicted. */
 int32_t bicache_lookup_prefix(const bicache_ctx* ctx, uint64_t key, int32_t* prefix_id, int32_t* m);
 

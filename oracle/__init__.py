@@ -30,6 +30,9 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
                    orthogonally mixed tensors with cos = a / sqrt(a^2 + b^2);
                    scalar-loop brute force; hand-written threshold and
                    averaging cases).
+  xxh64/prefix_key (Sec. 5.2, k = h(p))
+                   pinned (the published digests of the empty input and of "a",
+                   and the `xxhash` library on random inputs of every tail length).
 """
 from .bicache_oracle import (  # noqa: F401
     OracleError,
@@ -44,6 +47,8 @@ from .bicache_oracle import (  # noqa: F401
     kv_similarity,
     depth_from_similarity,
     build_depth_table,
+    xxh64,
+    prefix_key,
     merge,
     attend,
     attend_full,

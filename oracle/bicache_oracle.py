@@ -13,7 +13,9 @@ Everything here is written from the paper's statement of the method:
   * Eq. 5  (deep layers l > b: the prefix KVs computed within the request are
     kept and reused across denoising steps, recomputed every Delta steps),
   * Eq. 3 + Sec. 4.2/5.1 (profiler: cosine similarity between cached and
-    reference prefix KVs per layer -> depth b_i under threshold tau -> table T).
+    reference prefix KVs per layer -> depth b_i under threshold tau -> table T),
+  * Sec. 5.2 + implementation appendix (k = h(p): a deterministic 64-bit hash,
+    XXH64, of the prefix's token ids is the cache key).
 
 All floating-point work is numpy float64.  A matrix product (numpy matmul) is
 used as a library step; there is no tiling, fusion, online softmax or any
@@ -543,3 +545,64 @@ def build_depth_table(ratio_idx, depths, num_layers):
             last = sums[idx] // cnts[idx]
         table.append(last)
     return table
+
+
+# ---------------------------------------------------------------------------
+# Cache key (Sec. 5.2 "k = h(p)"; implementation appendix: a 64-bit xxHash of the
+# tokenised prefix).  XXH64 with seed 0 over the token ids as little-endian
+# 32-bit integers, written out from the algorithm's published description.
+# ---------------------------------------------------------------------------
+
+_M64 = (1 << 64) - 1
+_XP1, _XP2, _XP3 = 0x9E3779B185EBCA87, 0xC2B2AE3D27D4EB4F, 0x165667B19E3779F9
+_XP4, _XP5 = 0x85EBCA77C2B2AE63, 0x27D4EB2F165667C5
+
+
+def _rotl(x, r):
+    return ((x << r) | (x >> (64 - r))) & _M64
+
+
+def _xround(acc, lane):
+    return (_rotl((acc + lane * _XP2) & _M64, 31) * _XP1) & _M64
+
+
+def xxh64(data, seed=0):
+    """XXH64 of a bytes object."""
+    n = len(data)
+    pos = 0
+    if n >= 32:
+        v = [(seed + _XP1 + _XP2) & _M64, (seed + _XP2) & _M64, seed & _M64, (seed - _XP1) & _M64]
+        while pos + 32 <= n:
+            for i in range(4):
+                v[i] = _xround(v[i], int.from_bytes(data[pos + 8 * i:pos + 8 * i + 8], "little"))
+            pos += 32
+        h = (_rotl(v[0], 1) + _rotl(v[1], 7) + _rotl(v[2], 12) + _rotl(v[3], 18)) & _M64
+        for i in range(4):
+            h = ((h ^ _xround(0, v[i])) * _XP1 + _XP4) & _M64
+    else:
+        h = (seed + _XP5) & _M64
+    h = (h + n) & _M64
+    while pos + 8 <= n:
+        h ^= _xround(0, int.from_bytes(data[pos:pos + 8], "little"))
+        h = (_rotl(h, 27) * _XP1 + _XP4) & _M64
+        pos += 8
+    if pos + 4 <= n:
+        h ^= (int.from_bytes(data[pos:pos + 4], "little") * _XP1) & _M64
+        h = (_rotl(h, 23) * _XP2 + _XP3) & _M64
+        pos += 4
+    while pos < n:
+        h ^= (data[pos] * _XP5) & _M64
+        h = (_rotl(h, 11) * _XP1) & _M64
+        pos += 1
+    h ^= h >> 33
+    h = (h * _XP2) & _M64
+    h ^= h >> 29
+    h = (h * _XP3) & _M64
+    h ^= h >> 32
+    return h
+
+
+def prefix_key(tokens):
+    """k = h(p): the 64-bit key of a prefix given as a sequence of token ids."""
+    raw = b"".join(int(t).to_bytes(4, "little", signed=True) for t in tokens)
+    return xxh64(raw, 0)

@@ -26,7 +26,7 @@ EXPORTED = [
     "bicache_is_refresh_step", "bicache_reserve_prefix", "bicache_update_prefix_layer", "bicache_attend_step",
     "bicache_prefix_similarity", "bicache_prefix_similarity_async", "bicache_depth_from_similarity",
     "bicache_build_depth_table",
-    "bicache_device_status", "bicache_set_wait_budget", "bicache_launch_count", "bicache_last_error",
+    "bicache_hash_tokens", "bicache_device_status", "bicache_set_wait_budget", "bicache_launch_count", "bicache_last_error",
 ]
 
 
@@ -113,6 +113,8 @@ def load_library():
                                                C.c_int64, C.c_int64, vp, C.c_int64, C.c_float, vp]
     lib.bicache_device_status.restype = C.c_int32
     lib.bicache_device_status.argtypes = [vp, vp, C.c_int32]
+    lib.bicache_hash_tokens.restype = C.c_uint64
+    lib.bicache_hash_tokens.argtypes = [i32p, C.c_int64]
     lib.bicache_set_wait_budget.restype = C.c_int32
     lib.bicache_set_wait_budget.argtypes = [vp, C.c_int64]
     lib.bicache_launch_count.restype = C.c_int64
@@ -381,3 +383,10 @@ def build_depth_table(ratio_idx, depth, num_layers):
     if st != OK:
         raise BiCacheError(st, "bicache_build_depth_table")
     return out.tolist()
+
+
+def hash_tokens(tokens):
+    """bicache_hash_tokens: the 64-bit store key of a prefix given as token ids."""
+    lib = load_library()
+    a = np.ascontiguousarray(tokens, dtype=np.int32)
+    return int(lib.bicache_hash_tokens(a.ctypes.data_as(C.POINTER(C.c_int32)), len(a)))

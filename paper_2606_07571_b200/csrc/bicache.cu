@@ -744,6 +744,54 @@ int32_t bicache_build_depth_table(const int32_t* ratio_idx, const int32_t* depth
   return BICACHE_OK;
 }
 
+// XXH64 (seed 0) of the token ids taken as little-endian 32-bit integers: the 64-bit identifier of a
+// tokenised prefix (Sec. 5.2 "k = h(p)").  Input length is a multiple of four bytes, so the tail is at
+// most one 8-byte lane, one 4-byte lane and no single bytes.
+uint64_t bicache_hash_tokens(const int32_t* tokens, int64_t n) {
+  constexpr uint64_t P1 = 0x9E3779B185EBCA87ull, P2 = 0xC2B2AE3D27D4EB4Full, P3 = 0x165667B19E3779F9ull,
+                     P4 = 0x85EBCA77C2B2AE63ull, P5 = 0x27D4EB2F165667C5ull;
+  auto rotl = [](uint64_t x, int r) { return (x << r) | (x >> (64 - r)); };
+  auto round = [&](uint64_t acc, uint64_t lane) { return rotl(acc + lane * P2, 31) * P1; };
+  auto lane64 = [&](int64_t i) {                     // tokens i, i + 1 as one little-endian 64-bit lane
+    return (uint64_t)(uint32_t)tokens[i] | ((uint64_t)(uint32_t)tokens[i + 1] << 32);
+  };
+  if (n < 0 || (n > 0 && !tokens)) return 0;
+  const uint64_t bytes = (uint64_t)n * 4;
+  int64_t i = 0;
+  uint64_t h;
+  if (n >= 8) {
+    uint64_t v1 = P1 + P2, v2 = P2, v3 = 0, v4 = 0 - P1;
+    for (; i + 8 <= n; i += 8) {
+      v1 = round(v1, lane64(i));
+      v2 = round(v2, lane64(i + 2));
+      v3 = round(v3, lane64(i + 4));
+      v4 = round(v4, lane64(i + 6));
+    }
+    h = rotl(v1, 1) + rotl(v2, 7) + rotl(v3, 12) + rotl(v4, 18);
+    h = (h ^ round(0, v1)) * P1 + P4;
+    h = (h ^ round(0, v2)) * P1 + P4;
+    h = (h ^ round(0, v3)) * P1 + P4;
+    h = (h ^ round(0, v4)) * P1 + P4;
+  } else {
+    h = P5;
+  }
+  h += bytes;
+  for (; i + 2 <= n; i += 2) {
+    h ^= round(0, lane64(i));
+    h = rotl(h, 27) * P1 + P4;
+  }
+  if (i < n) {
+    h ^= (uint64_t)(uint32_t)tokens[i] * P1;
+    h = rotl(h, 23) * P2 + P3;
+  }
+  h ^= h >> 33;
+  h *= P2;
+  h ^= h >> 29;
+  h *= P3;
+  h ^= h >> 32;
+  return h;
+}
+
 int32_t bicache_is_refresh_step(int32_t t, int32_t delta) {
   if (t < 1 || delta < 1) return -1;
   return (t - 1) % delta == 0 ? 1 : 0;

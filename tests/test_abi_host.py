@@ -224,3 +224,20 @@ def test_profiler_host_pieces_match_oracle(lib):
     assert lib.bicache_prefix_similarity(ctx, 0, None, None, 8, sp, None) == binding.ERR_INVALID        # stride < m rows
     assert lib.bicache_prefix_similarity(ctx, 0, None, None, 1 << 20, sp, None) == binding.ERR_UNSUPPORTED
     lib.bicache_destroy(ctx)
+
+
+def test_hash_tokens_matches_oracle(lib):
+    """k = h(p): the library's key of a token sequence against the oracle's XXH64, every tail length."""
+    rng = np.random.default_rng(3)
+    for n in list(range(0, 40)) + [127, 128, 129, 2048, 16385]:
+        toks = rng.integers(-2 ** 31, 2 ** 31, n, dtype=np.int64).astype(np.int32)
+        assert binding.hash_tokens(toks) == oracle.prefix_key(toks.tolist()), n
+    assert binding.hash_tokens([]) == 0xEF46DB3751D8E999
+    a, b = binding.hash_tokens([5, 6, 7]), binding.hash_tokens([5, 6, 8])
+    assert a != b                                             # one token apart, another key
+    # the key drives the store: same tokens hit, other tokens miss
+    ctx = host_ctx(lib, L=1, Hq=1, Hkv=1, pages=4)
+    assert put(lib, ctx, a, 16)[:3] == (binding.OK, 0, 0)
+    assert put(lib, ctx, binding.hash_tokens([5, 6, 7]), 16)[:3] == (binding.OK, 0, 1)
+    assert put(lib, ctx, b, 16)[:3] == (binding.OK, 1, 0)
+    lib.bicache_destroy(ctx)

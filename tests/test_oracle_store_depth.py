@@ -150,3 +150,18 @@ def test_workload_recipes_are_deterministic_and_shaped():
     assert q.shape == (4 * 96, 4, 64) and (q == q2).all()
     small = workloads.scaled_down(w, num_layers=2, max_requests=12, prefix_div=16, suffix_div=8)
     assert small.num_requests == 12 and small.req_prefix == sorted(small.req_prefix)
+
+
+def test_prefix_key_is_xxh64_of_the_token_ids():
+    """Pins for the oracle's hash: the published XXH64 digests of the empty input and of "a", and the
+    xxhash library (a third party's implementation) on inputs of every tail length."""
+    xxhash = pytest.importorskip("xxhash")
+    assert oracle.xxh64(b"") == 0xEF46DB3751D8E999
+    assert oracle.xxh64(b"a") == 0xD24EC4F1A98C6E5B
+    rng = np.random.default_rng(0)
+    for n in list(range(0, 80)) + [255, 256, 1000]:
+        data = rng.integers(0, 256, n, dtype=np.uint8).tobytes()
+        assert oracle.xxh64(data) == xxhash.xxh64(data).intdigest(), n
+        assert oracle.xxh64(data, 12345) == xxhash.xxh64(data, seed=12345).intdigest(), n
+    toks = [1, 2, 3, -1, 2 ** 31 - 1]
+    assert oracle.prefix_key(toks) == xxhash.xxh64(np.asarray(toks, dtype="<i4").tobytes()).intdigest()
