@@ -211,7 +211,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   int num_splits = 1, tiles_per_split = 0;
   if (unsplit_items > 0 && unsplit_items < 2LL * ctx->sm_count && max_key_tiles >= 8) {
     const int key_tiles = max_key_tiles;
-    const double c_tile = 3000.0, c_cta = 8000.0;          // SM clocks
+    const double c_tile = 3300.0, c_cta = 12000.0;         // SM clocks, fitted on the small-suffix shapes
     auto cost = [&](int nsplit, int tps) {
       const long long ctas = unsplit_items * nsplit;
       const double waves = (double)((ctas + ctx->sm_count - 1) / ctx->sm_count);
