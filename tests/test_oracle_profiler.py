@@ -86,3 +86,34 @@ def test_table_from_profiled_depths_hand_case():
         oracle.build_depth_table([101], [1], 32)
     with pytest.raises(oracle.InvalidArgument):
         oracle.build_depth_table([5], [33], 32)
+
+
+def test_similarity_distance_bound():
+    """1 - cos(a, b) <= |a - b|^2 / (2 |a| |b|), with equality when |a| = |b| (the paper's auxiliary
+    lemma on cosine similarity and distance): an inequality and an identity the oracle's similarity
+    must satisfy, computed here from norms of differences only."""
+    rng = np.random.default_rng(3)
+    L, m, Hkv, D = 4, 11, 2, 8
+    k, v = rng.standard_normal((L, m, Hkv, D)), rng.standard_normal((L, m, Hkv, D))
+    st, pid = _store_with(k, v)
+    kr = k + 0.3 * rng.standard_normal(k.shape)
+    vr = 1.7 * v + 0.1 * rng.standard_normal(v.shape)
+    sim = oracle.kv_similarity(st, pid, kr, vr)
+    for l in range(L):
+        a = np.concatenate([k[l].ravel(), v[l].ravel()])
+        b = np.concatenate([kr[l].ravel(), vr[l].ravel()])
+        bound = np.linalg.norm(a - b) ** 2 / (2 * np.linalg.norm(a) * np.linalg.norm(b))
+        assert 1 - sim[l] <= bound + 1e-12
+        assert 1 - sim[l] > 0
+    # equal norms: the bound is attained
+    for l in range(L):
+        a = np.concatenate([k[l].ravel(), v[l].ravel()])
+        b = np.concatenate([kr[l].ravel(), vr[l].ravel()])
+        s = np.linalg.norm(a) / np.linalg.norm(b)
+        kr[l] *= s
+        vr[l] *= s
+    sim = oracle.kv_similarity(st, pid, kr, vr)
+    for l in range(L):
+        a = np.concatenate([k[l].ravel(), v[l].ravel()])
+        b = np.concatenate([kr[l].ravel(), vr[l].ravel()])
+        assert abs((1 - sim[l]) - np.linalg.norm(a - b) ** 2 / (2 * np.linalg.norm(a) * np.linalg.norm(b))) < 1e-12
