@@ -33,6 +33,9 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
   xxh64/prefix_key (Sec. 5.2, k = h(p))
                    pinned (the published digests of the empty input and of "a",
                    and the `xxhash` library on random inputs of every tail length).
+  project_kv (Eq. 1)
+                   pinned (scalar-loop brute force, selector weights that copy
+                   chosen hidden components, linearity).
 """
 from .bicache_oracle import (  # noqa: F401
     OracleError,
@@ -49,6 +52,7 @@ from .bicache_oracle import (  # noqa: F401
     build_depth_table,
     xxh64,
     prefix_key,
+    project_kv,
     merge,
     attend,
     attend_full,

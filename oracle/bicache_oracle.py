@@ -15,7 +15,8 @@ Everything here is written from the paper's statement of the method:
   * Eq. 3 + Sec. 4.2/5.1 (profiler: cosine similarity between cached and
     reference prefix KVs per layer -> depth b_i under threshold tau -> table T),
   * Sec. 5.2 + implementation appendix (k = h(p): a deterministic 64-bit hash,
-    XXH64, of the prefix's token ids is the cache key).
+    XXH64, of the prefix's token ids is the cache key),
+  * Eq. 1  (k = W^K h, v = W^V h: the prefix KVs a miss computes and stores).
 
 All floating-point work is numpy float64.  A matrix product (numpy matmul) is
 used as a library step; there is no tiling, fusion, online softmax or any
@@ -606,3 +607,30 @@ def prefix_key(tokens):
     """k = h(p): the 64-bit key of a prefix given as a sequence of token ids."""
     raw = b"".join(int(t).to_bytes(4, "little", signed=True) for t in tokens)
     return xxh64(raw, 0)
+
+
+# ---------------------------------------------------------------------------
+# Eq. 1: the key and value vectors of a token are linear projections of its
+# hidden state, k = W^K h, v = W^V h (W^K, W^V of shape [d_k, d] per layer).
+# ---------------------------------------------------------------------------
+
+def project_kv(h, wk, wv, num_kv_heads, head_dim):
+    """Prefix KVs from hidden states, every layer (Eq. 1).
+
+    h [L, m, d]; wk, wv [L, Hkv * D, d] (row o of a weight produces output
+    component o; components are ordered head-major: o = head * D + dim).
+    Returns k, v of shape [L, m, Hkv, D], ready for `PagedPrefixStore.put`.
+    """
+    h = np.asarray(h, dtype=np.float64)
+    wk = np.asarray(wk, dtype=np.float64)
+    wv = np.asarray(wv, dtype=np.float64)
+    L, m, d = h.shape
+    out = num_kv_heads * head_dim
+    if wk.shape != (L, out, d) or wv.shape != (L, out, d):
+        raise InvalidArgument("bad projection weight shape")
+    k = np.empty((L, m, num_kv_heads, head_dim))
+    v = np.empty((L, m, num_kv_heads, head_dim))
+    for l in range(L):
+        k[l] = (h[l] @ wk[l].T).reshape(m, num_kv_heads, head_dim)
+        v[l] = (h[l] @ wv[l].T).reshape(m, num_kv_heads, head_dim)
+    return k, v

@@ -165,3 +165,34 @@ def test_prefix_key_is_xxh64_of_the_token_ids():
         assert oracle.xxh64(data, 12345) == xxhash.xxh64(data, seed=12345).intdigest(), n
     toks = [1, 2, 3, -1, 2 ** 31 - 1]
     assert oracle.prefix_key(toks) == xxhash.xxh64(np.asarray(toks, dtype="<i4").tobytes()).intdigest()
+
+
+def test_project_kv_is_eq1():
+    """k = W^K h, v = W^V h per token and layer: scalar loops, selector weights, linearity."""
+    rng = np.random.default_rng(4)
+    L, m, d, Hkv, D = 2, 5, 7, 2, 3
+    h = rng.standard_normal((L, m, d))
+    wk, wv = rng.standard_normal((L, Hkv * D, d)), rng.standard_normal((L, Hkv * D, d))
+    k, v = oracle.project_kv(h, wk, wv, Hkv, D)
+    assert k.shape == v.shape == (L, m, Hkv, D)
+    for l in range(L):
+        for t in range(m):
+            for hd in range(Hkv):
+                for j in range(D):
+                    o = hd * D + j
+                    assert abs(k[l, t, hd, j] - sum(wk[l, o, c] * h[l, t, c] for c in range(d))) < 1e-12
+                    assert abs(v[l, t, hd, j] - sum(wv[l, o, c] * h[l, t, c] for c in range(d))) < 1e-12
+    # a weight row that is a unit vector copies that hidden component
+    sel = np.zeros((L, Hkv * D, d))
+    for o in range(Hkv * D):
+        sel[:, o, o % d] = 1.0
+    k2, _ = oracle.project_kv(h, sel, sel, Hkv, D)
+    for o in range(Hkv * D):
+        assert np.array_equal(k2[:, :, o // D, o % D], h[:, :, o % d])
+    # linear in the hidden states
+    h2 = rng.standard_normal((L, m, d))
+    ka, va = oracle.project_kv(2.0 * h + h2, wk, wv, Hkv, D)
+    kb, vb = oracle.project_kv(h2, wk, wv, Hkv, D)
+    assert np.allclose(ka, 2.0 * k + kb, atol=1e-12) and np.allclose(va, 2.0 * v + vb, atol=1e-12)
+    with pytest.raises(oracle.InvalidArgument):
+        oracle.project_kv(h, wk[:, :-1], wv, Hkv, D)
