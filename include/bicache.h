@@ -219,6 +219,26 @@ int32_t bicache_reserve_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, int32_
 int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, const void* k,
                                     const void* v, int64_t kv_row_stride, void* stream);
 
+/* Read ONE layer of a stored prefix back as dense rows (the inverse of bicache_update_prefix_layer; the
+ * store's in-page element order is private, this call is how a caller sees the values): k_out, v_out
+ * device, rows [m][Hkv][D] of the context's dtype, `kv_row_stride` elements between rows, 16-byte
+ * aligned.  Copies on `stream`; bit-exact.  NOTFOUND / INVALID as for the update call. */
+int32_t bicache_read_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, void* k_out, void* v_out,
+                                  int64_t kv_row_stride, void* stream);
+
+/* Compute ONE layer's prefix K/V from the layer's input hidden states and write them into the pages
+ * of an existing prefix (Eq. 1: k = W^K h, v = W^V h per token, feeding the store H[k] of Sec. 5.2):
+ *   K[t][o] = sum_c h[t][c] * w_k[o][c],  V likewise,  o = head * D + dim,
+ * bf16 inputs, fp32 accumulation, one rounding to bf16.  h: device, [m][d_model] bf16 with
+ * `h_row_stride` elements between rows; w_k, w_v: device, [Hkv * D][d_model] bf16, rows contiguous.
+ * All 16-byte aligned; d_model and h_row_stride multiples of 8.  The dense K/V never exist in memory:
+ * the kernel (tensor cores) writes page images directly; unused slots of the last page become zero.
+ * Runs on `stream`.  UNSUPPORTED unless the context is bf16 with head_dim 128; NOTFOUND / INVALID as
+ * for the update call; a device-side wait that gives up is reported by bicache_device_status. */
+int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, const void* h,
+                                     int64_t h_row_stride, const void* w_k, const void* w_v, int32_t d_model,
+                                     void* stream);
+
 /* One layer of denoising step t with both kinds of reuse.  Request i owns seqlen[i] = N_i rows from
  * row_off[i] (prefix rows first).  Per request, in this order:
  *   layer < depth[i] and shared_id[i] >= 0      -> suffix rows attend over [shared cached prefix | own

@@ -24,6 +24,7 @@ EXPORTED = [
     "bicache_prefix_pages", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
     "bicache_attend_layer", "bicache_attend_full_static",
     "bicache_is_refresh_step", "bicache_reserve_prefix", "bicache_update_prefix_layer", "bicache_attend_step",
+    "bicache_read_prefix_layer", "bicache_project_prefix_layer",
     "bicache_prefix_similarity", "bicache_prefix_similarity_async", "bicache_depth_from_similarity",
     "bicache_build_depth_table",
     "bicache_hash_tokens", "bicache_device_status", "bicache_set_wait_budget", "bicache_launch_count", "bicache_last_error",
@@ -96,6 +97,10 @@ def load_library():
     lib.bicache_reserve_prefix.argtypes = [vp, C.c_uint64, C.c_int32, i32p, i32p, i32p, C.c_int32]
     lib.bicache_update_prefix_layer.restype = C.c_int32
     lib.bicache_update_prefix_layer.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, C.c_int64, vp]
+    lib.bicache_read_prefix_layer.restype = C.c_int32
+    lib.bicache_read_prefix_layer.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, C.c_int64, vp]
+    lib.bicache_project_prefix_layer.restype = C.c_int32
+    lib.bicache_project_prefix_layer.argtypes = [vp, C.c_int32, C.c_int32, vp, C.c_int64, vp, vp, C.c_int32, vp]
     lib.bicache_attend_step.restype = C.c_int32
     lib.bicache_attend_step.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, i32p, i32p, i32p, i64p, i32p,
                                         vp, vp, vp, C.c_int64, C.c_int64, vp, C.c_int64, vp, C.c_float, vp]
@@ -236,6 +241,23 @@ class BiCache:
         st = self.lib.bicache_update_prefix_layer(self.ctx, prefix_id, layer, k.data_ptr(), v.data_ptr(),
                                                   k.stride(0), self._stream())
         self._check(st, "bicache_update_prefix_layer")
+
+    def read_prefix_layer(self, prefix_id, layer, k_out, v_out):
+        """One layer of a stored prefix as dense rows: k_out, v_out [m, Hkv, D] (rows may be strided)."""
+        assert k_out.is_cuda and v_out.is_cuda and k_out.dtype == self.dtype and k_out.shape == v_out.shape
+        assert k_out.stride()[1:] == (self.D, 1) and v_out.stride() == k_out.stride()
+        st = self.lib.bicache_read_prefix_layer(self.ctx, prefix_id, layer, k_out.data_ptr(), v_out.data_ptr(),
+                                                k_out.stride(0), self._stream())
+        self._check(st, "bicache_read_prefix_layer")
+
+    def project_prefix_layer(self, prefix_id, layer, h, w_k, w_v):
+        """Eq. 1 into the store: h [m, d_model] (rows may be strided), w_k, w_v [Hkv * D, d_model]."""
+        assert h.is_cuda and w_k.is_cuda and w_v.is_cuda and h.dtype == w_k.dtype == w_v.dtype == self.dtype
+        assert h.dim() == 2 and h.stride(1) == 1 and w_k.is_contiguous() and w_v.is_contiguous()
+        assert w_k.shape == w_v.shape == (self.Hkv * self.D, h.shape[1])
+        st = self.lib.bicache_project_prefix_layer(self.ctx, prefix_id, layer, h.data_ptr(), h.stride(0),
+                                                   w_k.data_ptr(), w_v.data_ptr(), h.shape[1], self._stream())
+        self._check(st, "bicache_project_prefix_layer")
 
     def prefix_similarity(self, prefix_id, k_ref, v_ref):
         """Eq. 3 per layer: cosine between the cached K/V of a prefix and k_ref, v_ref [L, m, Hkv, D]."""

@@ -21,6 +21,7 @@
 #include "common.cuh"
 #include "simt_kernels.cuh"
 #include "tc_attention.cuh"
+#include "project_kv.cuh"
 
 using namespace bicache;
 
@@ -494,6 +495,7 @@ int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
   }
   if (tensor_ok) {
     cudaError_t e = configure_tc_attention();
+    if (e == cudaSuccess) e = configure_project_kv();
     if (e != cudaSuccess) {
       delete ctx;
       return BICACHE_ERR_CUDA;
@@ -655,6 +657,102 @@ int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t
     ce = cudaGetLastError();
   }
   if (ce != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("update_prefix_layer: ") + cudaGetErrorString(ce));
+  return BICACHE_OK;
+}
+
+int32_t bicache_read_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, void* k_out, void* v_out,
+                                  int64_t kv_row_stride, void* stream_) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  const bicache_config& cfg = ctx->cfg;
+  auto found = ctx->by_id.find(prefix_id);
+  if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+  if (layer < 0 || layer >= cfg.num_layers) return fail(ctx, BICACHE_ERR_INVALID, "layer out of range");
+  const PrefixEntry& e = *found->second;
+  const int64_t row_elems = (int64_t)cfg.num_kv_heads * cfg.head_dim;
+  if (kv_row_stride < row_elems || (kv_row_stride * ctx->esize) % 16)
+    return fail(ctx, BICACHE_ERR_INVALID, "bad row stride");
+  if (ctx->host_only) return fail(ctx, BICACHE_ERR_UNSUPPORTED, "host-only context");
+  if (!k_out || !v_out || !aligned16(k_out) || !aligned16(v_out))
+    return fail(ctx, BICACHE_ERR_INVALID, "bad k/v pointer");
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int need = (int)e.pages.size();
+  cudaError_t ce =
+      cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+  if (ce == cudaSuccess && e.m > 0) {
+    const int chunks_per_row = cfg.head_dim * ctx->esize / 16;
+    const long long total = (long long)e.m * cfg.num_kv_heads * chunks_per_row;
+    const int threads = 256;
+    const int blocks = (int)std::min<long long>((total + threads - 1) / threads, (long long)ctx->sm_count * 16);
+    const PoolView pv = pool_view(ctx);
+    gather_prefix_kernel<<<blocks, threads, 0, stream>>>(
+        pv.k + (long long)layer * pv.layer_bytes, pv.v + (long long)layer * pv.layer_bytes,
+        static_cast<char*>(k_out), static_cast<char*>(v_out), ctx->d_put_pages, e.m, cfg.num_kv_heads,
+        chunks_per_row, kv_row_stride * ctx->esize, pv.page_bytes, pv.swizzled);
+    ctx->launches++;
+    ce = cudaGetLastError();
+  }
+  if (ce != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("read_prefix_layer: ") + cudaGetErrorString(ce));
+  return BICACHE_OK;
+}
+
+// bf16 matrix [rows][cols] with `row_stride` elements between rows; box = (64 columns, box_rows),
+// 128-byte swizzle, zero fill outside.
+static bool encode_map_2d(CUtensorMap* m, const void* base, long long rows, long long cols, long long row_stride,
+                          int box_rows) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_stride * 2};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, const void* h,
+                                     int64_t h_row_stride, const void* w_k, const void* w_v, int32_t d_model,
+                                     void* stream_) {
+  if (!ctx) return BICACHE_ERR_INVALID;
+  const bicache_config& cfg = ctx->cfg;
+  if (!ctx->tensor_ok && !(ctx->host_only && cfg.dtype == BICACHE_BF16 && cfg.head_dim == 128))
+    return fail(ctx, BICACHE_ERR_UNSUPPORTED, "projection needs a bf16 context with head_dim 128");
+  auto found = ctx->by_id.find(prefix_id);
+  if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+  if (layer < 0 || layer >= cfg.num_layers) return fail(ctx, BICACHE_ERR_INVALID, "layer out of range");
+  if (d_model <= 0 || d_model % 8 || h_row_stride < d_model || h_row_stride % 8)
+    return fail(ctx, BICACHE_ERR_INVALID, "d_model and the row stride must be positive multiples of 8");
+  const PrefixEntry& e = *found->second;
+  if (ctx->host_only) return BICACHE_OK;
+  if (!h || !w_k || !w_v || !aligned16(h) || !aligned16(w_k) || !aligned16(w_v))
+    return fail(ctx, BICACHE_ERR_INVALID, "bad h/w pointer");
+  if (e.m == 0) return BICACHE_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int need = (int)e.pages.size();
+  CUtensorMap tm_h, tm_wk, tm_wv;
+  const long long out_rows = (long long)cfg.num_kv_heads * cfg.head_dim;
+  if (!encode_map_2d(&tm_h, h, e.m, d_model, h_row_stride, proj::kBM) ||
+      !encode_map_2d(&tm_wk, w_k, out_rows, d_model, d_model, proj::kBN) ||
+      !encode_map_2d(&tm_wv, w_v, out_rows, d_model, d_model, proj::kBN))
+    return fail(ctx, BICACHE_ERR_CUDA, "project_prefix_layer: tensor map encoding failed");
+  cudaError_t ce =
+      cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+  if (ce == cudaSuccess) {
+    const PoolView pv = pool_view(ctx);
+    proj::ProjArgs a;
+    a.pool_k = static_cast<char*>(cfg.k_pool) + (long long)layer * pv.layer_bytes;
+    a.pool_v = static_cast<char*>(cfg.v_pool) + (long long)layer * pv.layer_bytes;
+    a.pages = ctx->d_put_pages;
+    a.m = e.m;
+    a.d_model = d_model;
+    a.num_kv_heads = cfg.num_kv_heads;
+    a.m_tiles = (e.m + proj::kBM - 1) / proj::kBM;
+    a.n_tiles = (cfg.num_kv_heads + 1) / 2;
+    ce = launch_project_kv(a, ctx->d_status, ctx->sm_count, tm_h, tm_wk, tm_wv, ctx->wait_cycles, stream);
+    ctx->launches++;
+  }
+  if (ce != cudaSuccess)
+    return fail(ctx, BICACHE_ERR_CUDA, std::string("project_prefix_layer: ") + cudaGetErrorString(ce));
   return BICACHE_OK;
 }
 

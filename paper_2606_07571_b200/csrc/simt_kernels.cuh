@@ -92,6 +92,30 @@ __global__ void scatter_prefix_kernel(const char* __restrict__ src_k, const char
 }
 
 // ---------------------------------------------------------------------------------------------
+// The inverse for one layer: pool pages -> dense rows [m][Hkv][D] (K and V).  One thread moves one
+// 16-byte chunk of each.
+// ---------------------------------------------------------------------------------------------
+__global__ void gather_prefix_kernel(const char* __restrict__ pool_k, const char* __restrict__ pool_v,
+                                     char* __restrict__ dst_k, char* __restrict__ dst_v,
+                                     const int* __restrict__ pages, int m, int num_kv_heads, int chunks_per_row,
+                                     long long dst_row_stride_bytes, int page_bytes, int swizzled) {
+  const long long total = (long long)m * num_kv_heads * chunks_per_row;
+  const int row_bytes = chunks_per_row * 16;
+  for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+       idx += (long long)gridDim.x * blockDim.x) {
+    long long rem = idx;
+    const int c16 = (int)(rem % chunks_per_row); rem /= chunks_per_row;
+    const int hk = (int)(rem % num_kv_heads); rem /= num_kv_heads;
+    const int t = (int)rem;
+    const long long po = ((long long)pages[t / kPageSize] * num_kv_heads + hk) * page_bytes +
+                         page_chunk_offset(swizzled != 0, t % kPageSize, c16, row_bytes);
+    const long long d = (long long)t * dst_row_stride_bytes + (long long)hk * row_bytes + c16 * 16;
+    *reinterpret_cast<uint4*>(dst_k + d) = *reinterpret_cast<const uint4*>(pool_k + po);
+    *reinterpret_cast<uint4*>(dst_v + d) = *reinterpret_cast<const uint4*>(pool_v + po);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Profiler reduction (Eq. 3): for every layer the three sums behind
 //   sim_l = cos(KV$_l, KVref_l) = <a, b> / (|a| |b|),
 // a = the cached prefix's K and V of layer l read through the page table, b = the reference K and V

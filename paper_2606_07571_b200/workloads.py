@@ -128,6 +128,19 @@ def draw_prefix_kv(w: Workload, g: int, device="cpu", layers=None):
     return torch.stack(ks), torch.stack(vs)
 
 
+def draw_hidden_and_weights(m, d_model, num_kv_heads, head_dim, seed, dtype=torch.bfloat16, device="cpu"):
+    """Inputs of the K/V projection of one layer: hidden states h [m, d_model] ~ N(0, 1) (the scale
+    of a normalised residual stream) and weights w_k, w_v [Hkv * D, d_model] ~ N(0, 1 / d_model), so
+    that the projected K/V have unit variance like the drawn ones."""
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed * 1000003 + 15485863)
+    h = _normal((m, d_model), gen, dtype, device, 1.0)
+    out = num_kv_heads * head_dim
+    w_k = _normal((out, d_model), gen, dtype, device, d_model ** -0.5)
+    w_v = _normal((out, d_model), gen, dtype, device, d_model ** -0.5)
+    return h, w_k, w_v
+
+
 def prefix_key(w: Workload, g: int) -> int:
     """A 64-bit identifier standing in for the hash of the prefix's token ids."""
     return (0x9E3779B97F4A7C15 * (g + 1) + w.seed) & 0xFFFFFFFFFFFFFFFF
