@@ -59,6 +59,7 @@ struct bicache_ctx {
   int esize = 2;
   bool swizzled = false;
   bool tensor_ok = false;
+  int proj_pairs = 0;                                             // CTA pairs of the projection kernel the device runs at once
   bool host_only = false;                                         // cfg.device < 0: bookkeeping only
   int path = BICACHE_PATH_AUTO;
   std::deque<int32_t> free_pages;
@@ -495,7 +496,7 @@ int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
   }
   if (tensor_ok) {
     cudaError_t e = configure_tc_attention();
-    if (e == cudaSuccess) e = configure_project_kv();
+    if (e == cudaSuccess) e = configure_project_kv(&ctx->proj_pairs);
     if (e != cudaSuccess) {
       delete ctx;
       return BICACHE_ERR_CUDA;
@@ -732,8 +733,8 @@ int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_
   CUtensorMap tm_h, tm_wk, tm_wv;
   const long long out_rows = (long long)cfg.num_kv_heads * cfg.head_dim;
   if (!encode_map_2d(&tm_h, h, e.m, d_model, h_row_stride, proj::kBM) ||
-      !encode_map_2d(&tm_wk, w_k, out_rows, d_model, d_model, proj::kBN) ||
-      !encode_map_2d(&tm_wv, w_v, out_rows, d_model, d_model, proj::kBN))
+      !encode_map_2d(&tm_wk, w_k, out_rows, d_model, d_model, proj::kBN / 2) ||
+      !encode_map_2d(&tm_wv, w_v, out_rows, d_model, d_model, proj::kBN / 2))
     return fail(ctx, BICACHE_ERR_CUDA, "project_prefix_layer: tensor map encoding failed");
   cudaError_t ce =
       cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
@@ -746,9 +747,9 @@ int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_
     a.m = e.m;
     a.d_model = d_model;
     a.num_kv_heads = cfg.num_kv_heads;
-    a.m_tiles = (e.m + proj::kBM - 1) / proj::kBM;
+    a.m_tiles = (e.m + 2 * proj::kBM - 1) / (2 * proj::kBM);
     a.n_tiles = (cfg.num_kv_heads + 1) / 2;
-    ce = launch_project_kv(a, ctx->d_status, ctx->sm_count, tm_h, tm_wk, tm_wv, ctx->wait_cycles, stream);
+    ce = launch_project_kv(a, ctx->d_status, ctx->proj_pairs, tm_h, tm_wk, tm_wv, ctx->wait_cycles, stream);
     ctx->launches++;
   }
   if (ce != cudaSuccess)

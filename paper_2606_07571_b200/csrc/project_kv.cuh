@@ -4,19 +4,28 @@
 // tensor: every (page, kv head) slice of the pool is produced as the 4 KB operand image the
 // attention kernel reads and leaves shared memory as one bulk copy.
 //
-// A persistent tcgen05 GEMM.  One output tile is 128 tokens x 256 output features (two KV heads
-// of K, or two of V); the contraction runs over d in blocks of 64 (one 128-byte swizzled row per
-// token / feature and block).  Warp 0 feeds a four-stage ring of (H tile 16 KB, W tile 32 KB) by
-// TMA, warp 1 issues the MMAs (M = 128, N = 256, K = 16) into one of two 256-column TMEM
-// accumulators, warps 2-5 drain the other accumulator: TMEM -> registers -> bf16 -> page images
-// in shared memory -> eight 4 KB bulk copies per head.  Tiles are handed out statically
-// (tile = block + i * grid) with all tiles of a token block adjacent, so that the H tile is
-// shared through L2 by the CTAs working on it.
+// A persistent tcgen05 GEMM on CTA pairs (clusters of two, the two-SM MMA).  One output tile of
+// a pair is 256 tokens x 256 output features (two KV heads of K, or two of V): CTA r of the pair
+// owns tokens 128 r .. 128 r + 127 of the tile (its rows of A and of the accumulator, in its own
+// TMEM) and stages rows 128 r .. 128 r + 127 of the W tile (its half of B), so every SM stages
+// and reads half of the B operand a one-CTA tile would.  The contraction runs over d in blocks of
+// 64 (one 128-byte swizzled row per token / feature and block).  Per CTA: warp 0 feeds a
+// six-stage ring of (H tile 16 KB, W half tile 16 KB) by TMA, the loads of both CTAs completing
+// on one barrier in CTA 0; warp 1 of CTA 0 issues the MMAs (cta_group::2, M = 256, N = 256,
+// K = 16) into one of two 256-column TMEM accumulators; warps 2-5 drain the other accumulator:
+// TMEM -> registers -> bf16 -> page images in shared memory -> eight 4 KB bulk copies per head.
+// One tcgen05.commit with a CTA mask releases a stage, or hands over an accumulator, in both
+// CTAs; the epilogue warps of CTA 1 release the accumulator on CTA 0's barrier through the
+// cluster's shared address space.  Tiles are handed out statically (tile = pair + i * pairs) with
+// all tiles of a token block adjacent, so that the H tile is shared through L2.
 //
-// Every wait is bounded (SM clock); a wait that gives up raises the CTA's abort flag, the roles
-// leave their loops, loads and MMAs in flight are waited for, TMEM is released and the context's
-// sticky status word is set.
+// Every wait is bounded (SM clock) and on a barrier of the waiting CTA; a wait that gives up
+// raises the CTA's abort flag, the roles leave their loops (the partner's waits then run out
+// too), loads and MMAs in flight are waited for, the pair meets at a cluster barrier, TMEM is
+// released and the context's sticky status word is set.
 #pragma once
+
+#include <cooperative_groups.h>
 
 #include "tc_attention.cuh"
 
@@ -25,24 +34,24 @@ namespace proj {
 
 using namespace tc;
 
-constexpr int kBM = 128;                       // tokens per tile
+constexpr int kBM = 128;                       // tokens per tile and CTA (256 per pair)
 constexpr int kBN = 256;                       // output features per tile (two heads of 128 dims)
 constexpr int kBK = 64;                        // contraction block: 64 bf16 = one 128-byte row
-constexpr int kStages = 4;
-constexpr int kABytes = kBM * kBK * 2;         // 16 KB
-constexpr int kBBytes = kBN * kBK * 2;         // 32 KB
+constexpr int kStages = 6;
+constexpr int kABytes = kBM * kBK * 2;         // 16 KB: this CTA's tokens
+constexpr int kBBytes = (kBN / 2) * kBK * 2;   // 16 KB: this CTA's half of the W tile
 constexpr int kProjStageBytes = kABytes + kBBytes;
 constexpr int kOutBytes = 8 * kPageBytes;      // 128 tokens of one head = eight page images
 constexpr int kProjThreads = 192;
 constexpr int kEpiWarps = 4;
-// fp32 accumulate, bf16 A and B (both K-major), M = 128, N = 256
-constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+// fp32 accumulate, bf16 A and B (both K-major), M = 256 (over the pair), N = 256
+constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
 
 struct Sync {
-  unsigned long long full[kStages];      // stage holds its two tiles
-  unsigned long long empty[kStages];     // the MMAs reading the stage have completed
+  unsigned long long full[kStages];      // CTA 0 only: the stage holds its tiles in BOTH CTAs
+  unsigned long long empty[kStages];     // the MMAs reading the stage (in both CTAs) have completed
   unsigned long long acc_full[2];        // the accumulator holds a finished tile
-  unsigned long long acc_empty[2];       // the epilogue has read the accumulator
+  unsigned long long acc_empty[2];       // CTA 0 only: the epilogues of both CTAs have read the accumulator
   unsigned long long epi;                // barrier of the four epilogue warps
   unsigned long long drain;
   long long wait_cycles;                 // budget of every wait; directly before abort_flag (mbar_wait reads it)
@@ -60,7 +69,7 @@ struct ProjArgs {
   int m;                     // prefix tokens
   int d_model;
   int num_kv_heads;
-  int m_tiles;               // ceil(m / 128)
+  int m_tiles;               // ceil(m / 256): token blocks of a CTA pair
   int n_tiles;               // per matrix: ceil(Hkv / 2)
 };
 
@@ -70,9 +79,67 @@ __device__ __forceinline__ void tma_load_2d(unsigned dst, const void* tmap, int 
       ::"r"(dst), "l"(reinterpret_cast<unsigned long long>(tmap)), "r"(c0), "r"(c1), "r"(bar)
       : "memory");
 }
+// The same load issued by either CTA of a pair, completing on the barrier at `bar`'s offset in the
+// pair's FIRST CTA (bit 24 of a shared-window address is the CTA's rank in the pair): one barrier
+// there collects the bytes of both CTAs' stages.  No multicast: each CTA's data goes to its own
+// shared memory.
+__device__ __forceinline__ void tma_load_2d_pair(unsigned dst, const void* tmap, int c0, int c1, unsigned bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<unsigned long long>(tmap)), "r"(c0), "r"(c1), "r"(bar & 0xFEFFFFFFu)
+      : "memory");
+}
 __device__ __forceinline__ void bulk_copy_s2g(void* dst, unsigned src, unsigned bytes) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes)
                : "memory");
+}
+
+// arrive on the barrier at the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ void mbar_arrive_remote(unsigned local_bar, unsigned rank) {
+  unsigned raddr;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(local_bar), "r"(rank));
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(raddr) : "memory");
+}
+// The two-SM MMA, issued by one elected lane of a converged warp of the pair's first CTA.  The
+// descriptors name the same shared-memory offsets in both CTAs: CTA r supplies rows 128 r .. of A
+// and rows N/2 r .. of B and receives rows 128 r .. of D in its own TMEM.
+__device__ __forceinline__ void mma2_ss_elect(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                              unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred P, Q;\n\t"
+      "elect.sync _|P, 0xffffffff;\n\t"
+      "setp.ne.b32 Q, %4, 0;\n\t"
+      "@P tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, Q;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+// commit of the two-SM MMAs issued so far by this thread: arrives on the barrier at this offset in
+// both CTAs of the pair
+__device__ __forceinline__ void mma2_commit_both_elect(unsigned bar) {
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "elect.sync _|P, 0xffffffff;\n\t"
+      "@P tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
+      ::"r"(bar), "h"((unsigned short)3)
+      : "memory");
+}
+// the same, arriving in this CTA only
+__device__ __forceinline__ void mma2_commit_local_elect(unsigned bar) {
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "elect.sync _|P, 0xffffffff;\n\t"
+      "@P tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+      ::"r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(unsigned smem_slot, unsigned cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(unsigned taddr, unsigned cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
 
 struct TileCoord {
@@ -89,12 +156,14 @@ __device__ __forceinline__ TileCoord tile_coord(int tile, int n_tiles) {
 
 }  // namespace proj
 
-__global__ void __launch_bounds__(proj::kProjThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(proj::kProjThreads, 1)
 project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtensorMap tm_h,
                   const __grid_constant__ CUtensorMap tm_wk, const __grid_constant__ CUtensorMap tm_wv,
                   long long wait_cycles) {
   using namespace proj;
+  namespace cg = cooperative_groups;
   extern __shared__ unsigned char smem_raw[];
+  // the same offsets in both CTAs of the pair: the MMA descriptors name them once for both
   unsigned char* smem =
       reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* const out_stage = smem + kStages * kProjStageBytes;
@@ -102,6 +171,9 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
   volatile int* abort_flag = &sy->abort_flag;
   const unsigned ring = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned rank = cluster.block_rank();              // 0: issues the pair's MMAs
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
 
   if (tid == 0) {
     sy->wait_cycles = wait_cycles;
@@ -113,18 +185,18 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&sy->acc_full[i]), 1);
-      mbar_init(smem_u32(&sy->acc_empty[i]), kEpiWarps);
+      mbar_init(smem_u32(&sy->acc_empty[i]), 2 * kEpiWarps);
     }
     mbar_init(smem_u32(&sy->epi), kEpiWarps);
     mbar_init(smem_u32(&sy->drain), 1);
     fence_barrier_init();
   }
-  if (warp == 1) {
-    tmem_alloc(smem_u32(&sy->tmem_base), 512);
-    tmem_relinquish();
+  if (warp == 1) {                                          // the same warp in both CTAs
+    tmem_alloc2(smem_u32(&sy->tmem_base), 512);
+    tmem_relinquish2();
   }
   tc_fence_before();
-  __syncthreads();
+  cluster.sync();                                           // barriers of both CTAs exist before any remote arrival
   tc_fence_after();
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&sy->tmem_base);
   const bool dead = *reinterpret_cast<volatile int*>(&sy->dead) != 0;
@@ -133,10 +205,13 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
 
   if (warp == 0) {
     // ===================================== TMA producer =====================================
+    // this CTA's 128 tokens of the H tile and its 128 rows of the W tile
     bool ok = !dead;
     int it = 0;                              // stage uses over the life of the CTA
-    int armed[kStages] = {-1, -1, -1, -1};
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
+    int armed[kStages];
+#pragma unroll
+    for (int i = 0; i < kStages; ++i) armed[i] = -1;
+    for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
       const TileCoord c = tile_coord(tile, a.n_tiles);
       const void* tm_w = c.which ? (const void*)&tm_wv : (const void*)&tm_wk;
       for (int kb = 0; kb < KB; ++kb, ++it) {
@@ -146,26 +221,36 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
         if (lane == 0) {
           const unsigned full = smem_u32(&sy->full[s]);
           const unsigned dst = ring + s * kProjStageBytes;
-          mbar_arrive_expect_tx(full, (unsigned)kProjStageBytes);
-          tma_load_2d(dst, &tm_h, kb * kBK, c.mt * kBM, full);
-          tma_load_2d(dst + kABytes, tm_w, kb * kBK, c.nt * kBN, full);
+          if (rank == 0) mbar_arrive_expect_tx(full, 2u * kProjStageBytes);   // the bytes of both CTAs
+          tma_load_2d_pair(dst, &tm_h, kb * kBK, (c.mt * 2 + (int)rank) * kBM, full);
+          tma_load_2d_pair(dst + kABytes, tm_w, kb * kBK, c.nt * kBN + (int)rank * (kBN / 2), full);
           armed[s] = it;
         }
       }
     }
-    // After a give-up, loads may still be in flight: wait (bounded) for the barriers armed last.
+    // After a give-up, loads may still be in flight.  CTA 0 waits (bounded) for the barriers it
+    // armed last, which count the bytes of both CTAs.  CTA 1 cannot see those barriers: if it has
+    // issued loads it waits out the same limit before it joins the pair's last barrier.
     if (!dead && (!ok || *abort_flag) && lane == 0) {
       for (int s = 0; s < kStages; ++s)
-        if (armed[s] >= 0)
-          for (unsigned n = 0; n < 4096 && !mbar_try_wait(smem_u32(&sy->full[s]), (armed[s] / kStages) & 1); ++n)
-            __nanosleep(256);
+        if (armed[s] >= 0) {
+          if (rank == 0) {
+            for (unsigned n = 0; n < 4096 && !mbar_try_wait(smem_u32(&sy->full[s]), (armed[s] / kStages) & 1); ++n)
+              __nanosleep(256);
+          } else {
+            for (unsigned n = 0; n < 4096; ++n) __nanosleep(256);
+            break;
+          }
+        }
     }
+  } else if (warp == 1 && rank == 1) {
+    // CTA 1's warp 1 only owns the pair's TMEM allocation with its counterpart
   } else if (warp == 1) {
-    // ====================================== MMA issue ======================================
+    // ================================== CTA 0: MMA issue ===================================
     bool ok = !dead;
     if (ok) {
       int it = 0, tl = 0;
-      for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tl) {
+      for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tl) {
         const int buf = tl & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->acc_empty[buf]), ((tl >> 1) & 1) ^ 1, abort_flag));
         if (!ok) break;
@@ -173,7 +258,8 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
         const unsigned d_tmem = tmem + buf * kBN;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % kStages;
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->full[s]), (it / kStages) & 1, abort_flag));
+          const unsigned ph = (it / kStages) & 1;
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->full[s]), ph, abort_flag));
           if (!ok) break;
           tc_fence_after();
           // both operands K-major, rows of 128 bytes, 8-row groups 1024 bytes apart; a K step of
@@ -182,25 +268,25 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
           const unsigned long long b_desc = make_desc(ring + s * kProjStageBytes + kABytes, 16, 1024);
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k)
-            mma_ss_elect(d_tmem, a_desc + 2 * k, b_desc + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
-          mma_commit_elect(smem_u32(&sy->empty[s]));
+            mma2_ss_elect(d_tmem, a_desc + 2 * k, b_desc + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
+          mma2_commit_both_elect(smem_u32(&sy->empty[s]));
         }
         if (!ok) break;
-        mma_commit_elect(smem_u32(&sy->acc_full[buf]));
+        mma2_commit_both_elect(smem_u32(&sy->acc_full[buf]));
       }
-      // Whatever happened, let every MMA issued so far finish before TMEM is released.
+      // Whatever happened, let every MMA issued so far finish before the pair's TMEM is released.
       __syncwarp();
-      mma_commit_elect(smem_u32(&sy->drain));
+      mma2_commit_local_elect(smem_u32(&sy->drain));
       mbar_wait_issued(smem_u32(&sy->drain), 0);
     }
     __syncwarp();
   } else {
     // ====================================== epilogue =======================================
-    // Warp w reads TMEM lanes 32 (w & 3) .. + 31: thread = one token of the tile.  Per head:
-    // 128 fp32 -> bf16, written as 16-byte chunks into the token's slot of its page image
-    // (page = token / 16); when all four warps are done, eight threads copy one page each.
+    // Warp w reads TMEM lanes 32 (w & 3) .. + 31: thread = one token of this CTA's half of the
+    // tile.  Per head: 128 fp32 -> bf16, written as 16-byte chunks into the token's slot of its
+    // page image (page = token / 16); when all four warps are done, eight threads copy one page each.
     const int q = warp & 3;
-    const int e = q * 32 + lane;                             // token within the tile
+    const int e = q * 32 + lane;                             // token within this CTA's 128
     const unsigned lane_base = (unsigned)(q * 32) << 16;
     unsigned char* const my_row = out_stage + (e >> 4) * kPageBytes;
     const int slot = e & 15;
@@ -214,9 +300,10 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
       return done;
     };
     int tl = 0;
-    for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++tl) {
+    for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tl) {
       const TileCoord c = tile_coord(tile, a.n_tiles);
       const int buf = tl & 1;
+      const int tok_base = (c.mt * 2 + (int)rank) * kBM;     // first token of this CTA's half
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->acc_full[buf]), (tl >> 1) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
@@ -248,15 +335,18 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
           // the accumulator has been read: the MMAs of the tile after next may overwrite it
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&sy->acc_empty[buf]));
+          if (lane == 0) {
+            if (rank == 0) mbar_arrive(smem_u32(&sy->acc_empty[buf]));
+            else mbar_arrive_remote(smem_u32(&sy->acc_empty[buf]), 0);
+          }
         }
         fence_proxy_async();                                 // the bulk copies read what the threads wrote
         ok = epi_sync();
         if (!ok) break;
         if (e < 8) {
-          const int tok0 = c.mt * kBM + e * kPageSize;
+          const int tok0 = tok_base + e * kPageSize;
           if (head_valid && tok0 < a.m) {
-            const int page = a.pages[c.mt * 8 + e];
+            const int page = a.pages[tok0 / kPageSize];
             char* dst = (c.which ? a.pool_v : a.pool_k) + ((long long)page * a.num_kv_heads + head) * kPageBytes;
             bulk_copy_s2g(dst, smem_u32(out_stage + e * kPageBytes), kPageBytes);
           }
@@ -265,28 +355,39 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
       }
     }
     if (e < 8) bulk_wait_all();                              // this thread's page copies have completed
-    tc_fence_before();
   }
 
-  __syncthreads();
-  if (warp == 1) {
-    tc_fence_after();
-    tmem_dealloc(tmem, 512);
-  }
+  // The pair leaves together: CTA 0's MMAs read CTA 1's shared memory and write its TMEM.
+  tc_fence_before();
+  cluster.sync();
+  tc_fence_after();
+  if (warp == 1) tmem_dealloc2(tmem, 512);
   if (tid == 0 && !dead && *abort_flag) atomicCAS(status, kDevOk, kDevTimeout);
 }
 
-inline cudaError_t configure_project_kv() {
-  return cudaFuncSetAttribute(project_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, proj::kProjSmemBytes);
+// Sets the kernel's shared-memory limit and returns how many CTA pairs the device runs at once.
+inline cudaError_t configure_project_kv(int* max_pairs) {
+  cudaError_t e =
+      cudaFuncSetAttribute(project_kv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, proj::kProjSmemBytes);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(2, 1, 1);
+  cfg.blockDim = dim3(proj::kProjThreads, 1, 1);
+  cfg.dynamicSmemBytes = proj::kProjSmemBytes;
+  int n = 0;
+  e = cudaOccupancyMaxActiveClusters(&n, project_kv_kernel, &cfg);
+  if (e != cudaSuccess) return e;
+  *max_pairs = n;
+  return n > 0 ? cudaSuccess : cudaErrorLaunchOutOfResources;
 }
 
-inline cudaError_t launch_project_kv(const proj::ProjArgs& a, int* status, int num_sms, const CUtensorMap& tm_h,
+inline cudaError_t launch_project_kv(const proj::ProjArgs& a, int* status, int max_pairs, const CUtensorMap& tm_h,
                                      const CUtensorMap& tm_wk, const CUtensorMap& tm_wv, long long wait_cycles,
                                      cudaStream_t stream) {
   const int total = a.m_tiles * 2 * a.n_tiles;
   if (total <= 0) return cudaSuccess;
-  const int grid = total < num_sms ? total : num_sms;
-  project_kv_kernel<<<grid, proj::kProjThreads, proj::kProjSmemBytes, stream>>>(
+  const int pairs = total < max_pairs ? total : max_pairs;
+  project_kv_kernel<<<2 * pairs, proj::kProjThreads, proj::kProjSmemBytes, stream>>>(
       a, status, tm_h, tm_wk, tm_wv, wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
   return cudaGetLastError();
 }
