@@ -733,8 +733,8 @@ int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_
   CUtensorMap tm_h, tm_wk, tm_wv;
   const long long out_rows = (long long)cfg.num_kv_heads * cfg.head_dim;
   if (!encode_map_2d(&tm_h, h, e.m, d_model, h_row_stride, proj::kBM) ||
-      !encode_map_2d(&tm_wk, w_k, out_rows, d_model, d_model, proj::kBN / 2) ||
-      !encode_map_2d(&tm_wv, w_v, out_rows, d_model, d_model, proj::kBN / 2))
+      !encode_map_2d(&tm_wk, w_k, out_rows, d_model, d_model, 64) ||
+      !encode_map_2d(&tm_wv, w_v, out_rows, d_model, d_model, 64))
     return fail(ctx, BICACHE_ERR_CUDA, "project_prefix_layer: tensor map encoding failed");
   cudaError_t ce =
       cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
@@ -749,6 +749,7 @@ int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_
     a.num_kv_heads = cfg.num_kv_heads;
     a.m_tiles = (e.m + 2 * proj::kBM - 1) / (2 * proj::kBM);
     a.n_tiles = (cfg.num_kv_heads + 1) / 2;
+    a.full_tiles = 0;                                   // set by the launcher
     ce = launch_project_kv(a, ctx->d_status, ctx->proj_pairs, tm_h, tm_wk, tm_wv, ctx->wait_cycles, stream);
     ctx->launches++;
   }

@@ -46,6 +46,8 @@ constexpr int kProjThreads = 192;
 constexpr int kEpiWarps = 4;
 // fp32 accumulate, bf16 A and B (both K-major), M = 256 (over the pair), N = 256
 constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((256u >> 4) << 24);
+// the same with N = 128: one head (the tiles of the last, partial round are split in two)
+constexpr unsigned kIdescHalf = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((256u >> 4) << 24);
 
 struct Sync {
   unsigned long long full[kStages];      // CTA 0 only: the stage holds its tiles in BOTH CTAs
@@ -71,6 +73,9 @@ struct ProjArgs {
   int num_kv_heads;
   int m_tiles;               // ceil(m / 256): token blocks of a CTA pair
   int n_tiles;               // per matrix: ceil(Hkv / 2)
+  int full_tiles;            // tiles 0 .. full_tiles - 1 are worked on whole (whole rounds of the grid);
+                             // each tile after them is split into its two heads, so that the last
+                             // round takes half the time
 };
 
 __device__ __forceinline__ void tma_load_2d(unsigned dst, const void* tmap, int c0, int c1, unsigned bar) {
@@ -144,13 +149,25 @@ __device__ __forceinline__ void tmem_dealloc2(unsigned taddr, unsigned cols) {
 
 struct TileCoord {
   int mt, nt, which;         // token block, feature block of the matrix, 0: K, 1: V
+  int half;                  // -1: both heads of the feature block; 0 / 1: that head only
+  int valid;
 };
-__device__ __forceinline__ TileCoord tile_coord(int tile, int n_tiles) {
+// work unit `idx` of the launch (a pair takes idx = pair, pair + pairs, ...)
+__device__ __forceinline__ TileCoord tile_coord(int idx, const ProjArgs& a) {
   TileCoord c;
-  c.mt = tile / (2 * n_tiles);
-  const int rem = tile - c.mt * 2 * n_tiles;
-  c.which = rem / n_tiles;
-  c.nt = rem - c.which * n_tiles;
+  const int total = a.m_tiles * 2 * a.n_tiles;
+  int tile = idx;
+  c.half = -1;
+  if (idx >= a.full_tiles) {
+    const int j = idx - a.full_tiles;
+    tile = a.full_tiles + (j >> 1);
+    c.half = j & 1;
+  }
+  c.valid = tile < total;
+  c.mt = tile / (2 * a.n_tiles);
+  const int rem = tile - c.mt * 2 * a.n_tiles;
+  c.which = rem / a.n_tiles;
+  c.nt = rem - c.which * a.n_tiles;
   return c;
 }
 
@@ -200,7 +217,6 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
   tc_fence_after();
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&sy->tmem_base);
   const bool dead = *reinterpret_cast<volatile int*>(&sy->dead) != 0;
-  const int total_tiles = a.m_tiles * 2 * a.n_tiles;
   const int KB = (a.d_model + kBK - 1) / kBK;
 
   if (warp == 0) {
@@ -211,9 +227,13 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
     int armed[kStages];
 #pragma unroll
     for (int i = 0; i < kStages; ++i) armed[i] = -1;
-    for (int tile = pair; tile < total_tiles && ok; tile += num_pairs) {
-      const TileCoord c = tile_coord(tile, a.n_tiles);
+    for (int idx = pair; ok; idx += num_pairs) {
+      const TileCoord c = tile_coord(idx, a);
+      if (!c.valid) break;
       const void* tm_w = c.which ? (const void*)&tm_wv : (const void*)&tm_wk;
+      // rows of W this CTA stages: its half of the tile's features (64-row boxes)
+      const int w_row = c.nt * kBN + (c.half < 0 ? (int)rank * 128 : c.half * 128 + (int)rank * 64);
+      const unsigned stage_tx = c.half < 0 ? 2u * kProjStageBytes : 2u * (kABytes + kBBytes / 2);
       for (int kb = 0; kb < KB; ++kb, ++it) {
         const int s = it % kStages;
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->empty[s]), ((it / kStages) & 1) ^ 1, abort_flag));
@@ -221,9 +241,10 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
         if (lane == 0) {
           const unsigned full = smem_u32(&sy->full[s]);
           const unsigned dst = ring + s * kProjStageBytes;
-          if (rank == 0) mbar_arrive_expect_tx(full, 2u * kProjStageBytes);   // the bytes of both CTAs
+          if (rank == 0) mbar_arrive_expect_tx(full, stage_tx);               // the bytes of both CTAs
           tma_load_2d_pair(dst, &tm_h, kb * kBK, (c.mt * 2 + (int)rank) * kBM, full);
-          tma_load_2d_pair(dst + kABytes, tm_w, kb * kBK, c.nt * kBN + (int)rank * (kBN / 2), full);
+          tma_load_2d_pair(dst + kABytes, tm_w, kb * kBK, w_row, full);
+          if (c.half < 0) tma_load_2d_pair(dst + kABytes + kBBytes / 2, tm_w, kb * kBK, w_row + 64, full);
           armed[s] = it;
         }
       }
@@ -250,7 +271,10 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
     bool ok = !dead;
     if (ok) {
       int it = 0, tl = 0;
-      for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tl) {
+      for (int idx = pair; ok; idx += num_pairs, ++tl) {
+        const TileCoord c = tile_coord(idx, a);
+        if (!c.valid) break;
+        const unsigned idesc = c.half < 0 ? kIdesc : kIdescHalf;
         const int buf = tl & 1;
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->acc_empty[buf]), ((tl >> 1) & 1) ^ 1, abort_flag));
         if (!ok) break;
@@ -268,7 +292,7 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
           const unsigned long long b_desc = make_desc(ring + s * kProjStageBytes + kABytes, 16, 1024);
 #pragma unroll
           for (int k = 0; k < kBK / 16; ++k)
-            mma2_ss_elect(d_tmem, a_desc + 2 * k, b_desc + 2 * k, kIdesc, (kb | k) ? 1u : 0u);
+            mma2_ss_elect(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) ? 1u : 0u);
           mma2_commit_both_elect(smem_u32(&sy->empty[s]));
         }
         if (!ok) break;
@@ -300,16 +324,19 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
       return done;
     };
     int tl = 0;
-    for (int tile = pair; tile < total_tiles && ok; tile += num_pairs, ++tl) {
-      const TileCoord c = tile_coord(tile, a.n_tiles);
+    for (int idx = pair; ok; idx += num_pairs, ++tl) {
+      const TileCoord c = tile_coord(idx, a);
+      if (!c.valid) break;
+      const int hh_begin = c.half < 0 ? 0 : c.half, hh_end = c.half < 0 ? 2 : c.half + 1;
       const int buf = tl & 1;
       const int tok_base = (c.mt * 2 + (int)rank) * kBM;     // first token of this CTA's half
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->acc_full[buf]), (tl >> 1) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
 #pragma unroll 1
-      for (int hh = 0; hh < 2; ++hh) {
+      for (int hh = hh_begin; hh < hh_end; ++hh) {
         const int head = c.nt * 2 + hh;
+        const int col = buf * kBN + (c.half < 0 ? hh * 128 : 0);   // a split tile's head sits in the first columns
         const bool head_valid = head < a.num_kv_heads;
         if (e < 8) bulk_wait_read();                         // the previous copies have read the staging pages
         ok = epi_sync();
@@ -318,7 +345,7 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
 #pragma unroll
           for (int cc = 0; cc < 4; ++cc) {
             unsigned r[32];
-            tmem_ld32(tmem + buf * kBN + hh * 128 + cc * 32 + lane_base, r);
+            tmem_ld32(tmem + col + cc * 32 + lane_base, r);
             tmem_wait_ld();
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -331,7 +358,7 @@ project_kv_kernel(proj::ProjArgs a, int* status, const __grid_constant__ CUtenso
             }
           }
         }
-        if (hh == 1) {
+        if (hh == hh_end - 1) {
           // the accumulator has been read: the MMAs of the tile after next may overwrite it
           tc_fence_before();
           __syncwarp();
@@ -386,9 +413,16 @@ inline cudaError_t launch_project_kv(const proj::ProjArgs& a, int* status, int m
                                      cudaStream_t stream) {
   const int total = a.m_tiles * 2 * a.n_tiles;
   if (total <= 0) return cudaSuccess;
-  const int pairs = total < max_pairs ? total : max_pairs;
+  // Whole rounds of the grid work on whole tiles.  If the tiles left for the last round occupy at
+  // most half of the pairs they are split in two (one head each), which halves that round; a
+  // fuller last round is better off with whole tiles (a split tile stages H for half the work).
+  proj::ProjArgs b = a;
+  const int left = total % max_pairs;
+  b.full_tiles = 2 * left <= max_pairs ? total - left : total;
+  const int units = b.full_tiles + 2 * (total - b.full_tiles);
+  const int pairs = units < max_pairs ? units : max_pairs;
   project_kv_kernel<<<2 * pairs, proj::kProjThreads, proj::kProjSmemBytes, stream>>>(
-      a, status, tm_h, tm_wk, tm_wv, wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
+      b, status, tm_h, tm_wk, tm_wv, wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
   return cudaGetLastError();
 }
 
