@@ -476,6 +476,28 @@ def main():
     roofline_put = None
     put_bytes = 4 * w.num_layers * w.prefix_lens[0] * w.num_kv_heads * w.head_dim * (2 if w.dtype == torch.bfloat16 else 4)
     roofline_sim = None
+    # ---- prefix K/V projection into the store (Eq. 1), one layer of prefix 0, off the per-step path ----
+    roofline_proj = None
+    if w.dtype == torch.bfloat16 and w.head_dim == 128:
+        m0, d_model = w.prefix_lens[0], w.num_q_heads * w.head_dim
+        hh, wk_, wv_ = workloads.draw_hidden_and_weights(m0, d_model, w.num_kv_heads, w.head_dim, 1, device="cuda")
+        ts = []
+        for i in range(8):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            bc.project_prefix_layer(pid[0], 0, hh, wk_, wv_)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        del hh, wk_, wv_
+        ms_proj = sorted(ts[3:])[len(ts[3:]) // 2]
+        proj_flops = 2.0 * m0 * d_model * 2 * w.num_kv_heads * w.head_dim
+        tf = proj_flops / (ms_proj * 1e-3) / 1e12
+        roofline_proj = {"bound": "tensor", "kernel": "project_kv_kernel (project_prefix_layer of prefix 0, one layer)",
+                         "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
+                         "peak_source": peaks["source"], "flops_per_launch": proj_flops, "ms_per_launch": ms_proj,
+                         "d_model": d_model, "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("project")}
     if put_bytes >= (256 << 20):
         kc, vc = workloads.draw_prefix_kv(w, 0, "cuda")
         # profiler reduction (Eq. 3): cached prefix 0 against a reference K/V of the same shape; reads both once
@@ -525,7 +547,7 @@ def main():
                 "tflops": flops / (step_ms_max * 1e-3) / 1e12, "step_flops": flops,
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
                 "roofline": roofline, "roofline_attend": roofline_attend, "roofline_put": roofline_put,
-                "roofline_similarity": roofline_sim,
+                "roofline_similarity": roofline_sim, "roofline_project": roofline_proj,
                 "cpu_baseline": cpu}
         print(json.dumps(line))
     if dist is not None:

@@ -241,3 +241,32 @@ def test_hash_tokens_matches_oracle(lib):
     assert put(lib, ctx, binding.hash_tokens([5, 6, 7]), 16)[:3] == (binding.OK, 0, 1)
     assert put(lib, ctx, b, 16)[:3] == (binding.OK, 1, 0)
     lib.bicache_destroy(ctx)
+
+
+def test_projection_and_read_back_argument_checks_on_host_context(lib):
+    """Eq. 1 into the store / layer read-back: ids, layers, shapes and strides are checked on the
+    host, before anything would launch."""
+    ctx = host_ctx(lib, L=2, Hq=4, Hkv=2, D=128, pages=4)
+    pid, hit = C.c_int32(-1), C.c_int32(-1)
+    pages = np.full(4, -1, dtype=np.int32)
+    pp = pages.ctypes.data_as(C.POINTER(C.c_int32))
+    assert lib.bicache_reserve_prefix(ctx, C.c_uint64(5), 40, C.byref(pid), C.byref(hit), pp, 4) == binding.OK
+    proj = lib.bicache_project_prefix_layer
+    assert proj(ctx, pid.value + 9, 0, None, 512, None, None, 512, None) == binding.ERR_NOTFOUND
+    assert proj(ctx, pid.value, 2, None, 512, None, None, 512, None) == binding.ERR_INVALID      # layer
+    assert proj(ctx, pid.value, 0, None, 512, None, None, 508, None) == binding.ERR_INVALID      # d_model % 8
+    assert proj(ctx, pid.value, 0, None, 504, None, None, 512, None) == binding.ERR_INVALID      # stride < d_model
+    assert proj(ctx, pid.value, 0, None, 516, None, None, 512, None) == binding.ERR_INVALID      # stride % 8
+    assert proj(ctx, pid.value, 0, None, 0, None, None, 0, None) == binding.ERR_INVALID
+    assert proj(ctx, pid.value, 1, None, 520, None, None, 512, None) == binding.OK               # host-only: no launch
+    read = lib.bicache_read_prefix_layer
+    assert read(ctx, pid.value + 9, 0, None, None, 256, None) == binding.ERR_NOTFOUND
+    assert read(ctx, pid.value, 2, None, None, 256, None) == binding.ERR_INVALID
+    assert read(ctx, pid.value, 0, None, None, 255, None) == binding.ERR_INVALID
+    assert read(ctx, pid.value, 0, None, None, 256, None) == binding.ERR_UNSUPPORTED             # nothing to read from
+    lib.bicache_destroy(ctx)
+    # only bf16 with head_dim 128 has the projection
+    f32 = host_ctx(lib, L=1, Hq=2, Hkv=2, D=64, pages=4, dtype=binding.F32)
+    assert lib.bicache_reserve_prefix(f32, C.c_uint64(5), 40, C.byref(pid), C.byref(hit), pp, 4) == binding.OK
+    assert proj(f32, pid.value, 0, None, 512, None, None, 512, None) == binding.ERR_UNSUPPORTED
+    lib.bicache_destroy(f32)
