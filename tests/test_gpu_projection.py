@@ -167,3 +167,16 @@ def test_projection_status_codes():
                                                   64, None)
         f32._check(st, "bicache_project_prefix_layer")
     assert ei.value.status == binding.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3])
+def test_projection_random_shapes(seed):
+    """Seeded random small shapes: any head count, token count and d_model (multiple of 8), down to
+    one token, one head and a d_model below the 64-wide contraction block."""
+    rng = np.random.default_rng(100 + seed)
+    for _ in range(4):
+        Hkv = int(rng.integers(1, 9))
+        m = int(rng.choice([1, 15, 16, 17, int(rng.integers(18, 600))]))
+        d_model = 8 * int(rng.choice([1, 7, 8, 9, int(rng.integers(10, 100))]))
+        _check_projection(Hkv=Hkv, m=m, d_model=d_model, L=1, strided=bool(rng.integers(0, 2)),
+                          seed=int(rng.integers(1, 1000)))

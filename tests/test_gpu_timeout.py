@@ -46,3 +46,29 @@ def test_tiny_wait_budget_reports_timeout_and_context_recovers(Hq, Hkv, lens):
     err = np.abs(workloads.to_f64(out) - ref)
     assert err.max() <= 2e-2 and err.mean() <= 2e-3
     bc.close()
+
+
+def test_projection_tiny_wait_budget_reports_timeout_and_context_recovers():
+    """The same for the projection kernel, whose CTAs work in pairs: both CTAs of a pair give up,
+    wait for their loads, meet at the pair's barrier and release the pair's tensor memory."""
+    Hkv, D, m, d_model = 4, 128, 700, 512
+    bc = binding.BiCache(1, Hkv, Hkv, D, (m + 15) // 16 + 1, torch.bfloat16, 16, 1)
+    pid, _, _ = bc.reserve_prefix(3, m)
+    h, w_k, w_v = workloads.draw_hidden_and_weights(m, d_model, Hkv, D, 9, device="cuda")
+    bc.set_wait_budget(1)
+    bc.project_prefix_layer(pid, 0, h, w_k, w_v)
+    assert bc.device_status() == binding.ERR_TIMEOUT
+    bc.project_prefix_layer(pid, 0, h, w_k, w_v)            # a launch on a flagged context does no work
+    assert bc.device_status(clear=True) == binding.ERR_TIMEOUT
+    assert bc.device_status() == binding.OK
+    bc.set_wait_budget(0)
+    bc.project_prefix_layer(pid, 0, h, w_k, w_v)
+    assert bc.device_status() == binding.OK
+    rk, rv = oracle.project_kv(workloads.to_f64(h)[None], workloads.to_f64(w_k)[None], workloads.to_f64(w_v)[None],
+                               Hkv, D)
+    gk = torch.empty(m, Hkv, D, dtype=torch.bfloat16, device="cuda")
+    gv = torch.empty_like(gk)
+    bc.read_prefix_layer(pid, 0, gk, gv)
+    for got, ref in ((gk, rk[0]), (gv, rv[0])):
+        assert np.all(np.abs(workloads.to_f64(got) - ref) <= np.abs(ref) * 2.0 ** -8 + 1e-3)
+    bc.close()
