@@ -444,12 +444,29 @@ merge_partials_kernel(ScheduleView s, TensorArgs t) {
 #pragma unroll
   for (int i = 0; i < kSimtMaxD / 32; ++i) acc[i] = 0.f;
   if (any) {
-    for (int sp = 0; sp < s.num_splits; ++sp) {
-      const float w = expf(t.part_lse[pr0 + sp * split_stride] - mx) * inv_tot;
-      const float* po = t.part_o + (pr0 + sp * split_stride) * D;
+    // Lane l holds the weights of splits l, l + 32, ...; the partial rows of eight splits are
+    // loaded before any is used, so that their latencies overlap.
+    for (int base = 0; base < s.num_splits; base += 32) {
+      const int mine = base + lane;
+      const float w_lane = mine < s.num_splits ? expf(t.part_lse[pr0 + mine * split_stride] - mx) * inv_tot : 0.f;
+      const int cnt = min(32, s.num_splits - base);
+      for (int s0 = 0; s0 < cnt; s0 += 8) {
+        float v[8][kSimtMaxD / 32];
+        float w[8];
 #pragma unroll
-      for (int i = 0; i < kSimtMaxD / 32; ++i)
-        if (lane + 32 * i < D) acc[i] = fmaf(w, po[lane + 32 * i], acc[i]);
+        for (int u = 0; u < 8; ++u) {
+          const int sp = min(s0 + u, cnt - 1);               // a clamped repeat gets weight 0 below
+          const float w_sp = __shfl_sync(0xffffffffu, w_lane, sp);
+          w[u] = s0 + u < cnt ? w_sp : 0.f;
+          const float* po = t.part_o + (pr0 + (long long)(base + sp) * split_stride) * D;
+#pragma unroll
+          for (int i = 0; i < kSimtMaxD / 32; ++i) v[u][i] = lane + 32 * i < D ? po[lane + 32 * i] : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+#pragma unroll
+          for (int i = 0; i < kSimtMaxD / 32; ++i) acc[i] = fmaf(w[u], v[u][i], acc[i]);
+      }
     }
   }
 #pragma unroll
