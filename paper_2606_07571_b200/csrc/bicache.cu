@@ -22,6 +22,7 @@
 #include "simt_kernels.cuh"
 #include "tc_attention.cuh"
 #include "project_kv.cuh"
+#include "tc_decode.cuh"
 
 using namespace bicache;
 
@@ -44,13 +45,18 @@ struct PrefixEntry {
 struct CachedSchedule {
   bool valid = false;
   uint64_t last_use = 0;
-  int kind = 0;                               // 0 attend, 1 attend_full
+  int kind = 0;                               // 0 attend, 1 attend_full, 2 attend through the key-range kernel
   std::vector<int32_t> prefix_id;
   std::vector<int64_t> row_off;
   std::vector<int32_t> seqlen;
   int num_items = 0, num_splits = 1, tiles_per_split = 0, total_tokens = 0;
   size_t reqs_off = 0, pages_off = 0, items_off = 0;   // byte offsets inside the slot
+  size_t ditems_off = 0;                      // kind 2: the key-range items
+  size_t tok_rows_off = 0;                    // kind 2: row of every token of the call
+  int num_ditems = 0;
 };
+constexpr int kMaxDecodeItems = 1024;
+constexpr int kMaxDecodeTokens = 4096;        // tokens of a call served by the key-range kernel
 
 }  // namespace
 
@@ -112,7 +118,9 @@ size_t slot_bytes_for(const bicache_config* c, int64_t max_rows, int32_t max_req
   const long long max_items = std::max<long long>(tiles * c->num_kv_heads, 1) + 2LL * kTargetCtas;
   return align_up((size_t)max_req * sizeof(ReqMeta) + 16, 256) +
          align_up((size_t)c->num_pages * sizeof(int) + 16, 256) +
-         align_up((size_t)max_items * sizeof(WorkItem) + 16, 256);
+         align_up((size_t)max_items * sizeof(WorkItem) + 16, 256) +
+         align_up((size_t)kMaxDecodeItems * sizeof(dec::DecodeItem) + 16, 256) +
+         align_up((size_t)kMaxDecodeTokens * sizeof(long long) + 16, 256);
 }
 
 size_t partial_bytes_for(const bicache_config* c) {
@@ -173,7 +181,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
     if (!c.valid || c.kind != kind || (int)c.seqlen.size() != R) continue;
     if (std::memcmp(c.row_off.data(), row_off, sizeof(int64_t) * R) != 0) continue;
     if (std::memcmp(c.seqlen.data(), seqlen, sizeof(int32_t) * R) != 0) continue;
-    if (kind == 0 && std::memcmp(c.prefix_id.data(), prefix_id, sizeof(int32_t) * R) != 0) continue;
+    if (kind != 1 && std::memcmp(c.prefix_id.data(), prefix_id, sizeof(int32_t) * R) != 0) continue;
     c.last_use = ctx->use_counter;
     return s;
   }
@@ -192,7 +200,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
     r.page_off = 0;
     r.tok_off = (int)tok;
     tok += seqlen[i];
-    if (kind == 0 && prefix_id[i] >= 0) {
+    if (kind != 1 && prefix_id[i] >= 0) {
       const PrefixEntry& e = *ctx->by_id.at(prefix_id[i]);
       r.m = e.m;
       if (prefix_id[i] != last_pid) {
@@ -211,7 +219,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   // splits minimises a simple cost model: waves of CTAs (one CTA per SM) times the time of one CTA
   // (a fixed prologue/epilogue plus a per-key-tile cost), plus the merge pass over the partials.
   int num_splits = 1, tiles_per_split = 0;
-  if (unsplit_items > 0 && unsplit_items < 2LL * ctx->sm_count && max_key_tiles >= 8) {
+  if (kind != 2 && unsplit_items > 0 && unsplit_items < 2LL * ctx->sm_count && max_key_tiles >= 8) {
     const int key_tiles = max_key_tiles;
     const double c_tile = 3300.0, c_cta = 12000.0;         // SM clocks, fitted on the small-suffix shapes
     auto cost = [&](int nsplit, int tps) {
@@ -235,8 +243,58 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
     }
   }
   std::vector<WorkItem> items;
+  std::vector<dec::DecodeItem> ditems;
+  if (kind == 2) {
+    // Key-range kernel (few query rows against long cached prefixes).  Row space of the prefix ranges:
+    // all requests of a prefix group, their tokens concatenated; of the own-key range: each request.  Ranges 0 .. sp-1 split the prefix keys, range sp holds the own keys.
+    struct Group { int first, last; int n, tok_off; };
+    std::vector<Group> groups;
+    for (int i = 0; i < R; ++i) {
+      if (groups.empty() || prefix_id[i] != prefix_id[groups.back().first])
+        groups.push_back(Group{i, i, 0, reqs[i].tok_off});
+      Group& g = groups.back();
+      g.last = i;
+      g.n += seqlen[i];
+    }
+    long long base_items = 0;
+    int tiles64_max = 1;
+    for (const Group& g : groups) {
+      if (g.n <= 0) continue;
+      base_items += (long long)((g.n * (long long)G + 127) / 128) * Hkv;
+      tiles64_max = std::max(tiles64_max, (reqs[g.first].m + 63) / 64);
+    }
+    int sp = (int)std::max<long long>(1, 2LL * ctx->sm_count / std::max<long long>(1, base_items));
+    sp = std::min(sp, std::max(1, tiles64_max / 4));
+    sp = std::min(sp, 63);
+    while (sp > 1 && tok * ctx->cfg.num_q_heads * (sp + 1) > ctx->part_capacity_rowheads) --sp;
+    for (const Group& g : groups) {
+      if (g.n <= 0) continue;
+      const ReqMeta& r0m = reqs[g.first];
+      const int tiles = (r0m.m + 63) / 64, tps = (tiles + sp - 1) / sp;
+      for (int s = 0; s < sp; ++s) {
+        const int kb = s * tps * 64;
+        const int kc = std::max(0, std::min(r0m.m - kb, tps * 64));
+        for (int hk = 0; hk < Hkv; ++hk)
+          for (int r0 = 0; r0 < g.n * G; r0 += 128)
+            ditems.push_back(dec::DecodeItem{0, g.first, g.last - g.first + 1, g.n, g.tok_off, hk, r0, 0,
+                                             kc > 0 ? kb : 0, kc, r0m.page_off, s});
+      }
+    }
+    // long ranges first; the own-key ranges (short) fill the tail of the launch
+    std::stable_sort(ditems.begin(), ditems.end(),
+                     [](const dec::DecodeItem& a, const dec::DecodeItem& b) { return a.key_count > b.key_count; });
+    for (int i = 0; i < R; ++i) {
+      if (reqs[i].n <= 0) continue;
+      for (int hk = 0; hk < Hkv; ++hk)
+        for (int r0 = 0; r0 < reqs[i].n * G; r0 += 128)
+          ditems.push_back(dec::DecodeItem{reqs[i].row_off, i, 1, reqs[i].n, reqs[i].tok_off, hk, r0, 1, 0, reqs[i].n,
+                                           0, sp});
+    }
+    num_splits = sp + 1;                                   // what the merge kernel combines
+    tiles_per_split = 0;
+  }
   items.reserve((size_t)unsplit_items * num_splits);
-  for (int sp = 0; sp < num_splits; ++sp) {
+  for (int sp = 0; sp < (kind == 2 ? 1 : num_splits); ++sp) {
     const size_t first = items.size();
     for (int i = 0; i < R; ++i) {
       if (reqs[i].n <= 0) continue;
@@ -254,8 +312,16 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   const size_t reqs_off = 0;
   const size_t pages_off = align_up(reqs_off + reqs.size() * sizeof(ReqMeta) + 16, 256);
   const size_t items_off = align_up(pages_off + pages.size() * sizeof(int) + 16, 256);
-  const size_t total = items_off + items.size() * sizeof(WorkItem);
-  if (total > ctx->slot_bytes) {
+  const size_t ditems_off = align_up(items_off + items.size() * sizeof(WorkItem) + 16, 256);
+  std::vector<long long> tok_rows;
+  if (kind == 2) {
+    tok_rows.reserve((size_t)tok);
+    for (int i = 0; i < R; ++i)
+      for (int a = 0; a < reqs[i].n; ++a) tok_rows.push_back(reqs[i].row_off + a);
+  }
+  const size_t tok_rows_off = align_up(ditems_off + ditems.size() * sizeof(dec::DecodeItem) + 16, 256);
+  const size_t total = tok_rows_off + tok_rows.size() * sizeof(long long);
+  if (total > ctx->slot_bytes || (int)ditems.size() > kMaxDecodeItems || (long long)tok_rows.size() > kMaxDecodeTokens) {
     *status = fail(ctx, BICACHE_ERR_NOMEM, "workspace too small for this batch's schedule");
     return -1;
   }
@@ -268,6 +334,8 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   if (!reqs.empty()) std::memcpy(blob.data() + reqs_off, reqs.data(), reqs.size() * sizeof(ReqMeta));
   if (!pages.empty()) std::memcpy(blob.data() + pages_off, pages.data(), pages.size() * sizeof(int));
   if (!items.empty()) std::memcpy(blob.data() + items_off, items.data(), items.size() * sizeof(WorkItem));
+  if (!ditems.empty()) std::memcpy(blob.data() + ditems_off, ditems.data(), ditems.size() * sizeof(dec::DecodeItem));
+  if (!tok_rows.empty()) std::memcpy(blob.data() + tok_rows_off, tok_rows.data(), tok_rows.size() * sizeof(long long));
   CachedSchedule& c = ctx->slots[victim];
   c.valid = false;
   if (total > 0) {
@@ -283,7 +351,10 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   c.prefix_id.assign(prefix_id ? prefix_id : nullptr, prefix_id ? prefix_id + R : nullptr);
   c.row_off.assign(row_off, row_off + R);
   c.seqlen.assign(seqlen, seqlen + R);
-  c.num_items = (int)items.size();
+  c.num_items = (int)items.size() * (kind == 2 ? num_splits : 1);   // kind 2 stores the first range's items only
+  c.ditems_off = ditems_off;
+  c.tok_rows_off = tok_rows_off;
+  c.num_ditems = (int)ditems.size();
   c.num_splits = num_splits;
   c.tiles_per_split = tiles_per_split;
   c.total_tokens = (int)tok;
@@ -346,8 +417,34 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   }
   if (total == 0) return BICACHE_OK;
 
+  // the tensor-core kernels take the row maximum before scaling, which needs a positive scale
+  const bool use_tensor = ctx->tensor_ok && ctx->path != BICACHE_PATH_SIMT && softmax_scale > 0.f;
+  // Few query rows per prefix group against a long cached prefix (block-query decoding): the
+  // bandwidth-bound regime, served by the key-range kernel.  Conditions: every request has a cached
+  // prefix of at least 1024 tokens and the rows of a group's requests pack into at most two
+  // 128-row tiles per KV head.
+  bool key_ranges = kind == 0 && use_tensor;
+  if (key_ranges) {
+    const int G = cfg.num_q_heads / cfg.num_kv_heads;
+    long long group_rows = 0;
+    for (int i = 0; i < R && key_ranges; ++i) {
+      if (prefix_id[i] < 0) { key_ranges = false; break; }
+      if (i == 0 || prefix_id[i] != prefix_id[i - 1]) group_rows = 0;
+      if (ctx->by_id.at(prefix_id[i])->m < 1024) key_ranges = false;
+      group_rows += seqlen[i];
+      if (group_rows * G > 256) key_ranges = false;
+    }
+  }
   int st = BICACHE_OK;
-  const int slot = prepare_schedule(ctx, kind, R, prefix_id, row_off, seqlen, stream, &st);
+  int slot = -1;
+  if (key_ranges) {
+    slot = prepare_schedule(ctx, 2, R, prefix_id, row_off, seqlen, stream, &st);
+    if (slot < 0) {                                      // does not fit the schedule slot: the general path
+      key_ranges = false;
+      ctx->last_error.clear();
+    }
+  }
+  if (slot < 0) slot = prepare_schedule(ctx, kind, R, prefix_id, row_off, seqlen, stream, &st);
   if (slot < 0) return st;
   const CachedSchedule& c = ctx->slots[slot];
   char* base = ctx->d_slots + (size_t)slot * ctx->slot_bytes;
@@ -378,10 +475,11 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   t.total_tokens = c.total_tokens;
   const PoolView pool = pool_view(ctx);
 
-  // the tensor-core kernel takes the row maximum before scaling, which needs a positive scale
-  const bool use_tensor = ctx->tensor_ok && ctx->path != BICACHE_PATH_SIMT && softmax_scale > 0.f;
   cudaError_t e;
-  if (use_tensor) {
+  if (key_ranges) {
+    e = launch_tc_decode(reinterpret_cast<const dec::DecodeItem*>(base + c.ditems_off), c.num_ditems, sv.reqs,
+                         sv.pages, pool, t, ctx->d_status, ctx->wait_cycles, stream);
+  } else if (use_tensor) {
     // rows the tensors are known to have: up to the end of the last request
     long long rows_total = 0;
     for (int i = 0; i < R; ++i) rows_total = std::max<long long>(rows_total, row_off[i] + seqlen[i]);
@@ -406,7 +504,11 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   }
   ctx->launches++;
   if (e != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
-  if (c.num_splits > 1) {
+  if (key_ranges) {
+    e = launch_merge_ranges(t, reinterpret_cast<const long long*>(base + c.tok_rows_off), c.num_splits, stream);
+    ctx->launches++;
+    if (e != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("merge launch: ") + cudaGetErrorString(e));
+  } else if (c.num_splits > 1) {
     const int grid = c.num_items / c.num_splits * (kTileRows / kMergeRowsPerBlock);
     if (cfg.dtype == BICACHE_F32)
       merge_partials_kernel<float><<<grid, kMergeRowsPerBlock * 32, 0, stream>>>(sv, t);
@@ -497,6 +599,7 @@ int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
   if (tensor_ok) {
     cudaError_t e = configure_tc_attention();
     if (e == cudaSuccess) e = configure_project_kv(&ctx->proj_pairs);
+    if (e == cudaSuccess) e = configure_tc_decode();
     if (e != cudaSuccess) {
       delete ctx;
       return BICACHE_ERR_CUDA;

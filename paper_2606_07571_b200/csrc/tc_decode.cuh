@@ -1,0 +1,471 @@
+// Few query rows against many keys (block-query decoding shapes): the bandwidth-bound form of
+// Eq. 2 / Eq. 4.  One CTA computes, for up to 128 packed query rows of one KV head and one RANGE of
+// keys, the normalised partial result and its log-sum-exp; a merge kernel combines the ranges
+// (the identity behind the log-sum-exp merge: softmax over a union of key sets).  The query rows of
+// ALL requests of a prefix group sit in one tile when their rows are adjacent in memory, so the
+// cached prefix is read once per group, not once per request; each request's own keys are one
+// more range, handled by CTAs of the same launch.
+//
+// Why a second kernel: with one 128-row tile per CTA the big kernel's chain S -> softmax -> P V
+// runs once per 128 keys with nothing to overlap it, and one CTA per SM cannot keep HBM busy.
+// Here a CTA is small (96 KB of shared memory, 256 TMEM columns: two CTAs per SM), key tiles are
+// 64 keys, and S is double-buffered in TMEM: S(j+1) = Q K(j+1)^T is issued before the softmax of
+// tile j ends.  Roles: warps 0-3 softmax (one thread per row), warp 4 MMA issue and TMEM, warp 5
+// gathers Q and stages K tiles, warp 6 stages V tiles (cached pages: one 4 KB bulk copy per page,
+// a pool page already is the operand image; own rows: 16-byte gathers into the same image).
+// Every wait is bounded, as in the big kernel.
+#pragma once
+
+#include "tc_attention.cuh"
+
+namespace bicache {
+namespace dec {
+
+using namespace tc;
+
+constexpr int kKeys = 64;                          // keys per tile
+constexpr int kKvTileBytes = kKeys * 128 * 2;      // 16 KB
+constexpr int kQBytes = 128 * 128 * 2;             // 32 KB
+constexpr int kDecStages = 2;
+constexpr int kDecThreads = 224;
+constexpr int kDecTmemCols = 256;                  // S0 0-63, S1 64-127 (P over the first 32 of each), O 128-255
+// fp32 accumulate, bf16 A and B (both K-major), M = 128, N = 64
+constexpr unsigned kIdescS64 = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
+
+struct DecodeItem {
+  long long row_off;     // kind 1: first row of the request (its own keys are rows row_off .. + n - 1 of k / v)
+  int req_first;         // the row space: requests req_first .. req_first + req_count - 1 of the call, their
+  int req_count;         // tokens concatenated (a request, or all requests of a prefix group)
+  int n;                 // tokens in the row space
+  int tok_off;           // index of the row space's first token among the call's tokens (partials)
+  int kv_head;
+  int row0;              // first packed row of the item (multiple of 128)
+  int kind;              // 0: cached prefix keys (paged), 1: the rows' own keys
+  int key_begin;         // first key of the range (multiple of 64)
+  int key_count;         // keys in the range (0: the item only writes the neutral partial)
+  int page_off;          // kind 0: index of the prefix's first page id in the schedule's page list
+  int slot;              // which partial this range is
+};
+
+struct DecSync {
+  unsigned long long q_full;
+  unsigned long long k_full[kDecStages], k_free[kDecStages];
+  unsigned long long v_full[kDecStages], v_free[kDecStages];
+  unsigned long long s_full[2];          // S of a key tile is in TMEM
+  unsigned long long p_full[2];          // P of the tile is in TMEM (and O rescaled if it had to be)
+  unsigned long long pv_done;            // O += P V of a tile has completed (one phase per tile)
+  unsigned long long o_done;             // O += P V of the LAST tile has completed
+  unsigned long long drain;
+  long long wait_cycles;                 // directly before abort_flag (mbar_wait reads it)
+  int abort_flag;
+  unsigned tmem_base;
+  int dead;
+};
+constexpr int kDecSmemBytes = 1024 + kQBytes + 2 * kDecStages * kKvTileBytes + (int)sizeof(DecSync);
+static_assert(2 * (kDecSmemBytes + 1024) <= 232448, "two CTAs per SM");
+
+}  // namespace dec
+
+__global__ void __launch_bounds__(dec::kDecThreads, 2)
+tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __restrict__ reqs,
+                 const int* __restrict__ pages, PoolView pool, TensorArgs t, int* status, long long wait_cycles) {
+  using namespace dec;
+  extern __shared__ unsigned char smem_raw[];
+  unsigned char* smem =
+      reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  DecSync* sy = reinterpret_cast<DecSync*>(smem + kQBytes + 2 * kDecStages * kKvTileBytes);
+  volatile int* abort_flag = &sy->abort_flag;
+  const unsigned q_smem = smem_u32(smem);
+  const unsigned k_ring = q_smem + kQBytes, v_ring = k_ring + kDecStages * kKvTileBytes;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // the merge kernel that follows may be placed on the SMs from now on (it waits for this grid's end)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const DecodeItem it = items[blockIdx.x];
+  const int G = t.Hq / t.Hkv;
+  const int T = (it.key_count + kKeys - 1) / kKeys;
+
+  if (tid == 0) {
+    sy->wait_cycles = wait_cycles;
+    sy->dead = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
+    sy->abort_flag = (sy->dead || wait_cycles < kStrictBudget) ? 1 : 0;
+    mbar_init(smem_u32(&sy->q_full), 32);
+    for (int i = 0; i < kDecStages; ++i) {
+      mbar_init(smem_u32(&sy->k_full[i]), 32);
+      mbar_init(smem_u32(&sy->k_free[i]), 1);
+      mbar_init(smem_u32(&sy->v_full[i]), 32);
+      mbar_init(smem_u32(&sy->v_free[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&sy->s_full[i]), 1);
+      mbar_init(smem_u32(&sy->p_full[i]), 128);
+    }
+    mbar_init(smem_u32(&sy->pv_done), 1);
+    mbar_init(smem_u32(&sy->o_done), 1);
+    mbar_init(smem_u32(&sy->drain), 1);
+    fence_barrier_init();
+  }
+  if (warp == 4) {
+    tmem_alloc(smem_u32(&sy->tmem_base), kDecTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&sy->tmem_base);
+  const bool dead = *reinterpret_cast<volatile int*>(&sy->dead) != 0;
+  const unsigned tmem_o = tmem + 128;
+
+  if (warp < 4) {
+    // ================================ softmax and epilogue =================================
+    const int row = warp * 32 + lane;                        // row of the tile = TMEM lane
+    const unsigned lane_base = (unsigned)(warp * 32) << 16;
+    const float sl2 = t.scale * 1.4426950408889634f;         // scores are handled in the log2 domain
+    float m_ref = -INFINITY, l_sum = 0.f;
+    bool ok = !dead;
+    for (int j = 0; j < T && ok; ++j) {
+      const int b = j & 1;
+      const int cnt = min(kKeys, it.key_count - j * kKeys);
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->s_full[b]), (j >> 1) & 1, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      unsigned r[64];
+      tmem_ld32(tmem + b * 64 + lane_base, r);
+      tmem_ld32(tmem + b * 64 + 32 + lane_base, r + 32);
+      tmem_wait_ld();
+      if (cnt < kKeys) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+          if (i >= cnt) r[i] = 0xff800000u;                  // -inf: columns past the last key
+      }
+      float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < 64; i += 4) {
+        mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+        mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+      }
+      const float mx = fmaxf(mx0, mx1) * sl2;                // scale > 0
+      if (j == 0) {
+        m_ref = mx;
+      } else if (__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+        // Rare: a row's maximum exceeds the reference by more than 2^8.  O must be rescaled, and
+        // S of this tile was issued before O += P V of the previous one: wait for that first.
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->pv_done), (j - 1) & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        float alpha = 1.f;
+        if (mx > m_ref + 8.f) {
+          alpha = ex2(m_ref - mx);
+          m_ref = mx;
+        }
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          unsigned o[32];
+          tmem_ld32(tmem_o + c * 32 + lane_base, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+          tmem_st32(tmem_o + c * 32 + lane_base, o);
+        }
+        tmem_wait_st();
+        l_sum *= alpha;
+      }
+      const unsigned long long sl2_2 = pack2(sl2, sl2), neg_m2 = pack2(-m_ref, -m_ref);
+      unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const unsigned long long xa =
+            fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+        const unsigned long long xb =
+            fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+        float x0, x1, x2, x3;
+        unpack2(xa, x0, x1);
+        unpack2(xb, x2, x3);
+        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+        acc_a = add2(acc_a, pack2(p0, p1));
+        acc_b = add2(acc_b, pack2(p2, p3));
+        r[2 * i] = pack_bf16(p0, p1);
+        r[2 * i + 1] = pack_bf16(p2, p3);
+      }
+      tmem_st32(tmem + b * 64 + lane_base, r);               // P over the first 32 columns of this S
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(smem_u32(&sy->p_full[b]));
+      float s0, s1, s2, s3;
+      unpack2(acc_a, s0, s1);
+      unpack2(acc_b, s2, s3);
+      l_sum += (s0 + s1) + (s2 + s3);
+    }
+    // -------- epilogue: the normalised partial of this key range and its log-sum-exp --------
+    if (ok) {
+      const int p = it.row0 + row;                           // packed row of the row space
+      const bool row_valid = p < it.n * G;
+      const int a = p / G;
+      const int h = it.kv_head * G + (p - a * G);
+      const long long pr = ((long long)it.slot * t.total_tokens + it.tok_off + a) * t.Hq + h;
+      if (T > 0) {
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->o_done), 0, abort_flag));
+        if (ok) {
+          tc_fence_after();
+          const float inv = 1.f / l_sum;
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            unsigned o[32];
+            tmem_ld32(tmem_o + c * 32 + lane_base, o);
+            tmem_wait_ld();
+            if (row_valid) {
+              float* po = t.part_o + pr * 128 + c * 32;
+#pragma unroll
+              for (int i = 0; i < 32; i += 4)
+                *reinterpret_cast<float4*>(po + i) =
+                    make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv,
+                                __uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+            }
+          }
+          if (row_valid) t.part_lse[pr] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+        }
+      } else if (row_valid) {
+        float* po = t.part_o + pr * 128;
+#pragma unroll 4
+        for (int i = 0; i < 128; i += 4) *reinterpret_cast<float4*>(po + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+        t.part_lse[pr] = -INFINITY;
+      }
+    }
+    tc_fence_before();
+  } else if (warp == 4) {
+    // ====================================== MMA issue ======================================
+    bool ok = !dead && T > 0;
+    if (ok) {
+      const unsigned long long q_desc = make_desc(q_smem, 16, 2048);
+      // a K step of 16 dims: 32 bytes inside the swizzled row; dims 64.. sit 1024 bytes further
+      auto kstep = [](int k) { return (unsigned long long)((k & 3) * 2 + (k >> 2) * 64); };
+      auto issue_s = [&](int j) {
+        const int b = j & 1;
+        bool good = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->k_full[b]), (j >> 1) & 1, abort_flag));
+        if (!good) return false;
+        tc_fence_after();
+        const unsigned long long k_desc = make_desc(k_ring + b * kKvTileBytes, 16, 2048);
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          mma_ss_elect(tmem + b * 64, q_desc + kstep(k), k_desc + kstep(k), kIdescS64, k > 0 ? 1u : 0u);
+        mma_commit_elect(smem_u32(&sy->s_full[b]));
+        mma_commit_elect(smem_u32(&sy->k_free[b]));
+        return true;
+      };
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->q_full), 0, abort_flag));
+      if (ok) ok = issue_s(0);
+      for (int j = 0; j < T && ok; ++j) {
+        const int b = j & 1;
+        if (j + 1 < T) {
+          ok = issue_s(j + 1);
+          if (!ok) break;
+        }
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->p_full[b]), (j >> 1) & 1, abort_flag));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->v_full[b]), (j >> 1) & 1, abort_flag));
+        if (!ok) break;
+        tc_fence_after();
+        // V is the MN-major operand: 64-dim halves 1024 bytes apart, 8-key groups 2048 bytes; a K
+        // step of 16 keys is one page image (4096 bytes).  Steps past the last key are skipped.
+        const unsigned long long v_desc = make_desc(v_ring + b * kKvTileBytes, 1024, 2048);
+        const int cnt = min(kKeys, it.key_count - j * kKeys);
+        const int ksteps = (cnt + 15) >> 4;
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+          mma_ts_elect(tmem_o, tmem + b * 64 + k * 8, v_desc + (unsigned long long)(k * 256), kIdescPV,
+                       (j > 0 || k > 0) ? 1u : 0u, k < ksteps ? 1u : 0u);
+        mma_commit_elect(smem_u32(&sy->v_free[b]));
+        mma_commit_elect(smem_u32(&sy->pv_done));
+        if (j == T - 1) mma_commit_elect(smem_u32(&sy->o_done));
+      }
+      // Whatever happened, let every MMA issued so far finish before TMEM is released.
+      __syncwarp();
+      mma_commit_elect(smem_u32(&sy->drain));
+      mbar_wait_issued(smem_u32(&sy->drain), 0);
+    }
+    __syncwarp();
+  } else {
+    // ======================================= loads ========================================
+    // Warp 5 gathers the Q tile, then stages the K tiles; warp 6 stages the V tiles.
+    const int is_v = warp - 5;
+    const int r0 = lane >> 4, c16 = lane & 15;
+    bool ok = !dead;
+    int armed[kDecStages] = {-1, -1};        // the last tile armed with bulk copies, per stage
+    if (ok && !is_v && T > 0) {
+      // Packed row p = token a * G + head jj of the KV group; rows past the end are zero-filled.
+      // Token a of the row space is token tok_off + a of the call: the request that holds it is
+      // found by walking the space's requests (a only grows along a lane's rows).
+      const int packed_rows = it.n * G;
+      const char* const q_head = t.q + ((long long)it.kv_head * G * 128) * 2 + c16 * 16;
+      int kreq = it.req_first;
+      const int kreq_end = it.req_first + it.req_count;
+      ReqMeta rq = reqs[kreq];
+#pragma unroll 2
+      for (int i = 0; i < 64; ++i) {
+        const int prow = it.row0 + r0 + 2 * i;
+        const bool valid = prow < packed_rows;
+        const char* src = q_head;
+        if (valid) {
+          const int a = prow / G, jj = prow - a * G;
+          const int tg = it.tok_off + a;
+          while (tg >= rq.tok_off + rq.n && kreq + 1 < kreq_end) rq = reqs[++kreq];
+          src = q_head + ((rq.row_off + (tg - rq.tok_off)) * t.q_stride + jj * 128) * 2;
+        }
+        cp_async16(q_smem + tile_chunk_offset(r0 + 2 * i, c16), src, valid ? 16u : 0u);
+      }
+      cp_async_commit();
+      cp_async_wait<0>();
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&sy->q_full));
+    }
+    const unsigned ring = is_v ? v_ring : k_ring;
+    for (int j = 0; j < T && ok; ++j) {
+      const int b = j & 1;
+      const unsigned free_bar = smem_u32(is_v ? &sy->v_free[b] : &sy->k_free[b]);
+      const unsigned full = smem_u32(is_v ? &sy->v_full[b] : &sy->k_full[b]);
+      ok = __all_sync(0xffffffffu, mbar_wait(free_bar, ((j >> 1) & 1) ^ 1, abort_flag));
+      if (!ok) break;
+      const unsigned dst = ring + b * kKvTileBytes;
+      const int key0 = it.key_begin + j * kKeys;
+      const int cnt = min(kKeys, it.key_count - j * kKeys);
+      if (it.kind == 0) {
+        // cached prefix: one bulk copy per page (a pool page already is the tile image), each issued
+        // by its own lane so that the page-table reads overlap
+        const int npages = (cnt + kPageSize - 1) / kPageSize;
+        if (lane < npages) {
+          const char* pool_base = is_v ? pool.v : pool.k;
+          bulk_copy_g2s(dst + lane * kPageBytes,
+                        pool_base + pool_slice_offset(pool, t.layer, pages[it.page_off + key0 / kPageSize + lane],
+                                                      it.kv_head),
+                        kPageBytes, full);
+        }
+        // every lane arrives, so the phase cannot complete before lane 0 has announced the bytes
+        if (lane == 0) {
+          mbar_arrive_expect_tx(full, (unsigned)(npages * kPageBytes));
+          armed[b] = j;
+        } else {
+          mbar_arrive(full);
+        }
+      } else {
+        // the rows' own keys: 16-byte gathers into the page-image layout, zero-filled past the end
+        const char* rowp = (is_v ? t.v : t.k) + ((it.row_off + key0) * t.kv_stride + (long long)it.kv_head * 128) * 2 +
+                           c16 * 16;
+        const long long row_bytes = t.kv_stride * 2;
+        const char* src = rowp + r0 * row_bytes;
+#pragma unroll 4
+        for (int i = 0; i < kKeys / 2; ++i) {
+          const bool valid = r0 + 2 * i < cnt;
+          cp_async16(dst + tile_chunk_offset(r0 + 2 * i, c16), valid ? src : rowp, valid ? 16u : 0u);
+          src += 2 * row_bytes;
+        }
+        cp_async_commit();
+        cp_async_wait<0>();
+        fence_proxy_async();
+        mbar_arrive(full);
+      }
+    }
+    cp_async_wait<0>();
+    // After a give-up, bulk copies may still be in flight: wait (bounded) for the barriers armed last.
+    if (!dead && (!ok || *abort_flag) && lane == 0) {
+      for (int b = 0; b < kDecStages; ++b)
+        if (armed[b] >= 0) {
+          const unsigned full = smem_u32(is_v ? &sy->v_full[b] : &sy->k_full[b]);
+          for (unsigned n = 0; n < 4096 && !mbar_try_wait(full, (armed[b] >> 1) & 1); ++n) __nanosleep(256);
+        }
+    }
+  }
+
+  __syncthreads();
+  if (warp == 4) {
+    tc_fence_after();
+    tmem_dealloc(tmem, kDecTmemCols);
+  }
+  if (tid == 0 && !dead && *abort_flag) atomicCAS(status, kDevOk, kDevTimeout);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Merge of the key ranges (the log-sum-exp merge): for every (token, query head) of the call,
+//   lse = log sum_s exp(lse_s),  o = sum_s exp(lse_s - lse) o_s
+// over the num_slots partials, written as the bf16 output row.  One warp per (token, head), one
+// float4 of the 128 dims per lane; the rows of eight ranges are loaded before any is used.
+// Launched as a programmatic dependent of the key-range kernel: the grid is placed while that
+// kernel still runs and waits here for its memory to be visible.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMergeWarps = 8;
+
+__global__ void __launch_bounds__(kMergeWarps * 32)
+merge_ranges_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse,
+                    const long long* __restrict__ tok_rows, int total_tokens, int Hq, int num_slots,
+                    char* __restrict__ out, long long out_stride, float* __restrict__ lse_out) {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const long long pr = (long long)blockIdx.x * kMergeWarps + warp;     // token * Hq + head
+  if (pr >= (long long)total_tokens * Hq) return;
+  const int tg = (int)(pr / Hq), h = (int)(pr - (long long)tg * Hq);
+  const long long row = tok_rows[tg];
+  const long long slot_stride = (long long)total_tokens * Hq;
+  const float l0 = lane < num_slots ? part_lse[pr + lane * slot_stride] : -INFINITY;
+  const float l1 = lane + 32 < num_slots ? part_lse[pr + (lane + 32) * slot_stride] : -INFINITY;
+  const float mx = warp_max(fmaxf(l0, l1));
+  const bool any = mx > -INFINITY;
+  float w0 = any ? expf(l0 - mx) : 0.f, w1 = any ? expf(l1 - mx) : 0.f;
+  const float tot = warp_sum(w0 + w1);
+  const float inv = any ? 1.f / tot : 0.f;
+  w0 *= inv;
+  w1 *= inv;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s0 = 0; s0 < num_slots; s0 += 8) {
+    float4 v[8];
+    float w[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int sl = min(s0 + u, num_slots - 1);             // a clamped repeat gets weight 0
+      const float ws = __shfl_sync(0xffffffffu, sl < 32 ? w0 : w1, sl & 31);
+      w[u] = s0 + u < num_slots ? ws : 0.f;
+      v[u] = *reinterpret_cast<const float4*>(part_o + (pr + sl * slot_stride) * 128 + lane * 4);
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      acc.x = fmaf(w[u], v[u].x, acc.x);
+      acc.y = fmaf(w[u], v[u].y, acc.y);
+      acc.z = fmaf(w[u], v[u].z, acc.z);
+      acc.w = fmaf(w[u], v[u].w, acc.w);
+    }
+  }
+  uint2 o2;
+  o2.x = tc::pack_bf16(acc.x, acc.y);
+  o2.y = tc::pack_bf16(acc.z, acc.w);
+  *reinterpret_cast<uint2*>(out + (row * out_stride + (long long)h * 128) * 2 + lane * 8) = o2;
+  if (lane == 0 && lse_out != nullptr) lse_out[row * Hq + h] = any ? mx + logf(tot) : -INFINITY;
+}
+
+inline cudaError_t launch_merge_ranges(const TensorArgs& t, const long long* tok_rows, int num_slots,
+                                       cudaStream_t stream) {
+  const long long row_heads = (long long)t.total_tokens * t.Hq;
+  if (row_heads <= 0) return cudaSuccess;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)((row_heads + kMergeWarps - 1) / kMergeWarps), 1, 1);
+  cfg.blockDim = dim3(kMergeWarps * 32, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, merge_ranges_kernel, (const float*)t.part_o, (const float*)t.part_lse, tok_rows,
+                            t.total_tokens, t.Hq, num_slots, t.out, t.out_stride, t.lse);
+}
+
+inline cudaError_t configure_tc_decode() {
+  return cudaFuncSetAttribute(tc_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dec::kDecSmemBytes);
+}
+
+inline cudaError_t launch_tc_decode(const dec::DecodeItem* items, int num_items, const ReqMeta* reqs, const int* pages,
+                                    const PoolView& pool,
+                                    const TensorArgs& t, int* status, long long wait_cycles, cudaStream_t stream) {
+  if (num_items <= 0) return cudaSuccess;
+  tc_decode_kernel<<<num_items, dec::kDecThreads, dec::kDecSmemBytes, stream>>>(
+      items, reqs, pages, pool, t, status, wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
+  return cudaGetLastError();
+}
+
+}  // namespace bicache
