@@ -280,16 +280,19 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
                                              kc > 0 ? kb : 0, kc, r0m.page_off, s});
       }
     }
-    // long ranges first; the own-key ranges (short) fill the tail of the launch
+    // long prefix ranges first
     std::stable_sort(ditems.begin(), ditems.end(),
                      [](const dec::DecodeItem& a, const dec::DecodeItem& b) { return a.key_count > b.key_count; });
+    // The own-key ranges (one short tile or two each) go in front of everything: they leave their
+    // SM slots within a few microseconds, whereas at the end they would be a round of their own.
+    std::vector<dec::DecodeItem> own;
     for (int i = 0; i < R; ++i) {
       if (reqs[i].n <= 0) continue;
       for (int hk = 0; hk < Hkv; ++hk)
         for (int r0 = 0; r0 < reqs[i].n * G; r0 += 128)
-          ditems.push_back(dec::DecodeItem{reqs[i].row_off, i, 1, reqs[i].n, reqs[i].tok_off, hk, r0, 1, 0, reqs[i].n,
-                                           0, sp});
+          own.push_back(dec::DecodeItem{reqs[i].row_off, i, 1, reqs[i].n, reqs[i].tok_off, hk, r0, 1, 0, reqs[i].n, 0, sp});
     }
+    ditems.insert(ditems.begin(), own.begin(), own.end());
     num_splits = sp + 1;                                   // what the merge kernel combines
     tiles_per_split = 0;
   }

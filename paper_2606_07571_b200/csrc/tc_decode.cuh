@@ -11,7 +11,7 @@
 // Here a CTA is small (96 KB of shared memory, 256 TMEM columns: two CTAs per SM), key tiles are
 // 64 keys, and S is double-buffered in TMEM: S(j+1) = Q K(j+1)^T is issued before the softmax of
 // tile j ends.  Roles: warps 0-3 softmax (one thread per row), warp 4 MMA issue and TMEM, warp 5
-// gathers Q and stages K tiles, warp 6 stages V tiles (cached pages: one 4 KB bulk copy per page,
+// stages K tiles, warp 6 gathers Q and stages V tiles (cached pages: one 4 KB bulk copy per page,
 // a pool page already is the operand image; own rows: 16-byte gathers into the same image).
 // Every wait is bounded, as in the big kernel.
 #pragma once
@@ -284,12 +284,13 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     __syncwarp();
   } else {
     // ======================================= loads ========================================
-    // Warp 5 gathers the Q tile, then stages the K tiles; warp 6 stages the V tiles.
+    // Warp 5 stages the K tiles; warp 6 gathers the Q tile (needed together with the first K tile,
+    // so the two loads overlap), then stages the V tiles.
     const int is_v = warp - 5;
     const int r0 = lane >> 4, c16 = lane & 15;
     bool ok = !dead;
     int armed[kDecStages] = {-1, -1};        // the last tile armed with bulk copies, per stage
-    if (ok && !is_v && T > 0) {
+    if (ok && is_v && T > 0) {
       // Packed row p = token a * G + head jj of the KV group; rows past the end are zero-filled.
       // Token a of the row space is token tok_off + a of the call: the request that holds it is
       // found by walking the space's requests (a only grows along a lane's rows).
@@ -391,13 +392,17 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
 // ---------------------------------------------------------------------------------------------
 constexpr int kMergeWarps = 8;
 
+// kSlotWarps = 1: one warp per (token, head), eight per block.  kSlotWarps = 8: the eight warps of a
+// block share one (token, head), warp w taking ranges w, w + 8, ...; for many ranges and few rows.
+template <int kSlotWarps>
 __global__ void __launch_bounds__(kMergeWarps * 32)
 merge_ranges_kernel(const float* __restrict__ part_o, const float* __restrict__ part_lse,
                     const long long* __restrict__ tok_rows, int total_tokens, int Hq, int num_slots,
                     char* __restrict__ out, long long out_stride, float* __restrict__ lse_out) {
+  __shared__ float4 red[kSlotWarps == 1 ? 1 : kMergeWarps][32];
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long pr = (long long)blockIdx.x * kMergeWarps + warp;     // token * Hq + head
+  const long long pr = kSlotWarps == 1 ? (long long)blockIdx.x * kMergeWarps + warp : (long long)blockIdx.x;   // token * Hq + head
   if (pr >= (long long)total_tokens * Hq) return;
   const int tg = (int)(pr / Hq), h = (int)(pr - (long long)tg * Hq);
   const long long row = tok_rows[tg];
@@ -412,14 +417,17 @@ merge_ranges_kernel(const float* __restrict__ part_o, const float* __restrict__ 
   w0 *= inv;
   w1 *= inv;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s0 = 0; s0 < num_slots; s0 += 8) {
+  // this warp's ranges: first, first + kSlotWarps, ...; eight of them are loaded before any is used
+  const int first = kSlotWarps == 1 ? 0 : warp;
+  for (int s0 = first; s0 < num_slots; s0 += 8 * kSlotWarps) {
     float4 v[8];
     float w[8];
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
-      const int sl = min(s0 + u, num_slots - 1);             // a clamped repeat gets weight 0
+      const int want = s0 + u * kSlotWarps;
+      const int sl = min(want, num_slots - 1);               // a clamped repeat gets weight 0
       const float ws = __shfl_sync(0xffffffffu, sl < 32 ? w0 : w1, sl & 31);
-      w[u] = s0 + u < num_slots ? ws : 0.f;
+      w[u] = want < num_slots ? ws : 0.f;
       v[u] = *reinterpret_cast<const float4*>(part_o + (pr + sl * slot_stride) * 128 + lane * 4);
     }
 #pragma unroll
@@ -428,6 +436,19 @@ merge_ranges_kernel(const float* __restrict__ part_o, const float* __restrict__ 
       acc.y = fmaf(w[u], v[u].y, acc.y);
       acc.z = fmaf(w[u], v[u].z, acc.z);
       acc.w = fmaf(w[u], v[u].w, acc.w);
+    }
+  }
+  if (kSlotWarps > 1) {
+    red[warp][lane] = acc;
+    __syncthreads();
+    if (warp != 0) return;
+#pragma unroll
+    for (int w = 1; w < kMergeWarps; ++w) {
+      const float4 o = red[w][lane];
+      acc.x += o.x;
+      acc.y += o.y;
+      acc.z += o.z;
+      acc.w += o.w;
     }
   }
   uint2 o2;
@@ -441,8 +462,9 @@ inline cudaError_t launch_merge_ranges(const TensorArgs& t, const long long* tok
                                        cudaStream_t stream) {
   const long long row_heads = (long long)t.total_tokens * t.Hq;
   if (row_heads <= 0) return cudaSuccess;
+  const bool slot_warps = num_slots > 16;                   // many ranges: spread them over the block's warps
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)((row_heads + kMergeWarps - 1) / kMergeWarps), 1, 1);
+  cfg.gridDim = dim3((unsigned)(slot_warps ? row_heads : (row_heads + kMergeWarps - 1) / kMergeWarps), 1, 1);
   cfg.blockDim = dim3(kMergeWarps * 32, 1, 1);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
@@ -451,7 +473,10 @@ inline cudaError_t launch_merge_ranges(const TensorArgs& t, const long long* tok
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, merge_ranges_kernel, (const float*)t.part_o, (const float*)t.part_lse, tok_rows,
+  if (slot_warps)
+    return cudaLaunchKernelEx(&cfg, merge_ranges_kernel<8>, (const float*)t.part_o, (const float*)t.part_lse, tok_rows,
+                              t.total_tokens, t.Hq, num_slots, t.out, t.out_stride, t.lse);
+  return cudaLaunchKernelEx(&cfg, merge_ranges_kernel<1>, (const float*)t.part_o, (const float*)t.part_lse, tok_rows,
                             t.total_tokens, t.Hq, num_slots, t.out, t.out_stride, t.lse);
 }
 
