@@ -338,6 +338,17 @@ int32_t bicache_attend_full_static(int32_t dtype, int32_t num_q_heads, int32_t n
 /* Number of kernels this context has launched so far (for benchmarks' launch accounting). */
 int64_t bicache_launch_count(const bicache_ctx* ctx);
 
+/* Which attention kernel the context's last attention call launched (for tests and benchmarks):
+ * 0 none yet; BICACHE_KERNEL_SIMT the CUDA-core kernel (fp32, head dims other than 128, forced);
+ * BICACHE_KERNEL_TENSOR the tensor-core kernel over two 128-row query tiles per work item;
+ * BICACHE_KERNEL_KEY_RANGES the tensor-core kernel for few query rows against a long cached prefix
+ * (bicache_attend only; chosen when every request has a cached prefix of at least 1024 tokens and the
+ * suffix rows of each prefix group, all requests together, times Hq / Hkv are at most 256): the group's
+ * rows share tiles, the prefix keys are split into ranges over the CTAs, each request's own keys are
+ * one more range, and a merge kernel applies the log-sum-exp merge (exact up to rounding). */
+enum { BICACHE_KERNEL_SIMT = 1, BICACHE_KERNEL_TENSOR = 2, BICACHE_KERNEL_KEY_RANGES = 3 };
+int32_t bicache_last_attention_kernel(const bicache_ctx* ctx);
+
 /* Human-readable text for the last error of this context (host string, valid until next call). */
 const char* bicache_last_error(const bicache_ctx* ctx);
 

@@ -14,6 +14,7 @@ import torch
 OK, ERR_INVALID, ERR_NOMEM, ERR_NOTFOUND, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = range(7)
 F32, BF16 = 0, 1
 PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
+KERNEL_SIMT, KERNEL_TENSOR, KERNEL_KEY_RANGES = 1, 2, 3
 _STATUS_NAMES = ["OK", "INVALID", "NOMEM", "NOTFOUND", "CUDA", "TIMEOUT", "UNSUPPORTED"]
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbicache.so")
@@ -27,7 +28,7 @@ EXPORTED = [
     "bicache_read_prefix_layer", "bicache_project_prefix_layer",
     "bicache_prefix_similarity", "bicache_prefix_similarity_async", "bicache_depth_from_similarity",
     "bicache_build_depth_table",
-    "bicache_hash_tokens", "bicache_device_status", "bicache_set_wait_budget", "bicache_launch_count", "bicache_last_error",
+    "bicache_hash_tokens", "bicache_device_status", "bicache_set_wait_budget", "bicache_launch_count", "bicache_last_attention_kernel", "bicache_last_error",
 ]
 
 
@@ -126,6 +127,8 @@ def load_library():
     lib.bicache_launch_count.argtypes = [vp]
     lib.bicache_last_error.restype = C.c_char_p
     lib.bicache_last_error.argtypes = [vp]
+    lib.bicache_last_attention_kernel.restype = C.c_int32
+    lib.bicache_last_attention_kernel.argtypes = [vp]
     _lib = lib
     return lib
 
@@ -359,6 +362,9 @@ class BiCache:
 
     def set_wait_budget(self, sm_cycles):
         self._check(self.lib.bicache_set_wait_budget(self.ctx, sm_cycles), "bicache_set_wait_budget")
+
+    def last_attention_kernel(self):
+        return self.lib.bicache_last_attention_kernel(self.ctx)
 
     def launch_count(self):
         return int(self.lib.bicache_launch_count(self.ctx))

@@ -65,6 +65,7 @@ struct bicache_ctx {
   int esize = 2;
   bool swizzled = false;
   bool tensor_ok = false;
+  int last_kernel = 0;                                            // which attention kernel the last call launched
   int proj_pairs = 0;                                             // CTA pairs of the projection kernel the device runs at once
   bool host_only = false;                                         // cfg.device < 0: bookkeeping only
   int path = BICACHE_PATH_AUTO;
@@ -263,7 +264,12 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
       base_items += (long long)((g.n * (long long)G + 127) / 128) * Hkv;
       tiles64_max = std::max(tiles64_max, (reqs[g.first].m + 63) / 64);
     }
-    int sp = (int)std::max<long long>(1, 2LL * ctx->sm_count / std::max<long long>(1, base_items));
+    // ranges per prefix: what fills the two CTA slots of every SM once, next to the own-key CTAs
+    long long own_items = 0;
+    for (int i = 0; i < R; ++i)
+      if (reqs[i].n > 0) own_items += (long long)((reqs[i].n * (long long)G + 127) / 128) * Hkv;
+    const long long slots_left = std::max<long long>(2LL * ctx->sm_count - own_items, ctx->sm_count);
+    int sp = (int)std::max<long long>(1, slots_left / std::max<long long>(1, base_items));
     sp = std::min(sp, std::max(1, tiles64_max / 4));
     sp = std::min(sp, 63);
     while (sp > 1 && tok * ctx->cfg.num_q_heads * (sp + 1) > ctx->part_capacity_rowheads) --sp;
@@ -479,6 +485,7 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   const PoolView pool = pool_view(ctx);
 
   cudaError_t e;
+  ctx->last_kernel = key_ranges ? BICACHE_KERNEL_KEY_RANGES : use_tensor ? BICACHE_KERNEL_TENSOR : BICACHE_KERNEL_SIMT;
   if (key_ranges) {
     e = launch_tc_decode(reinterpret_cast<const dec::DecodeItem*>(base + c.ditems_off), c.num_ditems, sv.reqs,
                          sv.pages, pool, t, ctx->d_status, ctx->wait_cycles, stream);
@@ -1190,7 +1197,8 @@ int32_t bicache_device_status(bicache_ctx* ctx, void* stream, int32_t clear) {
     return fail(ctx, BICACHE_ERR_CUDA, "status read failed");
   if (clear && word != 0) cudaMemset(ctx->d_status, 0, kStatusBytes);
   if (word == kDevOk) return BICACHE_OK;
-  return fail(ctx, word == kDevTimeout ? BICACHE_ERR_TIMEOUT : BICACHE_ERR_CUDA, "device-side wait gave up");
+  if (word == kDevTimeout) return fail(ctx, BICACHE_ERR_TIMEOUT, "device-side wait gave up");
+  return fail(ctx, BICACHE_ERR_CUDA, "a kernel reported an internal error");
 }
 
 #ifdef BICACHE_TRACE
@@ -1207,6 +1215,8 @@ int32_t bicache_set_wait_budget(bicache_ctx* ctx, int64_t sm_cycles) {
 }
 
 int64_t bicache_launch_count(const bicache_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int32_t bicache_last_attention_kernel(const bicache_ctx* ctx) { return ctx ? ctx->last_kernel : 0; }
 
 const char* bicache_last_error(const bicache_ctx* ctx) { return ctx ? ctx->last_error.c_str() : "null context"; }
 

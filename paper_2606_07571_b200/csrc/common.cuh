@@ -68,5 +68,6 @@ __host__ __device__ inline long long pool_slice_offset(const PoolView& p, int la
 // Sticky device status word codes (first error wins).
 constexpr int kDevOk = 0;
 constexpr int kDevTimeout = 5;
+constexpr int kDevInternal = 6;   // a kernel found its own launch state wrong (shared-memory alignment)
 
 }  // namespace bicache

@@ -8,7 +8,7 @@
 //
 // Why a second kernel: with one 128-row tile per CTA the big kernel's chain S -> softmax -> P V
 // runs once per 128 keys with nothing to overlap it, and one CTA per SM cannot keep HBM busy.
-// Here a CTA is small (96 KB of shared memory, 256 TMEM columns: two CTAs per SM), key tiles are
+// Here a CTA is small (112 KB of shared memory, 256 TMEM columns: two CTAs per SM), key tiles are
 // 64 keys, and S is double-buffered in TMEM: S(j+1) = Q K(j+1)^T is issued before the softmax of
 // tile j ends.  Roles: warps 0-3 softmax (one thread per row), warp 4 MMA issue and TMEM, warp 5
 // stages K tiles, warp 6 gathers Q and stages V tiles (cached pages: one 4 KB bulk copy per page,
@@ -26,7 +26,8 @@ using namespace tc;
 constexpr int kKeys = 64;                          // keys per tile
 constexpr int kKvTileBytes = kKeys * 128 * 2;      // 16 KB
 constexpr int kQBytes = 128 * 128 * 2;             // 32 KB
-constexpr int kDecStages = 2;
+constexpr int kKStages = 3;                        // K tiles are consumed one tile early (S is double-buffered)
+constexpr int kVStages = 2;
 constexpr int kDecThreads = 224;
 constexpr int kDecTmemCols = 256;                  // S0 0-63, S1 64-127 (P over the first 32 of each), O 128-255
 // fp32 accumulate, bf16 A and B (both K-major), M = 128, N = 64
@@ -49,8 +50,8 @@ struct DecodeItem {
 
 struct DecSync {
   unsigned long long q_full;
-  unsigned long long k_full[kDecStages], k_free[kDecStages];
-  unsigned long long v_full[kDecStages], v_free[kDecStages];
+  unsigned long long k_full[kKStages], k_free[kKStages];
+  unsigned long long v_full[kVStages], v_free[kVStages];
   unsigned long long s_full[2];          // S of a key tile is in TMEM
   unsigned long long p_full[2];          // P of the tile is in TMEM (and O rescaled if it had to be)
   unsigned long long pv_done;            // O += P V of a tile has completed (one phase per tile)
@@ -61,8 +62,8 @@ struct DecSync {
   unsigned tmem_base;
   int dead;
 };
-constexpr int kDecSmemBytes = 1024 + kQBytes + 2 * kDecStages * kKvTileBytes + (int)sizeof(DecSync);
-static_assert(2 * (kDecSmemBytes + 1024) <= 232448, "two CTAs per SM");
+constexpr int kDecSmemBytes = kQBytes + (kKStages + kVStages) * kKvTileBytes + (int)sizeof(DecSync);
+static_assert(2 * (kDecSmemBytes + 1024) <= 233472, "two CTAs per SM");
 
 }  // namespace dec
 
@@ -70,13 +71,15 @@ __global__ void __launch_bounds__(dec::kDecThreads, 2)
 tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __restrict__ reqs,
                  const int* __restrict__ pages, PoolView pool, TensorArgs t, int* status, long long wait_cycles) {
   using namespace dec;
-  extern __shared__ unsigned char smem_raw[];
-  unsigned char* smem =
-      reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  DecSync* sy = reinterpret_cast<DecSync*>(smem + kQBytes + 2 * kDecStages * kKvTileBytes);
+  // No room for alignment slack with two CTAs per SM: the kernel has no static shared memory, the
+  // dynamic window starts 1024-byte aligned (the swizzled tiles need that), and a CTA that finds
+  // otherwise reports an error instead of computing.
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  unsigned char* const smem = smem_raw;
+  DecSync* sy = reinterpret_cast<DecSync*>(smem + kQBytes + (kKStages + kVStages) * kKvTileBytes);
   volatile int* abort_flag = &sy->abort_flag;
   const unsigned q_smem = smem_u32(smem);
-  const unsigned k_ring = q_smem + kQBytes, v_ring = k_ring + kDecStages * kKvTileBytes;
+  const unsigned k_ring = q_smem + kQBytes, v_ring = k_ring + kKStages * kKvTileBytes;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // the merge kernel that follows may be placed on the SMs from now on (it waits for this grid's end)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -86,12 +89,15 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
 
   if (tid == 0) {
     sy->wait_cycles = wait_cycles;
+    if ((q_smem & 1023u) != 0) atomicCAS(status, kDevOk, kDevInternal);
     sy->dead = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
     sy->abort_flag = (sy->dead || wait_cycles < kStrictBudget) ? 1 : 0;
     mbar_init(smem_u32(&sy->q_full), 32);
-    for (int i = 0; i < kDecStages; ++i) {
+    for (int i = 0; i < kKStages; ++i) {
       mbar_init(smem_u32(&sy->k_full[i]), 32);
       mbar_init(smem_u32(&sy->k_free[i]), 1);
+    }
+    for (int i = 0; i < kVStages; ++i) {
       mbar_init(smem_u32(&sy->v_full[i]), 32);
       mbar_init(smem_u32(&sy->v_free[i]), 1);
     }
@@ -239,16 +245,16 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
       // a K step of 16 dims: 32 bytes inside the swizzled row; dims 64.. sit 1024 bytes further
       auto kstep = [](int k) { return (unsigned long long)((k & 3) * 2 + (k >> 2) * 64); };
       auto issue_s = [&](int j) {
-        const int b = j & 1;
-        bool good = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->k_full[b]), (j >> 1) & 1, abort_flag));
+        const int b = j & 1, ks = j % kKStages;
+        bool good = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->k_full[ks]), (j / kKStages) & 1, abort_flag));
         if (!good) return false;
         tc_fence_after();
-        const unsigned long long k_desc = make_desc(k_ring + b * kKvTileBytes, 16, 2048);
+        const unsigned long long k_desc = make_desc(k_ring + ks * kKvTileBytes, 16, 2048);
 #pragma unroll
         for (int k = 0; k < 8; ++k)
           mma_ss_elect(tmem + b * 64, q_desc + kstep(k), k_desc + kstep(k), kIdescS64, k > 0 ? 1u : 0u);
         mma_commit_elect(smem_u32(&sy->s_full[b]));
-        mma_commit_elect(smem_u32(&sy->k_free[b]));
+        mma_commit_elect(smem_u32(&sy->k_free[ks]));
         return true;
       };
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->q_full), 0, abort_flag));
@@ -289,7 +295,8 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     const int is_v = warp - 5;
     const int r0 = lane >> 4, c16 = lane & 15;
     bool ok = !dead;
-    int armed[kDecStages] = {-1, -1};        // the last tile armed with bulk copies, per stage
+    const int stages = is_v ? kVStages : kKStages;
+    int armed[kKStages] = {-1, -1, -1};      // the last tile armed with bulk copies, per stage
     if (ok && is_v && T > 0) {
       // Packed row p = token a * G + head jj of the KV group; rows past the end are zero-filled.
       // Token a of the row space is token tok_off + a of the call: the request that holds it is
@@ -319,10 +326,10 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     }
     const unsigned ring = is_v ? v_ring : k_ring;
     for (int j = 0; j < T && ok; ++j) {
-      const int b = j & 1;
+      const int b = j % stages;
       const unsigned free_bar = smem_u32(is_v ? &sy->v_free[b] : &sy->k_free[b]);
       const unsigned full = smem_u32(is_v ? &sy->v_full[b] : &sy->k_full[b]);
-      ok = __all_sync(0xffffffffu, mbar_wait(free_bar, ((j >> 1) & 1) ^ 1, abort_flag));
+      ok = __all_sync(0xffffffffu, mbar_wait(free_bar, ((j / stages) & 1) ^ 1, abort_flag));
       if (!ok) break;
       const unsigned dst = ring + b * kKvTileBytes;
       const int key0 = it.key_begin + j * kKeys;
@@ -366,10 +373,10 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     cp_async_wait<0>();
     // After a give-up, bulk copies may still be in flight: wait (bounded) for the barriers armed last.
     if (!dead && (!ok || *abort_flag) && lane == 0) {
-      for (int b = 0; b < kDecStages; ++b)
+      for (int b = 0; b < stages; ++b)
         if (armed[b] >= 0) {
           const unsigned full = smem_u32(is_v ? &sy->v_full[b] : &sy->k_full[b]);
-          for (unsigned n = 0; n < 4096 && !mbar_try_wait(full, (armed[b] >> 1) & 1); ++n) __nanosleep(256);
+          for (unsigned n = 0; n < 4096 && !mbar_try_wait(full, (armed[b] / stages) & 1); ++n) __nanosleep(256);
         }
     }
   }

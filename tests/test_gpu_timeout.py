@@ -72,3 +72,36 @@ def test_projection_tiny_wait_budget_reports_timeout_and_context_recovers():
     for got, ref in ((gk, rk[0]), (gv, rv[0])):
         assert np.all(np.abs(workloads.to_f64(got) - ref) <= np.abs(ref) * 2.0 ** -8 + 1e-3)
     bc.close()
+
+
+def test_key_range_kernel_tiny_wait_budget_reports_timeout_and_context_recovers():
+    """The same for the kernel that serves few query rows against a long cached prefix."""
+    Hq, Hkv, D, m, n = 4, 2, 128, 2000, [7, 12]
+    w = workloads.Workload("kr-timeout", 1, Hq, Hkv, D, torch.bfloat16, 16, [m], [0, 0], n, softmax_scale=D ** -0.5)
+    bc = binding.BiCache(1, Hq, Hkv, D, w.pages_needed() + 1, torch.bfloat16, w.total_rows, 2)
+    st = oracle.PagedPrefixStore(1, Hkv, D, 16, w.pages_needed() + 1)
+    kc, vc = workloads.draw_prefix_kv(w, 0, "cuda")
+    pid = bc.put_prefix(1, kc, vc)[0]
+    opid = st.put(1, workloads.to_f64(kc), workloads.to_f64(vc))[0]
+    q, k, v = workloads.draw_full_qkv(w, "cuda")
+    out = torch.zeros_like(q)
+    args = (0, [pid, pid], w.suffix_row_off, w.suffix_lens, q, k, v, out, None, w.softmax_scale)
+    bc.set_wait_budget(1)
+    bc.attend(*args)
+    assert bc.last_attention_kernel() == binding.KERNEL_KEY_RANGES
+    assert bc.device_status() == binding.ERR_TIMEOUT
+    bc.attend(*args)                                        # a launch on a flagged context does no work
+    assert bc.device_status(clear=True) == binding.ERR_TIMEOUT
+    assert bc.device_status() == binding.OK
+    bc.set_wait_budget(0)
+    out.zero_()
+    bc.attend(*args)
+    assert bc.device_status() == binding.OK
+    ref, _ = oracle.attend(st, 0, [opid, opid], w.suffix_row_off, w.suffix_lens,
+                           *(workloads.to_f64(x) for x in (q, k, v)), w.softmax_scale)
+    mask = np.zeros(w.total_rows, dtype=bool)
+    for o, nn in zip(w.suffix_row_off, w.suffix_lens):
+        mask[o:o + nn] = True
+    err = np.abs(workloads.to_f64(out)[mask] - ref[mask])
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3
+    bc.close()
