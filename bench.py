@@ -180,10 +180,13 @@ class Job:
 
 
 def time_call(fn, iters, flush):
-    """Average device time of fn() over `iters` runs, each preceded by an L2 flush (untimed)."""
+    """Average device time of fn() over `iters` runs, each preceded by an L2 flush (untimed): the
+    256 MB buffer is written, then read back, so that the timed kernel starts with an L2 full of
+    foreign but CLEAN lines and does not pay for writing the flusher's dirty lines back."""
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
     for a, b in ev:
         flush.zero_()
+        flush.max()
         a.record()
         fn()
         b.record()
@@ -399,6 +402,15 @@ def main():
                        "peak": peak, "unit": "TFLOP/s", "frac": tf_attend / peak,
                        "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("attend"),
                        "flops_per_launch": w.attend_flops(), "ms_per_launch": ms_attend}
+    call_attend()
+    if bc.last_attention_kernel() == 3:                    # the key-range kernel (BICACHE_KERNEL_KEY_RANGES)
+        # few query rows against a long cached prefix: the launch is bound by reading the prefix once
+        gbs = w.attend_bytes() / (ms_attend * 1e-3) / 1e9
+        roofline_attend = {"bound": "hbm", "kernel": "tc_decode_kernel + merge_ranges_kernel (attend call)",
+                           "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                           "peak_source": peaks["source"], "bytes_per_launch": w.attend_bytes(),
+                           "ms_per_launch": ms_attend, "tflops": tf_attend,
+                           "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("attend")}
 
     # ---- end to end: host buffers, copies inside the timed region ------------------------------
     e2e = None

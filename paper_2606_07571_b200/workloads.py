@@ -91,6 +91,15 @@ class Workload:
         return 4 * self.head_dim * self.num_q_heads * sum(
             n * (self.prefix_lens[g] + n) for g, n in zip(self.req_prefix, self.suffix_lens))
 
+    def attend_bytes(self):
+        """Algorithmic bytes of one `attend` launch: every group's cached K and V once, every
+        request's suffix Q, K, V read and output written once."""
+        e = 2 if self.dtype == torch.bfloat16 else 4
+        groups = sorted(set(self.req_prefix))
+        b = sum(2 * self.prefix_lens[g] * self.num_kv_heads * self.head_dim * e for g in groups)
+        b += sum(2 * n * (self.num_q_heads + self.num_kv_heads) * self.head_dim * e for n in self.suffix_lens)
+        return b
+
     def full_flops(self):
         """Algorithmic FLOPs of one deep layer with every request recomputing."""
         return 4 * self.head_dim * self.num_q_heads * sum(N * N for N in self.full_lens)
