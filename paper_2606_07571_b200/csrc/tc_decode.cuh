@@ -306,18 +306,25 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
       int kreq = it.req_first;
       const int kreq_end = it.req_first + it.req_count;
       ReqMeta rq = reqs[kreq];
-#pragma unroll 2
+      // this lane's rows are it.row0 + r0 + 2 i: token a and head jj advance without divisions
+      int prow = it.row0 + r0;
+      int a = prow / G, jj = prow - a * G;
+#pragma unroll 4
       for (int i = 0; i < 64; ++i) {
-        const int prow = it.row0 + r0 + 2 * i;
         const bool valid = prow < packed_rows;
         const char* src = q_head;
         if (valid) {
-          const int a = prow / G, jj = prow - a * G;
           const int tg = it.tok_off + a;
           while (tg >= rq.tok_off + rq.n && kreq + 1 < kreq_end) rq = reqs[++kreq];
           src = q_head + ((rq.row_off + (tg - rq.tok_off)) * t.q_stride + jj * 128) * 2;
         }
         cp_async16(q_smem + tile_chunk_offset(r0 + 2 * i, c16), src, valid ? 16u : 0u);
+        prow += 2;
+        jj += 2;
+        while (jj >= G) {                           // at most twice (G >= 1)
+          jj -= G;
+          ++a;
+        }
       }
       cp_async_commit();
       cp_async_wait<0>();
