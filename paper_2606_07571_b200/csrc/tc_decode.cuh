@@ -11,7 +11,7 @@
 // Here a CTA is small (112 KB of shared memory, 256 TMEM columns: two CTAs per SM), key tiles are
 // 64 keys, and S is double-buffered in TMEM: S(j+1) = Q K(j+1)^T is issued before the softmax of
 // tile j ends.  Roles: warps 0-3 softmax (one thread per row), warp 4 MMA issue and TMEM, warp 5
-// stages K tiles, warp 6 gathers Q and stages V tiles (cached pages: one 4 KB bulk copy per page,
+// stages K tiles, warp 6 stages V tiles (the softmax warps gather Q before their first tile) (cached pages: one 4 KB bulk copy per page,
 // a pool page already is the operand image; own rows: 16-byte gathers into the same image).
 // Every wait is bounded, as in the big kernel.
 #pragma once
@@ -64,6 +64,20 @@ struct DecSync {
 };
 constexpr int kDecSmemBytes = kQBytes + (kKStages + kVStages) * kKvTileBytes + (int)sizeof(DecSync);
 static_assert(2 * (kDecSmemBytes + 1024) <= 233472, "two CTAs per SM");
+static_assert(128 * 528 <= (kKStages + kVStages) * kKvTileBytes, "the partial rows are staged over the K/V rings");
+
+#ifdef BICACHE_DEC_TRACE
+// Debug build only: nanosecond stamps of one CTA (slot = role event).
+__device__ unsigned long long g_dec_trace[64];
+__device__ __forceinline__ unsigned long long dec_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+#define DEC_STAMP(slot) do { if (blockIdx.x == BICACHE_DEC_TRACE) g_dec_trace[slot] = dec_now(); } while (0)
+#else
+#define DEC_STAMP(slot) do { } while (0)
+#endif
 
 }  // namespace dec
 
@@ -83,6 +97,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // the merge kernel that follows may be placed on the SMs from now on (it waits for this grid's end)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (threadIdx.x == 0) DEC_STAMP(0);
   const DecodeItem it = items[blockIdx.x];
   const int G = t.Hq / t.Hkv;
   const int T = (it.key_count + kKeys - 1) / kKeys;
@@ -92,7 +107,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     if ((q_smem & 1023u) != 0) atomicCAS(status, kDevOk, kDevInternal);
     sy->dead = (*reinterpret_cast<volatile int*>(status) != 0) ? 1 : 0;
     sy->abort_flag = (sy->dead || wait_cycles < kStrictBudget) ? 1 : 0;
-    mbar_init(smem_u32(&sy->q_full), 32);
+    mbar_init(smem_u32(&sy->q_full), 128);
     for (int i = 0; i < kKStages; ++i) {
       mbar_init(smem_u32(&sy->k_full[i]), 32);
       mbar_init(smem_u32(&sy->k_free[i]), 1);
@@ -120,6 +135,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&sy->tmem_base);
   const bool dead = *reinterpret_cast<volatile int*>(&sy->dead) != 0;
   const unsigned tmem_o = tmem + 128;
+  if (tid == 0) DEC_STAMP(1);
 
   if (warp < 4) {
     // ================================ softmax and epilogue =================================
@@ -128,12 +144,51 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     const float sl2 = t.scale * 1.4426950408889634f;         // scores are handled in the log2 domain
     float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = !dead;
+    if (ok && T > 0) {
+      // The Q tile, gathered by the 128 threads that have nothing else to do yet (one warp alone
+      // needs 5 us for its 64 passes): warp w fetches rows 32 w .. 32 w + 31, lane l the 16-byte chunk
+      // (l & 15) of rows 32 w + (l >> 4) + 2 i.  Packed row p = token a * G + head jj of the KV
+      // group; rows past the end are zero-filled.  Token a of the row space is token tok_off + a of
+      // the call: the request that holds it is found by walking the space's requests (a only grows
+      // along a lane's rows).
+      const int r0 = warp * 32 + (lane >> 4), c16 = lane & 15;
+      const int packed_rows = it.n * G;
+      const char* const q_head = t.q + ((long long)it.kv_head * G * 128) * 2 + c16 * 16;
+      int kreq = it.req_first;
+      const int kreq_end = it.req_first + it.req_count;
+      ReqMeta rq = reqs[kreq];
+      int prow = it.row0 + r0;
+      int a = prow / G, jj = prow - a * G;
+#pragma unroll 4
+      for (int i = 0; i < 16; ++i) {
+        const bool valid = prow < packed_rows;
+        const char* src = q_head;
+        if (valid) {
+          const int tg = it.tok_off + a;
+          while (tg >= rq.tok_off + rq.n && kreq + 1 < kreq_end) rq = reqs[++kreq];
+          src = q_head + ((rq.row_off + (tg - rq.tok_off)) * t.q_stride + jj * 128) * 2;
+        }
+        cp_async16(q_smem + tile_chunk_offset(r0 + 2 * i, c16), src, valid ? 16u : 0u);
+        prow += 2;
+        jj += 2;
+        while (jj >= G) {                           // at most twice (G >= 1)
+          jj -= G;
+          ++a;
+        }
+      }
+      cp_async_commit();
+      if (tid == 0) DEC_STAMP(6);
+      cp_async_wait<0>();
+      fence_proxy_async();
+      mbar_arrive(smem_u32(&sy->q_full));
+    }
     for (int j = 0; j < T && ok; ++j) {
       const int b = j & 1;
       const int cnt = min(kKeys, it.key_count - j * kKeys);
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->s_full[b]), (j >> 1) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
+      if (tid == 0 && j < 8) DEC_STAMP(10 + j);
       unsigned r[64];
       tmem_ld32(tmem + b * 64 + lane_base, r);
       tmem_ld32(tmem + b * 64 + 32 + lane_base, r + 32);
@@ -196,6 +251,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(smem_u32(&sy->p_full[b]));
+      if (tid == 0 && j < 8) DEC_STAMP(20 + j);
       float s0, s1, s2, s3;
       unpack2(acc_a, s0, s1);
       unpack2(acc_b, s2, s3);
@@ -212,22 +268,34 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->o_done), 0, abort_flag));
         if (ok) {
           tc_fence_after();
+          if (tid == 0) DEC_STAMP(2);
+          // Each thread holds one row of the partial (128 fp32 = 512 bytes, contiguous in the
+          // workspace).  Written from registers, a warp's stores would touch 32 rows at a time; so
+          // the row goes to shared memory first (the K/V rings are free by now: every tile has been
+          // consumed; rows 528 bytes apart keep the 16-byte stores conflict-free) and leaves as one
+          // 512-byte bulk copy per row.
           const float inv = 1.f / l_sum;
+          unsigned char* const stage_row = smem + kQBytes + row * 528;
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
             unsigned o[32];
             tmem_ld32(tmem_o + c * 32 + lane_base, o);
             tmem_wait_ld();
-            if (row_valid) {
-              float* po = t.part_o + pr * 128 + c * 32;
 #pragma unroll
-              for (int i = 0; i < 32; i += 4)
-                *reinterpret_cast<float4*>(po + i) =
-                    make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv,
-                                __uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
-            }
+            for (int i = 0; i < 32; i += 4)
+              *reinterpret_cast<float4*>(stage_row + (c * 32 + i) * 4) =
+                  make_float4(__uint_as_float(o[i]) * inv, __uint_as_float(o[i + 1]) * inv,
+                              __uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
           }
-          if (row_valid) t.part_lse[pr] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+          fence_proxy_async();
+          if (row_valid) {
+            asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], 512;"
+                         ::"l"(t.part_o + pr * 128), "r"(smem_u32(stage_row)) : "memory");
+            bulk_commit_group();
+            t.part_lse[pr] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
+            bulk_wait_all();
+          }
+          if (tid == 0) DEC_STAMP(3);
         }
       } else if (row_valid) {
         float* po = t.part_o + pr * 128;
@@ -258,7 +326,9 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
         return true;
       };
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->q_full), 0, abort_flag));
+      if (lane == 0) DEC_STAMP(4);
       if (ok) ok = issue_s(0);
+      if (lane == 0) DEC_STAMP(5);
       for (int j = 0; j < T && ok; ++j) {
         const int b = j & 1;
         if (j + 1 < T) {
@@ -290,47 +360,12 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     __syncwarp();
   } else {
     // ======================================= loads ========================================
-    // Warp 5 stages the K tiles; warp 6 gathers the Q tile (needed together with the first K tile,
-    // so the two loads overlap), then stages the V tiles.
+    // Warp 5 stages the K tiles, warp 6 the V tiles.
     const int is_v = warp - 5;
     const int r0 = lane >> 4, c16 = lane & 15;
     bool ok = !dead;
     const int stages = is_v ? kVStages : kKStages;
     int armed[kKStages] = {-1, -1, -1};      // the last tile armed with bulk copies, per stage
-    if (ok && is_v && T > 0) {
-      // Packed row p = token a * G + head jj of the KV group; rows past the end are zero-filled.
-      // Token a of the row space is token tok_off + a of the call: the request that holds it is
-      // found by walking the space's requests (a only grows along a lane's rows).
-      const int packed_rows = it.n * G;
-      const char* const q_head = t.q + ((long long)it.kv_head * G * 128) * 2 + c16 * 16;
-      int kreq = it.req_first;
-      const int kreq_end = it.req_first + it.req_count;
-      ReqMeta rq = reqs[kreq];
-      // this lane's rows are it.row0 + r0 + 2 i: token a and head jj advance without divisions
-      int prow = it.row0 + r0;
-      int a = prow / G, jj = prow - a * G;
-#pragma unroll 4
-      for (int i = 0; i < 64; ++i) {
-        const bool valid = prow < packed_rows;
-        const char* src = q_head;
-        if (valid) {
-          const int tg = it.tok_off + a;
-          while (tg >= rq.tok_off + rq.n && kreq + 1 < kreq_end) rq = reqs[++kreq];
-          src = q_head + ((rq.row_off + (tg - rq.tok_off)) * t.q_stride + jj * 128) * 2;
-        }
-        cp_async16(q_smem + tile_chunk_offset(r0 + 2 * i, c16), src, valid ? 16u : 0u);
-        prow += 2;
-        jj += 2;
-        while (jj >= G) {                           // at most twice (G >= 1)
-          jj -= G;
-          ++a;
-        }
-      }
-      cp_async_commit();
-      cp_async_wait<0>();
-      fence_proxy_async();
-      mbar_arrive(smem_u32(&sy->q_full));
-    }
     const unsigned ring = is_v ? v_ring : k_ring;
     for (int j = 0; j < T && ok; ++j) {
       const int b = j % stages;
@@ -354,6 +389,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
         }
         // every lane arrives, so the phase cannot complete before lane 0 has announced the bytes
         if (lane == 0) {
+          if (!is_v && j == 0) DEC_STAMP(7);
           mbar_arrive_expect_tx(full, (unsigned)(npages * kPageBytes));
           armed[b] = j;
         } else {
@@ -394,6 +430,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     tmem_dealloc(tmem, kDecTmemCols);
   }
   if (tid == 0 && !dead && *abort_flag) atomicCAS(status, kDevOk, kDevTimeout);
+  if (tid == 0) DEC_STAMP(8);
 }
 
 // ---------------------------------------------------------------------------------------------
