@@ -342,8 +342,8 @@ int64_t bicache_launch_count(const bicache_ctx* ctx);
  * 0 none yet; BICACHE_KERNEL_SIMT the CUDA-core kernel (fp32, head dims other than 128, forced);
  * BICACHE_KERNEL_TENSOR the tensor-core kernel over two 128-row query tiles per work item;
  * BICACHE_KERNEL_KEY_RANGES the tensor-core kernel for few query rows against a long cached prefix
- * (bicache_attend only; chosen when every request has a cached prefix of at least 1024 tokens and the
- * suffix rows of each prefix group, all requests together, times Hq / Hkv are at most 256): the group's
+ * (bicache_attend only; chosen when every request has a cached prefix of at least 1024 tokens and at
+ * most 128 * Hkv / Hq suffix tokens, and the call is small enough for the kernel's tables): the group's
  * rows share tiles, the prefix keys are split into ranges over the CTAs, each request's own keys are
  * one more range, and a merge kernel applies the log-sum-exp merge (exact up to rounding). */
 enum { BICACHE_KERNEL_SIMT = 1, BICACHE_KERNEL_TENSOR = 2, BICACHE_KERNEL_KEY_RANGES = 3 };

@@ -55,7 +55,7 @@ struct CachedSchedule {
   size_t tok_rows_off = 0;                    // kind 2: row of every token of the call
   int num_ditems = 0;
 };
-constexpr int kMaxDecodeItems = 1024;
+constexpr int kMaxDecodeItems = 4096;
 constexpr int kMaxDecodeTokens = 4096;        // tokens of a call served by the key-range kernel
 
 }  // namespace
@@ -273,6 +273,10 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
     sp = std::min(sp, std::max(1, tiles64_max / 4));
     sp = std::min(sp, 63);
     while (sp > 1 && tok * ctx->cfg.num_q_heads * (sp + 1) > ctx->part_capacity_rowheads) --sp;
+    if (tok * ctx->cfg.num_q_heads * (sp + 1) > ctx->part_capacity_rowheads) {
+      *status = fail(ctx, BICACHE_ERR_NOMEM, "the partial results of this batch do not fit the workspace");
+      return -1;                                          // the caller falls back to the general kernel
+    }
     for (const Group& g : groups) {
       if (g.n <= 0) continue;
       const ReqMeta& r0m = reqs[g.first];
@@ -430,19 +434,17 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   const bool use_tensor = ctx->tensor_ok && ctx->path != BICACHE_PATH_SIMT && softmax_scale > 0.f;
   // Few query rows per prefix group against a long cached prefix (block-query decoding): the
   // bandwidth-bound regime, served by the key-range kernel.  Conditions: every request has a cached
-  // prefix of at least 1024 tokens and the rows of a group's requests pack into at most two
-  // 128-row tiles per KV head.
+  // prefix of at least 1024 tokens and at most 128 packed rows per KV head (a request with more fills
+  // the general kernel's tiles by itself), and the call's tokens fit the kernel's tables.
   bool key_ranges = kind == 0 && use_tensor;
   if (key_ranges) {
     const int G = cfg.num_q_heads / cfg.num_kv_heads;
-    long long group_rows = 0;
     for (int i = 0; i < R && key_ranges; ++i) {
       if (prefix_id[i] < 0) { key_ranges = false; break; }
-      if (i == 0 || prefix_id[i] != prefix_id[i - 1]) group_rows = 0;
       if (ctx->by_id.at(prefix_id[i])->m < 1024) key_ranges = false;
-      group_rows += seqlen[i];
-      if (group_rows * G > 256) key_ranges = false;
+      if ((long long)seqlen[i] * G > 128) key_ranges = false;
     }
+    if (total > kMaxDecodeTokens) key_ranges = false;
   }
   int st = BICACHE_OK;
   int slot = -1;

@@ -86,9 +86,15 @@ def test_subset_of_requests_and_peaked_scores():
 
 
 def test_outside_the_regime_the_general_kernel_runs():
-    """A short prefix, or too many rows per group, keeps the general tensor-core kernel."""
+    """A short prefix, or a request with more than 128 packed rows, keeps the general tensor-core kernel."""
     _run(4, 2, [700], [0, 0], [10, 10], expect=binding.KERNEL_TENSOR)
     _run(2, 2, [1100], [0, 0], [200, 100], expect=binding.KERNEL_TENSOR)
+
+
+def test_group_of_many_short_requests_several_row_tiles():
+    """Seven requests of up to 100 tokens in one group: 470 packed rows per KV head = four row tiles
+    per key range, requests straddling the tile boundaries; a second group of one request."""
+    _run(4, 4, [1400, 1100], [0, 0, 0, 0, 0, 0, 0, 1], [100, 64, 1, 90, 15, 100, 100, 128], shuffle=True)
 
 
 @pytest.mark.parametrize("seed", [0, 1, 2, 3, 4, 5])
@@ -100,13 +106,9 @@ def test_seeded_random_shapes(seed):
     prefix_lens = [int(rng.integers(1024, 2600)) for _ in range(groups)]
     req_prefix, suffix_lens = [], []
     for g in range(groups):
-        budget = 256 // G                                   # tokens of a group: at most 256 packed rows
-        for _ in range(int(rng.integers(1, 5))):
-            n = int(rng.integers(0, max(1, budget // 2) + 1))
-            n = min(n, budget)
-            budget -= n
+        for _ in range(int(rng.integers(1, 7))):
             req_prefix.append(g)
-            suffix_lens.append(n)
+            suffix_lens.append(int(rng.integers(0, 128 // G + 1)))   # a request: at most 128 packed rows
     if sum(suffix_lens) == 0:
         suffix_lens[0] = 1
     _run(Hkv * G, Hkv, prefix_lens, req_prefix, suffix_lens, shuffle=bool(rng.integers(0, 2)))
