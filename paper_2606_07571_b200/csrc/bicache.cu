@@ -53,6 +53,7 @@ struct CachedSchedule {
   size_t reqs_off = 0, pages_off = 0, items_off = 0;   // byte offsets inside the slot
   size_t ditems_off = 0;                      // kind 2: the key-range items
   size_t tok_rows_off = 0;                    // kind 2: row of every token of the call
+  size_t tok_span_off = 0;                    // kind 2: the tokens of every token's own request
   int num_ditems = 0;
 };
 constexpr int kMaxDecodeItems = 4096;
@@ -121,7 +122,8 @@ size_t slot_bytes_for(const bicache_config* c, int64_t max_rows, int32_t max_req
          align_up((size_t)c->num_pages * sizeof(int) + 16, 256) +
          align_up((size_t)max_items * sizeof(WorkItem) + 16, 256) +
          align_up((size_t)kMaxDecodeItems * sizeof(dec::DecodeItem) + 16, 256) +
-         align_up((size_t)kMaxDecodeTokens * sizeof(long long) + 16, 256);
+         align_up((size_t)kMaxDecodeTokens * sizeof(long long) + 16, 256) +
+         align_up((size_t)kMaxDecodeTokens * sizeof(int2) + 16, 256);
 }
 
 size_t partial_bytes_for(const bicache_config* c) {
@@ -246,8 +248,9 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   std::vector<WorkItem> items;
   std::vector<dec::DecodeItem> ditems;
   if (kind == 2) {
-    // Key-range kernel (few query rows against long cached prefixes).  Row space of the prefix ranges:
-    // all requests of a prefix group, their tokens concatenated; of the own-key range: each request.  Ranges 0 .. sp-1 split the prefix keys, range sp holds the own keys.
+    // Key-range kernel (few query rows against long cached prefixes).  Row space: all requests of a
+    // prefix group, their tokens concatenated.  Ranges 0 .. sp-1 split the prefix keys; the CTAs of
+    // range 0 also cover the own keys of the requests that have rows in their row tile.
     struct Group { int first, last; int n, tok_off; };
     std::vector<Group> groups;
     for (int i = 0; i < R; ++i) {
@@ -264,16 +267,12 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
       base_items += (long long)((g.n * (long long)G + 127) / 128) * Hkv;
       tiles64_max = std::max(tiles64_max, (reqs[g.first].m + 63) / 64);
     }
-    // ranges per prefix: what fills the two CTA slots of every SM once, next to the own-key CTAs
-    long long own_items = 0;
-    for (int i = 0; i < R; ++i)
-      if (reqs[i].n > 0) own_items += (long long)((reqs[i].n * (long long)G + 127) / 128) * Hkv;
-    const long long slots_left = std::max<long long>(2LL * ctx->sm_count - own_items, ctx->sm_count);
-    int sp = (int)std::max<long long>(1, slots_left / std::max<long long>(1, base_items));
+    // ranges per prefix: what fills the two CTA slots of every SM once, at least 4 key tiles each
+    int sp = (int)std::max<long long>(1, 2LL * ctx->sm_count / std::max<long long>(1, base_items));
     sp = std::min(sp, std::max(1, tiles64_max / 4));
-    sp = std::min(sp, 63);
-    while (sp > 1 && tok * ctx->cfg.num_q_heads * (sp + 1) > ctx->part_capacity_rowheads) --sp;
-    if (tok * ctx->cfg.num_q_heads * (sp + 1) > ctx->part_capacity_rowheads) {
+    sp = std::min(sp, 64);
+    while (sp > 1 && tok * ctx->cfg.num_q_heads * sp > ctx->part_capacity_rowheads) --sp;
+    if (tok * ctx->cfg.num_q_heads * sp > ctx->part_capacity_rowheads) {
       *status = fail(ctx, BICACHE_ERR_NOMEM, "the partial results of this batch do not fit the workspace");
       return -1;                                          // the caller falls back to the general kernel
     }
@@ -285,25 +284,31 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
         const int kb = s * tps * 64;
         const int kc = std::max(0, std::min(r0m.m - kb, tps * 64));
         for (int hk = 0; hk < Hkv; ++hk)
-          for (int r0 = 0; r0 < g.n * G; r0 += 128)
-            ditems.push_back(dec::DecodeItem{0, g.first, g.last - g.first + 1, g.n, g.tok_off, hk, r0, 0,
-                                             kc > 0 ? kb : 0, kc, r0m.page_off, s});
+          for (int r0 = 0; r0 < g.n * G; r0 += 128) {
+            int own_begin = 0, own_count = 0;
+            if (s == 0) {
+              // the requests that own tokens r0 / G .. (last row of the tile) / G of the group
+              const int a_first = r0 / G, a_last = (std::min(r0 + 128, g.n * G) - 1) / G;
+              int lo = -1, hi = -1;
+              for (int i = g.first; i <= g.last; ++i) {
+                const int b0 = reqs[i].tok_off - g.tok_off, b1 = b0 + reqs[i].n;
+                if (reqs[i].n <= 0 || b1 <= a_first || b0 > a_last) continue;
+                if (lo < 0) lo = b0;
+                hi = b1;
+              }
+              own_begin = lo;
+              own_count = hi - lo;
+            }
+            ditems.push_back(dec::DecodeItem{g.n, g.tok_off, hk, r0, kc > 0 ? kb : 0, kc, r0m.page_off, s, own_begin,
+                                             own_count});
+          }
       }
     }
-    // long prefix ranges first
-    std::stable_sort(ditems.begin(), ditems.end(),
-                     [](const dec::DecodeItem& a, const dec::DecodeItem& b) { return a.key_count > b.key_count; });
-    // The own-key ranges (one short tile or two each) go in front of everything: they leave their
-    // SM slots within a few microseconds, whereas at the end they would be a round of their own.
-    std::vector<dec::DecodeItem> own;
-    for (int i = 0; i < R; ++i) {
-      if (reqs[i].n <= 0) continue;
-      for (int hk = 0; hk < Hkv; ++hk)
-        for (int r0 = 0; r0 < reqs[i].n * G; r0 += 128)
-          own.push_back(dec::DecodeItem{reqs[i].row_off, i, 1, reqs[i].n, reqs[i].tok_off, hk, r0, 1, 0, reqs[i].n, 0, sp});
-    }
-    ditems.insert(ditems.begin(), own.begin(), own.end());
-    num_splits = sp + 1;                                   // what the merge kernel combines
+    // long ranges first
+    std::stable_sort(ditems.begin(), ditems.end(), [](const dec::DecodeItem& a, const dec::DecodeItem& b) {
+      return a.key_count + a.own_count > b.key_count + b.own_count;
+    });
+    num_splits = sp;                                       // what the merge kernel combines
     tiles_per_split = 0;
   }
   items.reserve((size_t)unsplit_items * num_splits);
@@ -327,13 +332,19 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   const size_t items_off = align_up(pages_off + pages.size() * sizeof(int) + 16, 256);
   const size_t ditems_off = align_up(items_off + items.size() * sizeof(WorkItem) + 16, 256);
   std::vector<long long> tok_rows;
+  std::vector<int2> tok_span;                              // per token: the call's tokens of its own request
   if (kind == 2) {
     tok_rows.reserve((size_t)tok);
+    tok_span.reserve((size_t)tok);
     for (int i = 0; i < R; ++i)
-      for (int a = 0; a < reqs[i].n; ++a) tok_rows.push_back(reqs[i].row_off + a);
+      for (int a = 0; a < reqs[i].n; ++a) {
+        tok_rows.push_back(reqs[i].row_off + a);
+        tok_span.push_back(make_int2(reqs[i].tok_off, reqs[i].tok_off + reqs[i].n));
+      }
   }
   const size_t tok_rows_off = align_up(ditems_off + ditems.size() * sizeof(dec::DecodeItem) + 16, 256);
-  const size_t total = tok_rows_off + tok_rows.size() * sizeof(long long);
+  const size_t tok_span_off = align_up(tok_rows_off + tok_rows.size() * sizeof(long long) + 16, 256);
+  const size_t total = tok_span_off + tok_span.size() * sizeof(int2);
   if (total > ctx->slot_bytes || (int)ditems.size() > kMaxDecodeItems || (long long)tok_rows.size() > kMaxDecodeTokens) {
     *status = fail(ctx, BICACHE_ERR_NOMEM, "workspace too small for this batch's schedule");
     return -1;
@@ -349,6 +360,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   if (!items.empty()) std::memcpy(blob.data() + items_off, items.data(), items.size() * sizeof(WorkItem));
   if (!ditems.empty()) std::memcpy(blob.data() + ditems_off, ditems.data(), ditems.size() * sizeof(dec::DecodeItem));
   if (!tok_rows.empty()) std::memcpy(blob.data() + tok_rows_off, tok_rows.data(), tok_rows.size() * sizeof(long long));
+  if (!tok_span.empty()) std::memcpy(blob.data() + tok_span_off, tok_span.data(), tok_span.size() * sizeof(int2));
   CachedSchedule& c = ctx->slots[victim];
   c.valid = false;
   if (total > 0) {
@@ -367,6 +379,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   c.num_items = (int)items.size() * (kind == 2 ? num_splits : 1);   // kind 2 stores the first range's items only
   c.ditems_off = ditems_off;
   c.tok_rows_off = tok_rows_off;
+  c.tok_span_off = tok_span_off;
   c.num_ditems = (int)ditems.size();
   c.num_splits = num_splits;
   c.tiles_per_split = tiles_per_split;
@@ -489,8 +502,10 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   cudaError_t e;
   ctx->last_kernel = key_ranges ? BICACHE_KERNEL_KEY_RANGES : use_tensor ? BICACHE_KERNEL_TENSOR : BICACHE_KERNEL_SIMT;
   if (key_ranges) {
-    e = launch_tc_decode(reinterpret_cast<const dec::DecodeItem*>(base + c.ditems_off), c.num_ditems, sv.reqs,
-                         sv.pages, pool, t, ctx->d_status, ctx->wait_cycles, stream);
+    e = launch_tc_decode(reinterpret_cast<const dec::DecodeItem*>(base + c.ditems_off), c.num_ditems,
+                         reinterpret_cast<const long long*>(base + c.tok_rows_off),
+                         reinterpret_cast<const int2*>(base + c.tok_span_off), sv.pages, pool, t, ctx->d_status,
+                         ctx->wait_cycles, stream);
   } else if (use_tensor) {
     // rows the tensors are known to have: up to the end of the last request
     long long rows_total = 0;

@@ -2,9 +2,11 @@
 // Eq. 2 / Eq. 4.  One CTA computes, for up to 128 packed query rows of one KV head and one RANGE of
 // keys, the normalised partial result and its log-sum-exp; a merge kernel combines the ranges
 // (the identity behind the log-sum-exp merge: softmax over a union of key sets).  The query rows of
-// ALL requests of a prefix group sit in one tile when their rows are adjacent in memory, so the
-// cached prefix is read once per group, not once per request; each request's own keys are one
-// more range, handled by CTAs of the same launch.
+// ALL requests of a prefix group share tiles (token t of the group is row tok_rows[t] of q), so the
+// cached prefix is read once per group, not once per request.  The requests' own keys ride along
+// with the first range: after its prefix tiles that CTA runs over the own rows of the requests in its
+// row tile, every query row masked to the keys of its own request (a block-diagonal mask: Eq. 2
+// per request).
 //
 // Why a second kernel: with one 128-row tile per CTA the big kernel's chain S -> softmax -> P V
 // runs once per 128 keys with nothing to overlap it, and one CTA per SM cannot keep HBM busy.
@@ -34,18 +36,16 @@ constexpr int kDecTmemCols = 256;                  // S0 0-63, S1 64-127 (P over
 constexpr unsigned kIdescS64 = (1u << 4) | (1u << 7) | (1u << 10) | ((64u >> 3) << 17) | ((128u >> 4) << 24);
 
 struct DecodeItem {
-  long long row_off;     // kind 1: first row of the request (its own keys are rows row_off .. + n - 1 of k / v)
-  int req_first;         // the row space: requests req_first .. req_first + req_count - 1 of the call, their
-  int req_count;         // tokens concatenated (a request, or all requests of a prefix group)
-  int n;                 // tokens in the row space
-  int tok_off;           // index of the row space's first token among the call's tokens (partials)
+  int n;                 // tokens in the row space: all requests of a prefix group, concatenated
+  int tok_off;           // index of the row space's first token among the call's tokens
   int kv_head;
   int row0;              // first packed row of the item (multiple of 128)
-  int kind;              // 0: cached prefix keys (paged), 1: the rows' own keys
-  int key_begin;         // first key of the range (multiple of 64)
-  int key_count;         // keys in the range (0: the item only writes the neutral partial)
-  int page_off;          // kind 0: index of the prefix's first page id in the schedule's page list
+  int key_begin;         // first cached prefix key of the range (multiple of 64)
+  int key_count;         // cached keys in the range (0: none)
+  int page_off;          // index of the prefix's first page id in the schedule's page list
   int slot;              // which partial this range is
+  int own_begin;         // range 0 only: the own keys it also covers are tokens tok_off + own_begin ..
+  int own_count;         // .. + own_count - 1 of the call (the requests that have rows in this row tile)
 };
 
 struct DecSync {
@@ -82,8 +82,9 @@ __device__ __forceinline__ unsigned long long dec_now() {
 }  // namespace dec
 
 __global__ void __launch_bounds__(dec::kDecThreads, 2)
-tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __restrict__ reqs,
-                 const int* __restrict__ pages, PoolView pool, TensorArgs t, int* status, long long wait_cycles) {
+tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __restrict__ tok_rows,
+                 const int2* __restrict__ tok_span, const int* __restrict__ pages, PoolView pool, TensorArgs t,
+                 int* status, long long wait_cycles) {
   using namespace dec;
   // No room for alignment slack with two CTAs per SM: the kernel has no static shared memory, the
   // dynamic window starts 1024-byte aligned (the swizzled tiles need that), and a CTA that finds
@@ -100,7 +101,12 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
   if (threadIdx.x == 0) DEC_STAMP(0);
   const DecodeItem it = items[blockIdx.x];
   const int G = t.Hq / t.Hkv;
-  const int T = (it.key_count + kKeys - 1) / kKeys;
+  // key tiles: the cached range first, then (range 0) the own keys
+  const int T_pre = (it.key_count + kKeys - 1) / kKeys;
+  const int T = T_pre + (it.own_count + kKeys - 1) / kKeys;
+  auto tile_cnt = [&](int j) {
+    return j < T_pre ? min(kKeys, it.key_count - j * kKeys) : min(kKeys, it.own_count - (j - T_pre) * kKeys);
+  };
 
   if (tid == 0) {
     sy->wait_cycles = wait_cycles;
@@ -144,30 +150,23 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     const float sl2 = t.scale * 1.4426950408889634f;         // scores are handled in the log2 domain
     float m_ref = -INFINITY, l_sum = 0.f;
     bool ok = !dead;
+    // the call's tokens that are this row's own keys (its request); none for a row past the end
+    int2 span = make_int2(0, 0);
+    if (T > T_pre && it.row0 + row < it.n * G) span = tok_span[it.tok_off + (it.row0 + row) / G];
     if (ok && T > 0) {
-      // The Q tile, gathered by the 128 threads that have nothing else to do yet (one warp alone
-      // needs 5 us for its 64 passes): warp w fetches rows 32 w .. 32 w + 31, lane l the 16-byte chunk
-      // (l & 15) of rows 32 w + (l >> 4) + 2 i.  Packed row p = token a * G + head jj of the KV
-      // group; rows past the end are zero-filled.  Token a of the row space is token tok_off + a of
-      // the call: the request that holds it is found by walking the space's requests (a only grows
-      // along a lane's rows).
+      // The Q tile, gathered by the 128 threads that have nothing else to do yet: warp w fetches rows
+      // 32 w .. 32 w + 31, lane l the 16-byte chunk (l & 15) of rows 32 w + (l >> 4) + 2 i.  Packed row
+      // p = token a * G + head jj of the KV group; rows past the end are zero-filled.
       const int r0 = warp * 32 + (lane >> 4), c16 = lane & 15;
       const int packed_rows = it.n * G;
       const char* const q_head = t.q + ((long long)it.kv_head * G * 128) * 2 + c16 * 16;
-      int kreq = it.req_first;
-      const int kreq_end = it.req_first + it.req_count;
-      ReqMeta rq = reqs[kreq];
       int prow = it.row0 + r0;
       int a = prow / G, jj = prow - a * G;
 #pragma unroll 4
       for (int i = 0; i < 16; ++i) {
         const bool valid = prow < packed_rows;
         const char* src = q_head;
-        if (valid) {
-          const int tg = it.tok_off + a;
-          while (tg >= rq.tok_off + rq.n && kreq + 1 < kreq_end) rq = reqs[++kreq];
-          src = q_head + ((rq.row_off + (tg - rq.tok_off)) * t.q_stride + jj * 128) * 2;
-        }
+        if (valid) src = q_head + (tok_rows[it.tok_off + a] * t.q_stride + jj * 128) * 2;
         cp_async16(q_smem + tile_chunk_offset(r0 + 2 * i, c16), src, valid ? 16u : 0u);
         prow += 2;
         jj += 2;
@@ -184,7 +183,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
     }
     for (int j = 0; j < T && ok; ++j) {
       const int b = j & 1;
-      const int cnt = min(kKeys, it.key_count - j * kKeys);
+      const int cnt = tile_cnt(j);
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->s_full[b]), (j >> 1) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
@@ -193,7 +192,16 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
       tmem_ld32(tmem + b * 64 + lane_base, r);
       tmem_ld32(tmem + b * 64 + 32 + lane_base, r + 32);
       tmem_wait_ld();
-      if (cnt < kKeys) {
+      if (j >= T_pre) {
+        // own keys: column i is token tok_off + own_begin + 64 (j - T_pre) + i of the call; a row
+        // sees the tokens of its own request only (every row has seen a cached tile before, so its
+        // reference maximum is finite even if this whole tile is masked for it)
+        const int tok0 = it.tok_off + it.own_begin + (j - T_pre) * kKeys;
+        const int lo = span.x - tok0, hi = span.y - tok0;
+#pragma unroll
+        for (int i = 0; i < 64; ++i)
+          if (i < lo || i >= hi) r[i] = 0xff800000u;
+      } else if (cnt < kKeys) {
 #pragma unroll
         for (int i = 0; i < 64; ++i)
           if (i >= cnt) r[i] = 0xff800000u;                  // -inf: columns past the last key
@@ -342,7 +350,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
         // V is the MN-major operand: 64-dim halves 1024 bytes apart, 8-key groups 2048 bytes; a K
         // step of 16 keys is one page image (4096 bytes).  Steps past the last key are skipped.
         const unsigned long long v_desc = make_desc(v_ring + b * kKvTileBytes, 1024, 2048);
-        const int cnt = min(kKeys, it.key_count - j * kKeys);
+        const int cnt = tile_cnt(j);
         const int ksteps = (cnt + 15) >> 4;
 #pragma unroll
         for (int k = 0; k < 4; ++k)
@@ -375,8 +383,8 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
       if (!ok) break;
       const unsigned dst = ring + b * kKvTileBytes;
       const int key0 = it.key_begin + j * kKeys;
-      const int cnt = min(kKeys, it.key_count - j * kKeys);
-      if (it.kind == 0) {
+      const int cnt = tile_cnt(j);
+      if (j < T_pre) {
         // cached prefix: one bulk copy per page (a pool page already is the tile image), each issued
         // by its own lane so that the page-table reads overlap
         const int npages = (cnt + kPageSize - 1) / kPageSize;
@@ -396,16 +404,17 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const ReqMeta* __res
           mbar_arrive(full);
         }
       } else {
-        // the rows' own keys: 16-byte gathers into the page-image layout, zero-filled past the end
-        const char* rowp = (is_v ? t.v : t.k) + ((it.row_off + key0) * t.kv_stride + (long long)it.kv_head * 128) * 2 +
-                           c16 * 16;
-        const long long row_bytes = t.kv_stride * 2;
-        const char* src = rowp + r0 * row_bytes;
+        // own keys: 16-byte gathers into the page-image layout, zero-filled past the end; key r of the
+        // tile is token tok0 + r of the call, row tok_rows[tok0 + r] of k / v
+        const int tok0 = it.tok_off + it.own_begin + (j - T_pre) * kKeys;
+        const char* const base = (is_v ? t.v : t.k) + ((long long)it.kv_head * 128) * 2 + c16 * 16;
 #pragma unroll 4
         for (int i = 0; i < kKeys / 2; ++i) {
-          const bool valid = r0 + 2 * i < cnt;
-          cp_async16(dst + tile_chunk_offset(r0 + 2 * i, c16), valid ? src : rowp, valid ? 16u : 0u);
-          src += 2 * row_bytes;
+          const int r = r0 + 2 * i;
+          const bool valid = r < cnt;
+          const char* src = base;
+          if (valid) src = base + tok_rows[tok0 + r] * t.kv_stride * 2;
+          cp_async16(dst + tile_chunk_offset(r, c16), src, valid ? 16u : 0u);
         }
         cp_async_commit();
         cp_async_wait<0>();
@@ -535,12 +544,12 @@ inline cudaError_t configure_tc_decode() {
   return cudaFuncSetAttribute(tc_decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, dec::kDecSmemBytes);
 }
 
-inline cudaError_t launch_tc_decode(const dec::DecodeItem* items, int num_items, const ReqMeta* reqs, const int* pages,
-                                    const PoolView& pool,
+inline cudaError_t launch_tc_decode(const dec::DecodeItem* items, int num_items, const long long* tok_rows,
+                                    const int2* tok_span, const int* pages, const PoolView& pool,
                                     const TensorArgs& t, int* status, long long wait_cycles, cudaStream_t stream) {
   if (num_items <= 0) return cudaSuccess;
   tc_decode_kernel<<<num_items, dec::kDecThreads, dec::kDecSmemBytes, stream>>>(
-      items, reqs, pages, pool, t, status, wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
+      items, tok_rows, tok_span, pages, pool, t, status, wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
   return cudaGetLastError();
 }
 
