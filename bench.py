@@ -34,7 +34,8 @@ UNIT = "tokens/s"
 # DRAM bytes (read + write) of one launch of the dominant kernel, from ncu captures summarised
 # under profiles/ (None until a capture of that workload exists).
 NCU_TRAFFIC_BYTES = {"config2": {"full": 651.3e6, "attend": 138.2e6},
-                     "config3": {"put": 2104.6e6, "similarity": 2147.6e6, "project": 218.0e6}}     # profiles/tc_attention_kernel_config2.md
+                     "config3": {"put": 2104.6e6, "similarity": 2147.6e6, "project": 218.0e6},
+                     "b2": {"attend": 274.1e6}}     # profiles/tc_attention_kernel_config2.md
 
 
 def load_peaks():
@@ -406,10 +407,41 @@ def main():
     if bc.last_attention_kernel() == 3:                    # the key-range kernel (BICACHE_KERNEL_KEY_RANGES)
         # few query rows against a long cached prefix: the launch is bound by reading the prefix once
         gbs = w.attend_bytes() / (ms_attend * 1e-3) / 1e9
+        # The same call replayed from a CUDA graph (ten calls per replay): what a serving loop that
+        # captures its steps sees, without the host time of the Python binding per call.  Only for
+        # prefixes larger than L2, where back-to-back calls still read the keys from HBM.
+        graph_ms = None
+        if w.attend_bytes() > (200 << 20):
+            try:
+                st = torch.cuda.Stream()
+                with torch.cuda.stream(st):
+                    call_attend()
+                    torch.cuda.synchronize()
+                    g = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(g, stream=st):
+                        for _ in range(10):
+                            call_attend()
+                    ts = []
+                    for _ in range(5):
+                        flush.zero_()
+                        flush.max()
+                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a.record(st)
+                        g.replay()
+                        b.record(st)
+                        torch.cuda.synchronize()
+                        ts.append(a.elapsed_time(b) / 10)
+                graph_ms = sorted(ts)[len(ts) // 2]
+            except Exception:                              # capture not available: the figure is left out
+                graph_ms = None
         roofline_attend = {"bound": "hbm", "kernel": "tc_decode_kernel + merge_ranges_kernel (attend call)",
                            "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                            "peak_source": peaks["source"], "bytes_per_launch": w.attend_bytes(),
                            "ms_per_launch": ms_attend, "tflops": tf_attend,
+                           "graph_replay": (None if graph_ms is None else
+                                            {"ms_per_call": graph_ms, "calls_per_replay": 10,
+                                             "achieved": w.attend_bytes() / (graph_ms * 1e-3) / 1e9,
+                                             "frac": w.attend_bytes() / (graph_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}),
                            "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("attend")}
 
     # ---- end to end: host buffers, copies inside the timed region ------------------------------
