@@ -1,5 +1,5 @@
-"""Parity at the benchmark's full sizes (configurations 3-5), in the launch configuration the
-benchmark times: the layer-dispatch call at selected layers, compared with the oracle on sampled
+"""Parity at the benchmark's full sizes (configurations 3-5 and two of the small-suffix shapes), in the
+launch configuration the benchmark times: the layer-dispatch call at selected layers, compared with the oracle on sampled
 rows, each computed over all of its keys.  Sampled per layer: tile-boundary rows of the shortest and
 longest requests and random (request, head, row) triples."""
 import numpy as np
@@ -13,7 +13,7 @@ from paper_2606_07571_b200 import binding, workloads
 pytestmark = pytest.mark.gpu
 
 
-def run_config(name, layers_to_check, n_random=24):
+def run_config(name, layers_to_check, n_random=24, key_ranges=False):
     entry.build()
     w = workloads.CONFIGS[name]()
     L = w.num_layers
@@ -50,6 +50,9 @@ def run_config(name, layers_to_check, n_random=24):
         out.fill_(7.0)
         bc.attend_layer(layer, depth, req_pid, w.full_row_off, w.full_lens, q, k, v, out, lse, w.softmax_scale)
         assert bc.device_status() == binding.OK
+        if key_ranges and layer < int(min(depth)):
+            # every request reuses at this layer: one attend call, served by the key-range kernel
+            assert bc.last_attention_kernel() == binding.KERNEL_KEY_RANGES
         worst = 0.0
         errs = []
         for i in picked:
@@ -100,3 +103,13 @@ def test_config4_full_size_sampled():
 
 def test_config5_full_size_sampled():
     run_config("config5", [0, 20, 21])          # depth is 21 for every request: last reuse layer, first full layer
+
+
+@pytest.mark.parametrize("name", ["b2", "b3"])
+def test_small_suffix_shapes_full_size_sampled(name):
+    """Block-query shapes at full size (prefix 16384, 1 and 4 requests of 32 tokens, 32 layers): the
+    shallow layers go through the key-range kernel, the deep ones through full attention."""
+    w = workloads.CONFIGS[name]()
+    d = oracle.reuse_depth(w.req_prefix_len(), w.suffix_lens, workloads.standin_depth_table(w.num_layers),
+                           w.num_layers)
+    run_config(name, sorted({0, int(d.min()) - 1, int(d.min())}), key_ranges=True)
