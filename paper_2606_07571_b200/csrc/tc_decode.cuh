@@ -12,10 +12,10 @@
 // runs once per 128 keys with nothing to overlap it, and one CTA per SM cannot keep HBM busy.
 // Here a CTA is small (112 KB of shared memory, 256 TMEM columns: two CTAs per SM), key tiles are
 // 64 keys, and S is double-buffered in TMEM: S(j+1) = Q K(j+1)^T is issued before the softmax of
-// tile j ends.  Roles: warps 0-3 softmax (one thread per row), warp 4 MMA issue and TMEM, warp 5
-// stages K tiles, warp 6 stages V tiles (the softmax warps gather Q before their first tile) (cached pages: one 4 KB bulk copy per page,
-// a pool page already is the operand image; own rows: 16-byte gathers into the same image).
-// Every wait is bounded, as in the big kernel.
+// tile j ends.  Roles: warps 0-3 softmax (one thread per row; they also gather the Q tile before
+// their first key tile), warp 4 MMA issue and TMEM, warp 5 stages K tiles, warp 6 stages V tiles
+// (cached pages: one 4 KB bulk copy per page, a pool page already is the operand image; own rows:
+// 16-byte gathers into the same image).  Every wait is bounded, as in the big kernel.
 #pragma once
 
 #include "tc_attention.cuh"
