@@ -543,8 +543,29 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
         float alpha = 1.f;
         unsigned long long acc_a = pack2(0.f, 0.f), acc_b = pack2(0.f, 0.f);
         bool stored = false;                                   // P already stored and signalled
-        if (j > 0 && cnt >= kTileKeys) {
-          // Common case (a full tile after the first): the exponentials use the reference maximum of
+        // A ragged tile: columns past the last key become -inf (their exponentials are exactly 0).
+        if (cnt < kTileKeys) {
+#pragma unroll
+          for (int i = 0; i < 128; ++i)
+            if (i >= cnt) r[i] = 0xff800000u;
+        }
+        // The first tile of an item takes its own row maximum as the reference (a short extra pass);
+        // everything else is one code path for every tile: this code runs once per key tile and
+        // must stay in the instruction cache, which a separate first-tile path (11 KB of straight-
+        // line code met once per item) did not.
+        if (j == 0) {
+          float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+          for (int i = 0; i < 128; i += 8) {
+            mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
+            mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
+            mx2 = max3(mx2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
+            mx3 = max3(mx3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
+          }
+          m_ref = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sl2;   // scale > 0; finite: a tile has a key
+        }
+        {
+          // The exponentials use the reference maximum of
           // the earlier tiles and do not wait for this tile's maximum, which is computed alongside.
           // P of the first 64 keys is handed to the tensor pipe before the second half is computed.
           // If the row maximum turns out to exceed the reference by more than 2^8 (rare: checked per
@@ -630,8 +651,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               tmem_wait_ld();
 #pragma unroll
               for (int i = 0; i < 16; ++i) {
-                const float p0 = ex2(fmaf(__uint_as_float(s4[2 * i]), sl2, neg_m));
-                const float p1 = ex2(fmaf(__uint_as_float(s4[2 * i + 1]), sl2, neg_m));
+                // (the scores come from TMEM again: columns past the last key of a ragged tile are masked here)
+                const float p0 = c * 32 + 2 * i < cnt ? ex2(fmaf(__uint_as_float(s4[2 * i]), sl2, neg_m)) : 0.f;
+                const float p1 = c * 32 + 2 * i + 1 < cnt ? ex2(fmaf(__uint_as_float(s4[2 * i + 1]), sl2, neg_m)) : 0.f;
                 ps += p0 + p1;
                 r[c * 16 + i] = pack_bf16(p0, p1);
               }
@@ -647,56 +669,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               for (int i = 0; i < 32; ++i) s4[i] = __float_as_uint(__uint_as_float(s4[i]) * alpha);
               tmem_st32(tmem_o + c * 32, s4);
             }
-          }
-        } else {
-          // First tile of the item, or a ragged tile: maximum first, every exponential on the exp
-          // unit so that masked columns give exactly 0.
-          if (cnt < kTileKeys) {
-#pragma unroll
-            for (int i = 0; i < 128; ++i)
-              if (i >= cnt) r[i] = 0xff800000u;                // -inf: columns past the last key
-          }
-          float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-          for (int i = 0; i < 128; i += 8) {
-            mx0 = max3(mx0, __uint_as_float(r[i]), __uint_as_float(r[i + 1]));
-            mx1 = max3(mx1, __uint_as_float(r[i + 2]), __uint_as_float(r[i + 3]));
-            mx2 = max3(mx2, __uint_as_float(r[i + 4]), __uint_as_float(r[i + 5]));
-            mx3 = max3(mx3, __uint_as_float(r[i + 6]), __uint_as_float(r[i + 7]));
-          }
-          const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sl2;   // scale > 0
-          if (j == 0) {
-            m_ref = mx;
-          } else if (mx > m_ref + 8.f) {
-            alpha = ex2(m_ref - mx);
-            m_ref = mx;
-          }
-          if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-              unsigned o[32];
-              tmem_ld32(tmem_o + c * 32, o);
-              tmem_wait_ld();
-#pragma unroll
-              for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
-              tmem_st32(tmem_o + c * 32, o);
-            }
-          }
-          const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const unsigned long long xa =
-                fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
-            const unsigned long long xb =
-                fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
-            float x0, x1, x2, x3;
-            unpack2(xa, x0, x1);
-            unpack2(xb, x2, x3);
-            const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
-            acc_a = add2(acc_a, pack2(p0, p1));
-            acc_b = add2(acc_b, pack2(p2, p3));
-            r[2 * i] = pack_bf16(p0, p1);
-            r[2 * i + 1] = pack_bf16(p2, p3);
           }
         }
         if (!stored) {
