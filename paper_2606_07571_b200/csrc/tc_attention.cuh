@@ -256,6 +256,34 @@ __device__ __forceinline__ void mma_ts_batch4(unsigned el, unsigned o_tmem, unsi
       ::"r"(o_tmem), "r"(p_tmem), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "r"(idesc), "r"(acc0), "r"(el)
       : "memory");
 }
+// The same for a ragged key tile: up to four K steps of 16 keys, P read from TMEM at p + 8 k; the first accumulates iff
+// acc0; only the first n_on steps are issued (a ragged key tile has fewer than eight steps).
+__device__ __forceinline__ void mma_ts_batch4_first(unsigned el, unsigned o_tmem, unsigned p_tmem,
+                                                    const unsigned long long (&b)[4], unsigned idesc, unsigned acc0,
+                                                    int n_on) {
+  asm volatile(
+      "{\n\t.reg .pred P, T, Q, E0, E1, E2, E3;\n\t.reg .b32 p1, p2, p3;\n\t"
+      "setp.ne.b32 P, %8, 0;\n\t"
+      "setp.eq.u32 T, 0, 0;\n\t"
+      "setp.ne.b32 Q, %7, 0;\n\t"
+      "setp.gt.s32 E0, %9, 0;\n\t"
+      "setp.gt.s32 E1, %9, 1;\n\t"
+      "setp.gt.s32 E2, %9, 2;\n\t"
+      "setp.gt.s32 E3, %9, 3;\n\t"
+      "and.pred E0, E0, P;\n\t"
+      "and.pred E1, E1, P;\n\t"
+      "and.pred E2, E2, P;\n\t"
+      "and.pred E3, E3, P;\n\t"
+      "add.u32 p1, %1, 8;\n\t"
+      "add.u32 p2, %1, 16;\n\t"
+      "add.u32 p3, %1, 24;\n\t"
+      "@E0 tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %6, Q;\n\t"
+      "@E1 tcgen05.mma.cta_group::1.kind::f16 [%0], [p1], %3, %6, T;\n\t"
+      "@E2 tcgen05.mma.cta_group::1.kind::f16 [%0], [p2], %4, %6, T;\n\t"
+      "@E3 tcgen05.mma.cta_group::1.kind::f16 [%0], [p3], %5, %6, T;\n\t}"
+      ::"r"(o_tmem), "r"(p_tmem), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "r"(idesc), "r"(acc0), "r"(el), "r"(n_on)
+      : "memory");
+}
 // tcgen05.commit by the same elected lane (a commit covers the MMAs its own thread issued)
 __device__ __forceinline__ void mma_commit_pred(unsigned el, unsigned bar) {
   asm volatile(
@@ -1035,16 +1063,11 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       // four of the eight MMAs (K steps of 16 keys) of O_X += P_X V
       auto issue_pv = [&](unsigned o_tmem, unsigned p_tmem, unsigned long long vd, unsigned v_step, int half,
                           unsigned acc0, int ksteps) {
-        if (ksteps == 8) {
-          unsigned long long b[4];
+        unsigned long long b[4];
 #pragma unroll
-          for (int k = 0; k < 4; ++k) b[k] = vd + (half * 4 + k) * v_step;
-          mma_ts_batch4(el, o_tmem, p_tmem + half * 32, b, kIdescPV, half ? 1u : acc0);
-        } else {
-#pragma unroll
-          for (int k = half * 4; k < half * 4 + 4; ++k)
-            mma_ts_elect(o_tmem, p_tmem + k * 8, vd + k * v_step, kIdescPV, k > 0 ? 1u : acc0, k < ksteps ? 1u : 0u);
-        }
+        for (int k = 0; k < 4; ++k) b[k] = vd + (half * 4 + k) * v_step;
+        if (ksteps == 8) mma_ts_batch4(el, o_tmem, p_tmem + half * 32, b, kIdescPV, half ? 1u : acc0);
+        else mma_ts_batch4_first(el, o_tmem, p_tmem + half * 32, b, kIdescPV, half ? 1u : acc0, ksteps - half * 4);
       };
       int n_it = 0;
       int c0 = 0, c1 = 0;        // key tiles each query tile has been through (phase of p_half)
