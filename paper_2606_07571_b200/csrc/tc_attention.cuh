@@ -109,24 +109,22 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity) {
 }
 // Bounded wait.  try_wait suspends the thread in hardware until the phase completes or a short
 // system time limit passes, so the loop itself needs no sleep; the SM clock bounds the total.
-// Returns false if the CTA's abort flag is up or (raising it) if the budget runs out.
+// Returns false if the CTA's abort flag is up or (raising it) if the budget runs out.  Kept small:
+// the kernels wait at some sixty places, every one an inlined copy, and their code has to stay in
+// the instruction cache.
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (unsigned it = 1;; ++it) {
+  // the budget sits in shared memory directly before the abort flag
+  const long long t_end = clock64() + *reinterpret_cast<const volatile long long*>(abort_flag - 2);
+#pragma unroll 1
+  while (!*abort_flag && clock64() < t_end)
     if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 1u) {
-      if (*abort_flag) return false;
-      // the budget sits in shared memory directly before the abort flag
-      if (clock64() - t0 > *reinterpret_cast<const volatile long long*>(abort_flag - 2)) break;
-    }
-  }
   *abort_flag = 1;
   return false;
 }
 // A budget below this is the tests' way to walk the give-up path with barriers that all complete:
-// the abort flag is up from the start, so every wait that is not over within its first two polls
-// gives up, and the launch reports a timeout.
+// the abort flag is up from the start, so every wait that is not over at its first poll gives up,
+// and the launch reports a timeout.
 constexpr long long kStrictBudget = 1024;
 // Wait for work that is certain to finish (MMAs already issued): the default budget, whatever the
 // per-wait budget or the abort flag say, because tensor memory must not be released under them.
