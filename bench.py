@@ -33,7 +33,7 @@ UNIT = "tokens/s"
 
 # DRAM bytes (read + write) of one launch of the dominant kernel, from ncu captures summarised
 # under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {"config2": {"full": 651.3e6, "attend": 138.2e6},     # profiles/tc_attention_kernel_config2.md
+NCU_TRAFFIC_BYTES = {"config2": {"full": 647.9e6, "attend": 135.3e6},     # profiles/tc_attention_kernel_config2.md
                      "config3": {"put": 2104.6e6, "similarity": 2147.6e6,    # profiles/hbm_kernels_config3.md
                                  "project": 218.0e6},                         # profiles/project_kv_kernel_config3.md
                      "b2": {"attend": 274.1e6}}                               # profiles/key_range_kernels_b2.md
