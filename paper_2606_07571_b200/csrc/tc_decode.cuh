@@ -318,6 +318,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
     bool ok = !dead && T > 0;
     if (ok) {
       const unsigned long long q_desc = make_desc(q_smem, 16, 2048);
+      const unsigned el = elect_one() ? 1u : 0u;               // the lane that issues every MMA of this warp
       // a K step of 16 dims: 32 bytes inside the swizzled row; dims 64.. sit 1024 bytes further
       auto kstep = [](int k) { return (unsigned long long)((k & 3) * 2 + (k >> 2) * 64); };
       auto issue_s = [&](int j) {
@@ -326,11 +327,15 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
         if (!good) return false;
         tc_fence_after();
         const unsigned long long k_desc = make_desc(k_ring + ks * kKvTileBytes, 16, 2048);
+        unsigned long long qa[8], kb[8];
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
-          mma_ss_elect(tmem + b * 64, q_desc + kstep(k), k_desc + kstep(k), kIdescS64, k > 0 ? 1u : 0u);
-        mma_commit_elect(smem_u32(&sy->s_full[b]));
-        mma_commit_elect(smem_u32(&sy->k_free[ks]));
+        for (int k = 0; k < 8; ++k) {
+          qa[k] = q_desc + kstep(k);
+          kb[k] = k_desc + kstep(k);
+        }
+        mma_ss_batch8(el, tmem + b * 64, qa, kb, kIdescS64);   // one predicated group instead of eight elections
+        mma_commit_pred(el, smem_u32(&sy->s_full[b]));
+        mma_commit_pred(el, smem_u32(&sy->k_free[ks]));
         return true;
       };
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->q_full), 0, abort_flag));
@@ -352,13 +357,11 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
         const unsigned long long v_desc = make_desc(v_ring + b * kKvTileBytes, 1024, 2048);
         const int cnt = tile_cnt(j);
         const int ksteps = (cnt + 15) >> 4;
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-          mma_ts_elect(tmem_o, tmem + b * 64 + k * 8, v_desc + (unsigned long long)(k * 256), kIdescPV,
-                       (j > 0 || k > 0) ? 1u : 0u, k < ksteps ? 1u : 0u);
-        mma_commit_elect(smem_u32(&sy->v_free[b]));
-        mma_commit_elect(smem_u32(&sy->pv_done));
-        if (j == T - 1) mma_commit_elect(smem_u32(&sy->o_done));
+        const unsigned long long vb[4] = {v_desc, v_desc + 256ull, v_desc + 512ull, v_desc + 768ull};
+        mma_ts_batch4_first(el, tmem_o, tmem + b * 64, vb, kIdescPV, j > 0 ? 1u : 0u, ksteps);
+        mma_commit_pred(el, smem_u32(&sy->v_free[b]));
+        mma_commit_pred(el, smem_u32(&sy->pv_done));
+        if (j == T - 1) mma_commit_pred(el, smem_u32(&sy->o_done));
       }
       // Whatever happened, let every MMA issued so far finish before TMEM is released.
       __syncwarp();
