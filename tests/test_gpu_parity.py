@@ -117,6 +117,7 @@ def tiny(name, L, Hq, Hkv, D, dtype, ms, req_prefix, ns, shuffle=False, std=1.0,
 def test_config1_tiny_fp32():
     c = Case(workloads.config1())
     c.compare_all()
+    assert c.bc.last_attention_kernel() == binding.KERNEL_SIMT      # fp32, D = 64: the CUDA-core kernel
     c.close()
 
 
