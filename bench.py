@@ -4,12 +4,12 @@
 One "step" is one denoising step's attention: reuse-depth rule, prefix-store lookups (hits), the
 per-layer dispatch, and for every layer the shallow-layer call (suffix queries over cached prefix
 K/V + own suffix K/V) and/or the deep-layer fallback (full bidirectional attention), all through
-the C ABI.  The default workload is the LLaDA-8B-shaped single layer (prefix 1024, 16 requests x
-256 suffix tokens, bf16): being one layer, its step runs the layer once as a shallow layer (every
-request reuses, as the depth rule says) and once as a deep layer (every request recomputes), so
-that every stage of the path is inside the timed region.
+the C ABI.  The default workload is the largest single-GPU configuration by FLOPs per step, the
+Dream-7B-shaped 28-layer GQA stack with a 16384-token prefix (`config5`); the other configurations
+and the small-suffix (bandwidth-bound) shapes are measured in the same run at a few steps each and
+reported as the `per_config` list of the same JSON line.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config2] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload config5] [--impl reference]
 
 Prints ONE JSON line (rank 0).
 """
@@ -30,13 +30,27 @@ import torch
 
 METRIC = "prefix_reuse_attention_suffix_tokens_per_s_per_denoising_step"
 UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "config5"
+# what the default run measures besides its own workload: (workload, timed steps)
+PER_CONFIG = (("config2", 20), ("config3", 8), ("config4", 4))
+SMALL_SUFFIX = ("b1", "b2", "b3", "b4")
 
-# DRAM bytes (read + write) of one launch of the dominant kernel, from ncu captures summarised
-# under profiles/ (None until a capture of that workload exists).
-NCU_TRAFFIC_BYTES = {"config2": {"full": 647.9e6, "attend": 135.3e6},     # profiles/tc_attention_kernel_config2.md
-                     "config3": {"put": 2104.6e6, "similarity": 2147.6e6,    # profiles/hbm_kernels_config3.md
-                                 "project": 218.0e6},                         # profiles/project_kv_kernel_config3.md
-                     "b2": {"attend": 274.1e6}}                               # profiles/key_range_kernels_b2.md
+# DRAM bytes (read + write) of one launch, from the ncu captures summarised under profiles/ (the file
+# is named beside each figure; a capture is of the kernel as it was when the summary was written).
+# None: no capture of that launch exists.
+NCU_TRAFFIC = {
+    "config2": {"full": (647.9e6, "profiles/tc_attention_kernel_config2.md"),
+                "attend": (135.3e6, "profiles/tc_attention_kernel_config2.md")},
+    "config3": {"put": (2104.6e6, "profiles/hbm_kernels_config3.md"),
+                "similarity": (2147.6e6, "profiles/hbm_kernels_config3.md"),
+                "project": (218.0e6, "profiles/project_kv_kernel_config3.md")},
+    "b2": {"attend": (274.1e6, "profiles/key_range_kernels_b2.md")},
+}
+
+
+def traffic_of(workload, which):
+    t = NCU_TRAFFIC.get(workload, {}).get(which)
+    return (None, None) if t is None else t
 
 
 def load_peaks():
@@ -44,7 +58,7 @@ def load_peaks():
     if os.path.exists(path):
         with open(path) as f:
             p = json.load(f)
-        return {"bf16_tflops": p["bf16_tflops"], "bf16_tflops_sustained": p.get("bf16_tflops_sustained"),
+        return {"bf16_tflops": p["bf16_tflops"], "bf16_tflops_sustained": p.get("bf16_tflops_sustained") or p["bf16_tflops"],
                 "hbm_gbs": p["hbm_gbs"], "source": "measured"}
     return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
 
@@ -131,10 +145,29 @@ class Job:
         self.out = torch.empty_like(self.q)
         self.single_layer = w.num_layers == 1
         self.out2 = torch.empty_like(self.q) if self.single_layer else None
+        self.depth = self.bc.reuse_depth(w.req_prefix_len(), w.suffix_lens)
         torch.cuda.synchronize()
 
-    def step(self, q=None, k=None, v=None, out=None, out2=None):
-        """One denoising step's attention through the C ABI."""
+    def close(self):
+        self.bc.close()
+        for name in ("q", "k", "v", "out", "out2", "bc"):
+            setattr(self, name, None)
+        torch.cuda.empty_cache()
+
+    def calls_per_step(self):
+        """The layer calls of one step as (layer, kind): kind 'attend' / 'full' when every request of
+        the call takes the same path in that layer (one kernel launch of known FLOPs), else 'mixed'."""
+        w = self.w
+        if self.single_layer:
+            return [(0, "attend"), (0, "full")]
+        if self.delta > 0:
+            return [(l, "mixed") for l in range(w.num_layers)]
+        lo, hi = int(min(self.depth)), int(max(self.depth))
+        return [(l, "attend" if l < lo else "full" if l >= hi else "mixed") for l in range(w.num_layers)]
+
+    def step(self, q=None, k=None, v=None, out=None, out2=None, events=None):
+        """One denoising step's attention through the C ABI.  `events`: a list that receives one
+        (start, end) CUDA event pair per layer call, in the order of calls_per_step()."""
         w, bc = self.w, self.bc
         q = self.q if q is None else q
         k = self.k if k is None else k
@@ -144,35 +177,47 @@ class Job:
         depth = bc.reuse_depth(w.req_prefix_len(), w.suffix_lens)                     # depth rule
         pid = [bc.lookup_prefix(key)[0] for key in self.keys]                         # store hits
         req_pid = [pid[g] for g in w.req_prefix]
+
+        def timed(fn):
+            if events is None:
+                fn()
+                return
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            events.append((a, b))
+
         if self.single_layer:
             # shallow-layer pass (depths from the rule) then deep-layer pass (all recompute)
-            bc.attend_layer(0, depth, req_pid, w.full_row_off, w.full_lens, q, k, v, out, None, w.softmax_scale)
-            bc.attend_layer(0, [0] * w.num_requests, req_pid, w.full_row_off, w.full_lens, q, k, v, out2, None,
-                            w.softmax_scale)
+            timed(lambda: bc.attend_layer(0, depth, req_pid, w.full_row_off, w.full_lens, q, k, v, out, None,
+                                          w.softmax_scale))
+            timed(lambda: bc.attend_layer(0, [0] * w.num_requests, req_pid, w.full_row_off, w.full_lens, q, k, v,
+                                          out2, None, w.softmax_scale))
         elif self.delta > 0:
             # deep layers keep the request's own prefix K/V and recompute them every delta steps
             for l in range(w.num_layers):
-                bc.attend_step(l, self.t, self.delta, depth, req_pid, self.private, w.full_row_off, w.full_lens,
-                               q, k, v, out, None, w.softmax_scale)
+                timed(lambda: bc.attend_step(l, self.t, self.delta, depth, req_pid, self.private, w.full_row_off,
+                                             w.full_lens, q, k, v, out, None, w.softmax_scale))
             self.t += 1
         else:
             for l in range(w.num_layers):
-                bc.attend_layer(l, depth, req_pid, w.full_row_off, w.full_lens, q, k, v, out, None,
-                                w.softmax_scale)
+                timed(lambda: bc.attend_layer(l, depth, req_pid, w.full_row_off, w.full_lens, q, k, v, out, None,
+                                              w.softmax_scale))
         return depth
 
     def step_flops(self):
         w = self.w
-        depth = self.bc.reuse_depth(w.req_prefix_len(), w.suffix_lens)
+        depth = self.depth
         per_req_attend = [4 * w.head_dim * w.num_q_heads * n * (w.prefix_lens[g] + n)
                           for g, n in zip(w.req_prefix, w.suffix_lens)]
         per_req_full = [4 * w.head_dim * w.num_q_heads * N * N for N in w.full_lens]
         if self.single_layer:
-            return sum(per_req_attend) + sum(per_req_full), depth
+            return sum(per_req_attend) + sum(per_req_full)
         tot = 0
         for i in range(w.num_requests):
             tot += int(depth[i]) * per_req_attend[i] + (w.num_layers - int(depth[i])) * per_req_full[i]
-        return tot, depth
+        return tot
 
     def reuse_step_flops(self):
         """A step between two refresh steps: every layer reads a cached prefix (shared or kept)."""
@@ -204,47 +249,307 @@ def max_over_ranks(value, dist, device):
     return float(t.item())
 
 
-def oracle_one_request(w, workloads, oracle, i):
-    """The oracle on request i of the workload: one shallow-layer and one deep-layer pass (all heads).
-    Returns (seconds of the shallow pass, seconds of the deep pass)."""
-    g = w.req_prefix[i]
-    m, n = w.prefix_lens[g], w.suffix_lens[i]
-    sub = workloads.Workload("sample", 1, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, 16, [m], [0], [n],
-                             softmax_scale=w.softmax_scale, seed=w.seed + i)
-    kc, vc = workloads.draw_prefix_kv(sub, 0, "cpu")
-    q, k, v = workloads.draw_full_qkv(sub, "cpu")
-    st = oracle.PagedPrefixStore(1, w.num_kv_heads, w.head_dim, 16, sub.pages_needed())
-    qd, kd, vd = (workloads.to_f64(x) for x in (q, k, v))
-    pid, _, _ = st.put(1, workloads.to_f64(kc), workloads.to_f64(vc))
-    t0 = time.perf_counter()
-    oracle.attend(st, 0, [pid], sub.suffix_row_off, sub.suffix_lens, qd, kd, vd, w.softmax_scale)
-    t1 = time.perf_counter()
-    oracle.attend_full(sub.full_row_off, sub.full_lens, qd, kd, vd, w.softmax_scale)
-    t2 = time.perf_counter()
-    return (t1 - t0), (t2 - t1)
+def tensor_roofline(kernel, flops, ms, peaks, sustained, launches, traffic):
+    """The roofline record of a tensor-pipe-bound launch.  `sustained`: the launch was timed inside
+    a long step (seconds of back-to-back kernels under the power cap), so the denominator is the
+    sustained matmul peak; a launch timed alone takes the burst peak."""
+    tf = flops / (ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    return {"bound": "tensor", "kernel": kernel, "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+            "peak_source": peaks["source"] + (" sustained (launch timed inside a long step)" if sustained
+                                              else " burst (launch timed alone or inside a millisecond step)"),
+            "frac_of_burst": tf / peaks["bf16_tflops"], "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
+            "traffic": traffic[0], "traffic_source": traffic[1],
+            "flops_per_launch": flops, "ms_per_launch": ms, "launches_timed": launches}
 
 
-def oracle_step_seconds(w, workloads, oracle, depth, budget_s=12.0):
-    """Time of one whole step for the oracle.  Requests are sampled (median length first, then
-    spread over the length distribution) until about `budget_s` seconds of oracle work are done;
-    the step time is the sampled time scaled by the step's algorithmic FLOPs over the sample's."""
-    order = np.argsort(w.suffix_lens)
-    R = w.num_requests
+def measure_steps(job, name, steps, warmup, flush, peaks, rank, local_rank, world, dist):
+    """Warm-up, then `steps` timed steps (each preceded by an untimed L2 flush), with one CUDA event
+    pair per layer call so that the launches of the dominant kernels are timed where they run."""
+    w = job.w
+    for _ in range(warmup):
+        flush.zero_()
+        job.step()
+    assert job.bc.device_status() == 0
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = job.bc.launch_count()
+    job.t = 1                                         # the timed steps are denoising steps 1 .. K
+    ev, per_call = [], []
+    for _ in range(steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        calls = []
+        flush.zero_()
+        a.record()
+        job.step(events=calls)
+        b.record()
+        ev.append((a, b))
+        per_call.append(calls)
+    torch.cuda.synchronize()
+    launches = job.bc.launch_count() - launches0
+    per_step_ms = [a.elapsed_time(b) for a, b in ev]
+    step_ms = sum(per_step_ms) / steps
+    if step_ms * steps < 400.0:
+        # a short sustained stretch so that the clock sampler sees the kernels under load
+        t_end = time.time() + 0.5
+        while time.time() < t_end:
+            job.step()
+            torch.cuda.synchronize()
+    clocks = sampler.stop() if rank == 0 else None
+    assert job.bc.device_status() == 0
+    step_ms_max = max_over_ranks(step_ms, dist, "cuda")
+    if dist is not None:
+        dist.barrier()
+
+    flops = job.step_flops()
+    refresh_info = None
+    if job.delta > 0:
+        is_ref = [(t - 1) % job.delta == 0 for t in range(1, steps + 1)]
+        ref_ms = [m for m, r in zip(per_step_ms, is_ref) if r]
+        reu_ms = [m for m, r in zip(per_step_ms, is_ref) if not r]
+        flops = (len(ref_ms) * flops + len(reu_ms) * job.reuse_step_flops()) / steps   # mean FLOPs per step
+        refresh_info = {"delta": job.delta, "refresh_steps": len(ref_ms), "reuse_steps": len(reu_ms),
+                        "ms_refresh_step": sum(ref_ms) / max(1, len(ref_ms)),
+                        "ms_reuse_step": sum(reu_ms) / max(1, len(reu_ms)) if reu_ms else None}
+
+    # launches timed in place: the layer calls in which every request takes the same path
+    kinds = job.calls_per_step()
+    in_place = {"attend": [], "full": []}
+    for calls in per_call:
+        for (layer, kind), (a, b) in zip(kinds, calls):
+            if kind in in_place:
+                in_place[kind].append(a.elapsed_time(b))
+    sustained = step_ms >= 50.0          # the stacks: tens of milliseconds to a second of back-to-back kernels
+    roofline = roofline_attend = None
+    if in_place["full"]:
+        roofline = tensor_roofline("tc_attention_kernel (attend_full launch, every request recomputes)",
+                                   w.full_flops(), sum(in_place["full"]) / len(in_place["full"]), peaks, sustained,
+                                   len(in_place["full"]), traffic_of(name, "full"))
+    if in_place["attend"]:
+        roofline_attend = tensor_roofline("tc_attention_kernel (attend launch, every request reuses)",
+                                          w.attend_flops(), sum(in_place["attend"]) / len(in_place["attend"]), peaks,
+                                          sustained, len(in_place["attend"]), traffic_of(name, "attend"))
+    depth = job.depth
+    return {"value": world * w.suffix_tokens / (step_ms_max * 1e-3), "ms_per_step": step_ms_max, "steps": steps,
+            "warmup": warmup, "tflops": flops / (step_ms_max * 1e-3) / 1e12, "step_flops": flops,
+            "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "roofline_attend": roofline_attend,
+            "config": dict(config_keys(w, depth), deep_layer_refresh=refresh_info)}
+
+
+def measure_calls_alone(job, name, flush, peaks):
+    """The `attend` and `attend_full` calls of one layer over all requests, each timed alone after an L2
+    flush (CUDA events around the single call): the burst-peak view of the same two launches."""
+    w, bc = job.w, job.bc
+    pid = [bc.lookup_prefix(key)[0] for key in job.keys]
+    req_pid = [pid[g] for g in w.req_prefix]
+
+    def call_attend():
+        bc.attend(0, req_pid, w.suffix_row_off, w.suffix_lens, job.q, job.k, job.v, job.out, None, w.softmax_scale)
+
+    def call_full():
+        bc.attend_full(0, w.full_row_off, w.full_lens, job.q, job.k, job.v, job.out, None, w.softmax_scale)
+
+    iters = 10 if w.full_flops() < 5e13 else 3
+    call_attend()
+    kernel = bc.last_attention_kernel()
+    call_full()
+    ms_attend = time_call(call_attend, iters, flush)
+    ms_full = time_call(call_full, iters, flush)
+    full = tensor_roofline("tc_attention_kernel (attend_full call alone)", w.full_flops(), ms_full, peaks, False,
+                           iters, traffic_of(name, "full"))
+    if kernel != 3:                                    # not the key-range kernel
+        attend = tensor_roofline("tc_attention_kernel (attend call alone)", w.attend_flops(), ms_attend, peaks, False,
+                                 iters, traffic_of(name, "attend"))
+        return {"attend_full": full, "attend": attend}
+    # few query rows against a long cached prefix: the call is bound by reading the prefix once
+    gbs = w.attend_bytes() / (ms_attend * 1e-3) / 1e9
+    # The same call replayed from a CUDA graph (ten calls per replay): what a serving loop that
+    # captures its steps sees, without the host time of the Python binding per call.  Only for
+    # prefixes larger than L2, where back-to-back calls still read the keys from HBM.
+    graph_ms = None
+    if w.attend_bytes() > (200 << 20):
+        try:
+            st = torch.cuda.Stream()
+            with torch.cuda.stream(st):
+                call_attend()
+                torch.cuda.synchronize()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=st):
+                    for _ in range(10):
+                        call_attend()
+                ts = []
+                for _ in range(5):
+                    flush.zero_()
+                    flush.max()
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record(st)
+                    g.replay()
+                    b.record(st)
+                    torch.cuda.synchronize()
+                    ts.append(a.elapsed_time(b) / 10)
+            graph_ms = sorted(ts)[len(ts) // 2]
+        except Exception:                              # capture not available: the figure is left out
+            graph_ms = None
+    tr = traffic_of(name, "attend")
+    attend = {"bound": "hbm", "kernel": "tc_decode_kernel (+ merge) (attend call alone)",
+              "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+              "peak_source": peaks["source"], "bytes_per_launch": w.attend_bytes(), "ms_per_launch": ms_attend,
+              "launches_timed": iters, "tflops": w.attend_flops() / (ms_attend * 1e-3) / 1e12,
+              "graph_replay": (None if graph_ms is None else
+                               {"ms_per_call": graph_ms, "calls_per_replay": 10,
+                                "achieved": w.attend_bytes() / (graph_ms * 1e-3) / 1e9,
+                                "frac": w.attend_bytes() / (graph_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}),
+              "traffic": tr[0], "traffic_source": tr[1]}
+    return {"attend_full": full, "attend": attend}
+
+
+def pinned_like(t, chunk_bytes=1 << 30):
+    """Pinned host buffers for a [rows, ...] tensor, in chunks of at most `chunk_bytes` (a list of
+    (first row, buffer)): one allocation per gigabyte instead of one of many."""
+    rows = t.shape[0]
+    row_bytes = max(1, t[0].numel() * t.element_size())
+    step = max(1, chunk_bytes // row_bytes)
+    return [(r0, torch.empty((min(step, rows - r0),) + tuple(t.shape[1:]), dtype=t.dtype, pin_memory=True))
+            for r0 in range(0, rows, step)]
+
+
+def measure_e2e(job, steps, world, dist):
+    """The same step with HOST inputs and outputs: every step uploads its Q, K, V from pinned host
+    memory and downloads its output(s); the copies are inside the timed region."""
+    w = job.w
+    host_in = []
+    for x in (job.q, job.k, job.v):
+        chunks = pinned_like(x)
+        for r0, c in chunks:
+            c.copy_(x[r0:r0 + c.shape[0]])
+        host_in.append(chunks)
+    n_out = 2 if job.single_layer else 1
+    # Two buffer sets and three streams: the upload of step i + 1 and the download of step i - 1
+    # run while step i computes (every step still uploads its own inputs and downloads its own
+    # outputs; the figure is the steady-state time per step of that pipeline).
+    dev = [tuple(torch.empty_like(x) for x in (job.q, job.k, job.v)) +
+           tuple(torch.empty_like(job.out) for _ in range(n_out)) for _ in range(2)]
+    host_out = [[pinned_like(job.out) for _ in range(n_out)] for _ in range(2)]
+    s_c = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def upload(dst, chunks):
+        for r0, c in chunks:
+            dst[r0:r0 + c.shape[0]].copy_(c, non_blocking=True)
+
+    def download(chunks, src):
+        for r0, c in chunks:
+            c.copy_(src[r0:r0 + c.shape[0]], non_blocking=True)
+
+    def run(n):
+        ev_in = [torch.cuda.Event() for _ in range(2)]
+        ev_done = [torch.cuda.Event() for _ in range(2)]
+        ev_out = [torch.cuda.Event() for _ in range(2)]
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0.record(s_c)
+        s_in.wait_event(t0)
+        for i in range(n):
+            b = i % 2
+            bq, bk, bv = dev[b][:3]
+            bo = dev[b][3:]
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_done[b])            # step i - 2 no longer reads this buffer set
+                upload(bq, host_in[0])
+                upload(bk, host_in[1])
+                upload(bv, host_in[2])
+                ev_in[b].record(s_in)
+            s_c.wait_event(ev_in[b])
+            if i >= 2:
+                s_c.wait_event(ev_out[b])                  # its outputs of step i - 2 are on the host
+            job.step(bq, bk, bv, bo[0], bo[1] if n_out == 2 else None)
+            ev_done[b].record(s_c)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[b])
+                for j in range(n_out):
+                    download(host_out[b][j], bo[j])
+                ev_out[b].record(s_out)
+        s_c.wait_event(ev_out[0])
+        if n > 1:
+            s_c.wait_event(ev_out[1])
+        t1.record(s_c)
+        torch.cuda.synchronize()
+        return t0.elapsed_time(t1) / n
+
+    run(2)
+    e2e_ms = max_over_ranks(run(steps), dist, "cuda")
+    h2d = sum(x.numel() * x.element_size() for x in (job.q, job.k, job.v))
+    d2h = job.out.numel() * job.out.element_size() * n_out
+    del dev, host_out, host_in
+    torch.cuda.empty_cache()
+    return {"value": world * w.suffix_tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "how": "pinned host buffers (1 GiB chunks); upload, compute and download of consecutive steps overlap "
+                   "(two device buffer sets, three streams); time of %d steps / %d" % (steps, steps)}
+
+
+# ---- the oracle as a timed CPU baseline ------------------------------------------------------------
+
+def oracle_sample_plan(w, flop_budget):
+    """Which part of a step the oracle is timed on: (request, KV head, query rows of the deep-layer pass)
+    units, median-length request first and then spread over the length distribution, until about
+    `flop_budget` algorithmic FLOPs are planned.  A unit is the shallow-layer pass (all suffix rows) and the
+    deep-layer pass (the first `rows` rows) of the query heads that share one KV head."""
+    R, G = w.num_requests, w.num_q_heads // w.num_kv_heads
+    order = np.argsort(w.suffix_lens, kind="stable")
     picks = [int(order[R // 2])] + [int(order[(j * 7919) % R]) for j in range(1, R)]
-    seen, ta, tf, fa, ff = [], 0.0, 0.0, 0.0, 0.0
+    plan, seen, used = [], set(), 0.0
     for i in picks:
         if i in seen:
             continue
-        a, f = oracle_one_request(w, workloads, oracle, i)
+        seen.add(i)
         n, m = w.suffix_lens[i], w.prefix_lens[w.req_prefix[i]]
-        seen.append(i)
-        ta, tf = ta + a, tf + f
-        fa += 4.0 * w.head_dim * w.num_q_heads * n * (m + n)
-        ff += 4.0 * w.head_dim * w.num_q_heads * (m + n) ** 2
-        if ta + tf >= budget_s:
+        N = m + n
+        fa = 4.0 * w.head_dim * G * n * N
+        left = max(flop_budget - used - fa, 0.25 * flop_budget)
+        rows = int(min(N, max(64, left // (4.0 * w.head_dim * G * N))))
+        plan.append((i, (7 * i) % w.num_kv_heads, rows))
+        used += fa + 4.0 * w.head_dim * G * rows * N
+        if used >= flop_budget:
             break
+    return plan
+
+
+def oracle_run_plan(w, workloads, oracle, plan):
+    """Runs the oracle on the planned units.  Returns (seconds shallow, seconds deep, FLOPs shallow, FLOPs deep)."""
+    G = w.num_q_heads // w.num_kv_heads
+    ta = tf = fa = ff = 0.0
+    for i, hk, rows in plan:
+        g = w.req_prefix[i]
+        m, n = w.prefix_lens[g], w.suffix_lens[i]
+        sub = workloads.Workload("sample", 1, G, 1, w.head_dim, w.dtype, 16, [m], [0], [n],
+                                 softmax_scale=w.softmax_scale, seed=w.seed + 131 * i + hk)
+        kc, vc = workloads.draw_prefix_kv(sub, 0, "cpu")
+        q, k, v = workloads.draw_full_qkv(sub, "cpu")
+        st = oracle.PagedPrefixStore(1, 1, w.head_dim, 16, sub.pages_needed())
+        qd, kd, vd = (workloads.to_f64(x) for x in (q, k, v))
+        pid, _, _ = st.put(1, workloads.to_f64(kc), workloads.to_f64(vc))
+        t0 = time.perf_counter()
+        oracle.attend(st, 0, [pid], sub.suffix_row_off, sub.suffix_lens, qd, kd, vd, w.softmax_scale)
+        t1 = time.perf_counter()
+        # deep-layer pass of the first `rows` query rows over all N keys (Eq. 2 row by row is independent)
+        oracle.attention(qd[:rows], kd, vd, w.softmax_scale)
+        t2 = time.perf_counter()
+        ta, tf = ta + (t1 - t0), tf + (t2 - t1)
+        fa += 4.0 * w.head_dim * G * n * (m + n)
+        ff += 4.0 * w.head_dim * G * rows * (m + n)
+    return ta, tf, fa, ff
+
+
+def oracle_step_estimate(w, depth, ta, tf, fa, ff):
+    """Whole-step time of the oracle: the sampled times scaled by the step's algorithmic FLOPs."""
     tot = 0.0
-    for j in range(R):
+    for j in range(w.num_requests):
         nj, mj = w.suffix_lens[j], w.prefix_lens[w.req_prefix[j]]
         fa_j = 4.0 * w.head_dim * w.num_q_heads * nj * (mj + nj)
         ff_j = 4.0 * w.head_dim * w.num_q_heads * (mj + nj) ** 2
@@ -252,9 +557,16 @@ def oracle_step_seconds(w, workloads, oracle, depth, budget_s=12.0):
             tot += ta * fa_j / fa + tf * ff_j / ff
         else:
             tot += int(depth[j]) * ta * fa_j / fa + (w.num_layers - int(depth[j])) * tf * ff_j / ff
-    desc = ("%d of %d requests (all heads), one shallow-layer and one deep-layer oracle pass each, %.1f s of "
-            "oracle work; step time = sampled time scaled by algorithmic FLOPs" % (len(seen), R, ta + tf))
-    return tot, desc, ta + tf
+    return tot
+
+
+def plan_text(w, plan, seconds):
+    units = ", ".join("request %d KV head %d (%d of %d deep-layer query rows)"
+                      % (i, hk, rows, w.prefix_lens[w.req_prefix[i]] + w.suffix_lens[i]) for i, hk, rows in plan[:3])
+    more = "" if len(plan) <= 3 else " and %d more" % (len(plan) - 3)
+    return ("%d (request, KV head) unit(s): %s%s; per unit one shallow-layer oracle pass (all suffix rows) and one "
+            "deep-layer pass (the stated rows, all keys), %.1f s of oracle work; step time = sampled time scaled "
+            "by algorithmic FLOPs" % (len(plan), units, more, seconds))
 
 
 def host_cores():
@@ -266,8 +578,20 @@ def host_cores():
         return len(os.sched_getaffinity(0))
 
 
+def config_keys(w, depth):
+    """The `config` object both arms print."""
+    return {"workload": w.name, "note": w.note, "layers": w.num_layers, "requests": w.num_requests,
+            "suffix_tokens": w.suffix_tokens,
+            "l2": "flushed before every timed step (256 MB write); the tensors of a step exceed L2",
+            "step": ("shallow-layer pass + deep-layer pass of the single layer"
+                     if w.num_layers == 1 else "all layers, per-request depths from the rule"),
+            "depth_min": int(min(depth)), "depth_max": int(max(depth)), "deep_layer_refresh": None}
+
+
 def run_reference(args, w):
-    """The oracle arm: the CPU oracle as it stands, timed on the host cores."""
+    """The oracle arm: the CPU oracle as it stands, timed on the host cores.  Every step (warm-up steps
+    included) runs the same bounded sample of the workload; `ms_per_step` is the measured time of that
+    sample, `value` the tokens/s of a whole step at the sampled rate."""
     import oracle
     from paper_2606_07571_b200 import workloads
     rank = int(os.environ.get("RANK", "0"))
@@ -275,37 +599,120 @@ def run_reference(args, w):
         return
     table = workloads.standin_depth_table(w.num_layers)
     depth = oracle.reuse_depth(w.req_prefix_len(), w.suffix_lens, table, w.num_layers)
-    for _ in range(min(args.warmup, 1)):
-        oracle_step_seconds(w, workloads, oracle, depth)
-    times, desc = [], ""
-    for _ in range(max(1, min(args.steps, 3))):
-        t, desc, _ = oracle_step_seconds(w, workloads, oracle, depth)
-        times.append(t)
-    sec = float(np.mean(times))
-    value = w.suffix_tokens / sec
-    cores = host_cores()
+    plan = oracle_sample_plan(w, args.ref_flops)
+    for _ in range(args.warmup):
+        oracle_run_plan(w, workloads, oracle, plan)
+    times, est = [], []
+    for _ in range(args.steps):
+        ta, tf, fa, ff = oracle_run_plan(w, workloads, oracle, plan)
+        times.append(ta + tf)
+        est.append(oracle_step_estimate(w, depth, ta, tf, fa, ff))
+    sec_sample, sec_step = float(np.mean(times)), float(np.mean(est))
+    value = w.suffix_tokens / sec_step
+    desc = plan_text(w, plan, sec_sample) + "; every step repeats this sample"
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": w.name, "note": w.note},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_sample * 1e3,
+            "ms_per_whole_step_extrapolated": sec_step * 1e3, "sample_fraction_of_step": sec_sample / sec_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_keys(w, depth),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": desc},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
+
+
+def measure_extras(job, name, flush, peaks):
+    """Off the per-step path: prefix put (scatter into page images), the profiler's similarity
+    reduction (Eq. 3) and the K/V projection into the store (Eq. 1), each on prefix 0."""
+    w, bc, workloads = job.w, job.bc, job.workloads
+    pid = [bc.lookup_prefix(key)[0] for key in job.keys]
+    es = 2 if w.dtype == torch.bfloat16 else 4
+    put_bytes = 4 * w.num_layers * w.prefix_lens[0] * w.num_kv_heads * w.head_dim * es
+    out = {"roofline_put": None, "roofline_similarity": None, "roofline_project": None}
+    if w.dtype == torch.bfloat16 and w.head_dim == 128:
+        m0, d_model = w.prefix_lens[0], w.num_q_heads * w.head_dim
+        hh, wk_, wv_ = workloads.draw_hidden_and_weights(m0, d_model, w.num_kv_heads, w.head_dim, 1, device="cuda")
+        ts = []
+        for i in range(8):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            bc.project_prefix_layer(pid[0], 0, hh, wk_, wv_)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        del hh, wk_, wv_
+        ms_proj = sorted(ts[3:])[len(ts[3:]) // 2]
+        proj_flops = 2.0 * m0 * d_model * 2 * w.num_kv_heads * w.head_dim
+        tf = proj_flops / (ms_proj * 1e-3) / 1e12
+        tr = traffic_of(name, "project")
+        out["roofline_project"] = {
+            "bound": "tensor", "kernel": "project_kv_kernel (project_prefix_layer of prefix 0, one layer)",
+            "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
+            "peak_source": peaks["source"] + " burst", "flops_per_launch": proj_flops, "ms_per_launch": ms_proj,
+            "d_model": d_model, "traffic": tr[0], "traffic_source": tr[1]}
+    if put_bytes >= (256 << 20):
+        # Timed last: every put of a fresh key evicts the oldest prefix (FIFO), the workload's own first.
+        kc, vc = workloads.draw_prefix_kv(w, 0, "cuda")
+        ts = []
+        sim_dev = torch.zeros(w.num_layers, dtype=torch.float32, device="cuda")
+        for i in range(5):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            bc.prefix_similarity_async(pid[0], kc, vc, sim_dev)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        ms_sim = sorted(ts[1:])[len(ts[1:]) // 2]
+        gbs = put_bytes / (ms_sim * 1e-3) / 1e9
+        tr = traffic_of(name, "similarity")
+        out["roofline_similarity"] = {
+            "bound": "hbm", "kernel": "kv_similarity_partial_kernel (prefix_similarity of prefix 0)",
+            "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+            "peak_source": peaks["source"], "bytes_per_launch": put_bytes, "ms_per_launch": ms_sim,
+            "traffic": tr[0], "traffic_source": tr[1]}
+        ts = []
+        for i in range(5):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            bc.put_prefix(0x7000000000000000 + i, kc, vc)
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        del kc, vc
+        ms_put = sorted(ts[1:])[len(ts[1:]) // 2]
+        gbs = put_bytes / (ms_put * 1e-3) / 1e9
+        tr = traffic_of(name, "put")
+        out["roofline_put"] = {
+            "bound": "hbm", "kernel": "scatter_prefix_kernel (put_prefix of prefix 0, all layers)",
+            "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+            "peak_source": peaks["source"], "bytes_per_launch": put_bytes, "ms_per_launch": ms_put,
+            "traffic": tr[0], "traffic_source": tr[1]}
+    return out
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="config2")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the put / similarity / projection launches")
+    ap.add_argument("--per-config", choices=("auto", "on", "off"), default="auto",
+                    help="also measure the other configurations and the small-suffix shapes (auto: when the "
+                         "default workload runs on one GPU)")
+    ap.add_argument("--cpu-flops", type=float, default=1.5e12, help="algorithmic FLOPs of the cpu_baseline sample")
+    ap.add_argument("--ref-flops", type=float, default=2.5e11,
+                    help="algorithmic FLOPs of the sample one step of --impl reference runs")
     ap.add_argument("--delta", type=int, default=0,
                     help="refresh interval of the deep layers' kept prefix K/V (Eq. 5); 0: recompute every step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    args.steps = max(args.steps, 1)
 
     from paper_2606_07571_b200 import workloads
     w = workloads.CONFIGS[args.workload]()
@@ -329,271 +736,71 @@ def main():
             entry.build()
     peaks = load_peaks()
     job = Job(w, local_rank, args.delta)
-    flops, depth = job.step_flops()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")       # 2x the 126 MB L2
 
-    # ---- device-resident timing: K steps, each preceded by an (untimed) L2 flush -------------
-    for _ in range(args.warmup):
-        flush.zero_()
-        job.step()
-    assert job.bc.device_status() == 0
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    launches0 = job.bc.launch_count()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    job.t = 1                                         # the timed steps are denoising steps 1 .. K
-    for a, b in ev:
-        flush.zero_()
-        a.record()
-        job.step()
-        b.record()
-    torch.cuda.synchronize()
-    launches = job.bc.launch_count() - launches0
-    per_step_ms = [a.elapsed_time(b) for a, b in ev]
-    step_ms = sum(per_step_ms) / args.steps
-    refresh_info = None
-    if job.delta > 0:
-        is_ref = [(t - 1) % job.delta == 0 for t in range(1, args.steps + 1)]
-        ref_ms = [m for m, r in zip(per_step_ms, is_ref) if r]
-        reu_ms = [m for m, r in zip(per_step_ms, is_ref) if not r]
-        flops = (len(ref_ms) * flops + len(reu_ms) * job.reuse_step_flops()) / args.steps   # mean FLOPs per step
-        refresh_info = {"delta": job.delta, "refresh_steps": len(ref_ms), "reuse_steps": len(reu_ms),
-                        "ms_refresh_step": sum(ref_ms) / max(1, len(ref_ms)),
-                        "ms_reuse_step": sum(reu_ms) / max(1, len(reu_ms)) if reu_ms else None}
-    # a short sustained stretch so that the clock sampler sees the kernels under load
-    t_end = time.time() + 0.6
-    while time.time() < t_end:
-        job.step()
-        torch.cuda.synchronize()
-    clocks = sampler.stop() if rank == 0 else None
-    assert job.bc.device_status() == 0
-    step_ms_max = max_over_ranks(step_ms, dist, "cuda")
-    if dist is not None:
-        dist.barrier()
-    value = world * w.suffix_tokens / (step_ms_max * 1e-3)
+    rec = measure_steps(job, args.workload, args.steps, args.warmup, flush, peaks, rank, local_rank, world, dist)
+    alone = measure_calls_alone(job, args.workload, flush, peaks)
+    # where no layer has every request on one path, the launch timed alone stands in
+    if rec["roofline"] is None:
+        rec["roofline"] = alone["attend_full"]
+    if rec["roofline_attend"] is None or alone["attend"]["bound"] == "hbm":
+        rec["roofline_attend"] = alone["attend"]
 
-    # ---- per-call timing for the roofline (CUDA events around the single kernel launch) ------
-    bc = job.bc
-    pid = [bc.lookup_prefix(key)[0] for key in job.keys]
-    req_pid = [pid[g] for g in w.req_prefix]
-    layer_mid = 0
-
-    def call_attend():
-        bc.attend(layer_mid, req_pid, w.suffix_row_off, w.suffix_lens, job.q, job.k, job.v, job.out, None,
-                  w.softmax_scale)
-
-    def call_full():
-        bc.attend_full(layer_mid, w.full_row_off, w.full_lens, job.q, job.k, job.v, job.out, None, w.softmax_scale)
-
-    iters = 10 if w.full_flops() < 5e13 else 3
-    call_attend(); call_full()
-    ms_attend = time_call(call_attend, iters, flush)
-    ms_full = time_call(call_full, iters, flush)
-    tf_attend = w.attend_flops() / (ms_attend * 1e-3) / 1e12
-    tf_full = w.full_flops() / (ms_full * 1e-3) / 1e12
-    peak = peaks["bf16_tflops"]
-    roofline = {"bound": "tensor", "kernel": "tc_attention_kernel (attend_full launch)", "achieved": tf_full,
-                "peak": peak, "unit": "TFLOP/s", "frac": tf_full / peak, "peak_source": peaks["source"] + " burst",
-                "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("full"),
-                "flops_per_launch": w.full_flops(), "ms_per_launch": ms_full}
-    roofline_attend = {"bound": "tensor", "kernel": "tc_attention_kernel (attend launch)", "achieved": tf_attend,
-                       "peak": peak, "unit": "TFLOP/s", "frac": tf_attend / peak,
-                       "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("attend"),
-                       "flops_per_launch": w.attend_flops(), "ms_per_launch": ms_attend}
-    call_attend()
-    if bc.last_attention_kernel() == 3:                    # the key-range kernel (BICACHE_KERNEL_KEY_RANGES)
-        # few query rows against a long cached prefix: the launch is bound by reading the prefix once
-        gbs = w.attend_bytes() / (ms_attend * 1e-3) / 1e9
-        # The same call replayed from a CUDA graph (ten calls per replay): what a serving loop that
-        # captures its steps sees, without the host time of the Python binding per call.  Only for
-        # prefixes larger than L2, where back-to-back calls still read the keys from HBM.
-        graph_ms = None
-        if w.attend_bytes() > (200 << 20):
-            try:
-                st = torch.cuda.Stream()
-                with torch.cuda.stream(st):
-                    call_attend()
-                    torch.cuda.synchronize()
-                    g = torch.cuda.CUDAGraph()
-                    with torch.cuda.graph(g, stream=st):
-                        for _ in range(10):
-                            call_attend()
-                    ts = []
-                    for _ in range(5):
-                        flush.zero_()
-                        flush.max()
-                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                        a.record(st)
-                        g.replay()
-                        b.record(st)
-                        torch.cuda.synchronize()
-                        ts.append(a.elapsed_time(b) / 10)
-                graph_ms = sorted(ts)[len(ts) // 2]
-            except Exception:                              # capture not available: the figure is left out
-                graph_ms = None
-        roofline_attend = {"bound": "hbm", "kernel": "tc_decode_kernel + merge_ranges_kernel (attend call)",
-                           "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                           "peak_source": peaks["source"], "bytes_per_launch": w.attend_bytes(),
-                           "ms_per_launch": ms_attend, "tflops": tf_attend,
-                           "graph_replay": (None if graph_ms is None else
-                                            {"ms_per_call": graph_ms, "calls_per_replay": 10,
-                                             "achieved": w.attend_bytes() / (graph_ms * 1e-3) / 1e9,
-                                             "frac": w.attend_bytes() / (graph_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}),
-                           "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("attend")}
-
-    # ---- end to end: host buffers, copies inside the timed region ------------------------------
     e2e = None
-    if not args.no_e2e and w.total_rows * w.num_q_heads * w.head_dim * 2 < (4 << 30):
-        hq, hk, hv = (x.to("cpu").pin_memory() for x in (job.q, job.k, job.v))
-        ho = torch.empty_like(hq).pin_memory()
-        ho2 = torch.empty_like(hq).pin_memory() if job.single_layer else None
-        dq, dk, dv = (torch.empty_like(x) for x in (job.q, job.k, job.v))
+    if not args.no_e2e:
+        e2e = measure_e2e(job, max(3, min(args.steps, 6 if rec["ms_per_step"] > 100 else 16)), world, dist)
 
-        # Two buffer sets and three streams: the upload of step i + 1 and the download of step i - 1
-        # run while step i computes (every step still uploads its own inputs and downloads its own
-        # outputs; the figure is the steady-state time per step of that pipeline).
-        dev = [(dq, dk, dv, torch.empty_like(job.out), torch.empty_like(job.out) if ho2 is not None else None),
-               (torch.empty_like(dq), torch.empty_like(dk), torch.empty_like(dv), torch.empty_like(job.out),
-                torch.empty_like(job.out) if ho2 is not None else None)]
-        host_out = [(ho, ho2), (torch.empty_like(ho).pin_memory(), torch.empty_like(ho).pin_memory() if ho2 is not None else None)]
-        s_c = torch.cuda.current_stream()
-        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
-
-        def e2e_run(n):
-            ev_in = [torch.cuda.Event() for _ in range(2)]
-            ev_done = [torch.cuda.Event() for _ in range(2)]
-            ev_out = [torch.cuda.Event() for _ in range(2)]
-            t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            t0.record(s_c)
-            s_in.wait_event(t0)
-            for i in range(n):
-                b = i % 2
-                bq, bk, bv, bo, bo2 = dev[b]
-                with torch.cuda.stream(s_in):
-                    if i >= 2:
-                        s_in.wait_event(ev_done[b])            # step i - 2 no longer reads this buffer set
-                    bq.copy_(hq, non_blocking=True)
-                    bk.copy_(hk, non_blocking=True)
-                    bv.copy_(hv, non_blocking=True)
-                    ev_in[b].record(s_in)
-                s_c.wait_event(ev_in[b])
-                if i >= 2:
-                    s_c.wait_event(ev_out[b])                  # its outputs of step i - 2 are on the host
-                job.step(bq, bk, bv, bo, bo2)
-                ev_done[b].record(s_c)
-                with torch.cuda.stream(s_out):
-                    s_out.wait_event(ev_done[b])
-                    host_out[b][0].copy_(bo, non_blocking=True)
-                    if bo2 is not None:
-                        host_out[b][1].copy_(bo2, non_blocking=True)
-                    ev_out[b].record(s_out)
-            s_c.wait_event(ev_out[0])
-            s_c.wait_event(ev_out[1])
-            t1.record(s_c)
-            torch.cuda.synchronize()
-            return t0.elapsed_time(t1) / n
-
-        e2e_run(3)
-        n_e2e = max(4, min(args.steps, 16))
-        e2e_ms = e2e_run(n_e2e)
-        e2e_ms = max_over_ranks(e2e_ms, dist, "cuda")
-        h2d = sum(x.numel() * x.element_size() for x in (hq, hk, hv))
-        d2h = ho.numel() * ho.element_size() * (2 if ho2 is not None else 1)
-        e2e = {"value": world * w.suffix_tokens / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "how": "pinned host buffers; upload, compute and download of consecutive steps overlap "
-                      "(two buffer sets, three streams); time of %d steps / %d" % (n_e2e, n_e2e)}
-
-    # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only) ---------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
-        sec, desc, _ = oracle_step_seconds(w, workloads, oracle, depth)
-        cpu = {"value": w.suffix_tokens / sec, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": desc}
+        plan = oracle_sample_plan(w, args.cpu_flops)
+        ta, tf, fa, ff = oracle_run_plan(w, workloads, oracle, plan)
+        sec = oracle_step_estimate(w, job.depth, ta, tf, fa, ff)
+        cpu = {"value": w.suffix_tokens / sec, "unit": UNIT, "cores": host_cores(), "kind": "oracle",
+               "sample": plan_text(w, plan, ta + tf)}
 
-    # ---- prefix store put (bandwidth-bound scatter into page images), off the per-step path ----
-    # Timed last: every put of a fresh key evicts the oldest prefix (FIFO), the workload's own first.
-    roofline_put = None
-    put_bytes = 4 * w.num_layers * w.prefix_lens[0] * w.num_kv_heads * w.head_dim * (2 if w.dtype == torch.bfloat16 else 4)
-    roofline_sim = None
-    # ---- prefix K/V projection into the store (Eq. 1), one layer of prefix 0, off the per-step path ----
-    roofline_proj = None
-    if w.dtype == torch.bfloat16 and w.head_dim == 128:
-        m0, d_model = w.prefix_lens[0], w.num_q_heads * w.head_dim
-        hh, wk_, wv_ = workloads.draw_hidden_and_weights(m0, d_model, w.num_kv_heads, w.head_dim, 1, device="cuda")
-        ts = []
-        for i in range(8):
-            flush.zero_()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            bc.project_prefix_layer(pid[0], 0, hh, wk_, wv_)
-            b.record()
-            torch.cuda.synchronize()
-            ts.append(a.elapsed_time(b))
-        del hh, wk_, wv_
-        ms_proj = sorted(ts[3:])[len(ts[3:]) // 2]
-        proj_flops = 2.0 * m0 * d_model * 2 * w.num_kv_heads * w.head_dim
-        tf = proj_flops / (ms_proj * 1e-3) / 1e12
-        roofline_proj = {"bound": "tensor", "kernel": "project_kv_kernel (project_prefix_layer of prefix 0, one layer)",
-                         "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"],
-                         "peak_source": peaks["source"], "flops_per_launch": proj_flops, "ms_per_launch": ms_proj,
-                         "d_model": d_model, "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("project")}
-    if put_bytes >= (256 << 20):
-        kc, vc = workloads.draw_prefix_kv(w, 0, "cuda")
-        # profiler reduction (Eq. 3): cached prefix 0 against a reference K/V of the same shape; reads both once
-        ts = []
-        sim_dev = torch.zeros(w.num_layers, dtype=torch.float32, device="cuda")
-        for i in range(5):
-            flush.zero_()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            bc.prefix_similarity_async(pid[0], kc, vc, sim_dev)
-            b.record()
-            torch.cuda.synchronize()
-            ts.append(a.elapsed_time(b))
-        ms_sim = sorted(ts[1:])[len(ts[1:]) // 2]
-        gbs = put_bytes / (ms_sim * 1e-3) / 1e9
-        roofline_sim = {"bound": "hbm", "kernel": "kv_similarity_partial_kernel (prefix_similarity of prefix 0)",
-                        "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                        "peak_source": peaks["source"], "bytes_per_launch": put_bytes, "ms_per_launch": ms_sim,
-                        "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("similarity")}
-        ts = []
-        for i in range(5):
-            flush.zero_()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            bc.put_prefix(0x7000000000000000 + i, kc, vc)
-            b.record()
-            torch.cuda.synchronize()
-            ts.append(a.elapsed_time(b))
-        del kc, vc
-        ms_put = sorted(ts[1:])[len(ts[1:]) // 2]
-        gbs = put_bytes / (ms_put * 1e-3) / 1e9
-        roofline_put = {"bound": "hbm", "kernel": "scatter_prefix_kernel (put_prefix of prefix 0, all layers)",
-                        "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
-                        "peak_source": peaks["source"], "bytes_per_launch": put_bytes, "ms_per_launch": ms_put,
-                        "traffic": NCU_TRAFFIC_BYTES.get(args.workload, {}).get("put")}
+    extras = {"roofline_put": None, "roofline_similarity": None, "roofline_project": None}
+    if not args.no_extras:
+        extras = measure_extras(job, args.workload, flush, peaks)
+    job.close()
+
+    # ---- the other configurations and the small-suffix shapes, a few steps each ----------------------
+    per_config = None
+    want_sub = args.per_config == "on" or (args.per_config == "auto" and args.workload == DEFAULT_WORKLOAD
+                                           and world == 1 and args.delta == 0)
+    if want_sub and rank == 0 and world == 1:
+        per_config = []
+        for name, steps in PER_CONFIG:
+            if name == args.workload:
+                continue
+            sj = Job(workloads.CONFIGS[name](), local_rank)
+            r = measure_steps(sj, name, steps, 3, flush, peaks, 0, local_rank, 1, None)
+            a = measure_calls_alone(sj, name, flush, peaks)
+            sj.close()
+            per_config.append({"workload": sj.w.name, "value": r["value"], "unit": UNIT, "ms_per_step": r["ms_per_step"],
+                               "steps": steps, "warmup": 3, "tflops": r["tflops"], "gpu_launches": r["gpu_launches"],
+                               "roofline": r["roofline"] or a["attend_full"],
+                               "roofline_attend": r["roofline_attend"] or a["attend"],
+                               "calls_alone": a, "clocks": r["clocks"], "config": r["config"]})
+        for name in SMALL_SUFFIX:
+            sw = workloads.CONFIGS[name]()
+            sj = Job(sw, local_rank)
+            sampler = ClockSampler(local_rank)
+            sampler.start()
+            a = measure_calls_alone(sj, name, flush, peaks)
+            clocks = sampler.stop()
+            sj.close()
+            per_config.append({"workload": sw.name, "note": sw.note, "roofline_attend": a["attend"], "clocks": clocks})
 
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": step_ms_max, "higher_is_better": True, "scaling": "weak",
+        line = {"metric": METRIC, "value": rec["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": rec["ms_per_step"], "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16" if w.dtype == torch.bfloat16 else "f32", "data": "synthetic",
-                "config": {"workload": w.name, "note": w.note, "layers": w.num_layers, "requests": w.num_requests,
-                           "suffix_tokens": w.suffix_tokens, "l2": "flushed between timed steps (256 MB write)",
-                           "step": ("shallow-layer pass + deep-layer pass of the single layer"
-                                    if job.single_layer else "all layers, per-request depths from the rule"),
-                           "depth_min": int(min(depth)), "depth_max": int(max(depth)),
-                           "deep_layer_refresh": refresh_info},
-                "tflops": flops / (step_ms_max * 1e-3) / 1e12, "step_flops": flops,
-                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-                "roofline": roofline, "roofline_attend": roofline_attend, "roofline_put": roofline_put,
-                "roofline_similarity": roofline_sim, "roofline_project": roofline_proj,
-                "cpu_baseline": cpu}
+                "config": rec["config"], "tflops": rec["tflops"], "step_flops": rec["step_flops"],
+                "clocks": rec["clocks"], "e2e": e2e, "gpu_launches": rec["gpu_launches"],
+                "roofline": rec["roofline"], "roofline_attend": rec["roofline_attend"], "calls_alone": alone,
+                "roofline_put": extras["roofline_put"], "roofline_similarity": extras["roofline_similarity"],
+                "roofline_project": extras["roofline_project"], "cpu_baseline": cpu, "per_config": per_config}
         print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
