@@ -7,7 +7,7 @@
  * library is the attention of one denoising step under that scheme:
  *
  *   bicache_put_prefix    KV store H: insert the prefix KVs of all L layers
- *                         (Sec. 5.2 "On a miss ... stores them in H[k]"),
+ *                         under the prefix's key (Sec. 5.2, the miss case),
  *                         paged, with first-in-first-out eviction
  *                         (implementation appendix).
  *   bicache_reuse_depth   r = shared-prefix tokens / all tokens of the input
@@ -95,7 +95,11 @@ typedef struct {
 size_t bicache_pool_bytes(const bicache_config* cfg);
 
 /* Workspace needed to run batches of at most max_requests requests and max_total_rows query rows
- * per call (bicache_attend: suffix rows; bicache_attend_full: all rows). */
+ * per call (bicache_attend: suffix rows; bicache_attend_full: all rows).  Besides the fixed areas
+ * (status, partial results of key-split calls, page-list staging) it holds the schedule arena: the
+ * device-resident descriptions of the batches seen so far, kept so that the layers of a denoising step
+ * and the following steps upload nothing.  The size asked for holds min(2 L + 4, 72) schedules of the
+ * largest batch; a smaller workspace still works as long as two schedules fit (more uploads). */
 size_t bicache_workspace_bytes(const bicache_config* cfg, int64_t max_total_rows, int32_t max_requests);
 
 /* Create a context.  Clears the library's part of the workspace with a synchronous memset.
@@ -180,15 +184,16 @@ int32_t bicache_attend_full(bicache_ctx* ctx, int32_t layer, int32_t R,
                             void* out, int64_t out_row_stride, float* lse_out,
                             float softmax_scale, void* stream);
 
-/* Layer-partitioned dispatch of one layer (Sec. 5.2: "for each layer l, determine whether l <= b"):
+/* Layer-partitioned dispatch of one layer (Sec. 5.2: the per-layer test l <= b of the online phase):
  * request i, whose whole input (prefix rows, then suffix rows) occupies seqlen[i] = N_i rows from
  * row_off[i], goes through bicache_attend on its suffix rows (row_off[i] + m_i, N_i - m_i rows, m_i =
  * length of prefix_id[i]) if layer < depth[i] and prefix_id[i] >= 0, and through bicache_attend_full
  * on all its rows otherwise.  depth, prefix_id, row_off, seqlen: host arrays of length R; the reusing
  * requests' prefix ids must be grouped.  Tensor arguments as for bicache_attend.  Outputs: suffix rows
  * of reusing requests, all rows of the others.  INVALID if a reusing request is shorter than its
- * prefix; other errors as for the two calls.  The reuse half is validated and enqueued first; if
- * the second half then fails validation the first has already been enqueued. */
+ * prefix; other errors as for the two calls.  Both halves are validated and their schedules placed in the
+ * workspace before either is launched: an error the host can detect (bad arguments, an evicted id, a
+ * schedule that does not fit the workspace) leaves out and lse_out untouched and launches no kernel. */
 int32_t bicache_attend_layer(bicache_ctx* ctx, int32_t layer, int32_t R, const int32_t* depth,
                              const int32_t* prefix_id, const int64_t* row_off, const int32_t* seqlen,
                              const void* q, const void* k, const void* v,
@@ -251,8 +256,9 @@ int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_
  *                                                                                       (Eq. 5, recompute).
  * depth, shared_id, private_id, row_off, seqlen: host arrays of length R (requests of one shared prefix
  * need not be contiguous here: the call groups them).  Tensor arguments, outputs and errors as for
- * bicache_attend_layer; INVALID also if t < 1 or delta < 1.  Everything is validated before the first
- * launch. */
+ * bicache_attend_layer; INVALID also if t < 1 or delta < 1.  Everything the host can check (both
+ * attention calls and the ids, lengths and strides of the layer updates) is checked, and both schedules
+ * are placed in the workspace, before the first launch. */
 int32_t bicache_attend_step(bicache_ctx* ctx, int32_t layer, int32_t t, int32_t delta, int32_t R,
                             const int32_t* depth, const int32_t* shared_id, const int32_t* private_id,
                             const int64_t* row_off, const int32_t* seqlen,
@@ -313,8 +319,12 @@ int32_t bicache_set_wait_budget(bicache_ctx* ctx, int64_t sm_cycles);
  * running, a process whose GPU budget was handed out before this library was loaded.  The calls
  * above need a context and a caller-allocated workspace; this one needs neither.  Its scratch
  * (partial results of BICACHE_STATIC_KEY_SPLITS key ranges) is a fixed array inside the library's
- * device image: about 8.1 MB on every GPU that loads the library, held until the process exits.
- * The call allocates and frees nothing, on the host or on the device.
+ * device image: 4096 x 4 x 129 floats = 8,454,144 bytes (8.06 MiB) on every GPU that runs this entry
+ * point, held until the process exits.  The call itself allocates and frees nothing, on the host or
+ * on the device.  One caveat for callers with a fixed memory budget: CUDA loads a library's device
+ * code lazily, so the FIRST call on a device is when the driver loads this entry point's module and
+ * backs the array; make that call at start-up, where an out-of-memory answer (BICACHE_ERR_CUDA) can
+ * still be handled, and count the 8.06 MiB into the budget.
  *
  * Computes what bicache_attend_full computes for a single request occupying rows 0..n_rows-1:
  * every row attends, without a mask, over all n_rows keys.  dtype: BICACHE_F32 or BICACHE_BF16;
@@ -324,7 +334,8 @@ int32_t bicache_set_wait_budget(bicache_ctx* ctx, int64_t sm_cycles);
  *   UNSUPPORTED  dtype or head_dim outside the list above
  *   INVALID      null pointers, bad strides or head counts
  * The first call on each device looks up the array's device address (a host-side set-up step that
- * enqueues nothing); make that first call before starting any stream capture.  All calls on a
+ * enqueues nothing and is cached in plain, unsynchronised host state: make the first call from one
+ * thread, before starting any stream capture, and do not call again on a device after resetting it).  All calls on a
  * device share the one array and every call overwrites the part it uses, so nothing has to be
  * cleared between calls - but two calls whose kernels may overlap on the GPU (different streams,
  * or different threads) race on it.  Issue them on one stream, or serialise them yourself. */
@@ -337,6 +348,12 @@ int32_t bicache_attend_full_static(int32_t dtype, int32_t num_q_heads, int32_t n
 
 /* Number of kernels this context has launched so far (for benchmarks' launch accounting). */
 int64_t bicache_launch_count(const bicache_ctx* ctx);
+
+/* Number of schedules this context has uploaded to the device so far.  A batch whose metadata
+ * (request offsets, lengths, prefix ids) equals that of an earlier call reuses the cached schedule, so
+ * in steady state a denoising step uploads none.  An upload goes through pinned host memory owned by
+ * the context and does not make the host wait for the stream. */
+int64_t bicache_schedule_uploads(const bicache_ctx* ctx);
 
 /* Which attention kernel the context's last attention call launched (for tests and benchmarks):
  * 0 none yet; BICACHE_KERNEL_SIMT the CUDA-core kernel (fp32, head dims other than 128, forced);

@@ -492,9 +492,9 @@ def attend_step(store, layer, t, delta, depth, shared_id, private_id, full_row_o
 def kv_similarity(store, prefix_id, k_ref, v_ref):
     """sim_l = cos(KV$_l, KVref_l) for every layer l (Eq. 3).
 
-    "Each KV representation is flattened into a single vector" (Sec. 4.1
-    footnote) is read as: layer l's keys and values of all prefix positions
-    and heads, concatenated, form one vector per side.  k_ref, v_ref:
+    The flattening the Sec. 4.1 footnote speaks of is read as: layer l's keys
+    and values of all prefix positions and heads, concatenated, form one vector
+    per side.  k_ref, v_ref:
     [L, m, Hkv, D].  A zero vector on either side gives similarity 0.
     """
     k_ref = np.asarray(k_ref, dtype=np.float64)

@@ -28,7 +28,7 @@ EXPORTED = [
     "bicache_read_prefix_layer", "bicache_project_prefix_layer",
     "bicache_prefix_similarity", "bicache_prefix_similarity_async", "bicache_depth_from_similarity",
     "bicache_build_depth_table",
-    "bicache_hash_tokens", "bicache_device_status", "bicache_set_wait_budget", "bicache_launch_count", "bicache_last_attention_kernel", "bicache_last_error",
+    "bicache_hash_tokens", "bicache_device_status", "bicache_set_wait_budget", "bicache_launch_count", "bicache_schedule_uploads", "bicache_last_attention_kernel", "bicache_last_error",
 ]
 
 
@@ -125,6 +125,8 @@ def load_library():
     lib.bicache_set_wait_budget.argtypes = [vp, C.c_int64]
     lib.bicache_launch_count.restype = C.c_int64
     lib.bicache_launch_count.argtypes = [vp]
+    lib.bicache_schedule_uploads.restype = C.c_int64
+    lib.bicache_schedule_uploads.argtypes = [vp]
     lib.bicache_last_error.restype = C.c_char_p
     lib.bicache_last_error.argtypes = [vp]
     lib.bicache_last_attention_kernel.restype = C.c_int32
@@ -155,7 +157,7 @@ class BiCache:
     """One library context plus the torch-owned device buffers it needs."""
 
     def __init__(self, num_layers, num_q_heads, num_kv_heads, head_dim, num_pages, dtype,
-                 max_total_rows, max_requests, device=0, page_size=16, free_order=None):
+                 max_total_rows, max_requests, device=0, page_size=16, free_order=None, workspace_bytes=None):
         self.lib = load_library()
         if not torch.cuda.is_available():
             raise RuntimeError("BiCache needs a CUDA device; there is no CPU path")
@@ -166,6 +168,8 @@ class BiCache:
                      _dtype_code(dtype), device)
         pool_bytes = self.lib.bicache_pool_bytes(C.byref(cfg))
         ws_bytes = self.lib.bicache_workspace_bytes(C.byref(cfg), int(max_total_rows), int(max_requests))
+        if workspace_bytes is not None:          # a caller that sizes the workspace itself
+            ws_bytes = int(workspace_bytes)
         if pool_bytes == 0 or ws_bytes == 0:
             raise BiCacheError(ERR_INVALID, "bicache_pool_bytes/workspace_bytes")
         # torch allocations are 512-byte aligned
@@ -369,6 +373,9 @@ class BiCache:
     def launch_count(self):
         return int(self.lib.bicache_launch_count(self.ctx))
 
+    def schedule_uploads(self):
+        return int(self.lib.bicache_schedule_uploads(self.ctx))
+
 
 STATIC_MAX_ROW_HEADS = 4096
 
@@ -382,6 +389,11 @@ def attend_full_static(q, k, v, out, scale=None):
     lib = load_library()
     n, Hq, D = q.shape
     Hkv = k.shape[1]
+    for t in (q, k, v, out):
+        assert t.is_cuda and t.device == q.device and t.dtype == q.dtype and t.dim() == 3
+        assert t.stride(2) == 1 and t.stride(1) == D, "heads must be dense within a row"
+    assert k.shape == v.shape == (n, Hkv, D) and out.shape == q.shape
+    assert q.device.index == torch.cuda.current_device(), "the call runs on the current device"
     scale = D ** -0.5 if scale is None else scale
     return lib.bicache_attend_full_static(_dtype_code(q.dtype), Hq, Hkv, D, n, q.data_ptr(), k.data_ptr(),
                                           v.data_ptr(), q.stride(0), k.stride(0), out.data_ptr(), out.stride(0),

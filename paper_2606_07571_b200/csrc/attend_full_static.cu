@@ -27,10 +27,15 @@ constexpr int kStaticFloatsPerPartial = kStaticMaxD + 1;              // o[D] an
 constexpr size_t kStaticScratchFloats = (size_t)kStaticMaxRowHeads * kStaticSplits * kStaticFloatsPerPartial;
 constexpr int kMaxDevices = 64;
 
-// The scratch itself: about 8.1 MB of every GPU that loads this library, until the process exits.
+// The scratch itself: 4096 x 4 x 129 floats = 8,454,144 bytes (8.06 MiB) of every GPU that loads this
+// library's device code, until the process exits.  With CUDA's lazy module loading the device code of
+// this file is loaded, and the array backed, by the first call on a device (the address lookup below).
 // In host code this name is only a handle; the device address comes from cudaGetSymbolAddress.
 static __device__ __align__(256) float g_static_scratch[kStaticScratchFloats];
 
+// Device address of the array, per device, looked up once.  Plain host state: not synchronised between
+// host threads, and stale after a cudaDeviceReset of that device (a process that resets a device must not
+// call this entry point on it again).
 float* g_scratch_addr[kMaxDevices] = {nullptr};
 
 template <typename T> __device__ __forceinline__ float ld_elem(const T* p);

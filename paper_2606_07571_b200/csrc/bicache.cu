@@ -28,7 +28,9 @@ using namespace bicache;
 
 namespace {
 
-constexpr int kNumSlots = 4;                 // cached schedules kept on the device
+constexpr bool kTiledAttend = false;          // row tiles shared by the requests of a prefix group
+constexpr int kMaxCached = 192;              // cached schedules a context keeps track of
+constexpr int kStageBufs = 4;                // pinned staging buffers of the schedule uploads
 constexpr size_t kStatusBytes = 256;
 constexpr int kTargetCtas = 296;             // two waves of 148 SMs: aim of the key split
 constexpr long long kMaxPartialRowHeads = (long long)kTargetCtas * kTileRows;
@@ -42,19 +44,23 @@ struct PrefixEntry {
   std::vector<int32_t> pages;
 };
 
+// A schedule kept on the device: where it lives in the schedule arena and what batch it describes.
 struct CachedSchedule {
   bool valid = false;
-  uint64_t last_use = 0;
+  uint64_t last_use = 0;                      // API-call counter of the last use (entries of the running call are pinned)
+  uint64_t hash = 0;                          // of (kind, R, row_off, seqlen, prefix_id)
   int kind = 0;                               // 0 attend, 1 attend_full, 2 attend through the key-range kernel
   std::vector<int32_t> prefix_id;
   std::vector<int64_t> row_off;
   std::vector<int32_t> seqlen;
   int num_items = 0, num_splits = 1, tiles_per_split = 0, total_tokens = 0;
-  size_t reqs_off = 0, pages_off = 0, items_off = 0;   // byte offsets inside the slot
+  size_t off = 0, bytes = 0;                  // place in the arena
+  size_t reqs_off = 0, pages_off = 0, items_off = 0;   // byte offsets inside the schedule
   size_t ditems_off = 0;                      // kind 2: the key-range items
   size_t tok_rows_off = 0;                    // kind 2: row of every token of the call
   size_t tok_span_off = 0;                    // kind 2: the tokens of every token's own request
   int num_ditems = 0;
+  int num_tiles = 0;                          // tiled schedules: row tiles behind the items (at ditems_off)
 };
 constexpr int kMaxDecodeItems = 4096;
 constexpr int kMaxDecodeTokens = 4096;        // tokens of a call served by the key-range kernel
@@ -79,14 +85,23 @@ struct bicache_ctx {
   // workspace carving
   int* d_status = nullptr;
   long long wait_cycles = 0;       // SM-clock budget of the device-side waits (0: the kernel's default)
-  char* d_slots = nullptr;
-  size_t slot_bytes = 0;
+  // Schedule arena (the part of the workspace behind the fixed areas): schedules are placed one after
+  // the other and the place wraps around, evicting what it overwrites.
+  char* d_arena = nullptr;
+  size_t arena_bytes = 0, arena_head = 0;
+  // Pinned staging for the uploads, so that a schedule miss never makes the host wait for the stream.
+  char* h_stage[kStageBufs] = {nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t stage_ev[kStageBufs] = {nullptr, nullptr, nullptr, nullptr};
+  bool stage_used[kStageBufs] = {false, false, false, false};
+  size_t stage_bytes = 0;
+  int stage_next = 0;
+  int64_t schedule_uploads = 0;
   float* d_part_o = nullptr;
   float* d_part_lse = nullptr;
   long long part_capacity_rowheads = 0;
   int* d_put_pages = nullptr;                                     // page list staging for put_prefix
-  CachedSchedule slots[kNumSlots];
-  uint64_t use_counter = 0;
+  std::vector<CachedSchedule> sched;                              // kMaxCached entries
+  uint64_t use_counter = 0;                                       // one tick per API call
   int64_t launches = 0;
   int sm_count = 148;
   std::string last_error;
@@ -114,17 +129,24 @@ bool sane(const bicache_config* c) {
          c->num_q_heads % c->num_kv_heads == 0 && c->num_pages >= 1 && c->head_dim >= 1;
 }
 
-size_t slot_bytes_for(const bicache_config* c, int64_t max_rows, int32_t max_req) {
+// Upper bound of the bytes of one schedule of at most max_req requests and max_rows rows.
+size_t schedule_bytes_for(const bicache_config* c, int64_t max_rows, int32_t max_req) {
   const int G = c->num_q_heads / c->num_kv_heads;
   const long long tiles = (max_rows * G + kTileRows - 1) / kTileRows + max_req;
   const long long max_items = std::max<long long>(tiles * c->num_kv_heads, 1) + 2LL * kTargetCtas;
   return align_up((size_t)max_req * sizeof(ReqMeta) + 16, 256) +
          align_up((size_t)c->num_pages * sizeof(int) + 16, 256) +
          align_up((size_t)max_items * sizeof(WorkItem) + 16, 256) +
-         align_up((size_t)kMaxDecodeItems * sizeof(dec::DecodeItem) + 16, 256) +
+         std::max(align_up((size_t)kMaxDecodeItems * sizeof(dec::DecodeItem) + 16, 256),
+                  align_up((size_t)tiles * sizeof(RowTile) + 16, 256)) +
          align_up((size_t)kMaxDecodeTokens * sizeof(long long) + 16, 256) +
          align_up((size_t)kMaxDecodeTokens * sizeof(int2) + 16, 256);
 }
+
+// How many schedules of the largest size the arena is asked to hold: a denoising step alternates
+// between at most two schedules per distinct depth value (the reuse set and the recompute set change
+// membership only there), and a set's schedule is smaller than the bound above, so this holds a step.
+int arena_schedules_for(const bicache_config* c) { return std::min(2 * c->num_layers + 4, 72); }
 
 size_t partial_bytes_for(const bicache_config* c) {
   return align_up((size_t)kMaxPartialRowHeads * (c->head_dim + 1) * sizeof(float), 256);
@@ -174,19 +196,84 @@ bool encode_map(CUtensorMap* m, const void* base, long long rows, int heads, lon
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Build (or find) the device-resident schedule for this batch.  Returns the slot index or -1.
-int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id, const int64_t* row_off,
-                     const int32_t* seqlen, cudaStream_t stream, int* status) {
+uint64_t fnv1a(uint64_t h, const void* data, size_t bytes) {
+  const unsigned char* p = static_cast<const unsigned char*>(data);
+  for (size_t i = 0; i < bytes; ++i) h = (h ^ p[i]) * 0x100000001b3ull;
+  return h;
+}
+
+// A pinned staging buffer of at least `bytes` bytes whose previous upload has completed.
+char* staging_buffer(bicache_ctx* ctx, size_t bytes, int* index) {
+  if (bytes > ctx->stage_bytes) {
+    // grow: rare (the first batches of a context); every upload in flight must finish first
+    for (int i = 0; i < kStageBufs; ++i) {
+      if (ctx->stage_used[i]) cudaEventSynchronize(ctx->stage_ev[i]);
+      ctx->stage_used[i] = false;
+      if (ctx->h_stage[i]) cudaFreeHost(ctx->h_stage[i]);
+      ctx->h_stage[i] = nullptr;
+    }
+    const size_t want = align_up(bytes + bytes / 2, 4096);
+    for (int i = 0; i < kStageBufs; ++i)
+      if (cudaHostAlloc(reinterpret_cast<void**>(&ctx->h_stage[i]), want, cudaHostAllocDefault) != cudaSuccess) {
+        ctx->h_stage[i] = nullptr;
+        ctx->stage_bytes = 0;
+        return nullptr;
+      }
+    ctx->stage_bytes = want;
+  }
+  const int i = ctx->stage_next;
+  ctx->stage_next = (i + 1) % kStageBufs;
+  if (ctx->stage_used[i]) cudaEventSynchronize(ctx->stage_ev[i]);   // kStageBufs uploads ago: long done
+  *index = i;
+  return ctx->h_stage[i];
+}
+
+// Room for `bytes` in the schedule arena: schedules follow one another and the place wraps around;
+// what the new schedule would overwrite is dropped from the cache, except schedules of the running API
+// call (they are about to be launched), which are stepped over.  Returns the offset or (size_t)-1.
+size_t arena_place(bicache_ctx* ctx, size_t bytes) {
+  bytes = align_up(bytes, 256);
+  if (bytes > ctx->arena_bytes) return (size_t)-1;
+  size_t head = ctx->arena_head;
+  for (int attempt = 0; attempt < 8; ++attempt) {
+    if (head + bytes > ctx->arena_bytes) head = 0;
+    bool moved = false;
+    for (CachedSchedule& c : ctx->sched) {
+      if (!c.valid || c.off >= head + bytes || c.off + c.bytes <= head) continue;
+      if (c.last_use == ctx->use_counter) {               // pinned: try behind it
+        head = c.off + c.bytes;
+        moved = true;
+        break;
+      }
+      c.valid = false;
+    }
+    if (!moved) {
+      ctx->arena_head = head + bytes;
+      return head;
+    }
+  }
+  return (size_t)-1;
+}
+
+// Build (or find) the device-resident schedule for this batch.  Returns its index in ctx->sched or -1.
+// `tiled`: kind 0 on the tensor path - the query rows of a prefix group are packed into row tiles.
+int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int R, const int32_t* prefix_id,
+                     const int64_t* row_off, const int32_t* seqlen, cudaStream_t stream, int* status) {
   *status = BICACHE_OK;
-  ctx->use_counter++;
-  for (int s = 0; s < kNumSlots; ++s) {
-    CachedSchedule& c = ctx->slots[s];
-    if (!c.valid || c.kind != kind || (int)c.seqlen.size() != R) continue;
+  const int key_kind = kind + (tiled ? 8 : 0);
+  uint64_t hash = fnv1a(0xcbf29ce484222325ull, &key_kind, sizeof(key_kind));
+  hash = fnv1a(hash, &R, sizeof(R));
+  hash = fnv1a(hash, row_off, sizeof(int64_t) * R);
+  hash = fnv1a(hash, seqlen, sizeof(int32_t) * R);
+  if (kind != 1) hash = fnv1a(hash, prefix_id, sizeof(int32_t) * R);
+  for (size_t s = 0; s < ctx->sched.size(); ++s) {
+    CachedSchedule& c = ctx->sched[s];
+    if (!c.valid || c.hash != hash || c.kind != key_kind || (int)c.seqlen.size() != R) continue;
     if (std::memcmp(c.row_off.data(), row_off, sizeof(int64_t) * R) != 0) continue;
     if (std::memcmp(c.seqlen.data(), seqlen, sizeof(int32_t) * R) != 0) continue;
     if (kind != 1 && std::memcmp(c.prefix_id.data(), prefix_id, sizeof(int32_t) * R) != 0) continue;
     c.last_use = ctx->use_counter;
-    return s;
+    return (int)s;
   }
   const int Hkv = ctx->cfg.num_kv_heads, G = ctx->cfg.num_q_heads / Hkv;
   std::vector<ReqMeta> reqs(R);
@@ -246,6 +333,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
     }
   }
   std::vector<WorkItem> items;
+  std::vector<RowTile> tiles;
   std::vector<dec::DecodeItem> ditems;
   if (kind == 2) {
     // Key-range kernel (few query rows against long cached prefixes).  Row space: all requests of a
@@ -279,7 +367,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
     for (const Group& g : groups) {
       if (g.n <= 0) continue;
       const ReqMeta& r0m = reqs[g.first];
-      const int tiles = (r0m.m + 63) / 64, tps = (tiles + sp - 1) / sp;
+      const int ktiles = (r0m.m + 63) / 64, tps = (ktiles + sp - 1) / sp;
       for (int s = 0; s < sp; ++s) {
         const int kb = s * tps * 64;
         const int kc = std::max(0, std::min(r0m.m - kb, tps * 64));
@@ -311,25 +399,86 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
     num_splits = sp;                                       // what the merge kernel combines
     tiles_per_split = 0;
   }
-  items.reserve((size_t)unsplit_items * num_splits);
-  for (int sp = 0; sp < (kind == 2 ? 1 : num_splits); ++sp) {
-    const size_t first = items.size();
+  if (tiled && num_splits == 1) {
+    // Row tiles of up to 256 packed rows.  The requests of a prefix group (consecutive requests with the
+    // same cached prefix) share tiles: a tile is a list of segments, each a run of one request's packed
+    // rows, so that a staged prefix tile serves the rows of several requests and ragged suffixes do
+    // not leave tile rows empty.  Segments start on multiples of `seg_align` rows (what the 8-row TMA
+    // boxes of the Q tile need); a request without a cached prefix gets tiles of its own.
+    const int seg_align = (8 % G == 0) ? 8 : 1;
+    std::vector<int> tile_cost;                            // key tiles of every row tile
+    RowTile cur = RowTile{};
+    int fill = 0, cur_cost = 0;
+    auto flush = [&]() {
+      if (cur.nseg > 0) {
+        cur.nrows = cur.seg[cur.nseg - 1].begin + cur.seg[cur.nseg - 1].count;
+        tiles.push_back(cur);
+        tile_cost.push_back(cur_cost);
+      }
+      cur = RowTile{};
+      fill = 0;
+      cur_cost = 0;
+    };
     for (int i = 0; i < R; ++i) {
       if (reqs[i].n <= 0) continue;
-      const int prow = reqs[i].n * G;
-      for (int hk = 0; hk < Hkv; ++hk)
-        for (int r0 = 0; r0 < prow; r0 += kTileRows) items.push_back(WorkItem{i, hk, r0, sp});
+      const bool joins = cur.nseg > 0 && reqs[i].m > 0 && prefix_id[i] == prefix_id[cur.seg[0].req];
+      if (!joins) flush();
+      int prow = 0, left = reqs[i].n * G;
+      while (left > 0) {
+        if (cur.nseg == kMaxSegs || fill >= kTileRows) flush();
+        if (cur.nseg == 0) {
+          cur.m = reqs[i].m;
+          cur.page_off = reqs[i].page_off;
+          cur_cost = (reqs[i].m + kTileKeys - 1) / kTileKeys;
+        }
+        const int take = std::min(left, kTileRows - fill);
+        cur.seg[cur.nseg++] = RowSeg{i, prow, fill, take};
+        cur_cost += (reqs[i].n + kTileKeys - 1) / kTileKeys;
+        fill = (int)align_up((size_t)(fill + take), (size_t)seg_align);
+        prow += take;
+        left -= take;
+      }
     }
-    // Longest key range first (the tail of the launch is then made of short items); items of one
-    // KV head and request stay adjacent so that concurrently running CTAs share K/V tiles in L2.
-    std::stable_sort(items.begin() + first, items.end(), [&](const WorkItem& a, const WorkItem& b) {
-      const int ka = reqs[a.req].m + reqs[a.req].n, kb = reqs[b.req].m + reqs[b.req].n;
-      return ka > kb;
+    flush();
+    // Items in the order (run of tiles with one prefix, KV head, tile): CTAs that run side by side then
+    // read the same cached K/V tiles and share them in L2.  Then longest key range first (in steps of
+    // four key tiles, so that neighbours mostly stay neighbours): the tail of the launch is made of
+    // short items.
+    items.reserve(tiles.size() * Hkv);
+    for (size_t t0 = 0; t0 < tiles.size();) {
+      size_t t1 = t0 + 1;
+      while (t1 < tiles.size() && tiles[t1].m > 0 && tiles[t1].page_off == tiles[t0].page_off && tiles[t1].m == tiles[t0].m)
+        ++t1;
+      for (int hk = 0; hk < Hkv; ++hk)
+        for (size_t tI = t0; tI < t1; ++tI) items.push_back(WorkItem{(int)tI, hk, 0, 0});
+      t0 = t1;
+    }
+    std::stable_sort(items.begin(), items.end(), [&](const WorkItem& a, const WorkItem& b) {
+      return tile_cost[a.req] / 4 > tile_cost[b.req] / 4;
     });
+  } else {
+    tiled = false;
+    items.reserve((size_t)unsplit_items * num_splits);
+    for (int sp = 0; sp < (kind == 2 ? 1 : num_splits); ++sp) {
+      const size_t first = items.size();
+      for (int i = 0; i < R; ++i) {
+        if (reqs[i].n <= 0) continue;
+        const int prow = reqs[i].n * G;
+        for (int hk = 0; hk < Hkv; ++hk)
+          for (int r0 = 0; r0 < prow; r0 += kTileRows) items.push_back(WorkItem{i, hk, r0, sp});
+      }
+      // Longest key range first (the tail of the launch is then made of short items); items of one
+      // KV head and request stay adjacent so that concurrently running CTAs share K/V tiles in L2.
+      std::stable_sort(items.begin() + first, items.end(), [&](const WorkItem& a, const WorkItem& b) {
+        const int ka = reqs[a.req].m + reqs[a.req].n, kb = reqs[b.req].m + reqs[b.req].n;
+        return ka > kb;
+      });
+    }
   }
   const size_t reqs_off = 0;
   const size_t pages_off = align_up(reqs_off + reqs.size() * sizeof(ReqMeta) + 16, 256);
   const size_t items_off = align_up(pages_off + pages.size() * sizeof(int) + 16, 256);
+  // the key-range items (kind 2) or the row tiles (tiled schedules) follow the items
   const size_t ditems_off = align_up(items_off + items.size() * sizeof(WorkItem) + 16, 256);
   std::vector<long long> tok_rows;
   std::vector<int2> tok_span;                              // per token: the call's tokens of its own request
@@ -342,37 +491,61 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
         tok_span.push_back(make_int2(reqs[i].tok_off, reqs[i].tok_off + reqs[i].n));
       }
   }
-  const size_t tok_rows_off = align_up(ditems_off + ditems.size() * sizeof(dec::DecodeItem) + 16, 256);
+  const size_t second_bytes = kind == 2 ? ditems.size() * sizeof(dec::DecodeItem) : tiles.size() * sizeof(RowTile);
+  const size_t tok_rows_off = align_up(ditems_off + second_bytes + 16, 256);
   const size_t tok_span_off = align_up(tok_rows_off + tok_rows.size() * sizeof(long long) + 16, 256);
   const size_t total = tok_span_off + tok_span.size() * sizeof(int2);
-  if (total > ctx->slot_bytes || (int)ditems.size() > kMaxDecodeItems || (long long)tok_rows.size() > kMaxDecodeTokens) {
+  if ((int)ditems.size() > kMaxDecodeItems || (long long)tok_rows.size() > kMaxDecodeTokens) {
+    *status = fail(ctx, BICACHE_ERR_NOMEM, "batch too large for the key-range kernel's tables");
+    return -1;
+  }
+  int victim = -1;
+  for (size_t s = 0; s < ctx->sched.size(); ++s)
+    if (!ctx->sched[s].valid) { victim = (int)s; break; }
+  if (victim < 0) {                                        // every entry in use: drop the least recently used
+    victim = 0;
+    for (size_t s = 0; s < ctx->sched.size(); ++s)
+      if (ctx->sched[s].last_use < ctx->sched[victim].last_use) victim = (int)s;
+    if (ctx->sched[victim].last_use == ctx->use_counter) {
+      *status = fail(ctx, BICACHE_ERR_NOMEM, "workspace too small for this batch's schedule");
+      return -1;
+    }
+    ctx->sched[victim].valid = false;
+  }
+  const size_t place = arena_place(ctx, total);
+  if (place == (size_t)-1) {
     *status = fail(ctx, BICACHE_ERR_NOMEM, "workspace too small for this batch's schedule");
     return -1;
   }
-  int victim = 0;
-  for (int s = 0; s < kNumSlots; ++s) {
-    if (!ctx->slots[s].valid) { victim = s; break; }
-    if (ctx->slots[s].last_use < ctx->slots[victim].last_use) victim = s;
-  }
-  std::vector<char> blob(total, 0);
-  if (!reqs.empty()) std::memcpy(blob.data() + reqs_off, reqs.data(), reqs.size() * sizeof(ReqMeta));
-  if (!pages.empty()) std::memcpy(blob.data() + pages_off, pages.data(), pages.size() * sizeof(int));
-  if (!items.empty()) std::memcpy(blob.data() + items_off, items.data(), items.size() * sizeof(WorkItem));
-  if (!ditems.empty()) std::memcpy(blob.data() + ditems_off, ditems.data(), ditems.size() * sizeof(dec::DecodeItem));
-  if (!tok_rows.empty()) std::memcpy(blob.data() + tok_rows_off, tok_rows.data(), tok_rows.size() * sizeof(long long));
-  if (!tok_span.empty()) std::memcpy(blob.data() + tok_span_off, tok_span.data(), tok_span.size() * sizeof(int2));
-  CachedSchedule& c = ctx->slots[victim];
+  CachedSchedule& c = ctx->sched[victim];
   c.valid = false;
   if (total > 0) {
-    // Pageable source: the runtime stages it before returning, so `blob` may die with this scope.
-    cudaError_t e = cudaMemcpyAsync(ctx->d_slots + (size_t)victim * ctx->slot_bytes, blob.data(), total,
-                                    cudaMemcpyHostToDevice, stream);
+    int sb = 0;
+    char* blob = staging_buffer(ctx, total, &sb);
+    if (!blob) {
+      *status = fail(ctx, BICACHE_ERR_NOMEM, "no pinned host memory for the schedule upload");
+      return -1;
+    }
+    if (!reqs.empty()) std::memcpy(blob + reqs_off, reqs.data(), reqs.size() * sizeof(ReqMeta));
+    if (!pages.empty()) std::memcpy(blob + pages_off, pages.data(), pages.size() * sizeof(int));
+    if (!items.empty()) std::memcpy(blob + items_off, items.data(), items.size() * sizeof(WorkItem));
+    if (!ditems.empty()) std::memcpy(blob + ditems_off, ditems.data(), ditems.size() * sizeof(dec::DecodeItem));
+    if (!tiles.empty()) std::memcpy(blob + ditems_off, tiles.data(), tiles.size() * sizeof(RowTile));
+    if (!tok_rows.empty()) std::memcpy(blob + tok_rows_off, tok_rows.data(), tok_rows.size() * sizeof(long long));
+    if (!tok_span.empty()) std::memcpy(blob + tok_span_off, tok_span.data(), tok_span.size() * sizeof(int2));
+    cudaError_t e = cudaMemcpyAsync(ctx->d_arena + place, blob, total, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->stage_ev[sb], stream);
     if (e != cudaSuccess) {
       *status = fail(ctx, BICACHE_ERR_CUDA, std::string("schedule upload: ") + cudaGetErrorString(e));
       return -1;
     }
+    ctx->stage_used[sb] = true;
+    ctx->schedule_uploads++;
   }
-  c.kind = kind;
+  c.kind = key_kind;
+  c.hash = hash;
+  c.off = place;
+  c.bytes = align_up(total, 256);
   c.prefix_id.assign(prefix_id ? prefix_id : nullptr, prefix_id ? prefix_id + R : nullptr);
   c.row_off.assign(row_off, row_off + R);
   c.seqlen.assign(seqlen, seqlen + R);
@@ -381,6 +554,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
   c.tok_rows_off = tok_rows_off;
   c.tok_span_off = tok_span_off;
   c.num_ditems = (int)ditems.size();
+  c.num_tiles = (int)tiles.size();
   c.num_splits = num_splits;
   c.tiles_per_split = tiles_per_split;
   c.total_tokens = (int)tok;
@@ -393,13 +567,34 @@ int prepare_schedule(bicache_ctx* ctx, int kind, int R, const int32_t* prefix_id
 }
 
 void drop_schedules(bicache_ctx* ctx) {
-  for (int s = 0; s < kNumSlots; ++s) ctx->slots[s].valid = false;
+  for (CachedSchedule& c : ctx->sched) c.valid = false;
 }
 
-int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const int32_t* prefix_id,
-                  const int64_t* row_off, const int32_t* seqlen, const void* q, const void* k, const void* v,
-                  int64_t q_row_stride, int64_t kv_row_stride, void* out, int64_t out_row_stride,
-                  float* lse_out, float softmax_scale, void* stream_) {
+// The pinned staging buffers and their events (the only non-heap host resources of a context).
+void destroy_host_resources(bicache_ctx* ctx) {
+  for (int i = 0; i < kStageBufs; ++i) {
+    if (ctx->stage_ev[i]) cudaEventDestroy(ctx->stage_ev[i]);
+    if (ctx->h_stage[i]) cudaFreeHost(ctx->h_stage[i]);
+    ctx->stage_ev[i] = nullptr;
+    ctx->h_stage[i] = nullptr;
+  }
+}
+
+// One attention call, validated and with its schedule on the device, not yet launched.
+struct PreparedCall {
+  bool empty = true;           // nothing to launch
+  int entry = -1;              // index in ctx->sched
+  bool key_ranges = false, use_tensor = false;
+  TcTensorMaps maps;
+};
+
+// Everything the host can check, then the schedule (found in the cache or built and uploaded) and the
+// tensor maps.  Launches no kernel and writes no output.
+int prepare_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const int32_t* prefix_id,
+                      const int64_t* row_off, const int32_t* seqlen, const void* q, const void* k, const void* v,
+                      int64_t q_row_stride, int64_t kv_row_stride, void* out, int64_t out_row_stride,
+                      float* lse_out, float softmax_scale, void* stream_, PreparedCall* pc) {
+  *pc = PreparedCall();
   if (!ctx) return BICACHE_ERR_INVALID;
   if (ctx->host_only) return fail(ctx, BICACHE_ERR_UNSUPPORTED, "host-only context has no device path");
   const bicache_config& cfg = ctx->cfg;
@@ -444,12 +639,12 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   if (total == 0) return BICACHE_OK;
 
   // the tensor-core kernels take the row maximum before scaling, which needs a positive scale
-  const bool use_tensor = ctx->tensor_ok && ctx->path != BICACHE_PATH_SIMT && softmax_scale > 0.f;
+  pc->use_tensor = ctx->tensor_ok && ctx->path != BICACHE_PATH_SIMT && softmax_scale > 0.f;
   // Few query rows per prefix group against a long cached prefix (block-query decoding): the
   // bandwidth-bound regime, served by the key-range kernel.  Conditions: every request has a cached
   // prefix of at least 1024 tokens and at most 128 packed rows per KV head (a request with more fills
   // the general kernel's tiles by itself), and the call's tokens fit the kernel's tables.
-  bool key_ranges = kind == 0 && use_tensor;
+  bool key_ranges = kind == 0 && pc->use_tensor;
   if (key_ranges) {
     const int G = cfg.num_q_heads / cfg.num_kv_heads;
     for (int i = 0; i < R && key_ranges; ++i) {
@@ -460,22 +655,57 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
     if (total > kMaxDecodeTokens) key_ranges = false;
   }
   int st = BICACHE_OK;
-  int slot = -1;
+  int entry = -1;
   if (key_ranges) {
-    slot = prepare_schedule(ctx, 2, R, prefix_id, row_off, seqlen, stream, &st);
-    if (slot < 0) {                                      // does not fit the schedule slot: the general path
+    entry = prepare_schedule(ctx, 2, false, R, prefix_id, row_off, seqlen, stream, &st);
+    if (entry < 0) {                                     // does not fit: the general path
       key_ranges = false;
       ctx->last_error.clear();
     }
   }
-  if (slot < 0) slot = prepare_schedule(ctx, kind, R, prefix_id, row_off, seqlen, stream, &st);
-  if (slot < 0) return st;
-  const CachedSchedule& c = ctx->slots[slot];
-  char* base = ctx->d_slots + (size_t)slot * ctx->slot_bytes;
+  if (entry < 0)
+    entry = prepare_schedule(ctx, kind, kind == 0 && pc->use_tensor && kTiledAttend, R, prefix_id, row_off, seqlen,
+                             stream, &st);
+  if (entry < 0) return st;
+  pc->entry = entry;
+  pc->key_ranges = key_ranges;
+  if (pc->use_tensor && !key_ranges) {
+    // rows the tensors are known to have: up to the end of the last request
+    long long rows_total = 0;
+    for (int i = 0; i < R; ++i) rows_total = std::max<long long>(rows_total, row_off[i] + seqlen[i]);
+    const int G = cfg.num_q_heads / cfg.num_kv_heads;
+    TcTensorMaps& maps = pc->maps;
+    maps.q_tma = (128 % G == 0) ? 1 : 0;
+    maps.q8_tma = (8 % G == 0) ? 1 : 0;
+    bool okm = encode_map(&maps.k, k, rows_total, cfg.num_kv_heads, kv_row_stride, 1, 128) &&
+               encode_map(&maps.v, v, rows_total, cfg.num_kv_heads, kv_row_stride, 1, 128) &&
+               encode_map(&maps.q, q, rows_total, cfg.num_q_heads, q_row_stride, maps.q_tma ? G : 1,
+                          maps.q_tma ? 128 / G : 128) &&
+               encode_map(&maps.q8, q, rows_total, cfg.num_q_heads, q_row_stride, maps.q8_tma ? G : 1,
+                          maps.q8_tma ? 8 / G : 8);
+    maps.o_tma = (32 % G == 0) ? 1 : 0;
+    okm = okm && encode_map(&maps.o, out, rows_total, cfg.num_q_heads, out_row_stride, maps.o_tma ? G : 1,
+                            maps.o_tma ? 32 / G : 32);
+    if (!okm) return fail(ctx, BICACHE_ERR_CUDA, "tensor map encoding failed");
+  }
+  pc->empty = false;
+  return BICACHE_OK;
+}
+
+// The kernel launches of a prepared call.
+int launch_attention(bicache_ctx* ctx, const PreparedCall& pc, int32_t layer, const void* q, const void* k,
+                     const void* v, int64_t q_row_stride, int64_t kv_row_stride, void* out, int64_t out_row_stride,
+                     float* lse_out, float softmax_scale, void* stream_) {
+  if (pc.empty) return BICACHE_OK;
+  const bicache_config& cfg = ctx->cfg;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const CachedSchedule& c = ctx->sched[pc.entry];
+  char* base = ctx->d_arena + c.off;
   ScheduleView sv;
   sv.reqs = reinterpret_cast<const ReqMeta*>(base + c.reqs_off);
   sv.pages = reinterpret_cast<const int*>(base + c.pages_off);
   sv.items = reinterpret_cast<const WorkItem*>(base + c.items_off);
+  sv.tiles = c.num_tiles > 0 ? reinterpret_cast<const RowTile*>(base + c.ditems_off) : nullptr;
   sv.num_items = c.num_items;
   sv.num_splits = c.num_splits;
   sv.tiles_per_split = c.tiles_per_split;
@@ -491,7 +721,7 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   t.out_stride = out_row_stride;
   t.Hq = cfg.num_q_heads;
   t.Hkv = cfg.num_kv_heads;
-  t.D = D;
+  t.D = cfg.head_dim;
   t.layer = layer;
   t.scale = softmax_scale;
   t.part_o = ctx->d_part_o;
@@ -500,28 +730,14 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   const PoolView pool = pool_view(ctx);
 
   cudaError_t e;
-  ctx->last_kernel = key_ranges ? BICACHE_KERNEL_KEY_RANGES : use_tensor ? BICACHE_KERNEL_TENSOR : BICACHE_KERNEL_SIMT;
-  if (key_ranges) {
+  ctx->last_kernel = pc.key_ranges ? BICACHE_KERNEL_KEY_RANGES : pc.use_tensor ? BICACHE_KERNEL_TENSOR : BICACHE_KERNEL_SIMT;
+  if (pc.key_ranges) {
     e = launch_tc_decode(reinterpret_cast<const dec::DecodeItem*>(base + c.ditems_off), c.num_ditems,
                          reinterpret_cast<const long long*>(base + c.tok_rows_off),
                          reinterpret_cast<const int2*>(base + c.tok_span_off), sv.pages, pool, t, ctx->d_status,
                          ctx->wait_cycles, stream);
-  } else if (use_tensor) {
-    // rows the tensors are known to have: up to the end of the last request
-    long long rows_total = 0;
-    for (int i = 0; i < R; ++i) rows_total = std::max<long long>(rows_total, row_off[i] + seqlen[i]);
-    const int G = cfg.num_q_heads / cfg.num_kv_heads;
-    TcTensorMaps maps;
-    maps.q_tma = (128 % G == 0) ? 1 : 0;
-    bool okm = encode_map(&maps.k, k, rows_total, cfg.num_kv_heads, kv_row_stride, 1, 128) &&
-               encode_map(&maps.v, v, rows_total, cfg.num_kv_heads, kv_row_stride, 1, 128) &&
-               encode_map(&maps.q, q, rows_total, cfg.num_q_heads, q_row_stride, maps.q_tma ? G : 1,
-                          maps.q_tma ? 128 / G : 128);
-    maps.o_tma = (32 % G == 0) ? 1 : 0;
-    okm = okm && encode_map(&maps.o, out, rows_total, cfg.num_q_heads, out_row_stride, maps.o_tma ? G : 1,
-                            maps.o_tma ? 32 / G : 32);
-    if (!okm) return fail(ctx, BICACHE_ERR_CUDA, "tensor map encoding failed");
-    e = launch_tc_attention(sv, pool, t, ctx->d_status, ctx->sm_count, maps, ctx->wait_cycles, stream);
+  } else if (pc.use_tensor) {
+    e = launch_tc_attention(sv, pool, t, ctx->d_status, ctx->sm_count, pc.maps, ctx->wait_cycles, stream);
   } else if (cfg.dtype == BICACHE_F32) {
     simt_attention_kernel<float><<<c.num_items, kSimtWarps * 32, 0, stream>>>(sv, pool, t);
     e = cudaGetLastError();
@@ -531,7 +747,7 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   }
   ctx->launches++;
   if (e != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("attention launch: ") + cudaGetErrorString(e));
-  if (key_ranges) {
+  if (pc.key_ranges) {
     e = launch_merge_ranges(t, reinterpret_cast<const long long*>(base + c.tok_rows_off), c.num_splits, stream);
     ctx->launches++;
     if (e != cudaSuccess) return fail(ctx, BICACHE_ERR_CUDA, std::string("merge launch: ") + cudaGetErrorString(e));
@@ -548,6 +764,19 @@ int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const in
   return BICACHE_OK;
 }
 
+int run_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, const int32_t* prefix_id,
+                  const int64_t* row_off, const int32_t* seqlen, const void* q, const void* k, const void* v,
+                  int64_t q_row_stride, int64_t kv_row_stride, void* out, int64_t out_row_stride,
+                  float* lse_out, float softmax_scale, void* stream) {
+  if (ctx) ctx->use_counter++;
+  PreparedCall pc;
+  const int st = prepare_attention(ctx, kind, layer, R, prefix_id, row_off, seqlen, q, k, v, q_row_stride,
+                                   kv_row_stride, out, out_row_stride, lse_out, softmax_scale, stream, &pc);
+  if (st != BICACHE_OK) return st;
+  return launch_attention(ctx, pc, layer, q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                          softmax_scale, stream);
+}
+
 }  // namespace
 
 extern "C" {
@@ -560,7 +789,7 @@ size_t bicache_pool_bytes(const bicache_config* cfg) {
 
 size_t bicache_workspace_bytes(const bicache_config* cfg, int64_t max_total_rows, int32_t max_requests) {
   if (!sane(cfg) || max_total_rows < 0 || max_requests < 0) return 0;
-  return kStatusBytes + kNumSlots * slot_bytes_for(cfg, max_total_rows, max_requests) +
+  return kStatusBytes + (size_t)arena_schedules_for(cfg) * schedule_bytes_for(cfg, max_total_rows, max_requests) +
          partial_bytes_for(cfg) + align_up((size_t)cfg->num_pages * sizeof(int) + 16, 256);
 }
 
@@ -579,7 +808,7 @@ int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
     if ((reinterpret_cast<uintptr_t>(cfg->k_pool) & 255) || (reinterpret_cast<uintptr_t>(cfg->v_pool) & 255) ||
         (reinterpret_cast<uintptr_t>(cfg->workspace) & 255))
       return BICACHE_ERR_INVALID;
-    if (cfg->workspace_bytes < kStatusBytes + part + put_pages + kNumSlots * slot_bytes_for(cfg, 0, 0))
+    if (cfg->workspace_bytes < kStatusBytes + part + put_pages + 2 * schedule_bytes_for(cfg, 0, 0))
       return BICACHE_ERR_NOMEM;
   }
   std::vector<int32_t> order(cfg->num_pages);
@@ -614,12 +843,20 @@ int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
   ctx->d_part_lse = ctx->d_part_o + (size_t)kMaxPartialRowHeads * cfg->head_dim;
   ctx->part_capacity_rowheads = kMaxPartialRowHeads;
   ctx->d_put_pages = reinterpret_cast<int*>(ws + kStatusBytes + part);
-  ctx->d_slots = ws + kStatusBytes + part + put_pages;
-  ctx->slot_bytes = (cfg->workspace_bytes - (kStatusBytes + part + put_pages)) / kNumSlots / 256 * 256;
+  ctx->d_arena = ws + kStatusBytes + part + put_pages;
+  ctx->arena_bytes = (cfg->workspace_bytes - (kStatusBytes + part + put_pages)) / 256 * 256;
+  ctx->sched.resize(kMaxCached);
+  for (int i = 0; i < kStageBufs; ++i)
+    if (cudaEventCreateWithFlags(&ctx->stage_ev[i], cudaEventDisableTiming) != cudaSuccess) {
+      destroy_host_resources(ctx);
+      delete ctx;
+      return BICACHE_ERR_CUDA;
+    }
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) == cudaSuccess && sms > 0)
     ctx->sm_count = sms;
   if (cudaMemset(ws, 0, kStatusBytes) != cudaSuccess) {
+    destroy_host_resources(ctx);
     delete ctx;
     return BICACHE_ERR_CUDA;
   }
@@ -628,6 +865,7 @@ int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
     if (e == cudaSuccess) e = configure_project_kv(&ctx->proj_pairs);
     if (e == cudaSuccess) e = configure_tc_decode();
     if (e != cudaSuccess) {
+      destroy_host_resources(ctx);
       delete ctx;
       return BICACHE_ERR_CUDA;
     }
@@ -644,6 +882,7 @@ int32_t bicache_destroy(bicache_ctx* ctx) {
   }
   cudaSetDevice(ctx->cfg.device);
   cudaError_t e = cudaDeviceSynchronize();
+  destroy_host_resources(ctx);
   delete ctx;
   return e == cudaSuccess ? BICACHE_OK : BICACHE_ERR_CUDA;
 }
@@ -1112,24 +1351,31 @@ int32_t bicache_attend_layer(bicache_ctx* ctx, int32_t layer, int32_t R, const i
       f_len.push_back(seqlen[i]);
     }
   }
-  // Validate both halves before launching either, so that an error leaves the outputs untouched.
+  // Both halves are validated and their schedules prepared before either is launched, so that an error
+  // the host can detect leaves the outputs untouched.
+  ctx->use_counter++;
+  PreparedCall pr, pf;
   if (!r_len.empty()) {
     for (size_t i = 1; i < r_pid.size(); ++i)
       if (r_pid[i] != r_pid[i - 1] &&
           std::find(r_pid.begin(), r_pid.begin() + i, r_pid[i]) != r_pid.begin() + i)
         return fail(ctx, BICACHE_ERR_INVALID, "requests of one prefix are not contiguous");
-    const int32_t st = run_attention(ctx, 0, layer, (int32_t)r_len.size(), r_pid.data(), r_off.data(), r_len.data(),
-                                     q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
-                                     softmax_scale, stream);
+    const int32_t st = prepare_attention(ctx, 0, layer, (int32_t)r_len.size(), r_pid.data(), r_off.data(),
+                                         r_len.data(), q, k, v, q_row_stride, kv_row_stride, out, out_row_stride,
+                                         lse_out, softmax_scale, stream, &pr);
     if (st != BICACHE_OK) return st;
   }
   if (!f_len.empty()) {
-    const int32_t st = run_attention(ctx, 1, layer, (int32_t)f_len.size(), nullptr, f_off.data(), f_len.data(),
-                                     q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
-                                     softmax_scale, stream);
+    const int32_t st = prepare_attention(ctx, 1, layer, (int32_t)f_len.size(), nullptr, f_off.data(), f_len.data(),
+                                         q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                                         softmax_scale, stream, &pf);
     if (st != BICACHE_OK) return st;
   }
-  return BICACHE_OK;
+  int32_t st = launch_attention(ctx, pr, layer, q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                                softmax_scale, stream);
+  if (st != BICACHE_OK) return st;
+  return launch_attention(ctx, pf, layer, q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                          softmax_scale, stream);
 }
 
 int32_t bicache_attend_step(bicache_ctx* ctx, int32_t layer, int32_t t, int32_t delta, int32_t R,
@@ -1175,30 +1421,40 @@ int32_t bicache_attend_step(bicache_ctx* ctx, int32_t layer, int32_t t, int32_t 
   }
   // requests of one prefix side by side, in order of first appearance
   std::stable_sort(reuse.begin(), reuse.end(), [](const Reuse& a, const Reuse& b) { return a.order < b.order; });
+  // Everything the host can check comes before the first launch: both attention calls are validated and
+  // prepared, and the arguments of the layer updates are the same tensors and strides.
+  ctx->use_counter++;
+  PreparedCall pr, pf;
+  std::vector<int32_t> r_pid, r_len;
+  std::vector<int64_t> r_off;
   if (!reuse.empty()) {
-    std::vector<int32_t> r_pid, r_len;
-    std::vector<int64_t> r_off;
     for (const Reuse& r : reuse) {
       r_pid.push_back(r.pid);
       r_off.push_back(r.off);
       r_len.push_back(r.len);
     }
-    const int32_t st = run_attention(ctx, 0, layer, (int32_t)r_len.size(), r_pid.data(), r_off.data(), r_len.data(),
-                                     q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
-                                     softmax_scale, stream);
+    const int32_t st = prepare_attention(ctx, 0, layer, (int32_t)r_len.size(), r_pid.data(), r_off.data(),
+                                         r_len.data(), q, k, v, q_row_stride, kv_row_stride, out, out_row_stride,
+                                         lse_out, softmax_scale, stream, &pr);
     if (st != BICACHE_OK) return st;
   }
   if (!f_len.empty()) {
-    const int32_t st = run_attention(ctx, 1, layer, (int32_t)f_len.size(), nullptr, f_off.data(), f_len.data(),
-                                     q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
-                                     softmax_scale, stream);
+    const int32_t st = prepare_attention(ctx, 1, layer, (int32_t)f_len.size(), nullptr, f_off.data(), f_len.data(),
+                                         q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                                         softmax_scale, stream, &pf);
     if (st != BICACHE_OK) return st;
   }
+  int32_t st = launch_attention(ctx, pr, layer, q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                                softmax_scale, stream);
+  if (st != BICACHE_OK) return st;
+  st = launch_attention(ctx, pf, layer, q, k, v, q_row_stride, kv_row_stride, out, out_row_stride, lse_out,
+                        softmax_scale, stream);
+  if (st != BICACHE_OK) return st;
   // refresh: the prefix rows just used become the kept K/V of this layer (Eq. 5, first case)
   for (size_t i = 0; i < upd_id.size(); ++i) {
     const char* kp = static_cast<const char*>(k) + upd_off[i] * kv_row_stride * ctx->esize;
     const char* vp = static_cast<const char*>(v) + upd_off[i] * kv_row_stride * ctx->esize;
-    const int32_t st = bicache_update_prefix_layer(ctx, upd_id[i], layer, kp, vp, kv_row_stride, stream);
+    st = bicache_update_prefix_layer(ctx, upd_id[i], layer, kp, vp, kv_row_stride, stream);
     if (st != BICACHE_OK) return st;
   }
   return BICACHE_OK;
@@ -1239,6 +1495,8 @@ int32_t bicache_set_wait_budget(bicache_ctx* ctx, int64_t sm_cycles) {
 }
 
 int64_t bicache_launch_count(const bicache_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int64_t bicache_schedule_uploads(const bicache_ctx* ctx) { return ctx ? ctx->schedule_uploads : 0; }
 
 int32_t bicache_last_attention_kernel(const bicache_ctx* ctx) { return ctx ? ctx->last_kernel : 0; }
 

@@ -29,11 +29,32 @@ struct WorkItem {
   int split;           // index of the key split this item covers (0 when the keys are not split)
 };
 
+// Row tiles (tensor-core `attend` schedules): up to 256 packed query rows that share every key tile of a
+// cached prefix.  A tile is a list of segments; segment k is rows [begin, begin + count) of the tile =
+// packed rows prow0 .. of request `req`.  All requests of a tile have the same cached prefix; after the
+// prefix tiles the tile walks the own rows of every segment's request in turn, and a query row takes part
+// only in the key tiles of its own request.  In a tiled schedule WorkItem::req is the index of the row tile.
+constexpr int kMaxSegs = 8;
+struct RowSeg {
+  int req;
+  int prow0;
+  int begin;
+  int count;
+};
+struct RowTile {
+  int m;               // cached prefix length of the tile's requests (0: a request without prefix, one segment)
+  int page_off;        // index of the prefix's first page id inside the schedule's page list
+  int nrows;           // end of the last segment
+  int nseg;
+  RowSeg seg[kMaxSegs];
+};
+
 // Device view of a schedule: everything a kernel needs besides the tensors.
 struct ScheduleView {
   const ReqMeta* reqs;
   const int* pages;          // concatenated page lists
   const WorkItem* items;
+  const RowTile* tiles;      // nullptr: items name (request, first packed row) themselves
   int num_items;
   int num_splits;            // > 1: item covers key tiles [split * tiles_per_split, (split + 1) * tiles_per_split)
   int tiles_per_split;       // key tiles: ceil(m/128) prefix tiles followed by ceil(n/128) own tiles

@@ -1279,6 +1279,8 @@ inline cudaError_t configure_tc_attention() {
 // q with a box of 32 packed rows (the rows of one softmax warp).
 struct TcTensorMaps {
   CUtensorMap q, k, v, o;
+  CUtensorMap q8;            // q again with a box of 8 packed rows (row tiles made of several segments)
+  int q8_tma;                // 0: G does not divide 8
   int q_tma;                 // 0: G does not divide 128, Q is gathered instead
   int o_tma;                 // 0: G does not divide 32, the output rows are copied out by the warps
 };

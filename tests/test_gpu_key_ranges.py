@@ -51,7 +51,7 @@ def _run(Hq, Hkv, prefix_lens, req_prefix, suffix_lens, reqs=None, shuffle=False
         mask[o:o + n] = True
     err = np.abs(got[mask] - ref[mask])
     assert err.max() <= 2e-2 and err.mean() <= 2e-3, (float(err.max()), float(err.mean()))
-    assert np.abs(got_lse[mask] - ref_lse[mask]).max() <= 1e-2
+    assert np.abs(got_lse[mask] - ref_lse[mask]).max() <= 1e-3
     assert (got[~mask] == 7.0).all() and (got_lse[~mask] == 7.0).all()          # untouched rows
     bc.close()
 

@@ -1,4 +1,4 @@
-"""The allocation-free entry point against the regular one.
+"""The allocation-free entry point against the regular one and against the oracle.
 
 bicache_attend_full_static serves callers that cannot allocate device memory (its scratch is a
 fixed array inside the library).  It must give what bicache_attend_full gives, call after call:
@@ -11,7 +11,8 @@ import pytest
 import torch
 
 import __graft_entry__ as entry
-from paper_2606_07571_b200 import binding
+import oracle
+from paper_2606_07571_b200 import binding, workloads
 
 pytestmark = pytest.mark.gpu
 
@@ -44,6 +45,50 @@ def test_static_entry_point_matches_regular_one_twice_in_a_row(dtype, tol):
         err = (out.double() - ref.double()).abs()
         assert torch.isfinite(out).all()
         assert err.max().item() <= tol and err.mean().item() <= tol / 10
+        # and against the definition itself (Eq. 2 over the request's own rows)
+        want, _ = oracle.attend_full([0], [n], *(workloads.to_f64(x) for x in (q, k, v)), D ** -0.5)
+        err = np.abs(workloads.to_f64(out) - want)
+        assert err.max() <= tol and err.mean() <= tol / 10
+
+
+@pytest.mark.parametrize("D", [32, 96])
+def test_static_entry_point_other_head_dims_match_the_oracle(D):
+    entry.build()
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(11 + D)
+    n, Hq, Hkv = 70, 6, 3
+    q = torch.randn(n, Hq, D, generator=gen, device="cuda").to(torch.bfloat16)
+    k = torch.randn(n, Hkv, D, generator=gen, device="cuda").to(torch.bfloat16)
+    v = torch.randn(n, Hkv, D, generator=gen, device="cuda").to(torch.bfloat16)
+    out = torch.full_like(q, 5.0)
+    assert binding.attend_full_static(q, k, v, out, D ** -0.5) == binding.OK
+    torch.cuda.synchronize()
+    want, _ = oracle.attend_full([0], [n], *(workloads.to_f64(x) for x in (q, k, v)), D ** -0.5)
+    err = np.abs(workloads.to_f64(out) - want)
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3
+
+
+def test_static_entry_point_capacity_edge():
+    """Exactly BICACHE_STATIC_MAX_ROW_HEADS row-heads are served (and correct), one more is refused."""
+    entry.build()
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    n, Hq, Hkv, D = 128, 32, 8, 64                                            # 128 * 32 = 4096 row-heads
+    assert n * Hq == binding.STATIC_MAX_ROW_HEADS
+    q = torch.randn(n, Hq, D, generator=gen, device="cuda").to(torch.bfloat16)
+    k = torch.randn(n, Hkv, D, generator=gen, device="cuda").to(torch.bfloat16)
+    v = torch.randn(n, Hkv, D, generator=gen, device="cuda").to(torch.bfloat16)
+    out = torch.full_like(q, 5.0)
+    assert binding.attend_full_static(q, k, v, out, D ** -0.5) == binding.OK
+    torch.cuda.synchronize()
+    want, _ = oracle.attend_full([0], [n], *(workloads.to_f64(x) for x in (q, k, v)), D ** -0.5)
+    err = np.abs(workloads.to_f64(out) - want)
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3
+    q1 = torch.zeros(4097, 1, D, dtype=torch.bfloat16, device="cuda")         # 4097 row-heads
+    out1 = torch.full_like(q1, 5.0)
+    assert binding.attend_full_static(q1, q1, q1, out1) == binding.ERR_NOMEM
+    torch.cuda.synchronize()
+    assert (out1 == 5.0).all()
 
 
 def test_static_entry_point_rejects_what_does_not_fit():
