@@ -28,7 +28,7 @@ using namespace bicache;
 
 namespace {
 
-constexpr bool kTiledAttend = false;          // row tiles shared by the requests of a prefix group
+constexpr bool kTiledAttend = true;           // row tiles shared by the requests of a prefix group
 constexpr int kMaxCached = 192;              // cached schedules a context keeps track of
 constexpr int kStageBufs = 4;                // pinned staging buffers of the schedule uploads
 constexpr size_t kStatusBytes = 256;
@@ -61,6 +61,7 @@ struct CachedSchedule {
   size_t tok_span_off = 0;                    // kind 2: the tokens of every token's own request
   int num_ditems = 0;
   int num_tiles = 0;                          // tiled schedules: row tiles behind the items (at ditems_off)
+  bool shared_tiles = false;                  // ... and some tile holds rows of several requests
 };
 constexpr int kMaxDecodeItems = 4096;
 constexpr int kMaxDecodeTokens = 4096;        // tokens of a call served by the key-range kernel
@@ -403,9 +404,11 @@ int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int R, const int32_
     // Row tiles of up to 256 packed rows.  The requests of a prefix group (consecutive requests with the
     // same cached prefix) share tiles: a tile is a list of segments, each a run of one request's packed
     // rows, so that a staged prefix tile serves the rows of several requests and ragged suffixes do
-    // not leave tile rows empty.  Segments start on multiples of `seg_align` rows (what the 8-row TMA
-    // boxes of the Q tile need); a request without a cached prefix gets tiles of its own.
-    const int seg_align = (8 % G == 0) ? 8 : 1;
+    // not leave tile rows empty.  Segments start on multiples of 8 rows (what the 8-row TMA boxes of the
+    // Q tile need), which is why requests share tiles only when the query heads of a KV group divide 8;
+    // a request without a cached prefix gets tiles of its own.
+    const bool pack = 8 % G == 0;                          // else every request keeps tiles of its own
+    const int seg_align = 8;
     std::vector<int> tile_cost;                            // key tiles of every row tile
     RowTile cur = RowTile{};
     int fill = 0, cur_cost = 0;
@@ -421,7 +424,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int R, const int32_
     };
     for (int i = 0; i < R; ++i) {
       if (reqs[i].n <= 0) continue;
-      const bool joins = cur.nseg > 0 && reqs[i].m > 0 && prefix_id[i] == prefix_id[cur.seg[0].req];
+      const bool joins = pack && cur.nseg > 0 && reqs[i].m > 0 && prefix_id[i] == prefix_id[cur.seg[0].req];
       if (!joins) flush();
       int prow = 0, left = reqs[i].n * G;
       while (left > 0) {
@@ -555,6 +558,8 @@ int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int R, const int32_
   c.tok_span_off = tok_span_off;
   c.num_ditems = (int)ditems.size();
   c.num_tiles = (int)tiles.size();
+  c.shared_tiles = false;
+  for (const RowTile& tl : tiles) c.shared_tiles = c.shared_tiles || tl.nseg > 1;
   c.num_splits = num_splits;
   c.tiles_per_split = tiles_per_split;
   c.total_tokens = (int)tok;
@@ -706,6 +711,7 @@ int launch_attention(bicache_ctx* ctx, const PreparedCall& pc, int32_t layer, co
   sv.pages = reinterpret_cast<const int*>(base + c.pages_off);
   sv.items = reinterpret_cast<const WorkItem*>(base + c.items_off);
   sv.tiles = c.num_tiles > 0 ? reinterpret_cast<const RowTile*>(base + c.ditems_off) : nullptr;
+  sv.shared_tiles = c.shared_tiles ? 1 : 0;
   sv.num_items = c.num_items;
   sv.num_splits = c.num_splits;
   sv.tiles_per_split = c.tiles_per_split;

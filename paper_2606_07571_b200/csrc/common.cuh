@@ -55,6 +55,7 @@ struct ScheduleView {
   const int* pages;          // concatenated page lists
   const WorkItem* items;
   const RowTile* tiles;      // nullptr: items name (request, first packed row) themselves
+  int shared_tiles;          // some row tile holds rows of more than one request
   int num_items;
   int num_splits;            // > 1: item covers key tiles [split * tiles_per_split, (split + 1) * tiles_per_split)
   int tiles_per_split;       // key tiles: ceil(m/128) prefix tiles followed by ceil(n/128) own tiles

@@ -53,11 +53,24 @@ constexpr long long kWaitCycles = 400000000LL;   // default budget of a bounded 
 
 // shared-memory layout (dynamic, 1024-byte aligned by hand): Q_A, Q_B, ring, output staging
 // (4 KB per softmax warp), barriers and item records
-struct ItemInfo {                        // one work item, written by the fetching lane of warp 9
+// One work item as the roles see it, written by warp 9.  Its query rows are `nseg` segments; segment k
+// is rows [begin, begin + count) of the item = packed rows prow0 .. of one request.  An item of a plain
+// schedule has one segment; an item of a tiled schedule has one per request with rows in its row tile
+// (all of one prefix group).  Key tiles: the cached prefix's, then every segment's request's own rows.
+struct SegInfo {
+  long long row_off;                     // first row of the request in q / k / v / out
+  int n;                                 // its rows: queries and own keys
+  int prow0, begin, count;
+  int tok_off;                           // its first token in the call's token numbering (key-split partials)
+  int tile_end;                          // key tiles of the item up to and including this request's own tiles
+};
+struct ItemInfo {
   int valid;                             // 0: the items are exhausted
-  int kv_head, row0, split;
-  int n, m, page_off, tok_off;
-  long long row_off;
+  int kv_head, split;
+  int m, page_off;
+  int nseg, nrows;                       // segments; end of the last one
+  int all_tiles;                         // ceil(m / 128) + sum over the segments of ceil(n / 128)
+  SegInfo seg[kMaxSegs];
 };
 struct alignas(8) Barriers {
   unsigned long long info_full[2];       // item record (double-buffered by item parity) is written
@@ -71,6 +84,12 @@ struct alignas(8) Barriers {
   unsigned long long o_done[2];          // the last O += P V of the item has completed (per query tile)
   unsigned long long o_free[2];          // the epilogue has read O out of TMEM (per query tile)
   unsigned long long drain;
+  // What the K loader found out about the key tiles, for the MMA warp and the softmax warps (which
+  // then need no per-tile arithmetic of their own): entry (t & 7) describes the t-th key tile the CTA
+  // has staged: keys | dense layout << 8 | (segment + 1) << 16 (segment -1: cached prefix).  A ring
+  // of 8 is deep enough: the loaders run at most two tiles ahead of the MMAs, the softmax less than
+  // one tile behind them.
+  int tile_meta[8];
   long long wait_cycles;                 // SM-clock budget of every wait; directly before abort_flag (mbar_wait reads it)
   int abort_flag;
   unsigned tmem_base;
@@ -403,17 +422,19 @@ __device__ __forceinline__ unsigned tile_chunk_offset(int r, int c16) {
   return (unsigned)((r >> 4) * kPageBytes) + page_chunk_offset(true, r & 15, c16, 256);
 }
 
-// Geometry of one work item, derived from its record.
+// Geometry of one work item, derived from its record.  n0 / end0: rows of the first segment's request
+// and the end of its own key tiles, kept in registers because most items have one segment and their
+// per-tile arithmetic must not touch shared memory.
 struct Geo {
-  int valid, m, n, prefix_tiles, tile_begin, T, b_active;
+  int valid, m, nseg, prefix_tiles, tile_begin, T, b_active, n0, end0;
 };
-__device__ __forceinline__ Geo read_geo(const ItemInfo* inf, int num_splits, int tiles_per_split, int G) {
+__device__ __forceinline__ Geo read_geo(const ItemInfo* inf, int num_splits, int tiles_per_split) {
   Geo g;
   g.valid = inf->valid;
   g.m = inf->m;
-  g.n = inf->n;
+  g.nseg = inf->nseg;
   g.prefix_tiles = (g.m + kTileKeys - 1) / kTileKeys;
-  const int all_tiles = g.prefix_tiles + (g.n + kTileKeys - 1) / kTileKeys;
+  const int all_tiles = inf->all_tiles;
   int tb = 0, te = all_tiles;
   if (num_splits > 1) {
     tb = min(all_tiles, inf->split * tiles_per_split);
@@ -421,33 +442,90 @@ __device__ __forceinline__ Geo read_geo(const ItemInfo* inf, int num_splits, int
   }
   g.tile_begin = tb;
   g.T = g.valid ? te - tb : 0;
-  g.b_active = inf->row0 + 128 < g.n * G;                   // the item has a second query tile
+  g.b_active = inf->nrows > 128;                            // the item has a second query tile
+  g.n0 = inf->seg[0].n;
+  g.end0 = inf->seg[0].tile_end;
   return g;
 }
 // The same, with every field broadcast from lane 0 of a converged warp: the compiler then knows the
 // values to be warp-uniform and keeps what derives from them (loop counters, MMA descriptors) in
 // the uniform datapath, which the MMA issue path needs to run at full rate.
-__device__ __forceinline__ Geo read_geo_uniform(const ItemInfo* inf, int num_splits, int tiles_per_split, int G) {
-  Geo g = read_geo(inf, num_splits, tiles_per_split, G);
+__device__ __forceinline__ Geo read_geo_uniform(const ItemInfo* inf, int num_splits, int tiles_per_split) {
+  Geo g = read_geo(inf, num_splits, tiles_per_split);
   g.valid = __shfl_sync(0xffffffffu, g.valid, 0);
   g.m = __shfl_sync(0xffffffffu, g.m, 0);
-  g.n = __shfl_sync(0xffffffffu, g.n, 0);
+  g.nseg = __shfl_sync(0xffffffffu, g.nseg, 0);
   g.prefix_tiles = __shfl_sync(0xffffffffu, g.prefix_tiles, 0);
   g.tile_begin = __shfl_sync(0xffffffffu, g.tile_begin, 0);
   g.T = __shfl_sync(0xffffffffu, g.T, 0);
   g.b_active = __shfl_sync(0xffffffffu, g.b_active, 0);
+  g.n0 = __shfl_sync(0xffffffffu, g.n0, 0);
+  g.end0 = __shfl_sync(0xffffffffu, g.end0, 0);
   return g;
 }
-// keys of key tile j of the item
-__device__ __forceinline__ int tile_keys(const Geo& g, int j) {
+// Key tile j of the item: which keys it holds.  seg < 0: keys key0 .. of the cached prefix; else own
+// rows key0 .. of segment seg's request.  Tiles of the prefix and of the first segment are resolved from
+// registers; only the later segments of a shared row tile read the item record.
+struct TileRef {
+  int seg, key0, cnt;
+};
+__device__ __forceinline__ TileRef tile_ref(const ItemInfo* inf, const Geo& g, int j) {
   const int jg = g.tile_begin + j;
-  return jg < g.prefix_tiles ? min(kTileKeys, g.m - jg * kTileKeys)
-                             : min(kTileKeys, g.n - (jg - g.prefix_tiles) * kTileKeys);
+  TileRef r;
+  if (jg < g.prefix_tiles) {
+    r.seg = -1;
+    r.key0 = jg * kTileKeys;
+    r.cnt = min(kTileKeys, g.m - r.key0);
+    return r;
+  }
+  if (jg < g.end0) {
+    r.seg = 0;
+    r.key0 = (jg - g.prefix_tiles) * kTileKeys;
+    r.cnt = min(kTileKeys, g.n0 - r.key0);
+    return r;
+  }
+  int k = 1, start = g.end0;
+  while (k + 1 < g.nseg && jg >= inf->seg[k].tile_end) {
+    start = inf->seg[k].tile_end;
+    ++k;
+  }
+  r.seg = k;
+  r.key0 = (jg - start) * kTileKeys;
+  r.cnt = min(kTileKeys, inf->seg[k].n - r.key0);
+  return r;
 }
-// a key tile is in the dense (TMA) layout iff it is a full tile of the request's own rows
-__device__ __forceinline__ bool tile_dense(const Geo& g, int j) {
+// The same for a converged warp, the result warp-uniform to the compiler as well: what comes from the
+// item record is broadcast from lane 0 (see read_geo_uniform).
+__device__ __forceinline__ TileRef tile_ref_uniform(const ItemInfo* inf, const Geo& g, int j) {
   const int jg = g.tile_begin + j;
-  return jg >= g.prefix_tiles && g.n - (jg - g.prefix_tiles) * kTileKeys >= kTileKeys;
+  TileRef r;
+  if (jg < g.end0) {
+    const bool pre = jg < g.prefix_tiles;
+    r.seg = pre ? -1 : 0;
+    r.key0 = (pre ? jg : jg - g.prefix_tiles) * kTileKeys;
+    r.cnt = min(kTileKeys, (pre ? g.m : g.n0) - r.key0);
+    return r;
+  }
+  r = tile_ref(inf, g, j);
+  r.seg = __shfl_sync(0xffffffffu, r.seg, 0);
+  r.key0 = __shfl_sync(0xffffffffu, r.key0, 0);
+  r.cnt = __shfl_sync(0xffffffffu, r.cnt, 0);
+  return r;
+}
+// Keys of key tile j of an item with ONE segment, from registers only; dense: a full tile of own rows.
+__device__ __forceinline__ int tile_keys_single(const Geo& g, int j, bool& dense) {
+  const int jg = g.tile_begin + j;
+  const bool pre = jg < g.prefix_tiles;
+  const int cnt = min(kTileKeys, pre ? g.m - jg * kTileKeys : g.n0 - (jg - g.prefix_tiles) * kTileKeys);
+  dense = !pre && cnt >= kTileKeys;
+  return cnt;
+}
+// the segment that holds row p of the item, or -1
+__device__ __forceinline__ int seg_of_row(const ItemInfo* inf, int nseg, int p) {
+  int k = -1;
+  for (int i = 0; i < nseg; ++i)
+    if (p >= inf->seg[i].begin && p < inf->seg[i].begin + inf->seg[i].count) k = i;
+  return k;
 }
 
 #ifdef BICACHE_TRACE
@@ -462,11 +540,15 @@ __device__ long long g_trace[3 * 1024];
 }  // namespace tc
 
 
+// kShared: the schedule holds row tiles with several segments (requests of a prefix group sharing a
+// tile); that instantiation takes its per-tile key counts from the K loader's notes.  The plain one keeps
+// them in registers and carries none of the shared-tile code in its loops.
+template <bool kShared>
 __global__ void __launch_bounds__(tc::kThreads, 1)
 tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
                     const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o, int q_tma,
-                    int o_tma, long long wait_cycles) {
+                    const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_o,
+                    const __grid_constant__ CUtensorMap tm_q8, int q_tma, int o_tma, long long wait_cycles) {
   using namespace tc;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* smem =
@@ -542,22 +624,43 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
     int n_it = 0;                // items seen by this CTA
     int c_tile = 0;              // key tiles this query tile has processed (phase of s_full / p_half)
     int e_item = 0;              // items this query tile has taken part in (phase of o_done)
+    int tg = 0;                  // key tiles of all items so far (index into the tile descriptions)
     int ti = 0; (void)ti;
     while (ok) {
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->info_full[n_it & 1]), (n_it >> 1) & 1, abort_flag));
       if (!ok) break;
       const ItemInfo* inf = &bars->info[n_it & 1];
-      const Geo g = read_geo_uniform(inf, s.num_splits, s.tiles_per_split, G);
+      const Geo g = read_geo_uniform(inf, s.num_splits, s.tiles_per_split);
       if (!g.valid) break;
       const int T = g.T;
       const bool active = X == 0 || g.b_active;
+      // The segment (request) this thread's row belongs to; -1: a padding row.  With several segments a
+      // row takes part only in the own-key tiles of its own request (the prefix tiles come first, so its
+      // reference maximum is finite by then); with one segment padding rows just run along.
+      const int vseg = seg_of_row(inf, g.nseg, X * 128 + gt);
       float m_ref = -INFINITY, l_sum = 0.f;
       for (int j = 0; j < T && active; ++j) {
-        const int cnt = tile_keys(g, j);
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_full[X]), c_tile & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
         if (tid == 0) BICACHE_STAMP(0, ti); if (tid == 128) BICACHE_STAMP(2, ti);
+        // Keys of the tile.  The plain kernel works them out from registers; the kernel for row tiles
+        // shared by several requests reads what the K loader wrote down (two code paths side by side in
+        // this loop cost more than either alone, hence two kernels).  In a shared tile a row takes part only in the own keys of its own request: for the
+        // other rows the reference maximum used below is +inf, which makes every exponential exactly 0
+        // (and the row's own maximum -inf, so it never asks for a rescale): no branch, no code of its
+        // own in this loop.
+        int cnt;
+        bool mine = true;
+        if (!kShared) {
+          bool dense_unused;
+          cnt = tile_keys_single(g, j, dense_unused);
+        } else {
+          const int meta = __shfl_sync(0xffffffffu, *reinterpret_cast<volatile int*>(&bars->tile_meta[(tg + j) & 7]), 0);
+          cnt = meta & 255;
+          const int tseg = (meta >> 16) - 1;
+          mine = tseg < 0 || tseg == vseg;
+        }
         // the whole row of S into registers: four loads in flight, one wait
         unsigned r[128];
         tmem_ld32(tmem_s, r);
@@ -596,7 +699,8 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           // P of the first 64 keys is handed to the tensor pipe before the second half is computed.
           // If the row maximum turns out to exceed the reference by more than 2^8 (rare: checked per
           // warp before anything is handed over), the tile is redone below with the new reference.
-          const unsigned long long neg_m2 = pack2(-m_ref, -m_ref);
+          const float neg_m_eff = mine ? -m_ref : -INFINITY;
+          const unsigned long long neg_m2 = pack2(neg_m_eff, neg_m_eff);
           float mx0 = -INFINITY, mx1 = -INFINITY;
           // first half of the exponentials, with the maximum over all 128 scores computed alongside
           // (independent instructions that fill the exp unit's latency)
@@ -626,7 +730,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             r[2 * i] = pack_bf16(p0, p1);
             r[2 * i + 1] = pack_bf16(p2, p3);
           }
-          const float mx = fmaxf(mx0, mx1) * sl2;              // scale > 0
+          const float mx = mine ? fmaxf(mx0, mx1) * sl2 : -INFINITY;   // scale > 0
 
           if (!__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
             tmem_st32(tmem_s, r);
@@ -669,7 +773,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               m_ref = mx;
             }
             unsigned s4[32];
-            const float neg_m = -m_ref;
+            const float neg_m = mine ? -m_ref : -INFINITY;
             float ps = 0.f;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -716,11 +820,11 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       if (!ok) break;
       // ------------------------------- epilogue -------------------------------------------
       if (active) {
-        const int row0 = inf->row0, kv_head = inf->kv_head;
-        const long long row_off = inf->row_off;
-        const int packed_rows = g.n * G;
-        const int prow = row0 + X * 128 + gt;                // packed row of this thread
-        const bool row_valid = prow < packed_rows;
+        const int kv_head = inf->kv_head;
+        const bool row_valid = vseg >= 0;
+        const SegInfo* sg = &inf->seg[row_valid ? vseg : 0];
+        const long long row_off = sg->row_off;
+        const int prow = sg->prow0 + (X * 128 + gt - sg->begin);   // packed row of this thread within its request
         const int a = prow / G;
         const int h = kv_head * G + (prow - a * G);
         unsigned o[128];
@@ -746,7 +850,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
         if (s.num_splits > 1) {
           // key-split call: normalised fp32 partial and its lse, merged by a second kernel
           if (row_valid) {
-            const long long pr = ((long long)inf->split * t.total_tokens + inf->tok_off + a) * t.Hq + h;
+            const long long pr = ((long long)inf->split * t.total_tokens + sg->tok_off + a) * t.Hq + h;
             float* po = t.part_o + pr * 128;
 #pragma unroll
             for (int i = 0; i < 128; i += 4)
@@ -761,8 +865,13 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           // one TMA store writes the half out; a warp whose rows are not all valid, or a head
           // grouping the box cannot express, copies the staged rows out itself, four rows per
           // instruction.
-          const int p0w = row0 + X * 128 + (warp & 3) * 32;  // first packed row of this warp
-          const bool by_tma = o_tma && p0w + 32 <= packed_rows;
+          // (a warp whose 32 rows lie in one segment on whole tokens; else every row finds its own place)
+          const int seg_first = __shfl_sync(0xffffffffu, vseg, 0), seg_last = __shfl_sync(0xffffffffu, vseg, 31);
+          const int prow_first = __shfl_sync(0xffffffffu, prow, 0);
+          const bool by_tma = o_tma && seg_first >= 0 && seg_first == seg_last && prow_first % G == 0;
+          const int tok_first = (int)__shfl_sync(0xffffffffu, (int)row_off, 0) + prow_first / G;
+          // byte offset of this thread's output row (one 64-dim half is added below); -1: a padding row
+          const long long my_dst = row_valid ? ((row_off + a) * t.out_stride + (long long)h * 128) * 2 : -1;
 #pragma unroll
           for (int hh = 0; hh < 2; ++hh) {
             if (lane == 0) bulk_wait_read();                 // the previous store has read the staging rows
@@ -781,7 +890,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               fence_proxy_async();
               __syncwarp();
               if (lane == 0) {
-                tma_store_3d(&tm_o, smem_u32(stage), hh * 64, kv_head * G, (int)row_off + p0w / G);
+                tma_store_3d(&tm_o, smem_u32(stage), hh * 64, kv_head * G, tok_first);
                 bulk_commit_group();
               }
             } else {
@@ -790,14 +899,10 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
 #pragma unroll 2
               for (int it = 0; it < 8; ++it) {
                 const int row = it * 4 + (lane >> 3);
-                const int pr = p0w + row;
-                if (pr < packed_rows) {
-                  const int a2 = pr / G, jj = pr - a2 * G;
-                  char* dst = t.out + ((row_off + a2) * t.out_stride + (long long)(kv_head * G + jj) * 128 + hh * 64) * 2 +
-                              ch * 16;
-                  *reinterpret_cast<uint4*>(dst) =
+                const long long dst_off = __shfl_sync(0xffffffffu, my_dst, row);
+                if (dst_off >= 0)
+                  *reinterpret_cast<uint4*>(t.out + dst_off + hh * 128 + ch * 16) =
                       *reinterpret_cast<const uint4*>(stage + row * 128 + ((ch ^ (row & 7)) << 4));
-                }
               }
               __syncwarp();
             }
@@ -809,6 +914,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->info_free[n_it & 1]));
       ++n_it;
+      tg += T;
     }
     if (lane == 0) bulk_wait_all();                          // the output stores of this warp have completed
     tc_fence_before();
@@ -820,34 +926,84 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
     bool ok = !dead;
     int n_it = 0;
     int eq[2] = {0, 0};          // items each query tile has taken part in (phase of q_free / q_full)
+    // The record of item `idx` (the whole warp works on it; lane k fills segment k).
     auto write_info = [&](ItemInfo* dst, int idx) {
       if (idx < s.num_items) {
         const WorkItem wi = s.items[idx];
-        const ReqMeta rq = s.reqs[wi.req];
-        dst->kv_head = wi.kv_head;
-        dst->row0 = wi.row0;
-        dst->split = wi.split;
-        dst->n = rq.n;
-        dst->m = rq.m;
-        dst->page_off = rq.page_off;
-        dst->tok_off = rq.tok_off;
-        dst->row_off = rq.row_off;
-        dst->valid = 1;
-      } else {
+        if (s.tiles != nullptr) {
+          const RowTile* tl = s.tiles + wi.req;
+          const int nseg = tl->nseg, m = tl->m;
+          const int pt = (m + kTileKeys - 1) / kTileKeys;
+          SegInfo si;
+          int own = 0;
+          if (lane < nseg) {
+            const RowSeg sg = tl->seg[lane];
+            const ReqMeta rq = s.reqs[sg.req];
+            si.row_off = rq.row_off;
+            si.n = rq.n;
+            si.prow0 = sg.prow0;
+            si.begin = sg.begin;
+            si.count = sg.count;
+            si.tok_off = rq.tok_off;
+            own = (rq.n + kTileKeys - 1) / kTileKeys;
+          }
+          int scan = own;                                 // inclusive prefix sum over the segments
+#pragma unroll
+          for (int o = 1; o < kMaxSegs; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, scan, o);
+            if (lane >= o) scan += up;
+          }
+          if (lane < nseg) {
+            si.tile_end = pt + scan;
+            dst->seg[lane] = si;
+          }
+          const int all_tiles = pt + __shfl_sync(0xffffffffu, scan, nseg - 1);
+          if (lane == 0) {
+            dst->kv_head = wi.kv_head;
+            dst->split = wi.split;
+            dst->m = m;
+            dst->page_off = tl->page_off;
+            dst->nseg = nseg;
+            dst->nrows = tl->nrows;
+            dst->all_tiles = all_tiles;
+            dst->valid = 1;
+          }
+        } else if (lane == 0) {
+          const ReqMeta rq = s.reqs[wi.req];
+          const int pt = (rq.m + kTileKeys - 1) / kTileKeys, own = (rq.n + kTileKeys - 1) / kTileKeys;
+          SegInfo si;
+          si.row_off = rq.row_off;
+          si.n = rq.n;
+          si.prow0 = wi.row0;
+          si.begin = 0;
+          si.count = min(kTileRows, rq.n * G - wi.row0);
+          si.tok_off = rq.tok_off;
+          si.tile_end = pt + own;
+          dst->seg[0] = si;
+          dst->kv_head = wi.kv_head;
+          dst->split = wi.split;
+          dst->m = rq.m;
+          dst->page_off = rq.page_off;
+          dst->nseg = 1;
+          dst->nrows = si.count;
+          dst->all_tiles = pt + own;
+          dst->valid = 1;
+        }
+      } else if (lane == 0) {
         dst->valid = 0;
       }
+      __syncwarp();                                       // every lane's part is written before lane 0 signals
     };
-    if (ok && lane == 0) {
+    if (ok) {
       write_info(&bars->info[0], (int)blockIdx.x);
-      mbar_arrive(smem_u32(&bars->info_full[0]));
+      if (lane == 0) mbar_arrive(smem_u32(&bars->info_full[0]));
     }
     __syncwarp();
     while (ok) {
       const ItemInfo* inf = &bars->info[n_it & 1];
-      const Geo g = read_geo_uniform(inf, s.num_splits, s.tiles_per_split, G);
+      const Geo g = read_geo_uniform(inf, s.num_splits, s.tiles_per_split);
       if (!g.valid) break;
       if (g.T > 0) {
-        const int packed_rows = g.n * G;
         for (int x = 0; x < 2 && ok; ++x) {
           if (x == 1 && !g.b_active) break;
           ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_free[x]), (eq[x] & 1) ^ 1, abort_flag));
@@ -855,11 +1011,26 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           ++eq[x];
           const unsigned qf = smem_u32(&bars->q_full[x]);
           const unsigned q_dst = q_smem + x * kTileBytes;
-          if (q_tma) {
-            // 128 packed rows = 128 / G tokens x G heads of the KV group: one TMA box per 64-dim half,
-            // in the dense swizzled layout (row r at r * 128 bytes, halves 16 KB apart)
+          const SegInfo* s0 = &inf->seg[0];
+          if (kShared && g.nseg > 1) {
+            // Rows of several requests (only built when the heads of a KV group divide 8): 16 boxes of 8
+            // packed rows per 64-dim half, one per lane, each from the request that owns its rows
+            // (segments start on multiples of 8 rows); a box past the last segment is filled with zeros
+            // (a coordinate outside the tensor).  Dense swizzled layout: row r at r * 128 bytes, halves
+            // 16 KB apart.
+            const int box = lane & 15, half = lane >> 4;
+            const int k = seg_of_row(inf, g.nseg, x * 128 + box * 8);
+            int tok = 0x3fffffff;
+            if (k >= 0) tok = (int)inf->seg[k].row_off + (inf->seg[k].prow0 + x * 128 + box * 8 - inf->seg[k].begin) / G;
+            tma_load_3d(q_dst + half * (kTileBytes / 2) + box * 1024, &tm_q8, half * 64, inf->kv_head * G, tok, qf);
+            if (lane == 0) mbar_arrive_expect_tx(qf, (unsigned)kTileBytes);
+            else mbar_arrive(qf);
+          } else if (q_tma) {
+            // 128 packed rows = 128 / G tokens x G heads of the KV group (the schedule starts such an
+            // item on a whole token): one TMA box per 64-dim half, in the dense swizzled layout (row r
+            // at r * 128 bytes, halves 16 KB apart)
             if (lane == 0) {
-              const int tok = (int)inf->row_off + (inf->row0 + x * 128) / G;
+              const int tok = (int)s0->row_off + (s0->prow0 + x * 128) / G;
               mbar_arrive_expect_tx(qf, (unsigned)kTileBytes);
               tma_load_3d(q_dst, &tm_q, 0, inf->kv_head * G, tok, qf);
               tma_load_3d(q_dst + kTileBytes / 2, &tm_q, 64, inf->kv_head * G, tok, qf);
@@ -869,12 +1040,13 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           } else {
             // gathers into the page-image layout: packed row p = token a * G + head jj of the KV
             // group; rows past the end are zero-filled
+            const int packed_rows = s0->n * G;
             const int r0 = lane >> 4, c16 = lane & 15;
-            int prow = inf->row0 + x * 128 + r0;
+            int prow = s0->prow0 + x * 128 + r0;
             const int a0 = prow / G;
             int jj = prow - a0 * G;
             const long long q_row_bytes = t.q_stride * 2;
-            const char* q_base = t.q + (inf->row_off * t.q_stride + (long long)inf->kv_head * G * 128) * 2 + c16 * 16;
+            const char* q_base = t.q + (s0->row_off * t.q_stride + (long long)inf->kv_head * G * 128) * 2 + c16 * 16;
             const char* src_row = q_base + a0 * q_row_bytes;
 #pragma unroll 4
             for (int i = 0; i < 64; ++i) {
@@ -896,16 +1068,18 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
         if (!ok) break;
       }
       // the next item: its record slot must have been released by every role (item n - 1)
-      if (lane == 0) {
+      {
         const int nn = n_it + 1;
-        ok = mbar_wait(smem_u32(&bars->info_free[nn & 1]), ((nn >> 1) & 1) ^ 1, abort_flag);
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->info_free[nn & 1]), ((nn >> 1) & 1) ^ 1, abort_flag));
         if (ok) {
-          write_info(&bars->info[nn & 1], (int)gridDim.x + atomicAdd(next_item, 1));
-          mbar_arrive(smem_u32(&bars->info_full[nn & 1]));
+          int idx = 0;
+          if (lane == 0) idx = (int)gridDim.x + atomicAdd(next_item, 1);
+          idx = __shfl_sync(0xffffffffu, idx, 0);
+          write_info(&bars->info[nn & 1], idx);
+          if (lane == 0) mbar_arrive(smem_u32(&bars->info_full[nn & 1]));
         }
       }
-      ok = __all_sync(0xffffffffu, ok);
-      __syncwarp();                                          // lane 0's record is visible to the warp
+      __syncwarp();
       ++n_it;
     }
     cp_async_wait<0>();
@@ -935,10 +1109,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->info_full[n_it & 1]), (n_it >> 1) & 1, abort_flag));
       if (!ok) break;
       const ItemInfo* inf = &bars->info[n_it & 1];
-      const Geo g = read_geo_uniform(inf, s.num_splits, s.tiles_per_split, G);
+      const Geo g = read_geo_uniform(inf, s.num_splits, s.tiles_per_split);
       if (!g.valid) break;
       const int kv_head = inf->kv_head;
-      const long long row_off = inf->row_off;
       const int* pages = s.pages + inf->page_off;
       for (int j = 0; j < g.T; ++j) {
         const int u = U + 2 * j + is_v;
@@ -948,6 +1121,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
         if (!ok) break;
         const unsigned dst = ring_smem + slot * kTileBytes;
         const unsigned full = smem_u32(&bars->full[slot]);
+        const TileRef tr = tile_ref_uniform(inf, g, j);
+        if (kShared && !is_v && lane == 0)       // before this lane's arrival on `full`, which publishes it
+          bars->tile_meta[(u >> 1) & 7] = tr.cnt | ((tr.seg >= 0 && tr.cnt >= kTileKeys) ? 256 : 0) | ((tr.seg + 1) << 16);
         if (jg < g.prefix_tiles) {
           // cached prefix tile: one bulk copy per page (a pool page already is the tile image), each
           // issued by its own lane so that the page-table reads overlap
@@ -967,8 +1143,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           }
           continue;
         }
-        const int key0 = (jg - g.prefix_tiles) * kTileKeys;
-        const int cnt = min(kTileKeys, g.n - key0);
+        // own rows of one of the item's requests
+        const long long row_off = inf->seg[tr.seg].row_off;
+        const int key0 = tr.key0, cnt = tr.cnt;
         if (cnt >= kTileKeys) {
           // a full tile of the request's own rows: two TMA boxes (dense swizzled layout)
           if (lane == 0) {
@@ -1073,7 +1250,14 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       unsigned u = 0;            // ring use of the current key tile's K; its V is u + 1, the next tile's K u + 2
       int ti = 0; (void)ti;
       ok = BICACHE_WAIT(smem_u32(&bars->info_full[0]), 0);
-      Geo cur = read_geo_uniform(&bars->info[0], s.num_splits, s.tiles_per_split, G);
+      Geo cur = read_geo_uniform(&bars->info[0], s.num_splits, s.tiles_per_split);
+      // keys | dense << 8 of the key tile whose K has ring use uu, as the K loader described it (valid once
+      // that slot's `full` barrier has been waited for); warp-uniform like the geometry
+      auto read_meta = [&](unsigned uu) -> int {
+        return __shfl_sync(0xffffffffu, *reinterpret_cast<volatile int*>(&bars->tile_meta[(uu >> 1) & 7]), 0);
+      };
+      bool dn = false;           // layout of the current key tile
+      int ksteps = 8;            // its keys, in steps of 16
       bool pre = false;          // the first S of the current item was issued at the end of the previous one
       while (ok && cur.valid) {
         Geo nxt;
@@ -1082,12 +1266,18 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
         const int T = cur.T;
         if (T > 0) {
           const bool b_on = cur.b_active;
-          bool dn = tile_dense(cur, 0);                        // layout of the current key tile
           if (!pre) {
             // the first S of an item that could not be issued ahead (the CTA's first item)
             ok = BICACHE_WAIT(bar_full + (u & 3) * 8, (u >> 2) & 1) && BICACHE_WAIT(bar_qfull, e0 & 1);
             if (!ok) break;
             tc_fence_after();
+            if (!kShared) {
+              ksteps = (tile_keys_single(cur, 0, dn) + 15) >> 4;
+            } else {
+              const int meta = read_meta(u);
+              dn = (meta & 256) != 0;
+              ksteps = ((meta & 255) + 15) >> 4;
+            }
             const unsigned long long kd0 = (dn ? kb_dense : kb_img) + (u & 3) * kSlotUnits;
             issue_s(tmem_u, q_desc0, kd0, dn ? 1024u : 64u);
             mma_commit_pred(el, bar_s);
@@ -1107,7 +1297,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           // V of the first key tile; the previous item's epilogue must have read O_A out of TMEM
           ok = BICACHE_WAIT(bar_full + ((u + 1) & 3) * 8, ((u + 1) >> 2) & 1) && BICACHE_WAIT(bar_ofree, (e0 & 1) ^ 1);
           if (!ok) break;
-          int ksteps = (tile_keys(cur, 0) + 15) >> 4;
           // One key tile.  The body exists twice: the lean one for every tile but the last, and the
           // one for the last tile, which also looks at the next item.
           auto tile_iter = [&](auto last_c, int j) {
@@ -1126,25 +1315,31 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             // ---- shadow of A's second half of the exponentials: what follows the O of this iteration ----
             bool s_on0 = true, s_on1 = b_on;                   // an S follows O_A / O_B
             bool q_last = j + 2 == T;                           // ... and it is the last S of its item
-            bool dn_next;
+            bool dn_next = false;
+            int ks_next = 8;
             if (!last) {
-              dn_next = tile_dense(cur, j + 1);
+              if (!kShared) ks_next = (tile_keys_single(cur, j + 1, dn_next) + 15) >> 4;
             } else {
               // the next item (fetched long ago): its first S follows this item's last O
               const int nn = n_it + 1;
               ok = BICACHE_WAIT(smem_u32(&bars->info_full[nn & 1]), (nn >> 1) & 1);
               if (!ok) return;
-              nxt = read_geo_uniform(&bars->info[nn & 1], s.num_splits, s.tiles_per_split, G);
+              nxt = read_geo_uniform(&bars->info[nn & 1], s.num_splits, s.tiles_per_split);
               have_next = true;
               can_pre = nxt.valid && nxt.T > 0;
               s_on0 = can_pre;
               s_on1 = can_pre && nxt.b_active;
               q_last = nxt.T == 1;
-              dn_next = can_pre && tile_dense(nxt, 0);
+              if (!kShared && can_pre) ks_next = (tile_keys_single(nxt, 0, dn_next) + 15) >> 4;
             }
             if (s_on0) {
               ok = BICACHE_WAIT(bar_full + sn * 8, ((u + 2) >> 2) & 1);
               if (!ok) return;
+              if (kShared) {
+                const int meta = read_meta(u + 2);
+                dn_next = (meta & 256) != 0;
+                ks_next = ((meta & 255) + 15) >> 4;
+              }
             }
             const unsigned long long k_desc = (dn_next ? kb_dense : kb_img) + sn * kSlotUnits;
             const unsigned k_hi = dn_next ? 1024u : 64u;
@@ -1182,8 +1377,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               tc_fence_after();
                             issue_pv(tmem_o1, tmem_s1, v_desc, v_step, 0, acc0, ksteps);
             }
-            // ---- shadow of B's second half: the next tile's key count ----
-            const int ks_next = last ? 8 : (tile_keys(cur, j + 1) + 15) >> 4;
             // ---- tile B: second half, then the next S_B ----
             if (b_on) {
               ok = BICACHE_WAIT(bar_p + 24, c1 & 1);
@@ -1227,7 +1420,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           const int nn = n_it + 1;
           ok = BICACHE_WAIT(smem_u32(&bars->info_full[nn & 1]), (nn >> 1) & 1);
           if (!ok) break;
-          nxt = read_geo_uniform(&bars->info[nn & 1], s.num_splits, s.tiles_per_split, G);
+          nxt = read_geo_uniform(&bars->info[nn & 1], s.num_splits, s.tiles_per_split);
         }
         if (elect_one()) mbar_arrive(smem_u32(&bars->info_free[n_it & 1]));
         __syncwarp();
@@ -1266,12 +1459,17 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
 
 inline cudaError_t configure_tc_attention() {
   cudaFuncAttributes attr;
-  cudaError_t e = cudaFuncGetAttributes(&attr, tc_attention_kernel);
-  if (e != cudaSuccess) return e;
-  // the register pool the kernel redistributes is the launch allocation of the CTA
-  if (attr.numRegs * tc::kThreads < 2 * tc::kGroupThreads * tc::kSoftmaxRegs + 128 * tc::kOtherRegs)
-    return cudaErrorLaunchOutOfResources;
-  return cudaFuncSetAttribute(tc_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes);
+  for (int shared = 0; shared < 2; ++shared) {
+    const void* fn = shared ? (const void*)tc_attention_kernel<true> : (const void*)tc_attention_kernel<false>;
+    cudaError_t e = cudaFuncGetAttributes(&attr, fn);
+    if (e != cudaSuccess) return e;
+    // the register pool the kernel redistributes is the launch allocation of the CTA
+    if (attr.numRegs * tc::kThreads < 2 * tc::kGroupThreads * tc::kSoftmaxRegs + 128 * tc::kOtherRegs)
+      return cudaErrorLaunchOutOfResources;
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::kSmemBytes);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
 }
 
 // Tensor maps of one call: q [rows][Hq][128] with a box of (64 dims, G heads, 128 / G rows) so that
@@ -1291,9 +1489,14 @@ inline cudaError_t launch_tc_attention(const ScheduleView& s, const PoolView& po
                                        int* status, int num_sms, const TcTensorMaps& maps, long long wait_cycles,
                                        cudaStream_t stream) {
   const int grid = s.num_items < num_sms ? s.num_items : num_sms;
-  tc_attention_kernel<<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(
-      s, pool, t, status, maps.q, maps.k, maps.v, maps.o, maps.q_tma, maps.o_tma,
-      wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
+  if (s.tiles != nullptr && s.shared_tiles)
+    tc_attention_kernel<true><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(
+        s, pool, t, status, maps.q, maps.k, maps.v, maps.o, maps.q8, maps.q_tma, maps.o_tma,
+        wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
+  else
+    tc_attention_kernel<false><<<grid, tc::kThreads, tc::kSmemBytes, stream>>>(
+        s, pool, t, status, maps.q, maps.k, maps.v, maps.o, maps.q8, maps.q_tma, maps.o_tma,
+        wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
   return cudaGetLastError();
 }
 
