@@ -1480,20 +1480,6 @@ int32_t bicache_device_status(bicache_ctx* ctx, void* stream, int32_t clear) {
   return fail(ctx, BICACHE_ERR_CUDA, "a kernel reported an internal error");
 }
 
-#ifdef BICACHE_DEC_TRACE
-// Debug build only: copy the traced key-range CTA's time stamps to the host.
-int32_t bicache_debug_read_dec_trace(unsigned long long* out, int32_t n) {
-  return cudaMemcpyFromSymbol(out, bicache::dec::g_dec_trace, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : 4;
-}
-#endif
-
-#ifdef BICACHE_TRACE
-// Debug build only: copy the traced CTA's clock stamps to the host.
-int32_t bicache_debug_read_trace(long long* out, int32_t n) {
-  return cudaMemcpyFromSymbol(out, bicache::tc::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : 4;
-}
-#endif
-
 int32_t bicache_set_wait_budget(bicache_ctx* ctx, int64_t sm_cycles) {
   if (!ctx || sm_cycles < 0) return BICACHE_ERR_INVALID;
   ctx->wait_cycles = sm_cycles;

@@ -528,14 +528,6 @@ __device__ __forceinline__ int seg_of_row(const ItemInfo* inf, int nseg, int p) 
   return k;
 }
 
-#ifdef BICACHE_TRACE
-// Debug build only: per-phase SM clock stamps of one CTA (three roles x 1024 slots).
-__device__ long long g_trace[3 * 1024];
-#define BICACHE_STAMP(role, idx) \
-  do { if (blockIdx.x == BICACHE_TRACE && (idx) < 1024) g_trace[(role) * 1024 + (idx)++] = clock64(); } while (0)
-#else
-#define BICACHE_STAMP(role, idx) do { } while (0)
-#endif
 
 }  // namespace tc
 
@@ -561,9 +553,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
   int* const ctas_done = status + 17;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-#ifdef BICACHE_TRACE
-  if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1000] = clock64();
-#endif
   const int G = t.Hq / t.Hkv;
 
   if (tid == 0) {
@@ -595,9 +584,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-#ifdef BICACHE_TRACE
-  if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1001] = clock64();
-#endif
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&bars->tmem_base);
   const bool dead = *reinterpret_cast<volatile int*>(&bars->dead) != 0;   // an earlier launch or CTA gave up: do no work
 
@@ -625,7 +611,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
     int c_tile = 0;              // key tiles this query tile has processed (phase of s_full / p_half)
     int e_item = 0;              // items this query tile has taken part in (phase of o_done)
     int tg = 0;                  // key tiles of all items so far (index into the tile descriptions)
-    int ti = 0; (void)ti;
     while (ok) {
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->info_full[n_it & 1]), (n_it >> 1) & 1, abort_flag));
       if (!ok) break;
@@ -643,7 +628,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->s_full[X]), c_tile & 1, abort_flag));
         if (!ok) break;
         tc_fence_after();
-        if (tid == 0) BICACHE_STAMP(0, ti); if (tid == 128) BICACHE_STAMP(2, ti);
         // Keys of the tile.  The plain kernel works them out from registers; the kernel for row tiles
         // shared by several requests reads what the K loader wrote down (two code paths side by side in
         // this loop cost more than either alone, hence two kernels).  In a shared tile a row takes part only in the own keys of its own request: for the
@@ -764,7 +748,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(smem_u32(&bars->p_half[X][1]));
-            if (tid == 0) BICACHE_STAMP(0, ti); if (tid == 128) BICACHE_STAMP(2, ti);
             stored = true;
           } else {
             // redo with the new reference: S is still intact in TMEM
@@ -833,7 +816,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           if (!ok) break;
           tc_fence_after();
           ++e_item;
-          if (tid == 0) BICACHE_STAMP(0, ti); if (tid == 128) BICACHE_STAMP(2, ti);
           tmem_ld32(tmem_o, o);
           tmem_ld32(tmem_o + 32, o + 32);
           tmem_ld32(tmem_o + 64, o + 64);
@@ -909,7 +891,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           }
           if (row_valid && t.lse != nullptr) t.lse[(row_off + a) * t.Hq + h] = lse;
         }
-        if (tid == 0) BICACHE_STAMP(0, ti); if (tid == 128) BICACHE_STAMP(2, ti);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&bars->info_free[n_it & 1]));
@@ -1248,7 +1229,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
       int c0 = 0, c1 = 0;        // key tiles each query tile has been through (phase of p_half)
       int e0 = 0, e1 = 0;        // items each query tile has taken part in (phase of q_full / o_free)
       unsigned u = 0;            // ring use of the current key tile's K; its V is u + 1, the next tile's K u + 2
-      int ti = 0; (void)ti;
       ok = BICACHE_WAIT(smem_u32(&bars->info_full[0]), 0);
       Geo cur = read_geo_uniform(&bars->info[0], s.num_splits, s.tiles_per_split);
       // keys | dense << 8 of the key tile whose K has ring use uu, as the K loader described it (valid once
@@ -1308,10 +1288,8 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             // ---- tile A: first half of O += P V as soon as P of keys 0-63 is there ----
             ok = BICACHE_WAIT(bar_p, c0 & 1);
             if (!ok) return;
-            if (lane == 0) BICACHE_STAMP(1, ti);
             tc_fence_after();
                         issue_pv(tmem_o0, tmem_u, v_desc, v_step, 0, acc0, ksteps);
-            if (lane == 0) BICACHE_STAMP(1, ti);
             // ---- shadow of A's second half of the exponentials: what follows the O of this iteration ----
             bool s_on0 = true, s_on1 = b_on;                   // an S follows O_A / O_B
             bool q_last = j + 2 == T;                           // ... and it is the last S of its item
@@ -1343,11 +1321,9 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             }
             const unsigned long long k_desc = (dn_next ? kb_dense : kb_img) + sn * kSlotUnits;
             const unsigned k_hi = dn_next ? 1024u : 64u;
-            if (lane == 0) BICACHE_STAMP(1, ti);
             // ---- tile A: second half, then the next S_A back to back ----
             ok = BICACHE_WAIT(bar_p + 8, c0 & 1);
             if (!ok) return;
-            if (lane == 0) BICACHE_STAMP(1, ti);
             tc_fence_after();
                         issue_pv(tmem_o0, tmem_u, v_desc, v_step, 1, acc0, ksteps);
             ++c0;
@@ -1364,7 +1340,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               mma_commit_pred(el, bar_s);
               if (q_last) mma_commit_pred(el, bar_qfree);
             }
-            if (lane == 0) BICACHE_STAMP(1, ti);
             // ---- tile B: first half ----
             if (b_on) {
               if (j == 0) {
@@ -1373,7 +1348,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               }
               ok = BICACHE_WAIT(bar_p + 16, c1 & 1);
               if (!ok) return;
-              if (lane == 0) BICACHE_STAMP(1, ti);
               tc_fence_after();
                             issue_pv(tmem_o1, tmem_s1, v_desc, v_step, 0, acc0, ksteps);
             }
@@ -1398,7 +1372,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               mma_commit_pred(el, bar_s + 8);
               if (q_last) mma_commit_pred(el, bar_qfree + 8);
             }
-            if (lane == 0) BICACHE_STAMP(1, ti);
             // release V of this tile and K of the next
             mma_commit_pred(el, bar_free + sv * 8);
             if (s_on0) mma_commit_pred(el, bar_free + sn * 8);
@@ -1438,9 +1411,6 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
   }
 
   __syncthreads();
-#ifdef BICACHE_TRACE
-  if (tid == 0 && blockIdx.x == BICACHE_TRACE) g_trace[2 * 1024 + 1002] = clock64();
-#endif
   if (warp == kMmaWarp) {
     tc_fence_after();
     tmem_dealloc(tmem, kTmemCols);

@@ -66,18 +66,6 @@ constexpr int kDecSmemBytes = kQBytes + (kKStages + kVStages) * kKvTileBytes + (
 static_assert(2 * (kDecSmemBytes + 1024) <= 233472, "two CTAs per SM");
 static_assert(128 * 528 <= (kKStages + kVStages) * kKvTileBytes, "the partial rows are staged over the K/V rings");
 
-#ifdef BICACHE_DEC_TRACE
-// Debug build only: nanosecond stamps of one CTA (slot = role event).
-__device__ unsigned long long g_dec_trace[64];
-__device__ __forceinline__ unsigned long long dec_now() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-#define DEC_STAMP(slot) do { if (blockIdx.x == BICACHE_DEC_TRACE) g_dec_trace[slot] = dec_now(); } while (0)
-#else
-#define DEC_STAMP(slot) do { } while (0)
-#endif
 
 }  // namespace dec
 
@@ -98,7 +86,6 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   // the merge kernel that follows may be placed on the SMs from now on (it waits for this grid's end)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  if (threadIdx.x == 0) DEC_STAMP(0);
   const DecodeItem it = items[blockIdx.x];
   const int G = t.Hq / t.Hkv;
   // key tiles: the cached range first, then (range 0) the own keys
@@ -141,7 +128,6 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
   const unsigned tmem = *reinterpret_cast<volatile unsigned*>(&sy->tmem_base);
   const bool dead = *reinterpret_cast<volatile int*>(&sy->dead) != 0;
   const unsigned tmem_o = tmem + 128;
-  if (tid == 0) DEC_STAMP(1);
 
   if (warp < 4) {
     // ================================ softmax and epilogue =================================
@@ -176,7 +162,6 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
         }
       }
       cp_async_commit();
-      if (tid == 0) DEC_STAMP(6);
       cp_async_wait<0>();
       fence_proxy_async();
       mbar_arrive(smem_u32(&sy->q_full));
@@ -187,7 +172,6 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->s_full[b]), (j >> 1) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
-      if (tid == 0 && j < 8) DEC_STAMP(10 + j);
       unsigned r[64];
       tmem_ld32(tmem + b * 64 + lane_base, r);
       tmem_ld32(tmem + b * 64 + 32 + lane_base, r + 32);
@@ -259,7 +243,6 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(smem_u32(&sy->p_full[b]));
-      if (tid == 0 && j < 8) DEC_STAMP(20 + j);
       float s0, s1, s2, s3;
       unpack2(acc_a, s0, s1);
       unpack2(acc_b, s2, s3);
@@ -276,7 +259,6 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->o_done), 0, abort_flag));
         if (ok) {
           tc_fence_after();
-          if (tid == 0) DEC_STAMP(2);
           // Each thread holds one row of the partial (128 fp32 = 512 bytes, contiguous in the
           // workspace).  Written from registers, a warp's stores would touch 32 rows at a time; so
           // the row goes to shared memory first (the K/V rings are free by now: every tile has been
@@ -303,7 +285,6 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
             t.part_lse[pr] = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
             bulk_wait_all();
           }
-          if (tid == 0) DEC_STAMP(3);
         }
       } else if (row_valid) {
         float* po = t.part_o + pr * 128;
@@ -339,9 +320,7 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
         return true;
       };
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&sy->q_full), 0, abort_flag));
-      if (lane == 0) DEC_STAMP(4);
       if (ok) ok = issue_s(0);
-      if (lane == 0) DEC_STAMP(5);
       for (int j = 0; j < T && ok; ++j) {
         const int b = j & 1;
         if (j + 1 < T) {
@@ -400,7 +379,6 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
         }
         // every lane arrives, so the phase cannot complete before lane 0 has announced the bytes
         if (lane == 0) {
-          if (!is_v && j == 0) DEC_STAMP(7);
           mbar_arrive_expect_tx(full, (unsigned)(npages * kPageBytes));
           armed[b] = j;
         } else {
@@ -442,7 +420,6 @@ tc_decode_kernel(const dec::DecodeItem* __restrict__ items, const long long* __r
     tmem_dealloc(tmem, kDecTmemCols);
   }
   if (tid == 0 && !dead && *abort_flag) atomicCAS(status, kDevOk, kDevTimeout);
-  if (tid == 0) DEC_STAMP(8);
 }
 
 // ---------------------------------------------------------------------------------------------
