@@ -39,11 +39,17 @@ SMALL_SUFFIX = ("b1", "b2", "b3", "b4")
 # is named beside each figure; a capture is of the kernel as it was when the summary was written).
 # None: no capture of that launch exists.
 NCU_TRAFFIC = {
-    "config2": {"full": (647.9e6, "profiles/tc_attention_kernel_config2.md"),
-                "attend": (135.3e6, "profiles/tc_attention_kernel_config2.md")},
-    "config3": {"put": (2104.6e6, "profiles/hbm_kernels_config3.md"),
+    "config2": {"full": (652.3e6, "profiles/tc_attention_kernel_config2.md"),
+                "attend": (130.4e6, "profiles/tc_attention_kernel_config2.md")},
+    "config3": {"attend": (848.6e6, "profiles/tc_attention_kernel_config3_attend.md"),
+                "put": (2104.6e6, "profiles/hbm_kernels_config3.md"),
                 "similarity": (2147.6e6, "profiles/hbm_kernels_config3.md"),
                 "project": (218.0e6, "profiles/project_kv_kernel_config3.md")},
+    # captured with 4 of the 32 requests and scaled by the units processed (see the file)
+    "config5": {"full": (8848.0e6, "profiles/tc_attention_kernel_config5_traffic.md (4-request capture, scaled)"),
+                "attend": (402.0e6, "profiles/tc_attention_kernel_config5_traffic.md (4-request capture, scaled)")},
+    "config5s": {"full": (1106.0e6, "profiles/tc_attention_kernel_config5_traffic.md"),
+                 "attend": (79.7e6, "profiles/tc_attention_kernel_config5_traffic.md")},
     "b2": {"attend": (274.1e6, "profiles/key_range_kernels_b2.md")},
 }
 

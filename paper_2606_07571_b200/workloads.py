@@ -234,9 +234,18 @@ def scaled_down(w: Workload, num_layers=None, max_requests=None, prefix_div=1, s
                     shuffle_pages=w.shuffle_pages, note=w.note + " (scaled down)")
 
 
+def config5_small():
+    """Four of config 5's 32 requests (same prefix, same lengths): a case small enough for a full
+    profiler capture; DRAM traffic per launch scales with the number of requests."""
+    w = config5()
+    return Workload("config5-dream-gqa-4req", w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim, w.dtype, 16,
+                    w.prefix_lens, [0] * 4, [1024] * 4, softmax_scale=w.softmax_scale,
+                    note="config 5 with 4 of its 32 requests (profiling case)")
+
+
 CONFIGS = {
     "config1": config1, "config2": config2, "config3": config3,
-    "config4": config4, "config5": config5,
+    "config4": config4, "config5": config5, "config5s": config5_small,
     "b1": lambda: small_suffix("b1"), "b2": lambda: small_suffix("b2"),
     "b3": lambda: small_suffix("b3"), "b4": lambda: small_suffix("b4"),
 }
