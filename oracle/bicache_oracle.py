@@ -94,15 +94,20 @@ def reuse_depth(prefix_len, nonshared_len, table, num_layers):
 class PagedPrefixStore:
     """Prefix-KV store over fixed-size pages with FIFO eviction.
 
-    One page index addresses the same slot in every layer.  Token t of a
-    prefix lives in page pages[t // P], slot t % P.  The free list is a FIFO
-    queue: pages are taken from its head; an evicted prefix's pages are
-    appended to its tail in page-table order.  Prefix ids come from a counter
-    that is never reused.
+    Every layer has its own pages and its own free queue (a FIFO: pages are
+    taken from its head; an evicted prefix's pages are appended to its tail in
+    page-table order).  A prefix owns pages in the layers first_layer .. L-1
+    only: a shared prefix (put) in all of them, a request's kept deep-layer
+    prefix (reserve, Eq. 5) from its shallow depth on - the shallow layers of
+    such a request never read its own prefix KVs.  Token t of a prefix lives, in
+    layer l, in page pages_l[t // P], slot t % P.  As long as every prefix owns
+    all layers the queues move in lockstep and a prefix has the same page list
+    in every layer.  Layer l holds layer_pages[l] pages (default: num_pages in
+    every layer).  Prefix ids come from a counter that is never reused.
     """
 
     def __init__(self, num_layers, num_kv_heads, head_dim, page_size, num_pages,
-                 free_order=None):
+                 free_order=None, layer_pages=None):
         self.L = int(num_layers)
         self.Hkv = int(num_kv_heads)
         self.D = int(head_dim)
@@ -113,68 +118,105 @@ class PagedPrefixStore:
         free_order = [int(p) for p in free_order]
         if sorted(free_order) != list(range(self.num_pages)):
             raise InvalidArgument("free_order must be a permutation of the pages")
-        self.free = deque(free_order)
+        if layer_pages is None:
+            layer_pages = [self.num_pages] * self.L
+        self.layer_pages = [int(c) for c in layer_pages]
+        if len(self.layer_pages) != self.L or any(c < 1 or c > self.num_pages for c in self.layer_pages):
+            raise InvalidArgument("layer_pages needs one capacity in 1..num_pages per layer")
+        # layer l's queue: the pages below its capacity, in the given order
+        self.free = [deque(p for p in free_order if p < c) for c in self.layer_pages]
         # [layer][page][slot][kv head][dim]
         shape = (self.L, self.num_pages, self.P, self.Hkv, self.D)
         self.k_pool = np.zeros(shape, dtype=np.float64)
         self.v_pool = np.zeros(shape, dtype=np.float64)
         self.by_key = OrderedDict()   # key -> prefix id, in insertion order
-        self.entries = {}             # prefix id -> (key, m, [pages])
+        self.entries = {}             # prefix id -> (key, m, first_layer, [pages of layer first_layer, ...])
         self.next_id = 0
 
     def pages_needed(self, m):
         return (int(m) + self.P - 1) // self.P
 
+    def _insert(self, key, m, first_layer):
+        """Hit / miss / FIFO eviction / allocation in the layers first_layer .. L-1.
+        Returns (prefix_id, was_hit, pages of layer first_layer)."""
+        m = int(m)
+        first_layer = int(first_layer)
+        if m < 1:
+            raise InvalidArgument("empty prefix")
+        if not 0 <= first_layer < self.L:
+            raise InvalidArgument("first layer out of range")
+        key = int(key)
+        if key in self.by_key:
+            pid = self.by_key[key]
+            if self.entries[pid][1] != m or self.entries[pid][2] != first_layer:
+                raise InvalidArgument("key already present with another length or first layer")
+            return pid, True, list(self.entries[pid][3][0])
+        need = self.pages_needed(m)
+        layers = range(first_layer, self.L)
+        if any(need > self.layer_pages[l] for l in layers):
+            raise OutOfPages("prefix larger than a layer's pool")
+        while any(len(self.free[l]) < need for l in layers):
+            old_key, old_id = next(iter(self.by_key.items()))   # oldest insertion
+            del self.by_key[old_key]
+            _, _, old_first, old_pages = self.entries.pop(old_id)
+            for j, plist in enumerate(old_pages):
+                for p in plist:
+                    self.free[old_first + j].append(p)
+        pages = [[self.free[l].popleft() for _ in range(need)] for l in layers]
+        pid = self.next_id
+        self.next_id += 1
+        self.by_key[key] = pid
+        self.entries[pid] = (key, m, first_layer, pages)
+        return pid, False, list(pages[0])
+
     def put(self, key, k, v):
-        """Insert prefix KVs k, v of shape [L, m, Hkv, D].  Returns
-        (prefix_id, was_hit, pages)."""
+        """Insert prefix KVs k, v of shape [L, m, Hkv, D] (all layers).  Returns
+        (prefix_id, was_hit, pages of layer 0)."""
         k = np.asarray(k, dtype=np.float64)
         v = np.asarray(v, dtype=np.float64)
         if k.shape != v.shape or k.ndim != 4 or k.shape[0] != self.L \
                 or k.shape[2] != self.Hkv or k.shape[3] != self.D:
             raise InvalidArgument("bad prefix KV shape")
         m = k.shape[1]
-        if m < 1:
-            raise InvalidArgument("empty prefix")
-        key = int(key)
-        if key in self.by_key:
-            pid = self.by_key[key]
-            if self.entries[pid][1] != m:
-                raise InvalidArgument("key already present with another length")
-            return pid, True, list(self.entries[pid][2])
-        need = self.pages_needed(m)
-        if need > self.num_pages:
-            raise OutOfPages("prefix larger than the whole pool")
-        while len(self.free) < need:
-            old_key, old_id = next(iter(self.by_key.items()))   # oldest insertion
-            del self.by_key[old_key]
-            for p in self.entries.pop(old_id)[2]:
-                self.free.append(p)
-        pages = [self.free.popleft() for _ in range(need)]
-        pid = self.next_id
-        self.next_id += 1
-        self.by_key[key] = pid
-        self.entries[pid] = (key, m, pages)
-        for t in range(m):
-            self.k_pool[:, pages[t // self.P], t % self.P] = k[:, t]
-            self.v_pool[:, pages[t // self.P], t % self.P] = v[:, t]
-        return pid, False, list(pages)
+        pid, hit, pages0 = self._insert(key, m, 0)
+        if not hit:
+            pages = self.entries[pid][3]
+            for l in range(self.L):
+                for t in range(m):
+                    self.k_pool[l, pages[l][t // self.P], t % self.P] = k[l, t]
+                    self.v_pool[l, pages[l][t // self.P], t % self.P] = v[l, t]
+        return pid, hit, pages0
 
-    def reserve(self, key, m):
-        """Allocate pages for a prefix of m tokens without writing any KV (the
-        per-request deep-layer cache of Eq. 5, filled layer by layer at refresh
-        steps).  Same allocation and eviction rules as `put`."""
-        zeros = np.zeros((self.L, int(m), self.Hkv, self.D), dtype=np.float64)
-        return self.put(key, zeros, zeros)
+    def reserve(self, key, m, first_layer=0):
+        """Allocate pages for a prefix of m tokens in the layers first_layer .. L-1
+        without writing any KV (the per-request deep-layer cache of Eq. 5, which
+        only layers past the request's shallow depth keep; filled layer by layer
+        at refresh steps).  Same hit / miss / eviction rules as `put`.  Returns
+        (prefix_id, was_hit, pages of layer first_layer)."""
+        pid, hit, pages0 = self._insert(key, m, first_layer)
+        if not hit:
+            pages = self.entries[pid][3]
+            for j, plist in enumerate(pages):
+                for p in plist:
+                    self.k_pool[first_layer + j, p] = 0.0
+                    self.v_pool[first_layer + j, p] = 0.0
+        return pid, hit, pages0
+
+    def _layer_pages(self, prefix_id, layer):
+        if prefix_id not in self.entries:
+            raise NotFound("unknown or evicted prefix id")
+        _, _, first, pages = self.entries[prefix_id]
+        if not first <= layer < self.L:
+            raise InvalidArgument("the prefix owns no pages in this layer")
+        return pages[layer - first]
 
     def update_layer(self, prefix_id, layer, k, v):
         """Overwrite one layer of an existing prefix with k, v [m, Hkv, D]
         (Eq. 5, refresh step: KV^use <- KV^ref of the current step)."""
         if not 0 <= layer < self.L:
             raise InvalidArgument("layer out of range")
-        if prefix_id not in self.entries:
-            raise NotFound("unknown or evicted prefix id")
-        _, m, pages = self.entries[prefix_id]
+        pages = self._layer_pages(prefix_id, layer)
+        m = self.entries[prefix_id][1]
         k = np.asarray(k, dtype=np.float64)
         v = np.asarray(v, dtype=np.float64)
         if k.shape != (m, self.Hkv, self.D) or v.shape != k.shape:
@@ -190,10 +232,18 @@ class PagedPrefixStore:
         pid = self.by_key[key]
         return pid, self.entries[pid][1]
 
-    def pages(self, prefix_id):
+    def first_layer(self, prefix_id):
         if prefix_id not in self.entries:
             raise NotFound("unknown or evicted prefix id")
-        return list(self.entries[prefix_id][2])
+        return self.entries[prefix_id][2]
+
+    def pages(self, prefix_id, layer=None):
+        """Page list of a live prefix in `layer` (default: its first layer)."""
+        if prefix_id not in self.entries:
+            raise NotFound("unknown or evicted prefix id")
+        if layer is None:
+            layer = self.entries[prefix_id][2]
+        return list(self._layer_pages(prefix_id, int(layer)))
 
     def prefix_len(self, prefix_id):
         if prefix_id not in self.entries:
@@ -205,9 +255,8 @@ class PagedPrefixStore:
         two arrays [m, Hkv, D]."""
         if not 0 <= layer < self.L:
             raise InvalidArgument("layer out of range")
-        if prefix_id not in self.entries:
-            raise NotFound("unknown or evicted prefix id")
-        _, m, pages = self.entries[prefix_id]
+        pages = self._layer_pages(prefix_id, layer)
+        m = self.entries[prefix_id][1]
         k = np.empty((m, self.Hkv, self.D), dtype=np.float64)
         v = np.empty((m, self.Hkv, self.D), dtype=np.float64)
         for t in range(m):

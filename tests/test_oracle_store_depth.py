@@ -99,7 +99,7 @@ def test_store_traces_against_model(trace, num_pages, seed):
             assert (hit, pid, pages) == (want[0] == "hit", want[1], want[2])
         # conservation: every page is free or owned exactly once
         owned = [p for pid in real.entries for p in real.pages(pid)]
-        assert sorted(owned + list(real.free)) == list(range(num_pages))
+        assert sorted(owned + list(real.free[0])) == list(range(num_pages))
         # live keys agree, evicted keys are gone
         live = {e[0] for e in model.live}
         for k in range(7):
@@ -133,6 +133,120 @@ def test_store_fifo_not_lru_and_ids_never_reused():
         s.put(11, kv(17), kv(17))
     with pytest.raises(oracle.InvalidArgument):
         oracle.PagedPrefixStore(1, 1, 2, 16, 4, free_order=[0, 1, 1, 2])
+
+
+# -- store with per-layer page lists (a kept deep-layer prefix owns layers first_layer .. L-1 only) ------
+
+class LayeredModel:
+    """Independent model of the per-layer store: an owner array per layer (which prefix holds each page)
+    and, per layer, the order in which pages became free, replayed from the events."""
+
+    def __init__(self, L, caps, P, order):
+        self.L, self.P = L, P
+        self.caps = caps
+        self.freed_at = [{p: i for i, p in enumerate(q for q in order if q < caps[l])} for l in range(L)]
+        self.tick = len(order)
+        self.live = []          # [key, m, first, {layer: pages}, id]
+        self.count = 0
+
+    def free_list(self, l):
+        return [p for p, _ in sorted(self.freed_at[l].items(), key=lambda kv: kv[1])]
+
+    def insert(self, key, m, first):
+        for e in self.live:
+            if e[0] == key:
+                return ("hit", e[4], e[3][first]) if (e[1], e[2]) == (m, first) else ("invalid",)
+        need = -(-m // self.P)
+        if any(need > self.caps[l] for l in range(first, self.L)):
+            return ("nomem",)
+        while any(len(self.freed_at[l]) < need for l in range(first, self.L)):
+            old = self.live.pop(0)
+            for l, pages in old[3].items():
+                for p in pages:
+                    self.freed_at[l][p] = self.tick
+                    self.tick += 1
+        got = {}
+        for l in range(first, self.L):
+            got[l] = self.free_list(l)[:need]
+            for p in got[l]:
+                del self.freed_at[l][p]
+        self.live.append([key, m, first, got, self.count])
+        self.count += 1
+        return ("miss", self.count - 1, got[first])
+
+
+@given(st.lists(st.tuples(st.integers(0, 7), st.integers(1, 40), st.integers(0, 2)), min_size=1, max_size=40),
+       st.integers(2, 10), st.integers(0, 3), st.booleans())
+@settings(max_examples=150, deadline=None)
+def test_layered_store_traces_against_model(trace, num_pages, seed, shrink_shallow):
+    P, L, H, D = 8, 3, 1, 2
+    order = list(range(num_pages)) if seed == 0 else np.random.default_rng(seed).permutation(num_pages).tolist()
+    caps = [max(1, num_pages // 2), max(1, (3 * num_pages) // 4), num_pages] if shrink_shallow else [num_pages] * L
+    real = oracle.PagedPrefixStore(L, H, D, P, num_pages, free_order=order, layer_pages=caps)
+    model = LayeredModel(L, caps, P, order)
+    for key, m, first in trace:
+        want = model.insert(key, m, first)
+        if want[0] == "invalid":
+            with pytest.raises(oracle.InvalidArgument):
+                real.reserve(key, m, first)
+        elif want[0] == "nomem":
+            with pytest.raises(oracle.OutOfPages):
+                real.reserve(key, m, first)
+        else:
+            pid, hit, pages = real.reserve(key, m, first)
+            assert (hit, pid, pages) == (want[0] == "hit", want[1], want[2])
+        # per layer: every page below the layer's capacity is free or owned exactly once, and the
+        # free queue has the model's order
+        for l in range(L):
+            owned = [p for e in model.live if l in e[3] for p in e[3][l]]
+            assert sorted(owned + list(real.free[l])) == list(range(caps[l]))
+            assert list(real.free[l]) == model.free_list(l)
+        for e in model.live:
+            for l in range(L):
+                if l in e[3]:
+                    assert real.pages(e[4], l) == e[3][l]
+                else:
+                    with pytest.raises(oracle.InvalidArgument):
+                        real.pages(e[4], l)
+
+
+def test_layered_store_hand_sequence():
+    """Three layers of four pages.  A full-depth prefix, then a deep-only one (layers 1-2), then a
+    full-depth one that no longer fits layer 1 without evicting the oldest prefix: FIFO order is by
+    insertion, whatever layers a prefix owns, and the lists of the third prefix differ by layer."""
+    s = oracle.PagedPrefixStore(3, 1, 2, 16, 4)
+    a, _, pa = s.reserve(1, 32)                  # pages 0, 1 in every layer
+    b, _, pb = s.reserve(2, 32, first_layer=1)   # pages 2, 3 in layers 1 and 2; layer 0 untouched
+    assert (a, pa, b, pb) == (0, [0, 1], 1, [2, 3])
+    assert [list(q) for q in s.free] == [[2, 3], [], []]
+    with pytest.raises(oracle.InvalidArgument):
+        s.pages(b, 0)
+    with pytest.raises(oracle.InvalidArgument):
+        s.prefix_kv(0, b)
+    assert s.reserve(2, 32, first_layer=1)[1] is True
+    with pytest.raises(oracle.InvalidArgument):
+        s.reserve(2, 32, first_layer=2)          # same key, another first layer
+    c, hit, pc = s.reserve(3, 32)                # layers 1, 2 are full: the oldest prefix (key 1) goes
+    assert (c, hit) == (2, False)
+    assert [s.pages(c, l) for l in range(3)] == [[2, 3], [0, 1], [0, 1]]
+    assert [list(q) for q in s.free] == [[0, 1], [], []]
+    with pytest.raises(oracle.NotFound):
+        s.lookup(1)
+    # values written to one layer are read back from that layer only
+    kv = np.arange(32 * 2, dtype=np.float64).reshape(32, 1, 2)
+    s.update_layer(b, 2, kv, kv + 1)
+    k2, v2 = s.prefix_kv(2, b)
+    assert (k2 == kv).all() and (v2 == kv + 1).all()
+    k1, _ = s.prefix_kv(1, b)
+    assert (k1 == 0).all()
+    with pytest.raises(oracle.InvalidArgument):
+        s.update_layer(b, 0, kv, kv)
+    with pytest.raises(oracle.InvalidArgument):
+        oracle.PagedPrefixStore(3, 1, 2, 16, 4, layer_pages=[4, 5, 4])
+    small = oracle.PagedPrefixStore(2, 1, 2, 16, 4, layer_pages=[1, 4])
+    with pytest.raises(oracle.OutOfPages):
+        small.reserve(9, 32)                      # two pages do not fit layer 0's single page
+    assert small.reserve(9, 32, first_layer=1)[2] == [0, 1]
 
 
 def test_workload_recipes_are_deterministic_and_shaped():
