@@ -132,11 +132,20 @@ class Job:
         self.delta = delta if w.num_layers > 1 else 0
         self.t = 1                                    # 1-based denoising step (Eq. 5)
         npages = w.pages_needed() + 1
-        if self.delta > 0:                            # per-request kept prefix K/V of the deep layers
-            npages += sum((w.prefix_lens[g] + 15) // 16 for g in w.req_prefix)
+        layer_pages = None
+        if self.delta > 0:
+            # Per-request kept prefix K/V of the deep layers (Eq. 5): request i keeps them from layer
+            # depth[i] on, so layer l's pool holds the shared prefixes plus the kept prefixes of the
+            # requests whose depth is at most l.
+            depth0 = host_reuse_depth(binding, w)
+            need = [(w.prefix_lens[g] + 15) // 16 for g in w.req_prefix]
+            layer_pages = [npages + sum(nd for nd, d in zip(need, depth0) if d <= l) for l in range(w.num_layers)]
+            npages = max(layer_pages)
         order = workloads.shuffled_page_order(npages, 7) if w.shuffle_pages else None
         self.bc = binding.BiCache(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim, npages, w.dtype,
-                                  w.total_rows, w.num_requests, device=device, free_order=order)
+                                  w.total_rows, w.num_requests, device=device, free_order=order,
+                                  layer_pages=layer_pages)
+        self.pool_bytes = 2 * self.bc.k_pool.numel()
         self.bc.set_depth_table(workloads.standin_depth_table(w.num_layers))
         self.keys = [workloads.prefix_key(w, g) for g in range(len(w.prefix_lens))]
         for g in range(len(w.prefix_lens)):
@@ -145,8 +154,9 @@ class Job:
             del kc, vc
         self.private = [-1] * w.num_requests
         if self.delta > 0:
-            self.private = [self.bc.reserve_prefix(0x6000000000000000 + i, w.prefix_lens[g])[0]
-                            for i, g in enumerate(w.req_prefix)]
+            self.private = [self.bc.reserve_prefix(0x6000000000000000 + i, w.prefix_lens[g], first_layer=int(d))[0]
+                            if d < w.num_layers else -1
+                            for i, (g, d) in enumerate(zip(w.req_prefix, depth0))]
         self.q, self.k, self.v = workloads.draw_full_qkv(w, "cuda")
         self.out = torch.empty_like(self.q)
         self.single_layer = w.num_layers == 1
@@ -230,6 +240,31 @@ class Job:
         w = self.w
         return w.num_layers * sum(4 * w.head_dim * w.num_q_heads * n * (w.prefix_lens[g] + n)
                                   for g, n in zip(w.req_prefix, w.suffix_lens))
+
+
+def host_reuse_depth(binding, w):
+    """The depth rule through a host-only context of the library (no device work): needed before the
+    device context exists, to size the per-layer pools of the kept deep-layer prefixes."""
+    import ctypes as C
+    lib = binding.load_library()
+    cfg = binding.Config(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim, 16, 1, binding._dtype_code(w.dtype), -1)
+    ctx = C.c_void_p()
+    assert lib.bicache_create(C.byref(cfg), C.byref(ctx)) == binding.OK
+    i32p = C.POINTER(C.c_int32)
+    table = np.ascontiguousarray(w_table(w), dtype=np.int32)
+    assert lib.bicache_set_depth_table(ctx, table.ctypes.data_as(i32p), 101) == binding.OK
+    m = np.ascontiguousarray(w.req_prefix_len(), dtype=np.int32)
+    n = np.ascontiguousarray(w.suffix_lens, dtype=np.int32)
+    out = np.zeros(len(m), dtype=np.int32)
+    assert lib.bicache_reuse_depth(ctx, len(m), m.ctypes.data_as(i32p), n.ctypes.data_as(i32p),
+                                   out.ctypes.data_as(i32p)) == binding.OK
+    lib.bicache_destroy(ctx)
+    return out.tolist()
+
+
+def w_table(w):
+    from paper_2606_07571_b200 import workloads
+    return workloads.standin_depth_table(w.num_layers)
 
 
 def time_call(fn, iters, flush):
@@ -318,7 +353,8 @@ def measure_steps(job, name, steps, warmup, flush, peaks, rank, local_rank, worl
         ref_ms = [m for m, r in zip(per_step_ms, is_ref) if r]
         reu_ms = [m for m, r in zip(per_step_ms, is_ref) if not r]
         flops = (len(ref_ms) * flops + len(reu_ms) * job.reuse_step_flops()) / steps   # mean FLOPs per step
-        refresh_info = {"delta": job.delta, "refresh_steps": len(ref_ms), "reuse_steps": len(reu_ms),
+        refresh_info = {"delta": job.delta, "store_bytes": job.pool_bytes,
+                        "refresh_steps": len(ref_ms), "reuse_steps": len(reu_ms),
                         "ms_refresh_step": sum(ref_ms) / max(1, len(ref_ms)),
                         "ms_reuse_step": sum(reu_ms) / max(1, len(reu_ms)) if reu_ms else None}
 

@@ -73,7 +73,7 @@ typedef struct {
   int32_t head_dim;          /* D: 128 for the tensor-core path; any multiple of 32 up to 256
                                 on the SIMT path                                               */
   int32_t page_size;         /* tokens per page; must be 16                                    */
-  int32_t num_pages;         /* pool capacity; page p addresses the same slot in every layer   */
+  int32_t num_pages;         /* pages per layer (see layer_pages for layers that hold fewer)   */
   int32_t dtype;             /* BICACHE_F32 or BICACHE_BF16: type of q/k/v/out and the pools   */
   int32_t device;            /* CUDA device ordinal.  A negative value creates a host-only
                                 context: the store's bookkeeping and the depth rule work (pools
@@ -84,14 +84,20 @@ typedef struct {
   const int32_t* initial_free_order; /* host, num_pages entries, a permutation of 0..num_pages-1
                                 giving the initial order of the free-page queue; NULL = 0,1,2,...
                                 Read during bicache_create only.                               */
+  const int32_t* layer_pages; /* host, num_layers entries, or NULL: pages of each layer's pool,
+                                1 .. num_pages (NULL: num_pages everywhere).  Shallow layers may hold
+                                fewer: the kept deep-layer prefixes of Eq. 5 own no pages there.
+                                Layer l's free queue starts as the pages below its capacity in the
+                                initial order.  Read during bicache_create only.                 */
   void* k_pool;              /* device, bicache_pool_bytes() bytes, caller-owned               */
   void* v_pool;              /* device, same size                                              */
   void* workspace;           /* device scratch, caller-owned, 256-byte aligned                 */
   size_t workspace_bytes;    /* >= bicache_workspace_bytes() for the batches to be run         */
 } bicache_config;
 
-/* Bytes of ONE pool (K or V): L * num_pages * Hkv * page_size * D elements.  The order of
- * elements inside a page is private to the library: only bicache_put_prefix writes pools. */
+/* Bytes of ONE pool (K or V): (sum over the layers of their pages) * Hkv * page_size * D elements,
+ * the layers one after the other.  The order of elements inside a page is private to the library:
+ * only the library writes pools.  0 for an invalid configuration. */
 size_t bicache_pool_bytes(const bicache_config* cfg);
 
 /* Workspace needed to run batches of at most max_requests requests and max_total_rows query rows
@@ -122,13 +128,16 @@ int32_t bicache_set_depth_table(bicache_ctx* ctx, const int32_t* table, int32_t 
  * between layers (>= m*Hkv*D), rows dense.  m >= 1.
  *   key present with the same m : hit, nothing is written, *was_hit = 1.
  *   key present with another m  : INVALID.
- *   ceil(m/16) > num_pages      : NOMEM, nothing evicted.
- *   otherwise: evict whole prefixes, oldest insertion first (hits do not refresh age), until
- *   enough pages are free (their pages join the tail of the free queue in page-table order),
- *   take ceil(m/16) pages from the head of the queue, and enqueue the scatter of all L layers
- *   on `stream`.  The caller may free k, v once the stream has passed this point.
+ *   ceil(m/16) > a layer's pages : NOMEM, nothing evicted.
+ *   otherwise: every layer has its own free queue.  Evict whole prefixes, oldest insertion first
+ *   (hits do not refresh age), until every layer has enough free pages (an evicted prefix's pages
+ *   join the tail of their layer's queue in page-table order), take ceil(m/16) pages from the head of
+ *   every layer's queue, and enqueue the scatter of all L layers on `stream`.  The caller may free
+ *   k, v once the stream has passed this point.  While every prefix owns all layers (no
+ *   bicache_reserve_prefix_layers with a first layer > 0, no layer_pages) the queues move in
+ *   lockstep and a prefix has the same page list in every layer.
  * prefix_id (host, required) receives an id that is never reused.  was_hit (host, optional).
- * pages_out (host, optional, capacity pages_cap) receives the page ids in token order;
+ * pages_out (host, optional, capacity pages_cap) receives the page ids of layer 0 in token order;
  * INVALID if pages_cap is too small (checked before anything changes). */
 int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const void* v,
                            int64_t layer_stride, void* stream,
@@ -143,10 +152,15 @@ uint64_t bicache_hash_tokens(const int32_t* tokens, int64_t n);
 /* KV store lookup (Sec. 5.2 "On a cache hit").  NOTFOUND if the key is absent or evicted. */
 int32_t bicache_lookup_prefix(const bicache_ctx* ctx, uint64_t key, int32_t* prefix_id, int32_t* m);
 
-/* Page list of a live prefix, in token order.  *n receives the page count; pages_out (host) may be
- * NULL to query the count only.  NOTFOUND for an evicted id, INVALID if cap is too small. */
+/* Page list of a live prefix in its first layer, in token order.  *n receives the page count; pages_out
+ * (host) may be NULL to query the count only.  NOTFOUND for an evicted id, INVALID if cap is too small. */
 int32_t bicache_prefix_pages(const bicache_ctx* ctx, int32_t prefix_id, int32_t* pages_out, int32_t cap,
                              int32_t* n);
+
+/* The same for one layer (a negative layer: the prefix's first layer).  INVALID if the prefix owns no
+ * pages in that layer. */
+int32_t bicache_prefix_pages_layer(const bicache_ctx* ctx, int32_t prefix_id, int32_t layer, int32_t* pages_out,
+                                   int32_t cap, int32_t* n);
 
 /* (2) Per-request shallow depth (Sec. 5.1/5.2).  Host arrays of length R.  prefix_len[i] = m_i
  * shared-prefix tokens, nonshared_len[i] = n_i = every other token of the input string (prompt
@@ -216,6 +230,16 @@ int32_t bicache_is_refresh_step(int32_t t, int32_t delta);
 int32_t bicache_reserve_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, int32_t* prefix_id,
                                int32_t* was_hit, int32_t* pages_out, int32_t pages_cap);
 
+/* The same for a prefix that only the layers first_layer .. L-1 keep (Eq. 5: a request's own prefix K/V
+ * are kept in the layers past its shallow depth, so first_layer = depth[i]): pages are taken from, and
+ * on eviction returned to, the queues of those layers only; the shallow layers' pages stay free for
+ * other prefixes.  pages_out receives the list of layer first_layer.  A hit needs the same m and the
+ * same first_layer (INVALID otherwise).  Every call that names a layer for this prefix (update, read,
+ * project, the attention calls) answers INVALID for a layer below first_layer. */
+int32_t bicache_reserve_prefix_layers(bicache_ctx* ctx, uint64_t key, int32_t m, int32_t first_layer,
+                                      int32_t* prefix_id, int32_t* was_hit, int32_t* pages_out,
+                                      int32_t pages_cap);
+
 /* Overwrite ONE layer of an existing prefix (Eq. 5, refresh step: the kept K/V become the ones just
  * computed).  k, v: device, rows [m][Hkv][D] of the context's dtype, `kv_row_stride` elements between
  * consecutive rows (so k may point at the request's first row inside a packed [rows][Hkv][D] tensor),
@@ -277,7 +301,8 @@ int32_t bicache_attend_step(bicache_ctx* ctx, int32_t layer, int32_t t, int32_t 
  * length).  sim_out: HOST array of L floats.  Runs on `stream` and synchronises it before returning
  * (an offline call).  A zero vector on either side gives 0.  Uses the context's workspace as scratch.
  * NOTFOUND for an unknown or evicted id, INVALID for a bad pointer or stride, UNSUPPORTED on a
- * host-only context. */
+ * host-only context and for a prefix whose page list differs between layers (profile shared prefixes
+ * before any partial-depth reservation, or in a context of their own). */
 int32_t bicache_prefix_similarity(bicache_ctx* ctx, int32_t prefix_id, const void* k_ref, const void* v_ref,
                                   int64_t layer_stride, float* sim_out, void* stream);
 

@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbicache.
 EXPORTED = [
     "bicache_pool_bytes", "bicache_workspace_bytes", "bicache_create", "bicache_destroy",
     "bicache_set_path", "bicache_set_depth_table", "bicache_put_prefix", "bicache_lookup_prefix",
-    "bicache_prefix_pages", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
+    "bicache_prefix_pages", "bicache_prefix_pages_layer", "bicache_reserve_prefix_layers", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
     "bicache_attend_layer", "bicache_attend_full_static",
     "bicache_is_refresh_step", "bicache_reserve_prefix", "bicache_update_prefix_layer", "bicache_attend_step",
     "bicache_read_prefix_layer", "bicache_project_prefix_layer",
@@ -45,6 +45,7 @@ class Config(C.Structure):
         ("head_dim", C.c_int32), ("page_size", C.c_int32), ("num_pages", C.c_int32),
         ("dtype", C.c_int32), ("device", C.c_int32),
         ("initial_free_order", C.POINTER(C.c_int32)),
+        ("layer_pages", C.POINTER(C.c_int32)),
         ("k_pool", C.c_void_p), ("v_pool", C.c_void_p),
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
     ]
@@ -81,6 +82,10 @@ def load_library():
     lib.bicache_lookup_prefix.argtypes = [vp, C.c_uint64, i32p, i32p]
     lib.bicache_prefix_pages.restype = C.c_int32
     lib.bicache_prefix_pages.argtypes = [vp, C.c_int32, i32p, C.c_int32, i32p]
+    lib.bicache_prefix_pages_layer.restype = C.c_int32
+    lib.bicache_prefix_pages_layer.argtypes = [vp, C.c_int32, C.c_int32, i32p, C.c_int32, i32p]
+    lib.bicache_reserve_prefix_layers.restype = C.c_int32
+    lib.bicache_reserve_prefix_layers.argtypes = [vp, C.c_uint64, C.c_int32, C.c_int32, i32p, i32p, i32p, C.c_int32]
     lib.bicache_reuse_depth.restype = C.c_int32
     lib.bicache_reuse_depth.argtypes = [vp, C.c_int32, i32p, i32p, i32p]
     lib.bicache_attend.restype = C.c_int32
@@ -157,7 +162,8 @@ class BiCache:
     """One library context plus the torch-owned device buffers it needs."""
 
     def __init__(self, num_layers, num_q_heads, num_kv_heads, head_dim, num_pages, dtype,
-                 max_total_rows, max_requests, device=0, page_size=16, free_order=None, workspace_bytes=None):
+                 max_total_rows, max_requests, device=0, page_size=16, free_order=None, workspace_bytes=None,
+                 layer_pages=None):
         self.lib = load_library()
         if not torch.cuda.is_available():
             raise RuntimeError("BiCache needs a CUDA device; there is no CPU path")
@@ -166,6 +172,11 @@ class BiCache:
         self.L, self.Hq, self.Hkv, self.D = num_layers, num_q_heads, num_kv_heads, head_dim
         cfg = Config(num_layers, num_q_heads, num_kv_heads, head_dim, page_size, num_pages,
                      _dtype_code(dtype), device)
+        self._layer_pages = None
+        if layer_pages is not None:              # per-layer pool capacities
+            self._layer_pages, ptr = _i32(layer_pages)
+            assert len(self._layer_pages) == num_layers
+            cfg.layer_pages = ptr
         pool_bytes = self.lib.bicache_pool_bytes(C.byref(cfg))
         ws_bytes = self.lib.bicache_workspace_bytes(C.byref(cfg), int(max_total_rows), int(max_requests))
         if workspace_bytes is not None:          # a caller that sizes the workspace itself
@@ -230,15 +241,15 @@ class BiCache:
         self._check(st, "bicache_put_prefix")
         return pid.value, bool(hit.value), pages[:cap].tolist()
 
-    def reserve_prefix(self, key, m):
-        """Pages for a prefix of m tokens, no K/V written (Eq. 5's per-request cache).  Returns
-        (prefix_id, was_hit, pages)."""
+    def reserve_prefix(self, key, m, first_layer=0):
+        """Pages for a prefix of m tokens in the layers first_layer .. L-1, no K/V written (Eq. 5's
+        per-request cache).  Returns (prefix_id, was_hit, pages of layer first_layer)."""
         pid, hit = C.c_int32(-1), C.c_int32(0)
         cap = (m + 15) // 16
         pages = np.zeros(max(cap, 1), dtype=np.int32)
-        st = self.lib.bicache_reserve_prefix(self.ctx, C.c_uint64(key), m, C.byref(pid), C.byref(hit),
-                                             pages.ctypes.data_as(C.POINTER(C.c_int32)), cap)
-        self._check(st, "bicache_reserve_prefix")
+        st = self.lib.bicache_reserve_prefix_layers(self.ctx, C.c_uint64(key), m, first_layer, C.byref(pid),
+                                                    C.byref(hit), pages.ctypes.data_as(C.POINTER(C.c_int32)), cap)
+        self._check(st, "bicache_reserve_prefix_layers")
         return pid.value, bool(hit.value), pages[:cap].tolist()
 
     def update_prefix_layer(self, prefix_id, layer, k, v):
@@ -308,12 +319,15 @@ class BiCache:
                     "bicache_lookup_prefix")
         return pid.value, m.value
 
-    def prefix_pages(self, prefix_id):
+    def prefix_pages(self, prefix_id, layer=-1):
+        """Page list of a prefix in `layer` (default: its first layer)."""
         n = C.c_int32(0)
-        self._check(self.lib.bicache_prefix_pages(self.ctx, prefix_id, None, 0, C.byref(n)), "bicache_prefix_pages")
+        self._check(self.lib.bicache_prefix_pages_layer(self.ctx, prefix_id, layer, None, 0, C.byref(n)),
+                    "bicache_prefix_pages_layer")
         pages = np.zeros(max(n.value, 1), dtype=np.int32)
-        self._check(self.lib.bicache_prefix_pages(self.ctx, prefix_id, pages.ctypes.data_as(C.POINTER(C.c_int32)),
-                                                  n.value, C.byref(n)), "bicache_prefix_pages")
+        self._check(self.lib.bicache_prefix_pages_layer(self.ctx, prefix_id, layer,
+                                                        pages.ctypes.data_as(C.POINTER(C.c_int32)), n.value,
+                                                        C.byref(n)), "bicache_prefix_pages_layer")
         return pages[:n.value].tolist()
 
     def reuse_depth(self, prefix_len, nonshared_len):

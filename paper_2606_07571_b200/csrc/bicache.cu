@@ -37,12 +37,22 @@ constexpr long long kMaxPartialRowHeads = (long long)kTargetCtas * kTileRows;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// A stored prefix owns ceil(m / 16) pages in each of the layers first_layer .. L-1 (a shared prefix in all
+// of them; a request's kept deep-layer prefix, Eq. 5, from its shallow depth on).  Every layer has its own
+// free queue; as long as all prefixes own all layers the queues move in lockstep and a prefix has ONE
+// page list (`uniform`); otherwise `layer_pages[l - first_layer]` is the list of layer l.
 struct PrefixEntry {
   uint64_t key;
   int32_t id;
   int32_t m;
-  std::vector<int32_t> pages;
+  int32_t first_layer = 0;
+  bool uniform = true;
+  std::vector<int32_t> pages;                         // the list of layer first_layer
+  std::vector<std::vector<int32_t>> layer_pages;      // only if !uniform
 };
+inline const std::vector<int32_t>& pages_of(const PrefixEntry& e, int layer) {
+  return e.uniform ? e.pages : e.layer_pages[layer - e.first_layer];
+}
 
 // A schedule kept on the device: where it lives in the schedule arena and what batch it describes.
 struct CachedSchedule {
@@ -77,7 +87,10 @@ struct bicache_ctx {
   int proj_pairs = 0;                                             // CTA pairs of the projection kernel the device runs at once
   bool host_only = false;                                         // cfg.device < 0: bookkeeping only
   int path = BICACHE_PATH_AUTO;
-  std::deque<int32_t> free_pages;
+  std::vector<std::deque<int32_t>> free_pages;                   // one queue per layer
+  std::vector<int32_t> layer_cap;                                 // pages of each layer's pool
+  std::vector<long long> layer_off;                               // byte offset of each layer inside a pool
+  bool uniform_caps = true;                                       // every layer holds cfg.num_pages pages
   std::list<PrefixEntry> fifo;                                    // insertion order, oldest first
   std::unordered_map<uint64_t, std::list<PrefixEntry>::iterator> by_key;
   std::unordered_map<int32_t, std::list<PrefixEntry>::iterator> by_id;
@@ -155,6 +168,7 @@ size_t partial_bytes_for(const bicache_config* c) {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// The whole pools (layer stride = a full layer: only meaningful when every layer has the same capacity).
 PoolView pool_view(const bicache_ctx* ctx) {
   PoolView p;
   p.k = static_cast<const char*>(ctx->cfg.k_pool);
@@ -163,6 +177,13 @@ PoolView pool_view(const bicache_ctx* ctx) {
   p.num_kv_heads = ctx->cfg.num_kv_heads;
   p.layer_bytes = (long long)ctx->cfg.num_pages * ctx->cfg.num_kv_heads * p.page_bytes;
   p.swizzled = ctx->swizzled ? 1 : 0;
+  return p;
+}
+// One layer of the pools, addressed as layer 0 of the view.
+PoolView pool_view_layer(const bicache_ctx* ctx, int layer) {
+  PoolView p = pool_view(ctx);
+  p.k += ctx->layer_off[layer];
+  p.v += ctx->layer_off[layer];
   return p;
 }
 
@@ -258,10 +279,17 @@ size_t arena_place(bicache_ctx* ctx, size_t bytes) {
 
 // Build (or find) the device-resident schedule for this batch.  Returns its index in ctx->sched or -1.
 // `tiled`: kind 0 on the tensor path - the query rows of a prefix group are packed into row tiles.
-int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int R, const int32_t* prefix_id,
+int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int layer, int R, const int32_t* prefix_id,
                      const int64_t* row_off, const int32_t* seqlen, cudaStream_t stream, int* status) {
   *status = BICACHE_OK;
-  const int key_kind = kind + (tiled ? 8 : 0);
+  // A schedule holds the page lists of its prefixes.  They are the same in every layer unless some
+  // prefix has per-layer lists; only then is the schedule tied to the layer it was built for.
+  int layer_tag = 0;
+  if (kind != 1)
+    for (int i = 0; i < R; ++i)
+      if (prefix_id[i] >= 0 && (i == 0 || prefix_id[i] != prefix_id[i - 1]) && !ctx->by_id.at(prefix_id[i])->uniform)
+        layer_tag = layer + 1;
+  const int key_kind = kind + (tiled ? 8 : 0) + 16 * layer_tag;
   uint64_t hash = fnv1a(0xcbf29ce484222325ull, &key_kind, sizeof(key_kind));
   hash = fnv1a(hash, &R, sizeof(R));
   hash = fnv1a(hash, row_off, sizeof(int64_t) * R);
@@ -297,7 +325,8 @@ int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int R, const int32_
       if (prefix_id[i] != last_pid) {
         last_pid = prefix_id[i];
         last_page_off = (int)pages.size();
-        pages.insert(pages.end(), e.pages.begin(), e.pages.end());
+        const std::vector<int32_t>& pl = pages_of(e, layer);
+        pages.insert(pages.end(), pl.begin(), pl.end());
       }
       r.page_off = last_page_off;
     }
@@ -636,8 +665,11 @@ int prepare_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, cons
         if (std::find(seen.begin(), seen.end(), p) != seen.end())
           return fail(ctx, BICACHE_ERR_INVALID, "requests of one prefix are not contiguous");
         seen.push_back(p);
-        if (ctx->by_id.find(p) == ctx->by_id.end())
+        auto found = ctx->by_id.find(p);
+        if (found == ctx->by_id.end())
           return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
+        if (found->second->first_layer > layer)
+          return fail(ctx, BICACHE_ERR_INVALID, "the prefix owns no pages in this layer");
       }
     }
   }
@@ -662,15 +694,15 @@ int prepare_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, cons
   int st = BICACHE_OK;
   int entry = -1;
   if (key_ranges) {
-    entry = prepare_schedule(ctx, 2, false, R, prefix_id, row_off, seqlen, stream, &st);
+    entry = prepare_schedule(ctx, 2, false, layer, R, prefix_id, row_off, seqlen, stream, &st);
     if (entry < 0) {                                     // does not fit: the general path
       key_ranges = false;
       ctx->last_error.clear();
     }
   }
   if (entry < 0)
-    entry = prepare_schedule(ctx, kind, kind == 0 && pc->use_tensor && kTiledAttend, R, prefix_id, row_off, seqlen,
-                             stream, &st);
+    entry = prepare_schedule(ctx, kind, kind == 0 && pc->use_tensor && kTiledAttend, layer, R, prefix_id, row_off,
+                             seqlen, stream, &st);
   if (entry < 0) return st;
   pc->entry = entry;
   pc->key_ranges = key_ranges;
@@ -728,12 +760,12 @@ int launch_attention(bicache_ctx* ctx, const PreparedCall& pc, int32_t layer, co
   t.Hq = cfg.num_q_heads;
   t.Hkv = cfg.num_kv_heads;
   t.D = cfg.head_dim;
-  t.layer = layer;
+  t.layer = 0;                                  // the pool view below starts at this call's layer
   t.scale = softmax_scale;
   t.part_o = ctx->d_part_o;
   t.part_lse = ctx->d_part_lse;
   t.total_tokens = c.total_tokens;
-  const PoolView pool = pool_view(ctx);
+  const PoolView pool = pool_view_layer(ctx, layer);
 
   cudaError_t e;
   ctx->last_kernel = pc.key_ranges ? BICACHE_KERNEL_KEY_RANGES : pc.use_tensor ? BICACHE_KERNEL_TENSOR : BICACHE_KERNEL_SIMT;
@@ -790,7 +822,13 @@ extern "C" {
 size_t bicache_pool_bytes(const bicache_config* cfg) {
   if (!sane(cfg)) return 0;
   const size_t es = cfg->dtype == BICACHE_F32 ? 4 : 2;
-  return (size_t)cfg->num_layers * cfg->num_pages * cfg->num_kv_heads * cfg->page_size * cfg->head_dim * es;
+  size_t pages = 0;
+  for (int l = 0; l < cfg->num_layers; ++l) {
+    const int32_t c = cfg->layer_pages ? cfg->layer_pages[l] : cfg->num_pages;
+    if (c < 1 || c > cfg->num_pages) return 0;
+    pages += (size_t)c;
+  }
+  return pages * cfg->num_kv_heads * cfg->page_size * cfg->head_dim * es;
 }
 
 size_t bicache_workspace_bytes(const bicache_config* cfg, int64_t max_total_rows, int32_t max_requests) {
@@ -809,6 +847,9 @@ int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
   const bool host_only = cfg->device < 0;
   const size_t part = partial_bytes_for(cfg);
   const size_t put_pages = align_up((size_t)cfg->num_pages * sizeof(int) + 16, 256);
+  if (cfg->layer_pages)
+    for (int l = 0; l < cfg->num_layers; ++l)
+      if (cfg->layer_pages[l] < 1 || cfg->layer_pages[l] > cfg->num_pages) return BICACHE_ERR_INVALID;
   if (!host_only) {
     if (!cfg->k_pool || !cfg->v_pool || !cfg->workspace) return BICACHE_ERR_INVALID;
     if ((reinterpret_cast<uintptr_t>(cfg->k_pool) & 255) || (reinterpret_cast<uintptr_t>(cfg->v_pool) & 255) ||
@@ -835,10 +876,26 @@ int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
   ctx->host_only = host_only;
   ctx->cfg = *cfg;
   ctx->cfg.initial_free_order = nullptr;
+  ctx->cfg.layer_pages = nullptr;
   ctx->esize = esize;
   ctx->swizzled = swz;
   ctx->tensor_ok = tensor_ok;
-  ctx->free_pages.assign(order.begin(), order.end());
+  // per layer: capacity, place inside a pool, and the free queue (the pages below the layer's capacity,
+  // in the initial order)
+  ctx->free_pages.resize(cfg->num_layers);
+  ctx->layer_cap.resize(cfg->num_layers);
+  ctx->layer_off.resize(cfg->num_layers);
+  long long off = 0;
+  const long long slice = (long long)cfg->num_kv_heads * kPageSize * cfg->head_dim * esize;
+  for (int l = 0; l < cfg->num_layers; ++l) {
+    const int32_t cap = cfg->layer_pages ? cfg->layer_pages[l] : cfg->num_pages;
+    ctx->layer_cap[l] = cap;
+    ctx->layer_off[l] = off;
+    off += (long long)cap * slice;
+    if (cap != cfg->num_pages) ctx->uniform_caps = false;
+    for (int32_t pg : order)
+      if (pg < cap) ctx->free_pages[l].push_back(pg);
+  }
   if (host_only) {
     *out = ctx;
     return BICACHE_OK;
@@ -910,20 +967,23 @@ int32_t bicache_set_depth_table(bicache_ctx* ctx, const int32_t* table, int32_t 
 }  // extern "C"
 
 namespace {
-// Insert a prefix: hit / miss / FIFO eviction / page allocation, and (write = true) the scatter of all
-// layers' K/V into the page images.
+// Insert a prefix that owns the layers first_layer .. L-1: hit / miss / FIFO eviction / page allocation
+// per layer, and (write = true, first_layer = 0) the scatter of all layers' K/V into the page images.
 int32_t put_impl(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const void* v, int64_t layer_stride,
                  void* stream_, int32_t* prefix_id, int32_t* was_hit, int32_t* pages_out, int32_t pages_cap,
-                 bool write) {
+                 bool write, int32_t first_layer) {
   if (!ctx) return BICACHE_ERR_INVALID;
   if (!prefix_id) return fail(ctx, BICACHE_ERR_INVALID, "prefix_id is required");
   if (m < 1) return fail(ctx, BICACHE_ERR_INVALID, "empty prefix");
   const bicache_config& cfg = ctx->cfg;
+  const int L = cfg.num_layers;
+  if (first_layer < 0 || first_layer >= L) return fail(ctx, BICACHE_ERR_INVALID, "first layer out of range");
   const int need = (m + kPageSize - 1) / kPageSize;
   auto found = ctx->by_key.find(key);
   if (found != ctx->by_key.end()) {
     const PrefixEntry& e = *found->second;
-    if (e.m != m) return fail(ctx, BICACHE_ERR_INVALID, "key already present with another length");
+    if (e.m != m || e.first_layer != first_layer)
+      return fail(ctx, BICACHE_ERR_INVALID, "key already present with another length or first layer");
     if (pages_out && pages_cap < need) return fail(ctx, BICACHE_ERR_INVALID, "pages_out too small");
     *prefix_id = e.id;
     if (was_hit) *was_hit = 1;
@@ -935,11 +995,18 @@ int32_t put_impl(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const
   const int64_t row_elems = (int64_t)cfg.num_kv_heads * cfg.head_dim;
   if (write && (layer_stride < (int64_t)m * row_elems || (layer_stride * ctx->esize) % 16))
     return fail(ctx, BICACHE_ERR_INVALID, "bad layer stride");
-  if (need > cfg.num_pages) return fail(ctx, BICACHE_ERR_NOMEM, "prefix larger than the whole pool");
+  for (int l = first_layer; l < L; ++l)
+    if (need > ctx->layer_cap[l]) return fail(ctx, BICACHE_ERR_NOMEM, "prefix larger than a layer's pool");
   if (pages_out && pages_cap < need) return fail(ctx, BICACHE_ERR_INVALID, "pages_out too small");
-  while ((int)ctx->free_pages.size() < need) {
+  auto lacking = [&]() {
+    for (int l = first_layer; l < L; ++l)
+      if ((int)ctx->free_pages[l].size() < need) return true;
+    return false;
+  };
+  while (lacking()) {
     PrefixEntry& old = ctx->fifo.front();
-    for (int32_t p : old.pages) ctx->free_pages.push_back(p);
+    for (int l = old.first_layer; l < L; ++l)
+      for (int32_t pg : pages_of(old, l)) ctx->free_pages[l].push_back(pg);
     ctx->by_key.erase(old.key);
     ctx->by_id.erase(old.id);
     ctx->fifo.pop_front();
@@ -948,32 +1015,61 @@ int32_t put_impl(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const
   PrefixEntry e;
   e.key = key;
   e.m = m;
+  e.first_layer = first_layer;
   e.id = ctx->next_id++;
-  e.pages.resize(need);
-  for (int i = 0; i < need; ++i) {
-    e.pages[i] = ctx->free_pages.front();
-    ctx->free_pages.pop_front();
-  }
+  std::vector<std::vector<int32_t>> lists(L - first_layer, std::vector<int32_t>(need));
+  for (int l = first_layer; l < L; ++l)
+    for (int i = 0; i < need; ++i) {
+      lists[l - first_layer][i] = ctx->free_pages[l].front();
+      ctx->free_pages[l].pop_front();
+    }
+  e.uniform = true;
+  for (size_t j = 1; j < lists.size(); ++j) e.uniform = e.uniform && lists[j] == lists[0];
+  e.pages = lists[0];
+  if (!e.uniform) e.layer_pages = lists;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   cudaError_t ce = cudaSuccess;
-  if (write)
-    ce = cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
-  if (ce == cudaSuccess && write) {
+  if (write) {
     const int chunks_per_row = cfg.head_dim * ctx->esize / 16;
-    const long long total = (long long)cfg.num_layers * need * kPageSize * cfg.num_kv_heads * chunks_per_row;
     const int threads = 256;
-    const int blocks = (int)std::min<long long>((total + threads - 1) / threads, (long long)ctx->sm_count * 16);
     const PoolView pv = pool_view(ctx);
-    scatter_prefix_kernel<<<blocks, threads, 0, stream>>>(
-        static_cast<const char*>(k), static_cast<const char*>(v), static_cast<char*>(cfg.k_pool),
-        static_cast<char*>(cfg.v_pool), ctx->d_put_pages, need, m, cfg.num_layers, cfg.num_kv_heads,
-        chunks_per_row, layer_stride * ctx->esize, (long long)row_elems * ctx->esize, pv.layer_bytes,
-        pv.page_bytes, pv.swizzled);
-    ctx->launches++;
-    ce = cudaGetLastError();
+    if (e.uniform && ctx->uniform_caps) {
+      // one page list and one layer stride: all layers in one launch
+      ce = cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+      if (ce == cudaSuccess) {
+        const long long total = (long long)L * need * kPageSize * cfg.num_kv_heads * chunks_per_row;
+        const int blocks = (int)std::min<long long>((total + threads - 1) / threads, (long long)ctx->sm_count * 16);
+        scatter_prefix_kernel<<<blocks, threads, 0, stream>>>(
+            static_cast<const char*>(k), static_cast<const char*>(v), static_cast<char*>(cfg.k_pool),
+            static_cast<char*>(cfg.v_pool), ctx->d_put_pages, need, m, L, cfg.num_kv_heads, chunks_per_row,
+            layer_stride * ctx->esize, (long long)row_elems * ctx->esize, pv.layer_bytes, pv.page_bytes, pv.swizzled);
+        ctx->launches++;
+        ce = cudaGetLastError();
+      }
+    } else {
+      // the lists or the layers' places differ: one launch per layer (the staging of the list is reused in
+      // stream order)
+      const long long total = (long long)need * kPageSize * cfg.num_kv_heads * chunks_per_row;
+      const int blocks = (int)std::min<long long>((total + threads - 1) / threads, (long long)ctx->sm_count * 16);
+      for (int l = 0; l < L && ce == cudaSuccess; ++l) {
+        ce = cudaMemcpyAsync(ctx->d_put_pages, lists[l].data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+        if (ce != cudaSuccess) break;
+        scatter_prefix_kernel<<<blocks, threads, 0, stream>>>(
+            static_cast<const char*>(k) + (long long)l * layer_stride * ctx->esize,
+            static_cast<const char*>(v) + (long long)l * layer_stride * ctx->esize,
+            static_cast<char*>(cfg.k_pool) + ctx->layer_off[l], static_cast<char*>(cfg.v_pool) + ctx->layer_off[l],
+            ctx->d_put_pages, need, m, 1, cfg.num_kv_heads, chunks_per_row, 0, (long long)row_elems * ctx->esize,
+            pv.layer_bytes, pv.page_bytes, pv.swizzled);
+        ctx->launches++;
+        ce = cudaGetLastError();
+      }
+    }
   }
   if (ce != cudaSuccess) {
-    for (auto it = e.pages.rbegin(); it != e.pages.rend(); ++it) ctx->free_pages.push_front(*it);
+    for (int l = first_layer; l < L; ++l) {
+      const std::vector<int32_t>& pl = lists[l - first_layer];
+      for (auto it = pl.rbegin(); it != pl.rend(); ++it) ctx->free_pages[l].push_front(*it);
+    }
     ctx->next_id--;
     return fail(ctx, BICACHE_ERR_CUDA, std::string("put_prefix: ") + cudaGetErrorString(ce));
   }
@@ -993,12 +1089,18 @@ extern "C" {
 int32_t bicache_put_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, const void* k, const void* v,
                            int64_t layer_stride, void* stream, int32_t* prefix_id, int32_t* was_hit,
                            int32_t* pages_out, int32_t pages_cap) {
-  return put_impl(ctx, key, m, k, v, layer_stride, stream, prefix_id, was_hit, pages_out, pages_cap, true);
+  return put_impl(ctx, key, m, k, v, layer_stride, stream, prefix_id, was_hit, pages_out, pages_cap, true, 0);
 }
 
 int32_t bicache_reserve_prefix(bicache_ctx* ctx, uint64_t key, int32_t m, int32_t* prefix_id, int32_t* was_hit,
                                int32_t* pages_out, int32_t pages_cap) {
-  return put_impl(ctx, key, m, nullptr, nullptr, 0, nullptr, prefix_id, was_hit, pages_out, pages_cap, false);
+  return put_impl(ctx, key, m, nullptr, nullptr, 0, nullptr, prefix_id, was_hit, pages_out, pages_cap, false, 0);
+}
+
+int32_t bicache_reserve_prefix_layers(bicache_ctx* ctx, uint64_t key, int32_t m, int32_t first_layer,
+                                      int32_t* prefix_id, int32_t* was_hit, int32_t* pages_out, int32_t pages_cap) {
+  return put_impl(ctx, key, m, nullptr, nullptr, 0, nullptr, prefix_id, was_hit, pages_out, pages_cap, false,
+                  first_layer);
 }
 
 int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, const void* k,
@@ -1009,6 +1111,7 @@ int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t
   if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
   if (layer < 0 || layer >= cfg.num_layers) return fail(ctx, BICACHE_ERR_INVALID, "layer out of range");
   const PrefixEntry& e = *found->second;
+  if (layer < e.first_layer) return fail(ctx, BICACHE_ERR_INVALID, "the prefix owns no pages in this layer");
   const int64_t row_elems = (int64_t)cfg.num_kv_heads * cfg.head_dim;
   if (kv_row_stride < row_elems || (kv_row_stride * ctx->esize) % 16)
     return fail(ctx, BICACHE_ERR_INVALID, "bad row stride");
@@ -1017,7 +1120,7 @@ int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const int need = (int)e.pages.size();
   cudaError_t ce =
-      cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+      cudaMemcpyAsync(ctx->d_put_pages, pages_of(e, layer).data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
   if (ce == cudaSuccess) {
     const int chunks_per_row = cfg.head_dim * ctx->esize / 16;
     const long long total = (long long)need * kPageSize * cfg.num_kv_heads * chunks_per_row;
@@ -1026,8 +1129,8 @@ int32_t bicache_update_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t
     const PoolView pv = pool_view(ctx);
     scatter_prefix_kernel<<<blocks, threads, 0, stream>>>(
         static_cast<const char*>(k), static_cast<const char*>(v),
-        static_cast<char*>(cfg.k_pool) + (long long)layer * pv.layer_bytes,
-        static_cast<char*>(cfg.v_pool) + (long long)layer * pv.layer_bytes, ctx->d_put_pages, need, e.m, 1,
+        static_cast<char*>(cfg.k_pool) + ctx->layer_off[layer],
+        static_cast<char*>(cfg.v_pool) + ctx->layer_off[layer], ctx->d_put_pages, need, e.m, 1,
         cfg.num_kv_heads, chunks_per_row, 0, kv_row_stride * ctx->esize, pv.layer_bytes, pv.page_bytes, pv.swizzled);
     ctx->launches++;
     ce = cudaGetLastError();
@@ -1044,6 +1147,7 @@ int32_t bicache_read_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t l
   if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
   if (layer < 0 || layer >= cfg.num_layers) return fail(ctx, BICACHE_ERR_INVALID, "layer out of range");
   const PrefixEntry& e = *found->second;
+  if (layer < e.first_layer) return fail(ctx, BICACHE_ERR_INVALID, "the prefix owns no pages in this layer");
   const int64_t row_elems = (int64_t)cfg.num_kv_heads * cfg.head_dim;
   if (kv_row_stride < row_elems || (kv_row_stride * ctx->esize) % 16)
     return fail(ctx, BICACHE_ERR_INVALID, "bad row stride");
@@ -1053,7 +1157,7 @@ int32_t bicache_read_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t l
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   const int need = (int)e.pages.size();
   cudaError_t ce =
-      cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+      cudaMemcpyAsync(ctx->d_put_pages, pages_of(e, layer).data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
   if (ce == cudaSuccess && e.m > 0) {
     const int chunks_per_row = cfg.head_dim * ctx->esize / 16;
     const long long total = (long long)e.m * cfg.num_kv_heads * chunks_per_row;
@@ -1061,7 +1165,7 @@ int32_t bicache_read_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t l
     const int blocks = (int)std::min<long long>((total + threads - 1) / threads, (long long)ctx->sm_count * 16);
     const PoolView pv = pool_view(ctx);
     gather_prefix_kernel<<<blocks, threads, 0, stream>>>(
-        pv.k + (long long)layer * pv.layer_bytes, pv.v + (long long)layer * pv.layer_bytes,
+        pv.k + ctx->layer_off[layer], pv.v + ctx->layer_off[layer],
         static_cast<char*>(k_out), static_cast<char*>(v_out), ctx->d_put_pages, e.m, cfg.num_kv_heads,
         chunks_per_row, kv_row_stride * ctx->esize, pv.page_bytes, pv.swizzled);
     ctx->launches++;
@@ -1099,6 +1203,7 @@ int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_
   if (d_model <= 0 || d_model % 8 || h_row_stride < d_model || h_row_stride % 8)
     return fail(ctx, BICACHE_ERR_INVALID, "d_model and the row stride must be positive multiples of 8");
   const PrefixEntry& e = *found->second;
+  if (layer < e.first_layer) return fail(ctx, BICACHE_ERR_INVALID, "the prefix owns no pages in this layer");
   if (ctx->host_only) return BICACHE_OK;
   if (!h || !w_k || !w_v || !aligned16(h) || !aligned16(w_k) || !aligned16(w_v))
     return fail(ctx, BICACHE_ERR_INVALID, "bad h/w pointer");
@@ -1112,12 +1217,12 @@ int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_
       !encode_map_2d(&tm_wv, w_v, out_rows, d_model, d_model, 64))
     return fail(ctx, BICACHE_ERR_CUDA, "project_prefix_layer: tensor map encoding failed");
   cudaError_t ce =
-      cudaMemcpyAsync(ctx->d_put_pages, e.pages.data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
+      cudaMemcpyAsync(ctx->d_put_pages, pages_of(e, layer).data(), sizeof(int) * need, cudaMemcpyHostToDevice, stream);
   if (ce == cudaSuccess) {
     const PoolView pv = pool_view(ctx);
     proj::ProjArgs a;
-    a.pool_k = static_cast<char*>(cfg.k_pool) + (long long)layer * pv.layer_bytes;
-    a.pool_v = static_cast<char*>(cfg.v_pool) + (long long)layer * pv.layer_bytes;
+    a.pool_k = static_cast<char*>(cfg.k_pool) + ctx->layer_off[layer];
+    a.pool_v = static_cast<char*>(cfg.v_pool) + ctx->layer_off[layer];
     a.pages = ctx->d_put_pages;
     a.m = e.m;
     a.d_model = d_model;
@@ -1145,6 +1250,8 @@ int32_t bicache_prefix_similarity_async(bicache_ctx* ctx, int32_t prefix_id, con
   if (layer_stride < (int64_t)e.m * row_elems || (layer_stride * ctx->esize) % 16)
     return fail(ctx, BICACHE_ERR_INVALID, "bad layer stride");
   if (ctx->host_only) return fail(ctx, BICACHE_ERR_UNSUPPORTED, "host-only context");
+  if (e.first_layer != 0 || !e.uniform || !ctx->uniform_caps)
+    return fail(ctx, BICACHE_ERR_UNSUPPORTED, "the similarity needs a prefix with one page list for all layers");
   if (!k_ref || !v_ref || !aligned16(k_ref) || !aligned16(v_ref))
     return fail(ctx, BICACHE_ERR_INVALID, "bad k/v pointer");
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -1281,18 +1388,27 @@ int32_t bicache_lookup_prefix(const bicache_ctx* ctx, uint64_t key, int32_t* pre
   return BICACHE_OK;
 }
 
-int32_t bicache_prefix_pages(const bicache_ctx* ctx, int32_t prefix_id, int32_t* pages_out, int32_t cap,
-                             int32_t* n) {
+int32_t bicache_prefix_pages_layer(const bicache_ctx* ctx, int32_t prefix_id, int32_t layer, int32_t* pages_out,
+                                   int32_t cap, int32_t* n) {
   if (!ctx) return BICACHE_ERR_INVALID;
   auto found = ctx->by_id.find(prefix_id);
   if (found == ctx->by_id.end()) return fail(ctx, BICACHE_ERR_NOTFOUND, "unknown or evicted prefix id");
   const PrefixEntry& e = *found->second;
-  if (n) *n = (int32_t)e.pages.size();
+  if (layer < 0) layer = e.first_layer;
+  if (layer < e.first_layer || layer >= ctx->cfg.num_layers)
+    return fail(ctx, BICACHE_ERR_INVALID, "the prefix owns no pages in this layer");
+  const std::vector<int32_t>& pl = pages_of(e, layer);
+  if (n) *n = (int32_t)pl.size();
   if (pages_out) {
-    if (cap < (int32_t)e.pages.size()) return fail(ctx, BICACHE_ERR_INVALID, "pages_out too small");
-    std::copy(e.pages.begin(), e.pages.end(), pages_out);
+    if (cap < (int32_t)pl.size()) return fail(ctx, BICACHE_ERR_INVALID, "pages_out too small");
+    std::copy(pl.begin(), pl.end(), pages_out);
   }
   return BICACHE_OK;
+}
+
+int32_t bicache_prefix_pages(const bicache_ctx* ctx, int32_t prefix_id, int32_t* pages_out, int32_t cap,
+                             int32_t* n) {
+  return bicache_prefix_pages_layer(ctx, prefix_id, -1, pages_out, cap, n);
 }
 
 int32_t bicache_reuse_depth(const bicache_ctx* ctx, int32_t R, const int32_t* prefix_len,

@@ -270,3 +270,74 @@ def test_projection_and_read_back_argument_checks_on_host_context(lib):
     assert lib.bicache_reserve_prefix(f32, C.c_uint64(5), 40, C.byref(pid), C.byref(hit), pp, 4) == binding.OK
     assert proj(f32, pid.value, 0, None, 512, None, None, 512, None) == binding.ERR_UNSUPPORTED
     lib.bicache_destroy(f32)
+
+
+@given(st.lists(st.tuples(st.integers(0, 7), st.integers(1, 80), st.integers(0, 2)), min_size=1, max_size=40),
+       st.integers(2, 10), st.integers(0, 3), st.booleans())
+@settings(max_examples=120, deadline=None)
+def test_layered_store_traces_match_oracle_bit_exactly(trace, num_pages, seed, shrink_shallow):
+    """Prefixes that own only the layers from a first layer on (the kept deep-layer K/V of Eq. 5), with
+    per-layer free queues and, optionally, smaller pools in the shallow layers: ids, hit flags, error
+    codes and the page list of EVERY layer equal the oracle's after every call."""
+    entry.build()
+    lib = binding.load_library()
+    L = 3
+    order = list(range(num_pages)) if seed == 0 else np.random.default_rng(seed).permutation(num_pages).tolist()
+    caps = [max(1, num_pages // 2), max(1, (3 * num_pages) // 4), num_pages] if shrink_shallow else None
+    cfg = binding.Config(L, 2, 1, 128, 16, num_pages, binding.BF16, -1)
+    keep = np.ascontiguousarray(order, dtype=np.int32)
+    cfg.initial_free_order = keep.ctypes.data_as(C.POINTER(C.c_int32))
+    keep2 = None
+    if caps is not None:
+        keep2 = np.ascontiguousarray(caps, dtype=np.int32)
+        cfg.layer_pages = keep2.ctypes.data_as(C.POINTER(C.c_int32))
+    ctx = C.c_void_p()
+    assert lib.bicache_create(C.byref(cfg), C.byref(ctx)) == binding.OK
+    ref = oracle.PagedPrefixStore(L, 1, 128, 16, num_pages, free_order=order, layer_pages=caps)
+    i32p = C.POINTER(C.c_int32)
+    live = {}
+    for key, m, first in trace:
+        pid, hit = C.c_int32(-1), C.c_int32(-1)
+        cap = (m + 15) // 16
+        pages = np.full(cap, -1, dtype=np.int32)
+        st_ = lib.bicache_reserve_prefix_layers(ctx, C.c_uint64(key), m, first, C.byref(pid), C.byref(hit),
+                                                pages.ctypes.data_as(i32p), cap)
+        try:
+            opid, ohit, opages = ref.reserve(key, m, first)
+        except oracle.InvalidArgument:
+            assert st_ == binding.ERR_INVALID
+            continue
+        except oracle.OutOfPages:
+            assert st_ == binding.ERR_NOMEM
+            continue
+        assert st_ == binding.OK and (pid.value, bool(hit.value), pages.tolist()) == (opid, ohit, opages)
+        live[opid] = first
+        for p_id in list(live):
+            if p_id not in ref.entries:                     # evicted by this call
+                n = C.c_int32(0)
+                assert lib.bicache_prefix_pages(ctx, p_id, None, 0, C.byref(n)) == binding.ERR_NOTFOUND
+                del live[p_id]
+                continue
+            for l in range(L):
+                n = C.c_int32(0)
+                buf = np.full(16, -1, dtype=np.int32)
+                st2 = lib.bicache_prefix_pages_layer(ctx, p_id, l, buf.ctypes.data_as(i32p), 16, C.byref(n))
+                if l < live[p_id]:
+                    assert st2 == binding.ERR_INVALID
+                else:
+                    assert st2 == binding.OK and buf[:n.value].tolist() == ref.pages(p_id, l)
+    lib.bicache_destroy(ctx)
+
+
+def test_pool_bytes_with_layer_capacities(lib):
+    cfg = binding.Config(3, 2, 1, 128, 16, 8, binding.BF16, -1)
+    full = lib.bicache_pool_bytes(C.byref(cfg))
+    assert full == 3 * 8 * 1 * 16 * 128 * 2
+    caps = np.array([2, 5, 8], dtype=np.int32)
+    cfg.layer_pages = caps.ctypes.data_as(C.POINTER(C.c_int32))
+    assert lib.bicache_pool_bytes(C.byref(cfg)) == (2 + 5 + 8) * 16 * 128 * 2
+    bad = np.array([2, 9, 8], dtype=np.int32)
+    cfg.layer_pages = bad.ctypes.data_as(C.POINTER(C.c_int32))
+    assert lib.bicache_pool_bytes(C.byref(cfg)) == 0
+    ctx = C.c_void_p()
+    assert lib.bicache_create(C.byref(cfg), C.byref(ctx)) == binding.ERR_INVALID
