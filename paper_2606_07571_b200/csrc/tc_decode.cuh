@@ -445,8 +445,17 @@ merge_ranges_kernel(const float* __restrict__ part_o, const float* __restrict__ 
   const long long pr = kSlotWarps == 1 ? (long long)blockIdx.x * kMergeWarps + warp : (long long)blockIdx.x;   // token * Hq + head
   if (pr >= (long long)total_tokens * Hq) return;
   const int tg = (int)(pr / Hq), h = (int)(pr - (long long)tg * Hq);
-  const long long row = tok_rows[tg];
   const long long slot_stride = (long long)total_tokens * Hq;
+  // Up to 16 ranges (the common case): every range's row is requested before anything else, so that the
+  // row loads, the lse loads and the row-table load are one round trip instead of three.
+  const bool few = kSlotWarps == 1 && num_slots <= 16;
+  float4 pre[16];
+  if (few) {
+#pragma unroll
+    for (int u = 0; u < 16; ++u)
+      pre[u] = *reinterpret_cast<const float4*>(part_o + (pr + min(u, num_slots - 1) * slot_stride) * 128 + lane * 4);
+  }
+  const long long row = tok_rows[tg];
   const float l0 = lane < num_slots ? part_lse[pr + lane * slot_stride] : -INFINITY;
   const float l1 = lane + 32 < num_slots ? part_lse[pr + (lane + 32) * slot_stride] : -INFINITY;
   const float mx = warp_max(fmaxf(l0, l1));
@@ -459,7 +468,17 @@ merge_ranges_kernel(const float* __restrict__ part_o, const float* __restrict__ 
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   // this warp's ranges: first, first + kSlotWarps, ...; eight of them are loaded before any is used
   const int first = kSlotWarps == 1 ? 0 : warp;
-  for (int s0 = first; s0 < num_slots; s0 += 8 * kSlotWarps) {
+  if (few) {
+#pragma unroll
+    for (int u = 0; u < 16; ++u) {
+      const float w = u < num_slots ? __shfl_sync(0xffffffffu, w0, u) : 0.f;
+      acc.x = fmaf(w, pre[u].x, acc.x);
+      acc.y = fmaf(w, pre[u].y, acc.y);
+      acc.z = fmaf(w, pre[u].z, acc.z);
+      acc.w = fmaf(w, pre[u].w, acc.w);
+    }
+  }
+  for (int s0 = few ? num_slots : first; s0 < num_slots; s0 += 8 * kSlotWarps) {
     float4 v[8];
     float w[8];
 #pragma unroll
