@@ -436,8 +436,32 @@ def measure_calls_alone(job, name, flush, peaks):
             graph_ms = sorted(ts)[len(ts) // 2]
         except Exception:                              # capture not available: the figure is left out
             graph_ms = None
+    # Host time of one call: through the Python binding (marshalling of the metadata lists every call)
+    # and through the C ABI itself with the arguments marshalled once (what a C caller pays).  Enqueue
+    # only: 100 calls back to back, then one synchronisation.
+    import ctypes as C
+    from paper_2606_07571_b200 import binding as _b
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(100):
+        call_attend()
+    host_binding_us = (time.perf_counter() - t0) / 100 * 1e6
+    torch.cuda.synchronize()
+    pid_a, pid_p = _b._i32(req_pid)
+    off_a, off_p = _b._i64(w.suffix_row_off)
+    len_a, len_p = _b._i32(w.suffix_lens)
+    qp, kp, vp_, qs, ks, op, os_, lp = bc._tensor_args(job.q, job.k, job.v, job.out, None)
+    args = (bc.ctx, 0, len(len_a), pid_p, off_p, len_p, qp, kp, vp_, qs, ks, op, os_, lp, C.c_float(w.softmax_scale),
+            bc._stream())
+    t0 = time.perf_counter()
+    for _ in range(100):
+        bc.lib.bicache_attend(*args)
+    host_c_us = (time.perf_counter() - t0) / 100 * 1e6
+    torch.cuda.synchronize()
+    assert bc.device_status() == 0
     tr = traffic_of(name, "attend")
     attend = {"bound": "hbm", "kernel": "tc_decode_kernel (+ merge) (attend call alone)",
+              "host_us_per_call": {"python_binding": host_binding_us, "c_abi_premarshalled": host_c_us},
               "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
               "peak_source": peaks["source"], "bytes_per_launch": w.attend_bytes(), "ms_per_launch": ms_attend,
               "launches_timed": iters, "tflops": w.attend_flops() / (ms_attend * 1e-3) / 1e12,
