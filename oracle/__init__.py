@@ -36,6 +36,10 @@ Parity status of each function (what pins it, see tests/test_oracle_*.py):
   project_kv (Eq. 1)
                    pinned (scalar-loop brute force, selector weights that copy
                    chosen hidden components, linearity).
+  rope_rotate      pinned (zero angle, quarter turn, scalar loop, norm of every
+                   pair preserved, inner products depend on the position
+                   difference only).  The paper names no position encoding: the
+                   angles are an input.
 """
 from .bicache_oracle import (  # noqa: F401
     OracleError,
@@ -53,6 +57,7 @@ from .bicache_oracle import (  # noqa: F401
     xxh64,
     prefix_key,
     project_kv,
+    rope_rotate,
     merge,
     attend,
     attend_full,

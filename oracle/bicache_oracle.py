@@ -663,11 +663,40 @@ def prefix_key(tokens):
 # hidden state, k = W^K h, v = W^V h (W^K, W^V of shape [d_k, d] per layer).
 # ---------------------------------------------------------------------------
 
-def project_kv(h, wk, wv, num_kv_heads, head_dim):
+def rope_rotate(x, cos, sin):
+    """Rotary position encoding of keys (or queries) in the half-split pairing:
+    for token t and every head, the pair (x[d], x[d + D/2]), d < D/2, is rotated
+    by the angle whose cosine and sine are cos[t, d], sin[t, d]:
+
+        x'[d]       = x[d] cos - x[d + D/2] sin
+        x'[d + D/2] = x[d + D/2] cos + x[d] sin
+
+    x [m, H, D]; cos, sin [m, D/2] (the caller's table: the paper names no
+    position encoding, so angles are an input, not computed here).
+    """
+    x = np.asarray(x, dtype=np.float64)
+    cos = np.asarray(cos, dtype=np.float64)
+    sin = np.asarray(sin, dtype=np.float64)
+    m, _, D = x.shape
+    if D % 2 or cos.shape != (m, D // 2) or sin.shape != cos.shape:
+        raise InvalidArgument("bad rotary table shape")
+    half = D // 2
+    out = np.empty_like(x)
+    for t in range(m):
+        lo, hi = x[t, :, :half], x[t, :, half:]
+        out[t, :, :half] = lo * cos[t] - hi * sin[t]
+        out[t, :, half:] = hi * cos[t] + lo * sin[t]
+    return out
+
+
+def project_kv(h, wk, wv, num_kv_heads, head_dim, rope=None):
     """Prefix KVs from hidden states, every layer (Eq. 1).
 
     h [L, m, d]; wk, wv [L, Hkv * D, d] (row o of a weight produces output
     component o; components are ordered head-major: o = head * D + dim).
+    rope: None (Eq. 1 as printed) or (cos, sin), each [m, D/2]: the keys (not
+    the values) are then rotated per token with `rope_rotate` after the
+    projection, the form in which a rotary model caches them.
     Returns k, v of shape [L, m, Hkv, D], ready for `PagedPrefixStore.put`.
     """
     h = np.asarray(h, dtype=np.float64)
@@ -682,4 +711,6 @@ def project_kv(h, wk, wv, num_kv_heads, head_dim):
     for l in range(L):
         k[l] = (h[l] @ wk[l].T).reshape(m, num_kv_heads, head_dim)
         v[l] = (h[l] @ wv[l].T).reshape(m, num_kv_heads, head_dim)
+        if rope is not None:
+            k[l] = rope_rotate(k[l], rope[0], rope[1])
     return k, v

@@ -117,3 +117,45 @@ def test_similarity_distance_bound():
         a = np.concatenate([k[l].ravel(), v[l].ravel()])
         b = np.concatenate([kr[l].ravel(), vr[l].ravel()])
         assert abs((1 - sim[l]) - np.linalg.norm(a - b) ** 2 / (2 * np.linalg.norm(a) * np.linalg.norm(b))) < 1e-12
+
+
+def test_rope_rotate_pins():
+    """The rotary rotation of keys that the projection may apply (the angles are an input): identity at
+    angle 0, a quarter turn maps (a, b) to (-b, a), a scalar loop, norms of pairs, and the property the
+    encoding exists for: <rot(q, p), rot(k, p')> depends on p - p' only."""
+    rng = np.random.default_rng(8)
+    m, H, D = 6, 3, 8
+    x = rng.standard_normal((m, H, D))
+    zero = np.zeros((m, D // 2))
+    assert np.array_equal(oracle.rope_rotate(x, np.ones((m, D // 2)), zero), x)
+    quarter = oracle.rope_rotate(x, zero, np.ones((m, D // 2)))
+    assert np.allclose(quarter[..., :D // 2], -x[..., D // 2:]) and np.allclose(quarter[..., D // 2:], x[..., :D // 2])
+    ang = rng.uniform(-3, 3, (m, D // 2))
+    got = oracle.rope_rotate(x, np.cos(ang), np.sin(ang))
+    for t in range(m):
+        for h in range(H):
+            for d in range(D // 2):
+                a, b = x[t, h, d], x[t, h, d + D // 2]
+                assert abs(got[t, h, d] - (a * math.cos(ang[t, d]) - b * math.sin(ang[t, d]))) < 1e-12
+                assert abs(got[t, h, d + D // 2] - (b * math.cos(ang[t, d]) + a * math.sin(ang[t, d]))) < 1e-12
+                assert abs(math.hypot(got[t, h, d], got[t, h, d + D // 2]) - math.hypot(a, b)) < 1e-12
+    # relative positions: angles pos * theta_d
+    theta = 10000.0 ** (-np.arange(D // 2) / (D // 2))
+    q, k = rng.standard_normal((1, 1, D)), rng.standard_normal((1, 1, D))
+
+    def at(v, pos):
+        return oracle.rope_rotate(v, np.cos(pos * theta)[None], np.sin(pos * theta)[None])[0, 0]
+
+    base = at(q, 7.0) @ at(k, 3.0)
+    assert abs(at(q, 104.0) @ at(k, 100.0) - base) < 1e-9
+    assert abs(at(q, 4.0) @ k[0, 0] - base) < 1e-9
+    assert abs(at(q, 8.0) @ at(k, 3.0) - base) > 1e-3          # another difference, another value
+    with pytest.raises(oracle.InvalidArgument):
+        oracle.rope_rotate(x, zero[:, :-1], zero[:, :-1])
+    # project_kv applies it to the keys only
+    L, d = 1, 5
+    hdn = rng.standard_normal((L, m, d))
+    wk, wv = rng.standard_normal((L, H * D, d)), rng.standard_normal((L, H * D, d))
+    k0, v0 = oracle.project_kv(hdn, wk, wv, H, D)
+    k1, v1 = oracle.project_kv(hdn, wk, wv, H, D, rope=(np.cos(ang), np.sin(ang)))
+    assert np.array_equal(v0, v1) and np.allclose(k1[0], oracle.rope_rotate(k0[0], np.cos(ang), np.sin(ang)))
