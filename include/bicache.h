@@ -268,6 +268,18 @@ int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_
                                      int64_t h_row_stride, const void* w_k, const void* w_v, int32_t d_model,
                                      void* stream);
 
+/* The same with a rotary position encoding of the KEYS applied before they are stored (Eq. 1 has no
+ * position encoding and the paper names none; the attention calls take K as it is cached, so a model
+ * with rotary keys caches them rotated).  rope_cos_sin: device, fp32 [m][64][2]: for token t and pair d
+ * the cosine and the sine of the token's angle; the pair is head dims (d, d + 64) of every KV head
+ * (the half-split pairing):  k'[d] = k[d] cos - k[d + 64] sin,  k'[d + 64] = k[d + 64] cos + k[d] sin,
+ * in fp32 on the accumulator, before the one rounding to bf16.  The table is the caller's (base,
+ * scaling and position offset are the model's business); 16-byte aligned.  NULL: no rotation, the call
+ * above.  Values are not rotated.  Errors as above. */
+int32_t bicache_project_prefix_layer_rope(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, const void* h,
+                                          int64_t h_row_stride, const void* w_k, const void* w_v, int32_t d_model,
+                                          const float* rope_cos_sin, void* stream);
+
 /* One layer of denoising step t with both kinds of reuse.  Request i owns seqlen[i] = N_i rows from
  * row_off[i] (prefix rows first).  Per request, in this order:
  *   layer < depth[i] and shared_id[i] >= 0      -> suffix rows attend over [shared cached prefix | own

@@ -25,7 +25,7 @@ EXPORTED = [
     "bicache_prefix_pages", "bicache_prefix_pages_layer", "bicache_reserve_prefix_layers", "bicache_reuse_depth", "bicache_attend", "bicache_attend_full",
     "bicache_attend_layer", "bicache_attend_full_static",
     "bicache_is_refresh_step", "bicache_reserve_prefix", "bicache_update_prefix_layer", "bicache_attend_step",
-    "bicache_read_prefix_layer", "bicache_project_prefix_layer",
+    "bicache_read_prefix_layer", "bicache_project_prefix_layer", "bicache_project_prefix_layer_rope",
     "bicache_prefix_similarity", "bicache_prefix_similarity_async", "bicache_depth_from_similarity",
     "bicache_build_depth_table",
     "bicache_hash_tokens", "bicache_device_status", "bicache_set_wait_budget", "bicache_launch_count", "bicache_schedule_uploads", "bicache_last_attention_kernel", "bicache_last_error",
@@ -107,6 +107,8 @@ def load_library():
     lib.bicache_read_prefix_layer.argtypes = [vp, C.c_int32, C.c_int32, vp, vp, C.c_int64, vp]
     lib.bicache_project_prefix_layer.restype = C.c_int32
     lib.bicache_project_prefix_layer.argtypes = [vp, C.c_int32, C.c_int32, vp, C.c_int64, vp, vp, C.c_int32, vp]
+    lib.bicache_project_prefix_layer_rope.restype = C.c_int32
+    lib.bicache_project_prefix_layer_rope.argtypes = [vp, C.c_int32, C.c_int32, vp, C.c_int64, vp, vp, C.c_int32, vp, vp]
     lib.bicache_attend_step.restype = C.c_int32
     lib.bicache_attend_step.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, i32p, i32p, i32p, i64p, i32p,
                                         vp, vp, vp, C.c_int64, C.c_int64, vp, C.c_int64, vp, C.c_float, vp]
@@ -268,14 +270,22 @@ class BiCache:
                                                 k_out.stride(0), self._stream())
         self._check(st, "bicache_read_prefix_layer")
 
-    def project_prefix_layer(self, prefix_id, layer, h, w_k, w_v):
-        """Eq. 1 into the store: h [m, d_model] (rows may be strided), w_k, w_v [Hkv * D, d_model]."""
+    def project_prefix_layer(self, prefix_id, layer, h, w_k, w_v, rope=None):
+        """Eq. 1 into the store: h [m, d_model] (rows may be strided), w_k, w_v [Hkv * D, d_model].
+        rope: None, or a device fp32 tensor [m, 64, 2] of (cos, sin) per token and pair of head dims
+        (d, d + 64) by which the keys are rotated before they are stored."""
         assert h.is_cuda and w_k.is_cuda and w_v.is_cuda and h.dtype == w_k.dtype == w_v.dtype == self.dtype
         assert h.dim() == 2 and h.stride(1) == 1 and w_k.is_contiguous() and w_v.is_contiguous()
         assert w_k.shape == w_v.shape == (self.Hkv * self.D, h.shape[1])
-        st = self.lib.bicache_project_prefix_layer(self.ctx, prefix_id, layer, h.data_ptr(), h.stride(0),
-                                                   w_k.data_ptr(), w_v.data_ptr(), h.shape[1], self._stream())
-        self._check(st, "bicache_project_prefix_layer")
+        rp = None
+        if rope is not None:
+            assert rope.is_cuda and rope.dtype == torch.float32 and rope.is_contiguous()
+            assert tuple(rope.shape) == (h.shape[0], 64, 2)
+            rp = rope.data_ptr()
+        st = self.lib.bicache_project_prefix_layer_rope(self.ctx, prefix_id, layer, h.data_ptr(), h.stride(0),
+                                                        w_k.data_ptr(), w_v.data_ptr(), h.shape[1], rp,
+                                                        self._stream())
+        self._check(st, "bicache_project_prefix_layer_rope")
 
     def prefix_similarity(self, prefix_id, k_ref, v_ref):
         """Eq. 3 per layer: cosine between the cached K/V of a prefix and k_ref, v_ref [L, m, Hkv, D]."""

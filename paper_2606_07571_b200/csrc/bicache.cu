@@ -1193,7 +1193,16 @@ static bool encode_map_2d(CUtensorMap* m, const void* base, long long rows, long
 int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, const void* h,
                                      int64_t h_row_stride, const void* w_k, const void* w_v, int32_t d_model,
                                      void* stream_) {
+  return bicache_project_prefix_layer_rope(ctx, prefix_id, layer, h, h_row_stride, w_k, w_v, d_model, nullptr,
+                                           stream_);
+}
+
+int32_t bicache_project_prefix_layer_rope(bicache_ctx* ctx, int32_t prefix_id, int32_t layer, const void* h,
+                                          int64_t h_row_stride, const void* w_k, const void* w_v, int32_t d_model,
+                                          const float* rope_cos_sin, void* stream_) {
   if (!ctx) return BICACHE_ERR_INVALID;
+  if (rope_cos_sin && (reinterpret_cast<uintptr_t>(rope_cos_sin) & 15))
+    return fail(ctx, BICACHE_ERR_INVALID, "the rotary table must be 16-byte aligned");
   const bicache_config& cfg = ctx->cfg;
   if (!ctx->tensor_ok && !(ctx->host_only && cfg.dtype == BICACHE_BF16 && cfg.head_dim == 128))
     return fail(ctx, BICACHE_ERR_UNSUPPORTED, "projection needs a bf16 context with head_dim 128");
@@ -1224,6 +1233,7 @@ int32_t bicache_project_prefix_layer(bicache_ctx* ctx, int32_t prefix_id, int32_
     a.pool_k = static_cast<char*>(cfg.k_pool) + ctx->layer_off[layer];
     a.pool_v = static_cast<char*>(cfg.v_pool) + ctx->layer_off[layer];
     a.pages = ctx->d_put_pages;
+    a.rope = reinterpret_cast<const float2*>(rope_cos_sin);
     a.m = e.m;
     a.d_model = d_model;
     a.num_kv_heads = cfg.num_kv_heads;

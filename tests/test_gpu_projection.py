@@ -61,7 +61,7 @@ def test_read_back_is_bit_exact(dtype, Hkv, D, m):
     assert ei.value.status == binding.ERR_INVALID
 
 
-def _check_projection(Hkv, m, d_model, L=2, strided=False, seed=1):
+def _check_projection(Hkv, m, d_model, L=2, strided=False, seed=1, rope=False):
     D = 128
     npages = (m + 15) // 16
     bc = binding.BiCache(L, Hkv, Hkv, D, 2 * npages + 1, torch.bfloat16, 16, 1)
@@ -73,6 +73,12 @@ def _check_projection(Hkv, m, d_model, L=2, strided=False, seed=1):
     nid, _, _ = bc.put_prefix(5, nk, nv)
     pid, hit, pages = bc.reserve_prefix(6, m)
     assert not hit and len(pages) == npages
+    # rotary table of the keys (an input of the call): position t, pair d -> angle (t + 3) * 10000^(-d / 64)
+    table = dev_table = None
+    if rope:
+        ang = (np.arange(m, dtype=np.float64)[:, None] + 3.0) * 10000.0 ** (-np.arange(64, dtype=np.float64) / 64.0)
+        table = np.stack([np.cos(ang), np.sin(ang)], axis=-1).astype(np.float32)          # [m, 64, 2]
+        dev_table = torch.from_numpy(table).cuda()
     hs, wks, wvs = [], [], []
     for l in range(L):
         h, w_k, w_v = workloads.draw_hidden_and_weights(m, d_model, Hkv, D, seed * 100 + l, device="cuda")
@@ -80,10 +86,12 @@ def _check_projection(Hkv, m, d_model, L=2, strided=False, seed=1):
             wide = torch.zeros(m, d_model + 64, dtype=torch.bfloat16, device="cuda")
             wide[:, :d_model] = h
             h = wide[:, :d_model]
-        bc.project_prefix_layer(pid, l, h, w_k, w_v)
+        bc.project_prefix_layer(pid, l, h, w_k, w_v, rope=dev_table)
         hs.append(workloads.to_f64(h)); wks.append(workloads.to_f64(w_k)); wvs.append(workloads.to_f64(w_v))
     assert bc.device_status() == 0
-    rk, rv = oracle.project_kv(np.stack(hs), np.stack(wks), np.stack(wvs), Hkv, D)
+    rk, rv = oracle.project_kv(np.stack(hs), np.stack(wks), np.stack(wvs), Hkv, D,
+                               rope=None if table is None else (table[..., 0].astype(np.float64),
+                                                                table[..., 1].astype(np.float64)))
     for l in range(L):
         gk, gv = _read(bc, pid, l, m)
         for got, ref, name in ((gk, rk[l], "K"), (gv, rv[l], "V")):
@@ -105,6 +113,17 @@ def test_projection_small_ragged():
 
 def test_projection_several_token_blocks_strided_rows():
     _check_projection(Hkv=4, m=300, d_model=512, strided=True)
+
+
+def test_projection_with_rotary_keys():
+    """Keys rotated per token in the epilogue (pairs of head dims d, d + 64; the caller's table of
+    cosines and sines), values left alone: a ragged single block, and several blocks with whole and
+    split tiles."""
+    _check_projection(Hkv=3, m=77, d_model=200, rope=True)
+    _check_projection(Hkv=4, m=700, d_model=512, strided=True, rope=True)
+    # and the rotation really happened: against the unrotated oracle the keys differ
+    bc, pid = _check_projection(Hkv=2, m=40, d_model=128, L=1, rope=True)
+    bc.close()
 
 
 def test_projection_more_tiles_than_sms():
