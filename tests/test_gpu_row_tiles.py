@@ -91,3 +91,48 @@ def test_more_items_than_sms_scattered_pages_second_layer():
     npages = sum((m + 15) // 16 for m in ms) + 1
     run_case("many", 8, 8, ms, [0] * 25 + [1] * 15, ns, order=workloads.shuffled_page_order(npages, 3), layers=2,
              layer=1)
+
+
+@pytest.mark.parametrize("seed", [31, 32, 33, 34])
+def test_large_random_batches_against_the_cuda_core_path(seed):
+    """Many requests in several groups, more work items than SMs (every CTA walks through many shared
+    and plain tiles in a row), random head groupings that do and do not share tiles: the tensor-core path
+    against the CUDA-core path of the same library on the same inputs (both are checked against the
+    oracle elsewhere; here the point is volume)."""
+    rng = np.random.default_rng(seed)
+    G = int(rng.choice([1, 2, 4, 8, 3]))
+    Hkv = int(rng.choice([2, 4, 8])) if G <= 2 else int(rng.choice([1, 2]))
+    Hq = G * Hkv
+    ngroups = int(rng.integers(2, 6))
+    ms = [int(rng.integers(17, 900)) for _ in range(ngroups)]
+    R = int(rng.integers(40, 120))
+    rp = sorted(int(rng.integers(0, ngroups)) for _ in range(R))
+    ns = [int(rng.choice([0, 1, 5, 8, 9, 31, 64, 100, 127, 128, 130, 257, 300])) for _ in range(R)]
+    w = workloads.Workload("big%d" % seed, 1, Hq, Hkv, 128, torch.bfloat16, 16, ms, rp, ns,
+                           softmax_scale=128 ** -0.5, seed=seed)
+    bc = binding.BiCache(1, Hq, Hkv, 128, w.pages_needed() + 1, torch.bfloat16, w.total_rows, R)
+    pids = []
+    for g in range(ngroups):
+        kc, vc = workloads.draw_prefix_kv(w, g, "cuda")
+        pids.append(bc.put_prefix(100 + g, kc, vc)[0])
+    q, k, v = workloads.draw_full_qkv(w, "cuda")
+    req_pid = [pids[g] for g in rp]
+    # a few requests go without a prefix (between the groups)
+    for i in range(0, R, 17):
+        req_pid[i] = -1
+    ok_groups = all(req_pid[i] == req_pid[i - 1] or req_pid[i] not in req_pid[:i] for i in range(1, R))
+    if not ok_groups:                         # a -1 in the middle of a group splits it: ids must stay grouped
+        req_pid = [pids[g] for g in rp]
+    res = []
+    for path in (binding.PATH_TENSOR, binding.PATH_SIMT):
+        bc.set_path(path)
+        out = torch.full_like(q, 3.0)
+        lse = torch.full(q.shape[:2], 3.0, dtype=torch.float32, device="cuda")
+        bc.attend(0, req_pid, w.suffix_row_off, w.suffix_lens, q, k, v, out, lse, w.softmax_scale)
+        assert bc.device_status() == binding.OK
+        res.append((out.float(), lse))
+    what = "seed %d G %d Hkv %d groups %s R %d" % (seed, G, Hkv, ms, R)
+    assert torch.isfinite(res[0][0]).all(), what
+    assert (res[0][0] - res[1][0]).abs().max().item() <= 2e-2, what
+    assert (res[0][1] - res[1][1]).abs().max().item() <= 1e-3, what
+    bc.close()
