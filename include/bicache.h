@@ -63,8 +63,13 @@ enum { BICACHE_F32 = 0, BICACHE_BF16 = 1 };
 
 /* Which kernels serve bf16 head_dim-128 attention.  AUTO picks the tensor-core
  * path when it applies; SIMT forces the plain CUDA-core kernels (used as an
- * on-device cross-check).  fp32 and other head dims always run SIMT. */
-enum { BICACHE_PATH_AUTO = 0, BICACHE_PATH_SIMT = 1, BICACHE_PATH_TENSOR = 2 };
+ * on-device cross-check).  fp32 and other head dims always run SIMT.
+ * TENSOR_PAIRS is TENSOR with bicache_attend_full on the variant of the tensor-core
+ * kernel that runs on pairs of SMs (one MMA over 256 query rows, each SM staging half
+ * of every K/V tile) whenever Hq / Hkv divides 32; it gives the same bits as the
+ * default kernel and is slower, so AUTO never picks it (it exists as a measured
+ * alternative and a cross-check). */
+enum { BICACHE_PATH_AUTO = 0, BICACHE_PATH_SIMT = 1, BICACHE_PATH_TENSOR = 2, BICACHE_PATH_TENSOR_PAIRS = 3 };
 
 typedef struct {
   int32_t num_layers;        /* L >= 1                                                         */
@@ -399,8 +404,9 @@ int64_t bicache_schedule_uploads(const bicache_ctx* ctx);
  * (bicache_attend only; chosen when every request has a cached prefix of at least 1024 tokens and at
  * most 128 * Hkv / Hq suffix tokens, and the call is small enough for the kernel's tables): the group's
  * rows share tiles, the prefix keys are split into ranges over the CTAs, each request's own keys are
- * one more range, and a merge kernel applies the log-sum-exp merge (exact up to rounding). */
-enum { BICACHE_KERNEL_SIMT = 1, BICACHE_KERNEL_TENSOR = 2, BICACHE_KERNEL_KEY_RANGES = 3 };
+ * one more range, and a merge kernel applies the log-sum-exp merge (exact up to rounding);
+ * BICACHE_KERNEL_TENSOR_PAIRS the tensor-core kernel on pairs of SMs (BICACHE_PATH_TENSOR_PAIRS). */
+enum { BICACHE_KERNEL_SIMT = 1, BICACHE_KERNEL_TENSOR = 2, BICACHE_KERNEL_KEY_RANGES = 3, BICACHE_KERNEL_TENSOR_PAIRS = 4 };
 int32_t bicache_last_attention_kernel(const bicache_ctx* ctx);
 
 /* Human-readable text for the last error of this context (host string, valid until next call). */

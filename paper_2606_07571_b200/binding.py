@@ -13,8 +13,8 @@ import torch
 
 OK, ERR_INVALID, ERR_NOMEM, ERR_NOTFOUND, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED = range(7)
 F32, BF16 = 0, 1
-PATH_AUTO, PATH_SIMT, PATH_TENSOR = 0, 1, 2
-KERNEL_SIMT, KERNEL_TENSOR, KERNEL_KEY_RANGES = 1, 2, 3
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_TENSOR_PAIRS = 0, 1, 2, 3
+KERNEL_SIMT, KERNEL_TENSOR, KERNEL_KEY_RANGES, KERNEL_TENSOR_PAIRS = 1, 2, 3, 4
 _STATUS_NAMES = ["OK", "INVALID", "NOMEM", "NOTFOUND", "CUDA", "TIMEOUT", "UNSUPPORTED"]
 
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libbicache.so")

@@ -22,6 +22,7 @@
 #include "simt_kernels.cuh"
 #include "tc_attention.cuh"
 #include "project_kv.cuh"
+#include "tc_attention_pair.cuh"
 #include "tc_decode.cuh"
 
 using namespace bicache;
@@ -84,6 +85,7 @@ struct bicache_ctx {
   bool swizzled = false;
   bool tensor_ok = false;
   int last_kernel = 0;                                            // which attention kernel the last call launched
+  int attn_pairs = 0;                                             // CTA pairs of the attention kernel on pairs the device runs at once
   int proj_pairs = 0;                                             // CTA pairs of the projection kernel the device runs at once
   bool host_only = false;                                         // cfg.device < 0: bookkeeping only
   int path = BICACHE_PATH_AUTO;
@@ -279,7 +281,8 @@ size_t arena_place(bicache_ctx* ctx, size_t bytes) {
 
 // Build (or find) the device-resident schedule for this batch.  Returns its index in ctx->sched or -1.
 // `tiled`: kind 0 on the tensor path - the query rows of a prefix group are packed into row tiles.
-int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int layer, int R, const int32_t* prefix_id,
+// `pairs`: kind 1 for the kernel on CTA pairs - items of 512 packed rows, the keys never split.
+int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, bool pairs, int layer, int R, const int32_t* prefix_id,
                      const int64_t* row_off, const int32_t* seqlen, cudaStream_t stream, int* status) {
   *status = BICACHE_OK;
   // A schedule holds the page lists of its prefixes.  They are the same in every layer unless some
@@ -289,7 +292,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int layer, int R, c
     for (int i = 0; i < R; ++i)
       if (prefix_id[i] >= 0 && (i == 0 || prefix_id[i] != prefix_id[i - 1]) && !ctx->by_id.at(prefix_id[i])->uniform)
         layer_tag = layer + 1;
-  const int key_kind = kind + (tiled ? 8 : 0) + 16 * layer_tag;
+  const int key_kind = kind + (tiled ? 8 : 0) + (pairs ? 16 : 0) + 32 * layer_tag;
   uint64_t hash = fnv1a(0xcbf29ce484222325ull, &key_kind, sizeof(key_kind));
   hash = fnv1a(hash, &R, sizeof(R));
   hash = fnv1a(hash, row_off, sizeof(int64_t) * R);
@@ -339,7 +342,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int layer, int R, c
   // splits minimises a simple cost model: waves of CTAs (one CTA per SM) times the time of one CTA
   // (a fixed prologue/epilogue plus a per-key-tile cost), plus the merge pass over the partials.
   int num_splits = 1, tiles_per_split = 0;
-  if (kind != 2 && unsplit_items > 0 && unsplit_items < 2LL * ctx->sm_count && max_key_tiles >= 8) {
+  if (kind != 2 && !pairs && unsplit_items > 0 && unsplit_items < 2LL * ctx->sm_count && max_key_tiles >= 8) {
     const int key_tiles = max_key_tiles;
     const double c_tile = 3300.0, c_cta = 12000.0;         // SM clocks, fitted on the small-suffix shapes
     auto cost = [&](int nsplit, int tps) {
@@ -490,6 +493,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int layer, int R, c
     });
   } else {
     tiled = false;
+    const int item_rows = pairs ? 2 * kTileRows : kTileRows;
     items.reserve((size_t)unsplit_items * num_splits);
     for (int sp = 0; sp < (kind == 2 ? 1 : num_splits); ++sp) {
       const size_t first = items.size();
@@ -497,7 +501,7 @@ int prepare_schedule(bicache_ctx* ctx, int kind, bool tiled, int layer, int R, c
         if (reqs[i].n <= 0) continue;
         const int prow = reqs[i].n * G;
         for (int hk = 0; hk < Hkv; ++hk)
-          for (int r0 = 0; r0 < prow; r0 += kTileRows) items.push_back(WorkItem{i, hk, r0, sp});
+          for (int r0 = 0; r0 < prow; r0 += item_rows) items.push_back(WorkItem{i, hk, r0, sp});
       }
       // Longest key range first (the tail of the launch is then made of short items); items of one
       // KV head and request stay adjacent so that concurrently running CTAs share K/V tiles in L2.
@@ -619,7 +623,9 @@ struct PreparedCall {
   bool empty = true;           // nothing to launch
   int entry = -1;              // index in ctx->sched
   bool key_ranges = false, use_tensor = false;
+  bool pairs = false;          // the tensor-core kernel on CTA pairs
   TcTensorMaps maps;
+  CUtensorMap k64;             // pairs: k with a box of 64 rows
 };
 
 // Everything the host can check, then the schedule (found in the cache or built and uploaded) and the
@@ -691,18 +697,23 @@ int prepare_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, cons
     }
     if (total > kMaxDecodeTokens) key_ranges = false;
   }
+  // The kernel on CTA pairs serves full attention only when asked for (it is the slower of the two on
+  // every shape measured: the hand-over between the two SMs lengthens the per-tile chain by more than
+  // the halved shared-memory traffic shortens it), and only when a 32-row output box holds whole tokens.
+  pc->pairs = kind == 1 && pc->use_tensor && ctx->path == BICACHE_PATH_TENSOR_PAIRS && ctx->attn_pairs > 0 &&
+              32 % (cfg.num_q_heads / cfg.num_kv_heads) == 0;
   int st = BICACHE_OK;
   int entry = -1;
   if (key_ranges) {
-    entry = prepare_schedule(ctx, 2, false, layer, R, prefix_id, row_off, seqlen, stream, &st);
+    entry = prepare_schedule(ctx, 2, false, false, layer, R, prefix_id, row_off, seqlen, stream, &st);
     if (entry < 0) {                                     // does not fit: the general path
       key_ranges = false;
       ctx->last_error.clear();
     }
   }
   if (entry < 0)
-    entry = prepare_schedule(ctx, kind, kind == 0 && pc->use_tensor && kTiledAttend, layer, R, prefix_id, row_off,
-                             seqlen, stream, &st);
+    entry = prepare_schedule(ctx, kind, kind == 0 && pc->use_tensor && kTiledAttend, pc->pairs, layer, R, prefix_id,
+                             row_off, seqlen, stream, &st);
   if (entry < 0) return st;
   pc->entry = entry;
   pc->key_ranges = key_ranges;
@@ -723,6 +734,7 @@ int prepare_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, cons
     maps.o_tma = (32 % G == 0) ? 1 : 0;
     okm = okm && encode_map(&maps.o, out, rows_total, cfg.num_q_heads, out_row_stride, maps.o_tma ? G : 1,
                             maps.o_tma ? 32 / G : 32);
+    if (pc->pairs) okm = okm && encode_map(&pc->k64, k, rows_total, cfg.num_kv_heads, kv_row_stride, 1, 64);
     if (!okm) return fail(ctx, BICACHE_ERR_CUDA, "tensor map encoding failed");
   }
   pc->empty = false;
@@ -768,12 +780,18 @@ int launch_attention(bicache_ctx* ctx, const PreparedCall& pc, int32_t layer, co
   const PoolView pool = pool_view_layer(ctx, layer);
 
   cudaError_t e;
-  ctx->last_kernel = pc.key_ranges ? BICACHE_KERNEL_KEY_RANGES : pc.use_tensor ? BICACHE_KERNEL_TENSOR : BICACHE_KERNEL_SIMT;
+  ctx->last_kernel = pc.key_ranges ? BICACHE_KERNEL_KEY_RANGES
+                     : pc.pairs    ? BICACHE_KERNEL_TENSOR_PAIRS
+                     : pc.use_tensor ? BICACHE_KERNEL_TENSOR
+                                     : BICACHE_KERNEL_SIMT;
   if (pc.key_ranges) {
     e = launch_tc_decode(reinterpret_cast<const dec::DecodeItem*>(base + c.ditems_off), c.num_ditems,
                          reinterpret_cast<const long long*>(base + c.tok_rows_off),
                          reinterpret_cast<const int2*>(base + c.tok_span_off), sv.pages, pool, t, ctx->d_status,
                          ctx->wait_cycles, stream);
+  } else if (pc.pairs) {
+    e = launch_tc_attention_pair(sv, t, ctx->d_status, ctx->attn_pairs, pc.maps.q, pc.k64, pc.maps.v, pc.maps.o,
+                                 ctx->wait_cycles, stream);
   } else if (pc.use_tensor) {
     e = launch_tc_attention(sv, pool, t, ctx->d_status, ctx->sm_count, pc.maps, ctx->wait_cycles, stream);
   } else if (cfg.dtype == BICACHE_F32) {
@@ -926,6 +944,7 @@ int32_t bicache_create(const bicache_config* cfg, bicache_ctx** out) {
   if (tensor_ok) {
     cudaError_t e = configure_tc_attention();
     if (e == cudaSuccess) e = configure_project_kv(&ctx->proj_pairs);
+    if (e == cudaSuccess) e = configure_tc_attention_pair(&ctx->attn_pairs);
     if (e == cudaSuccess) e = configure_tc_decode();
     if (e != cudaSuccess) {
       destroy_host_resources(ctx);
@@ -951,8 +970,8 @@ int32_t bicache_destroy(bicache_ctx* ctx) {
 }
 
 int32_t bicache_set_path(bicache_ctx* ctx, int32_t path) {
-  if (!ctx || path < BICACHE_PATH_AUTO || path > BICACHE_PATH_TENSOR) return BICACHE_ERR_INVALID;
-  if (path == BICACHE_PATH_TENSOR && !ctx->tensor_ok)
+  if (!ctx || path < BICACHE_PATH_AUTO || path > BICACHE_PATH_TENSOR_PAIRS) return BICACHE_ERR_INVALID;
+  if ((path == BICACHE_PATH_TENSOR || path == BICACHE_PATH_TENSOR_PAIRS) && !ctx->tensor_ok)
     return fail(ctx, BICACHE_ERR_UNSUPPORTED, "tensor-core path needs bf16 and head_dim 128");
   ctx->path = path;
   return BICACHE_OK;
