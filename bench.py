@@ -403,10 +403,21 @@ def measure_calls_alone(job, name, flush, peaks):
     ms_full = time_call(call_full, iters, flush)
     full = tensor_roofline("tc_attention_kernel (attend_full call alone)", w.full_flops(), ms_full, peaks, False,
                            iters, traffic_of(name, "full"))
+    # The same call on the variant of the kernel that runs on pairs of SMs (an opt-in path: the measured
+    # alternative, not what the steps use).
+    from paper_2606_07571_b200 import binding as _bind
+    pairs = None
+    if w.dtype == torch.bfloat16 and w.head_dim == 128 and 32 % (w.num_q_heads // w.num_kv_heads) == 0:
+        bc.set_path(_bind.PATH_TENSOR_PAIRS)
+        call_full()
+        if bc.last_attention_kernel() == _bind.KERNEL_TENSOR_PAIRS:
+            pairs = tensor_roofline("tc_attention_pair_kernel (attend_full call alone, opt-in path)", w.full_flops(),
+                                    time_call(call_full, iters, flush), peaks, False, iters, (None, None))
+        bc.set_path(_bind.PATH_AUTO)
     if kernel != 3:                                    # not the key-range kernel
         attend = tensor_roofline("tc_attention_kernel (attend call alone)", w.attend_flops(), ms_attend, peaks, False,
                                  iters, traffic_of(name, "attend"))
-        return {"attend_full": full, "attend": attend}
+        return {"attend_full": full, "attend": attend, "attend_full_cta_pairs": pairs}
     # few query rows against a long cached prefix: the call is bound by reading the prefix once
     gbs = w.attend_bytes() / (ms_attend * 1e-3) / 1e9
     # The same call replayed from a CUDA graph (ten calls per replay): what a serving loop that
@@ -470,7 +481,7 @@ def measure_calls_alone(job, name, flush, peaks):
                                 "achieved": w.attend_bytes() / (graph_ms * 1e-3) / 1e9,
                                 "frac": w.attend_bytes() / (graph_ms * 1e-3) / 1e9 / peaks["hbm_gbs"]}),
               "traffic": tr[0], "traffic_source": tr[1]}
-    return {"attend_full": full, "attend": attend}
+    return {"attend_full": full, "attend": attend, "attend_full_cta_pairs": pairs}
 
 
 def pinned_like(t, chunk_bytes=1 << 30):
