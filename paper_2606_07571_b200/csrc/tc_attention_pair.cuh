@@ -81,6 +81,11 @@ __device__ __forceinline__ unsigned map_to_rank(unsigned local, unsigned rank) {
 __device__ __forceinline__ void mbar_arrive_cluster(unsigned cluster_bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
+// The same without cluster-scope release (which costs a memory barrier on the arriving warp): for
+// hand-overs whose data lives in tensor memory and is ordered by the tcgen05 fences, not by this arrival.
+__device__ __forceinline__ void mbar_arrive_cluster_plain(unsigned cluster_bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
 __device__ __forceinline__ void st_cluster_u32(unsigned cluster_addr, unsigned v) {
   asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(v) : "memory");
 }
@@ -280,7 +285,7 @@ tc_attention_pair_kernel(ScheduleView s, TensorArgs t, int* status, const __grid
       __syncwarp();
       if (lane == 0) {
         if (rank == 0) mbar_arrive(local_bar);
-        else mbar_arrive_cluster(cluster_bar);
+        else mbar_arrive_cluster_plain(cluster_bar);
       }
     };
     const unsigned loc_p0 = smem_u32(&bars->p_half[X][0]), loc_p1 = smem_u32(&bars->p_half[X][1]);
