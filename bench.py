@@ -787,6 +787,9 @@ def main():
                     help="algorithmic FLOPs of the sample one step of --impl reference runs")
     ap.add_argument("--delta", type=int, default=0,
                     help="refresh interval of the deep layers' kept prefix K/V (Eq. 5); 0: recompute every step")
+    ap.add_argument("--attend-full-path", choices=("default", "pairs"), default="default",
+                    help="pairs: the timed steps run full attention on the CTA-pair variant of the tensor-core "
+                         "kernel (an opt-in path of the library; slower, see the design notes)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     args.steps = max(args.steps, 1)
@@ -813,9 +816,13 @@ def main():
             entry.build()
     peaks = load_peaks()
     job = Job(w, local_rank, args.delta)
+    if args.attend_full_path == "pairs":
+        job.bc.set_path(job.binding.PATH_TENSOR_PAIRS)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")       # 2x the 126 MB L2
 
     rec = measure_steps(job, args.workload, args.steps, args.warmup, flush, peaks, rank, local_rank, world, dist)
+    if args.attend_full_path == "pairs":
+        rec["config"]["attend_full_path"] = "cta pairs (opt-in)"
     alone = measure_calls_alone(job, args.workload, flush, peaks)
     # where no layer has every request on one path, the launch timed alone stands in
     if rec["roofline"] is None:
