@@ -80,7 +80,7 @@ struct alignas(8) Barriers {
   unsigned long long full[kRing];        // ring slot holds its tile
   unsigned long long free_[kRing];       // the MMAs reading the slot have completed
   unsigned long long s_full[2];          // S = Q K^T of the current key tile is in TMEM (per query tile)
-  unsigned long long p_half[2][2];       // P of keys 0-63 / 64-127 is in TMEM and O is rescaled (per query tile)
+  unsigned long long p_half[2][2];       // P of keys 0-95 / 96-127 is in TMEM and O is rescaled (per query tile)
   unsigned long long o_done[2];          // the last O += P V of the item has completed (per query tile)
   unsigned long long o_free[2];          // the epilogue has read O out of TMEM (per query tile)
   unsigned long long drain;
@@ -255,26 +255,8 @@ __device__ __forceinline__ void mma_ss_batch8(unsigned el, unsigned d_tmem, cons
         "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "l"(b[6]), "l"(b[7]), "r"(idesc), "r"(el)
       : "memory");
 }
-// O (+)= P V: four K steps of 16 keys, P read from TMEM at p + 8 k; the first accumulates iff acc0.
-__device__ __forceinline__ void mma_ts_batch4(unsigned el, unsigned o_tmem, unsigned p_tmem,
-                                              const unsigned long long (&b)[4], unsigned idesc, unsigned acc0) {
-  asm volatile(
-      "{\n\t.reg .pred P, T, Q;\n\t.reg .b32 p1, p2, p3;\n\t"
-      "setp.ne.b32 P, %8, 0;\n\t"
-      "setp.eq.u32 T, 0, 0;\n\t"
-      "setp.ne.b32 Q, %7, 0;\n\t"
-      "add.u32 p1, %1, 8;\n\t"
-      "add.u32 p2, %1, 16;\n\t"
-      "add.u32 p3, %1, 24;\n\t"
-      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %6, Q;\n\t"
-      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p1], %3, %6, T;\n\t"
-      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p2], %4, %6, T;\n\t"
-      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p3], %5, %6, T;\n\t}"
-      ::"r"(o_tmem), "r"(p_tmem), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "r"(idesc), "r"(acc0), "r"(el)
-      : "memory");
-}
-// The same for a ragged key tile: up to four K steps of 16 keys, P read from TMEM at p + 8 k; the first accumulates iff
-// acc0; only the first n_on steps are issued (a ragged key tile has fewer than eight steps).
+// O (+)= P V, up to four K steps of 16 keys (the key-range kernel's 64-key tiles): P read from TMEM at p + 8 k; the
+// first accumulates iff acc0; only the first n_on steps are issued.
 __device__ __forceinline__ void mma_ts_batch4_first(unsigned el, unsigned o_tmem, unsigned p_tmem,
                                                     const unsigned long long (&b)[4], unsigned idesc, unsigned acc0,
                                                     int n_on) {
@@ -299,6 +281,94 @@ __device__ __forceinline__ void mma_ts_batch4_first(unsigned el, unsigned o_tmem
       "@E2 tcgen05.mma.cta_group::1.kind::f16 [%0], [p2], %4, %6, T;\n\t"
       "@E3 tcgen05.mma.cta_group::1.kind::f16 [%0], [p3], %5, %6, T;\n\t}"
       ::"r"(o_tmem), "r"(p_tmem), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "r"(idesc), "r"(acc0), "r"(el), "r"(n_on)
+      : "memory");
+}
+// The split of O += P V that the kernel uses: P is handed over as keys 0-95 and keys 96-127, so that only
+// two K steps follow the last exponentials of a tile.  Six K steps; step k is issued iff k < n_on.
+__device__ __forceinline__ void mma_ts_batch6(unsigned el, unsigned o_tmem, unsigned p_tmem,
+                                              const unsigned long long (&b)[6], unsigned idesc, unsigned acc0, int n_on) {
+  asm volatile(
+      "{\n\t.reg .pred P, T, Q, E0, E1, E2, E3, E4, E5;\n\t.reg .b32 p1, p2, p3, p4, p5;\n\t"
+      "setp.ne.b32 P, %10, 0;\n\t"
+      "setp.eq.u32 T, 0, 0;\n\t"
+      "setp.ne.b32 Q, %9, 0;\n\t"
+      "setp.gt.s32 E0, %11, 0;\n\t"
+      "setp.gt.s32 E1, %11, 1;\n\t"
+      "setp.gt.s32 E2, %11, 2;\n\t"
+      "setp.gt.s32 E3, %11, 3;\n\t"
+      "setp.gt.s32 E4, %11, 4;\n\t"
+      "setp.gt.s32 E5, %11, 5;\n\t"
+      "and.pred E0, E0, P;\n\t"
+      "and.pred E1, E1, P;\n\t"
+      "and.pred E2, E2, P;\n\t"
+      "and.pred E3, E3, P;\n\t"
+      "and.pred E4, E4, P;\n\t"
+      "and.pred E5, E5, P;\n\t"
+      "add.u32 p1, %1, 8;\n\t"
+      "add.u32 p2, %1, 16;\n\t"
+      "add.u32 p3, %1, 24;\n\t"
+      "add.u32 p4, %1, 32;\n\t"
+      "add.u32 p5, %1, 40;\n\t"
+      "@E0 tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %8, Q;\n\t"
+      "@E1 tcgen05.mma.cta_group::1.kind::f16 [%0], [p1], %3, %8, T;\n\t"
+      "@E2 tcgen05.mma.cta_group::1.kind::f16 [%0], [p2], %4, %8, T;\n\t"
+      "@E3 tcgen05.mma.cta_group::1.kind::f16 [%0], [p3], %5, %8, T;\n\t"
+      "@E4 tcgen05.mma.cta_group::1.kind::f16 [%0], [p4], %6, %8, T;\n\t"
+      "@E5 tcgen05.mma.cta_group::1.kind::f16 [%0], [p5], %7, %8, T;\n\t}"
+      ::"r"(o_tmem), "r"(p_tmem), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "r"(idesc),
+        "r"(acc0), "r"(el), "r"(n_on)
+      : "memory");
+}
+// the same for a full key tile: no per-step predicates
+__device__ __forceinline__ void mma_ts_batch6_full(unsigned el, unsigned o_tmem, unsigned p_tmem,
+                                                   const unsigned long long (&b)[6], unsigned idesc, unsigned acc0) {
+  asm volatile(
+      "{\n\t.reg .pred P, T, Q;\n\t.reg .b32 p1, p2, p3, p4, p5;\n\t"
+      "setp.ne.b32 P, %10, 0;\n\t"
+      "setp.eq.u32 T, 0, 0;\n\t"
+      "setp.ne.b32 Q, %9, 0;\n\t"
+      "add.u32 p1, %1, 8;\n\t"
+      "add.u32 p2, %1, 16;\n\t"
+      "add.u32 p3, %1, 24;\n\t"
+      "add.u32 p4, %1, 32;\n\t"
+      "add.u32 p5, %1, 40;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %8, Q;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p1], %3, %8, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p2], %4, %8, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p3], %5, %8, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p4], %6, %8, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p5], %7, %8, T;\n\t}"
+      ::"r"(o_tmem), "r"(p_tmem), "l"(b[0]), "l"(b[1]), "l"(b[2]), "l"(b[3]), "l"(b[4]), "l"(b[5]), "r"(idesc),
+        "r"(acc0), "r"(el)
+      : "memory");
+}
+__device__ __forceinline__ void mma_ts_batch2_full(unsigned el, unsigned o_tmem, unsigned p_tmem,
+                                                   const unsigned long long (&b)[2], unsigned idesc) {
+  asm volatile(
+      "{\n\t.reg .pred P, T;\n\t.reg .b32 p1;\n\t"
+      "setp.ne.b32 P, %5, 0;\n\t"
+      "setp.eq.u32 T, 0, 0;\n\t"
+      "add.u32 p1, %1, 8;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %4, T;\n\t"
+      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [p1], %3, %4, T;\n\t}"
+      ::"r"(o_tmem), "r"(p_tmem), "l"(b[0]), "l"(b[1]), "r"(idesc), "r"(el)
+      : "memory");
+}
+// The last two K steps (keys 96-111, 112-127), always accumulating; step k is issued iff k < n_on.
+__device__ __forceinline__ void mma_ts_batch2(unsigned el, unsigned o_tmem, unsigned p_tmem,
+                                              const unsigned long long (&b)[2], unsigned idesc, int n_on) {
+  asm volatile(
+      "{\n\t.reg .pred P, T, E0, E1;\n\t.reg .b32 p1;\n\t"
+      "setp.ne.b32 P, %5, 0;\n\t"
+      "setp.eq.u32 T, 0, 0;\n\t"
+      "setp.gt.s32 E0, %6, 0;\n\t"
+      "setp.gt.s32 E1, %6, 1;\n\t"
+      "and.pred E0, E0, P;\n\t"
+      "and.pred E1, E1, P;\n\t"
+      "add.u32 p1, %1, 8;\n\t"
+      "@E0 tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %4, T;\n\t"
+      "@E1 tcgen05.mma.cta_group::1.kind::f16 [%0], [p1], %3, %4, T;\n\t}"
+      ::"r"(o_tmem), "r"(p_tmem), "l"(b[0]), "l"(b[1]), "r"(idesc), "r"(el), "r"(n_on)
       : "memory");
 }
 // tcgen05.commit by the same elected lane (a commit covers the MMAs its own thread issued)
@@ -331,6 +401,14 @@ __device__ __forceinline__ void tmem_st32(unsigned taddr, const unsigned* r) {
         "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
         "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
         "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(unsigned taddr, const unsigned* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+        "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
       : "memory");
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -680,13 +758,15 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
         {
           // The exponentials use the reference maximum of
           // the earlier tiles and do not wait for this tile's maximum, which is computed alongside.
-          // P of the first 64 keys is handed to the tensor pipe before the second half is computed.
+          // P of the first 96 keys is handed to the tensor pipe before the last 32 exponentials are computed
+          // (a 64 / 64 split left four K steps of P V behind the last exponential, 2 % slower; 112 / 16 is
+          // slower again: the first part then starts too late).
           // If the row maximum turns out to exceed the reference by more than 2^8 (rare: checked per
           // warp before anything is handed over), the tile is redone below with the new reference.
           const float neg_m_eff = mine ? -m_ref : -INFINITY;
           const unsigned long long neg_m2 = pack2(neg_m_eff, neg_m_eff);
           float mx0 = -INFINITY, mx1 = -INFINITY;
-          // first half of the exponentials, with the maximum over all 128 scores computed alongside
+          // the first 64 exponentials, with the maximum over all 128 scores computed alongside
           // (independent instructions that fill the exp unit's latency)
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
@@ -717,13 +797,30 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
           const float mx = mine ? fmaxf(mx0, mx1) * sl2 : -INFINITY;   // scale > 0
 
           if (!__any_sync(0xffffffffu, mx > m_ref + 8.f)) {
+            // keys 64-95 join the first hand-over, so that only two K steps of P V follow the last exponentials
+#pragma unroll
+            for (int i = 16; i < 24; ++i) {
+              const unsigned long long xa =
+                  fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
+              const unsigned long long xb =
+                  fma2(pack2(__uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3])), sl2_2, neg_m2);
+              float xa0, xa1, xb0, xb1;
+              unpack2(xa, xa0, xa1);
+              unpack2(xb, xb0, xb1);
+              const float p0 = ex2(xa0), p1 = ex2(xa1), p2 = ex2(xb0), p3 = ex2(xb1);
+              acc_a = add2(acc_a, pack2(p0, p1));
+              acc_b = add2(acc_b, pack2(p2, p3));
+              r[2 * i] = pack_bf16(p0, p1);
+              r[2 * i + 1] = pack_bf16(p2, p3);
+            }
             tmem_st32(tmem_s, r);
+            tmem_st16(tmem_s + 32, r + 32);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(smem_u32(&bars->p_half[X][0]));
 
 #pragma unroll
-            for (int i = 16; i < 32; ++i) {
+            for (int i = 24; i < 32; ++i) {
               const unsigned long long xa =
                   fma2(pack2(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1])), sl2_2, neg_m2);
               const unsigned long long xb =
@@ -744,7 +841,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               r[2 * i] = pack_bf16(p0, p1);
               r[2 * i + 1] = pack_bf16(p2, p3);
             }
-            tmem_st32(tmem_s + 32, r + 32);
+            tmem_st16(tmem_s + 48, r + 48);
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(smem_u32(&bars->p_half[X][1]));
@@ -1178,13 +1275,13 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
     // The whole warp runs this control flow converged and one elected lane issues each batch of
     // tcgen05 instructions.  Issue order inside an item:
     //   S_A(0) S_B(0) | O_A(0) S_A(1) | O_B(0) S_B(1) | O_A(1) S_A(2) | ...
-    // O_X(j) += P_X V is issued in two halves as P arrives, and the next S_X = Q_X K^T follows it
+    // O_X(j) += P_X V is issued in two parts as P arrives (six K steps, then two), and the next S_X = Q_X K^T follows it
     // back to back (it overwrites P_X; the tensor pipe runs MMAs in issue order).  After the last
     // O_X of an item the next S_X is the first one of the next item.  Alternating between the two
     // tiles keeps their softmaxes half a period apart, which the exp unit they share needs.
     // This warp shares its scheduler with two busy softmax warps and gets through its own
     // instructions slowly, so everything but the MMAs - waits for K/V tiles, descriptors, what
-    // follows each O - sits in the shadow of the waits for the second half of P.
+    // follows each O - sits in the shadow of the waits for the second part of P.
     bool ok = !dead;
     if (ok) {
       const unsigned bar_full = smem_u32(&bars->full[0]), bar_free = smem_u32(&bars->free_[0]);   // slot i: + 8 i
@@ -1216,14 +1313,22 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
         }
         mma_ss_batch8(el, d_tmem, a, b, kIdescQK);
       };
-      // four of the eight MMAs (K steps of 16 keys) of O_X += P_X V
+      // one part of the eight MMAs (K steps of 16 keys) of O_X += P_X V: half 0 = keys 0-95, half 1 = keys 96-127
       auto issue_pv = [&](unsigned o_tmem, unsigned p_tmem, unsigned long long vd, unsigned v_step, int half,
                           unsigned acc0, int ksteps) {
-        unsigned long long b[4];
+        if (half == 0) {
+          unsigned long long b[6];
 #pragma unroll
-        for (int k = 0; k < 4; ++k) b[k] = vd + (half * 4 + k) * v_step;
-        if (ksteps == 8) mma_ts_batch4(el, o_tmem, p_tmem + half * 32, b, kIdescPV, half ? 1u : acc0);
-        else mma_ts_batch4_first(el, o_tmem, p_tmem + half * 32, b, kIdescPV, half ? 1u : acc0, ksteps - half * 4);
+          for (int k = 0; k < 6; ++k) b[k] = vd + k * v_step;
+          if (ksteps == 8) mma_ts_batch6_full(el, o_tmem, p_tmem, b, kIdescPV, acc0);
+          else mma_ts_batch6(el, o_tmem, p_tmem, b, kIdescPV, acc0, ksteps);
+        } else {
+          unsigned long long b[2];
+#pragma unroll
+          for (int k = 0; k < 2; ++k) b[k] = vd + (6 + k) * v_step;
+          if (ksteps == 8) mma_ts_batch2_full(el, o_tmem, p_tmem + 48, b, kIdescPV);
+          else mma_ts_batch2(el, o_tmem, p_tmem + 48, b, kIdescPV, ksteps - 6);
+        }
       };
       int n_it = 0;
       int c0 = 0, c1 = 0;        // key tiles each query tile has been through (phase of p_half)
@@ -1263,8 +1368,8 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             mma_commit_pred(el, bar_s);
             if (T == 1) mma_commit_pred(el, bar_qfree);
             if (b_on) {
-              // Stagger the two query tiles by half a period: tile B starts when tile A's softmax is
-              // half done (started together, the two softmaxes share the exp unit and the MMAs of
+              // Stagger the two query tiles: tile B starts when tile A's softmax has handed over its
+              // first part of P (started together, the two softmaxes share the exp unit and the MMAs of
               // both tiles then queue behind each other).
               ok = BICACHE_WAIT(bar_p, c0 & 1) && BICACHE_WAIT(bar_qfull + 8, e1 & 1);
               if (!ok) break;
@@ -1285,12 +1390,12 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             const unsigned long long v_desc = (dn ? vb_dense : vb_img) + sv * kSlotUnits;
             const unsigned v_step = dn ? 128u : 256u;           // 16 keys further, in 16-byte units
             const unsigned acc0 = j > 0 ? 1u : 0u;
-            // ---- tile A: first half of O += P V as soon as P of keys 0-63 is there ----
+            // ---- tile A: first part of O += P V as soon as P of keys 0-95 is there ----
             ok = BICACHE_WAIT(bar_p, c0 & 1);
             if (!ok) return;
             tc_fence_after();
                         issue_pv(tmem_o0, tmem_u, v_desc, v_step, 0, acc0, ksteps);
-            // ---- shadow of A's second half of the exponentials: what follows the O of this iteration ----
+            // ---- shadow of A's last exponentials: what follows the O of this iteration ----
             bool s_on0 = true, s_on1 = b_on;                   // an S follows O_A / O_B
             bool q_last = j + 2 == T;                           // ... and it is the last S of its item
             bool dn_next = false;
@@ -1321,7 +1426,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
             }
             const unsigned long long k_desc = (dn_next ? kb_dense : kb_img) + sn * kSlotUnits;
             const unsigned k_hi = dn_next ? 1024u : 64u;
-            // ---- tile A: second half, then the next S_A back to back ----
+            // ---- tile A: second part, then the next S_A back to back ----
             ok = BICACHE_WAIT(bar_p + 8, c0 & 1);
             if (!ok) return;
             tc_fence_after();
@@ -1340,7 +1445,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               mma_commit_pred(el, bar_s);
               if (q_last) mma_commit_pred(el, bar_qfree);
             }
-            // ---- tile B: first half ----
+            // ---- tile B: first part ----
             if (b_on) {
               if (j == 0) {
                 ok = BICACHE_WAIT(bar_ofree + 8, (e1 & 1) ^ 1);  // the previous epilogue has read O_B
@@ -1351,7 +1456,7 @@ tc_attention_kernel(ScheduleView s, PoolView pool, TensorArgs t, int* status,
               tc_fence_after();
                             issue_pv(tmem_o1, tmem_s1, v_desc, v_step, 0, acc0, ksteps);
             }
-            // ---- tile B: second half, then the next S_B ----
+            // ---- tile B: second part, then the next S_B ----
             if (b_on) {
               ok = BICACHE_WAIT(bar_p + 24, c1 & 1);
               if (!ok) return;
