@@ -396,6 +396,8 @@ def measure_calls_alone(job, name, flush, peaks):
         bc.attend_full(0, w.full_row_off, w.full_lens, job.q, job.k, job.v, job.out, None, w.softmax_scale)
 
     iters = 10 if w.full_flops() < 5e13 else 3
+    from paper_2606_07571_b200 import binding as _bind
+    bc.set_path(_bind.PATH_AUTO)                       # whatever path the timed steps ran on
     call_attend()
     kernel = bc.last_attention_kernel()
     call_full()
@@ -405,9 +407,8 @@ def measure_calls_alone(job, name, flush, peaks):
                            iters, traffic_of(name, "full"))
     # The same call on the variant of the kernel that runs on pairs of SMs (an opt-in path: the measured
     # alternative, not what the steps use).
-    from paper_2606_07571_b200 import binding as _bind
     pairs = None
-    if w.dtype == torch.bfloat16 and w.head_dim == 128 and 32 % (w.num_q_heads // w.num_kv_heads) == 0:
+    if w.dtype == torch.bfloat16 and w.head_dim == 128:
         bc.set_path(_bind.PATH_TENSOR_PAIRS)
         call_full()
         if bc.last_attention_kernel() == _bind.KERNEL_TENSOR_PAIRS:

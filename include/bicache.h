@@ -66,9 +66,8 @@ enum { BICACHE_F32 = 0, BICACHE_BF16 = 1 };
  * on-device cross-check).  fp32 and other head dims always run SIMT.
  * TENSOR_PAIRS is TENSOR with bicache_attend_full on the variant of the tensor-core
  * kernel that runs on pairs of SMs (one MMA over 256 query rows, each SM staging half
- * of every K/V tile) whenever Hq / Hkv divides 32; it gives the same bits as the
- * default kernel and is slower, so AUTO never picks it (it exists as a measured
- * alternative and a cross-check). */
+ * of every K/V tile); it gives the same bits as the default kernel and is slower, so
+ * AUTO never picks it (it exists as a measured alternative and a cross-check). */
 enum { BICACHE_PATH_AUTO = 0, BICACHE_PATH_SIMT = 1, BICACHE_PATH_TENSOR = 2, BICACHE_PATH_TENSOR_PAIRS = 3 };
 
 typedef struct {

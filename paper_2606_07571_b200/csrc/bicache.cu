@@ -699,9 +699,8 @@ int prepare_attention(bicache_ctx* ctx, int kind, int32_t layer, int32_t R, cons
   }
   // The kernel on CTA pairs serves full attention only when asked for (it is the slower of the two on
   // every shape measured: the hand-over between the two SMs lengthens the per-tile chain by more than
-  // the halved shared-memory traffic shortens it), and only when a 32-row output box holds whole tokens.
-  pc->pairs = kind == 1 && pc->use_tensor && ctx->path == BICACHE_PATH_TENSOR_PAIRS && ctx->attn_pairs > 0 &&
-              32 % (cfg.num_q_heads / cfg.num_kv_heads) == 0;
+  // the halved shared-memory traffic shortens it).
+  pc->pairs = kind == 1 && pc->use_tensor && ctx->path == BICACHE_PATH_TENSOR_PAIRS && ctx->attn_pairs > 0;
   int st = BICACHE_OK;
   int entry = -1;
   if (key_ranges) {
@@ -791,7 +790,7 @@ int launch_attention(bicache_ctx* ctx, const PreparedCall& pc, int32_t layer, co
                          ctx->wait_cycles, stream);
   } else if (pc.pairs) {
     e = launch_tc_attention_pair(sv, t, ctx->d_status, ctx->attn_pairs, pc.maps.q, pc.k64, pc.maps.v, pc.maps.o,
-                                 ctx->wait_cycles, stream);
+                                 pc.maps.q_tma, pc.maps.o_tma, ctx->wait_cycles, stream);
   } else if (pc.use_tensor) {
     e = launch_tc_attention(sv, pool, t, ctx->d_status, ctx->sm_count, pc.maps, ctx->wait_cycles, stream);
   } else if (cfg.dtype == BICACHE_F32) {

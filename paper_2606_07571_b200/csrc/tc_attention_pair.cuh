@@ -205,7 +205,7 @@ __device__ __forceinline__ void mma2_commit_local_pred(unsigned el, unsigned bar
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(tc::kThreads, 1)
 tc_attention_pair_kernel(ScheduleView s, TensorArgs t, int* status, const __grid_constant__ CUtensorMap tm_q,
                          const __grid_constant__ CUtensorMap tm_k64, const __grid_constant__ CUtensorMap tm_v,
-                         const __grid_constant__ CUtensorMap tm_o, long long wait_cycles) {
+                         const __grid_constant__ CUtensorMap tm_o, int q_tma, int o_tma, long long wait_cycles) {
   using namespace tcp;
   namespace cg = cooperative_groups;
   extern __shared__ unsigned char smem_raw[];
@@ -458,7 +458,7 @@ tc_attention_pair_kernel(ScheduleView s, TensorArgs t, int* status, const __grid
           const float lse = (m_ref + log2f(l_sum)) * 0.6931471805599453f;
           const int seg_first = __shfl_sync(0xffffffffu, vseg, 0), seg_last = __shfl_sync(0xffffffffu, vseg, 31);
           const int prow_first = __shfl_sync(0xffffffffu, prow, 0);
-          const bool by_tma = seg_first >= 0 && seg_last >= 0 && prow_first % G == 0;
+          const bool by_tma = o_tma && seg_first >= 0 && seg_last >= 0 && prow_first % G == 0;
           const int tok_first = (int)row_off + prow_first / G;
           const long long my_dst = row_valid ? ((row_off + a) * t.out_stride + (long long)h * 128) * 2 : -1;
 #pragma unroll
@@ -557,15 +557,47 @@ tc_attention_pair_kernel(ScheduleView s, TensorArgs t, int* status, const __grid
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars->q_free[x]), (eq[x] & 1) ^ 1, abort_flag));
         if (!ok) break;
         ++eq[x];
-        if (lane == 0) {
-          const unsigned qf = smem_u32(&bars->q_full[x]);
-          const unsigned q_dst = q_smem + x * kTileBytes;
-          const SegInfo* s0 = &inf->seg[0];
-          const int tok = (int)s0->row_off + (s0->prow0 + x * 128) / G;
-          if (rank == 0) mbar_arrive_expect_tx(qf, 2u * kTileBytes);      // the Q tiles of both CTAs
-          tma_load_3d_pair(q_dst, &tm_q, 0, inf->kv_head * G, tok, qf);
-          tma_load_3d_pair(q_dst + kTileBytes / 2, &tm_q, 64, inf->kv_head * G, tok, qf);
-          if (rank != 0) mbar_arrive_remote(qf, 0);
+        const unsigned qf = smem_u32(&bars->q_full[x]);
+        const unsigned q_dst = q_smem + x * kTileBytes;
+        const SegInfo* s0 = &inf->seg[0];
+        if (q_tma) {
+          if (lane == 0) {
+            const int tok = (int)s0->row_off + (s0->prow0 + x * 128) / G;
+            if (rank == 0) mbar_arrive_expect_tx(qf, 2u * kTileBytes);      // the Q tiles of both CTAs
+            tma_load_3d_pair(q_dst, &tm_q, 0, inf->kv_head * G, tok, qf);
+            tma_load_3d_pair(q_dst + kTileBytes / 2, &tm_q, 64, inf->kv_head * G, tok, qf);
+            if (rank != 0) mbar_arrive_remote(qf, 0);
+          }
+        } else {
+          // gathers into the page-image layout (the heads of a KV group do not divide 128): packed row
+          // p = token a * G + head jj of the group; rows past the end are zero-filled
+          const int packed_rows = s0->n * G;
+          const int r0 = lane >> 4, c16 = lane & 15;
+          int prow = s0->prow0 + x * 128 + r0;
+          const int a0 = prow / G;
+          int jj = prow - a0 * G;
+          const long long q_row_bytes = t.q_stride * 2;
+          const char* q_base = t.q + (s0->row_off * t.q_stride + (long long)inf->kv_head * G * 128) * 2 + c16 * 16;
+          const char* src_row = q_base + a0 * q_row_bytes;
+#pragma unroll 4
+          for (int i = 0; i < 64; ++i) {
+            const bool valid = prow < packed_rows;
+            cp_async16(q_dst + tile_chunk_offset(r0 + 2 * i, c16), valid ? src_row + jj * 256 : q_base, valid ? 16u : 0u);
+            prow += 2;
+            jj += 2;
+            while (jj >= G) {
+              jj -= G;
+              src_row += q_row_bytes;
+            }
+          }
+          cp_async_commit();
+          cp_async_wait<0>();
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) {
+            if (rank == 0) mbar_arrive(qf);
+            else mbar_arrive_remote(qf, 0);
+          }
         }
         __syncwarp();
       }
@@ -715,7 +747,8 @@ tc_attention_pair_kernel(ScheduleView s, TensorArgs t, int* status, const __grid
       // image of a gathered ragged tile (8-row groups 2048 bytes apart, the 64-dim halves 1024 bytes) or
       // the dense layout TMA writes (8-row groups 1024 bytes apart, halves 8 KB).  V half, 128 keys x 64
       // dims, one layout: rows of 128 bytes, 8-key groups 1024 bytes apart.  Q as in the one-CTA kernel.
-      const unsigned long long q_desc0 = make_desc(q_smem, 16, 1024);
+      const unsigned q_hi = q_tma ? 1024u : 64u;
+      const unsigned long long q_desc0 = make_desc(q_smem, 16, q_tma ? 1024u : 2048u);
       const unsigned long long q_desc1 = q_desc0 + (kTileBytes >> 4);
       const unsigned long long kb_img = make_desc(ring_smem, 16, 2048), kb_dense = make_desc(ring_smem, 16, 1024);
       const unsigned long long vb = make_desc(ring_smem, 1024, 1024);
@@ -728,7 +761,7 @@ tc_attention_pair_kernel(ScheduleView s, TensorArgs t, int* status, const __grid
         unsigned long long a[8], b[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-          a[k] = qd + (k >> 2) * 1024u + (k & 3) * 2;
+          a[k] = qd + (k >> 2) * q_hi + (k & 3) * 2;
           b[k] = kd + (k >> 2) * k_hi + (k & 3) * 2;
         }
         mma2_ss_batch8(el, d_tmem, a, b, kIdescQK2);
@@ -928,14 +961,15 @@ inline cudaError_t configure_tc_attention_pair(int* max_pairs) {
   return n > 0 ? cudaSuccess : cudaErrorLaunchOutOfResources;
 }
 
-// Tensor maps of a launch on CTA pairs: q and o as in TcTensorMaps (G must divide 32); k64: [rows][Hkv][128]
+// Tensor maps of a launch on CTA pairs: q and o (and their flags) as in TcTensorMaps; k64: [rows][Hkv][128]
 // with a box of (64 dims, 1 head, 64 rows); v: the box of (64 dims, 1 head, 128 rows) of TcTensorMaps.
 inline cudaError_t launch_tc_attention_pair(const ScheduleView& s, const TensorArgs& t, int* status, int max_pairs,
                                             const CUtensorMap& tm_q, const CUtensorMap& tm_k64, const CUtensorMap& tm_v,
-                                            const CUtensorMap& tm_o, long long wait_cycles, cudaStream_t stream) {
+                                            const CUtensorMap& tm_o, int q_tma, int o_tma, long long wait_cycles,
+                                            cudaStream_t stream) {
   const int pairs = s.num_items < max_pairs ? s.num_items : max_pairs;
   tc_attention_pair_kernel<<<2 * pairs, tc::kThreads, tcp::kPairSmemBytes, stream>>>(
-      s, t, status, tm_q, tm_k64, tm_v, tm_o, wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
+      s, t, status, tm_q, tm_k64, tm_v, tm_o, q_tma, o_tma, wait_cycles > 0 ? wait_cycles : tc::kWaitCycles);
   return cudaGetLastError();
 }
 

@@ -1,6 +1,6 @@
 """The tensor-core kernel on pairs of SMs (`PATH_TENSOR_PAIRS`, full attention only) through the C ABI:
 against the oracle, against the default one-CTA kernel (same arithmetic in the same order: equal bits),
-the head groupings it leaves to the default kernel, and its give-up path."""
+head groupings that take the gather and copy-out paths, and its give-up path."""
 import numpy as np
 import pytest
 import torch
@@ -48,6 +48,8 @@ CASES = [
     (8, 2, [130, 64, 259, 1, 700]),            # four query heads per KV head
     (8, 1, [33, 200, 65]),                     # eight
     (32, 1, [17, 40]),                         # thirty-two: a token is a whole 32-row output box
+    (14, 2, [300, 40, 513]),                   # seven: Q by gathers, output rows copied out by the warps
+    (3, 1, [129, 700]),                        # three: gathers and copy-out as well
     (32, 32, [1100] * 6),                      # 96 items of 512 rows on 74 pairs
     (16, 16, [896, 600, 777] * 4),             # 192 items, no key splits in the default kernel: equal bits
 ]
@@ -92,16 +94,8 @@ def test_pairs_kernel_rescales_when_the_row_maximum_jumps():
     bc.close()
 
 
-def test_pairs_path_leaves_other_head_groupings_and_attend_to_the_default_kernel():
+def test_pairs_path_leaves_attend_to_the_default_kernel():
     D = 128
-    # seven query heads per KV head: a 32-row output box would cut a token
-    q, k, v, off = _inputs([300, 40], 14, 2, seed=3)
-    bc = binding.BiCache(1, 14, 2, D, 4, torch.bfloat16, 340, 2)
-    out_p, _, kern = _run(bc, binding.PATH_TENSOR_PAIRS, off, [300, 40], q, k, v, D ** -0.5)
-    assert kern == binding.KERNEL_TENSOR
-    out_s, _, _ = _run(bc, binding.PATH_TENSOR, off, [300, 40], q, k, v, D ** -0.5)
-    assert torch.equal(out_p, out_s)
-    bc.close()
     # attention over a cached prefix stays on the default kernels
     w = workloads.Workload("pairs_attend", 1, 4, 4, 128, torch.bfloat16, 16, [200], [0, 0], [300, 70],
                            softmax_scale=D ** -0.5, seed=77)
