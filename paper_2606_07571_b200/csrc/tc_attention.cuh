@@ -200,30 +200,7 @@ __device__ __forceinline__ void tmem_relinquish() {
 __device__ __forceinline__ void tmem_dealloc(unsigned taddr, unsigned cols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-// An MMA issued by one elected lane of a converged warp, without a branch: the election and the
-// accumulate flag are predicates inside one asm block.  `enable` = 0 skips the MMA.
-__device__ __forceinline__ void mma_ss_elect(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
-                                             unsigned idesc, unsigned accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred P, Q;\n\t"
-      "elect.sync _|P, 0xffffffff;\n\t"
-      "setp.ne.b32 Q, %4, 0;\n\t"
-      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, Q;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void mma_ts_elect(unsigned d_tmem, unsigned a_tmem, unsigned long long b_desc,
-                                             unsigned idesc, unsigned accumulate, unsigned enable) {
-  asm volatile(
-      "{\n\t.reg .pred P, Q, E;\n\t"
-      "elect.sync _|P, 0xffffffff;\n\t"
-      "setp.ne.b32 Q, %4, 0;\n\t"
-      "setp.ne.b32 E, %5, 0;\n\t"
-      "and.pred P, P, E;\n\t"
-      "@P tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, Q;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(enable)
-      : "memory");
-}
+// tcgen05.commit issued by one elected lane of a converged warp, without a branch
 __device__ __forceinline__ void mma_commit_elect(unsigned bar) {
   asm volatile(
       "{\n\t.reg .pred P;\n\t"

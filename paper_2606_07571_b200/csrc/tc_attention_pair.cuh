@@ -77,12 +77,9 @@ __device__ __forceinline__ unsigned map_to_rank(unsigned local, unsigned rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(local), "r"(rank));
   return raddr;
 }
-// arrival on a barrier named by a cluster address (this CTA's or the partner's)
-__device__ __forceinline__ void mbar_arrive_cluster(unsigned cluster_bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
-}
-// The same without cluster-scope release (which costs a memory barrier on the arriving warp): for
-// hand-overs whose data lives in tensor memory and is ordered by the tcgen05 fences, not by this arrival.
+// Arrival on a barrier named by a cluster address (this CTA's or the partner's), without a cluster-scope
+// release (which costs a memory barrier on the arriving warp): for hand-overs whose data lives in tensor
+// memory and is ordered by the tcgen05 fences, not by this arrival.
 __device__ __forceinline__ void mbar_arrive_cluster_plain(unsigned cluster_bar) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
